@@ -1,0 +1,180 @@
+/*
+ * arb.h -- C ABI of the Arbitrage hot path on one B200 (sm_100a).
+ *
+ * Three operations make up the data-parallel part of step-level speculative generation with an
+ * advantage-aware router (Algorithm 1 of the paper):
+ *
+ *   arb_attn      grouped-query attention of a batch of query chunks against per-sequence paged KV
+ *                 caches.  q_len = 1 is one autoregressive decode token of a draft or target step
+ *                 (Section 3.1: z_i ~ q(z_i | x, z_<i)); q_len = step length is the router's single
+ *                 forward over a completed draft step (Section 4.2, "one forward pass per step").
+ *   arb_route     the router decision (Section 4.2; Figure 1; Algorithm 1, "Routing decision"):
+ *                 y_hat = sigmoid(hidden_last . w + b); escalate to the target iff y_hat > tau,
+ *                 accept the draft step iff y_hat <= tau.
+ *   arb_rollback  the escalation branch of Algorithm 1: the target regenerates the step from the
+ *                 same prefix x, so a cache that absorbed the rejected draft step drops it by
+ *                 resetting its length; no KV bytes move.
+ *
+ * Conventions shared by every call
+ *   - Pointers are DEVICE pointers unless the argument says "host".  The caller owns every tensor;
+ *     the library owns only the arb_ctx (split-KV partials, arrival counters, a status word and
+ *     staging buffers), allocated by arb_create / grown by the *_host calls, never by arb_attn,
+ *     arb_route or arb_rollback.
+ *   - Calls enqueue work on `stream` and return; they do not synchronise (arb_poll_status and the
+ *     *_host calls do).  One arb_ctx must not be used from two streams at the same time: calls
+ *     share its workspace.
+ *   - Host-checkable problems (null pointer, bad dimension, pointer not 16-byte aligned,
+ *     unsupported head_dim / group size, workspace too small) return a non-zero arb_status and
+ *     launch nothing.  Problems only the device can see (page id out of range, seq_len < q_len,
+ *     seq_len beyond the block table, rollback below zero) set a bit in a device status word, the
+ *     offending sequence is skipped (its output rows are zero-filled) or clamped, and the kernel
+ *     carries on: nothing traps.  Read the bits with arb_poll_status.
+ *   - Layouts are dense row-major with the last index fastest.
+ */
+#ifndef ARB_H_
+#define ARB_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    ARB_OK = 0,
+    ARB_ERR_INVALID_ARG = 1,   /* null pointer, non-positive dimension, misaligned pointer */
+    ARB_ERR_UNSUPPORTED = 2,   /* head_dim, group size, page size or dtype outside the built set */
+    ARB_ERR_WORKSPACE = 3,     /* the ctx workspace is smaller than arb_attn_workspace_bytes() */
+    ARB_ERR_CUDA = 4,          /* a CUDA runtime call failed (allocation, launch, copy) */
+    ARB_ERR_DEVICE_STATUS = 5  /* arb_poll_status: the device status word is non-zero */
+} arb_status;
+
+typedef enum { ARB_F32 = 0, ARB_BF16 = 1 } arb_dtype;
+
+/* bits of the device status word (arb_poll_status) */
+enum {
+    ARB_DEV_BAD_SEQ_LEN = 1u,        /* q_len > 0 and (seq_len < q_len or seq_len > max_pages*page) */
+    ARB_DEV_BAD_PAGE = 2u,           /* block_table entry outside [0, num_pages) */
+    ARB_DEV_ROLLBACK_UNDERFLOW = 4u, /* step_len < 0 or step_len > seq_len */
+    ARB_DEV_WAIT_TIMEOUT = 8u        /* a bounded wait on an asynchronous copy or MMA gave up */
+};
+
+typedef struct CUstream_st *arb_stream_t; /* same type as cudaStream_t */
+typedef struct arb_ctx arb_ctx;
+
+/*
+ * Shape of one arb_attn call.  Notation: B = batch, Hq = num_q_heads, Hkv = num_kv_heads,
+ * g = Hq / Hkv (query heads h*g .. h*g+g-1 share KV head h), D = head_dim, P = page_size.
+ */
+typedef struct {
+    int32_t dtype;             /* arb_dtype of q, k_pages, v_pages and out; accumulation is fp32 */
+    int32_t batch;             /* 1 .. 1024 */
+    int32_t num_q_heads;       /* multiple of num_kv_heads, g <= 8 */
+    int32_t num_kv_heads;
+    int32_t head_dim;          /* 64 or 128 */
+    int32_t page_size;         /* 16 */
+    int32_t num_pages;         /* pages in the pool that k_pages / v_pages point to */
+    int32_t max_pages_per_seq; /* row length of block_table */
+    int32_t total_q;           /* sum of q_lens (rows of q and out); the host knows it */
+    int32_t max_q_len;         /* max of q_lens; 1 selects the decode kernel alone */
+    float softmax_scale;       /* <= 0 selects 1/sqrt(head_dim) */
+} arb_attn_params;
+
+/*
+ * Create a context on `device`.  workspace_bytes = 0 picks a default that covers every shape the
+ * library supports with batch * num_kv_heads <= 8192.  Allocates device memory; call it outside
+ * any stream capture.  Errors: ARB_ERR_INVALID_ARG, ARB_ERR_CUDA.
+ */
+arb_status arb_create(arb_ctx **ctx, int device, size_t workspace_bytes);
+arb_status arb_destroy(arb_ctx *ctx);
+
+/* Workspace an arb_attn call with these parameters needs (0 if the parameters are invalid). */
+size_t arb_attn_workspace_bytes(const arb_attn_params *params);
+
+/*
+ * Paged grouped-query attention (the forward passes of Algorithm 1's "Sample draft step",
+ * "Sample target step" and "Routing decision"; Section 3.1 for the token-by-token step).
+ *
+ *   q, out       [total_q, Hq, D]; rows packed by sequence: sequence b owns q_lens[b] consecutive
+ *                rows, in batch order.  out has q's dtype.
+ *   k_pages,
+ *   v_pages      [num_pages, Hkv, P, D]: one (page, kv head) tile is P*D contiguous elements.
+ *   block_table  int32 [B, max_pages_per_seq]; entry [b][j] is the pool page holding tokens
+ *                j*P .. j*P+P-1 of sequence b.  Entries at or beyond ceil(seq_len / P) are never
+ *                read.
+ *   seq_lens     int32 [B]: tokens in the cache INCLUDING the q_lens[b] new ones, whose K/V the
+ *                caller has already written.
+ *   q_lens       int32 [B]: 0 (idle slot, no rows), 1 (decode) or the step length.
+ *
+ * Query token i (0-based) of sequence b sits at position pos = seq_lens[b] - q_lens[b] + i and
+ * attends keys 0 .. pos inclusive:  out = sum_j softmax_j(scale * q . k_j) v_j.  Slots beyond
+ * pos are never used, not even multiplied by zero, so stale or non-finite values there (a rolled
+ * back step) cannot reach the output.
+ *
+ * Asynchronous on `stream`.  Errors: ARB_ERR_INVALID_ARG, ARB_ERR_UNSUPPORTED, ARB_ERR_WORKSPACE,
+ * ARB_ERR_CUDA; device-side: ARB_DEV_BAD_SEQ_LEN (rows zero-filled), ARB_DEV_BAD_PAGE (the bad
+ * page is skipped or replaced by page 0; that sequence's rows are unspecified but finite-safe).
+ */
+arb_status arb_attn(arb_ctx *ctx, const arb_attn_params *params, const void *q,
+                    const void *k_pages, const void *v_pages, const int32_t *block_table,
+                    const int32_t *seq_lens, const int32_t *q_lens, void *out,
+                    arb_stream_t stream);
+
+/*
+ * arb_attn for callers whose per-step tensors live in HOST memory (pinned memory makes the copies
+ * asynchronous).  q_host, block_table_host, seq_lens_host, q_lens_host and out_host are host
+ * pointers with the shapes above; k_pages and v_pages stay DEVICE pointers (the cache is resident
+ * state, not a per-step input).  Copies the inputs to staging buffers owned by ctx (grown here if
+ * too small -- the one call besides arb_create that may allocate), runs arb_attn, copies out back
+ * and synchronises `stream` before returning.
+ */
+arb_status arb_attn_host(arb_ctx *ctx, const arb_attn_params *params, const void *q_host,
+                         const void *k_pages, const void *v_pages,
+                         const int32_t *block_table_host, const int32_t *seq_lens_host,
+                         const int32_t *q_lens_host, void *out_host, arb_stream_t stream);
+
+/*
+ * Router head and threshold decision (Section 4.2: the score is the likelihood that the target
+ * outperforms the draft, reject iff y_hat > tau; Algorithm 1: accept iff y_hat <= tau; the
+ * classification head reads the final token's embedding).  A two-class softmax head (accept = 0,
+ * escalate = 1) is the same function with w = w1 - w0 and b = b1 - b0.
+ *
+ *   hidden     [n_steps, hidden_dim]; row i is the final-layer hidden state of the last token of
+ *              step i.  hidden_dim must be a multiple of 8.
+ *   w          [hidden_dim], same dtype as hidden.
+ *   b, tau     host scalars.
+ *   scores     fp32 [n_steps]: sigmoid(hidden_i . w + b), accumulated in fp32.
+ *   decisions  uint8 [n_steps]: 1 = escalate (score > tau), 0 = accept (score <= tau; a tie
+ *              accepts).
+ */
+arb_status arb_route(arb_ctx *ctx, int32_t dtype, int32_t n_steps, int32_t hidden_dim,
+                     const void *hidden, const void *w, float b, float tau, float *scores,
+                     uint8_t *decisions, arb_stream_t stream);
+
+/*
+ * Step rollback (Algorithm 1, escalation branch: the step is regenerated from the same prefix).
+ *   seq_lens[i] -= step_lens[i]  for every i with decisions == NULL or decisions[i] != 0.
+ * Block-table entries and page contents are left as they are; later attention ignores the stale
+ * slots and later appends overwrite them.  step_lens[i] < 0 leaves seq_lens[i] unchanged and
+ * step_lens[i] > seq_lens[i] clamps it to 0; both raise ARB_DEV_ROLLBACK_UNDERFLOW.
+ */
+arb_status arb_rollback(arb_ctx *ctx, int32_t batch, int32_t *seq_lens, const int32_t *step_lens,
+                        const uint8_t *decisions /* nullable */, arb_stream_t stream);
+
+/*
+ * Synchronise `stream`, read the device status word into *bits (nullable) and clear it together
+ * with the split-KV arrival counters.  Returns ARB_OK if the word was zero, else
+ * ARB_ERR_DEVICE_STATUS.
+ */
+arb_status arb_poll_status(arb_ctx *ctx, arb_stream_t stream, uint32_t *bits);
+
+/* Number of kernels the library has launched through this ctx since arb_create. */
+uint64_t arb_launch_count(const arb_ctx *ctx);
+
+const char *arb_status_string(arb_status status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* ARB_H_ */

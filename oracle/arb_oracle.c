@@ -1,0 +1,213 @@
+/*
+ * CPU oracle for the Arbitrage hot path: paged grouped-query attention, the router head and
+ * step rollback.  TEST INFRASTRUCTURE ONLY: the tests, the smoke check and the CPU-baseline leg of
+ * the benchmark call it; the product (the CUDA library) never does and shares no code with it.
+ *
+ * Everything is the plain definition written out in fp64, one key at a time in logical order:
+ * no tiling, no online softmax, no splits.  Inputs are the very bits the GPU reads (fp32 or
+ * bf16), widened exactly.  OpenMP only spreads independent output rows over cores.
+ *
+ * What each function follows:
+ *  - oracle_attn: the forward passes inside Algorithm 1 ("Sample draft step", "Sample target step",
+ *    and the router's forward over (x, z_d)) reduce, per layer, to causal scaled-dot-product
+ *    attention of the new tokens against the cached context x (Section 3.1: a step z is generated
+ *    token by token given x and z_<i).  The paper does not print the attention formula; this is the
+ *    textbook one, softmax(scale * q.k) v, with grouped-query head sharing and a paged cache.
+ *  - oracle_route: Section 4.2 (the router outputs y_hat, the likelihood that the target beats
+ *    the draft; reject iff y_hat > tau), Figure 1 caption and Algorithm 1 (accept iff
+ *    y_hat <= tau), with the classification head applied to the final-token embedding
+ *    (Section 4.2, "Training").  A two-class softmax head equals the sigmoid of the logit
+ *    difference, which is the single (w, b) used here.
+ *  - oracle_rollback: Algorithm 1, escalation branch: the target regenerates the step from the same
+ *    prefix x, so every cache that absorbed the rejected draft step forgets it.
+ *
+ * Pins (tests/test_oracle_*.py): rows of softmax sum to one; uniform keys give the mean of V;
+ * a single key returns its V; a dominant key returns its V; score-shift invariance; brute-force
+ * dense numpy attention; a library SDPA routine in fp64; page-permutation invariance; a chunk equals
+ * a sequence of decodes; GQA head sharing; hand-built router scores and the tie rule.
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+enum { ORACLE_F32 = 0, ORACLE_BF16 = 1 };
+
+/* status bits reported for inputs that have no defined result */
+enum {
+    ORACLE_BAD_SEQ_LEN = 1u,   /* seq_len < q_len, or seq_len > max_pages_per_seq * page_size */
+    ORACLE_BAD_PAGE = 2u,      /* block_table entry outside [0, num_pages) */
+    ORACLE_ROLLBACK_UNDERFLOW = 4u
+};
+
+static double widen(const void *base, int dtype, size_t idx)
+{
+    if (dtype == ORACLE_F32)
+        return (double)((const float *)base)[idx];
+    uint32_t bits = ((uint32_t)((const uint16_t *)base)[idx]) << 16;
+    float f;
+    memcpy(&f, &bits, sizeof f);
+    return (double)f;
+}
+
+/* element offset of K/V[page][kv_head][slot][0] in the head-major page layout
+ * [num_pages, num_kv_heads, page_size, head_dim] */
+static size_t kv_offset(long page, int kvh, int slot, int Hkv, int P, int D)
+{
+    return (((size_t)page * Hkv + kvh) * P + slot) * (size_t)D;
+}
+
+int oracle_num_threads(void)
+{
+#ifdef _OPENMP
+    return omp_get_max_threads();
+#else
+    return 1;
+#endif
+}
+
+/*
+ * One output row: query token `i` of sequence `b`, query head `h`.
+ *   pos = L_b - n_b + i;  keys j = 0..pos inclusive (a token sees itself)
+ *   s_j = scale * q . k_j ; p_j = exp(s_j - max) / sum ; out = sum_j p_j v_j
+ * If probs != NULL it receives p_0..p_pos.  Returns status bits (0 = fine).
+ */
+static unsigned attn_row(int dtype, int Hq, int Hkv, int D, int P, long num_pages, int max_pages,
+                         const void *q, const void *k_pages, const void *v_pages,
+                         const int32_t *block_row, long q_row, int h, long pos, double scale,
+                         double *out_row, double *probs)
+{
+    int g = Hq / Hkv;
+    int kvh = h / g;
+    long nkeys = pos + 1;
+    double *s = (double *)malloc(sizeof(double) * (size_t)nkeys);
+    size_t qoff = ((size_t)q_row * Hq + h) * (size_t)D;
+    unsigned status = 0;
+    (void)max_pages;
+
+    for (long j = 0; j < nkeys; ++j) {
+        long page = block_row[j / P];
+        if (page < 0 || page >= num_pages) { status |= ORACLE_BAD_PAGE; break; }
+        size_t koff = kv_offset(page, kvh, (int)(j % P), Hkv, P, D);
+        double acc = 0.0;
+        for (int d = 0; d < D; ++d)
+            acc += widen(q, dtype, qoff + d) * widen(k_pages, dtype, koff + d);
+        s[j] = scale * acc;
+    }
+    if (status) {
+        for (int d = 0; d < D; ++d) out_row[d] = 0.0;
+        free(s);
+        return status;
+    }
+    double mx = s[0];
+    for (long j = 1; j < nkeys; ++j) if (s[j] > mx) mx = s[j];
+    double Z = 0.0;
+    for (long j = 0; j < nkeys; ++j) { s[j] = exp(s[j] - mx); Z += s[j]; }
+    for (int d = 0; d < D; ++d) out_row[d] = 0.0;
+    for (long j = 0; j < nkeys; ++j) {
+        double p = s[j] / Z;
+        if (probs) probs[j] = p;
+        long page = block_row[j / P];
+        size_t voff = kv_offset(page, kvh, (int)(j % P), Hkv, P, D);
+        for (int d = 0; d < D; ++d)
+            out_row[d] += p * widen(v_pages, dtype, voff + d);
+    }
+    free(s);
+    return status;
+}
+
+/*
+ * Paged grouped-query attention.
+ *   q           [total_q, Hq, D]   rows packed by sequence (sequence b owns q_lens[b] rows)
+ *   k_pages,
+ *   v_pages     [num_pages, Hkv, P, D]
+ *   block_table int32 [B, max_pages]
+ *   seq_lens    int32 [B]  tokens in the cache INCLUDING the q_lens[b] new ones
+ *   q_lens      int32 [B]
+ *   out         fp64 [total_q, Hq, D]
+ * scale <= 0 means 1/sqrt(D).  Returns the OR of the status bits; a sequence with a bad length
+ * gets zero rows, a row that meets a bad page id gets zeros.
+ */
+unsigned oracle_attn(int dtype, int B, int Hq, int Hkv, int D, int P, long num_pages, int max_pages,
+                     const void *q, const void *k_pages, const void *v_pages,
+                     const int32_t *block_table, const int32_t *seq_lens, const int32_t *q_lens,
+                     double scale, double *out)
+{
+    if (scale <= 0.0) scale = 1.0 / sqrt((double)D);
+    long *row0 = (long *)malloc(sizeof(long) * (size_t)(B + 1));
+    row0[0] = 0;
+    for (int b = 0; b < B; ++b) row0[b + 1] = row0[b] + (q_lens[b] > 0 ? q_lens[b] : 0);
+    unsigned status = 0;
+
+    for (int b = 0; b < B; ++b) {
+        long n = q_lens[b], L = seq_lens[b];
+        if (n <= 0) continue;
+        if (L < n || L > (long)max_pages * P) {
+            status |= ORACLE_BAD_SEQ_LEN;
+            memset(out + (size_t)row0[b] * Hq * D, 0, sizeof(double) * (size_t)n * Hq * D);
+            continue;
+        }
+        unsigned st_b = 0;
+#pragma omp parallel for collapse(2) schedule(dynamic, 1) reduction(| : st_b)
+        for (long i = 0; i < n; ++i)
+            for (int h = 0; h < Hq; ++h) {
+                long row = row0[b] + i;
+                st_b |= attn_row(dtype, Hq, Hkv, D, P, num_pages, max_pages, q, k_pages, v_pages,
+                                 block_table + (size_t)b * max_pages, row, h, L - n + i, scale,
+                                 out + ((size_t)row * Hq + h) * D, NULL);
+            }
+        status |= st_b;
+    }
+    free(row0);
+    return status;
+}
+
+/* Same as one row of oracle_attn, also returning the softmax probabilities (length pos+1). */
+unsigned oracle_attn_row_probs(int dtype, int Hq, int Hkv, int D, int P, long num_pages,
+                               int max_pages, const void *q, const void *k_pages,
+                               const void *v_pages, const int32_t *block_row, long q_row, int h,
+                               long pos, double scale, double *out_row, double *probs)
+{
+    if (scale <= 0.0) scale = 1.0 / sqrt((double)D);
+    return attn_row(dtype, Hq, Hkv, D, P, num_pages, max_pages, q, k_pages, v_pages, block_row,
+                    q_row, h, pos, scale, out_row, probs);
+}
+
+/*
+ * Router head: z = hidden_i . w + b ; score = 1 / (1 + exp(-z)) ; decision = (score > tau).
+ * decision 1 = escalate to the target, 0 = accept the draft step (a tie accepts).
+ * The comparison is taken on the score rounded to fp32 against tau as fp32, the precision in which
+ * the score is stored and the threshold is given.
+ */
+void oracle_route(int dtype, int n_steps, int hidden_dim, const void *hidden, const void *w,
+                  double b, float tau, double *scores, uint8_t *decisions)
+{
+    for (int i = 0; i < n_steps; ++i) {
+        double z = b;
+        for (int k = 0; k < hidden_dim; ++k)
+            z += widen(hidden, dtype, (size_t)i * hidden_dim + k) * widen(w, dtype, (size_t)k);
+        double sc = 1.0 / (1.0 + exp(-z));
+        scores[i] = sc;
+        decisions[i] = ((float)sc > tau) ? 1 : 0;
+    }
+}
+
+/*
+ * Step rollback: seq_lens[i] -= step_lens[i] * (decisions ? decisions[i] != 0 : 1).
+ * No KV bytes move.  A step longer than the sequence clamps to 0 and raises a status bit.
+ */
+unsigned oracle_rollback(int B, int32_t *seq_lens, const int32_t *step_lens,
+                         const uint8_t *decisions)
+{
+    unsigned status = 0;
+    for (int i = 0; i < B; ++i) {
+        if (decisions && !decisions[i]) continue;
+        long r = (long)seq_lens[i] - (long)step_lens[i];
+        if (r < 0 || step_lens[i] < 0) { status |= ORACLE_ROLLBACK_UNDERFLOW; r = r < 0 ? 0 : seq_lens[i]; }
+        seq_lens[i] = (int32_t)r;
+    }
+    return status;
+}

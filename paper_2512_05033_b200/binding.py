@@ -1,0 +1,196 @@
+"""ctypes binding of the C-ABI library ``libarb.so`` (``include/arb.h``).
+
+Argument marshalling only: every step of the path runs in the CUDA kernels.  torch supplies device
+memory and streams; raw pointers cross the boundary.  Importing this module fails loudly when the
+library has not been built (``python -m paper_2512_05033_b200.build``): there is no fallback.
+"""
+from __future__ import annotations
+
+import ctypes
+from pathlib import Path
+
+import torch
+
+_LIB_PATH = Path(__file__).resolve().parent / "libarb.so"
+if not _LIB_PATH.exists():
+    raise ImportError(
+        f"{_LIB_PATH} is missing: build the CUDA library first "
+        "(python -m paper_2512_05033_b200.build); there is no CPU fallback")
+
+lib = ctypes.CDLL(str(_LIB_PATH))
+
+ARB_OK = 0
+ARB_ERR_INVALID_ARG, ARB_ERR_UNSUPPORTED, ARB_ERR_WORKSPACE, ARB_ERR_CUDA, ARB_ERR_DEVICE_STATUS = 1, 2, 3, 4, 5
+ARB_F32, ARB_BF16 = 0, 1
+DEV_BAD_SEQ_LEN, DEV_BAD_PAGE, DEV_ROLLBACK_UNDERFLOW, DEV_WAIT_TIMEOUT = 1, 2, 4, 8
+
+# every symbol include/arb.h declares
+EXPORTS = ("arb_create", "arb_destroy", "arb_attn_workspace_bytes", "arb_attn", "arb_attn_host",
+           "arb_route", "arb_rollback", "arb_poll_status", "arb_launch_count", "arb_status_string")
+
+
+class AttnParams(ctypes.Structure):
+    _fields_ = [("dtype", ctypes.c_int32), ("batch", ctypes.c_int32), ("num_q_heads", ctypes.c_int32),
+                ("num_kv_heads", ctypes.c_int32), ("head_dim", ctypes.c_int32), ("page_size", ctypes.c_int32),
+                ("num_pages", ctypes.c_int32), ("max_pages_per_seq", ctypes.c_int32),
+                ("total_q", ctypes.c_int32), ("max_q_len", ctypes.c_int32), ("softmax_scale", ctypes.c_float)]
+
+
+_vp, _i32, _f = ctypes.c_void_p, ctypes.c_int32, ctypes.c_float
+lib.arb_create.restype = ctypes.c_int
+lib.arb_create.argtypes = [ctypes.POINTER(_vp), ctypes.c_int, ctypes.c_size_t]
+lib.arb_destroy.restype = ctypes.c_int
+lib.arb_destroy.argtypes = [_vp]
+lib.arb_attn_workspace_bytes.restype = ctypes.c_size_t
+lib.arb_attn_workspace_bytes.argtypes = [ctypes.POINTER(AttnParams)]
+lib.arb_attn.restype = ctypes.c_int
+lib.arb_attn.argtypes = [_vp, ctypes.POINTER(AttnParams), _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp]
+lib.arb_attn_host.restype = ctypes.c_int
+lib.arb_attn_host.argtypes = [_vp, ctypes.POINTER(AttnParams), _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp]
+lib.arb_route.restype = ctypes.c_int
+lib.arb_route.argtypes = [_vp, _i32, _i32, _i32, _vp, _vp, _f, _f, _vp, _vp, _vp]
+lib.arb_rollback.restype = ctypes.c_int
+lib.arb_rollback.argtypes = [_vp, _i32, _vp, _vp, _vp, _vp]
+lib.arb_poll_status.restype = ctypes.c_int
+lib.arb_poll_status.argtypes = [_vp, _vp, ctypes.POINTER(ctypes.c_uint32)]
+lib.arb_launch_count.restype = ctypes.c_uint64
+lib.arb_launch_count.argtypes = [_vp]
+lib.arb_status_string.restype = ctypes.c_char_p
+lib.arb_status_string.argtypes = [ctypes.c_int]
+
+
+class ArbError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {lib.arb_status_string(status).decode()} (arb_status {status})")
+
+
+def _check(status: int, where: str):
+    if status != ARB_OK:
+        raise ArbError(status, where)
+
+
+def _dtype_code(t: torch.Tensor) -> int:
+    if t.dtype == torch.float32:
+        return ARB_F32
+    if t.dtype == torch.bfloat16:
+        return ARB_BF16
+    raise TypeError(f"arb takes fp32 or bf16 tensors, got {t.dtype}")
+
+
+def _stream_ptr(stream) -> int:
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return int(stream.cuda_stream)
+
+
+def _dev(t: torch.Tensor, name: str, dtype=None) -> int:
+    if not t.is_cuda or not t.is_contiguous():
+        raise ValueError(f"{name} must be a contiguous CUDA tensor")
+    if dtype is not None and t.dtype != dtype:
+        raise TypeError(f"{name} must be {dtype}, got {t.dtype}")
+    return t.data_ptr()
+
+
+def attn_params(q_dtype_code, batch, num_q_heads, num_kv_heads, head_dim, num_pages, max_pages_per_seq, total_q,
+                max_q_len, softmax_scale=0.0, page_size=16) -> AttnParams:
+    return AttnParams(q_dtype_code, batch, num_q_heads, num_kv_heads, head_dim, page_size, num_pages,
+                      max_pages_per_seq, total_q, max_q_len, softmax_scale)
+
+
+class Context:
+    """Owns one arb_ctx on a CUDA device (split-KV workspace, status word, staging buffers)."""
+
+    def __init__(self, device=0, workspace_bytes: int = 0):
+        self.device = torch.device("cuda", device) if isinstance(device, int) else torch.device(device)
+        torch.cuda.init()
+        h = _vp()
+        with torch.cuda.device(self.device):
+            _check(lib.arb_create(ctypes.byref(h), self.device.index or 0, workspace_bytes), "arb_create")
+        self._h = h
+
+    def close(self):
+        if getattr(self, "_h", None):
+            lib.arb_destroy(self._h)
+            self._h = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    # -- arb_attn -----------------------------------------------------------------------------
+    def params_for(self, q, k_pages, block_table, max_q_len: int, softmax_scale: float = 0.0) -> AttnParams:
+        total_q, Hq, D = q.shape
+        num_pages, Hkv, P, _ = k_pages.shape
+        B, max_pages = block_table.shape
+        return attn_params(_dtype_code(q), B, Hq, Hkv, D, num_pages, max_pages, total_q, max_q_len, softmax_scale, P)
+
+    def attn(self, q, k_pages, v_pages, block_table, seq_lens, q_lens, max_q_len: int, out=None,
+             softmax_scale: float = 0.0, stream=None, params: AttnParams | None = None):
+        """out[total_q, Hq, D] = paged GQA attention; all tensors on the device.  Asynchronous."""
+        if out is None:
+            out = torch.empty_like(q)
+        p = params or self.params_for(q, k_pages, block_table, max_q_len, softmax_scale)
+        st = lib.arb_attn(self._h, ctypes.byref(p), _dev(q, "q"), _dev(k_pages, "k_pages", q.dtype),
+                          _dev(v_pages, "v_pages", q.dtype), _dev(block_table, "block_table", torch.int32),
+                          _dev(seq_lens, "seq_lens", torch.int32), _dev(q_lens, "q_lens", torch.int32),
+                          _dev(out, "out", q.dtype), _stream_ptr(stream))
+        _check(st, "arb_attn")
+        return out
+
+    def attn_raw(self, p: AttnParams, q_ptr, k_ptr, v_ptr, bt_ptr, sl_ptr, ql_ptr, out_ptr, stream_ptr) -> int:
+        """Pointer-level call (no tensor checks) for timing loops; returns the arb_status."""
+        return lib.arb_attn(self._h, ctypes.byref(p), q_ptr, k_ptr, v_ptr, bt_ptr, sl_ptr, ql_ptr, out_ptr, stream_ptr)
+
+    def attn_host(self, q_host, k_pages, v_pages, block_table_host, seq_lens_host, q_lens_host, max_q_len: int,
+                  out_host=None, softmax_scale: float = 0.0, stream=None):
+        """Same with q / block_table / lengths / out in host memory (pinned for async copies).
+        Synchronises the stream before returning."""
+        if out_host is None:
+            out_host = torch.empty_like(q_host, pin_memory=True)
+        for t in (q_host, block_table_host, seq_lens_host, q_lens_host, out_host):
+            if t.is_cuda or not t.is_contiguous():
+                raise ValueError("host tensors must be contiguous CPU tensors")
+        p = self.params_for(q_host, k_pages, block_table_host, max_q_len, softmax_scale)
+        st = lib.arb_attn_host(self._h, ctypes.byref(p), q_host.data_ptr(), _dev(k_pages, "k_pages"),
+                               _dev(v_pages, "v_pages"), block_table_host.data_ptr(), seq_lens_host.data_ptr(),
+                               q_lens_host.data_ptr(), out_host.data_ptr(), _stream_ptr(stream))
+        _check(st, "arb_attn_host")
+        return out_host
+
+    # -- arb_route ----------------------------------------------------------------------------
+    def route(self, hidden, w, b: float, tau: float, scores=None, decisions=None, stream=None):
+        """scores fp32 [S] = sigmoid(hidden . w + b); decisions uint8 [S] = (score > tau)."""
+        S, H = hidden.shape
+        if scores is None:
+            scores = torch.empty(S, dtype=torch.float32, device=hidden.device)
+        if decisions is None:
+            decisions = torch.empty(S, dtype=torch.uint8, device=hidden.device)
+        st = lib.arb_route(self._h, _dtype_code(hidden), S, H, _dev(hidden, "hidden"), _dev(w, "w", hidden.dtype),
+                           float(b), float(tau), _dev(scores, "scores", torch.float32),
+                           _dev(decisions, "decisions", torch.uint8), _stream_ptr(stream))
+        _check(st, "arb_route")
+        return scores, decisions
+
+    # -- arb_rollback -------------------------------------------------------------------------
+    def rollback(self, seq_lens, step_lens, decisions=None, stream=None):
+        """In place: seq_lens[i] -= step_lens[i] where decisions is None or decisions[i] != 0."""
+        dp = None if decisions is None else _dev(decisions, "decisions", torch.uint8)
+        st = lib.arb_rollback(self._h, seq_lens.shape[0], _dev(seq_lens, "seq_lens", torch.int32),
+                              _dev(step_lens, "step_lens", torch.int32), dp, _stream_ptr(stream))
+        _check(st, "arb_rollback")
+        return seq_lens
+
+    # -- status -------------------------------------------------------------------------------
+    def poll_status(self, stream=None) -> int:
+        """Synchronises; returns the device status bits (and clears them)."""
+        bits = ctypes.c_uint32(0)
+        st = lib.arb_poll_status(self._h, _stream_ptr(stream), ctypes.byref(bits))
+        if st not in (ARB_OK, ARB_ERR_DEVICE_STATUS):
+            _check(st, "arb_poll_status")
+        return int(bits.value)
+
+    def launch_count(self) -> int:
+        return int(lib.arb_launch_count(self._h))

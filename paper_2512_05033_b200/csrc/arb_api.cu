@@ -1,0 +1,224 @@
+// C ABI of the arb library: argument validation, context and dispatch.  No arithmetic here.
+#include <new>
+
+#include "arb_common.cuh"
+
+using namespace arb;
+
+namespace {
+
+constexpr size_t kDefaultWorkspace = 48ull << 20;
+constexpr int kCounters = 1 << 16;
+
+inline bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+arb_status check_params(const arb_attn_params *p) {
+    if (p == nullptr) return ARB_ERR_INVALID_ARG;
+    if (p->batch < 1 || p->num_q_heads < 1 || p->num_kv_heads < 1 || p->num_pages < 1 || p->max_pages_per_seq < 1 ||
+        p->total_q < 0 || p->max_q_len < 0)
+        return ARB_ERR_INVALID_ARG;
+    if (p->num_q_heads % p->num_kv_heads != 0) return ARB_ERR_INVALID_ARG;
+    if (p->dtype != ARB_F32 && p->dtype != ARB_BF16) return ARB_ERR_UNSUPPORTED;
+    if (p->head_dim != 64 && p->head_dim != 128) return ARB_ERR_UNSUPPORTED;
+    if (p->page_size != kPage) return ARB_ERR_UNSUPPORTED;
+    if (p->num_q_heads / p->num_kv_heads > kMaxGroup) return ARB_ERR_UNSUPPORTED;
+    if (p->batch > kMaxBatch) return ARB_ERR_UNSUPPORTED;
+    if ((long long)p->batch * p->num_kv_heads > kCounters) return ARB_ERR_UNSUPPORTED;
+    if ((long long)p->max_pages_per_seq * kPage > (1ll << 30)) return ARB_ERR_UNSUPPORTED;
+    return ARB_OK;
+}
+
+struct DeviceGuard {
+    int prev = -1;
+    bool ok = true;
+    explicit DeviceGuard(int dev) {
+        ok = cudaGetDevice(&prev) == cudaSuccess;
+        if (ok && prev != dev) ok = cudaSetDevice(dev) == cudaSuccess;
+    }
+    ~DeviceGuard() {
+        if (prev >= 0) cudaSetDevice(prev);
+    }
+};
+
+}  // namespace
+
+extern "C" {
+
+arb_status arb_create(arb_ctx **out, int device, size_t workspace_bytes) {
+    if (out == nullptr || device < 0) return ARB_ERR_INVALID_ARG;
+    *out = nullptr;
+    DeviceGuard guard(device);
+    if (!guard.ok) return ARB_ERR_CUDA;
+    Ctx *c = new (std::nothrow) Ctx();
+    if (c == nullptr) return ARB_ERR_CUDA;
+    c->device = device;
+    int sms = 0;
+    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device) != cudaSuccess || sms < 1) {
+        delete c;
+        return ARB_ERR_CUDA;
+    }
+    c->num_sms = sms;
+    c->workspace_bytes = workspace_bytes ? workspace_bytes : kDefaultWorkspace;
+    c->counters_len = kCounters;
+    bool ok = cudaMalloc(&c->workspace, c->workspace_bytes) == cudaSuccess;
+    ok = ok && cudaMalloc(&c->counters, sizeof(int) * (c->counters_len + 4)) == cudaSuccess;
+    ok = ok && cudaMemset(c->counters, 0, sizeof(int) * (c->counters_len + 4)) == cudaSuccess;
+    if (!ok) {
+        cudaFree(c->workspace);
+        cudaFree(c->counters);
+        delete c;
+        cudaGetLastError();
+        return ARB_ERR_CUDA;
+    }
+    c->status = reinterpret_cast<uint32_t *>(c->counters + c->counters_len);
+    *out = reinterpret_cast<arb_ctx *>(c);
+    return ARB_OK;
+}
+
+arb_status arb_destroy(arb_ctx *ctx) {
+    if (ctx == nullptr) return ARB_ERR_INVALID_ARG;
+    Ctx *c = reinterpret_cast<Ctx *>(ctx);
+    DeviceGuard guard(c->device);
+    cudaFree(c->workspace);
+    cudaFree(c->counters);
+    cudaFree(c->stage);
+    delete c;
+    return ARB_OK;
+}
+
+size_t arb_attn_workspace_bytes(const arb_attn_params *params) {
+    if (check_params(params) != ARB_OK) return 0;
+    int dev = 0, sms = 148;
+    if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    cudaGetLastError();
+    if (sms < 148) sms = 148;
+    return decode_workspace_bytes(*params, sms);
+}
+
+arb_status arb_attn(arb_ctx *ctx, const arb_attn_params *params, const void *q, const void *k_pages,
+                    const void *v_pages, const int32_t *block_table, const int32_t *seq_lens,
+                    const int32_t *q_lens, void *out, arb_stream_t stream) {
+    if (ctx == nullptr) return ARB_ERR_INVALID_ARG;
+    arb_status st = check_params(params);
+    if (st != ARB_OK) return st;
+    if (!k_pages || !v_pages || !block_table || !seq_lens || !q_lens) return ARB_ERR_INVALID_ARG;
+    if (params->total_q == 0 || params->max_q_len == 0) return ARB_OK;  // nothing to do
+    if (!q || !out) return ARB_ERR_INVALID_ARG;
+    if (!aligned16(q) || !aligned16(out) || !aligned16(k_pages) || !aligned16(v_pages)) return ARB_ERR_INVALID_ARG;
+    if (params->max_q_len > params->total_q) return ARB_ERR_INVALID_ARG;
+    Ctx *c = reinterpret_cast<Ctx *>(ctx);
+    if (decode_workspace_bytes(*params, c->num_sms) > c->workspace_bytes) return ARB_ERR_WORKSPACE;
+    cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+
+    // q_len == 1 rows: the split-KV decode kernel.  It is launched whenever decode rows may exist
+    // (the host knows only the total and the maximum of q_lens).
+    const bool maybe_decode = params->max_q_len == 1 || params->total_q > params->max_q_len;
+    if (maybe_decode) {
+        st = launch_decode(c, *params, q, k_pages, v_pages, block_table, seq_lens, q_lens, out, s);
+        if (st != ARB_OK) return st;
+    }
+    if (params->max_q_len >= 2) {
+        st = launch_chunk_fma(c, *params, q, k_pages, v_pages, block_table, seq_lens, q_lens, out, 2,
+                              params->max_q_len, s);
+        if (st != ARB_OK) return st;
+    }
+    return ARB_OK;
+}
+
+arb_status arb_attn_host(arb_ctx *ctx, const arb_attn_params *params, const void *q_host, const void *k_pages,
+                         const void *v_pages, const int32_t *block_table_host, const int32_t *seq_lens_host,
+                         const int32_t *q_lens_host, void *out_host, arb_stream_t stream) {
+    if (ctx == nullptr) return ARB_ERR_INVALID_ARG;
+    arb_status st = check_params(params);
+    if (st != ARB_OK) return st;
+    if (!q_host || !out_host || !block_table_host || !seq_lens_host || !q_lens_host) return ARB_ERR_INVALID_ARG;
+    Ctx *c = reinterpret_cast<Ctx *>(ctx);
+    DeviceGuard guard(c->device);
+    if (!guard.ok) return ARB_ERR_CUDA;
+    cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+    const size_t esz = params->dtype == ARB_BF16 ? 2 : 4;
+    auto up = [](size_t x) { return (x + 255) & ~size_t(255); };
+    const size_t q_bytes = (size_t)params->total_q * params->num_q_heads * params->head_dim * esz;
+    const size_t bt_bytes = sizeof(int32_t) * (size_t)params->batch * params->max_pages_per_seq;
+    const size_t len_bytes = sizeof(int32_t) * (size_t)params->batch;
+    const size_t need = 2 * up(q_bytes) + up(bt_bytes) + 2 * up(len_bytes);
+    if (need > c->stage_bytes) {
+        if (cudaStreamSynchronize(s) != cudaSuccess) return ARB_ERR_CUDA;
+        cudaFree(c->stage);
+        c->stage = nullptr;
+        c->stage_bytes = 0;
+        if (cudaMalloc(&c->stage, need) != cudaSuccess) {
+            cudaGetLastError();
+            return ARB_ERR_CUDA;
+        }
+        c->stage_bytes = need;
+    }
+    char *dq = c->stage, *dout = dq + up(q_bytes), *dbt = dout + up(q_bytes);
+    char *dsl = dbt + up(bt_bytes), *dql = dsl + up(len_bytes);
+    bool ok = cudaMemcpyAsync(dq, q_host, q_bytes, cudaMemcpyHostToDevice, s) == cudaSuccess;
+    ok = ok && cudaMemcpyAsync(dbt, block_table_host, bt_bytes, cudaMemcpyHostToDevice, s) == cudaSuccess;
+    ok = ok && cudaMemcpyAsync(dsl, seq_lens_host, len_bytes, cudaMemcpyHostToDevice, s) == cudaSuccess;
+    ok = ok && cudaMemcpyAsync(dql, q_lens_host, len_bytes, cudaMemcpyHostToDevice, s) == cudaSuccess;
+    if (!ok) return ARB_ERR_CUDA;
+    st = arb_attn(ctx, params, dq, k_pages, v_pages, reinterpret_cast<int32_t *>(dbt),
+                  reinterpret_cast<int32_t *>(dsl), reinterpret_cast<int32_t *>(dql), dout, stream);
+    if (st != ARB_OK) return st;
+    if (cudaMemcpyAsync(out_host, dout, q_bytes, cudaMemcpyDeviceToHost, s) != cudaSuccess) return ARB_ERR_CUDA;
+    if (cudaStreamSynchronize(s) != cudaSuccess) return ARB_ERR_CUDA;
+    return ARB_OK;
+}
+
+arb_status arb_route(arb_ctx *ctx, int32_t dtype, int32_t n_steps, int32_t hidden_dim, const void *hidden,
+                     const void *w, float b, float tau, float *scores, uint8_t *decisions, arb_stream_t stream) {
+    if (ctx == nullptr || n_steps < 0 || hidden_dim < 1) return ARB_ERR_INVALID_ARG;
+    if (dtype != ARB_F32 && dtype != ARB_BF16) return ARB_ERR_UNSUPPORTED;
+    if (hidden_dim % 8 != 0) return ARB_ERR_UNSUPPORTED;
+    if (n_steps == 0) return ARB_OK;
+    if (!hidden || !w || !scores || !decisions) return ARB_ERR_INVALID_ARG;
+    if (!aligned16(hidden) || !aligned16(w)) return ARB_ERR_INVALID_ARG;
+    return launch_route(reinterpret_cast<Ctx *>(ctx), dtype, n_steps, hidden_dim, hidden, w, b, tau, scores,
+                        decisions, reinterpret_cast<cudaStream_t>(stream));
+}
+
+arb_status arb_rollback(arb_ctx *ctx, int32_t batch, int32_t *seq_lens, const int32_t *step_lens,
+                        const uint8_t *decisions, arb_stream_t stream) {
+    if (ctx == nullptr || batch < 0) return ARB_ERR_INVALID_ARG;
+    if (batch == 0) return ARB_OK;
+    if (!seq_lens || !step_lens) return ARB_ERR_INVALID_ARG;
+    return launch_rollback(reinterpret_cast<Ctx *>(ctx), batch, seq_lens, step_lens, decisions,
+                           reinterpret_cast<cudaStream_t>(stream));
+}
+
+arb_status arb_poll_status(arb_ctx *ctx, arb_stream_t stream, uint32_t *bits) {
+    if (ctx == nullptr) return ARB_ERR_INVALID_ARG;
+    Ctx *c = reinterpret_cast<Ctx *>(ctx);
+    cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+    uint32_t host = 0;
+    if (cudaMemcpyAsync(&host, c->status, sizeof(host), cudaMemcpyDeviceToHost, s) != cudaSuccess) return ARB_ERR_CUDA;
+    if (cudaStreamSynchronize(s) != cudaSuccess) return ARB_ERR_CUDA;
+    if (bits) *bits = host;
+    if (host != 0) {  // a kernel that gave up may have left arrival counters behind
+        if (cudaMemsetAsync(c->counters, 0, sizeof(int) * (c->counters_len + 4), s) != cudaSuccess) return ARB_ERR_CUDA;
+        if (cudaStreamSynchronize(s) != cudaSuccess) return ARB_ERR_CUDA;
+        return ARB_ERR_DEVICE_STATUS;
+    }
+    return ARB_OK;
+}
+
+uint64_t arb_launch_count(const arb_ctx *ctx) {
+    return ctx ? reinterpret_cast<const Ctx *>(ctx)->launches : 0;
+}
+
+const char *arb_status_string(arb_status status) {
+    switch (status) {
+        case ARB_OK: return "ok";
+        case ARB_ERR_INVALID_ARG: return "invalid argument";
+        case ARB_ERR_UNSUPPORTED: return "unsupported shape or dtype";
+        case ARB_ERR_WORKSPACE: return "workspace too small";
+        case ARB_ERR_CUDA: return "CUDA runtime error";
+        case ARB_ERR_DEVICE_STATUS: return "device status word is non-zero";
+        default: return "unknown status";
+    }
+}
+
+}  // extern "C"

@@ -1,0 +1,178 @@
+// Shared device helpers and the host-side context of the arb library (sm_100a only).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/arb.h"
+
+namespace arb {
+
+constexpr int kPage = 16;             // tokens per KV page
+constexpr int kMaxBatch = 1024;       // sequences per call (prefix tables live in shared memory)
+constexpr int kMaxGroup = 8;          // query heads per KV head
+constexpr long long kWaitCycles = 1ll << 31;  // bound of every mbarrier wait (about a second)
+
+// ---------------------------------------------------------------------------------------------
+// Host-side context
+// ---------------------------------------------------------------------------------------------
+struct Ctx {
+    int device = 0;
+    int num_sms = 0;
+    size_t workspace_bytes = 0;
+    char *workspace = nullptr;   // split-KV partials
+    int *counters = nullptr;     // arrival counters, one per (sequence, kv head); zero between calls
+    int counters_len = 0;
+    uint32_t *status = nullptr;  // device status word
+    uint64_t launches = 0;
+    // staging for the *_host entry points
+    char *stage = nullptr;
+    size_t stage_bytes = 0;
+};
+
+// ---------------------------------------------------------------------------------------------
+// Element types
+// ---------------------------------------------------------------------------------------------
+template <typename T>
+struct Elt;
+
+template <>
+struct Elt<float> {
+    static constexpr int kPerVec = 4;  // elements in one 16-byte vector
+    __device__ static __forceinline__ void unpack(const uint4 &v, float (&f)[4]) {
+        f[0] = __uint_as_float(v.x);
+        f[1] = __uint_as_float(v.y);
+        f[2] = __uint_as_float(v.z);
+        f[3] = __uint_as_float(v.w);
+    }
+    __device__ static __forceinline__ float to_float(float x) { return x; }
+    __device__ static __forceinline__ float from_float(float x) { return x; }
+};
+
+template <>
+struct Elt<__nv_bfloat16> {
+    static constexpr int kPerVec = 8;
+    // bf16 -> fp32 is a 16-bit shift: low half << 16, high half masked in place
+    __device__ static __forceinline__ void unpack(const uint4 &v, float (&f)[8]) {
+        f[0] = __uint_as_float(v.x << 16);
+        f[1] = __uint_as_float(v.x & 0xffff0000u);
+        f[2] = __uint_as_float(v.y << 16);
+        f[3] = __uint_as_float(v.y & 0xffff0000u);
+        f[4] = __uint_as_float(v.z << 16);
+        f[5] = __uint_as_float(v.z & 0xffff0000u);
+        f[6] = __uint_as_float(v.w << 16);
+        f[7] = __uint_as_float(v.w & 0xffff0000u);
+    }
+    __device__ static __forceinline__ float to_float(__nv_bfloat16 x) { return __bfloat162float(x); }
+    __device__ static __forceinline__ __nv_bfloat16 from_float(float x) { return __float2bfloat16_rn(x); }
+};
+
+// ---------------------------------------------------------------------------------------------
+// mbarrier and bulk-copy (TMA) wrappers
+// ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void *p) {
+    return static_cast<uint32_t>(__cvta_generic_to_shared(p));
+}
+
+__device__ __forceinline__ void mbar_init(uint64_t *bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
+}
+
+__device__ __forceinline__ void mbar_fence_init() {
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+}
+
+__device__ __forceinline__ void mbar_arrive(uint64_t *bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint64_t *bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes)
+                 : "memory");
+}
+
+__device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(smem_u32(bar)), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+
+// Wait for the phase with the given parity.  Every wait is bounded: after kWaitCycles, or as soon
+// as another thread of the block has given up (*abort != 0), it returns false and the caller
+// carries on with whatever is in shared memory; the status word then carries ARB_DEV_WAIT_TIMEOUT.
+__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volatile int *abort,
+                                          uint32_t *status) {
+    if (mbar_try_wait(bar, parity)) return true;
+    const long long t0 = clock64();
+    while (true) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if (*abort) return false;
+        if (clock64() - t0 > kWaitCycles) {
+            *abort = 1;
+            atomicOr(status, (uint32_t)ARB_DEV_WAIT_TIMEOUT);
+            return false;
+        }
+    }
+}
+
+// One contiguous global -> shared copy by the TMA unit; completion is counted in bytes on `bar`.
+// dst, src 16-byte aligned; bytes a multiple of 16.
+__device__ __forceinline__ void bulk_load(void *dst_smem, const void *src_gmem, uint32_t bytes, uint64_t *bar) {
+    asm volatile(
+        "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
+            smem_u32(dst_smem)),
+        "l"(src_gmem), "r"(bytes), "r"(smem_u32(bar))
+        : "memory");
+}
+
+__device__ __forceinline__ void named_barrier(int id, int threads) {
+    asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory");
+}
+
+__device__ __forceinline__ float fast_exp2(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
+// Transposing reduction of N per-lane values over an aligned group of W lanes (W a power of two,
+// N a multiple of W).  On return v[j], j < N/W, holds the group-wide sum of the original value
+// with index j + (N/W) * (lane % W).  N - N/W shuffles instead of N * log2(W).
+template <int N, int W>
+__device__ __forceinline__ void transpose_reduce(float (&v)[N], int lane_in_group) {
+    static_assert(N % W == 0, "value count must be a multiple of the group width");
+#pragma unroll
+    for (int w = W / 2, n = N / 2; w >= 1; w >>= 1, n >>= 1) {
+        const bool up = (lane_in_group & w) != 0;
+#pragma unroll
+        for (int i = 0; i < n; ++i) {
+            const float send = up ? v[i] : v[i + n];
+            const float keep = up ? v[i + n] : v[i];
+            v[i] = keep + __shfl_xor_sync(0xffffffffu, send, w);
+        }
+    }
+}
+
+// Launchers (one per translation unit)
+arb_status launch_decode(Ctx *ctx, const arb_attn_params &p, const void *q, const void *k_pages,
+                         const void *v_pages, const int32_t *block_table, const int32_t *seq_lens,
+                         const int32_t *q_lens, void *out, cudaStream_t stream);
+arb_status launch_chunk_fma(Ctx *ctx, const arb_attn_params &p, const void *q, const void *k_pages,
+                            const void *v_pages, const int32_t *block_table, const int32_t *seq_lens,
+                            const int32_t *q_lens, void *out, int n_lo, int n_hi, cudaStream_t stream);
+arb_status launch_route(Ctx *ctx, int dtype, int n_steps, int hidden_dim, const void *hidden, const void *w,
+                        float b, float tau, float *scores, uint8_t *decisions, cudaStream_t stream);
+arb_status launch_rollback(Ctx *ctx, int batch, int32_t *seq_lens, const int32_t *step_lens,
+                           const uint8_t *decisions, cudaStream_t stream);
+size_t decode_workspace_bytes(const arb_attn_params &p, int num_sms);
+int decode_grid(int num_sms);
+
+}  // namespace arb

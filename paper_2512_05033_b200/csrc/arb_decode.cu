@@ -1,0 +1,549 @@
+// Split-KV decode attention (q_len = 1) over paged KV, one persistent launch.
+//
+// Work decomposition.  The (sequence, kv head, page) triples of every decoding sequence form one
+// flat list, ordered sequence-major.  It is cut into gridDim.x equal ranges, one per CTA, so every
+// CTA streams the same number of pages whatever the length mix is.  Where a range crosses a
+// (sequence, kv head) boundary it splits into segments; a (sequence, kv head) whose pages span
+// several CTAs is finished by whichever of them arrives last (arrival counter + fence, no waiting).
+// The device derives all of this from seq_lens / q_lens in the kernel prologue, so the host never
+// reads a length.
+//
+// Inside a CTA one producer warp walks its pages and issues one bulk (TMA) copy per (page, head)
+// tile of K and of V -- 16 rows x head_dim, contiguous in the head-major page layout -- into a
+// shared-memory ring guarded by full/empty mbarriers.  Four consumer warps take tiles round-robin.
+// A segment is processed in sub-partitions of up to 512 tokens: q.K for every tile (fp32 FMAs on
+// the unpacked 16-byte vectors, reduced across the lanes of a row with a transposing shuffle
+// reduction) into a score buffer, one block-wide max / exp2 / sum pass, then P.V into per-lane
+// fp32 accumulators that live across sub-partitions (rescaled when the running max moves).
+#include "arb_common.cuh"
+
+namespace arb {
+
+namespace {
+
+constexpr int kConsWarps = 4;
+constexpr int kConsThreads = kConsWarps * 32;
+constexpr int kThreads = kConsThreads + 32;  // + producer warp
+constexpr int kStages = 16;
+constexpr int kSubPages = 32;                // pages per sub-partition
+constexpr int kSubTokens = kSubPages * kPage;
+constexpr int kMinChunk = 4;                 // fewest pages worth giving a CTA
+constexpr int kCtasPerSm = 2;
+
+struct DecodeArgs {
+    const char *q;
+    const char *k_pages;
+    const char *v_pages;
+    const int32_t *block_table;
+    const int32_t *seq_lens;
+    const int32_t *q_lens;
+    char *out;
+    float *part_o;    // [slots][G][D]   un-normalised partial outputs
+    float *part_ml;   // [slots][G][2]   running max (log2 domain) and sum
+    int *counters;    // [batch * Hkv]
+    uint32_t *status;
+    int batch, Hq, Hkv, num_pages, max_pages;
+    float scale_log2;  // softmax scale * log2(e)
+};
+
+template <typename T, int D, int G>
+struct Cfg {
+    static constexpr int EPL = Elt<T>::kPerVec;          // elements per lane (one 16-byte vector)
+    static constexpr int ROW_BYTES = D * (int)sizeof(T);
+    static constexpr int LPR = ROW_BYTES / 16;           // lanes per K/V row: 8, 16 or 32
+    static constexpr int RPP = 32 / LPR;                 // rows a warp reads per pass
+    static constexpr int NPASS = kPage / RPP;            // passes per tile
+    static constexpr int PB = NPASS < 8 ? NPASS : 8;     // passes per reduction batch
+    static constexpr int NB = NPASS / PB;
+    static constexpr int NV = PB * G;                    // partial dot products per lane and batch
+    static constexpr int NVP = (NV + LPR - 1) / LPR * LPR;
+    static constexpr int GP = (G + 3) / 4 * 4;           // heads padded to whole float4s
+    static constexpr int TILE_BYTES = kPage * ROW_BYTES;
+    static constexpr int RING_BYTES = kStages * TILE_BYTES;
+    static constexpr int LOGIT_BYTES = kSubTokens * GP * 4;
+    static constexpr int OSM_BYTES = kConsWarps * G * D * 4;
+    static constexpr int UNI_BYTES = LOGIT_BYTES > OSM_BYTES ? LOGIT_BYTES : OSM_BYTES;
+    static_assert(LPR == 8 || LPR == 16 || LPR == 32, "row must be 128, 256 or 512 bytes");
+};
+
+struct SmemTail {  // small fixed part after ring + score buffer
+    uint64_t full[kStages];
+    uint64_t empty[kStages];
+    float red_max[kConsWarps][kMaxGroup];
+    float red_sum[kConsWarps][kMaxGroup];
+    int abort;
+    int is_last;
+};
+
+template <typename T, int D, int G>
+size_t smem_bytes(int batch) {
+    using C = Cfg<T, D, G>;
+    return 128 + C::RING_BYTES + C::UNI_BYTES + sizeof(SmemTail) + sizeof(int) * (2 * (size_t)batch + 2);
+}
+
+struct Segment {
+    int b, kvh, pg0, pg1, L, bk, nparts, c_first;
+};
+
+// Next segment of the flat range [cur, r1); advances cur.  pref[b] = kv heads * pages of all
+// decoding sequences before b.
+__device__ __forceinline__ bool next_segment(int &cur, int r1, const int *pref, int B, int Hkv, int chunk,
+                                             const int32_t *seq_lens, Segment &s) {
+    if (cur >= r1) return false;
+    int lo = 0, hi = B;  // largest b with pref[b] <= cur
+    while (hi - lo > 1) {
+        const int mid = (lo + hi) >> 1;
+        if (pref[mid] <= cur) lo = mid; else hi = mid;
+    }
+    const int b = lo;
+    const int pages = (pref[b + 1] - pref[b]) / Hkv;
+    const int r = cur - pref[b];
+    const int kvh = r / pages;
+    const int pg0 = r - kvh * pages;
+    const int s0 = pref[b] + kvh * pages;  // flat range of this (sequence, kv head)
+    const int s1 = s0 + pages;
+    const int end = s1 < r1 ? s1 : r1;
+    s.b = b;
+    s.kvh = kvh;
+    s.pg0 = pg0;
+    s.pg1 = pg0 + (end - cur);
+    s.L = seq_lens[b];
+    s.bk = b * Hkv + kvh;
+    s.c_first = s0 / chunk;
+    s.nparts = (s1 - 1) / chunk - s.c_first + 1;
+    cur = end;
+    return true;
+}
+
+template <typename T, int D, int G>
+__global__ void __launch_bounds__(kThreads, kCtasPerSm) decode_kernel(const DecodeArgs a) {
+    using C = Cfg<T, D, G>;
+    constexpr int EPL = C::EPL, LPR = C::LPR, RPP = C::RPP, GP = C::GP;
+
+    extern __shared__ char smem_raw[];
+    char *base = reinterpret_cast<char *>((reinterpret_cast<uintptr_t>(smem_raw) + 127) & ~uintptr_t(127));
+    char *ring = base;
+    float *uni = reinterpret_cast<float *>(base + C::RING_BYTES);
+    SmemTail *tail = reinterpret_cast<SmemTail *>(base + C::RING_BYTES + C::UNI_BYTES);
+    int *pref = reinterpret_cast<int *>(tail + 1);  // [B + 1]
+    int *row0 = pref + a.batch + 1;                 // [B + 1]
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int B = a.batch, Hkv = a.Hkv;
+
+    // ---- prologue: lengths -> page counts and q row offsets, scanned by warp 0 -----------------
+    if (tid == 0) {
+        for (int s = 0; s < kStages; ++s) {
+            mbar_init(&tail->full[s], 1);
+            mbar_init(&tail->empty[s], 1);
+        }
+        tail->abort = 0;
+        tail->is_last = 0;
+        mbar_fence_init();
+        pref[0] = 0;
+        row0[0] = 0;
+    }
+    for (int b = tid; b < B; b += kThreads) {
+        const int n = a.q_lens[b], L = a.seq_lens[b];
+        int pages = 0;
+        if (n == 1) {
+            if (L >= 1 && L <= a.max_pages * kPage) {
+                pages = (L + kPage - 1) / kPage;
+            } else if (blockIdx.x == 0) {  // no defined result: flag it and zero the row
+                atomicOr(a.status, (uint32_t)ARB_DEV_BAD_SEQ_LEN);
+                int row = 0;
+                for (int i = 0; i < b; ++i) row += max(a.q_lens[i], 0);
+                T *o = reinterpret_cast<T *>(a.out) + (size_t)row * a.Hq * D;
+                for (int i = 0; i < a.Hq * D; ++i) o[i] = Elt<T>::from_float(0.f);
+            }
+        }
+        pref[b + 1] = pages * Hkv;
+        row0[b + 1] = n > 0 ? n : 0;
+    }
+    __syncthreads();
+    if (warp == 0) {
+        int carry_p = 0, carry_r = 0;
+        for (int b0 = 0; b0 < B; b0 += 32) {
+            const int b = b0 + lane;
+            int vp = b < B ? pref[b + 1] : 0;
+            int vr = b < B ? row0[b + 1] : 0;
+#pragma unroll
+            for (int off = 1; off < 32; off <<= 1) {
+                const int tp = __shfl_up_sync(0xffffffffu, vp, off);
+                const int tr = __shfl_up_sync(0xffffffffu, vr, off);
+                if (lane >= off) { vp += tp; vr += tr; }
+            }
+            if (b < B) { pref[b + 1] = vp + carry_p; row0[b + 1] = vr + carry_r; }
+            carry_p += __shfl_sync(0xffffffffu, vp, 31);
+            carry_r += __shfl_sync(0xffffffffu, vr, 31);
+        }
+    }
+    __syncthreads();
+
+    const int total = pref[B];
+    int chunk = (total + (int)gridDim.x - 1) / (int)gridDim.x;
+    if (chunk < kMinChunk) chunk = kMinChunk;
+    const long long r0l = (long long)blockIdx.x * chunk;
+    if (r0l >= total) return;  // whole CTA leaves together; no barrier is pending
+    const int r0 = (int)r0l;
+    const int r1 = min(total, r0 + chunk);
+    volatile int *abort = &tail->abort;
+
+    if (warp == kConsWarps) {
+        // ================================ producer warp ==========================================
+        uint32_t c = 0;
+        int cur = r0;
+        Segment s;
+        while (next_segment(cur, r1, pref, B, Hkv, chunk, a.seq_lens, s)) {
+            for (int sp0 = s.pg0; sp0 < s.pg1; sp0 += kSubPages) {
+                const int np = min(kSubPages, s.pg1 - sp0);
+                int pid = 0;
+                if (lane < np) {
+                    pid = a.block_table[(size_t)s.b * a.max_pages + sp0 + lane];
+                    if ((unsigned)pid >= (unsigned)a.num_pages) {
+                        atomicOr(a.status, (uint32_t)ARB_DEV_BAD_PAGE);
+                        pid = 0;
+                    }
+                }
+#pragma unroll 1
+                for (int ph = 0; ph < 2; ++ph) {
+                    const char *pool = ph ? a.v_pages : a.k_pages;
+#pragma unroll 1
+                    for (int i = 0; i < np; ++i, ++c) {
+                        const int pg = __shfl_sync(0xffffffffu, pid, i);
+                        if (lane == 0) {
+                            const uint32_t st = c % kStages, par = (c / kStages) & 1u;
+                            if (mbar_wait(&tail->empty[st], par ^ 1u, abort, a.status)) {
+                                mbar_arrive_expect_tx(&tail->full[st], C::TILE_BYTES);
+                                bulk_load(ring + st * C::TILE_BYTES,
+                                          pool + ((size_t)pg * Hkv + s.kvh) * C::TILE_BYTES, C::TILE_BYTES,
+                                          &tail->full[st]);
+                            }
+                        }
+                    }
+                }
+                __syncwarp();
+            }
+        }
+        // After a timeout the consumers may have left copies unconsumed: wait (bounded) for the
+        // last ring's worth so that no copy is in flight into this CTA's memory when it exits.
+        if (lane == 0 && *abort) {
+            const uint32_t n = c < (uint32_t)kStages ? c : (uint32_t)kStages;
+            for (uint32_t i = 0; i < n; ++i) {
+                const uint32_t cc = c - 1 - i;
+                const long long t0 = clock64();
+                while (!mbar_try_wait(&tail->full[cc % kStages], (cc / kStages) & 1u) &&
+                       clock64() - t0 < (1ll << 24)) {
+                }
+            }
+        }
+        return;
+    }
+
+    // ==================================== consumer warps ==========================================
+    const int lg = lane % LPR;  // lane within the row group (which 16-byte column of a row)
+    const int rg = lane / LPR;  // row group: which of the RPP rows of a pass
+    uint32_t c_base = 0;
+    int cur = r0;
+    Segment s;
+    while (next_segment(cur, r1, pref, B, Hkv, chunk, a.seq_lens, s)) {
+        const int qrow = row0[s.b];
+        float qf[G][EPL];
+#pragma unroll
+        for (int h = 0; h < G; ++h) {
+            const uint4 v = __ldg(reinterpret_cast<const uint4 *>(
+                a.q + (((size_t)qrow * a.Hq + s.kvh * G + h) * D + lg * EPL) * sizeof(T)));
+            Elt<T>::unpack(v, qf[h]);
+#pragma unroll
+            for (int e = 0; e < EPL; ++e) qf[h][e] *= a.scale_log2;
+        }
+        float m_run[G], l_run[G], o[G][EPL];
+#pragma unroll
+        for (int h = 0; h < G; ++h) {
+            m_run[h] = -INFINITY;
+            l_run[h] = 0.f;
+#pragma unroll
+            for (int e = 0; e < EPL; ++e) o[h][e] = 0.f;
+        }
+
+        for (int sp0 = s.pg0; sp0 < s.pg1; sp0 += kSubPages) {
+            const int np = min(kSubPages, s.pg1 - sp0);
+            const int ntok = min(s.L - sp0 * kPage, np * kPage);
+
+            // ---- phase A: scores of this warp's K tiles -------------------------------------------
+            for (int t = warp; t < np; t += kConsWarps) {
+                const uint32_t cc = c_base + t, st = cc % kStages, par = (cc / kStages) & 1u;
+                mbar_wait(&tail->full[st], par, abort, a.status);
+                const char *tile = ring + st * C::TILE_BYTES;
+#pragma unroll
+                for (int nb = 0; nb < C::NB; ++nb) {
+                    float acc[C::NVP];
+#pragma unroll
+                    for (int i = 0; i < C::NVP; ++i) acc[i] = 0.f;
+#pragma unroll
+                    for (int ps = 0; ps < C::PB; ++ps) {
+                        const int r = (nb * C::PB + ps) * RPP + rg;
+                        const uint4 kv = *reinterpret_cast<const uint4 *>(tile + r * C::ROW_BYTES + lg * 16);
+                        float kf[EPL];
+                        Elt<T>::unpack(kv, kf);
+#pragma unroll
+                        for (int h = 0; h < G; ++h)
+#pragma unroll
+                            for (int e = 0; e < EPL; ++e) acc[ps * G + h] = fmaf(qf[h][e], kf[e], acc[ps * G + h]);
+                    }
+                    transpose_reduce<C::NVP, LPR>(acc, lg);
+#pragma unroll
+                    for (int j = 0; j < C::NVP / LPR; ++j) {
+                        const int idx = j + (C::NVP / LPR) * lg;
+                        if (idx < C::NV) {
+                            const int ps = idx / G, h = idx - ps * G;
+                            const int token = t * kPage + (nb * C::PB + ps) * RPP + rg;
+                            uni[token * GP + h] = acc[j];
+                        }
+                    }
+                }
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&tail->empty[st]);
+            }
+            named_barrier(1, kConsThreads);
+
+            // ---- phase B: running max, exp2, running sum ------------------------------------------
+            float mloc[G];
+#pragma unroll
+            for (int h = 0; h < G; ++h) mloc[h] = -INFINITY;
+            for (int t = tid; t < ntok; t += kConsThreads) {
+#pragma unroll
+                for (int h4 = 0; h4 < GP; h4 += 4) {
+                    const float4 sv = *reinterpret_cast<const float4 *>(uni + t * GP + h4);
+                    if (h4 + 0 < G) mloc[h4 + 0] = fmaxf(mloc[h4 + 0], sv.x);
+                    if (h4 + 1 < G) mloc[h4 + 1] = fmaxf(mloc[h4 + 1], sv.y);
+                    if (h4 + 2 < G) mloc[h4 + 2] = fmaxf(mloc[h4 + 2], sv.z);
+                    if (h4 + 3 < G) mloc[h4 + 3] = fmaxf(mloc[h4 + 3], sv.w);
+                }
+            }
+#pragma unroll
+            for (int h = 0; h < G; ++h) {
+#pragma unroll
+                for (int off = 16; off >= 1; off >>= 1)
+                    mloc[h] = fmaxf(mloc[h], __shfl_xor_sync(0xffffffffu, mloc[h], off));
+                if (lane == 0) tail->red_max[warp][h] = mloc[h];
+            }
+            named_barrier(1, kConsThreads);
+            float factor[G], lloc[G];
+#pragma unroll
+            for (int h = 0; h < G; ++h) {
+                float m = m_run[h];
+#pragma unroll
+                for (int w = 0; w < kConsWarps; ++w) m = fmaxf(m, tail->red_max[w][h]);
+                factor[h] = fast_exp2(m_run[h] - m);  // 0 on the first sub-partition
+                m_run[h] = m;
+                lloc[h] = 0.f;
+            }
+            for (int t = tid; t < ntok; t += kConsThreads) {
+#pragma unroll
+                for (int h4 = 0; h4 < GP; h4 += 4) {
+                    float4 sv = *reinterpret_cast<const float4 *>(uni + t * GP + h4);
+                    if (h4 + 0 < G) { sv.x = fast_exp2(sv.x - m_run[h4 + 0]); lloc[h4 + 0] += sv.x; }
+                    if (h4 + 1 < G) { sv.y = fast_exp2(sv.y - m_run[h4 + 1]); lloc[h4 + 1] += sv.y; }
+                    if (h4 + 2 < G) { sv.z = fast_exp2(sv.z - m_run[h4 + 2]); lloc[h4 + 2] += sv.z; }
+                    if (h4 + 3 < G) { sv.w = fast_exp2(sv.w - m_run[h4 + 3]); lloc[h4 + 3] += sv.w; }
+                    *reinterpret_cast<float4 *>(uni + t * GP + h4) = sv;
+                }
+            }
+#pragma unroll
+            for (int h = 0; h < G; ++h) {
+#pragma unroll
+                for (int off = 16; off >= 1; off >>= 1) lloc[h] += __shfl_xor_sync(0xffffffffu, lloc[h], off);
+                if (lane == 0) tail->red_sum[warp][h] = lloc[h];
+            }
+            named_barrier(1, kConsThreads);
+#pragma unroll
+            for (int h = 0; h < G; ++h) {
+                float l = 0.f;
+#pragma unroll
+                for (int w = 0; w < kConsWarps; ++w) l += tail->red_sum[w][h];
+                l_run[h] = l_run[h] * factor[h] + l;
+#pragma unroll
+                for (int e = 0; e < EPL; ++e) o[h][e] *= factor[h];
+            }
+
+            // ---- phase C: P.V over this warp's V tiles --------------------------------------------
+            for (int t = warp; t < np; t += kConsWarps) {
+                const uint32_t cc = c_base + np + t, st = cc % kStages, par = (cc / kStages) & 1u;
+                mbar_wait(&tail->full[st], par, abort, a.status);
+                const char *tile = ring + st * C::TILE_BYTES;
+#pragma unroll
+                for (int ps = 0; ps < C::NPASS; ++ps) {
+                    const int r = ps * RPP + rg;
+                    const int token = t * kPage + r;
+                    if (token < ntok) {  // slots past the sequence end are never touched
+                        const uint4 vv = *reinterpret_cast<const uint4 *>(tile + r * C::ROW_BYTES + lg * 16);
+                        float vf[EPL];
+                        Elt<T>::unpack(vv, vf);
+                        float pf[GP];
+#pragma unroll
+                        for (int h4 = 0; h4 < GP; h4 += 4) {
+                            const float4 pv = *reinterpret_cast<const float4 *>(uni + token * GP + h4);
+                            pf[h4] = pv.x; pf[h4 + 1] = pv.y; pf[h4 + 2] = pv.z; pf[h4 + 3] = pv.w;
+                        }
+#pragma unroll
+                        for (int h = 0; h < G; ++h)
+#pragma unroll
+                            for (int e = 0; e < EPL; ++e) o[h][e] = fmaf(pf[h], vf[e], o[h][e]);
+                    }
+                }
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&tail->empty[st]);
+            }
+            named_barrier(1, kConsThreads);
+            c_base += 2u * np;
+        }
+
+        // ---- segment end: add up the warps' accumulators ---------------------------------------------
+#pragma unroll
+        for (int off = LPR; off < 32; off <<= 1)
+#pragma unroll
+            for (int h = 0; h < G; ++h)
+#pragma unroll
+                for (int e = 0; e < EPL; ++e) o[h][e] += __shfl_xor_sync(0xffffffffu, o[h][e], off);
+        if (rg == 0) {
+#pragma unroll
+            for (int h = 0; h < G; ++h)
+#pragma unroll
+                for (int e = 0; e < EPL; ++e) uni[(warp * G + h) * D + lg * EPL + e] = o[h][e];
+        }
+        named_barrier(1, kConsThreads);
+
+        const size_t out_base = ((size_t)qrow * a.Hq + s.kvh * G) * D;
+        if (s.nparts == 1) {
+            for (int idx = tid; idx < G * D; idx += kConsThreads) {
+                float acc = 0.f;
+#pragma unroll
+                for (int w = 0; w < kConsWarps; ++w) acc += uni[w * G * D + idx];
+                const int h = idx / D;
+                float l = l_run[0];
+#pragma unroll
+                for (int hh = 1; hh < G; ++hh) l = (h == hh) ? l_run[hh] : l;
+                reinterpret_cast<T *>(a.out)[out_base + idx] = Elt<T>::from_float(acc / l);
+            }
+            named_barrier(1, kConsThreads);
+        } else {
+            const size_t slot = (size_t)s.bk + blockIdx.x;
+            for (int idx = tid; idx < G * D; idx += kConsThreads) {
+                float acc = 0.f;
+#pragma unroll
+                for (int w = 0; w < kConsWarps; ++w) acc += uni[w * G * D + idx];
+                a.part_o[slot * G * D + idx] = acc;
+            }
+            if (tid == 0) {
+#pragma unroll
+                for (int h = 0; h < G; ++h) {
+                    a.part_ml[(slot * G + h) * 2 + 0] = m_run[h];
+                    a.part_ml[(slot * G + h) * 2 + 1] = l_run[h];
+                }
+            }
+            __threadfence();
+            named_barrier(1, kConsThreads);
+            if (tid == 0) {
+                const int old = atomicAdd(&a.counters[s.bk], 1);
+                const int last = (old == s.nparts - 1);
+                if (last) a.counters[s.bk] = 0;  // everyone has arrived: ready for the next call
+                tail->is_last = last;
+            }
+            named_barrier(1, kConsThreads);
+            if (tail->is_last) {
+                __threadfence();
+                const size_t slot0 = (size_t)s.bk + s.c_first;
+                for (int idx = tid; idx < G * D; idx += kConsThreads) {
+                    const int h = idx / D;
+                    float M = -INFINITY;
+                    for (int p = 0; p < s.nparts; ++p) M = fmaxf(M, __ldcg(&a.part_ml[((slot0 + p) * G + h) * 2]));
+                    float l = 0.f, acc = 0.f;
+                    for (int p = 0; p < s.nparts; ++p) {
+                        const float w = fast_exp2(__ldcg(&a.part_ml[((slot0 + p) * G + h) * 2]) - M);
+                        l = fmaf(w, __ldcg(&a.part_ml[((slot0 + p) * G + h) * 2 + 1]), l);
+                        acc = fmaf(w, __ldcg(&a.part_o[(slot0 + p) * G * D + idx]), acc);
+                    }
+                    reinterpret_cast<T *>(a.out)[out_base + idx] = Elt<T>::from_float(acc / l);
+                }
+            }
+            named_barrier(1, kConsThreads);
+        }
+    }
+}
+
+template <typename T, int D, int G>
+arb_status launch_one(Ctx *ctx, const DecodeArgs &args, cudaStream_t stream) {
+    const size_t smem = smem_bytes<T, D, G>(args.batch);
+    static bool attr_set[64] = {};
+    if (!attr_set[ctx->device & 63]) {
+        if (cudaFuncSetAttribute(decode_kernel<T, D, G>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 (int)smem_bytes<T, D, G>(kMaxBatch)) != cudaSuccess)
+            return ARB_ERR_CUDA;
+        attr_set[ctx->device & 63] = true;
+    }
+    decode_kernel<T, D, G><<<decode_grid(ctx->num_sms), kThreads, smem, stream>>>(args);
+    ctx->launches++;
+    return cudaGetLastError() == cudaSuccess ? ARB_OK : ARB_ERR_CUDA;
+}
+
+template <typename T, int D>
+arb_status launch_g(Ctx *ctx, int g, const DecodeArgs &args, cudaStream_t stream) {
+    switch (g) {
+        case 1: return launch_one<T, D, 1>(ctx, args, stream);
+        case 2: return launch_one<T, D, 2>(ctx, args, stream);
+        case 3: return launch_one<T, D, 3>(ctx, args, stream);
+        case 4: return launch_one<T, D, 4>(ctx, args, stream);
+        case 5: return launch_one<T, D, 5>(ctx, args, stream);
+        case 6: return launch_one<T, D, 6>(ctx, args, stream);
+        case 7: return launch_one<T, D, 7>(ctx, args, stream);
+        case 8: return launch_one<T, D, 8>(ctx, args, stream);
+        default: return ARB_ERR_UNSUPPORTED;
+    }
+}
+
+}  // namespace
+
+int decode_grid(int num_sms) { return num_sms * kCtasPerSm; }
+
+size_t decode_workspace_bytes(const arb_attn_params &p, int num_sms) {
+    const int g = p.num_q_heads / p.num_kv_heads;
+    const size_t slots = (size_t)p.batch * p.num_kv_heads + decode_grid(num_sms);
+    return slots * g * ((size_t)p.head_dim + 2) * sizeof(float);
+}
+
+arb_status launch_decode(Ctx *ctx, const arb_attn_params &p, const void *q, const void *k_pages,
+                         const void *v_pages, const int32_t *block_table, const int32_t *seq_lens,
+                         const int32_t *q_lens, void *out, cudaStream_t stream) {
+    const int g = p.num_q_heads / p.num_kv_heads;
+    const size_t slots = (size_t)p.batch * p.num_kv_heads + decode_grid(ctx->num_sms);
+    DecodeArgs a;
+    a.q = static_cast<const char *>(q);
+    a.k_pages = static_cast<const char *>(k_pages);
+    a.v_pages = static_cast<const char *>(v_pages);
+    a.block_table = block_table;
+    a.seq_lens = seq_lens;
+    a.q_lens = q_lens;
+    a.out = static_cast<char *>(out);
+    a.part_o = reinterpret_cast<float *>(ctx->workspace);
+    a.part_ml = a.part_o + slots * g * p.head_dim;
+    a.counters = ctx->counters;
+    a.status = ctx->status;
+    a.batch = p.batch;
+    a.Hq = p.num_q_heads;
+    a.Hkv = p.num_kv_heads;
+    a.num_pages = p.num_pages;
+    a.max_pages = p.max_pages_per_seq;
+    const float scale = p.softmax_scale > 0.f ? p.softmax_scale : 1.0f / sqrtf((float)p.head_dim);
+    a.scale_log2 = scale * 1.4426950408889634f;
+    if (p.dtype == ARB_BF16) {
+        if (p.head_dim == 128) return launch_g<__nv_bfloat16, 128>(ctx, g, a, stream);
+        if (p.head_dim == 64) return launch_g<__nv_bfloat16, 64>(ctx, g, a, stream);
+    } else if (p.dtype == ARB_F32) {
+        if (p.head_dim == 128) return launch_g<float, 128>(ctx, g, a, stream);
+        if (p.head_dim == 64) return launch_g<float, 64>(ctx, g, a, stream);
+    }
+    return ARB_ERR_UNSUPPORTED;
+}
+
+}  // namespace arb

@@ -1,0 +1,164 @@
+"""Parity of arb_attn (CUDA, through the C ABI) with the fp64 oracle, element by element."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2512_05033_b200 import workloads as wl
+from tests import helpers as H
+
+pytestmark = pytest.mark.gpu
+
+BF, F32 = torch.bfloat16, torch.float32
+
+DECODE_CASES = [
+    # (B, Hq, Hkv, D, dtype, seq_lens)                       what it covers
+    (1, 8, 2, 64, F32, [513]),                               # the tiny config: prefix 512 + 1
+    (1, 8, 2, 64, F32, [1]),                                 # a single key
+    (3, 12, 2, 128, BF, [16, 17, 15]),                       # page boundaries
+    (8, 12, 2, 128, BF, [1025, 2000, 3001, 777, 4096, 1, 640, 5555]),   # draft-shaped, ragged
+    (4, 32, 8, 128, BF, [4100, 9000, 33, 12000]),            # target-shaped heads
+    (2, 28, 4, 128, BF, [3000, 150]),                        # g = 7 (odd group)
+    (2, 6, 2, 64, BF, [700, 70]),                            # bf16, head_dim 64
+    (2, 4, 2, 128, F32, [900, 31]),                          # fp32, head_dim 128
+    (1, 5, 1, 128, BF, [40000]),                             # one long sequence over every CTA
+    (2, 3, 3, 64, F32, [260, 100]),                          # g = 1
+    (2, 16, 2, 128, BF, [2100, 900]),                        # g = 8
+]
+
+
+@pytest.mark.parametrize("case", DECODE_CASES)
+def test_decode_matches_oracle(case):
+    B, Hq, Hkv, D, dt, sl = case
+    inp = wl.small_attn_case(B, Hq, Hkv, D, dt, sl, [1] * B, seed=100 + len(sl) + Hq)
+    out, bits = H.gpu_attn(inp)
+    ref, st = H.oracle_attn(inp)
+    assert bits == 0 and st == 0
+    H.assert_close(out, ref, dt, tight=1e-3 if dt == BF else None)
+
+
+def test_decode_peaked_softmax():
+    """q scaled up so the softmax concentrates and outputs are O(1): the tolerance bites."""
+    inp = wl.small_attn_case(4, 12, 2, 128, BF, [3000, 513, 64, 1500], [1] * 4, seed=7, q_std=6.0)
+    out, bits = H.gpu_attn(inp)
+    ref, _ = H.oracle_attn(inp)
+    assert bits == 0
+    err = np.abs(out - ref)
+    # output is rounded to bf16 (2^-9 relative); the rest is the fp32 path
+    assert (err <= 2.0 ** -8 * np.abs(ref) + 2e-3).all(), err.max()
+
+
+def test_decode_idle_slots_and_scale():
+    inp = wl.small_attn_case(5, 8, 2, 64, F32, [100, 1, 300, 1, 47], [1, 0, 1, 0, 1], seed=31)
+    out, bits = H.gpu_attn(inp, scale=0.2)
+    ref, _ = H.oracle_attn(inp, scale=0.2)
+    assert bits == 0 and out.shape[0] == 3
+    H.assert_close(out, ref, F32)
+
+
+CHUNK_CASES = [
+    (1, 8, 2, 64, F32, [528], [16]),                         # the tiny config: 16-token chunk, prefix 512
+    (2, 12, 2, 128, BF, [300, 40], [7, 40]),                 # chunk == whole sequence (no prefix)
+    (3, 28, 4, 128, BF, [200, 90, 1000], [3, 1, 5]),         # decode and chunk rows in one call
+    (2, 4, 4, 64, BF, [33, 64], [2, 17]),
+    (2, 8, 1, 128, F32, [129, 50], [9, 2]),
+]
+
+
+@pytest.mark.parametrize("case", CHUNK_CASES)
+def test_chunk_matches_oracle(case):
+    B, Hq, Hkv, D, dt, sl, ql = case
+    inp = wl.small_attn_case(B, Hq, Hkv, D, dt, sl, ql, seed=200 + Hq)
+    out, bits = H.gpu_attn(inp)
+    ref, st = H.oracle_attn(inp)
+    assert bits == 0 and st == 0
+    H.assert_close(out, ref, dt, tight=1e-3 if dt == BF else None)
+
+
+def test_stale_slots_never_reach_the_output():
+    """Slots past each row's position hold NaN / 1e30 (a rolled-back step): the result must not change."""
+    inp = wl.small_attn_case(3, 12, 2, 128, BF, [1000, 37, 300], [1, 1, 6], seed=41, extra_tokens=40)
+    clean, bits = H.gpu_attn(inp)
+    assert bits == 0
+    k2, v2 = inp.k_pages.clone(), inp.v_pages.clone()
+    for b in range(3):
+        L = int(inp.seq_lens[b])
+        for j in range(L, L + 40):
+            pg = int(inp.block_table[b, j // wl.PAGE])
+            k2[pg, :, j % wl.PAGE] = float("nan")
+            v2[pg, :, j % wl.PAGE] = 1e30
+    pois = wl.AttnInputs(inp.shape, inp.q, k2, v2, inp.block_table, inp.seq_lens, inp.q_lens)
+    out, bits = H.gpu_attn(pois)
+    assert bits == 0
+    np.testing.assert_array_equal(out, clean)
+    ref, _ = H.oracle_attn(pois)
+    H.assert_close(out, ref, BF)
+
+
+def test_bad_length_is_flagged_and_zero_filled():
+    from paper_2512_05033_b200 import binding
+    inp = wl.small_attn_case(3, 8, 2, 64, F32, [50, 3, 20], [1, 5, 1], seed=51)   # seq_len < q_len in slot 1
+    out, bits = H.gpu_attn(inp)
+    ref, st = H.oracle_attn(inp)
+    assert bits & binding.DEV_BAD_SEQ_LEN and st & 1
+    assert (out[1:6] == 0).all()
+    H.assert_close(out, ref, F32)
+    # decode row with seq_len 0
+    inp = wl.small_attn_case(2, 8, 2, 64, F32, [0, 20], [1, 1], seed=52)
+    out, bits = H.gpu_attn(inp)
+    assert bits & binding.DEV_BAD_SEQ_LEN and (out[0] == 0).all()
+    ref, _ = H.oracle_attn(inp)
+    H.assert_close(out[1:], ref[1:], F32)
+    assert H.ctx().poll_status() == 0       # the word was cleared
+
+
+def test_bad_page_is_flagged_without_a_fault():
+    from paper_2512_05033_b200 import binding
+    inp = wl.small_attn_case(2, 8, 2, 64, F32, [100, 40], [1, 1], seed=53)
+    inp.block_table[0, 2] = inp.num_pages + 7
+    out, bits = H.gpu_attn(inp)
+    assert bits & binding.DEV_BAD_PAGE
+    good = wl.small_attn_case(2, 8, 2, 64, F32, [100, 40], [1, 1], seed=53)
+    ref, _ = H.oracle_attn(good)
+    H.assert_close(out[1:], ref[1:], F32)    # the other sequence is untouched
+    assert np.isfinite(out).all()
+
+
+def test_host_argument_errors():
+    from paper_2512_05033_b200 import binding
+    c = H.ctx()
+    inp = wl.small_attn_case(1, 8, 2, 64, F32, [40], [1], seed=54).to("cuda")
+    p = c.params_for(inp.q, inp.k_pages, inp.block_table, 1)
+    args = [inp.q.data_ptr(), inp.k_pages.data_ptr(), inp.v_pages.data_ptr(), inp.block_table.data_ptr(),
+            inp.seq_lens.data_ptr(), inp.q_lens.data_ptr(), torch.empty_like(inp.q).data_ptr(), 0]
+    assert c.attn_raw(p, *args) == binding.ARB_OK
+    bad = list(args); bad[1] = None
+    assert c.attn_raw(p, *bad) == binding.ARB_ERR_INVALID_ARG
+    bad = list(args); bad[0] = args[0] + 4
+    assert c.attn_raw(p, *bad) == binding.ARB_ERR_INVALID_ARG          # misaligned q
+    p2 = c.params_for(inp.q, inp.k_pages, inp.block_table, 1); p2.head_dim = 96
+    assert c.attn_raw(p2, *args) == binding.ARB_ERR_UNSUPPORTED
+    p3 = c.params_for(inp.q, inp.k_pages, inp.block_table, 1); p3.num_q_heads = 7
+    assert c.attn_raw(p3, *args) == binding.ARB_ERR_INVALID_ARG         # not a multiple of kv heads
+    small = binding.Context(0, workspace_bytes=1024)
+    assert small.attn_raw(p, *args) == binding.ARB_ERR_WORKSPACE
+    small.close()
+    torch.cuda.synchronize()
+
+
+def test_host_buffer_entry_point():
+    inp = wl.small_attn_case(3, 12, 2, 128, BF, [500, 90, 2000], [1, 4, 1], seed=55)
+    ref, _ = H.oracle_attn(inp)
+    c = H.ctx()
+    out = c.attn_host(inp.q.pin_memory(), inp.k_pages.cuda(), inp.v_pages.cuda(), inp.block_table.pin_memory(),
+                      inp.seq_lens.pin_memory(), inp.q_lens.pin_memory(), 4)
+    H.assert_close(out.double().numpy(), ref, BF)
+
+
+def test_repeated_calls_reuse_the_workspace():
+    """Arrival counters return to zero after every call: same answer five times in a row."""
+    inp = wl.small_attn_case(2, 12, 2, 128, BF, [9000, 5000], [1, 1], seed=56)
+    first, _ = H.gpu_attn(inp)
+    for _ in range(4):
+        again, bits = H.gpu_attn(inp)
+        assert bits == 0
+        np.testing.assert_array_equal(first, again)

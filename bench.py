@@ -1,0 +1,455 @@
+#!/usr/bin/env python
+"""Benchmark of the arb hot path on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+                    [--workload draft|target] [--layers L] [--no-graph] [--no-extras] [--profile]
+
+Headline workload: the draft-shaped decode configuration (batch 8, 12 query / 2 KV heads, head_dim
+128, bf16, page 16, prefix lengths uniform in [1024, 8192], q_len 1).  One step is one generated
+token's attention for the whole batch across 16 layers, each with its own KV pool, i.e. 16
+arb_attn calls (one kernel launch each, prepass and split combine fused in).  The pools together
+(about 600 MB) are several times the L2, so every call streams its KV from HBM.  The rows of the
+path that this workload does not contain (step-chunk attention, router head, rollback: there is no
+step boundary inside one decode token) are timed on the step-scoring workload and reported in
+"step_scoring" on the same line.
+
+value = KV-cache bytes attended per second over all ranks (GB/s).  Prints ONE JSON line on rank 0.
+"""
+from __future__ import annotations
+
+import argparse
+import hashlib
+import json
+import os
+import statistics
+import sys
+import threading
+import time
+from pathlib import Path
+
+import torch
+
+ROOT = Path(__file__).resolve().parent
+sys.path.insert(0, str(ROOT))
+
+from paper_2512_05033_b200 import workloads as wl  # noqa: E402
+
+METRIC = "attention KV HBM GB/s (% of B200 peak) and draft steps scored+routed/sec"
+LAYERS = 16
+NOMINAL_HBM_GBS = 8000.0
+FALLBACK_HBM_GBS = 6650.0
+
+
+# ------------------------------------------------------------------------------------------------
+# helpers
+# ------------------------------------------------------------------------------------------------
+def measured_peak():
+    f = ROOT / "MEASURED_PEAKS.json"
+    if f.exists():
+        try:
+            return float(json.loads(f.read_text())["hbm_gbs"]), "measured"
+        except Exception:
+            pass
+    return FALLBACK_HBM_GBS, "fallback"
+
+
+def attn_bytes(shape: wl.AttnShape, seq_lens, q_lens) -> dict:
+    """Algorithmic bytes of one arb_attn call: every visible KV token once per kv head, q and out
+    once, the block-table entries and the two length arrays."""
+    esz = 2 if shape.dtype == torch.bfloat16 else 4
+    tokens = int(seq_lens.sum())
+    rows = int(q_lens.sum())
+    kv = tokens * 2 * shape.num_kv_heads * shape.head_dim * esz
+    qo = 2 * rows * shape.num_q_heads * shape.head_dim * esz
+    table = int(((seq_lens + wl.PAGE - 1) // wl.PAGE).sum()) * 4 + 2 * 4 * int(seq_lens.numel())
+    return {"kv": kv, "qo": qo, "table": table, "total": kv + qo + table, "tokens": tokens}
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons through NVML (read-only) while the timed region runs."""
+
+    def __init__(self, index: int, period_s: float = 0.01):
+        self.index, self.period = index, period_s
+        self.samples, self.reasons = [], set()
+        self.max_mhz = None
+        self._stop = threading.Event()
+        self._thr = None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = int(pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM))
+        except Exception:
+            self.nv = None
+
+    def _loop(self):
+        nv = self.nv
+        names = {"hw_slowdown": 0x8, "sw_thermal_slowdown": 0x20, "hw_thermal_slowdown": 0x40,
+                 "sw_power_cap": 0x4, "hw_power_brake_slowdown": 0x80}
+        while not self._stop.is_set():
+            try:
+                self.samples.append(int(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM)))
+                try:
+                    r = int(nv.nvmlDeviceGetCurrentClocksEventReasons(self.h))
+                except Exception:
+                    r = int(nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h))
+                for k, bit in names.items():
+                    if r & bit:
+                        self.reasons.add(k)
+            except Exception:
+                pass
+            self._stop.wait(self.period)
+
+    def __enter__(self):
+        if self.nv is not None:
+            self._thr = threading.Thread(target=self._loop, daemon=True)
+            self._thr.start()
+        return self
+
+    def __exit__(self, *a):
+        self._stop.set()
+        if self._thr is not None:
+            self._thr.join()
+
+    def summary(self):
+        if not self.samples:
+            return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons), "samples": 0}
+        return {"sm_mhz": int(statistics.median(self.samples)), "sm_max_mhz": self.max_mhz,
+                "reasons": sorted(self.reasons), "samples": len(self.samples)}
+
+
+def cuda_physical_index(local: int) -> int:
+    vis = os.environ.get("CUDA_VISIBLE_DEVICES")
+    if vis:
+        try:
+            return int(vis.split(",")[local])
+        except Exception:
+            return local
+    return local
+
+
+# ------------------------------------------------------------------------------------------------
+# the decode workload
+# ------------------------------------------------------------------------------------------------
+class DecodeWorkload:
+    def __init__(self, shape: wl.AttnShape, layers: int, device, seed: int):
+        self.shape, self.layers = shape, layers
+        self.inp = wl.make_attn_inputs(shape, device=device, seed=seed)
+        self.pools = [(self.inp.k_pages, self.inp.v_pages)]
+        for l in range(1, layers):
+            self.pools.append(wl.make_kv_pool(shape, self.inp.num_pages, device, seed * 100 + l))
+        self.out = torch.empty_like(self.inp.q)
+        self.seq_cpu = self.inp.seq_lens.cpu().to(torch.int64)
+        self.ql_cpu = self.inp.q_lens.cpu().to(torch.int64)
+        self.bytes = attn_bytes(shape, self.seq_cpu, self.ql_cpu)
+
+    def step(self, ctx, params, stream_ptr):
+        i = self.inp
+        for k, v in self.pools:
+            st = ctx.attn_raw(params, i.q.data_ptr(), k.data_ptr(), v.data_ptr(), i.block_table.data_ptr(),
+                              i.seq_lens.data_ptr(), i.q_lens.data_ptr(), self.out.data_ptr(), stream_ptr)
+            if st != 0:
+                raise RuntimeError(f"arb_attn failed with status {st}")
+
+
+def time_steps(step_fn, steps, warmup, dist_barrier=None):
+    """W warm-up steps, then exactly K steps between CUDA events on the current stream."""
+    for _ in range(warmup):
+        step_fn()
+    torch.cuda.synchronize()
+    if dist_barrier:
+        dist_barrier()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(steps):
+        step_fn()
+    e1.record()
+    torch.cuda.synchronize()
+    if dist_barrier:
+        dist_barrier()
+    return e0.elapsed_time(e1)  # ms
+
+
+def make_step(ctx, work: DecodeWorkload, use_graph: bool):
+    """Returns (callable running one step on the current stream, kernel launches per step)."""
+    i = work.inp
+    params = ctx.params_for(i.q, i.k_pages, i.block_table, 1)
+    if not use_graph:
+        n0 = ctx.launch_count()
+        work.step(ctx, params, torch.cuda.current_stream().cuda_stream)
+        per_step = ctx.launch_count() - n0
+        return (lambda: work.step(ctx, params, torch.cuda.current_stream().cuda_stream)), per_step
+    # warm every code path outside capture (function attributes are set on first use)
+    work.step(ctx, params, torch.cuda.current_stream().cuda_stream)
+    torch.cuda.synchronize()
+    g = torch.cuda.CUDAGraph()
+    n0 = ctx.launch_count()
+    with torch.cuda.graph(g):
+        work.step(ctx, params, torch.cuda.current_stream().cuda_stream)
+    per_step = ctx.launch_count() - n0
+    return g.replay, per_step
+
+
+# ------------------------------------------------------------------------------------------------
+# our arm
+# ------------------------------------------------------------------------------------------------
+def run_ours(args):
+    from paper_2512_05033_b200 import binding
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist  # plumbing only: barrier and the max over ranks
+        dist.init_process_group("nccl", device_id=dev)
+    barrier = (lambda: dist.barrier()) if dist else None
+
+    ctx = binding.Context(local)
+    shape = wl.TARGET_DECODE if args.workload == "target" else wl.DRAFT_DECODE
+    layers = args.layers or (LAYERS if shape is wl.DRAFT_DECODE else 2)
+    work = DecodeWorkload(shape, layers, dev, seed=shape.seed + 1000 * rank)  # weak scaling: own batch per rank
+    use_graph = not (args.no_graph or args.profile)
+    step_fn, per_step = make_step(ctx, work, use_graph)
+
+    with ClockSampler(cuda_physical_index(local)) as clk:
+        ms = time_steps(step_fn, args.steps, args.warmup, barrier)
+    status_bits = ctx.poll_status()
+    t = torch.tensor([ms], dtype=torch.float64, device=dev)
+    if dist:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    ms_max = float(t.item())
+    ms_per_step = ms_max / args.steps
+    kv_per_step = work.bytes["kv"] * layers
+    value = world * kv_per_step / (ms_per_step * 1e-3) / 1e9  # same per-rank byte count up to the length draw
+
+    peak, peak_kind = measured_peak()
+    launch_us = ms / args.steps / per_step * 1e3  # this rank's average launch duration
+    achieved = work.bytes["total"] / (launch_us * 1e-6) / 1e9
+    traffic = read_traffic_note() if shape is wl.DRAFT_DECODE else None
+
+    result = {
+        "metric": METRIC, "value": round(value, 1), "unit": "GB/s", "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": round(ms_per_step, 5), "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": shape.name, "batch_per_gpu": shape.batch, "num_q_heads": shape.num_q_heads,
+                   "num_kv_heads": shape.num_kv_heads, "head_dim": shape.head_dim, "page_size": wl.PAGE,
+                   "kv_tokens_per_gpu": work.bytes["tokens"], "layers_per_step": layers,
+                   "kv_bytes_per_step_per_gpu": kv_per_step,
+                   "l2": f"inputs larger than L2: {layers} KV pools of {work.bytes['kv'] / 1e6:.1f} MB rotate",
+                   "launch": f"one CUDA graph of {per_step} kernels per step" if use_graph else "stream launches",
+                   "parallelism": f"dp{world} by sequence, no collective"},
+        "pct_of_nominal_8TBs": round(100 * value / world / NOMINAL_HBM_GBS, 2),
+        "gpu_launches": per_step * args.steps,
+        "device_status_bits": status_bits,
+        "clocks": clk.summary(),
+        "roofline": {"bound": "hbm", "kernel": "decode_kernel", "achieved": round(achieved, 1), "peak": peak,
+                     "peak_kind": f"of {peak_kind}", "unit": "GB/s", "frac": round(achieved / peak, 4),
+                     "traffic": traffic, "algorithmic_bytes_per_launch": work.bytes["total"],
+                     "avg_launch_us": round(launch_us, 3)},
+    }
+
+    if rank == 0 and not args.profile:
+        result["e2e"] = run_e2e(ctx, work, max(3, min(args.steps, 50)), world)
+        if world == 1:
+            if not args.no_extras:
+                result["target_shaped_decode"] = run_target_decode(ctx, dev, peak)
+                result["step_scoring"] = run_step_scoring(ctx, dev)
+            result["cpu_baseline"] = run_cpu_baseline(work)
+    if dist:
+        dist.barrier()
+        dist.destroy_process_group()
+    if rank == 0:
+        print(json.dumps(result), flush=True)
+
+
+def read_traffic_note():
+    """DRAM bytes per decode launch from the committed ncu summary; null once the kernel source has
+    changed since the counters were taken."""
+    note = ROOT / "profiles" / "decode_kernel_draft_shaped.traffic.txt"
+    if not note.exists():
+        return None
+    kv = dict(l.split("=", 1) for l in note.read_text().splitlines() if "=" in l and not l.startswith("#"))
+    src = ROOT / "paper_2512_05033_b200" / "csrc" / "arb_decode.cu"
+    if kv.get("source_sha1", "").strip() != hashlib.sha1(src.read_bytes()).hexdigest():
+        return None
+    try:
+        return float(kv["dram_bytes_per_launch"])
+    except Exception:
+        return None
+
+
+def run_e2e(ctx, work: DecodeWorkload, steps: int, world: int):
+    """Same step through arb_attn_host: per call, q / block table / lengths come from pinned host
+    memory and out goes back to pinned host memory, all inside the timed region.  The KV cache stays
+    resident: it is state of the generation loop, not an input of a step."""
+    i = work.inp
+    qh = i.q.cpu().pin_memory()
+    bth = i.block_table.cpu().pin_memory()
+    slh = i.seq_lens.cpu().pin_memory()
+    qlh = i.q_lens.cpu().pin_memory()
+    outh = torch.empty_like(qh).pin_memory()
+
+    def step():
+        for k, v in work.pools:
+            ctx.attn_host(qh, k, v, bth, slh, qlh, 1, out_host=outh)
+
+    for _ in range(3):
+        step()
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    for _ in range(steps):
+        step()
+    torch.cuda.synchronize()
+    dt = (time.perf_counter() - t0) / steps
+    h2d = (qh.numel() * qh.element_size() + bth.numel() * 4 + slh.numel() * 4 + qlh.numel() * 4) * work.layers
+    d2h = outh.numel() * outh.element_size() * work.layers
+    return {"value": round(world * work.bytes["kv"] * work.layers / dt / 1e9, 1), "unit": "GB/s",
+            "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": round(dt * 1e3, 4),
+            "note": "arb_attn_host per layer call; KV cache resident; measured on rank 0, scaled by ranks"}
+
+
+def run_target_decode(ctx, dev, peak):
+    """Supplementary: target-shaped decode (batch 16, 32/8 heads, prefixes in [4k, 32k]), 2 pools of 1.2 GB."""
+    shape = wl.TARGET_DECODE
+    work = DecodeWorkload(shape, 2, dev, seed=shape.seed)
+    step_fn, per_step = make_step(ctx, work, use_graph=False)
+    ms = time_steps(step_fn, 20, 3)
+    us = ms / 20 / per_step * 1e3
+    gbs = work.bytes["total"] / (us * 1e-6) / 1e9
+    return {"kv_tokens": work.bytes["tokens"], "us_per_call": round(us, 2), "gbs": round(gbs, 1),
+            "frac_of_measured": round(gbs / peak, 4), "pct_of_nominal_8TBs": round(100 * gbs / NOMINAL_HBM_GBS, 2)}
+
+
+def run_step_scoring(ctx, dev):
+    """Supplementary: step scoring + routing (batch 32, 28/4 heads, prefixes in [2k, 16k], steps of 16..128
+    tokens): chunk arb_attn (one layer call) + arb_route + arb_rollback per tau."""
+    shape = wl.STEP_SCORING
+    inp = wl.make_attn_inputs(shape, device=dev, seed=shape.seed)
+    r = wl.make_router_inputs(shape.batch, shape.hidden, shape.dtype, device=dev, seed=shape.seed,
+                              b_std=0.1 ** 0.5, taus=(0.3, 0.5, 0.7))
+    out = torch.empty_like(inp.q)
+    max_q = int(inp.q_lens.max())
+    step_lens = inp.q_lens.clone()
+    scores = torch.empty(shape.batch, dtype=torch.float32, device=dev)
+    dec = torch.empty(shape.batch, dtype=torch.uint8, device=dev)
+    seq0 = inp.seq_lens.clone()
+    res = {}
+    esc = {}
+
+    def one(tau):
+        inp.seq_lens.copy_(seq0)  # restore the lengths the previous rollback changed (outside the path)
+        ctx.attn(inp.q, inp.k_pages, inp.v_pages, inp.block_table, inp.seq_lens, inp.q_lens, max_q, out=out)
+        ctx.route(r.hidden, r.w, r.b, tau, scores=scores, decisions=dec)
+        ctx.rollback(inp.seq_lens, step_lens, dec)
+
+    for tau in r.taus:
+        one(tau)
+        torch.cuda.synchronize()
+        ms = time_steps(lambda: one(tau), 5, 3)
+        res[str(tau)] = round(shape.batch / (ms / 5 * 1e-3), 1)
+        esc[str(tau)] = float(dec.float().mean().item())
+    ms_route = time_steps(lambda: ctx.route(r.hidden, r.w, r.b, 0.5, scores=scores, decisions=dec), 200, 10)
+    b = attn_bytes(shape, seq0.cpu().to(torch.int64), inp.q_lens.cpu().to(torch.int64))
+    return {"steps_scored_routed_per_s": res, "escalation_rate": esc, "layer_calls_per_step": 1,
+            "route_only_steps_per_s": round(shape.batch / (ms_route / 200 * 1e-3), 1),
+            "kv_tokens": b["tokens"], "rows": int(inp.q_lens.sum())}
+
+
+def run_cpu_baseline(work: DecodeWorkload):
+    """The fp64 oracle, as it stands, on the host cores: whole steps of the same batch."""
+    from oracle import oracle
+    i = work.inp
+    bt, sl, ql = i.block_table.cpu(), i.seq_lens.cpu(), i.q_lens.cpu()
+    q = i.q.cpu()
+    pools = [(k.cpu(), v.cpu()) for k, v in work.pools]
+    done, t_used = 0, 0.0
+    while t_used < 10.0:  # whole steps (all layers) until about ten seconds of CPU work are done
+        for k, v in pools:
+            t0 = time.perf_counter()
+            oracle.attn(q, k, v, bt, sl, ql)
+            t_used += time.perf_counter() - t0
+            done += 1
+    return {"value": round(work.bytes["kv"] * done / t_used / 1e9, 4), "unit": "GB/s",
+            "cores": oracle.num_threads(), "kind": "oracle",
+            "sample": f"{done // work.layers} whole steps = {done} layer calls of the full draft-shaped batch "
+                      f"({work.bytes['tokens']} KV tokens each), {t_used:.1f} s"}
+
+
+# ------------------------------------------------------------------------------------------------
+# reference arm: the oracle on the host cores
+# ------------------------------------------------------------------------------------------------
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from oracle import oracle
+    shape = wl.DRAFT_DECODE
+    inp = wl.make_attn_inputs(shape, device="cpu", seed=shape.seed)
+    # calibrate on one sequence, then pick how many sequences of the batch one step covers so that
+    # the K timed steps end within about two minutes
+    sub = lambda m: (inp.q[:m], inp.block_table[:m], inp.seq_lens[:m], inp.q_lens[:m])
+    q, bt, sl, ql = sub(1)
+    oracle.attn(q, inp.k_pages, inp.v_pages, bt, sl, ql)
+    t0 = time.perf_counter()
+    oracle.attn(q, inp.k_pages, inp.v_pages, bt, sl, ql)
+    per_token = (time.perf_counter() - t0) / int(sl.sum())
+    budget = 120.0 / max(args.steps, 1)
+    m, tok = 1, int(inp.seq_lens[0])
+    while m < shape.batch and (tok + int(inp.seq_lens[m])) * per_token <= budget:
+        tok += int(inp.seq_lens[m])
+        m += 1
+    q, bt, sl, ql = sub(m)
+    step = lambda: oracle.attn(q, inp.k_pages, inp.v_pages, bt, sl, ql)
+    for _ in range(args.warmup):
+        step()
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        step()
+    dt = (time.perf_counter() - t0) / args.steps
+    b = attn_bytes(shape, sl.to(torch.int64), ql.to(torch.int64))
+    value = round(b["kv"] / dt / 1e9, 4)
+    sample = f"one layer call over the first {m} of {shape.batch} sequences ({b['tokens']} KV tokens) per step"
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": "GB/s",
+        "n_gpus": int(os.environ.get("WORLD_SIZE", "1")), "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": round(dt * 1e3, 3), "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f64", "data": "synthetic",
+        "config": {"workload": shape.name, "batch_per_gpu": shape.batch, "num_q_heads": shape.num_q_heads,
+                   "num_kv_heads": shape.num_kv_heads, "head_dim": shape.head_dim, "page_size": wl.PAGE,
+                   "sample": sample},
+        "cpu_baseline": {"value": value, "unit": "GB/s", "cores": oracle.num_threads(), "kind": "oracle",
+                         "sample": sample},
+        "e2e": {"value": value, "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=2000)
+    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--impl", choices=("ours", "reference"), default="ours")
+    ap.add_argument("--no-graph", action="store_true", help="launch on the stream instead of replaying a CUDA graph")
+    ap.add_argument("--no-extras", action="store_true", help="skip the supplementary workloads")
+    ap.add_argument("--workload", choices=("draft", "target"), default="draft",
+                    help="decode workload of the timed loop (the headline is draft)")
+    ap.add_argument("--layers", type=int, default=0, help="KV pools rotated per step (default 16 draft, 2 target)")
+    ap.add_argument("--profile", action="store_true",
+                    help="for runs under ncu: stream launches, no e2e / extras / CPU baseline")
+    args = ap.parse_args()
+    if args.warmup < 3:
+        args.warmup = 3
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

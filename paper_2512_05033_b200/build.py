@@ -51,7 +51,8 @@ def build(force: bool = False, verbose: bool = False) -> Path:
     objs = [OBJ / (s.stem + ".o") for s in _sources()]
     if force or jobs or _stale(LIB, objs):
         tmp = LIB.with_suffix(f".tmp{os.getpid()}.so")
-        subprocess.check_call([NVCC, "-shared", "-o", str(tmp), *map(str, objs), "-lcudart"])
+        subprocess.check_call([NVCC, "-shared", "-Wno-deprecated-gpu-targets", "-o", str(tmp), *map(str, objs),
+                               "-lcudart"])
         os.replace(tmp, LIB)
     return LIB
 

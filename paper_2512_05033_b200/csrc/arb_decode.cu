@@ -10,11 +10,20 @@
 //
 // Inside a CTA one producer warp walks its pages and issues one bulk (TMA) copy per (page, head)
 // tile of K and of V -- 16 rows x head_dim, contiguous in the head-major page layout -- into a
-// shared-memory ring guarded by full/empty mbarriers.  Four consumer warps take tiles round-robin.
-// A segment is processed in sub-partitions of up to 512 tokens: q.K for every tile (fp32 FMAs on
-// the unpacked 16-byte vectors, reduced across the lanes of a row with a transposing shuffle
-// reduction) into a score buffer, one block-wide max / exp2 / sum pass, then P.V into per-lane
-// fp32 accumulators that live across sub-partitions (rescaled when the running max moves).
+// shared-memory ring guarded by full/empty mbarriers; sixteen lanes issue in parallel, one ring
+// stage each.  Four consumer warps take tiles round-robin.  A segment is processed in
+// sub-partitions of up to 512 tokens: q.K for every tile into a score buffer, one block-wide
+// max / exp2 / sum pass, then P.V into per-lane fp32 accumulators that live across sub-partitions
+// (rescaled when the running max moves).
+//
+// Arithmetic.  bf16 q.K uses the mixed-precision FMA of sm_100 (bf16 x bf16 + fp32 -> fp32, the
+// product is exact), so neither operand is unpacked; eight lanes share a K row, each owning 16 of
+// its 128 dims, and the lanes' partial dot products meet in a transposing shuffle reduction.  P.V
+// keeps P in fp32: V is unpacked with one shift or mask per element, shared by the whole group.
+//
+// Split combine.  Partials of one (sequence, kv head) lie in consecutive workspace slots.  The CTA
+// that arrives last notes the job and, once its own pages are done and the ring is idle, pulls the
+// partials into shared memory with bulk copies and merges them there.
 #include "arb_common.cuh"
 
 namespace arb {
@@ -24,11 +33,10 @@ namespace {
 constexpr int kConsWarps = 4;
 constexpr int kConsThreads = kConsWarps * 32;
 constexpr int kThreads = kConsThreads + 32;  // + producer warp
-constexpr int kStages = 16;
 constexpr int kSubPages = 32;                // pages per sub-partition
 constexpr int kSubTokens = kSubPages * kPage;
 constexpr int kMinChunk = 4;                 // fewest pages worth giving a CTA
-constexpr int kCtasPerSm = 2;
+constexpr int kMaxCtasPerSm = 3;
 
 struct DecodeArgs {
     const char *q;
@@ -38,8 +46,8 @@ struct DecodeArgs {
     const int32_t *seq_lens;
     const int32_t *q_lens;
     char *out;
-    float *part_o;    // [slots][G][D]   un-normalised partial outputs
-    float *part_ml;   // [slots][G][2]   running max (log2 domain) and sum
+    float *part_o;    // [slots][G][D]    un-normalised partial outputs
+    float *part_ml;   // [slots][GP][2]   running max (log2 domain) and sum
     int *counters;    // [batch * Hkv]
     uint32_t *status;
     int batch, Hq, Hkv, num_pages, max_pages;
@@ -48,27 +56,40 @@ struct DecodeArgs {
 
 template <typename T, int D, int G>
 struct Cfg {
-    static constexpr int EPL = Elt<T>::kPerVec;          // elements per lane (one 16-byte vector)
+    static constexpr bool kBf16 = sizeof(T) == 2;
+    static constexpr int EPL = Elt<T>::kPerVec;          // elements in one 16-byte vector
     static constexpr int ROW_BYTES = D * (int)sizeof(T);
-    static constexpr int LPR = ROW_BYTES / 16;           // lanes per K/V row: 8, 16 or 32
+    // P.V mapping: one 16-byte vector per lane
+    static constexpr int LPR = ROW_BYTES / 16;           // lanes per V row: 8, 16 or 32
     static constexpr int RPP = 32 / LPR;                 // rows a warp reads per pass
-    static constexpr int NPASS = kPage / RPP;            // passes per tile
-    static constexpr int PB = NPASS < 8 ? NPASS : 8;     // passes per reduction batch
-    static constexpr int NB = NPASS / PB;
+    static constexpr int NPASS = kPage / RPP;
+    // q.K mapping: bf16 rows are shared by 8 lanes (CPL vectors each); fp32 rows as for P.V
+    static constexpr int QLPR = kBf16 ? 8 : LPR;
+    static constexpr int CPL = kBf16 ? ROW_BYTES / 128 : 1;  // 16-byte vectors per lane and row
+    static constexpr int QRPP = 32 / QLPR;
+    static constexpr int QNPASS = kPage / QRPP;
+    static constexpr int PB = QNPASS < 8 ? QNPASS : 8;   // passes per reduction batch
+    static constexpr int NB = QNPASS / PB;
     static constexpr int NV = PB * G;                    // partial dot products per lane and batch
-    static constexpr int NVP = (NV + LPR - 1) / LPR * LPR;
+    static constexpr int NVP = (NV + QLPR - 1) / QLPR * QLPR;
     static constexpr int GP = (G + 3) / 4 * 4;           // heads padded to whole float4s
     static constexpr int TILE_BYTES = kPage * ROW_BYTES;
-    static constexpr int RING_BYTES = kStages * TILE_BYTES;
+    static constexpr int CTAS = (kBf16 && G <= 4) ? 3 : 2;   // resident CTAs per SM aimed at
+    static constexpr int STAGES = (CTAS == 3) ? 12 : (TILE_BYTES > 4096 ? 8 : 16);
+    static constexpr int BATCH = STAGES < 16 ? STAGES : 16;  // producer lanes issuing side by side
+    static constexpr int RING_BYTES = STAGES * TILE_BYTES;
     static constexpr int LOGIT_BYTES = kSubTokens * GP * 4;
     static constexpr int OSM_BYTES = kConsWarps * G * D * 4;
     static constexpr int UNI_BYTES = LOGIT_BYTES > OSM_BYTES ? LOGIT_BYTES : OSM_BYTES;
     static_assert(LPR == 8 || LPR == 16 || LPR == 32, "row must be 128, 256 or 512 bytes");
 };
 
+constexpr int kMaxStages = 16;
+
 struct SmemTail {  // small fixed part after ring + score buffer
-    uint64_t full[kStages];
-    uint64_t empty[kStages];
+    uint64_t full[kMaxStages];
+    uint64_t empty[kMaxStages];
+    uint64_t cbar;  // split-combine staging
     float red_max[kConsWarps][kMaxGroup];
     float red_sum[kConsWarps][kMaxGroup];
     int abort;
@@ -115,10 +136,26 @@ __device__ __forceinline__ bool next_segment(int &cur, int r1, const int *pref, 
     return true;
 }
 
+// acc += q.lo * k.lo + q.hi * k.hi for two packed bf16 pairs; products are exact, sums round in fp32
+__device__ __forceinline__ float fma_bf16x2(uint32_t q, uint32_t k, float acc) {
+    asm("{\n\t.reg .b16 ql, qh, kl, kh;\n\t"
+        "mov.b32 {ql, qh}, %1;\n\t"
+        "mov.b32 {kl, kh}, %2;\n\t"
+        "fma.rn.f32.bf16 %0, ql, kl, %0;\n\t"
+        "fma.rn.f32.bf16 %0, qh, kh, %0;\n\t}"
+        : "+f"(acc)
+        : "r"(q), "r"(k));
+    return acc;
+}
+
+__device__ __forceinline__ void fence_proxy_async_all() { asm volatile("fence.proxy.async;" ::: "memory"); }
+
 template <typename T, int D, int G>
-__global__ void __launch_bounds__(kThreads, kCtasPerSm) decode_kernel(const DecodeArgs a) {
+__global__ void __launch_bounds__(kThreads, Cfg<T, D, G>::CTAS) decode_kernel(const DecodeArgs a) {
     using C = Cfg<T, D, G>;
     constexpr int EPL = C::EPL, LPR = C::LPR, RPP = C::RPP, GP = C::GP;
+    constexpr int QLPR = C::QLPR, QRPP = C::QRPP, CPL = C::CPL, STAGES = C::STAGES;
+    constexpr int QW = C::kBf16 ? CPL * 4 : EPL;  // 32-bit q registers per head and lane
 
     extern __shared__ char smem_raw[];
     char *base = reinterpret_cast<char *>((reinterpret_cast<uintptr_t>(smem_raw) + 127) & ~uintptr_t(127));
@@ -133,10 +170,11 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) decode_kernel(const Deco
 
     // ---- prologue: lengths -> page counts and q row offsets, scanned by warp 0 -----------------
     if (tid == 0) {
-        for (int s = 0; s < kStages; ++s) {
+        for (int s = 0; s < STAGES; ++s) {
             mbar_init(&tail->full[s], 1);
             mbar_init(&tail->empty[s], 1);
         }
+        mbar_init(&tail->cbar, 1);
         tail->abort = 0;
         tail->is_last = 0;
         mbar_fence_init();
@@ -191,6 +229,8 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) decode_kernel(const Deco
 
     if (warp == kConsWarps) {
         // ================================ producer warp ==========================================
+        // Lanes 0..BATCH-1 each own one ring stage at a time: wait until it is free, then issue the
+        // copy.  A batch never exceeds the ring, so a lane is at most one phase behind its barrier.
         uint32_t c = 0;
         int cur = r0;
         Segment s;
@@ -209,10 +249,11 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) decode_kernel(const Deco
                 for (int ph = 0; ph < 2; ++ph) {
                     const char *pool = ph ? a.v_pages : a.k_pages;
 #pragma unroll 1
-                    for (int i = 0; i < np; ++i, ++c) {
-                        const int pg = __shfl_sync(0xffffffffu, pid, i);
-                        if (lane == 0) {
-                            const uint32_t st = c % kStages, par = (c / kStages) & 1u;
+                    for (int i0 = 0; i0 < np; i0 += C::BATCH) {
+                        const int i = i0 + lane;
+                        const int pg = __shfl_sync(0xffffffffu, pid, i & 31);
+                        if (lane < C::BATCH && i < np) {
+                            const uint32_t cc = c + i, st = cc % STAGES, par = (cc / STAGES) & 1u;
                             if (mbar_wait(&tail->empty[st], par ^ 1u, abort, a.status)) {
                                 mbar_arrive_expect_tx(&tail->full[st], C::TILE_BYTES);
                                 bulk_load(ring + st * C::TILE_BYTES,
@@ -220,19 +261,20 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) decode_kernel(const Deco
                                           &tail->full[st]);
                             }
                         }
+                        __syncwarp();
                     }
+                    c += np;
                 }
-                __syncwarp();
             }
         }
         // After a timeout the consumers may have left copies unconsumed: wait (bounded) for the
         // last ring's worth so that no copy is in flight into this CTA's memory when it exits.
         if (lane == 0 && *abort) {
-            const uint32_t n = c < (uint32_t)kStages ? c : (uint32_t)kStages;
+            const uint32_t n = c < (uint32_t)STAGES ? c : (uint32_t)STAGES;
             for (uint32_t i = 0; i < n; ++i) {
                 const uint32_t cc = c - 1 - i;
                 const long long t0 = clock64();
-                while (!mbar_try_wait(&tail->full[cc % kStages], (cc / kStages) & 1u) &&
+                while (!mbar_try_wait(&tail->full[cc % STAGES], (cc / STAGES) & 1u) &&
                        clock64() - t0 < (1ll << 24)) {
                 }
             }
@@ -241,22 +283,40 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) decode_kernel(const Deco
     }
 
     // ==================================== consumer warps ==========================================
-    const int lg = lane % LPR;  // lane within the row group (which 16-byte column of a row)
-    const int rg = lane / LPR;  // row group: which of the RPP rows of a pass
+    const int lg = lane % LPR, rg = lane / LPR;      // P.V: vector column within a row, row of a pass
+    const int qlg = lane % QLPR, qrg = lane / QLPR;  // q.K: the same for its own row sharing
     uint32_t c_base = 0;
     int cur = r0;
     Segment s;
+    // split-combine jobs this CTA has to finish (only the first and last segment of a range can be
+    // part of a longer (sequence, kv head), so two slots are enough)
+    int pend_n = 0;
+    int pend_slot0[2], pend_parts[2];
+    size_t pend_out[2];
+
     while (next_segment(cur, r1, pref, B, Hkv, chunk, a.seq_lens, s)) {
         const int qrow = row0[s.b];
-        float qf[G][EPL];
+        // q of this kv head's group: packed bf16 pairs, or fp32 pre-multiplied by the scale
+        uint32_t qp[G][QW];
 #pragma unroll
         for (int h = 0; h < G; ++h) {
-            const uint4 v = __ldg(reinterpret_cast<const uint4 *>(
-                a.q + (((size_t)qrow * a.Hq + s.kvh * G + h) * D + lg * EPL) * sizeof(T)));
-            Elt<T>::unpack(v, qf[h]);
+            const char *qh = a.q + ((size_t)qrow * a.Hq + s.kvh * G + h) * D * sizeof(T);
+            if constexpr (C::kBf16) {
 #pragma unroll
-            for (int e = 0; e < EPL; ++e) qf[h][e] *= a.scale_log2;
+                for (int cp = 0; cp < CPL; ++cp) {
+                    const uint4 v = __ldg(reinterpret_cast<const uint4 *>(qh + (qlg + 8 * cp) * 16));
+                    qp[h][4 * cp + 0] = v.x; qp[h][4 * cp + 1] = v.y;
+                    qp[h][4 * cp + 2] = v.z; qp[h][4 * cp + 3] = v.w;
+                }
+            } else {
+                const uint4 v = __ldg(reinterpret_cast<const uint4 *>(qh + qlg * 16));
+                qp[h][0] = __float_as_uint(__uint_as_float(v.x) * a.scale_log2);
+                qp[h][1] = __float_as_uint(__uint_as_float(v.y) * a.scale_log2);
+                qp[h][2] = __float_as_uint(__uint_as_float(v.z) * a.scale_log2);
+                qp[h][3] = __float_as_uint(__uint_as_float(v.w) * a.scale_log2);
+            }
         }
+        const float sc = C::kBf16 ? a.scale_log2 : 1.0f;
         float m_run[G], l_run[G], o[G][EPL];
 #pragma unroll
         for (int h = 0; h < G; ++h) {
@@ -272,7 +332,7 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) decode_kernel(const Deco
 
             // ---- phase A: scores of this warp's K tiles -------------------------------------------
             for (int t = warp; t < np; t += kConsWarps) {
-                const uint32_t cc = c_base + t, st = cc % kStages, par = (cc / kStages) & 1u;
+                const uint32_t cc = c_base + t, st = cc % STAGES, par = (cc / STAGES) & 1u;
                 mbar_wait(&tail->full[st], par, abort, a.status);
                 const char *tile = ring + st * C::TILE_BYTES;
 #pragma unroll
@@ -282,23 +342,41 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) decode_kernel(const Deco
                     for (int i = 0; i < C::NVP; ++i) acc[i] = 0.f;
 #pragma unroll
                     for (int ps = 0; ps < C::PB; ++ps) {
-                        const int r = (nb * C::PB + ps) * RPP + rg;
-                        const uint4 kv = *reinterpret_cast<const uint4 *>(tile + r * C::ROW_BYTES + lg * 16);
-                        float kf[EPL];
-                        Elt<T>::unpack(kv, kf);
+                        const int r = (nb * C::PB + ps) * QRPP + qrg;
+                        if constexpr (C::kBf16) {
 #pragma unroll
-                        for (int h = 0; h < G; ++h)
+                            for (int cp = 0; cp < CPL; ++cp) {
+                                const uint4 kv = *reinterpret_cast<const uint4 *>(tile + r * C::ROW_BYTES +
+                                                                                  (qlg + 8 * cp) * 16);
 #pragma unroll
-                            for (int e = 0; e < EPL; ++e) acc[ps * G + h] = fmaf(qf[h][e], kf[e], acc[ps * G + h]);
+                                for (int h = 0; h < G; ++h) {
+                                    float x = acc[ps * G + h];
+                                    x = fma_bf16x2(qp[h][4 * cp + 0], kv.x, x);
+                                    x = fma_bf16x2(qp[h][4 * cp + 1], kv.y, x);
+                                    x = fma_bf16x2(qp[h][4 * cp + 2], kv.z, x);
+                                    x = fma_bf16x2(qp[h][4 * cp + 3], kv.w, x);
+                                    acc[ps * G + h] = x;
+                                }
+                            }
+                        } else {
+                            const uint4 kv = *reinterpret_cast<const uint4 *>(tile + r * C::ROW_BYTES + qlg * 16);
+                            float kf[EPL];
+                            Elt<T>::unpack(kv, kf);
+#pragma unroll
+                            for (int h = 0; h < G; ++h)
+#pragma unroll
+                                for (int e = 0; e < EPL; ++e)
+                                    acc[ps * G + h] = fmaf(__uint_as_float(qp[h][e]), kf[e], acc[ps * G + h]);
+                        }
                     }
-                    transpose_reduce<C::NVP, LPR>(acc, lg);
+                    transpose_reduce<C::NVP, QLPR>(acc, qlg);
 #pragma unroll
-                    for (int j = 0; j < C::NVP / LPR; ++j) {
-                        const int idx = j + (C::NVP / LPR) * lg;
+                    for (int j = 0; j < C::NVP / QLPR; ++j) {
+                        const int idx = j + (C::NVP / QLPR) * qlg;
                         if (idx < C::NV) {
                             const int ps = idx / G, h = idx - ps * G;
-                            const int token = t * kPage + (nb * C::PB + ps) * RPP + rg;
-                            uni[token * GP + h] = acc[j];
+                            const int token = t * kPage + (nb * C::PB + ps) * QRPP + qrg;
+                            uni[token * GP + h] = acc[j] * sc;
                         }
                     }
                 }
@@ -369,7 +447,7 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) decode_kernel(const Deco
 
             // ---- phase C: P.V over this warp's V tiles --------------------------------------------
             for (int t = warp; t < np; t += kConsWarps) {
-                const uint32_t cc = c_base + np + t, st = cc % kStages, par = (cc / kStages) & 1u;
+                const uint32_t cc = c_base + np + t, st = cc % STAGES, par = (cc / STAGES) & 1u;
                 mbar_wait(&tail->full[st], par, abort, a.status);
                 const char *tile = ring + st * C::TILE_BYTES;
 #pragma unroll
@@ -438,11 +516,12 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) decode_kernel(const Deco
             if (tid == 0) {
 #pragma unroll
                 for (int h = 0; h < G; ++h) {
-                    a.part_ml[(slot * G + h) * 2 + 0] = m_run[h];
-                    a.part_ml[(slot * G + h) * 2 + 1] = l_run[h];
+                    a.part_ml[(slot * GP + h) * 2 + 0] = m_run[h];
+                    a.part_ml[(slot * GP + h) * 2 + 1] = l_run[h];
                 }
             }
             __threadfence();
+            fence_proxy_async_all();  // the partials are read back through bulk copies
             named_barrier(1, kConsThreads);
             if (tid == 0) {
                 const int old = atomicAdd(&a.counters[s.bk], 1);
@@ -451,29 +530,102 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) decode_kernel(const Deco
                 tail->is_last = last;
             }
             named_barrier(1, kConsThreads);
-            if (tail->is_last) {
-                __threadfence();
-                const size_t slot0 = (size_t)s.bk + s.c_first;
-                for (int idx = tid; idx < G * D; idx += kConsThreads) {
-                    const int h = idx / D;
-                    float M = -INFINITY;
-                    for (int p = 0; p < s.nparts; ++p) M = fmaxf(M, __ldcg(&a.part_ml[((slot0 + p) * G + h) * 2]));
-                    float l = 0.f, acc = 0.f;
-                    for (int p = 0; p < s.nparts; ++p) {
-                        const float w = fast_exp2(__ldcg(&a.part_ml[((slot0 + p) * G + h) * 2]) - M);
-                        l = fmaf(w, __ldcg(&a.part_ml[((slot0 + p) * G + h) * 2 + 1]), l);
-                        acc = fmaf(w, __ldcg(&a.part_o[(slot0 + p) * G * D + idx]), acc);
-                    }
-                    reinterpret_cast<T *>(a.out)[out_base + idx] = Elt<T>::from_float(acc / l);
-                }
+            if (tail->is_last && pend_n < 2) {
+                pend_slot0[pend_n] = s.bk + s.c_first;
+                pend_parts[pend_n] = s.nparts;
+                pend_out[pend_n] = out_base;
+                ++pend_n;
             }
             named_barrier(1, kConsThreads);
         }
+    }
+
+    // ---- split combine of the (sequence, kv head)s this CTA was the last to reach -----------------
+    // All tiles have been consumed and the producer issues nothing more, so the ring is free:
+    // [ max/sum records of all parts | as many partial outputs as fit ].
+    uint32_t cphase = 0;
+    for (int j = 0; j < pend_n; ++j) {
+        const int nparts = pend_parts[j];
+        const size_t slot0 = (size_t)pend_slot0[j];
+        __threadfence();
+        const uint32_t ml_bytes = (uint32_t)nparts * GP * 8u;
+        const uint32_t ml_area = (ml_bytes + 127u) & ~127u;
+        float *ml = reinterpret_cast<float *>(ring);
+        float *po = reinterpret_cast<float *>(ring + ml_area);
+        const int per_piece = (C::RING_BYTES - (int)ml_area) / (G * D * 4);
+        if (per_piece < 1) {
+            // more parts than the ring can describe (far more CTAs than this part has SMs for):
+            // merge straight from global memory
+            for (int idx = tid; idx < G * D; idx += kConsThreads) {
+                const int h = idx / D;
+                float m = -INFINITY;
+                for (int p = 0; p < nparts; ++p) m = fmaxf(m, __ldcg(&a.part_ml[((slot0 + p) * GP + h) * 2]));
+                float l = 0.f, x = 0.f;
+                for (int p = 0; p < nparts; ++p) {
+                    const float w = fast_exp2(__ldcg(&a.part_ml[((slot0 + p) * GP + h) * 2]) - m);
+                    l = fmaf(w, __ldcg(&a.part_ml[((slot0 + p) * GP + h) * 2 + 1]), l);
+                    x = fmaf(w, __ldcg(&a.part_o[(slot0 + p) * G * D + idx]), x);
+                }
+                reinterpret_cast<T *>(a.out)[pend_out[j] + idx] = Elt<T>::from_float(x / l);
+            }
+            continue;
+        }
+        if (tid == 0) {
+            fence_proxy_async_all();
+            mbar_arrive_expect_tx(&tail->cbar, ml_bytes);
+            bulk_load(ml, a.part_ml + slot0 * GP * 2, ml_bytes, &tail->cbar);
+        }
+        mbar_wait(&tail->cbar, cphase, abort, a.status);
+        cphase ^= 1u;
+        named_barrier(1, kConsThreads);  // nobody is still polling this phase when the next copy is armed
+        constexpr int NK = (G * D + kConsThreads - 1) / kConsThreads;
+        float M[NK], lsum[NK], acc[NK];
+#pragma unroll
+        for (int k = 0; k < NK; ++k) {
+            const int idx = tid + k * kConsThreads;
+            const int h = idx < G * D ? idx / D : 0;
+            float m = -INFINITY;
+            for (int p = 0; p < nparts; ++p) m = fmaxf(m, ml[(p * GP + h) * 2]);
+            float l = 0.f;
+            for (int p = 0; p < nparts; ++p) l = fmaf(fast_exp2(ml[(p * GP + h) * 2] - m), ml[(p * GP + h) * 2 + 1], l);
+            M[k] = m;
+            lsum[k] = l;
+            acc[k] = 0.f;
+        }
+        for (int p0 = 0; p0 < nparts; p0 += per_piece) {
+            const int np = min(per_piece, nparts - p0);
+            if (tid == 0) {
+                const uint32_t bytes = (uint32_t)np * G * D * 4u;
+                mbar_arrive_expect_tx(&tail->cbar, bytes);
+                bulk_load(po, a.part_o + (slot0 + p0) * G * D, bytes, &tail->cbar);
+            }
+            mbar_wait(&tail->cbar, cphase, abort, a.status);
+            cphase ^= 1u;
+#pragma unroll
+            for (int k = 0; k < NK; ++k) {
+                const int idx = tid + k * kConsThreads;
+                if (idx < G * D) {
+                    const int h = idx / D;
+                    float x = acc[k];
+                    for (int p = 0; p < np; ++p)
+                        x = fmaf(fast_exp2(ml[((p0 + p) * GP + h) * 2] - M[k]), po[p * G * D + idx], x);
+                    acc[k] = x;
+                }
+            }
+            named_barrier(1, kConsThreads);  // everyone is done with this piece before the next lands
+        }
+#pragma unroll
+        for (int k = 0; k < NK; ++k) {
+            const int idx = tid + k * kConsThreads;
+            if (idx < G * D) reinterpret_cast<T *>(a.out)[pend_out[j] + idx] = Elt<T>::from_float(acc[k] / lsum[k]);
+        }
+        named_barrier(1, kConsThreads);
     }
 }
 
 template <typename T, int D, int G>
 arb_status launch_one(Ctx *ctx, const DecodeArgs &args, cudaStream_t stream) {
+    using C = Cfg<T, D, G>;
     const size_t smem = smem_bytes<T, D, G>(args.batch);
     static bool attr_set[64] = {};
     if (!attr_set[ctx->device & 63]) {
@@ -482,7 +634,7 @@ arb_status launch_one(Ctx *ctx, const DecodeArgs &args, cudaStream_t stream) {
             return ARB_ERR_CUDA;
         attr_set[ctx->device & 63] = true;
     }
-    decode_kernel<T, D, G><<<decode_grid(ctx->num_sms), kThreads, smem, stream>>>(args);
+    decode_kernel<T, D, G><<<ctx->num_sms * C::CTAS, kThreads, smem, stream>>>(args);
     ctx->launches++;
     return cudaGetLastError() == cudaSuccess ? ARB_OK : ARB_ERR_CUDA;
 }
@@ -502,21 +654,23 @@ arb_status launch_g(Ctx *ctx, int g, const DecodeArgs &args, cudaStream_t stream
     }
 }
 
-}  // namespace
+inline size_t slot_count(const arb_attn_params &p, int num_sms) {
+    return (size_t)p.batch * p.num_kv_heads + (size_t)num_sms * kMaxCtasPerSm;
+}
 
-int decode_grid(int num_sms) { return num_sms * kCtasPerSm; }
+}  // namespace
 
 size_t decode_workspace_bytes(const arb_attn_params &p, int num_sms) {
     const int g = p.num_q_heads / p.num_kv_heads;
-    const size_t slots = (size_t)p.batch * p.num_kv_heads + decode_grid(num_sms);
-    return slots * g * ((size_t)p.head_dim + 2) * sizeof(float);
+    const int gp = (g + 3) / 4 * 4;
+    return slot_count(p, num_sms) * ((size_t)g * p.head_dim + 2 * (size_t)gp) * sizeof(float) + 256;
 }
 
 arb_status launch_decode(Ctx *ctx, const arb_attn_params &p, const void *q, const void *k_pages,
                          const void *v_pages, const int32_t *block_table, const int32_t *seq_lens,
                          const int32_t *q_lens, void *out, cudaStream_t stream) {
     const int g = p.num_q_heads / p.num_kv_heads;
-    const size_t slots = (size_t)p.batch * p.num_kv_heads + decode_grid(ctx->num_sms);
+    const size_t slots = slot_count(p, ctx->num_sms);
     DecodeArgs a;
     a.q = static_cast<const char *>(q);
     a.k_pages = static_cast<const char *>(k_pages);
@@ -526,7 +680,7 @@ arb_status launch_decode(Ctx *ctx, const arb_attn_params &p, const void *q, cons
     a.q_lens = q_lens;
     a.out = static_cast<char *>(out);
     a.part_o = reinterpret_cast<float *>(ctx->workspace);
-    a.part_ml = a.part_o + slots * g * p.head_dim;
+    a.part_ml = a.part_o + ((slots * g * p.head_dim + 63) & ~size_t(63));  // keeps 256-byte alignment
     a.counters = ctx->counters;
     a.status = ctx->status;
     a.batch = p.batch;

@@ -172,10 +172,14 @@ def time_steps(step_fn, steps, warmup, dist_barrier=None):
     return e0.elapsed_time(e1)  # ms
 
 
-def make_step(ctx, work: DecodeWorkload, use_graph: bool):
-    """Returns (callable running one step on the current stream, kernel launches per step)."""
+def make_step(ctx, work: DecodeWorkload, use_graph: bool, overlap: bool = False):
+    """Returns (callable running one step on the current stream, kernel launches per step).
+    overlap: the layer calls of a step share q and read-only caches, so each may start under the
+    tail of the one before it (ARB_ATTN_OVERLAP_PREVIOUS)."""
+    from paper_2512_05033_b200 import binding
     i = work.inp
-    params = ctx.params_for(i.q, i.k_pages, i.block_table, 1)
+    params = ctx.params_for(i.q, i.k_pages, i.block_table, 1,
+                            flags=binding.ATTN_OVERLAP_PREVIOUS if overlap else 0)
     if not use_graph:
         n0 = ctx.launch_count()
         work.step(ctx, params, torch.cuda.current_stream().cuda_stream)
@@ -214,7 +218,8 @@ def run_ours(args):
     layers = args.layers or (LAYERS if shape is wl.DRAFT_DECODE else 2)
     work = DecodeWorkload(shape, layers, dev, seed=shape.seed + 1000 * rank)  # weak scaling: own batch per rank
     use_graph = not (args.no_graph or args.profile)
-    step_fn, per_step = make_step(ctx, work, use_graph)
+    overlap = not args.no_overlap
+    step_fn, per_step = make_step(ctx, work, use_graph, overlap)
 
     with ClockSampler(cuda_physical_index(local)) as clk:
         ms = time_steps(step_fn, args.steps, args.warmup, barrier)
@@ -242,6 +247,8 @@ def run_ours(args):
                    "kv_bytes_per_step_per_gpu": kv_per_step,
                    "l2": f"inputs larger than L2: {layers} KV pools of {work.bytes['kv'] / 1e6:.1f} MB rotate",
                    "launch": f"one CUDA graph of {per_step} kernels per step" if use_graph else "stream launches",
+                   "overlap": "layer calls launched as programmatic dependents (ARB_ATTN_OVERLAP_PREVIOUS)"
+                   if overlap else "none: every call waits for the one before it",
                    "parallelism": f"dp{world} by sequence, no collective"},
         "pct_of_nominal_8TBs": round(100 * value / world / NOMINAL_HBM_GBS, 2),
         "gpu_launches": per_step * args.steps,
@@ -257,6 +264,12 @@ def run_ours(args):
         result["e2e"] = run_e2e(ctx, work, max(3, min(args.steps, 50)), world)
         if world == 1:
             if not args.no_extras:
+                if overlap:  # the same loop with every call fully serialised behind the previous one
+                    fn2, _ = make_step(ctx, work, use_graph, overlap=False)
+                    ms2 = time_steps(fn2, max(20, args.steps // 4), 5)
+                    result["serialised_calls"] = {
+                        "gbs": round(kv_per_step / (ms2 / max(20, args.steps // 4) * 1e-3) / 1e9, 1),
+                        "us_per_call": round(ms2 / max(20, args.steps // 4) / per_step * 1e3, 3)}
                 result["target_shaped_decode"] = run_target_decode(ctx, dev, peak)
                 result["step_scoring"] = run_step_scoring(ctx, dev)
             result["cpu_baseline"] = run_cpu_baseline(work)
@@ -437,6 +450,8 @@ def main():
     ap.add_argument("--impl", choices=("ours", "reference"), default="ours")
     ap.add_argument("--no-graph", action="store_true", help="launch on the stream instead of replaying a CUDA graph")
     ap.add_argument("--no-extras", action="store_true", help="skip the supplementary workloads")
+    ap.add_argument("--no-overlap", action="store_true",
+                    help="do not let a layer call start under the tail of the previous one")
     ap.add_argument("--workload", choices=("draft", "target"), default="draft",
                     help="decode workload of the timed loop (the headline is draft)")
     ap.add_argument("--layers", type=int, default=0, help="KV pools rotated per step (default 16 draft, 2 target)")

@@ -79,7 +79,20 @@ typedef struct {
     int32_t total_q;           /* sum of q_lens (rows of q and out); the host knows it */
     int32_t max_q_len;         /* max of q_lens; 1 selects the decode kernel alone */
     float softmax_scale;       /* <= 0 selects 1/sqrt(head_dim) */
+    uint32_t flags;            /* ARB_ATTN_* bits, 0 for none */
 } arb_attn_params;
+
+/*
+ * arb_attn_params.flags.
+ * ARB_ATTN_OVERLAP_PREVIOUS: the caller states that no input of this call (q, k_pages, v_pages,
+ * block_table, seq_lens, q_lens) is written by the kernel that precedes it on the stream.  The
+ * decode kernel is then launched as a programmatic dependent of that kernel: it may start streaming
+ * KV while its predecessor is still finishing, and waits for the predecessor's completion only
+ * before its first write (out, workspace).  Results are the same as without the flag.  Typical
+ * use: the per-layer calls of one decode token when q and the KV cache of every layer are ready.
+ * Do not set it when the preceding kernel produces q, appends K/V or changes seq_lens.
+ */
+enum { ARB_ATTN_OVERLAP_PREVIOUS = 1u };
 
 /*
  * Create a context on `device`.  workspace_bytes = 0 picks a default that covers every shape the

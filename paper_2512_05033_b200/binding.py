@@ -23,6 +23,7 @@ ARB_OK = 0
 ARB_ERR_INVALID_ARG, ARB_ERR_UNSUPPORTED, ARB_ERR_WORKSPACE, ARB_ERR_CUDA, ARB_ERR_DEVICE_STATUS = 1, 2, 3, 4, 5
 ARB_F32, ARB_BF16 = 0, 1
 DEV_BAD_SEQ_LEN, DEV_BAD_PAGE, DEV_ROLLBACK_UNDERFLOW, DEV_WAIT_TIMEOUT = 1, 2, 4, 8
+ATTN_OVERLAP_PREVIOUS = 1
 
 # every symbol include/arb.h declares
 EXPORTS = ("arb_create", "arb_destroy", "arb_attn_workspace_bytes", "arb_attn", "arb_attn_host",
@@ -33,7 +34,8 @@ class AttnParams(ctypes.Structure):
     _fields_ = [("dtype", ctypes.c_int32), ("batch", ctypes.c_int32), ("num_q_heads", ctypes.c_int32),
                 ("num_kv_heads", ctypes.c_int32), ("head_dim", ctypes.c_int32), ("page_size", ctypes.c_int32),
                 ("num_pages", ctypes.c_int32), ("max_pages_per_seq", ctypes.c_int32),
-                ("total_q", ctypes.c_int32), ("max_q_len", ctypes.c_int32), ("softmax_scale", ctypes.c_float)]
+                ("total_q", ctypes.c_int32), ("max_q_len", ctypes.c_int32), ("softmax_scale", ctypes.c_float),
+                ("flags", ctypes.c_uint32)]
 
 
 _vp, _i32, _f = ctypes.c_void_p, ctypes.c_int32, ctypes.c_float
@@ -93,9 +95,9 @@ def _dev(t: torch.Tensor, name: str, dtype=None) -> int:
 
 
 def attn_params(q_dtype_code, batch, num_q_heads, num_kv_heads, head_dim, num_pages, max_pages_per_seq, total_q,
-                max_q_len, softmax_scale=0.0, page_size=16) -> AttnParams:
+                max_q_len, softmax_scale=0.0, page_size=16, flags=0) -> AttnParams:
     return AttnParams(q_dtype_code, batch, num_q_heads, num_kv_heads, head_dim, page_size, num_pages,
-                      max_pages_per_seq, total_q, max_q_len, softmax_scale)
+                      max_pages_per_seq, total_q, max_q_len, softmax_scale, flags)
 
 
 class Context:
@@ -121,11 +123,13 @@ class Context:
             pass
 
     # -- arb_attn -----------------------------------------------------------------------------
-    def params_for(self, q, k_pages, block_table, max_q_len: int, softmax_scale: float = 0.0) -> AttnParams:
+    def params_for(self, q, k_pages, block_table, max_q_len: int, softmax_scale: float = 0.0,
+                   flags: int = 0) -> AttnParams:
         total_q, Hq, D = q.shape
         num_pages, Hkv, P, _ = k_pages.shape
         B, max_pages = block_table.shape
-        return attn_params(_dtype_code(q), B, Hq, Hkv, D, num_pages, max_pages, total_q, max_q_len, softmax_scale, P)
+        return attn_params(_dtype_code(q), B, Hq, Hkv, D, num_pages, max_pages, total_q, max_q_len, softmax_scale, P,
+                           flags)
 
     def attn(self, q, k_pages, v_pages, block_table, seq_lens, q_lens, max_q_len: int, out=None,
              softmax_scale: float = 0.0, stream=None, params: AttnParams | None = None):

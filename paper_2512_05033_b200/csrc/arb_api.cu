@@ -25,6 +25,7 @@ arb_status check_params(const arb_attn_params *p) {
     if (p->batch > kMaxBatch) return ARB_ERR_UNSUPPORTED;
     if ((long long)p->batch * p->num_kv_heads > kCounters) return ARB_ERR_UNSUPPORTED;
     if ((long long)p->max_pages_per_seq * kPage > (1ll << 30)) return ARB_ERR_UNSUPPORTED;
+    if (p->flags & ~(uint32_t)ARB_ATTN_OVERLAP_PREVIOUS) return ARB_ERR_INVALID_ARG;
     return ARB_OK;
 }
 

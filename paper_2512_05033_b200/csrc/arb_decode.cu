@@ -89,7 +89,7 @@ constexpr int kMaxStages = 16;
 struct SmemTail {  // small fixed part after ring + score buffer
     uint64_t full[kMaxStages];
     uint64_t empty[kMaxStages];
-    uint64_t cbar;  // split-combine staging
+    uint64_t cbar[2];  // split-combine staging, one per buffer
     float red_max[kConsWarps][kMaxGroup];
     float red_sum[kConsWarps][kMaxGroup];
     int abort;
@@ -150,6 +150,13 @@ __device__ __forceinline__ float fma_bf16x2(uint32_t q, uint32_t k, float acc) {
 
 __device__ __forceinline__ void fence_proxy_async_all() { asm volatile("fence.proxy.async;" ::: "memory"); }
 
+// Programmatic dependent launch.  Both are no-ops in a kernel launched the ordinary way.
+//  - let_successor_start: the next kernel on the stream, if launched as a programmatic dependent,
+//    may begin once every CTA of this grid has passed this point or exited.
+//  - wait_for_predecessor: returns when the preceding kernel has completed and its writes are visible.
+__device__ __forceinline__ void let_successor_start() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void wait_for_predecessor() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
 template <typename T, int D, int G>
 __global__ void __launch_bounds__(kThreads, Cfg<T, D, G>::CTAS) decode_kernel(const DecodeArgs a) {
     using C = Cfg<T, D, G>;
@@ -168,13 +175,20 @@ __global__ void __launch_bounds__(kThreads, Cfg<T, D, G>::CTAS) decode_kernel(co
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int B = a.batch, Hkv = a.Hkv;
 
+    // Until wait_for_predecessor() this kernel only reads its inputs (and ORs error bits); every
+    // write to out, the workspace or the arrival counters comes after it.  A successor launched as
+    // a programmatic dependent does the same, so it can stream its KV under this kernel's tail and
+    // still cannot touch the shared workspace before this kernel is complete.
+    let_successor_start();
+
     // ---- prologue: lengths -> page counts and q row offsets, scanned by warp 0 -----------------
     if (tid == 0) {
         for (int s = 0; s < STAGES; ++s) {
             mbar_init(&tail->full[s], 1);
             mbar_init(&tail->empty[s], 1);
         }
-        mbar_init(&tail->cbar, 1);
+        mbar_init(&tail->cbar[0], 1);
+        mbar_init(&tail->cbar[1], 1);
         tail->abort = 0;
         tail->is_last = 0;
         mbar_fence_init();
@@ -188,6 +202,7 @@ __global__ void __launch_bounds__(kThreads, Cfg<T, D, G>::CTAS) decode_kernel(co
             if (L >= 1 && L <= a.max_pages * kPage) {
                 pages = (L + kPage - 1) / kPage;
             } else if (blockIdx.x == 0) {  // no defined result: flag it and zero the row
+                wait_for_predecessor();
                 atomicOr(a.status, (uint32_t)ARB_DEV_BAD_SEQ_LEN);
                 int row = 0;
                 for (int i = 0; i < b; ++i) row += max(a.q_lens[i], 0);
@@ -478,6 +493,7 @@ __global__ void __launch_bounds__(kThreads, Cfg<T, D, G>::CTAS) decode_kernel(co
         }
 
         // ---- segment end: add up the warps' accumulators ---------------------------------------------
+        wait_for_predecessor();  // first write of this CTA comes below; later calls return at once
 #pragma unroll
         for (int off = LPR; off < 32; off <<= 1)
 #pragma unroll
@@ -542,17 +558,18 @@ __global__ void __launch_bounds__(kThreads, Cfg<T, D, G>::CTAS) decode_kernel(co
 
     // ---- split combine of the (sequence, kv head)s this CTA was the last to reach -----------------
     // All tiles have been consumed and the producer issues nothing more, so the ring is free:
-    // [ max/sum records of all parts | as many partial outputs as fit ].
-    uint32_t cphase = 0;
+    // [ max/sum records of all parts | buffer A | buffer B ]; partial outputs stream through A and B
+    // while the previous piece is being added up.
+    uint32_t cph[2] = {0u, 0u};
     for (int j = 0; j < pend_n; ++j) {
         const int nparts = pend_parts[j];
         const size_t slot0 = (size_t)pend_slot0[j];
         __threadfence();
         const uint32_t ml_bytes = (uint32_t)nparts * GP * 8u;
         const uint32_t ml_area = (ml_bytes + 127u) & ~127u;
+        constexpr int PART_BYTES = G * D * 4;
         float *ml = reinterpret_cast<float *>(ring);
-        float *po = reinterpret_cast<float *>(ring + ml_area);
-        const int per_piece = (C::RING_BYTES - (int)ml_area) / (G * D * 4);
+        const int per_piece = ((C::RING_BYTES - (int)ml_area) / 2) / PART_BYTES;
         if (per_piece < 1) {
             // more parts than the ring can describe (far more CTAs than this part has SMs for):
             // merge straight from global memory
@@ -570,61 +587,79 @@ __global__ void __launch_bounds__(kThreads, Cfg<T, D, G>::CTAS) decode_kernel(co
             }
             continue;
         }
+        float *buf[2] = {reinterpret_cast<float *>(ring + ml_area),
+                         reinterpret_cast<float *>(ring + ml_area + per_piece * PART_BYTES)};
+        const int npieces = (nparts + per_piece - 1) / per_piece;
+        auto issue_piece = [&](int i, uint32_t extra) {  // thread 0 only
+            const int p0 = i * per_piece, np = min(per_piece, nparts - p0);
+            const uint32_t bytes = (uint32_t)np * PART_BYTES;
+            mbar_arrive_expect_tx(&tail->cbar[i & 1], bytes + extra);
+            bulk_load(buf[i & 1], a.part_o + (slot0 + p0) * G * D, bytes, &tail->cbar[i & 1]);
+        };
         if (tid == 0) {
             fence_proxy_async_all();
-            mbar_arrive_expect_tx(&tail->cbar, ml_bytes);
-            bulk_load(ml, a.part_ml + slot0 * GP * 2, ml_bytes, &tail->cbar);
+            issue_piece(0, ml_bytes);
+            bulk_load(ml, a.part_ml + slot0 * GP * 2, ml_bytes, &tail->cbar[0]);
+            if (npieces > 1) issue_piece(1, 0u);
         }
-        mbar_wait(&tail->cbar, cphase, abort, a.status);
-        cphase ^= 1u;
-        named_barrier(1, kConsThreads);  // nobody is still polling this phase when the next copy is armed
+        mbar_wait(&tail->cbar[0], cph[0], abort, a.status);
+        cph[0] ^= 1u;
+        // weights: warp w owns heads w, w + 4; the max slot of every record is overwritten by its weight
+        for (int h = warp; h < G; h += kConsWarps) {
+            float m = -INFINITY;
+            for (int p = lane; p < nparts; p += 32) m = fmaxf(m, ml[(p * GP + h) * 2]);
+#pragma unroll
+            for (int off = 16; off >= 1; off >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, off));
+            float l = 0.f;
+            for (int p = lane; p < nparts; p += 32) {
+                const float w = fast_exp2(ml[(p * GP + h) * 2] - m);
+                ml[(p * GP + h) * 2] = w;
+                l = fmaf(w, ml[(p * GP + h) * 2 + 1], l);
+            }
+#pragma unroll
+            for (int off = 16; off >= 1; off >>= 1) l += __shfl_xor_sync(0xffffffffu, l, off);
+            if (lane == 0) tail->red_sum[0][h] = l;
+        }
+        named_barrier(1, kConsThreads);
         constexpr int NK = (G * D + kConsThreads - 1) / kConsThreads;
-        float M[NK], lsum[NK], acc[NK];
+        float acc[NK];
+        int hk[NK];
 #pragma unroll
         for (int k = 0; k < NK; ++k) {
             const int idx = tid + k * kConsThreads;
-            const int h = idx < G * D ? idx / D : 0;
-            float m = -INFINITY;
-            for (int p = 0; p < nparts; ++p) m = fmaxf(m, ml[(p * GP + h) * 2]);
-            float l = 0.f;
-            for (int p = 0; p < nparts; ++p) l = fmaf(fast_exp2(ml[(p * GP + h) * 2] - m), ml[(p * GP + h) * 2 + 1], l);
-            M[k] = m;
-            lsum[k] = l;
+            hk[k] = idx < G * D ? idx / D : 0;
             acc[k] = 0.f;
         }
-        for (int p0 = 0; p0 < nparts; p0 += per_piece) {
-            const int np = min(per_piece, nparts - p0);
-            if (tid == 0) {
-                const uint32_t bytes = (uint32_t)np * G * D * 4u;
-                mbar_arrive_expect_tx(&tail->cbar, bytes);
-                bulk_load(po, a.part_o + (slot0 + p0) * G * D, bytes, &tail->cbar);
+        for (int i = 0; i < npieces; ++i) {
+            const int p0 = i * per_piece, np = min(per_piece, nparts - p0);
+            if (i > 0) {
+                mbar_wait(&tail->cbar[i & 1], cph[i & 1], abort, a.status);
+                cph[i & 1] ^= 1u;
             }
-            mbar_wait(&tail->cbar, cphase, abort, a.status);
-            cphase ^= 1u;
+            const float *po = buf[i & 1];
+#pragma unroll 2
+            for (int p = 0; p < np; ++p) {
 #pragma unroll
-            for (int k = 0; k < NK; ++k) {
-                const int idx = tid + k * kConsThreads;
-                if (idx < G * D) {
-                    const int h = idx / D;
-                    float x = acc[k];
-                    for (int p = 0; p < np; ++p)
-                        x = fmaf(fast_exp2(ml[((p0 + p) * GP + h) * 2] - M[k]), po[p * G * D + idx], x);
-                    acc[k] = x;
+                for (int k = 0; k < NK; ++k) {
+                    const int idx = tid + k * kConsThreads;
+                    if (idx < G * D) acc[k] = fmaf(ml[((p0 + p) * GP + hk[k]) * 2], po[p * G * D + idx], acc[k]);
                 }
             }
-            named_barrier(1, kConsThreads);  // everyone is done with this piece before the next lands
+            named_barrier(1, kConsThreads);  // everyone is done with this buffer before it is refilled
+            if (tid == 0 && i + 2 < npieces) issue_piece(i + 2, 0u);
         }
 #pragma unroll
         for (int k = 0; k < NK; ++k) {
             const int idx = tid + k * kConsThreads;
-            if (idx < G * D) reinterpret_cast<T *>(a.out)[pend_out[j] + idx] = Elt<T>::from_float(acc[k] / lsum[k]);
+            if (idx < G * D)
+                reinterpret_cast<T *>(a.out)[pend_out[j] + idx] = Elt<T>::from_float(acc[k] / tail->red_sum[0][hk[k]]);
         }
         named_barrier(1, kConsThreads);
     }
 }
 
 template <typename T, int D, int G>
-arb_status launch_one(Ctx *ctx, const DecodeArgs &args, cudaStream_t stream) {
+arb_status launch_one(Ctx *ctx, const DecodeArgs &args, bool overlap, cudaStream_t stream) {
     using C = Cfg<T, D, G>;
     const size_t smem = smem_bytes<T, D, G>(args.batch);
     static bool attr_set[64] = {};
@@ -634,22 +669,32 @@ arb_status launch_one(Ctx *ctx, const DecodeArgs &args, cudaStream_t stream) {
             return ARB_ERR_CUDA;
         attr_set[ctx->device & 63] = true;
     }
-    decode_kernel<T, D, G><<<ctx->num_sms * C::CTAS, kThreads, smem, stream>>>(args);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(ctx->num_sms * C::CTAS);
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = overlap ? 1 : 0;
+    const cudaError_t err = cudaLaunchKernelEx(&cfg, decode_kernel<T, D, G>, args);
     ctx->launches++;
-    return cudaGetLastError() == cudaSuccess ? ARB_OK : ARB_ERR_CUDA;
+    return err == cudaSuccess ? ARB_OK : ARB_ERR_CUDA;
 }
 
 template <typename T, int D>
-arb_status launch_g(Ctx *ctx, int g, const DecodeArgs &args, cudaStream_t stream) {
+arb_status launch_g(Ctx *ctx, int g, const DecodeArgs &args, bool overlap, cudaStream_t stream) {
     switch (g) {
-        case 1: return launch_one<T, D, 1>(ctx, args, stream);
-        case 2: return launch_one<T, D, 2>(ctx, args, stream);
-        case 3: return launch_one<T, D, 3>(ctx, args, stream);
-        case 4: return launch_one<T, D, 4>(ctx, args, stream);
-        case 5: return launch_one<T, D, 5>(ctx, args, stream);
-        case 6: return launch_one<T, D, 6>(ctx, args, stream);
-        case 7: return launch_one<T, D, 7>(ctx, args, stream);
-        case 8: return launch_one<T, D, 8>(ctx, args, stream);
+        case 1: return launch_one<T, D, 1>(ctx, args, overlap, stream);
+        case 2: return launch_one<T, D, 2>(ctx, args, overlap, stream);
+        case 3: return launch_one<T, D, 3>(ctx, args, overlap, stream);
+        case 4: return launch_one<T, D, 4>(ctx, args, overlap, stream);
+        case 5: return launch_one<T, D, 5>(ctx, args, overlap, stream);
+        case 6: return launch_one<T, D, 6>(ctx, args, overlap, stream);
+        case 7: return launch_one<T, D, 7>(ctx, args, overlap, stream);
+        case 8: return launch_one<T, D, 8>(ctx, args, overlap, stream);
         default: return ARB_ERR_UNSUPPORTED;
     }
 }
@@ -690,12 +735,13 @@ arb_status launch_decode(Ctx *ctx, const arb_attn_params &p, const void *q, cons
     a.max_pages = p.max_pages_per_seq;
     const float scale = p.softmax_scale > 0.f ? p.softmax_scale : 1.0f / sqrtf((float)p.head_dim);
     a.scale_log2 = scale * 1.4426950408889634f;
+    const bool overlap = (p.flags & ARB_ATTN_OVERLAP_PREVIOUS) != 0;
     if (p.dtype == ARB_BF16) {
-        if (p.head_dim == 128) return launch_g<__nv_bfloat16, 128>(ctx, g, a, stream);
-        if (p.head_dim == 64) return launch_g<__nv_bfloat16, 64>(ctx, g, a, stream);
+        if (p.head_dim == 128) return launch_g<__nv_bfloat16, 128>(ctx, g, a, overlap, stream);
+        if (p.head_dim == 64) return launch_g<__nv_bfloat16, 64>(ctx, g, a, overlap, stream);
     } else if (p.dtype == ARB_F32) {
-        if (p.head_dim == 128) return launch_g<float, 128>(ctx, g, a, stream);
-        if (p.head_dim == 64) return launch_g<float, 64>(ctx, g, a, stream);
+        if (p.head_dim == 128) return launch_g<float, 128>(ctx, g, a, overlap, stream);
+        if (p.head_dim == 64) return launch_g<float, 64>(ctx, g, a, overlap, stream);
     }
     return ARB_ERR_UNSUPPORTED;
 }

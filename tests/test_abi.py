@@ -35,7 +35,7 @@ def test_params_struct_matches_header_layout():
     from paper_2512_05033_b200 import build
     build.build()
     from paper_2512_05033_b200 import binding
-    assert ctypes.sizeof(binding.AttnParams) == 44
+    assert ctypes.sizeof(binding.AttnParams) == 48
     p = binding.attn_params(binding.ARB_BF16, 8, 12, 2, 128, 100, 10, 8, 1)
     # host-side validation needs no GPU: a bad head_dim is refused before anything is launched
     assert binding.lib.arb_attn_workspace_bytes(ctypes.byref(p)) > 0

@@ -162,3 +162,24 @@ def test_repeated_calls_reuse_the_workspace():
         again, bits = H.gpu_attn(inp)
         assert bits == 0
         np.testing.assert_array_equal(first, again)
+
+
+def test_overlap_flag_gives_identical_results():
+    """Back-to-back calls launched as programmatic dependents (ARB_ATTN_OVERLAP_PREVIOUS): each call
+    streams under the tail of the previous one; outputs must equal the serialised ones exactly."""
+    from paper_2512_05033_b200 import binding
+    c = H.ctx()
+    cases = [wl.small_attn_case(4, 12, 2, 128, BF, [5000 + 100 * i, 700, 3000, 64], [1] * 4, seed=70 + i).to("cuda")
+             for i in range(6)]
+    plain = [c.attn(d.q, d.k_pages, d.v_pages, d.block_table, d.seq_lens, d.q_lens, 1) for d in cases]
+    torch.cuda.synchronize()
+    outs = [torch.full_like(d.q, float("nan")) for d in cases]
+    for rep in range(3):
+        for d, o in zip(cases, outs):
+            p = c.params_for(d.q, d.k_pages, d.block_table, 1, flags=binding.ATTN_OVERLAP_PREVIOUS)
+            c.attn(d.q, d.k_pages, d.v_pages, d.block_table, d.seq_lens, d.q_lens, 1, out=o, params=p)
+    assert c.poll_status() == 0
+    for a, b in zip(plain, outs):
+        assert torch.equal(a, b)
+    ref, _ = H.oracle_attn(cases[0].to("cpu"))
+    H.assert_close(outs[0].double().cpu().numpy(), ref, BF)

@@ -10,11 +10,12 @@
 //
 // Inside a CTA one producer warp walks its pages and issues one bulk (TMA) copy per (page, head)
 // tile of K and of V -- 16 rows x head_dim, contiguous in the head-major page layout -- into a
-// shared-memory ring guarded by full/empty mbarriers; sixteen lanes issue in parallel, one ring
-// stage each.  Four consumer warps take tiles round-robin.  A segment is processed in
-// sub-partitions of up to 512 tokens: q.K for every tile into a score buffer, one block-wide
-// max / exp2 / sum pass, then P.V into per-lane fp32 accumulators that live across sub-partitions
-// (rescaled when the running max moves).
+// shared-memory ring guarded by full/empty mbarriers; up to sixteen lanes issue side by side, one
+// ring stage each.  Pages are taken in groups of kGroup; group j of a segment belongs to consumer
+// warp j mod 4, and its tiles enter the ring as K..K V..V.  Each consumer warp runs its own online
+// softmax: q.K for the group's K tiles into a per-warp score buffer, running max / exp2 / running
+// sum over those scores, then P.V over the group's V tiles into per-lane fp32 accumulators.  The
+// warps never meet until the segment ends, where their (max, sum, accumulator) triples are merged.
 //
 // Arithmetic.  bf16 q.K uses the mixed-precision FMA of sm_100 (bf16 x bf16 + fp32 -> fp32, the
 // product is exact), so neither operand is unpacked; eight lanes share a K row, each owning 16 of
@@ -33,10 +34,10 @@ namespace {
 constexpr int kConsWarps = 4;
 constexpr int kConsThreads = kConsWarps * 32;
 constexpr int kThreads = kConsThreads + 32;  // + producer warp
-constexpr int kSubPages = 32;                // pages per sub-partition
-constexpr int kSubTokens = kSubPages * kPage;
+constexpr int kGroup = 2;                    // pages per consumer work group
+constexpr int kGroupTokens = kGroup * kPage;
 constexpr int kMinChunk = 4;                 // fewest pages worth giving a CTA
-constexpr int kMaxCtasPerSm = 3;
+constexpr int kMaxCtasPerSm = 2;
 
 struct DecodeArgs {
     const char *q;
@@ -74,24 +75,28 @@ struct Cfg {
     static constexpr int NVP = (NV + QLPR - 1) / QLPR * QLPR;
     static constexpr int GP = (G + 3) / 4 * 4;           // heads padded to whole float4s
     static constexpr int TILE_BYTES = kPage * ROW_BYTES;
-    static constexpr int CTAS = (kBf16 && G <= 4) ? 3 : 2;   // resident CTAs per SM aimed at
-    static constexpr int STAGES = (CTAS == 3) ? 12 : (TILE_BYTES > 4096 ? 8 : 16);
-    static constexpr int BATCH = STAGES < 16 ? STAGES : 16;  // producer lanes issuing side by side
+    // Ring stage = tile counter mod STAGES and owner warp = (tile counter / tiles per group) mod 4.
+    // STAGES is a multiple of 4 groups, so a stage is only ever read by one warp: that warp has
+    // consumed fill k-1 before it waits for fill k, which is what a parity wait needs (a waiter two
+    // phases behind would pass at once).
+    static constexpr int STAGES = 16;
+    static constexpr int BATCH = 16;                         // producer lanes issuing side by side
     static constexpr int RING_BYTES = STAGES * TILE_BYTES;
-    static constexpr int LOGIT_BYTES = kSubTokens * GP * 4;
-    static constexpr int OSM_BYTES = kConsWarps * G * D * 4;
-    static constexpr int UNI_BYTES = LOGIT_BYTES > OSM_BYTES ? LOGIT_BYTES : OSM_BYTES;
+    static constexpr int CTAS = RING_BYTES > 65536 ? 1 : 2;  // resident CTAs per SM aimed at
+    static constexpr int SCORE_BYTES = kConsWarps * kGroupTokens * GP * 4;   // per-warp score buffers
+    static constexpr int REC = G * D + 2 * GP;                               // floats of one warp record
+    static constexpr int OSM_BYTES = kConsWarps * REC * 4;
     static_assert(LPR == 8 || LPR == 16 || LPR == 32, "row must be 128, 256 or 512 bytes");
+    static_assert(STAGES % (kConsWarps * 2 * kGroup) == 0, "a ring stage must always belong to the same warp");
 };
 
 constexpr int kMaxStages = 16;
 
-struct SmemTail {  // small fixed part after ring + score buffer
+struct SmemTail {  // small fixed part after ring + buffers
     uint64_t full[kMaxStages];
     uint64_t empty[kMaxStages];
     uint64_t cbar[2];  // split-combine staging, one per buffer
-    float red_max[kConsWarps][kMaxGroup];
-    float red_sum[kConsWarps][kMaxGroup];
+    float lsum[kMaxGroup];
     int abort;
     int is_last;
 };
@@ -99,7 +104,8 @@ struct SmemTail {  // small fixed part after ring + score buffer
 template <typename T, int D, int G>
 size_t smem_bytes(int batch) {
     using C = Cfg<T, D, G>;
-    return 128 + C::RING_BYTES + C::UNI_BYTES + sizeof(SmemTail) + sizeof(int) * (2 * (size_t)batch + 2);
+    return 128 + C::RING_BYTES + C::SCORE_BYTES + C::OSM_BYTES + sizeof(SmemTail) +
+           sizeof(int) * (3 * (size_t)batch + 2);
 }
 
 struct Segment {
@@ -107,9 +113,9 @@ struct Segment {
 };
 
 // Next segment of the flat range [cur, r1); advances cur.  pref[b] = kv heads * pages of all
-// decoding sequences before b.
-__device__ __forceinline__ bool next_segment(int &cur, int r1, const int *pref, int B, int Hkv, int chunk,
-                                             const int32_t *seq_lens, Segment &s) {
+// decoding sequences before b; slen[b] = seq_lens[b].
+__device__ __forceinline__ bool next_segment(int &cur, int r1, const int *pref, const int *slen, int B, int Hkv,
+                                             int chunk, Segment &s) {
     if (cur >= r1) return false;
     int lo = 0, hi = B;  // largest b with pref[b] <= cur
     while (hi - lo > 1) {
@@ -128,7 +134,7 @@ __device__ __forceinline__ bool next_segment(int &cur, int r1, const int *pref, 
     s.kvh = kvh;
     s.pg0 = pg0;
     s.pg1 = pg0 + (end - cur);
-    s.L = seq_lens[b];
+    s.L = slen[b];
     s.bk = b * Hkv + kvh;
     s.c_first = s0 / chunk;
     s.nparts = (s1 - 1) / chunk - s.c_first + 1;
@@ -163,14 +169,17 @@ __global__ void __launch_bounds__(kThreads, Cfg<T, D, G>::CTAS) decode_kernel(co
     constexpr int EPL = C::EPL, LPR = C::LPR, RPP = C::RPP, GP = C::GP;
     constexpr int QLPR = C::QLPR, QRPP = C::QRPP, CPL = C::CPL, STAGES = C::STAGES;
     constexpr int QW = C::kBf16 ? CPL * 4 : EPL;  // 32-bit q registers per head and lane
+    constexpr int REC = C::REC;
 
     extern __shared__ char smem_raw[];
     char *base = reinterpret_cast<char *>((reinterpret_cast<uintptr_t>(smem_raw) + 127) & ~uintptr_t(127));
     char *ring = base;
-    float *uni = reinterpret_cast<float *>(base + C::RING_BYTES);
-    SmemTail *tail = reinterpret_cast<SmemTail *>(base + C::RING_BYTES + C::UNI_BYTES);
+    float *score_all = reinterpret_cast<float *>(base + C::RING_BYTES);
+    float *osm = reinterpret_cast<float *>(base + C::RING_BYTES + C::SCORE_BYTES);
+    SmemTail *tail = reinterpret_cast<SmemTail *>(base + C::RING_BYTES + C::SCORE_BYTES + C::OSM_BYTES);
     int *pref = reinterpret_cast<int *>(tail + 1);  // [B + 1]
     int *row0 = pref + a.batch + 1;                 // [B + 1]
+    int *slen = row0 + a.batch + 1;                 // [B]
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int B = a.batch, Hkv = a.Hkv;
@@ -212,6 +221,7 @@ __global__ void __launch_bounds__(kThreads, Cfg<T, D, G>::CTAS) decode_kernel(co
         }
         pref[b + 1] = pages * Hkv;
         row0[b + 1] = n > 0 ? n : 0;
+        slen[b] = L;
     }
     __syncthreads();
     if (warp == 0) {
@@ -244,14 +254,15 @@ __global__ void __launch_bounds__(kThreads, Cfg<T, D, G>::CTAS) decode_kernel(co
 
     if (warp == kConsWarps) {
         // ================================ producer warp ==========================================
-        // Lanes 0..BATCH-1 each own one ring stage at a time: wait until it is free, then issue the
-        // copy.  A batch never exceeds the ring, so a lane is at most one phase behind its barrier.
+        // Tiles enter the ring group by group: K tiles of a group, then its V tiles.  Lanes
+        // 0..BATCH-1 each own one ring stage at a time: wait until it is free, then issue the copy.
+        // A batch never exceeds the ring, so a lane is at most one phase behind its barrier.
         uint32_t c = 0;
         int cur = r0;
         Segment s;
-        while (next_segment(cur, r1, pref, B, Hkv, chunk, a.seq_lens, s)) {
-            for (int sp0 = s.pg0; sp0 < s.pg1; sp0 += kSubPages) {
-                const int np = min(kSubPages, s.pg1 - sp0);
+        while (next_segment(cur, r1, pref, slen, B, Hkv, chunk, s)) {
+            for (int sp0 = s.pg0; sp0 < s.pg1; sp0 += 32) {
+                const int np = min(32, s.pg1 - sp0);
                 int pid = 0;
                 if (lane < np) {
                     pid = a.block_table[(size_t)s.b * a.max_pages + sp0 + lane];
@@ -260,26 +271,35 @@ __global__ void __launch_bounds__(kThreads, Cfg<T, D, G>::CTAS) decode_kernel(co
                         pid = 0;
                     }
                 }
+                const int full_tiles = (np / kGroup) * 2 * kGroup;  // tiles of the complete groups
+                const int rem = np % kGroup;
+                const int ntiles = 2 * np;
 #pragma unroll 1
-                for (int ph = 0; ph < 2; ++ph) {
-                    const char *pool = ph ? a.v_pages : a.k_pages;
-#pragma unroll 1
-                    for (int i0 = 0; i0 < np; i0 += C::BATCH) {
-                        const int i = i0 + lane;
-                        const int pg = __shfl_sync(0xffffffffu, pid, i & 31);
-                        if (lane < C::BATCH && i < np) {
-                            const uint32_t cc = c + i, st = cc % STAGES, par = (cc / STAGES) & 1u;
-                            if (mbar_wait(&tail->empty[st], par ^ 1u, abort, a.status)) {
-                                mbar_arrive_expect_tx(&tail->full[st], C::TILE_BYTES);
-                                bulk_load(ring + st * C::TILE_BYTES,
-                                          pool + ((size_t)pg * Hkv + s.kvh) * C::TILE_BYTES, C::TILE_BYTES,
-                                          &tail->full[st]);
-                            }
-                        }
-                        __syncwarp();
+                for (int i0 = 0; i0 < ntiles; i0 += C::BATCH) {
+                    const int i = i0 + lane;
+                    int page, is_v;
+                    if (i < full_tiles) {
+                        const int g = i / (2 * kGroup), r = i - g * 2 * kGroup;
+                        is_v = r / kGroup;
+                        page = g * kGroup + (r - is_v * kGroup);
+                    } else {
+                        const int r = i - full_tiles, d = rem > 0 ? rem : 1;
+                        is_v = r / d;
+                        page = (np / kGroup) * kGroup + (r - is_v * d);
                     }
-                    c += np;
+                    const int pg = __shfl_sync(0xffffffffu, pid, page & 31);
+                    if (lane < C::BATCH && i < ntiles) {
+                        const uint32_t cc = c + i, st = cc % STAGES, par = (cc / STAGES) & 1u;
+                        const char *pool = is_v ? a.v_pages : a.k_pages;
+                        if (mbar_wait(&tail->empty[st], par ^ 1u, abort, a.status)) {
+                            mbar_arrive_expect_tx(&tail->full[st], C::TILE_BYTES);
+                            bulk_load(ring + st * C::TILE_BYTES, pool + ((size_t)pg * Hkv + s.kvh) * C::TILE_BYTES,
+                                      C::TILE_BYTES, &tail->full[st]);
+                        }
+                    }
+                    __syncwarp();
                 }
+                c += ntiles;
             }
         }
         // After a timeout the consumers may have left copies unconsumed: wait (bounded) for the
@@ -300,7 +320,8 @@ __global__ void __launch_bounds__(kThreads, Cfg<T, D, G>::CTAS) decode_kernel(co
     // ==================================== consumer warps ==========================================
     const int lg = lane % LPR, rg = lane / LPR;      // P.V: vector column within a row, row of a pass
     const int qlg = lane % QLPR, qrg = lane / QLPR;  // q.K: the same for its own row sharing
-    uint32_t c_base = 0;
+    float *sc = score_all + warp * kGroupTokens * GP;  // this warp's scores / probabilities
+    uint32_t seg_base = 0;                             // ring counter of the segment's first tile
     int cur = r0;
     Segment s;
     // split-combine jobs this CTA has to finish (only the first and last segment of a range can be
@@ -309,7 +330,7 @@ __global__ void __launch_bounds__(kThreads, Cfg<T, D, G>::CTAS) decode_kernel(co
     int pend_slot0[2], pend_parts[2];
     size_t pend_out[2];
 
-    while (next_segment(cur, r1, pref, B, Hkv, chunk, a.seq_lens, s)) {
+    while (next_segment(cur, r1, pref, slen, B, Hkv, chunk, s)) {
         const int qrow = row0[s.b];
         // q of this kv head's group: packed bf16 pairs, or fp32 pre-multiplied by the scale
         uint32_t qp[G][QW];
@@ -331,7 +352,8 @@ __global__ void __launch_bounds__(kThreads, Cfg<T, D, G>::CTAS) decode_kernel(co
                 qp[h][3] = __float_as_uint(__uint_as_float(v.w) * a.scale_log2);
             }
         }
-        const float sc = C::kBf16 ? a.scale_log2 : 1.0f;
+        const float scl = C::kBf16 ? a.scale_log2 : 1.0f;
+        // m_run is the same in every lane of the warp; l_run is this lane's share of the sum
         float m_run[G], l_run[G], o[G][EPL];
 #pragma unroll
         for (int h = 0; h < G; ++h) {
@@ -341,13 +363,17 @@ __global__ void __launch_bounds__(kThreads, Cfg<T, D, G>::CTAS) decode_kernel(co
             for (int e = 0; e < EPL; ++e) o[h][e] = 0.f;
         }
 
-        for (int sp0 = s.pg0; sp0 < s.pg1; sp0 += kSubPages) {
-            const int np = min(kSubPages, s.pg1 - sp0);
-            const int ntok = min(s.L - sp0 * kPage, np * kPage);
+        const int seg_pages = s.pg1 - s.pg0;
+        const int ngroups = (seg_pages + kGroup - 1) / kGroup;
+        for (int gi = warp; gi < ngroups; gi += kConsWarps) {
+            const int p0 = s.pg0 + gi * kGroup;               // first page of the group
+            const int npg = min(kGroup, s.pg1 - p0);
+            const int ntok = min(s.L - p0 * kPage, npg * kPage);  // valid tokens of the group
+            const uint32_t gbase = seg_base + (uint32_t)gi * 2 * kGroup;
 
-            // ---- phase A: scores of this warp's K tiles -------------------------------------------
-            for (int t = warp; t < np; t += kConsWarps) {
-                const uint32_t cc = c_base + t, st = cc % STAGES, par = (cc / STAGES) & 1u;
+            // ---- q.K: scores of the group's K tiles ----------------------------------------------
+            for (int t = 0; t < npg; ++t) {
+                const uint32_t cc = gbase + t, st = cc % STAGES, par = (cc / STAGES) & 1u;
                 mbar_wait(&tail->full[st], par, abort, a.status);
                 const char *tile = ring + st * C::TILE_BYTES;
 #pragma unroll
@@ -391,92 +417,63 @@ __global__ void __launch_bounds__(kThreads, Cfg<T, D, G>::CTAS) decode_kernel(co
                         if (idx < C::NV) {
                             const int ps = idx / G, h = idx - ps * G;
                             const int token = t * kPage + (nb * C::PB + ps) * QRPP + qrg;
-                            uni[token * GP + h] = acc[j] * sc;
+                            sc[token * GP + h] = acc[j] * scl;
                         }
                     }
                 }
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&tail->empty[st]);
             }
-            named_barrier(1, kConsThreads);
 
-            // ---- phase B: running max, exp2, running sum ------------------------------------------
-            float mloc[G];
+            // ---- online softmax over the group's scores: one token per lane ---------------------
+            static_assert(kGroupTokens == 32, "one token per lane");
+            float sv[GP];
+            const bool tok_ok = lane < ntok;
 #pragma unroll
-            for (int h = 0; h < G; ++h) mloc[h] = -INFINITY;
-            for (int t = tid; t < ntok; t += kConsThreads) {
-#pragma unroll
-                for (int h4 = 0; h4 < GP; h4 += 4) {
-                    const float4 sv = *reinterpret_cast<const float4 *>(uni + t * GP + h4);
-                    if (h4 + 0 < G) mloc[h4 + 0] = fmaxf(mloc[h4 + 0], sv.x);
-                    if (h4 + 1 < G) mloc[h4 + 1] = fmaxf(mloc[h4 + 1], sv.y);
-                    if (h4 + 2 < G) mloc[h4 + 2] = fmaxf(mloc[h4 + 2], sv.z);
-                    if (h4 + 3 < G) mloc[h4 + 3] = fmaxf(mloc[h4 + 3], sv.w);
-                }
+            for (int h4 = 0; h4 < GP; h4 += 4) {
+                const float4 x = *reinterpret_cast<const float4 *>(sc + lane * GP + h4);
+                sv[h4] = x.x; sv[h4 + 1] = x.y; sv[h4 + 2] = x.z; sv[h4 + 3] = x.w;
             }
+            float mx[G];
+#pragma unroll
+            for (int h = 0; h < G; ++h) mx[h] = tok_ok ? sv[h] : -INFINITY;
+#pragma unroll
+            for (int off = 16; off >= 1; off >>= 1)
+#pragma unroll
+                for (int h = 0; h < G; ++h) mx[h] = fmaxf(mx[h], __shfl_xor_sync(0xffffffffu, mx[h], off));
 #pragma unroll
             for (int h = 0; h < G; ++h) {
-#pragma unroll
-                for (int off = 16; off >= 1; off >>= 1)
-                    mloc[h] = fmaxf(mloc[h], __shfl_xor_sync(0xffffffffu, mloc[h], off));
-                if (lane == 0) tail->red_max[warp][h] = mloc[h];
-            }
-            named_barrier(1, kConsThreads);
-            float factor[G], lloc[G];
-#pragma unroll
-            for (int h = 0; h < G; ++h) {
-                float m = m_run[h];
-#pragma unroll
-                for (int w = 0; w < kConsWarps; ++w) m = fmaxf(m, tail->red_max[w][h]);
-                factor[h] = fast_exp2(m_run[h] - m);  // 0 on the first sub-partition
+                const float m = fmaxf(m_run[h], mx[h]);      // finite: the group has a valid token
+                const float f = fast_exp2(m_run[h] - m);     // 0 for the first group
                 m_run[h] = m;
-                lloc[h] = 0.f;
-            }
-            for (int t = tid; t < ntok; t += kConsThreads) {
+                const float p = tok_ok ? fast_exp2(sv[h] - m) : 0.f;
+                sv[h] = p;
+                l_run[h] = fmaf(l_run[h], f, p);
 #pragma unroll
-                for (int h4 = 0; h4 < GP; h4 += 4) {
-                    float4 sv = *reinterpret_cast<const float4 *>(uni + t * GP + h4);
-                    if (h4 + 0 < G) { sv.x = fast_exp2(sv.x - m_run[h4 + 0]); lloc[h4 + 0] += sv.x; }
-                    if (h4 + 1 < G) { sv.y = fast_exp2(sv.y - m_run[h4 + 1]); lloc[h4 + 1] += sv.y; }
-                    if (h4 + 2 < G) { sv.z = fast_exp2(sv.z - m_run[h4 + 2]); lloc[h4 + 2] += sv.z; }
-                    if (h4 + 3 < G) { sv.w = fast_exp2(sv.w - m_run[h4 + 3]); lloc[h4 + 3] += sv.w; }
-                    *reinterpret_cast<float4 *>(uni + t * GP + h4) = sv;
-                }
+                for (int e = 0; e < EPL; ++e) o[h][e] *= f;
             }
 #pragma unroll
-            for (int h = 0; h < G; ++h) {
-#pragma unroll
-                for (int off = 16; off >= 1; off >>= 1) lloc[h] += __shfl_xor_sync(0xffffffffu, lloc[h], off);
-                if (lane == 0) tail->red_sum[warp][h] = lloc[h];
-            }
-            named_barrier(1, kConsThreads);
-#pragma unroll
-            for (int h = 0; h < G; ++h) {
-                float l = 0.f;
-#pragma unroll
-                for (int w = 0; w < kConsWarps; ++w) l += tail->red_sum[w][h];
-                l_run[h] = l_run[h] * factor[h] + l;
-#pragma unroll
-                for (int e = 0; e < EPL; ++e) o[h][e] *= factor[h];
-            }
+            for (int h4 = 0; h4 < GP; h4 += 4)
+                *reinterpret_cast<float4 *>(sc + lane * GP + h4) = make_float4(sv[h4], sv[h4 + 1], sv[h4 + 2], sv[h4 + 3]);
+            __syncwarp();
 
-            // ---- phase C: P.V over this warp's V tiles --------------------------------------------
-            for (int t = warp; t < np; t += kConsWarps) {
-                const uint32_t cc = c_base + np + t, st = cc % STAGES, par = (cc / STAGES) & 1u;
+            // ---- P.V over the group's V tiles -----------------------------------------------------
+            for (int t = 0; t < npg; ++t) {
+                const uint32_t cc = gbase + npg + t, st = cc % STAGES, par = (cc / STAGES) & 1u;
                 mbar_wait(&tail->full[st], par, abort, a.status);
                 const char *tile = ring + st * C::TILE_BYTES;
+                const float *pt = sc + t * kPage * GP;
+                if ((t + 1) * kPage <= ntok) {  // every slot of the tile is a real token
 #pragma unroll
-                for (int ps = 0; ps < C::NPASS; ++ps) {
-                    const int r = ps * RPP + rg;
-                    const int token = t * kPage + r;
-                    if (token < ntok) {  // slots past the sequence end are never touched
+                    for (int ps = 0; ps < C::NPASS; ++ps) {
+                        const int r = ps * RPP + rg;
                         const uint4 vv = *reinterpret_cast<const uint4 *>(tile + r * C::ROW_BYTES + lg * 16);
                         float vf[EPL];
                         Elt<T>::unpack(vv, vf);
                         float pf[GP];
 #pragma unroll
                         for (int h4 = 0; h4 < GP; h4 += 4) {
-                            const float4 pv = *reinterpret_cast<const float4 *>(uni + token * GP + h4);
+                            const float4 pv = *reinterpret_cast<const float4 *>(pt + r * GP + h4);
                             pf[h4] = pv.x; pf[h4 + 1] = pv.y; pf[h4 + 2] = pv.z; pf[h4 + 3] = pv.w;
                         }
 #pragma unroll
@@ -484,15 +481,30 @@ __global__ void __launch_bounds__(kThreads, Cfg<T, D, G>::CTAS) decode_kernel(co
 #pragma unroll
                             for (int e = 0; e < EPL; ++e) o[h][e] = fmaf(pf[h], vf[e], o[h][e]);
                     }
+                } else {  // ragged last page: slots past the sequence end are never touched
+#pragma unroll 1
+                    for (int ps = 0; ps < C::NPASS; ++ps) {
+                        const int r = ps * RPP + rg;
+                        if (t * kPage + r < ntok) {
+                            const uint4 vv = *reinterpret_cast<const uint4 *>(tile + r * C::ROW_BYTES + lg * 16);
+                            float vf[EPL];
+                            Elt<T>::unpack(vv, vf);
+#pragma unroll
+                            for (int h = 0; h < G; ++h) {
+                                const float p = pt[r * GP + h];
+#pragma unroll
+                                for (int e = 0; e < EPL; ++e) o[h][e] = fmaf(p, vf[e], o[h][e]);
+                            }
+                        }
+                    }
                 }
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&tail->empty[st]);
             }
-            named_barrier(1, kConsThreads);
-            c_base += 2u * np;
         }
+        seg_base += 2u * (uint32_t)seg_pages;
 
-        // ---- segment end: add up the warps' accumulators ---------------------------------------------
+        // ---- segment end: every warp leaves (max, sum, accumulator); all threads merge them ----------
         wait_for_predecessor();  // first write of this CTA comes below; later calls return at once
 #pragma unroll
         for (int off = LPR; off < 32; off <<= 1)
@@ -500,42 +512,48 @@ __global__ void __launch_bounds__(kThreads, Cfg<T, D, G>::CTAS) decode_kernel(co
             for (int h = 0; h < G; ++h)
 #pragma unroll
                 for (int e = 0; e < EPL; ++e) o[h][e] += __shfl_xor_sync(0xffffffffu, o[h][e], off);
+#pragma unroll
+        for (int off = 16; off >= 1; off >>= 1)
+#pragma unroll
+            for (int h = 0; h < G; ++h) l_run[h] += __shfl_xor_sync(0xffffffffu, l_run[h], off);
+        float *rec = osm + warp * REC;  // [m[GP] | l[GP] | o[G][D]]
         if (rg == 0) {
 #pragma unroll
             for (int h = 0; h < G; ++h)
 #pragma unroll
-                for (int e = 0; e < EPL; ++e) uni[(warp * G + h) * D + lg * EPL + e] = o[h][e];
+                for (int e = 0; e < EPL; ++e) rec[2 * GP + h * D + lg * EPL + e] = o[h][e];
+        }
+        if (lane == 0) {
+#pragma unroll
+            for (int h = 0; h < G; ++h) { rec[h] = m_run[h]; rec[GP + h] = l_run[h]; }
         }
         named_barrier(1, kConsThreads);
 
         const size_t out_base = ((size_t)qrow * a.Hq + s.kvh * G) * D;
-        if (s.nparts == 1) {
-            for (int idx = tid; idx < G * D; idx += kConsThreads) {
-                float acc = 0.f;
+        const size_t slot = (size_t)s.bk + blockIdx.x;
+        for (int idx = tid; idx < G * D; idx += kConsThreads) {
+            const int h = idx / D;
+            float M = -INFINITY;
 #pragma unroll
-                for (int w = 0; w < kConsWarps; ++w) acc += uni[w * G * D + idx];
-                const int h = idx / D;
-                float l = l_run[0];
+            for (int w = 0; w < kConsWarps; ++w) M = fmaxf(M, osm[w * REC + h]);
+            float l = 0.f, acc = 0.f;
 #pragma unroll
-                for (int hh = 1; hh < G; ++hh) l = (h == hh) ? l_run[hh] : l;
+            for (int w = 0; w < kConsWarps; ++w) {
+                const float f = fast_exp2(osm[w * REC + h] - M);  // 0 for a warp that had no group
+                l = fmaf(f, osm[w * REC + GP + h], l);
+                acc = fmaf(f, osm[w * REC + 2 * GP + idx], acc);
+            }
+            if (s.nparts == 1) {
                 reinterpret_cast<T *>(a.out)[out_base + idx] = Elt<T>::from_float(acc / l);
-            }
-            named_barrier(1, kConsThreads);
-        } else {
-            const size_t slot = (size_t)s.bk + blockIdx.x;
-            for (int idx = tid; idx < G * D; idx += kConsThreads) {
-                float acc = 0.f;
-#pragma unroll
-                for (int w = 0; w < kConsWarps; ++w) acc += uni[w * G * D + idx];
+            } else {
                 a.part_o[slot * G * D + idx] = acc;
-            }
-            if (tid == 0) {
-#pragma unroll
-                for (int h = 0; h < G; ++h) {
-                    a.part_ml[(slot * GP + h) * 2 + 0] = m_run[h];
-                    a.part_ml[(slot * GP + h) * 2 + 1] = l_run[h];
+                if (idx - h * D == 0) {
+                    a.part_ml[(slot * GP + h) * 2 + 0] = M;
+                    a.part_ml[(slot * GP + h) * 2 + 1] = l;
                 }
             }
+        }
+        if (s.nparts > 1) {
             __threadfence();
             fence_proxy_async_all();  // the partials are read back through bulk copies
             named_barrier(1, kConsThreads);
@@ -552,8 +570,8 @@ __global__ void __launch_bounds__(kThreads, Cfg<T, D, G>::CTAS) decode_kernel(co
                 pend_out[pend_n] = out_base;
                 ++pend_n;
             }
-            named_barrier(1, kConsThreads);
         }
+        named_barrier(1, kConsThreads);  // records and is_last are free for the next segment
     }
 
     // ---- split combine of the (sequence, kv head)s this CTA was the last to reach -----------------
@@ -618,7 +636,7 @@ __global__ void __launch_bounds__(kThreads, Cfg<T, D, G>::CTAS) decode_kernel(co
             }
 #pragma unroll
             for (int off = 16; off >= 1; off >>= 1) l += __shfl_xor_sync(0xffffffffu, l, off);
-            if (lane == 0) tail->red_sum[0][h] = l;
+            if (lane == 0) tail->lsum[h] = l;
         }
         named_barrier(1, kConsThreads);
         constexpr int NK = (G * D + kConsThreads - 1) / kConsThreads;
@@ -652,7 +670,7 @@ __global__ void __launch_bounds__(kThreads, Cfg<T, D, G>::CTAS) decode_kernel(co
         for (int k = 0; k < NK; ++k) {
             const int idx = tid + k * kConsThreads;
             if (idx < G * D)
-                reinterpret_cast<T *>(a.out)[pend_out[j] + idx] = Elt<T>::from_float(acc[k] / tail->red_sum[0][hk[k]]);
+                reinterpret_cast<T *>(a.out)[pend_out[j] + idx] = Elt<T>::from_float(acc[k] / tail->lsum[hk[k]]);
         }
         named_barrier(1, kConsThreads);
     }

@@ -119,8 +119,17 @@ arb_status arb_attn(arb_ctx *ctx, const arb_attn_params *params, const void *q, 
         if (st != ARB_OK) return st;
     }
     if (params->max_q_len >= 2) {
+        // Step chunks: a chunk with q_len * group >= 64 rows (bf16, head_dim 128) is a dense
+        // contraction and goes to the tcgen05 kernel; the rest, and every fp32 chunk, to the
+        // CUDA-core kernel.  Both kernels decide per sequence on the device.
+        int skip_rows = 0;
+        if (chunk_mma_supported(*params)) {
+            st = launch_chunk_mma(c, *params, q, k_pages, v_pages, block_table, seq_lens, q_lens, out, s);
+            if (st != ARB_OK) return st;
+            skip_rows = kChunkMmaMinRows;
+        }
         st = launch_chunk_fma(c, *params, q, k_pages, v_pages, block_table, seq_lens, q_lens, out, 2,
-                              params->max_q_len, s);
+                              params->max_q_len, skip_rows, s);
         if (st != ARB_OK) return st;
     }
     return ARB_OK;

@@ -1,7 +1,8 @@
 // Step-chunk attention, CUDA-core path: one CTA per (query row, kv head).
 //
 // This is the path for chunks that are not a dense contraction worth the tensor cores: fp32 inputs
-// (whose 1e-5 tolerance rules out tf32) and chunks with q_len * group < 64 rows.  Query token i of
+// (whose 1e-5 tolerance rules out tf32), head_dim 64, and chunks with q_len * group < 64 rows.  It
+// also zero-fills the rows of chunk sequences whose lengths are invalid, whatever their size.  Query token i of
 // a chunk of n tokens sits at position pos = L - n + i and attends keys 0..pos; the causal mask is
 // just each row's own key count.  K and V rows are read straight from global memory with 16-byte
 // loads (the rows of one chunk are re-read by neighbouring CTAs out of L2); each group of lanes that
@@ -26,7 +27,8 @@ struct ChunkArgs {
     char *out;
     uint32_t *status;
     int batch, Hq, Hkv, num_pages, max_pages;
-    int n_lo, n_hi;  // this kernel owns the sequences with n_lo <= q_len <= n_hi
+    int n_lo, n_hi;  // this kernel owns the sequences with n_lo <= q_len <= n_hi ...
+    int skip_rows;   // ... except valid ones with q_len * group >= skip_rows (> 0): the tensor-core kernel has them
     float scale_log2;
 };
 
@@ -80,6 +82,7 @@ __global__ void __launch_bounds__(kThreads) chunk_fma_kernel(const ChunkArgs a) 
         for (int idx = tid; idx < G * D; idx += kThreads) orow[idx] = Elt<T>::from_float(0.f);
         return;
     }
+    if (a.skip_rows > 0 && n * G >= a.skip_rows) return;
     const int i = row - row0[b];
     const int nkeys = L - n + i + 1;
     const int npages = (nkeys + kPage - 1) / kPage;
@@ -212,7 +215,8 @@ arb_status launch_g(Ctx *ctx, int g, const ChunkArgs &a, int total_q, cudaStream
 
 arb_status launch_chunk_fma(Ctx *ctx, const arb_attn_params &p, const void *q, const void *k_pages,
                             const void *v_pages, const int32_t *block_table, const int32_t *seq_lens,
-                            const int32_t *q_lens, void *out, int n_lo, int n_hi, cudaStream_t stream) {
+                            const int32_t *q_lens, void *out, int n_lo, int n_hi, int skip_rows,
+                            cudaStream_t stream) {
     ChunkArgs a;
     a.q = static_cast<const char *>(q);
     a.k_pages = static_cast<const char *>(k_pages);
@@ -229,6 +233,7 @@ arb_status launch_chunk_fma(Ctx *ctx, const arb_attn_params &p, const void *q, c
     a.max_pages = p.max_pages_per_seq;
     a.n_lo = n_lo;
     a.n_hi = n_hi;
+    a.skip_rows = skip_rows;
     const float scale = p.softmax_scale > 0.f ? p.softmax_scale : 1.0f / sqrtf((float)p.head_dim);
     a.scale_log2 = scale * 1.4426950408889634f;
     const int g = p.num_q_heads / p.num_kv_heads;

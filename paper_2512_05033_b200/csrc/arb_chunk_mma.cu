@@ -1,0 +1,584 @@
+// Step-chunk attention on the 5th-generation tensor cores (tcgen05 + TMEM), bf16, head_dim 128.
+//
+// A chunk of n query tokens against one KV head is a dense contraction once n * group >= 64:
+// the M = n * group query rows (token-major, the group's heads of one token are consecutive rows)
+// all read the same keys.  One work item is a tile of 128 query rows of one (sequence, kv head);
+// it walks the visible keys in tiles of 128 (eight pages):
+//
+//     S = Q K^T      tcgen05.mma, A = Q tile, B = K tile, both K-major in shared memory (128-byte
+//                    swizzle), fp32 accumulator in TMEM columns [0, 128)
+//     P = exp2(scale * S - m)   by the 128 softmax threads, one TMEM lane (= query row) each:
+//                    tcgen05.ld, causal / length mask, row max, exponentials, bf16 P written back to
+//                    shared memory in the K-major swizzled layout
+//     O += P V       tcgen05.mma, A = P, B = V tile read MN-major straight from its page layout,
+//                    fp32 accumulator in TMEM columns [128, 256)
+//
+// The running max is lazy: O is rescaled (tcgen05.ld / st) only when a row's max grows by more than
+// 2^8, otherwise the stale max keeps the exponentials bounded by 2^8 and nothing is touched.
+// K and V tiles are fetched page by page with tiled TMA copies (one 16 x 64 box per page and half
+// of head_dim, landing in the canonical swizzled layout) into a two-stage ring.  Roles: warps 0-3
+// softmax and epilogue, warp 4 TMA producer, warp 5 MMA issue and TMEM allocation.  Every mbarrier
+// wait is bounded; TMEM is released on every path.
+#include <cuda.h>  // CUtensorMap and its enums only; the encoder is looked up at run time
+
+#include "arb_common.cuh"
+
+namespace arb {
+
+namespace {
+
+constexpr int kD = 128;           // head_dim
+constexpr int kBM = 128;          // query rows per work item
+constexpr int kBN = 128;          // keys per KV tile
+constexpr int kTilePages = kBN / kPage;
+constexpr int kStages = 2;
+constexpr int kSoftmaxThreads = 128;
+constexpr int kThreads = 192;
+constexpr int kHalfBytes = 128 * 128;      // [128 rows x 64 bf16]: one 128-byte-swizzled half tile
+constexpr int kTileBytes = 2 * kHalfBytes;  // [128 x 128] bf16
+constexpr int kBoxBytes = kPage * 128;      // one TMA box: 16 rows x 64 bf16
+constexpr uint32_t kTmemCols = 256;         // S: columns 0..127, O: columns 128..255
+constexpr float kRescaleThreshold = 8.0f;   // log2 units
+
+struct MmaArgs {
+    const char *q;
+    const int32_t *block_table;
+    const int32_t *seq_lens;
+    const int32_t *q_lens;
+    char *out;
+    uint32_t *status;
+    int batch, Hq, Hkv, num_pages, max_pages;
+    int min_rows;  // sequences with q_len * group >= min_rows are handled here
+    float scale_log2;
+};
+
+struct Bars {
+    uint64_t q_full;             // 128 softmax threads wrote the Q tile
+    uint64_t k_full[kStages];    // TMA bytes of a K tile landed
+    uint64_t v_full[kStages];
+    uint64_t kv_empty[kStages];  // the MMAs that read the stage have completed
+    uint64_t s_full;             // S = Q K^T is in TMEM
+    uint64_t p_full;             // P is in shared memory, S may be overwritten
+    uint64_t o_full;             // O += P V has completed
+    uint32_t tmem_base;
+    int abort;
+};
+
+constexpr size_t kSmemFixed = 1024 /*alignment*/ + 2 * kTileBytes /*Q, P*/ + 2 * kStages * kTileBytes /*K, V*/ +
+                              sizeof(Bars);
+
+inline size_t mma_smem_bytes(int batch) { return kSmemFixed + sizeof(int) * (2 * (size_t)batch + 2); }
+
+// ---- tcgen05 / TMA wrappers -------------------------------------------------------------------
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+
+__device__ __forceinline__ void tmem_alloc(uint32_t *dst_smem, uint32_t cols) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(dst_smem)), "r"(cols)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t base, uint32_t cols) {
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(base), "r"(cols) : "memory");
+}
+
+// arrives on `bar` once every tcgen05 operation issued so far by this thread has completed
+__device__ __forceinline__ void mma_commit(uint64_t *bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar))
+                 : "memory");
+}
+
+// D[tmem] (+)= A[smem] * B[smem]; M = 128, K = 16 per instruction
+__device__ __forceinline__ void mma_f16_ss(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                           uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+
+// Shared-memory matrix descriptor, 128-byte swizzle: start address, leading / stride byte offsets
+// (all in 16-byte units), descriptor version 1 (sm_100), layout type 2 (SWIZZLE_128B).
+__device__ __forceinline__ uint64_t smem_desc(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
+    uint64_t d = 0;
+    d |= (uint64_t)((saddr >> 4) & 0x3FFFu);
+    d |= (uint64_t)((lbo_bytes >> 4) & 0x3FFFu) << 16;
+    d |= (uint64_t)((sbo_bytes >> 4) & 0x3FFFu) << 32;
+    d |= (uint64_t)1 << 46;
+    d |= (uint64_t)2 << 61;
+    return d;
+}
+
+// Instruction descriptor of kind::f16: fp32 accumulator, bf16 A and B, M = 128, N = 128.
+__host__ __device__ constexpr uint32_t instr_desc(bool b_mn_major) {
+    return (1u << 4)                       // accumulator format: f32
+           | (1u << 7) | (1u << 10)        // A, B format: bf16
+           | (0u << 15)                    // A is K-major
+           | ((b_mn_major ? 1u : 0u) << 16)
+           | ((uint32_t)(kBN >> 3) << 17)  // N
+           | ((uint32_t)(kBM >> 4) << 24); // M
+}
+
+__device__ __forceinline__ void tma_box_load(void *dst_smem, const CUtensorMap *map, int x, int y, uint64_t *bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+        ::"r"(smem_u32(dst_smem)), "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(smem_u32(bar))
+        : "memory");
+}
+
+#define ARB_R32(v, o)                                                                                       \
+    "=r"(v[o + 0]), "=r"(v[o + 1]), "=r"(v[o + 2]), "=r"(v[o + 3]), "=r"(v[o + 4]), "=r"(v[o + 5]), "=r"(v[o + 6]), \
+        "=r"(v[o + 7])
+// 32 consecutive fp32 columns of this thread's TMEM lane
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&v)[32]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : ARB_R32(v, 0), ARB_R32(v, 8), ARB_R32(v, 16), ARB_R32(v, 24)
+        : "r"(taddr)
+        : "memory");
+}
+#undef ARB_R32
+#define ARB_W8(v, o) "r"(v[o + 0]), "r"(v[o + 1]), "r"(v[o + 2]), "r"(v[o + 3]), "r"(v[o + 4]), "r"(v[o + 5]), "r"(v[o + 6]), "r"(v[o + 7])
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&v)[32]) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+        "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "
+        "%17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};"
+        ::"r"(taddr), ARB_W8(v, 0), ARB_W8(v, 8), ARB_W8(v, 16), ARB_W8(v, 24)
+        : "memory");
+}
+#undef ARB_W8
+__device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+    uint32_t r;
+    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+    return r;
+}
+
+struct Item {
+    int b, kvh, mt, n, L, rows_total, r_begin, rows_here, kv_len, ntiles, qrow0;
+};
+
+template <int G>
+__device__ __forceinline__ bool get_item(int item, int total, const int *pref, const int *row0, int B, int Hkv,
+                                         const MmaArgs &a, Item &it) {
+    if (item >= total) return false;
+    int lo = 0, hi = B;
+    while (hi - lo > 1) {
+        const int mid = (lo + hi) >> 1;
+        if (pref[mid] <= item) lo = mid; else hi = mid;
+    }
+    it.b = lo;
+    it.n = a.q_lens[lo];
+    it.L = a.seq_lens[lo];
+    it.rows_total = it.n * G;
+    const int mtiles = (it.rows_total + kBM - 1) / kBM;
+    const int r = item - pref[lo];
+    it.kvh = r / mtiles;
+    it.mt = r - it.kvh * mtiles;
+    it.r_begin = it.mt * kBM;
+    it.rows_here = min(kBM, it.rows_total - it.r_begin);
+    const int i_last = (it.r_begin + it.rows_here - 1) / G;
+    it.kv_len = it.L - it.n + i_last + 1;
+    it.ntiles = (it.kv_len + kBN - 1) / kBN;
+    it.qrow0 = row0[lo];
+    return true;
+}
+
+template <int G>
+__global__ void __launch_bounds__(kThreads, 1)
+chunk_mma_kernel(const MmaArgs a, const __grid_constant__ CUtensorMap k_map, const __grid_constant__ CUtensorMap v_map) {
+    extern __shared__ char smem_raw[];
+    char *base = reinterpret_cast<char *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    char *q_s = base;                                  // [2 halves][128 rows][128 B]
+    char *p_s = base + kTileBytes;
+    char *k_s = base + 2 * kTileBytes;                 // [stage][2 halves][128 keys][128 B]
+    char *v_s = k_s + kStages * kTileBytes;
+    Bars *bars = reinterpret_cast<Bars *>(v_s + kStages * kTileBytes);
+    int *pref = reinterpret_cast<int *>(bars + 1);     // [B + 1] work items before sequence b
+    int *row0 = pref + a.batch + 1;                    // [B + 1] q rows before sequence b
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int B = a.batch, Hkv = a.Hkv;
+
+    if (tid == 0) {
+        mbar_init(&bars->q_full, kSoftmaxThreads);
+        for (int s = 0; s < kStages; ++s) {
+            mbar_init(&bars->k_full[s], 1);
+            mbar_init(&bars->v_full[s], 1);
+            mbar_init(&bars->kv_empty[s], 1);
+        }
+        mbar_init(&bars->s_full, 1);
+        mbar_init(&bars->p_full, kSoftmaxThreads);
+        mbar_init(&bars->o_full, 1);
+        bars->abort = 0;
+        mbar_fence_init();
+        pref[0] = 0;
+        row0[0] = 0;
+    }
+    for (int b = tid; b < B; b += kThreads) {
+        const int n = a.q_lens[b], L = a.seq_lens[b];
+        int items = 0;
+        if (n >= 2 && n * G >= a.min_rows && L >= n && L <= a.max_pages * kPage) items = Hkv * ((n * G + kBM - 1) / kBM);
+        pref[b + 1] = items;
+        row0[b + 1] = n > 0 ? n : 0;
+    }
+    __syncthreads();
+    if (warp == 0) {
+        int carry_p = 0, carry_r = 0;
+        for (int b0 = 0; b0 < B; b0 += 32) {
+            const int b = b0 + lane;
+            int vp = b < B ? pref[b + 1] : 0;
+            int vr = b < B ? row0[b + 1] : 0;
+#pragma unroll
+            for (int off = 1; off < 32; off <<= 1) {
+                const int tp = __shfl_up_sync(0xffffffffu, vp, off);
+                const int tr = __shfl_up_sync(0xffffffffu, vr, off);
+                if (lane >= off) { vp += tp; vr += tr; }
+            }
+            if (b < B) { pref[b + 1] = vp + carry_p; row0[b + 1] = vr + carry_r; }
+            carry_p += __shfl_sync(0xffffffffu, vp, 31);
+            carry_r += __shfl_sync(0xffffffffu, vr, 31);
+        }
+    }
+    __syncthreads();
+    const int total = pref[B];
+    if ((int)blockIdx.x >= total) return;  // nothing for this CTA; no TMEM taken, no barrier pending
+
+    if (warp == 5) tmem_alloc(&bars->tmem_base, kTmemCols);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = bars->tmem_base;
+    volatile int *abort = &bars->abort;
+
+    if (warp == 4) {
+        // ===================================== TMA producer =========================================
+        uint32_t it = 0;  // KV tiles issued so far
+        Item w;
+        for (int item = blockIdx.x; get_item<G>(item, total, pref, row0, B, Hkv, a, w); item += gridDim.x) {
+            for (int j = 0; j < w.ntiles; ++j, ++it) {
+                const uint32_t s = it % kStages, par = (it / kStages) & 1u;
+                const int npages = min(kTilePages, (w.kv_len - j * kBN + kPage - 1) / kPage);
+                int pid = 0;
+                if (lane < npages) {
+                    pid = a.block_table[(size_t)w.b * a.max_pages + j * kTilePages + lane];
+                    if ((unsigned)pid >= (unsigned)a.num_pages) {
+                        atomicOr(a.status, (uint32_t)ARB_DEV_BAD_PAGE);
+                        pid = 0;
+                    }
+                }
+                bool ok = true;
+                if (lane == 0) ok = mbar_wait(&bars->kv_empty[s], par ^ 1u, abort, a.status);
+                ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+                if (ok) {
+                    if (lane == 0) {
+                        mbar_arrive_expect_tx(&bars->k_full[s], (uint32_t)npages * 2u * kBoxBytes);
+                        mbar_arrive_expect_tx(&bars->v_full[s], (uint32_t)npages * 2u * kBoxBytes);
+                    }
+                    __syncwarp();
+                    // lanes 0..15: (half, page) of K; the same lanes then issue V
+                    const int pg = lane & 7, half = (lane >> 3) & 1;
+                    const int row = (__shfl_sync(0xffffffffu, pid, pg) * Hkv + w.kvh) * kPage;
+                    if (lane < 16 && pg < npages) {
+                        char *kd = k_s + s * kTileBytes + half * kHalfBytes + pg * kBoxBytes;
+                        char *vd = v_s + s * kTileBytes + half * kHalfBytes + pg * kBoxBytes;
+                        tma_box_load(kd, &k_map, half * 64, row, &bars->k_full[s]);
+                        tma_box_load(vd, &v_map, half * 64, row, &bars->v_full[s]);
+                    }
+                }
+                __syncwarp();
+            }
+        }
+    } else if (warp == 5) {
+        // ====================================== MMA issue ===========================================
+        if (lane == 0) {
+            constexpr uint32_t idesc_qk = instr_desc(false), idesc_pv = instr_desc(true);
+            const uint32_t q_addr = smem_u32(q_s), p_addr = smem_u32(p_s);
+            uint32_t it = 0, nitem = 0;
+            Item w;
+            for (int item = blockIdx.x; get_item<G>(item, total, pref, row0, B, Hkv, a, w); item += gridDim.x, ++nitem) {
+                mbar_wait(&bars->q_full, nitem & 1u, abort, a.status);
+                for (int j = 0; j < w.ntiles; ++j, ++it) {
+                    const uint32_t s = it % kStages, par = (it / kStages) & 1u;
+                    const uint32_t k_addr = smem_u32(k_s + s * kTileBytes), v_addr = smem_u32(v_s + s * kTileBytes);
+                    // ---- S = Q K^T: 8 steps of 16 dims; 4 per 64-dim half; K-major operands, SBO = 8 rows
+                    mbar_wait(&bars->k_full[s], par, abort, a.status);
+                    tc_fence_after();
+#pragma unroll
+                    for (int ks = 0; ks < kD / 16; ++ks) {
+                        const uint32_t off = (ks >> 2) * kHalfBytes + (ks & 3) * 32;
+                        mma_f16_ss(tmem, smem_desc(q_addr + off, 16, 1024), smem_desc(k_addr + off, 16, 1024), idesc_qk,
+                                   ks > 0 ? 1u : 0u);
+                    }
+                    mma_commit(&bars->s_full);
+                    // ---- O += P V: 8 steps of 16 keys; P K-major; V MN-major: 64-dim halves LBO apart,
+                    //      8-key groups SBO apart
+                    mbar_wait(&bars->p_full, it & 1u, abort, a.status);
+                    mbar_wait(&bars->v_full[s], par, abort, a.status);
+                    tc_fence_after();
+#pragma unroll
+                    for (int ks = 0; ks < kBN / 16; ++ks) {
+                        const uint32_t p_off = (ks >> 2) * kHalfBytes + (ks & 3) * 32;
+                        mma_f16_ss(tmem + kBN, smem_desc(p_addr + p_off, 16, 1024),
+                                   smem_desc(v_addr + ks * 2 * 1024, kHalfBytes, 1024), idesc_pv,
+                                   (j > 0 || ks > 0) ? 1u : 0u);
+                    }
+                    mma_commit(&bars->kv_empty[s]);
+                    mma_commit(&bars->o_full);
+                }
+            }
+        }
+        __syncwarp();
+    } else {
+        // ================================ softmax and epilogue ====================================
+        const uint32_t lane_base = (uint32_t)(warp * 32) << 16;  // this warp's TMEM lane quadrant
+        const uint32_t s_tmem = tmem + lane_base, o_tmem = tmem + lane_base + kBN;
+        const int swz = tid & 7;
+        uint32_t it = 0, nitem = 0;
+        Item w;
+        for (int item = blockIdx.x; get_item<G>(item, total, pref, row0, B, Hkv, a, w); item += gridDim.x, ++nitem) {
+            const bool row_ok = tid < w.rows_here;
+            const int r = min(w.r_begin + tid, w.rows_total - 1);
+            const int tok = r / G, head = r - tok * G;
+            const int lim = w.L - w.n + tok + 1;  // keys this row may see
+            const size_t grow = ((size_t)(w.qrow0 + tok) * a.Hq + w.kvh * G + head) * kD;
+            // ---- Q tile: row `tid`, 16 chunks of 8 dims, chunk c of a half stored at c ^ (row & 7)
+            {
+                const uint4 *src = reinterpret_cast<const uint4 *>(a.q + grow * 2);
+#pragma unroll
+                for (int c = 0; c < 16; ++c) {
+                    const uint4 v = row_ok ? __ldg(src + c) : make_uint4(0, 0, 0, 0);
+                    *reinterpret_cast<uint4 *>(q_s + (c >> 3) * kHalfBytes + tid * 128 + (((c & 7) ^ swz) << 4)) = v;
+                }
+                fence_async_smem();
+                mbar_arrive(&bars->q_full);
+            }
+            float m_used = -INFINITY, l_sum = 0.f;
+            for (int j = 0; j < w.ntiles; ++j, ++it) {
+                const uint32_t s = it % kStages, par = (it / kStages) & 1u;
+                const int key0 = j * kBN;
+                const int nvis = lim - key0;  // columns < nvis are visible to this row (may be <= 0)
+                mbar_wait(&bars->s_full, it & 1u, abort, a.status);
+                tc_fence_after();
+                // ---- pass 1: row max of the visible scores
+                float mx = -INFINITY;
+#pragma unroll 1
+                for (int c4 = 0; c4 < 4; ++c4) {
+                    uint32_t v[32];
+                    tmem_ld32(s_tmem + c4 * 32, v);
+                    tmem_wait_ld();
+                    if (nvis >= (c4 + 1) * 32) {
+#pragma unroll
+                        for (int k = 0; k < 32; ++k) mx = fmaxf(mx, __uint_as_float(v[k]));
+                    } else {
+#pragma unroll
+                        for (int k = 0; k < 32; ++k)
+                            if (c4 * 32 + k < nvis) mx = fmaxf(mx, __uint_as_float(v[k]));
+                    }
+                }
+                const float m_tile = mx * a.scale_log2;  // -inf if this row sees nothing of the tile
+                float factor = 1.0f;
+                bool rescale = false;
+                if (m_tile > m_used + kRescaleThreshold || (m_used == -INFINITY && m_tile > -INFINITY)) {
+                    factor = fast_exp2(m_used - m_tile);  // 0 the first time
+                    rescale = j > 0;
+                    l_sum *= factor;
+                    m_used = m_tile;
+                }
+                if (__any_sync(0xffffffffu, rescale)) {
+                    // O of the previous tiles is complete: s_full of this tile was committed after them
+#pragma unroll 1
+                    for (int c4 = 0; c4 < 4; ++c4) {
+                        uint32_t v[32];
+                        tmem_ld32(o_tmem + c4 * 32, v);
+                        tmem_wait_ld();
+#pragma unroll
+                        for (int k = 0; k < 32; ++k) v[k] = __float_as_uint(__uint_as_float(v[k]) * factor);
+                        tmem_st32(o_tmem + c4 * 32, v);
+                    }
+                    tmem_wait_st();
+                }
+                // ---- pass 2: P = exp2(scale * S - m), bf16, into the swizzled K-major P tile
+                const float neg_m = (m_used == -INFINITY) ? 0.f : -m_used;
+#pragma unroll 1
+                for (int c4 = 0; c4 < 4; ++c4) {
+                    uint32_t v[32];
+                    tmem_ld32(s_tmem + c4 * 32, v);
+                    tmem_wait_ld();
+                    // The weights are rounded to bf16 BEFORE they are summed, so the tensor core's
+                    // numerator and the fp32 denominator use the very same weights and the result
+                    // stays a true convex combination of V rows.
+                    uint32_t pk[16];
+#pragma unroll
+                    for (int k = 0; k < 16; ++k) {
+                        const float e0 = fast_exp2(fmaf(__uint_as_float(v[2 * k]), a.scale_log2, neg_m));
+                        const float e1 = fast_exp2(fmaf(__uint_as_float(v[2 * k + 1]), a.scale_log2, neg_m));
+                        const uint32_t w = pack_bf16((c4 * 32 + 2 * k < nvis) ? e0 : 0.f,
+                                                     (c4 * 32 + 2 * k + 1 < nvis) ? e1 : 0.f);
+                        pk[k] = w;
+                        l_sum += __uint_as_float(w << 16) + __uint_as_float(w & 0xffff0000u);
+                    }
+                    char *prow = p_s + (c4 >> 1) * kHalfBytes + tid * 128;
+#pragma unroll
+                    for (int qd = 0; qd < 4; ++qd) {
+                        const int cc = (c4 & 1) * 4 + qd;
+                        *reinterpret_cast<uint4 *>(prow + ((cc ^ swz) << 4)) =
+                            make_uint4(pk[qd * 4 + 0], pk[qd * 4 + 1], pk[qd * 4 + 2], pk[qd * 4 + 3]);
+                    }
+                }
+                // ---- V rows past the last visible key of the item (stale slots, pages never loaded)
+                //      must not reach the tensor core, not even times zero
+                const int nvalid = w.kv_len - key0;
+                if (nvalid < kBN) {
+                    mbar_wait(&bars->v_full[s], par, abort, a.status);
+                    if (tid >= nvalid) {
+                        char *vrow = v_s + s * kTileBytes + tid * 128;
+#pragma unroll
+                        for (int c = 0; c < 8; ++c) {
+                            *reinterpret_cast<uint4 *>(vrow + c * 16) = make_uint4(0, 0, 0, 0);
+                            *reinterpret_cast<uint4 *>(vrow + kHalfBytes + c * 16) = make_uint4(0, 0, 0, 0);
+                        }
+                    }
+                }
+                fence_async_smem();
+                tc_fence_before();
+                mbar_arrive(&bars->p_full);
+            }
+            // ---- epilogue: O / l, bf16, one 256-byte row per thread
+            mbar_wait(&bars->o_full, (it - 1u) & 1u, abort, a.status);
+            tc_fence_after();
+            const float inv_l = 1.0f / l_sum;
+            uint4 *dst = reinterpret_cast<uint4 *>(a.out + grow * 2);
+#pragma unroll 1
+            for (int c4 = 0; c4 < 4; ++c4) {
+                uint32_t v[32];
+                tmem_ld32(o_tmem + c4 * 32, v);
+                tmem_wait_ld();
+                if (row_ok) {
+#pragma unroll
+                    for (int qd = 0; qd < 4; ++qd) {
+                        uint4 o4;
+                        o4.x = pack_bf16(__uint_as_float(v[qd * 8 + 0]) * inv_l, __uint_as_float(v[qd * 8 + 1]) * inv_l);
+                        o4.y = pack_bf16(__uint_as_float(v[qd * 8 + 2]) * inv_l, __uint_as_float(v[qd * 8 + 3]) * inv_l);
+                        o4.z = pack_bf16(__uint_as_float(v[qd * 8 + 4]) * inv_l, __uint_as_float(v[qd * 8 + 5]) * inv_l);
+                        o4.w = pack_bf16(__uint_as_float(v[qd * 8 + 6]) * inv_l, __uint_as_float(v[qd * 8 + 7]) * inv_l);
+                        dst[c4 * 4 + qd] = o4;
+                    }
+                }
+            }
+            tc_fence_before();
+        }
+    }
+
+    // ---- teardown: everyone is done with TMEM before the allocating warp frees it ------------------
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 5) {
+        tc_fence_after();
+        tmem_dealloc(tmem, kTmemCols);
+    }
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_tiled_fn() {
+    static EncodeTiledFn fn = nullptr;
+    static bool tried = false;
+    if (!tried) {
+        tried = true;
+        void *p = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) == cudaSuccess &&
+            qres == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(p);
+        cudaGetLastError();
+    }
+    return fn;
+}
+
+// 2-D view of a page pool: rows = (page, kv head, slot), 128 bf16 columns; box = one page-head, 64 columns
+bool make_pool_map(CUtensorMap *map, const void *pool, const arb_attn_params &p) {
+    EncodeTiledFn fn = encode_tiled_fn();
+    if (!fn) return false;
+    const cuuint64_t dims[2] = {(cuuint64_t)kD, (cuuint64_t)p.num_pages * p.num_kv_heads * kPage};
+    const cuuint64_t strides[1] = {(cuuint64_t)kD * 2};
+    const cuuint32_t box[2] = {64, (cuuint32_t)kPage};
+    const cuuint32_t estr[2] = {1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(pool), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+template <int G>
+arb_status launch_one(Ctx *ctx, const MmaArgs &a, const CUtensorMap &km, const CUtensorMap &vm, int max_items,
+                      cudaStream_t stream) {
+    const size_t smem = mma_smem_bytes(a.batch);
+    static bool attr_set[64] = {};
+    if (!attr_set[ctx->device & 63]) {
+        if (cudaFuncSetAttribute(chunk_mma_kernel<G>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 (int)mma_smem_bytes(kMaxBatch)) != cudaSuccess)
+            return ARB_ERR_CUDA;
+        attr_set[ctx->device & 63] = true;
+    }
+    const int grid = max_items < ctx->num_sms ? max_items : ctx->num_sms;
+    chunk_mma_kernel<G><<<grid, kThreads, smem, stream>>>(a, km, vm);
+    ctx->launches++;
+    return cudaGetLastError() == cudaSuccess ? ARB_OK : ARB_ERR_CUDA;
+}
+
+}  // namespace
+
+bool chunk_mma_supported(const arb_attn_params &p) {
+    const int g = p.num_q_heads / p.num_kv_heads;
+    return p.dtype == ARB_BF16 && p.head_dim == kD && p.max_q_len >= 2 && p.max_q_len * g >= kChunkMmaMinRows &&
+           encode_tiled_fn() != nullptr;
+}
+
+arb_status launch_chunk_mma(Ctx *ctx, const arb_attn_params &p, const void *q, const void *k_pages,
+                            const void *v_pages, const int32_t *block_table, const int32_t *seq_lens,
+                            const int32_t *q_lens, void *out, cudaStream_t stream) {
+    alignas(64) CUtensorMap km, vm;
+    if (!make_pool_map(&km, k_pages, p) || !make_pool_map(&vm, v_pages, p)) return ARB_ERR_CUDA;
+    MmaArgs a;
+    a.q = static_cast<const char *>(q);
+    a.block_table = block_table;
+    a.seq_lens = seq_lens;
+    a.q_lens = q_lens;
+    a.out = static_cast<char *>(out);
+    a.status = ctx->status;
+    a.batch = p.batch;
+    a.Hq = p.num_q_heads;
+    a.Hkv = p.num_kv_heads;
+    a.num_pages = p.num_pages;
+    a.max_pages = p.max_pages_per_seq;
+    a.min_rows = kChunkMmaMinRows;
+    const float scale = p.softmax_scale > 0.f ? p.softmax_scale : 1.0f / sqrtf((float)p.head_dim);
+    a.scale_log2 = scale * 1.4426950408889634f;
+    const int g = p.num_q_heads / p.num_kv_heads;
+    // upper bound of the work items from what the host knows: every row could sit in its own tile run
+    const long long bound = (long long)p.num_kv_heads * ((long long)p.total_q * g / kBM + p.batch);
+    const int max_items = (int)(bound < 1 ? 1 : (bound > (1 << 30) ? (1 << 30) : bound));
+    switch (g) {
+        case 1: return launch_one<1>(ctx, a, km, vm, max_items, stream);
+        case 2: return launch_one<2>(ctx, a, km, vm, max_items, stream);
+        case 3: return launch_one<3>(ctx, a, km, vm, max_items, stream);
+        case 4: return launch_one<4>(ctx, a, km, vm, max_items, stream);
+        case 5: return launch_one<5>(ctx, a, km, vm, max_items, stream);
+        case 6: return launch_one<6>(ctx, a, km, vm, max_items, stream);
+        case 7: return launch_one<7>(ctx, a, km, vm, max_items, stream);
+        case 8: return launch_one<8>(ctx, a, km, vm, max_items, stream);
+        default: return ARB_ERR_UNSUPPORTED;
+    }
+}
+
+}  // namespace arb

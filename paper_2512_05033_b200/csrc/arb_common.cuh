@@ -12,6 +12,7 @@ namespace arb {
 constexpr int kPage = 16;             // tokens per KV page
 constexpr int kMaxBatch = 1024;       // sequences per call (prefix tables live in shared memory)
 constexpr int kMaxGroup = 8;          // query heads per KV head
+constexpr int kChunkMmaMinRows = 64;  // q_len * group from which a chunk goes to the tensor cores
 constexpr long long kWaitCycles = 1ll << 31;  // bound of every mbarrier wait (about a second)
 
 // ---------------------------------------------------------------------------------------------
@@ -167,7 +168,12 @@ arb_status launch_decode(Ctx *ctx, const arb_attn_params &p, const void *q, cons
                          const int32_t *q_lens, void *out, cudaStream_t stream);
 arb_status launch_chunk_fma(Ctx *ctx, const arb_attn_params &p, const void *q, const void *k_pages,
                             const void *v_pages, const int32_t *block_table, const int32_t *seq_lens,
-                            const int32_t *q_lens, void *out, int n_lo, int n_hi, cudaStream_t stream);
+                            const int32_t *q_lens, void *out, int n_lo, int n_hi, int skip_rows,
+                            cudaStream_t stream);
+bool chunk_mma_supported(const arb_attn_params &p);
+arb_status launch_chunk_mma(Ctx *ctx, const arb_attn_params &p, const void *q, const void *k_pages,
+                            const void *v_pages, const int32_t *block_table, const int32_t *seq_lens,
+                            const int32_t *q_lens, void *out, cudaStream_t stream);
 arb_status launch_route(Ctx *ctx, int dtype, int n_steps, int hidden_dim, const void *hidden, const void *w,
                         float b, float tau, float *scores, uint8_t *decisions, cudaStream_t stream);
 arb_status launch_rollback(Ctx *ctx, int batch, int32_t *seq_lens, const int32_t *step_lens,

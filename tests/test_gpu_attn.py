@@ -56,6 +56,12 @@ def test_decode_idle_slots_and_scale():
 
 
 CHUNK_CASES = [
+    # chunks with q_len * group >= 64 rows in bf16 / head_dim 128 run on the tensor cores
+    (1, 32, 8, 128, BF, [300], [64]),                        # g = 4: 256 rows = two full row tiles
+    (2, 28, 4, 128, BF, [600, 2100], [16, 100]),             # g = 7: 112 rows (one ragged tile), 700 rows
+    (2, 12, 2, 128, BF, [131, 128], [128, 11]),              # chunk is almost the whole sequence; 66 rows
+    (4, 32, 8, 128, BF, [5000, 77, 1300, 256], [1, 30, 128, 5]),   # decode + tensor-core + CUDA-core chunks
+    (1, 16, 2, 128, BF, [4099], [19]),                       # g = 8: 152 rows, key count not a page multiple
     (1, 8, 2, 64, F32, [528], [16]),                         # the tiny config: 16-token chunk, prefix 512
     (2, 12, 2, 128, BF, [300, 40], [7, 40]),                 # chunk == whole sequence (no prefix)
     (3, 28, 4, 128, BF, [200, 90, 1000], [3, 1, 5]),         # decode and chunk rows in one call
@@ -71,7 +77,44 @@ def test_chunk_matches_oracle(case):
     out, bits = H.gpu_attn(inp)
     ref, st = H.oracle_attn(inp)
     assert bits == 0 and st == 0
-    H.assert_close(out, ref, dt, tight=1e-3 if dt == BF else None)
+    # chunks on the tensor cores carry bf16 softmax weights into the second product
+    on_mma = dt == BF and D == 128 and max(ql) * (Hq // Hkv) >= 64
+    H.assert_close(out, ref, dt, tight=(3e-3 if on_mma else 1e-3) if dt == BF else None)
+
+
+def test_large_chunk_peaked_and_stale_slots():
+    """Tensor-core chunk path: concentrated softmax, and NaN / 1e30 in the slots after the sequence end."""
+    inp = wl.small_attn_case(2, 28, 4, 128, BF, [1000, 333], [40, 64], seed=43, q_std=4.0, extra_tokens=50)
+    clean, bits = H.gpu_attn(inp)
+    assert bits == 0
+    ref, _ = H.oracle_attn(inp)
+    err = np.abs(clean - ref)
+    # The softmax weights enter the second product rounded to bf16 (relative 2^-9 each), the output is
+    # rounded to bf16 once more.  Gross bound for every element, exact bound on sampled rows.
+    vmax = float(inp.v_pages.abs().max())
+    assert (err <= 2.0 ** -8 * np.abs(ref) + 2.0 ** -9 * 2 * vmax).all(), err.max()
+    from oracle import oracle
+    rng = np.random.default_rng(0)
+    rows0 = np.cumsum([0] + [int(x) for x in inp.q_lens])
+    Vd = inp.v_pages.double().numpy()
+    for _ in range(48):
+        b = int(rng.integers(0, 2)); n = int(inp.q_lens[b]); L = int(inp.seq_lens[b])
+        i = int(rng.integers(0, n)); h = int(rng.integers(0, 28)); row = rows0[b] + i; pos = L - n + i
+        o, p, _ = oracle.attn_row_probs(inp.q, inp.k_pages, inp.v_pages, inp.block_table[b], row, h, pos)
+        bt = inp.block_table[b].numpy()
+        v = np.stack([Vd[bt[j // wl.PAGE], h // 7, j % wl.PAGE] for j in range(pos + 1)])      # [keys, D]
+        bound = 2.0 ** -9 * (p[:, None] * np.abs(v - o[None, :])).sum(axis=0) + 2.0 ** -8 * np.abs(o) + 1e-3
+        assert (np.abs(clean[row, h] - o) <= bound).all(), (b, i, h)
+    k2, v2 = inp.k_pages.clone(), inp.v_pages.clone()
+    for b in range(2):
+        L = int(inp.seq_lens[b])
+        for j in range(L, L + 50):
+            pg = int(inp.block_table[b, j // wl.PAGE])
+            k2[pg, :, j % wl.PAGE] = float("nan")
+            v2[pg, :, j % wl.PAGE] = 1e30
+    out, bits = H.gpu_attn(wl.AttnInputs(inp.shape, inp.q, k2, v2, inp.block_table, inp.seq_lens, inp.q_lens))
+    assert bits == 0
+    np.testing.assert_array_equal(out, clean)
 
 
 def test_stale_slots_never_reach_the_output():

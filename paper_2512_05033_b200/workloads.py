@@ -206,3 +206,48 @@ def small_attn_case(batch, num_q_heads, num_kv_heads, head_dim, dtype, seq_lens,
     v = normal((num_pages, num_kv_heads, PAGE, head_dim), 1.0, dtype, device, seed * 1000 + 3)
     return AttnInputs(shape, q, k, v, bt.to(device), seq.to(torch.int32).to(device),
                       ql.to(torch.int32).to(device))
+
+
+@dataclasses.dataclass
+class MixedLoopInputs:
+    """Everything the mixed serving loop draws: one KV pool whose slots already hold N(0,1) values
+    (so appending a token is just a longer seq_len), the starting lengths, and per iteration the
+    query lengths (even index + iteration: decode, q_len 1; odd: a step of 16..128 tokens), the query
+    rows and the router's hidden rows."""
+    shape: AttnShape
+    k_pages: torch.Tensor
+    v_pages: torch.Tensor
+    block_table: torch.Tensor      # int32 [B, max_pages], capacity for every append of the loop
+    seq_lens0: torch.Tensor        # int32 [B] lengths before the first iteration
+    q_lens: list                   # per iteration int32 [B]
+    q: list                        # per iteration [sum q_lens, Hq, D]
+    hidden: list                   # per iteration [B, hidden]
+    w: torch.Tensor
+    b: float
+    tau: float = 0.5
+
+
+def make_mixed_loop(shape: AttnShape = MIXED_LOOP, iterations: int = 10, device="cpu",
+                    seed: Optional[int] = None) -> MixedLoopInputs:
+    seed = shape.seed if seed is None else seed
+    gen = _cpu_gen(seed)
+    B = shape.batch
+    prefix = draw_prefix_lens(shape, gen)
+    idx = torch.arange(B)
+    q_lens, total_new = [], torch.zeros(B, dtype=torch.int64)
+    for it in range(iterations):
+        steps = torch.randint(shape.q_lo, shape.q_hi + 1, (B,), generator=gen)
+        ql = torch.where((idx + it) % 2 == 0, torch.ones(B, dtype=torch.int64), steps)
+        q_lens.append(ql)
+        total_new += ql
+    bt, num_pages = make_block_table(prefix, gen, extra_tokens=int(total_new.max()), headroom_pages=3)
+    H, Hk, D = shape.num_q_heads, shape.num_kv_heads, shape.head_dim
+    k = normal((num_pages, Hk, PAGE, D), 1.0, shape.dtype, device, seed * 1000 + 2)
+    v = normal((num_pages, Hk, PAGE, D), 1.0, shape.dtype, device, seed * 1000 + 3)
+    q = [normal((int(ql.sum()), H, D), 1.0, shape.dtype, device, seed * 1000 + 100 + it)
+         for it, ql in enumerate(q_lens)]
+    hidden = [normal((B, shape.hidden), 1.0, shape.dtype, device, seed * 1000 + 200 + it)
+              for it in range(iterations)]
+    w = normal((shape.hidden,), 1.0 / math.sqrt(shape.hidden), shape.dtype, device, seed * 1000 + 12)
+    return MixedLoopInputs(shape, k, v, bt.to(device), prefix.to(torch.int32).to(device),
+                           [x.to(torch.int32).to(device) for x in q_lens], q, hidden, w, 0.0, 0.5)

@@ -47,7 +47,8 @@ typedef enum {
     ARB_ERR_UNSUPPORTED = 2,   /* head_dim, group size, page size or dtype outside the built set */
     ARB_ERR_WORKSPACE = 3,     /* the ctx workspace is smaller than arb_attn_workspace_bytes() */
     ARB_ERR_CUDA = 4,          /* a CUDA runtime call failed (allocation, launch, copy) */
-    ARB_ERR_DEVICE_STATUS = 5  /* arb_poll_status: the device status word is non-zero */
+    ARB_ERR_DEVICE_STATUS = 5, /* arb_poll_status: the device status word is non-zero */
+    ARB_ERR_STATIC_LIMIT = 6   /* arb_attn_decode_static: the call needs more than the built-in scratch */
 } arb_status;
 
 typedef enum { ARB_F32 = 0, ARB_BF16 = 1 } arb_dtype;
@@ -146,6 +147,40 @@ arb_status arb_attn_host(arb_ctx *ctx, const arb_attn_params *params, const void
                          const void *k_pages, const void *v_pages,
                          const int32_t *block_table_host, const int32_t *seq_lens_host,
                          const int32_t *q_lens_host, void *out_host, arb_stream_t stream);
+
+/*
+ * Decode attention (q_len = 1 for every sequence) for callers that must not allocate.
+ *
+ * The paper has no counterpart to this call; it exists for the way the library gets embedded.
+ * Some hosts cannot afford a cudaMalloc at any point after start-up: a serving process that has
+ * already given every free byte of device memory to its KV-cache pool, or a plug-in that runs in
+ * the middle of another framework's operator, where an allocation would stall the whole device
+ * and may fail outright.  arb_create allocates, so such callers cannot hold an arb_ctx.  This
+ * entry point needs none: the split-KV partials, the arrival counters and the status word live in
+ * a fixed 4 MiB array that is part of the library image (every GPU that loads the library carries
+ * it until the process exits).  It calls no cudaMalloc, cudaFree or any other allocating routine.
+ *
+ * Arguments are those of arb_attn with params->max_q_len == 1 and params->total_q equal to the
+ * number of sequences with q_lens[b] == 1 (other q_lens must be 0).  device_status is an optional
+ * caller-owned device word: device-side problems (ARB_DEV_* bits) are OR-ed into it; pass NULL to
+ * ignore them.  Results equal arb_attn's.
+ *
+ * Limits and sharing.  The call is refused with ARB_ERR_STATIC_LIMIT, and nothing is launched,
+ * when batch * num_kv_heads > 1024 or when the call's scratch,
+ *     (batch * num_kv_heads + 2 * SM count) * (g * head_dim + 2 * roundup4(g)) * 4 + 4352 bytes,
+ * exceeds the 4 MiB array (the draft- and target-shaped decode workloads need under 1 MiB).  All
+ * calls in the process that target the same GPU share the one array and it keeps whatever the last call left:
+ * the counters and the internal status word are cleared on `stream` at the start of every call,
+ * but two calls that overlap on the GPU (different streams, or a programmatic dependent of each
+ * other) race on it and corrupt each other's results; ARB_ATTN_OVERLAP_PREVIOUS is therefore
+ * rejected with ARB_ERR_INVALID_ARG.  The current device must be the one the pointers live on.
+ * The first call on a device looks up the array's device address and sets the kernel's
+ * shared-memory attribute; make that first call before any stream capture begins.
+ */
+arb_status arb_attn_decode_static(const arb_attn_params *params, const void *q, const void *k_pages,
+                                  const void *v_pages, const int32_t *block_table,
+                                  const int32_t *seq_lens, const int32_t *q_lens, void *out,
+                                  uint32_t *device_status /* nullable */, arb_stream_t stream);
 
 /*
  * Router head and threshold decision (Section 4.2: the score is the likelihood that the target

@@ -21,12 +21,14 @@ lib = ctypes.CDLL(str(_LIB_PATH))
 
 ARB_OK = 0
 ARB_ERR_INVALID_ARG, ARB_ERR_UNSUPPORTED, ARB_ERR_WORKSPACE, ARB_ERR_CUDA, ARB_ERR_DEVICE_STATUS = 1, 2, 3, 4, 5
+ARB_ERR_STATIC_LIMIT = 6
 ARB_F32, ARB_BF16 = 0, 1
 DEV_BAD_SEQ_LEN, DEV_BAD_PAGE, DEV_ROLLBACK_UNDERFLOW, DEV_WAIT_TIMEOUT = 1, 2, 4, 8
 ATTN_OVERLAP_PREVIOUS = 1
 
 # every symbol include/arb.h declares
 EXPORTS = ("arb_create", "arb_destroy", "arb_attn_workspace_bytes", "arb_attn", "arb_attn_host",
+           "arb_attn_decode_static",
            "arb_route", "arb_rollback", "arb_poll_status", "arb_launch_count", "arb_status_string")
 
 
@@ -49,6 +51,8 @@ lib.arb_attn.restype = ctypes.c_int
 lib.arb_attn.argtypes = [_vp, ctypes.POINTER(AttnParams), _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp]
 lib.arb_attn_host.restype = ctypes.c_int
 lib.arb_attn_host.argtypes = [_vp, ctypes.POINTER(AttnParams), _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp]
+lib.arb_attn_decode_static.restype = ctypes.c_int
+lib.arb_attn_decode_static.argtypes = [ctypes.POINTER(AttnParams), _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp]
 lib.arb_route.restype = ctypes.c_int
 lib.arb_route.argtypes = [_vp, _i32, _i32, _i32, _vp, _vp, _f, _f, _vp, _vp, _vp]
 lib.arb_rollback.restype = ctypes.c_int
@@ -98,6 +102,29 @@ def attn_params(q_dtype_code, batch, num_q_heads, num_kv_heads, head_dim, num_pa
                 max_q_len, softmax_scale=0.0, page_size=16, flags=0) -> AttnParams:
     return AttnParams(q_dtype_code, batch, num_q_heads, num_kv_heads, head_dim, page_size, num_pages,
                       max_pages_per_seq, total_q, max_q_len, softmax_scale, flags)
+
+
+def attn_decode_static(q, k_pages, v_pages, block_table, seq_lens, q_lens, out=None, device_status=None,
+                       softmax_scale: float = 0.0, stream=None):
+    """Decode attention (every q_len 1 or 0) through arb_attn_decode_static: no arb_ctx, and no
+    allocation inside the library -- its scratch is a fixed array in the library image.  For hosts
+    that must not allocate after start-up (a server whose free memory all went to the KV pool, a
+    plug-in inside another framework's operator).  `out` should be passed in for the same reason;
+    it is created here only as a convenience.  Calls that overlap on the GPU race on the shared
+    scratch.  Returns out."""
+    if out is None:
+        out = torch.empty_like(q)
+    total_q, Hq, D = q.shape
+    num_pages, Hkv, P, _ = k_pages.shape
+    B, max_pages = block_table.shape
+    p = attn_params(_dtype_code(q), B, Hq, Hkv, D, num_pages, max_pages, total_q, 1, softmax_scale, P)
+    sp = None if device_status is None else _dev(device_status, "device_status", torch.int32)
+    st = lib.arb_attn_decode_static(ctypes.byref(p), _dev(q, "q"), _dev(k_pages, "k_pages", q.dtype),
+                                    _dev(v_pages, "v_pages", q.dtype), _dev(block_table, "block_table", torch.int32),
+                                    _dev(seq_lens, "seq_lens", torch.int32), _dev(q_lens, "q_lens", torch.int32),
+                                    _dev(out, "out", q.dtype), sp, _stream_ptr(stream))
+    _check(st, "arb_attn_decode_static")
+    return out
 
 
 class Context:

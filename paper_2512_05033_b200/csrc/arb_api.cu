@@ -135,6 +135,19 @@ arb_status arb_attn(arb_ctx *ctx, const arb_attn_params *params, const void *q, 
     return ARB_OK;
 }
 
+arb_status arb_attn_decode_static(const arb_attn_params *params, const void *q, const void *k_pages,
+                                  const void *v_pages, const int32_t *block_table, const int32_t *seq_lens,
+                                  const int32_t *q_lens, void *out, uint32_t *device_status, arb_stream_t stream) {
+    arb_status st = check_params(params);
+    if (st != ARB_OK) return st;
+    if (params->max_q_len != 1 || params->total_q < 1 || params->total_q > params->batch) return ARB_ERR_INVALID_ARG;
+    if (params->flags & ARB_ATTN_OVERLAP_PREVIOUS) return ARB_ERR_INVALID_ARG;  // calls share one scratch array
+    if (!q || !out || !k_pages || !v_pages || !block_table || !seq_lens || !q_lens) return ARB_ERR_INVALID_ARG;
+    if (!aligned16(q) || !aligned16(out) || !aligned16(k_pages) || !aligned16(v_pages)) return ARB_ERR_INVALID_ARG;
+    return launch_decode_static(*params, q, k_pages, v_pages, block_table, seq_lens, q_lens, out, device_status,
+                                reinterpret_cast<cudaStream_t>(stream));
+}
+
 arb_status arb_attn_host(arb_ctx *ctx, const arb_attn_params *params, const void *q_host, const void *k_pages,
                          const void *v_pages, const int32_t *block_table_host, const int32_t *seq_lens_host,
                          const int32_t *q_lens_host, void *out_host, arb_stream_t stream) {
@@ -227,6 +240,7 @@ const char *arb_status_string(arb_status status) {
         case ARB_ERR_WORKSPACE: return "workspace too small";
         case ARB_ERR_CUDA: return "CUDA runtime error";
         case ARB_ERR_DEVICE_STATUS: return "device status word is non-zero";
+        case ARB_ERR_STATIC_LIMIT: return "call exceeds the built-in scratch of the no-allocation entry point";
         default: return "unknown status";
     }
 }

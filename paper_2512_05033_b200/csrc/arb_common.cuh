@@ -178,6 +178,9 @@ arb_status launch_route(Ctx *ctx, int dtype, int n_steps, int hidden_dim, const 
                         float b, float tau, float *scores, uint8_t *decisions, cudaStream_t stream);
 arb_status launch_rollback(Ctx *ctx, int batch, int32_t *seq_lens, const int32_t *step_lens,
                            const uint8_t *decisions, cudaStream_t stream);
+arb_status launch_decode_static(const arb_attn_params &p, const void *q, const void *k_pages, const void *v_pages,
+                                const int32_t *block_table, const int32_t *seq_lens, const int32_t *q_lens,
+                                void *out, uint32_t *device_status, cudaStream_t stream);
 size_t decode_workspace_bytes(const arb_attn_params &p, int num_sms);
 int decode_grid(int num_sms);
 

@@ -721,7 +721,86 @@ inline size_t slot_count(const arb_attn_params &p, int num_sms) {
     return (size_t)p.batch * p.num_kv_heads + (size_t)num_sms * kMaxCtasPerSm;
 }
 
+// ---- scratch for arb_attn_decode_static ------------------------------------------------------------
+// In host code `g_static_scratch` is only a stand-in for the symbol, not a device address; the
+// address a kernel can use comes from cudaGetSymbolAddress, once per device.
+constexpr size_t kStaticScratchBytes = 4u << 20;
+constexpr int kStaticMaxBk = 1024;                              // batch * kv heads
+constexpr size_t kStaticCounterBytes = sizeof(int) * kStaticMaxBk + 256;   // counters, then the status word
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
+
+struct StaticSetup {
+    bool ready = false;
+    unsigned char *base = nullptr;
+    int num_sms = 0;
+};
+StaticSetup g_static_setup[64];
+
 }  // namespace
+
+arb_status launch_decode_static(const arb_attn_params &p, const void *q, const void *k_pages, const void *v_pages,
+                                const int32_t *block_table, const int32_t *seq_lens, const int32_t *q_lens,
+                                void *out, uint32_t *device_status, cudaStream_t stream) {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return ARB_ERR_CUDA;
+    StaticSetup &su = g_static_setup[dev];
+    if (!su.ready) {  // first call on this device: it is current, so the symbol resolves to its copy
+        void *ptr = nullptr;
+        if (cudaGetSymbolAddress(&ptr, g_static_scratch) != cudaSuccess || ptr == nullptr) {
+            cudaGetLastError();
+            return ARB_ERR_CUDA;
+        }
+        int sms = 0;
+        if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms < 1)
+            return ARB_ERR_CUDA;
+        su.base = static_cast<unsigned char *>(ptr);
+        su.num_sms = sms;
+        su.ready = true;
+    }
+    const int g = p.num_q_heads / p.num_kv_heads;
+    const int gp = (g + 3) / 4 * 4;
+    if ((long long)p.batch * p.num_kv_heads > kStaticMaxBk) return ARB_ERR_STATIC_LIMIT;
+    const size_t slots = (size_t)p.batch * p.num_kv_heads + (size_t)su.num_sms * kMaxCtasPerSm;
+    const size_t part_o_floats = (slots * g * p.head_dim + 63) & ~size_t(63);
+    const size_t need = kStaticCounterBytes + (part_o_floats + slots * gp * 2) * sizeof(float);
+    if (need > kStaticScratchBytes) return ARB_ERR_STATIC_LIMIT;
+
+    // [counters | internal status word | pad to 256 B][partial outputs][partial max/sum records]
+    int *counters = reinterpret_cast<int *>(su.base);
+    uint32_t *own_status = reinterpret_cast<uint32_t *>(su.base + sizeof(int) * kStaticMaxBk);
+    if (cudaMemsetAsync(su.base, 0, kStaticCounterBytes, stream) != cudaSuccess) return ARB_ERR_CUDA;
+
+    Ctx tmp;  // launch bookkeeping only; owns nothing
+    tmp.device = dev;
+    tmp.num_sms = su.num_sms;
+    DecodeArgs a;
+    a.q = static_cast<const char *>(q);
+    a.k_pages = static_cast<const char *>(k_pages);
+    a.v_pages = static_cast<const char *>(v_pages);
+    a.block_table = block_table;
+    a.seq_lens = seq_lens;
+    a.q_lens = q_lens;
+    a.out = static_cast<char *>(out);
+    a.part_o = reinterpret_cast<float *>(su.base + kStaticCounterBytes);
+    a.part_ml = a.part_o + part_o_floats;
+    a.counters = counters;
+    a.status = device_status ? device_status : own_status;
+    a.batch = p.batch;
+    a.Hq = p.num_q_heads;
+    a.Hkv = p.num_kv_heads;
+    a.num_pages = p.num_pages;
+    a.max_pages = p.max_pages_per_seq;
+    const float scale = p.softmax_scale > 0.f ? p.softmax_scale : 1.0f / sqrtf((float)p.head_dim);
+    a.scale_log2 = scale * 1.4426950408889634f;
+    if (p.dtype == ARB_BF16) {
+        if (p.head_dim == 128) return launch_g<__nv_bfloat16, 128>(&tmp, g, a, false, stream);
+        if (p.head_dim == 64) return launch_g<__nv_bfloat16, 64>(&tmp, g, a, false, stream);
+    } else if (p.dtype == ARB_F32) {
+        if (p.head_dim == 128) return launch_g<float, 128>(&tmp, g, a, false, stream);
+        if (p.head_dim == 64) return launch_g<float, 64>(&tmp, g, a, false, stream);
+    }
+    return ARB_ERR_UNSUPPORTED;
+}
 
 size_t decode_workspace_bytes(const arb_attn_params &p, int num_sms) {
     const int g = p.num_q_heads / p.num_kv_heads;

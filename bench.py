@@ -197,6 +197,24 @@ def make_step(ctx, work: DecodeWorkload, use_graph: bool, overlap: bool = False)
 
 
 # ------------------------------------------------------------------------------------------------
+# sharding over ranks: by sequence, every rank its own batch, no data-path collective
+# ------------------------------------------------------------------------------------------------
+def rank_seed(shape: wl.AttnShape, rank: int) -> int:
+    """Weak scaling: rank r draws its own batch of the same shape."""
+    return shape.seed + 1000 * rank
+
+
+def reduce_over_ranks(ms_local: float, kv_bytes_local: float, dist, device):
+    """(slowest rank's time, bytes of all ranks).  `dist` is torch.distributed or None."""
+    t = torch.tensor([ms_local], dtype=torch.float64, device=device)
+    b = torch.tensor([kv_bytes_local], dtype=torch.float64, device=device)
+    if dist is not None:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        dist.all_reduce(b, op=dist.ReduceOp.SUM)
+    return float(t.item()), float(b.item())
+
+
+# ------------------------------------------------------------------------------------------------
 # our arm
 # ------------------------------------------------------------------------------------------------
 def run_ours(args):
@@ -216,7 +234,7 @@ def run_ours(args):
     ctx = binding.Context(local)
     shape = wl.TARGET_DECODE if args.workload == "target" else wl.DRAFT_DECODE
     layers = args.layers or (LAYERS if shape is wl.DRAFT_DECODE else 2)
-    work = DecodeWorkload(shape, layers, dev, seed=shape.seed + 1000 * rank)  # weak scaling: own batch per rank
+    work = DecodeWorkload(shape, layers, dev, seed=rank_seed(shape, rank))
     use_graph = not (args.no_graph or args.profile)
     overlap = not args.no_overlap
     step_fn, per_step = make_step(ctx, work, use_graph, overlap)
@@ -224,13 +242,10 @@ def run_ours(args):
     with ClockSampler(cuda_physical_index(local)) as clk:
         ms = time_steps(step_fn, args.steps, args.warmup, barrier)
     status_bits = ctx.poll_status()
-    t = torch.tensor([ms], dtype=torch.float64, device=dev)
-    if dist:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    ms_max = float(t.item())
-    ms_per_step = ms_max / args.steps
     kv_per_step = work.bytes["kv"] * layers
-    value = world * kv_per_step / (ms_per_step * 1e-3) / 1e9  # same per-rank byte count up to the length draw
+    ms_max, kv_all_ranks = reduce_over_ranks(ms, kv_per_step, dist, dev)
+    ms_per_step = ms_max / args.steps
+    value = kv_all_ranks / (ms_per_step * 1e-3) / 1e9  # whole job: bytes of every rank over the slowest rank's time
 
     peak, peak_kind = measured_peak()
     launch_us = ms / args.steps / per_step * 1e3  # this rank's average launch duration
@@ -250,7 +265,7 @@ def run_ours(args):
                    "overlap": "layer calls launched as programmatic dependents (ARB_ATTN_OVERLAP_PREVIOUS)"
                    if overlap else "none: every call waits for the one before it",
                    "parallelism": f"dp{world} by sequence, no collective"},
-        "pct_of_nominal_8TBs": round(100 * value / world / NOMINAL_HBM_GBS, 2),
+        "pct_of_nominal_8TBs_per_gpu": round(100 * value / world / NOMINAL_HBM_GBS, 2),
         "gpu_launches": per_step * args.steps,
         "device_status_bits": status_bits,
         "clocks": clk.summary(),

@@ -92,8 +92,11 @@ typedef struct {
  * before its first write (out, workspace).  Results are the same as without the flag.  Typical
  * use: the per-layer calls of one decode token when q and the KV cache of every layer are ready.
  * Do not set it when the preceding kernel produces q, appends K/V or changes seq_lens.
+ * ARB_ATTN_NO_TENSOR_CORES: run decode and step chunks on the CUDA-core kernels even where the
+ * tensor-core kernels apply (bf16, head_dim 128).  Same results within the stated tolerances; for
+ * comparison runs and for keeping both paths under test.
  */
-enum { ARB_ATTN_OVERLAP_PREVIOUS = 1u };
+enum { ARB_ATTN_OVERLAP_PREVIOUS = 1u, ARB_ATTN_NO_TENSOR_CORES = 2u };
 
 /*
  * Create a context on `device`.  workspace_bytes = 0 picks a default that covers every shape the

@@ -25,6 +25,7 @@ ARB_ERR_STATIC_LIMIT = 6
 ARB_F32, ARB_BF16 = 0, 1
 DEV_BAD_SEQ_LEN, DEV_BAD_PAGE, DEV_ROLLBACK_UNDERFLOW, DEV_WAIT_TIMEOUT = 1, 2, 4, 8
 ATTN_OVERLAP_PREVIOUS = 1
+ATTN_NO_TENSOR_CORES = 2
 
 # every symbol include/arb.h declares
 EXPORTS = ("arb_create", "arb_destroy", "arb_attn_workspace_bytes", "arb_attn", "arb_attn_host",

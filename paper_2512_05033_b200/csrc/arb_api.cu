@@ -25,7 +25,7 @@ arb_status check_params(const arb_attn_params *p) {
     if (p->batch > kMaxBatch) return ARB_ERR_UNSUPPORTED;
     if ((long long)p->batch * p->num_kv_heads > kCounters) return ARB_ERR_UNSUPPORTED;
     if ((long long)p->max_pages_per_seq * kPage > (1ll << 30)) return ARB_ERR_UNSUPPORTED;
-    if (p->flags & ~(uint32_t)ARB_ATTN_OVERLAP_PREVIOUS) return ARB_ERR_INVALID_ARG;
+    if (p->flags & ~(uint32_t)(ARB_ATTN_OVERLAP_PREVIOUS | ARB_ATTN_NO_TENSOR_CORES)) return ARB_ERR_INVALID_ARG;
     return ARB_OK;
 }
 
@@ -114,8 +114,12 @@ arb_status arb_attn(arb_ctx *ctx, const arb_attn_params *params, const void *q, 
     // q_len == 1 rows: the split-KV decode kernel.  It is launched whenever decode rows may exist
     // (the host knows only the total and the maximum of q_lens).
     const bool maybe_decode = params->max_q_len == 1 || params->total_q > params->max_q_len;
+    const bool tensor_cores = (params->flags & ARB_ATTN_NO_TENSOR_CORES) == 0;
     if (maybe_decode) {
-        st = launch_decode(c, *params, q, k_pages, v_pages, block_table, seq_lens, q_lens, out, s);
+        if (tensor_cores && decode_mma_supported(*params))
+            st = launch_decode_mma(c, *params, q, k_pages, v_pages, block_table, seq_lens, q_lens, out, s);
+        else
+            st = launch_decode(c, *params, q, k_pages, v_pages, block_table, seq_lens, q_lens, out, s);
         if (st != ARB_OK) return st;
     }
     if (params->max_q_len >= 2) {
@@ -123,7 +127,7 @@ arb_status arb_attn(arb_ctx *ctx, const arb_attn_params *params, const void *q, 
         // contraction and goes to the tcgen05 kernel; the rest, and every fp32 chunk, to the
         // CUDA-core kernel.  Both kernels decide per sequence on the device.
         int skip_rows = 0;
-        if (chunk_mma_supported(*params)) {
+        if (tensor_cores && chunk_mma_supported(*params)) {
             st = launch_chunk_mma(c, *params, q, k_pages, v_pages, block_table, seq_lens, q_lens, out, s);
             if (st != ARB_OK) return st;
             skip_rows = kChunkMmaMinRows;

@@ -13,6 +13,7 @@ constexpr int kPage = 16;             // tokens per KV page
 constexpr int kMaxBatch = 1024;       // sequences per call (prefix tables live in shared memory)
 constexpr int kMaxGroup = 8;          // query heads per KV head
 constexpr int kChunkMmaMinRows = 64;  // q_len * group from which a chunk goes to the tensor cores
+constexpr int kDecodeMmaMinGroup = 1; // group size from which bf16 / head_dim 128 decode uses warp-level MMA
 constexpr long long kWaitCycles = 1ll << 31;  // bound of every mbarrier wait (about a second)
 
 // ---------------------------------------------------------------------------------------------
@@ -171,6 +172,10 @@ arb_status launch_chunk_fma(Ctx *ctx, const arb_attn_params &p, const void *q, c
                             const int32_t *q_lens, void *out, int n_lo, int n_hi, int skip_rows,
                             cudaStream_t stream);
 bool chunk_mma_supported(const arb_attn_params &p);
+bool decode_mma_supported(const arb_attn_params &p);
+arb_status launch_decode_mma(Ctx *ctx, const arb_attn_params &p, const void *q, const void *k_pages,
+                             const void *v_pages, const int32_t *block_table, const int32_t *seq_lens,
+                             const int32_t *q_lens, void *out, cudaStream_t stream);
 arb_status launch_chunk_mma(Ctx *ctx, const arb_attn_params &p, const void *q, const void *k_pages,
                             const void *v_pages, const int32_t *block_table, const int32_t *seq_lens,
                             const int32_t *q_lens, void *out, cudaStream_t stream);

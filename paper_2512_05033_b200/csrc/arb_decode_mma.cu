@@ -1,0 +1,728 @@
+// Split-KV decode attention (q_len = 1), bf16, head_dim 128: the group's query heads are padded to
+// the 16 rows of a warp-level tensor-core tile.
+//
+// Why tensor cores for a bandwidth-bound kernel: with CUDA-core FMAs a decode launch of the
+// draft-shaped workload (group size 6) executes 6.3 M warp instructions for 34 MB of KV, 10.7 k issue
+// slots per SM sub-partition, i.e. 5.4 us at one instruction per cycle -- as long as the 5.3 us the
+// bytes need at HBM speed.  The FMA form is issue-bound there.  Here one page (16 keys) costs a warp
+// 8 ldmatrix + 16 mma for q.K and the same for P.V, about a tenth of the instructions, so the kernel
+// goes back to being bound by memory and latency.  The rows 8..15 of the tile stay zero (g <= 8).
+//
+// Everything around the arithmetic is the scheme of the CUDA-core decode kernel: flat page list cut
+// into equal ranges per CTA, one producer warp feeding a 16-stage ring, page groups owned by one
+// consumer warp each with its own online softmax, last-arriver split combine staged through the idle
+// ring.  Differences: K/V tiles arrive as tiled TMA boxes (16 rows x 64 dims, 128-byte swizzle, two
+// per tile) so that ldmatrix reads them without bank conflicts; P is rounded to bf16 for the second
+// product (and summed after rounding, so numerator and denominator agree); results of a segment are
+// parked in shared memory and written out after the CTA's last page, so the wait for the previous
+// kernel (programmatic dependent launch) comes once, after all streaming.
+#include <cuda.h>  // CUtensorMap and its enums only; the encoder is looked up at run time
+
+#include "arb_common.cuh"
+
+namespace arb {
+
+namespace {
+
+constexpr int kD = 128;
+constexpr int kConsWarps = 4;
+constexpr int kConsThreads = kConsWarps * 32;
+constexpr int kThreads = kConsThreads + 32;
+constexpr int kGroup = 2;       // pages per consumer work group
+constexpr int kStages = 16;     // ring stages of one 4 KB tile each
+constexpr int kBatch = 16;      // producer lanes issuing side by side
+constexpr int kTileBytes = kPage * kD * 2;
+constexpr int kHalfTile = kTileBytes / 2;   // one TMA box: 16 rows x 64 bf16
+constexpr int kRingBytes = kStages * kTileBytes;
+constexpr int kMinChunk = 4;
+constexpr int kCtasPerSm = 2;
+constexpr int kParked = 2;      // segment results parked in shared memory before they are written
+static_assert(kStages % (kConsWarps * 2 * kGroup) == 0, "a ring stage must always belong to the same warp");
+
+struct Args {
+    const char *q;
+    const int32_t *block_table;
+    const int32_t *seq_lens;
+    const int32_t *q_lens;
+    char *out;
+    float *part_o;    // [slots][G][D]
+    float *part_ml;   // [slots][GP][2]
+    int *counters;
+    uint32_t *status;
+    int batch, Hq, Hkv, num_pages, max_pages;
+    float scale_log2;
+};
+
+struct Tail {
+    uint64_t full[kStages];
+    uint64_t empty[kStages];
+    uint64_t cbar[2];
+    float lsum[kMaxGroup];
+    int abort;
+    int flags[kParked];   // per parked segment: this CTA was the last to arrive
+};
+
+struct Parked {  // host-side view of what a parked segment needs besides its record
+    int bk, nparts, c_first;
+    size_t out_base;
+};
+
+template <int G>
+struct Cfg {
+    static constexpr int GP = (G + 3) / 4 * 4;
+    static constexpr int REC = G * kD + 2 * GP;            // [m[GP] | l[GP] | o[G][D]]
+    static constexpr int OSM_BYTES = kConsWarps * REC * 4;
+    static constexpr int PARK_BYTES = kParked * REC * 4;
+};
+
+template <int G>
+size_t smem_bytes(int batch) {
+    using C = Cfg<G>;
+    return 1024 + kRingBytes + C::OSM_BYTES + C::PARK_BYTES + sizeof(Tail) + sizeof(int) * (3 * (size_t)batch + 2);
+}
+
+struct Segment {
+    int b, kvh, pg0, pg1, L, bk, nparts, c_first;
+};
+
+__device__ __forceinline__ bool next_segment(int &cur, int r1, const int *pref, const int *slen, int B, int Hkv,
+                                             int chunk, Segment &s) {
+    if (cur >= r1) return false;
+    int lo = 0, hi = B;
+    while (hi - lo > 1) {
+        const int mid = (lo + hi) >> 1;
+        if (pref[mid] <= cur) lo = mid; else hi = mid;
+    }
+    const int b = lo;
+    const int pages = (pref[b + 1] - pref[b]) / Hkv;
+    const int r = cur - pref[b];
+    const int kvh = r / pages;
+    const int pg0 = r - kvh * pages;
+    const int s0 = pref[b] + kvh * pages;
+    const int s1 = s0 + pages;
+    const int end = s1 < r1 ? s1 : r1;
+    s.b = b;
+    s.kvh = kvh;
+    s.pg0 = pg0;
+    s.pg1 = pg0 + (end - cur);
+    s.L = slen[b];
+    s.bk = b * Hkv + kvh;
+    s.c_first = s0 / chunk;
+    s.nparts = (s1 - 1) / chunk - s.c_first + 1;
+    cur = end;
+    return true;
+}
+
+__device__ __forceinline__ void fence_proxy_async_all() { asm volatile("fence.proxy.async;" ::: "memory"); }
+__device__ __forceinline__ void let_successor_start() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void wait_for_predecessor() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
+__device__ __forceinline__ void tma_box_load(void *dst_smem, const CUtensorMap *map, int x, int y, uint64_t *bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+        ::"r"(smem_u32(dst_smem)), "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(smem_u32(bar))
+        : "memory");
+}
+
+// four 8x8 bf16 blocks; lanes 8i..8i+7 give the row addresses of block i
+__device__ __forceinline__ void ldmatrix_x4(uint32_t addr, uint32_t (&r)[4]) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0, %1, %2, %3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
+                 : "r"(addr));
+}
+__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t addr, uint32_t (&r)[4]) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0, %1, %2, %3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
+                 : "r"(addr));
+}
+// D(16x8, fp32) += A(16x16, bf16, row) * B(16x8, bf16, col)
+__device__ __forceinline__ void mma_16816(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+    asm volatile(
+        "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, "
+        "{%0, %1, %2, %3};"
+        : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+        : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+    uint32_t r;
+    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+    return r;
+}
+
+// byte offset of 16-byte chunk `c` (0..15 across the 256-byte row) of row `r` inside a swizzled tile
+__device__ __forceinline__ uint32_t tile_off(int r, int c) {
+    return (uint32_t)((c >> 3) * kHalfTile + r * 128 + (((c & 7) ^ (r & 7)) << 4));
+}
+
+template <int G>
+__global__ void __launch_bounds__(kThreads, kCtasPerSm)
+decode_mma_kernel(const Args a, const __grid_constant__ CUtensorMap k_map, const __grid_constant__ CUtensorMap v_map) {
+    using C = Cfg<G>;
+    constexpr int GP = C::GP, REC = C::REC;
+    static_assert(G >= 1 && G <= 8, "query heads of a group occupy rows 0..7 of the 16-row tile");
+
+    extern __shared__ char smem_raw[];
+    char *base = reinterpret_cast<char *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    char *ring = base;
+    float *osm = reinterpret_cast<float *>(base + kRingBytes);
+    float *park = reinterpret_cast<float *>(base + kRingBytes + C::OSM_BYTES);
+    Tail *tail = reinterpret_cast<Tail *>(base + kRingBytes + C::OSM_BYTES + C::PARK_BYTES);
+    int *pref = reinterpret_cast<int *>(tail + 1);
+    int *row0 = pref + a.batch + 1;
+    int *slen = row0 + a.batch + 1;
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int B = a.batch, Hkv = a.Hkv;
+
+    // Until wait_for_predecessor() only inputs are read; every write to out, the workspace or the
+    // arrival counters comes after it (see the CUDA-core decode kernel for the ordering argument).
+    let_successor_start();
+
+    if (tid == 0) {
+        for (int s = 0; s < kStages; ++s) {
+            mbar_init(&tail->full[s], 1);
+            mbar_init(&tail->empty[s], 1);
+        }
+        mbar_init(&tail->cbar[0], 1);
+        mbar_init(&tail->cbar[1], 1);
+        tail->abort = 0;
+        mbar_fence_init();
+        pref[0] = 0;
+        row0[0] = 0;
+    }
+    for (int b = tid; b < B; b += kThreads) {
+        const int n = a.q_lens[b], L = a.seq_lens[b];
+        int pages = 0;
+        if (n == 1) {
+            if (L >= 1 && L <= a.max_pages * kPage) {
+                pages = (L + kPage - 1) / kPage;
+            } else if (blockIdx.x == 0) {
+                wait_for_predecessor();
+                atomicOr(a.status, (uint32_t)ARB_DEV_BAD_SEQ_LEN);
+                int row = 0;
+                for (int i = 0; i < b; ++i) row += max(a.q_lens[i], 0);
+                __nv_bfloat16 *o = reinterpret_cast<__nv_bfloat16 *>(a.out) + (size_t)row * a.Hq * kD;
+                for (int i = 0; i < a.Hq * kD; ++i) o[i] = __float2bfloat16_rn(0.f);
+            }
+        }
+        pref[b + 1] = pages * Hkv;
+        row0[b + 1] = n > 0 ? n : 0;
+        slen[b] = L;
+    }
+    __syncthreads();
+    if (warp == 0) {
+        int carry_p = 0, carry_r = 0;
+        for (int b0 = 0; b0 < B; b0 += 32) {
+            const int b = b0 + lane;
+            int vp = b < B ? pref[b + 1] : 0;
+            int vr = b < B ? row0[b + 1] : 0;
+#pragma unroll
+            for (int off = 1; off < 32; off <<= 1) {
+                const int tp = __shfl_up_sync(0xffffffffu, vp, off);
+                const int tr = __shfl_up_sync(0xffffffffu, vr, off);
+                if (lane >= off) { vp += tp; vr += tr; }
+            }
+            if (b < B) { pref[b + 1] = vp + carry_p; row0[b + 1] = vr + carry_r; }
+            carry_p += __shfl_sync(0xffffffffu, vp, 31);
+            carry_r += __shfl_sync(0xffffffffu, vr, 31);
+        }
+    }
+    __syncthreads();
+
+    const int total = pref[B];
+    int chunk = (total + (int)gridDim.x - 1) / (int)gridDim.x;
+    if (chunk < kMinChunk) chunk = kMinChunk;
+    const long long r0l = (long long)blockIdx.x * chunk;
+    if (r0l >= total) return;
+    const int r0 = (int)r0l;
+    const int r1 = min(total, r0 + chunk);
+    volatile int *abort = &tail->abort;
+
+    if (warp == kConsWarps) {
+        // ================================ producer warp ==========================================
+        uint32_t c = 0;
+        int cur = r0;
+        Segment s;
+        while (next_segment(cur, r1, pref, slen, B, Hkv, chunk, s)) {
+            for (int sp0 = s.pg0; sp0 < s.pg1; sp0 += 32) {
+                const int np = min(32, s.pg1 - sp0);
+                int pid = 0;
+                if (lane < np) {
+                    pid = a.block_table[(size_t)s.b * a.max_pages + sp0 + lane];
+                    if ((unsigned)pid >= (unsigned)a.num_pages) {
+                        atomicOr(a.status, (uint32_t)ARB_DEV_BAD_PAGE);
+                        pid = 0;
+                    }
+                }
+                const int full_tiles = (np / kGroup) * 2 * kGroup;
+                const int rem = np % kGroup;
+                const int ntiles = 2 * np;
+#pragma unroll 1
+                for (int i0 = 0; i0 < ntiles; i0 += kBatch) {
+                    const int i = i0 + lane;
+                    int page, is_v;
+                    if (i < full_tiles) {
+                        const int g = i / (2 * kGroup), r = i - g * 2 * kGroup;
+                        is_v = r / kGroup;
+                        page = g * kGroup + (r - is_v * kGroup);
+                    } else {
+                        const int r = i - full_tiles, d = rem > 0 ? rem : 1;
+                        is_v = r / d;
+                        page = (np / kGroup) * kGroup + (r - is_v * d);
+                    }
+                    const int pg = __shfl_sync(0xffffffffu, pid, page & 31);
+                    if (lane < kBatch && i < ntiles) {
+                        const uint32_t cc = c + i, st = cc % kStages, par = (cc / kStages) & 1u;
+                        const CUtensorMap *map = is_v ? &v_map : &k_map;
+                        if (mbar_wait(&tail->empty[st], par ^ 1u, abort, a.status)) {
+                            mbar_arrive_expect_tx(&tail->full[st], kTileBytes);
+                            const int row = (pg * Hkv + s.kvh) * kPage;
+                            tma_box_load(ring + st * kTileBytes, map, 0, row, &tail->full[st]);
+                            tma_box_load(ring + st * kTileBytes + kHalfTile, map, 64, row, &tail->full[st]);
+                        }
+                    }
+                    __syncwarp();
+                }
+                c += ntiles;
+            }
+        }
+        if (lane == 0 && *abort) {
+            const uint32_t n = c < (uint32_t)kStages ? c : (uint32_t)kStages;
+            for (uint32_t i = 0; i < n; ++i) {
+                const uint32_t cc = c - 1 - i;
+                const long long t0 = clock64();
+                while (!mbar_try_wait(&tail->full[cc % kStages], (cc / kStages) & 1u) && clock64() - t0 < (1ll << 24)) {
+                }
+            }
+        }
+        return;
+    }
+
+    // ==================================== consumer warps ==========================================
+    const int gq = lane >> 2, tq = lane & 3;   // fragment coordinates: row / column pair
+    const bool row_ok = gq < G;                // this lane's row is a real query head
+    const uint32_t ring_addr = smem_u32(ring);
+    uint32_t seg_base = 0;
+    int cur = r0;
+    Segment s;
+    int n_parked = 0;
+    Parked pk[kParked];
+    int pend_n = 0;
+    int pend_slot0[2], pend_parts[2];
+    size_t pend_out[2];
+
+    // writes the parked segment results; returns after the arrival counters have been updated
+    auto flush = [&]() {
+        wait_for_predecessor();
+        bool any_multi = false;
+        for (int j = 0; j < n_parked; ++j) {
+            const float *rec = park + j * REC;
+            const size_t slot = (size_t)pk[j].bk + blockIdx.x;
+            for (int idx = tid; idx < G * kD; idx += kConsThreads) {
+                const int h = idx / kD;
+                if (pk[j].nparts == 1) {
+                    reinterpret_cast<__nv_bfloat16 *>(a.out)[pk[j].out_base + idx] =
+                        __float2bfloat16_rn(rec[2 * GP + idx] / rec[GP + h]);
+                } else {
+                    a.part_o[slot * G * kD + idx] = rec[2 * GP + idx];
+                    if (idx - h * kD == 0) {
+                        a.part_ml[(slot * GP + h) * 2 + 0] = rec[h];
+                        a.part_ml[(slot * GP + h) * 2 + 1] = rec[GP + h];
+                    }
+                }
+            }
+            any_multi |= pk[j].nparts > 1;
+        }
+        if (any_multi) {
+            fence_proxy_async_all();         // the partials are read back through bulk copies
+            named_barrier(1, kConsThreads);  // the block's stores are ordered before thread 0's fence
+            if (tid == 0) {
+                __threadfence();
+                fence_proxy_async_all();     // the partials are read back through bulk copies
+                for (int j = 0; j < n_parked; ++j) {
+                    int last = 0;
+                    if (pk[j].nparts > 1) {
+                        const int old = atomicAdd(&a.counters[pk[j].bk], 1);
+                        last = (old == pk[j].nparts - 1);
+                        if (last) a.counters[pk[j].bk] = 0;
+                    }
+                    tail->flags[j] = last;
+                }
+            }
+            named_barrier(1, kConsThreads);
+            for (int j = 0; j < n_parked; ++j) {
+                if (pk[j].nparts > 1 && tail->flags[j] && pend_n < 2) {
+                    pend_slot0[pend_n] = pk[j].bk + pk[j].c_first;
+                    pend_parts[pend_n] = pk[j].nparts;
+                    pend_out[pend_n] = pk[j].out_base;
+                    ++pend_n;
+                }
+            }
+        }
+        named_barrier(1, kConsThreads);  // parking slots and flags are free again
+        n_parked = 0;
+    };
+
+    while (next_segment(cur, r1, pref, slen, B, Hkv, chunk, s)) {
+        const int qrow = row0[s.b];
+        // A fragments of q (16 x 128, rows >= G zero): 8 k-slices of 16 dims
+        uint32_t qa[8][4];
+        {
+            const char *qh = a.q + ((size_t)qrow * a.Hq + s.kvh * G + gq) * kD * 2;
+#pragma unroll
+            for (int ks = 0; ks < 8; ++ks) {
+                qa[ks][0] = row_ok ? __ldg(reinterpret_cast<const uint32_t *>(qh + ks * 32 + tq * 4)) : 0u;
+                qa[ks][2] = row_ok ? __ldg(reinterpret_cast<const uint32_t *>(qh + ks * 32 + 16 + tq * 4)) : 0u;
+                qa[ks][1] = 0u;
+                qa[ks][3] = 0u;
+            }
+        }
+        // this lane's row (head gq): running max (the same in the 4 lanes of a row), its share of the
+        // sum, and 16 n-tiles of the output row: o[n][0..1] = dims 8n + 2 tq, + 1 (o[n][2..3]: rows 8..15)
+        float m_run = -INFINITY, l_run = 0.f;
+        float o[16][4];
+#pragma unroll
+        for (int n = 0; n < 16; ++n) { o[n][0] = o[n][1] = o[n][2] = o[n][3] = 0.f; }
+
+        const int seg_pages = s.pg1 - s.pg0;
+        const int ngroups = (seg_pages + kGroup - 1) / kGroup;
+        for (int gi = warp; gi < ngroups; gi += kConsWarps) {
+            const int p0 = s.pg0 + gi * kGroup;
+            const int npg = min(kGroup, s.pg1 - p0);
+            const int ntok = min(s.L - p0 * kPage, npg * kPage);
+            const uint32_t gbase = seg_base + (uint32_t)gi * 2 * kGroup;
+
+            // ---- S = q K^T for the group's pages: per page two n-tiles of 8 keys -----------------
+            float sc[kGroup * 2][4];
+#pragma unroll
+            for (int t = 0; t < kGroup; ++t) {
+#pragma unroll
+                for (int j = 0; j < 2; ++j) { sc[t * 2 + j][0] = sc[t * 2 + j][1] = sc[t * 2 + j][2] = sc[t * 2 + j][3] = 0.f; }
+                if (t < npg) {
+                    const uint32_t cc = gbase + t, st = cc % kStages, par = (cc / kStages) & 1u;
+                    mbar_wait(&tail->full[st], par, abort, a.status);
+                    const uint32_t tile = ring_addr + st * kTileBytes;
+#pragma unroll
+                    for (int j = 0; j < 2; ++j) {          // keys 8j .. 8j+7 of the page
+#pragma unroll
+                        for (int kp = 0; kp < 4; ++kp) {   // k-slices 2kp, 2kp+1
+                            uint32_t bfr[4];
+                            ldmatrix_x4(tile + tile_off(8 * j + (lane & 7), 4 * kp + (lane >> 3)), bfr);
+                            mma_16816(sc[t * 2 + j], qa[2 * kp], bfr[0], bfr[1]);
+                            mma_16816(sc[t * 2 + j], qa[2 * kp + 1], bfr[2], bfr[3]);
+                        }
+                    }
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&tail->empty[st]);
+                }
+            }
+
+            // ---- online softmax on the fragments: this lane has 2 scores per n-tile of its row ------
+            float mx = -INFINITY;
+#pragma unroll
+            for (int nt = 0; nt < kGroup * 2; ++nt) {
+#pragma unroll
+                for (int e = 0; e < 2; ++e) {
+                    const int key = nt * 8 + tq * 2 + e;
+                    const float v = (key < ntok) ? sc[nt][e] * a.scale_log2 : -INFINITY;
+                    sc[nt][e] = v;
+                    mx = fmaxf(mx, v);
+                }
+            }
+            mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
+            mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
+            const float m_new = fmaxf(m_run, mx);            // finite: the group has a visible key
+            const float f = fast_exp2(m_run - m_new);        // 0 for the first group
+            m_run = m_new;
+            uint32_t pa[kGroup][4];                          // A fragments of P: one k-slice per page
+            float lsum = 0.f;
+#pragma unroll
+            for (int t = 0; t < kGroup; ++t) {
+                const float p00 = fast_exp2(sc[2 * t][0] - m_new), p01 = fast_exp2(sc[2 * t][1] - m_new);
+                const float p10 = fast_exp2(sc[2 * t + 1][0] - m_new), p11 = fast_exp2(sc[2 * t + 1][1] - m_new);
+                const uint32_t w0 = pack_bf16(p00, p01), w1 = pack_bf16(p10, p11);
+                pa[t][0] = w0;   // row gq, keys 2 tq, +1
+                pa[t][2] = w1;   // row gq, keys 8 + 2 tq, +1
+                pa[t][1] = 0u;   // rows 8..15
+                pa[t][3] = 0u;
+                // the sum uses the rounded weights, like the tensor core
+                lsum += __uint_as_float(w0 << 16) + __uint_as_float(w0 & 0xffff0000u) +
+                        __uint_as_float(w1 << 16) + __uint_as_float(w1 & 0xffff0000u);
+            }
+            l_run = fmaf(l_run, f, lsum);
+            if (__any_sync(0xffffffffu, f != 1.0f)) {
+#pragma unroll
+                for (int n = 0; n < 16; ++n) { o[n][0] *= f; o[n][1] *= f; }
+            }
+
+            // ---- O += P V: per page 16 n-tiles of 8 dims, one k-slice of 16 keys ------------------
+#pragma unroll
+            for (int t = 0; t < kGroup; ++t) {
+                if (t < npg) {
+                    const uint32_t cc = gbase + npg + t, st = cc % kStages, par = (cc / kStages) & 1u;
+                    mbar_wait(&tail->full[st], par, abort, a.status);
+                    const uint32_t tile = ring_addr + st * kTileBytes;
+                    const int nvalid = ntok - t * kPage;
+                    if (nvalid < kPage) {
+                        // slots past the sequence end may hold anything; they must not reach the
+                        // tensor core, not even times zero: blank them in shared memory
+                        for (int i = lane; i < (kPage - nvalid) * 16; i += 32) {
+                            const int r = nvalid + (i >> 4), c = i & 15;
+                            *reinterpret_cast<uint4 *>(ring + st * kTileBytes + tile_off(r, c)) = make_uint4(0, 0, 0, 0);
+                        }
+                        __syncwarp();
+                    }
+#pragma unroll
+                    for (int np2 = 0; np2 < 8; ++np2) {    // dims 16 np2 .. 16 np2 + 15
+                        uint32_t bfr[4];
+                        // blocks: (keys 0-7, chunk 2np2), (keys 8-15, 2np2), (keys 0-7, 2np2+1), (keys 8-15, 2np2+1)
+                        ldmatrix_x4_trans(tile + tile_off((lane & 7) + ((lane >> 3) & 1) * 8, 2 * np2 + (lane >> 4)), bfr);
+                        mma_16816(o[2 * np2], pa[t], bfr[0], bfr[1]);
+                        mma_16816(o[2 * np2 + 1], pa[t], bfr[2], bfr[3]);
+                    }
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&tail->empty[st]);
+                }
+            }
+        }
+        seg_base += 2u * (uint32_t)seg_pages;
+
+        // ---- segment end: every warp leaves (max, sum, row accumulators); all threads merge them ------
+        l_run += __shfl_xor_sync(0xffffffffu, l_run, 1);
+        l_run += __shfl_xor_sync(0xffffffffu, l_run, 2);
+        float *rec = osm + warp * REC;
+        if (row_ok) {
+#pragma unroll
+            for (int n = 0; n < 16; ++n)
+                *reinterpret_cast<float2 *>(rec + 2 * GP + gq * kD + 8 * n + tq * 2) = make_float2(o[n][0], o[n][1]);
+            if (tq == 0) { rec[gq] = m_run; rec[GP + gq] = l_run; }
+        }
+        if (n_parked == kParked) flush();  // uniform across the consumer threads
+        named_barrier(1, kConsThreads);
+        float *dst = park + n_parked * REC;
+        for (int idx = tid; idx < G * kD; idx += kConsThreads) {
+            const int h = idx / kD;
+            float M = -INFINITY;
+#pragma unroll
+            for (int w = 0; w < kConsWarps; ++w) M = fmaxf(M, osm[w * REC + h]);
+            float l = 0.f, acc = 0.f;
+#pragma unroll
+            for (int w = 0; w < kConsWarps; ++w) {
+                const float ff = fast_exp2(osm[w * REC + h] - M);  // 0 for a warp that had no group
+                l = fmaf(ff, osm[w * REC + GP + h], l);
+                acc = fmaf(ff, osm[w * REC + 2 * GP + idx], acc);
+            }
+            dst[2 * GP + idx] = acc;
+            if (idx - h * kD == 0) { dst[h] = M; dst[GP + h] = l; }
+        }
+        pk[n_parked].bk = s.bk;
+        pk[n_parked].nparts = s.nparts;
+        pk[n_parked].c_first = s.c_first;
+        pk[n_parked].out_base = ((size_t)qrow * a.Hq + s.kvh * G) * kD;
+        ++n_parked;
+        named_barrier(1, kConsThreads);  // warp records are free for the next segment
+    }
+    if (n_parked > 0) flush();
+
+    // ---- split combine of the (sequence, kv head)s this CTA was the last to reach -----------------
+    // The ring is idle: [ max/sum records of all parts | buffer A | buffer B ].
+    uint32_t cph[2] = {0u, 0u};
+    for (int j = 0; j < pend_n; ++j) {
+        const int nparts = pend_parts[j];
+        const size_t slot0 = (size_t)pend_slot0[j];
+        __threadfence();
+        const uint32_t ml_bytes = (uint32_t)nparts * GP * 8u;
+        const uint32_t ml_area = (ml_bytes + 127u) & ~127u;
+        constexpr int PART_BYTES = G * kD * 4;
+        float *ml = reinterpret_cast<float *>(ring);
+        const int per_piece = ((kRingBytes - (int)ml_area) / 2) / PART_BYTES;
+        if (per_piece < 1) {
+            for (int idx = tid; idx < G * kD; idx += kConsThreads) {
+                const int h = idx / kD;
+                float m = -INFINITY;
+                for (int p = 0; p < nparts; ++p) m = fmaxf(m, __ldcg(&a.part_ml[((slot0 + p) * GP + h) * 2]));
+                float l = 0.f, x = 0.f;
+                for (int p = 0; p < nparts; ++p) {
+                    const float w = fast_exp2(__ldcg(&a.part_ml[((slot0 + p) * GP + h) * 2]) - m);
+                    l = fmaf(w, __ldcg(&a.part_ml[((slot0 + p) * GP + h) * 2 + 1]), l);
+                    x = fmaf(w, __ldcg(&a.part_o[(slot0 + p) * G * kD + idx]), x);
+                }
+                reinterpret_cast<__nv_bfloat16 *>(a.out)[pend_out[j] + idx] = __float2bfloat16_rn(x / l);
+            }
+            continue;
+        }
+        float *buf[2] = {reinterpret_cast<float *>(ring + ml_area),
+                         reinterpret_cast<float *>(ring + ml_area + per_piece * PART_BYTES)};
+        const int npieces = (nparts + per_piece - 1) / per_piece;
+        auto issue_piece = [&](int i, uint32_t extra) {
+            const int pp0 = i * per_piece, np = min(per_piece, nparts - pp0);
+            const uint32_t bytes = (uint32_t)np * PART_BYTES;
+            mbar_arrive_expect_tx(&tail->cbar[i & 1], bytes + extra);
+            bulk_load(buf[i & 1], a.part_o + (slot0 + pp0) * G * kD, bytes, &tail->cbar[i & 1]);
+        };
+        if (tid == 0) {
+            fence_proxy_async_all();
+            issue_piece(0, ml_bytes);
+            bulk_load(ml, a.part_ml + slot0 * GP * 2, ml_bytes, &tail->cbar[0]);
+            if (npieces > 1) issue_piece(1, 0u);
+        }
+        mbar_wait(&tail->cbar[0], cph[0], abort, a.status);
+        cph[0] ^= 1u;
+        for (int h = warp; h < G; h += kConsWarps) {
+            float m = -INFINITY;
+            for (int p = lane; p < nparts; p += 32) m = fmaxf(m, ml[(p * GP + h) * 2]);
+#pragma unroll
+            for (int off = 16; off >= 1; off >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, off));
+            float l = 0.f;
+            for (int p = lane; p < nparts; p += 32) {
+                const float w = fast_exp2(ml[(p * GP + h) * 2] - m);
+                ml[(p * GP + h) * 2] = w;
+                l = fmaf(w, ml[(p * GP + h) * 2 + 1], l);
+            }
+#pragma unroll
+            for (int off = 16; off >= 1; off >>= 1) l += __shfl_xor_sync(0xffffffffu, l, off);
+            if (lane == 0) tail->lsum[h] = l;
+        }
+        named_barrier(1, kConsThreads);
+        constexpr int NK = (G * kD + kConsThreads - 1) / kConsThreads;
+        float acc[NK];
+        int hk[NK];
+#pragma unroll
+        for (int k = 0; k < NK; ++k) {
+            const int idx = tid + k * kConsThreads;
+            hk[k] = idx < G * kD ? idx / kD : 0;
+            acc[k] = 0.f;
+        }
+        for (int i = 0; i < npieces; ++i) {
+            const int pp0 = i * per_piece, np = min(per_piece, nparts - pp0);
+            if (i > 0) {
+                mbar_wait(&tail->cbar[i & 1], cph[i & 1], abort, a.status);
+                cph[i & 1] ^= 1u;
+            }
+            const float *po = buf[i & 1];
+#pragma unroll 2
+            for (int p = 0; p < np; ++p) {
+#pragma unroll
+                for (int k = 0; k < NK; ++k) {
+                    const int idx = tid + k * kConsThreads;
+                    if (idx < G * kD) acc[k] = fmaf(ml[((pp0 + p) * GP + hk[k]) * 2], po[p * G * kD + idx], acc[k]);
+                }
+            }
+            named_barrier(1, kConsThreads);
+            if (tid == 0 && i + 2 < npieces) issue_piece(i + 2, 0u);
+        }
+#pragma unroll
+        for (int k = 0; k < NK; ++k) {
+            const int idx = tid + k * kConsThreads;
+            if (idx < G * kD)
+                reinterpret_cast<__nv_bfloat16 *>(a.out)[pend_out[j] + idx] = __float2bfloat16_rn(acc[k] / tail->lsum[hk[k]]);
+        }
+        named_barrier(1, kConsThreads);
+    }
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_tiled_fn() {
+    static EncodeTiledFn fn = nullptr;
+    static bool tried = false;
+    if (!tried) {
+        tried = true;
+        void *p = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) == cudaSuccess &&
+            qres == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(p);
+        cudaGetLastError();
+    }
+    return fn;
+}
+
+bool make_pool_map(CUtensorMap *map, const void *pool, const arb_attn_params &p) {
+    EncodeTiledFn fn = encode_tiled_fn();
+    if (!fn) return false;
+    const cuuint64_t dims[2] = {(cuuint64_t)kD, (cuuint64_t)p.num_pages * p.num_kv_heads * kPage};
+    const cuuint64_t strides[1] = {(cuuint64_t)kD * 2};
+    const cuuint32_t box[2] = {64, (cuuint32_t)kPage};
+    const cuuint32_t estr[2] = {1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(pool), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+template <int G>
+arb_status launch_one(Ctx *ctx, const Args &a, const CUtensorMap &km, const CUtensorMap &vm, bool overlap,
+                      cudaStream_t stream) {
+    const size_t smem = smem_bytes<G>(a.batch);
+    static bool attr_set[64] = {};
+    if (!attr_set[ctx->device & 63]) {
+        if (cudaFuncSetAttribute(decode_mma_kernel<G>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 (int)smem_bytes<G>(kMaxBatch)) != cudaSuccess)
+            return ARB_ERR_CUDA;
+        attr_set[ctx->device & 63] = true;
+    }
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(ctx->num_sms * kCtasPerSm);
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = overlap ? 1 : 0;
+    const cudaError_t err = cudaLaunchKernelEx(&cfg, decode_mma_kernel<G>, a, km, vm);
+    ctx->launches++;
+    return err == cudaSuccess ? ARB_OK : ARB_ERR_CUDA;
+}
+
+}  // namespace
+
+bool decode_mma_supported(const arb_attn_params &p) {
+    const int g = p.num_q_heads / p.num_kv_heads;
+    return p.dtype == ARB_BF16 && p.head_dim == kD && g >= kDecodeMmaMinGroup && g <= 8 && encode_tiled_fn() != nullptr;
+}
+
+arb_status launch_decode_mma(Ctx *ctx, const arb_attn_params &p, const void *q, const void *k_pages,
+                             const void *v_pages, const int32_t *block_table, const int32_t *seq_lens,
+                             const int32_t *q_lens, void *out, cudaStream_t stream) {
+    alignas(64) CUtensorMap km, vm;
+    if (!make_pool_map(&km, k_pages, p) || !make_pool_map(&vm, v_pages, p)) return ARB_ERR_CUDA;
+    const int g = p.num_q_heads / p.num_kv_heads;
+    const int gp = (g + 3) / 4 * 4;
+    (void)gp;
+    const size_t slots = (size_t)p.batch * p.num_kv_heads + (size_t)ctx->num_sms * kCtasPerSm;
+    Args a;
+    a.q = static_cast<const char *>(q);
+    a.block_table = block_table;
+    a.seq_lens = seq_lens;
+    a.q_lens = q_lens;
+    a.out = static_cast<char *>(out);
+    a.part_o = reinterpret_cast<float *>(ctx->workspace);
+    a.part_ml = a.part_o + ((slots * g * p.head_dim + 63) & ~size_t(63));
+    a.counters = ctx->counters;
+    a.status = ctx->status;
+    a.batch = p.batch;
+    a.Hq = p.num_q_heads;
+    a.Hkv = p.num_kv_heads;
+    a.num_pages = p.num_pages;
+    a.max_pages = p.max_pages_per_seq;
+    const float scale = p.softmax_scale > 0.f ? p.softmax_scale : 1.0f / sqrtf((float)p.head_dim);
+    a.scale_log2 = scale * 1.4426950408889634f;
+    const bool overlap = (p.flags & ARB_ATTN_OVERLAP_PREVIOUS) != 0;
+    switch (g) {
+        case 1: return launch_one<1>(ctx, a, km, vm, overlap, stream);
+        case 2: return launch_one<2>(ctx, a, km, vm, overlap, stream);
+        case 3: return launch_one<3>(ctx, a, km, vm, overlap, stream);
+        case 4: return launch_one<4>(ctx, a, km, vm, overlap, stream);
+        case 5: return launch_one<5>(ctx, a, km, vm, overlap, stream);
+        case 6: return launch_one<6>(ctx, a, km, vm, overlap, stream);
+        case 7: return launch_one<7>(ctx, a, km, vm, overlap, stream);
+        case 8: return launch_one<8>(ctx, a, km, vm, overlap, stream);
+        default: return ARB_ERR_UNSUPPORTED;
+    }
+}
+
+}  // namespace arb

@@ -15,13 +15,14 @@ def ctx():
     return _ctx
 
 
-def gpu_attn(inp, scale=0.0):
+def gpu_attn(inp, scale=0.0, flags=0):
     """inp: workloads.AttnInputs on the CPU.  Returns (out fp64 numpy, status bits)."""
     d = inp.to("cuda")
     max_q = int(inp.q_lens.max()) if inp.q_lens.numel() else 0
     out = torch.full_like(d.q, float("nan"))
     c = ctx()
-    c.attn(d.q, d.k_pages, d.v_pages, d.block_table, d.seq_lens, d.q_lens, max_q, out=out, softmax_scale=scale)
+    p = c.params_for(d.q, d.k_pages, d.block_table, max_q, scale, flags=flags)
+    c.attn(d.q, d.k_pages, d.v_pages, d.block_table, d.seq_lens, d.q_lens, max_q, out=out, params=p)
     bits = c.poll_status()
     return out.double().cpu().numpy(), bits
 

@@ -43,8 +43,9 @@ def test_static_entry_point_matches_arb_attn_twice_in_a_row():
     for inp in (first, second, first):
         out, ref = _both(binding, ctx, inp)
         assert np.isfinite(out).all()
-        assert np.abs(out - ref).max() <= 1e-2          # same kernel, same order of operations: equal in practice
-        np.testing.assert_array_equal(out, ref)
+        # arb_attn may take the tensor-core decode kernel, the static call always the CUDA-core one
+        assert np.abs(out - ref).max() <= 1e-2
+        assert (np.abs(out - ref) <= 2.0 ** -7 * np.abs(ref) + 3e-3).all()
     ctx.close()
 
 

@@ -37,6 +37,7 @@ constexpr int kRingBytes = kStages * kTileBytes;
 constexpr int kMinChunk = 4;
 constexpr int kCtasPerSm = 2;
 constexpr int kParked = 2;      // segment results parked in shared memory before they are written
+constexpr int kSmallCallPages = 64;   // up to this many pages per SM a call runs one CTA per SM
 static_assert(kStages % (kConsWarps * 2 * kGroup) == 0, "a ring stage must always belong to the same warp");
 
 struct Args {
@@ -229,8 +230,14 @@ decode_mma_kernel(const Args a, const __grid_constant__ CUtensorMap k_map, const
     }
     __syncthreads();
 
+    // Small calls use only the first half of the grid (one CTA per SM); the other CTAs leave at once
+    // and their slots are free for the next call, which -- launched as a programmatic dependent --
+    // then streams its KV while this call is still computing and combining.  Large calls use every
+    // CTA: two per SM keep more bytes in flight.
     const int total = pref[B];
-    int chunk = (total + (int)gridDim.x - 1) / (int)gridDim.x;
+    const int half_grid = ((int)gridDim.x + 1) / 2;
+    const int active = total <= half_grid * kSmallCallPages ? half_grid : (int)gridDim.x;
+    int chunk = (total + active - 1) / active;
     if (chunk < kMinChunk) chunk = kMinChunk;
     const long long r0l = (long long)blockIdx.x * chunk;
     if (r0l >= total) return;

@@ -58,7 +58,7 @@ struct Tail {
     uint64_t full[kStages];
     uint64_t empty[kStages];
     uint64_t cbar[2];
-    float lsum[kMaxGroup];
+    float lsum[2 * kMaxGroup];   // per combine job and head: sum of the weighted sums
     int abort;
     int flags[kParked];   // per parked segment: this CTA was the last to arrive
 };
@@ -532,18 +532,27 @@ decode_mma_kernel(const Args a, const __grid_constant__ CUtensorMap k_map, const
     if (n_parked > 0) flush();
 
     // ---- split combine of the (sequence, kv head)s this CTA was the last to reach -----------------
-    // The ring is idle: [ max/sum records of all parts | buffer A | buffer B ].
-    uint32_t cph[2] = {0u, 0u};
-    for (int j = 0; j < pend_n; ++j) {
-        const int nparts = pend_parts[j];
-        const size_t slot0 = (size_t)pend_slot0[j];
-        __threadfence();
-        const uint32_t ml_bytes = (uint32_t)nparts * GP * 8u;
-        const uint32_t ml_area = (ml_bytes + 127u) & ~127u;
-        constexpr int PART_BYTES = G * kD * 4;
-        float *ml = reinterpret_cast<float *>(ring);
-        const int per_piece = ((kRingBytes - (int)ml_area) / 2) / PART_BYTES;
-        if (per_piece < 1) {
+    // Up to two jobs, worked on side by side.  The ring is idle: each job gets half of it as a landing
+    // buffer for partial outputs (bulk copies, a piece at a time).  While the first pieces are in
+    // flight the warps read the parts' (max, sum) records straight from global memory and turn them
+    // into weights, kept where the warp records and parked segments used to be.
+    if (pend_n == 0) return;
+    constexpr int PART_BYTES = G * kD * 4;
+    constexpr int JOB_BYTES = kRingBytes / 2;
+    constexpr int PER_PIECE = JOB_BYTES / PART_BYTES;
+    constexpr int NK = (G * kD + kConsThreads - 1) / kConsThreads;
+    float *wsm = osm;                                        // [job][part][GP] weights
+    constexpr int WSM_FLOATS = (C::OSM_BYTES + C::PARK_BYTES) / 4;
+    const int wstride = WSM_FLOATS / 2;                      // floats per job
+    bool fits = true;
+    for (int j = 0; j < pend_n; ++j) fits = fits && pend_parts[j] * GP <= wstride;
+    __threadfence();
+    if (!fits) {
+        // more parts than the weight area can describe (one sequence over every CTA of a very large
+        // part): merge straight from global memory
+        for (int j = 0; j < pend_n; ++j) {
+            const int nparts = pend_parts[j];
+            const size_t slot0 = (size_t)pend_slot0[j];
             for (int idx = tid; idx < G * kD; idx += kConsThreads) {
                 const int h = idx / kD;
                 float m = -INFINITY;
@@ -556,75 +565,116 @@ decode_mma_kernel(const Args a, const __grid_constant__ CUtensorMap k_map, const
                 }
                 reinterpret_cast<__nv_bfloat16 *>(a.out)[pend_out[j] + idx] = __float2bfloat16_rn(x / l);
             }
-            continue;
         }
-        float *buf[2] = {reinterpret_cast<float *>(ring + ml_area),
-                         reinterpret_cast<float *>(ring + ml_area + per_piece * PART_BYTES)};
-        const int npieces = (nparts + per_piece - 1) / per_piece;
-        auto issue_piece = [&](int i, uint32_t extra) {
-            const int pp0 = i * per_piece, np = min(per_piece, nparts - pp0);
-            const uint32_t bytes = (uint32_t)np * PART_BYTES;
-            mbar_arrive_expect_tx(&tail->cbar[i & 1], bytes + extra);
-            bulk_load(buf[i & 1], a.part_o + (slot0 + pp0) * G * kD, bytes, &tail->cbar[i & 1]);
-        };
-        if (tid == 0) {
-            fence_proxy_async_all();
-            issue_piece(0, ml_bytes);
-            bulk_load(ml, a.part_ml + slot0 * GP * 2, ml_bytes, &tail->cbar[0]);
-            if (npieces > 1) issue_piece(1, 0u);
-        }
-        mbar_wait(&tail->cbar[0], cph[0], abort, a.status);
-        cph[0] ^= 1u;
+        return;
+    }
+    auto issue_piece = [&](int j, int i) {  // thread 0 only: piece i of job j into the job's buffer
+        const int pp0 = i * PER_PIECE, np = min(PER_PIECE, pend_parts[j] - pp0);
+        const uint32_t bytes = (uint32_t)np * PART_BYTES;
+        mbar_arrive_expect_tx(&tail->cbar[j], bytes);
+        bulk_load(ring + j * JOB_BYTES, a.part_o + ((size_t)pend_slot0[j] + pp0) * G * kD, bytes, &tail->cbar[j]);
+    };
+    if (tid == 0) {
+        fence_proxy_async_all();
+        for (int j = 0; j < pend_n; ++j) issue_piece(j, 0);
+    }
+    // weights: warp w owns heads w, w + 4 of every job; lanes stride over the parts
+    for (int j = 0; j < pend_n; ++j) {
+        const int nparts = pend_parts[j];
+        const float *mlg = a.part_ml + (size_t)pend_slot0[j] * GP * 2;
         for (int h = warp; h < G; h += kConsWarps) {
+            const bool small = nparts <= 128;   // the usual case: this lane's parts fit in registers
+            float mv[4], lv[4];
             float m = -INFINITY;
-            for (int p = lane; p < nparts; p += 32) m = fmaxf(m, ml[(p * GP + h) * 2]);
+            if (small) {
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    const int p = lane + 32 * u;
+                    mv[u] = p < nparts ? __ldcg(&mlg[(p * GP + h) * 2]) : -INFINITY;
+                    lv[u] = p < nparts ? __ldcg(&mlg[(p * GP + h) * 2 + 1]) : 0.f;
+                }
+#pragma unroll
+                for (int u = 0; u < 4; ++u) m = fmaxf(m, mv[u]);
+            } else {
+                for (int p = lane; p < nparts; p += 32) {
+                    const float x = __ldcg(&mlg[(p * GP + h) * 2]);
+                    wsm[j * wstride + p * GP + h] = x;
+                    m = fmaxf(m, x);
+                }
+            }
 #pragma unroll
             for (int off = 16; off >= 1; off >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, off));
             float l = 0.f;
-            for (int p = lane; p < nparts; p += 32) {
-                const float w = fast_exp2(ml[(p * GP + h) * 2] - m);
-                ml[(p * GP + h) * 2] = w;
-                l = fmaf(w, ml[(p * GP + h) * 2 + 1], l);
+            if (small) {
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    const int p = lane + 32 * u;
+                    if (p < nparts) {
+                        const float w = fast_exp2(mv[u] - m);
+                        wsm[j * wstride + p * GP + h] = w;
+                        l = fmaf(w, lv[u], l);
+                    }
+                }
+            } else {
+                for (int p = lane; p < nparts; p += 32) {
+                    const float w = fast_exp2(wsm[j * wstride + p * GP + h] - m);
+                    wsm[j * wstride + p * GP + h] = w;
+                    l = fmaf(w, __ldcg(&mlg[(p * GP + h) * 2 + 1]), l);
+                }
             }
 #pragma unroll
             for (int off = 16; off >= 1; off >>= 1) l += __shfl_xor_sync(0xffffffffu, l, off);
-            if (lane == 0) tail->lsum[h] = l;
+            if (lane == 0) tail->lsum[j * kMaxGroup + h] = l;
         }
-        named_barrier(1, kConsThreads);
-        constexpr int NK = (G * kD + kConsThreads - 1) / kConsThreads;
-        float acc[NK];
-        int hk[NK];
+    }
+    named_barrier(1, kConsThreads);
+    float acc[2][NK];
+    int hk[NK];
 #pragma unroll
-        for (int k = 0; k < NK; ++k) {
-            const int idx = tid + k * kConsThreads;
-            hk[k] = idx < G * kD ? idx / kD : 0;
-            acc[k] = 0.f;
-        }
-        for (int i = 0; i < npieces; ++i) {
-            const int pp0 = i * per_piece, np = min(per_piece, nparts - pp0);
-            if (i > 0) {
-                mbar_wait(&tail->cbar[i & 1], cph[i & 1], abort, a.status);
-                cph[i & 1] ^= 1u;
-            }
-            const float *po = buf[i & 1];
+    for (int k = 0; k < NK; ++k) {
+        const int idx = tid + k * kConsThreads;
+        hk[k] = idx < G * kD ? idx / kD : 0;
+        acc[0][k] = 0.f;
+        acc[1][k] = 0.f;
+    }
+    int max_pieces = 0;
+    for (int j = 0; j < pend_n; ++j) max_pieces = max(max_pieces, (pend_parts[j] + PER_PIECE - 1) / PER_PIECE);
+    for (int i = 0; i < max_pieces; ++i) {
+#pragma unroll
+        for (int j = 0; j < 2; ++j) {
+            if (j < pend_n && i * PER_PIECE < pend_parts[j]) {
+                const int pp0 = i * PER_PIECE, np = min(PER_PIECE, pend_parts[j] - pp0);
+                mbar_wait(&tail->cbar[j], (uint32_t)i & 1u, abort, a.status);
+                const float *po = reinterpret_cast<const float *>(ring + j * JOB_BYTES);
+                const float *wj = wsm + j * wstride + pp0 * GP;
 #pragma unroll 2
-            for (int p = 0; p < np; ++p) {
+                for (int p = 0; p < np; ++p) {
 #pragma unroll
-                for (int k = 0; k < NK; ++k) {
-                    const int idx = tid + k * kConsThreads;
-                    if (idx < G * kD) acc[k] = fmaf(ml[((pp0 + p) * GP + hk[k]) * 2], po[p * G * kD + idx], acc[k]);
+                    for (int k = 0; k < NK; ++k) {
+                        const int idx = tid + k * kConsThreads;
+                        if (idx < G * kD) acc[j][k] = fmaf(wj[p * GP + hk[k]], po[p * G * kD + idx], acc[j][k]);
+                    }
                 }
             }
-            named_barrier(1, kConsThreads);
-            if (tid == 0 && i + 2 < npieces) issue_piece(i + 2, 0u);
         }
+        if (i + 1 < max_pieces) {
+            named_barrier(1, kConsThreads);  // everyone is done with the buffers before they are refilled
+            if (tid == 0)
+                for (int j = 0; j < pend_n; ++j)
+                    if ((i + 1) * PER_PIECE < pend_parts[j]) issue_piece(j, i + 1);
+        }
+    }
 #pragma unroll
-        for (int k = 0; k < NK; ++k) {
-            const int idx = tid + k * kConsThreads;
-            if (idx < G * kD)
-                reinterpret_cast<__nv_bfloat16 *>(a.out)[pend_out[j] + idx] = __float2bfloat16_rn(acc[k] / tail->lsum[hk[k]]);
+    for (int j = 0; j < 2; ++j) {
+        if (j < pend_n) {
+#pragma unroll
+            for (int k = 0; k < NK; ++k) {
+                const int idx = tid + k * kConsThreads;
+                if (idx < G * kD)
+                    reinterpret_cast<__nv_bfloat16 *>(a.out)[pend_out[j] + idx] =
+                        __float2bfloat16_rn(acc[j][k] / tail->lsum[j * kMaxGroup + hk[k]]);
+            }
         }
-        named_barrier(1, kConsThreads);
     }
 }
 

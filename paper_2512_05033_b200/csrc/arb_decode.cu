@@ -620,6 +620,7 @@ __global__ void __launch_bounds__(kThreads, Cfg<T, D, G>::CTAS) decode_kernel(co
             bulk_load(ml, a.part_ml + slot0 * GP * 2, ml_bytes, &tail->cbar[0]);
             if (npieces > 1) issue_piece(1, 0u);
         }
+        __syncwarp();  // warp 0 reconverges before the wait and the weight phase
         mbar_wait(&tail->cbar[0], cph[0], abort, a.status);
         cph[0] ^= 1u;
         // weights: warp w owns heads w, w + 4; the max slot of every record is overwritten by its weight

@@ -538,9 +538,17 @@ decode_mma_kernel(const Args a, const __grid_constant__ CUtensorMap k_map, const
     // into weights, kept where the warp records and parked segments used to be.
     if (pend_n == 0) return;
     constexpr int PART_BYTES = G * kD * 4;
-    constexpr int JOB_BYTES = kRingBytes / 2;
-    constexpr int PER_PIECE = JOB_BYTES / PART_BYTES;
+    constexpr int CAP = kRingBytes / PART_BYTES;   // partial outputs the ring can hold at once
     constexpr int NK = (G * kD + kConsThreads - 1) / kConsThreads;
+    // landing buffers: the whole ring for one job, shared in proportion to their parts for two
+    int per_piece[2] = {CAP, 0}, buf_off[2] = {0, 0};
+    if (pend_n == 2) {
+        const int n0 = pend_parts[0], n1 = pend_parts[1];
+        int c0 = (n0 + n1 <= CAP) ? n0 : max(1, min(CAP - 1, CAP * n0 / (n0 + n1)));
+        per_piece[0] = c0;
+        per_piece[1] = CAP - c0;
+        buf_off[1] = c0 * PART_BYTES;
+    }
     float *wsm = osm;                                        // [job][part][GP] weights
     constexpr int WSM_FLOATS = (C::OSM_BYTES + C::PARK_BYTES) / 4;
     const int wstride = WSM_FLOATS / 2;                      // floats per job
@@ -569,62 +577,100 @@ decode_mma_kernel(const Args a, const __grid_constant__ CUtensorMap k_map, const
         return;
     }
     auto issue_piece = [&](int j, int i) {  // thread 0 only: piece i of job j into the job's buffer
-        const int pp0 = i * PER_PIECE, np = min(PER_PIECE, pend_parts[j] - pp0);
+        const int pp0 = i * per_piece[j], np = min(per_piece[j], pend_parts[j] - pp0);
         const uint32_t bytes = (uint32_t)np * PART_BYTES;
         mbar_arrive_expect_tx(&tail->cbar[j], bytes);
-        bulk_load(ring + j * JOB_BYTES, a.part_o + ((size_t)pend_slot0[j] + pp0) * G * kD, bytes, &tail->cbar[j]);
+        bulk_load(ring + buf_off[j], a.part_o + ((size_t)pend_slot0[j] + pp0) * G * kD, bytes, &tail->cbar[j]);
     };
     if (tid == 0) {
         fence_proxy_async_all();
         for (int j = 0; j < pend_n; ++j) issue_piece(j, 0);
     }
-    // weights: warp w owns heads w, w + 4 of every job; lanes stride over the parts
-    for (int j = 0; j < pend_n; ++j) {
-        const int nparts = pend_parts[j];
-        const float *mlg = a.part_ml + (size_t)pend_slot0[j] * GP * 2;
-        for (int h = warp; h < G; h += kConsWarps) {
-            const bool small = nparts <= 128;   // the usual case: this lane's parts fit in registers
-            float mv[4], lv[4];
-            float m = -INFINITY;
-            if (small) {
+    __syncwarp();  // warp 0 goes on as one: without this its lane 0 ran the next phase apart from the rest (5 us)
+    // weights: warp w owns heads w, w + 4 of every job; lanes stride over the parts.  In the usual
+    // case (at most 128 parts) every load of the warp is issued before the first one is used.
+    constexpr int HPW = (G + kConsWarps - 1) / kConsWarps;   // heads per warp
+    bool small = true;
+    for (int j = 0; j < pend_n; ++j) small = small && pend_parts[j] <= 128;
+    if (small) {
+        // every load first, from clamped (always valid) records, so that all of them are in flight
+        // together; what does not exist is masked afterwards
+        float2 raw[2][HPW][4];
+#pragma unroll
+        for (int j = 0; j < 2; ++j) {
+            const float *mlg = a.part_ml + (size_t)pend_slot0[j < pend_n ? j : 0] * GP * 2;
+            const int nparts = j < pend_n ? pend_parts[j] : 1;
+#pragma unroll
+            for (int hh = 0; hh < HPW; ++hh) {
+                const int hc = min(warp + hh * kConsWarps, G - 1);
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    const int pc = min(lane + 32 * u, nparts - 1);
+                    raw[j][hh][u] = __ldcg(reinterpret_cast<const float2 *>(mlg + (pc * GP + hc) * 2));
+                }
+            }
+        }
+        float mv[2][HPW][4], lv[2][HPW][4];
+#pragma unroll
+        for (int j = 0; j < 2; ++j) {
+            const int nparts = j < pend_n ? pend_parts[j] : 0;
+#pragma unroll
+            for (int hh = 0; hh < HPW; ++hh) {
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    const bool ok = lane + 32 * u < nparts && warp + hh * kConsWarps < G;
+                    mv[j][hh][u] = ok ? raw[j][hh][u].x : -INFINITY;
+                    lv[j][hh][u] = ok ? raw[j][hh][u].y : 0.f;
+                }
+            }
+        }
+#pragma unroll
+        for (int j = 0; j < 2; ++j) {
+            const int nparts = j < pend_n ? pend_parts[j] : 0;
+#pragma unroll
+            for (int hh = 0; hh < HPW; ++hh) {
+                const int h = warp + hh * kConsWarps;
+                float m = fmaxf(fmaxf(mv[j][hh][0], mv[j][hh][1]), fmaxf(mv[j][hh][2], mv[j][hh][3]));
+#pragma unroll
+                for (int off = 16; off >= 1; off >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, off));
+                float l = 0.f;
 #pragma unroll
                 for (int u = 0; u < 4; ++u) {
                     const int p = lane + 32 * u;
-                    mv[u] = p < nparts ? __ldcg(&mlg[(p * GP + h) * 2]) : -INFINITY;
-                    lv[u] = p < nparts ? __ldcg(&mlg[(p * GP + h) * 2 + 1]) : 0.f;
+                    if (p < nparts && h < G) {
+                        const float w = fast_exp2(mv[j][hh][u] - m);
+                        wsm[j * wstride + p * GP + h] = w;
+                        l = fmaf(w, lv[j][hh][u], l);
+                    }
                 }
 #pragma unroll
-                for (int u = 0; u < 4; ++u) m = fmaxf(m, mv[u]);
-            } else {
+                for (int off = 16; off >= 1; off >>= 1) l += __shfl_xor_sync(0xffffffffu, l, off);
+                if (lane == 0 && h < G && j < pend_n) tail->lsum[j * kMaxGroup + h] = l;
+            }
+        }
+    } else {
+        for (int j = 0; j < pend_n; ++j) {
+            const int nparts = pend_parts[j];
+            const float *mlg = a.part_ml + (size_t)pend_slot0[j] * GP * 2;
+            for (int h = warp; h < G; h += kConsWarps) {
+                float m = -INFINITY;
                 for (int p = lane; p < nparts; p += 32) {
                     const float x = __ldcg(&mlg[(p * GP + h) * 2]);
                     wsm[j * wstride + p * GP + h] = x;
                     m = fmaxf(m, x);
                 }
-            }
 #pragma unroll
-            for (int off = 16; off >= 1; off >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, off));
-            float l = 0.f;
-            if (small) {
-#pragma unroll
-                for (int u = 0; u < 4; ++u) {
-                    const int p = lane + 32 * u;
-                    if (p < nparts) {
-                        const float w = fast_exp2(mv[u] - m);
-                        wsm[j * wstride + p * GP + h] = w;
-                        l = fmaf(w, lv[u], l);
-                    }
-                }
-            } else {
+                for (int off = 16; off >= 1; off >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, off));
+                float l = 0.f;
                 for (int p = lane; p < nparts; p += 32) {
                     const float w = fast_exp2(wsm[j * wstride + p * GP + h] - m);
                     wsm[j * wstride + p * GP + h] = w;
                     l = fmaf(w, __ldcg(&mlg[(p * GP + h) * 2 + 1]), l);
                 }
-            }
 #pragma unroll
-            for (int off = 16; off >= 1; off >>= 1) l += __shfl_xor_sync(0xffffffffu, l, off);
-            if (lane == 0) tail->lsum[j * kMaxGroup + h] = l;
+                for (int off = 16; off >= 1; off >>= 1) l += __shfl_xor_sync(0xffffffffu, l, off);
+                if (lane == 0) tail->lsum[j * kMaxGroup + h] = l;
+            }
         }
     }
     named_barrier(1, kConsThreads);
@@ -638,14 +684,14 @@ decode_mma_kernel(const Args a, const __grid_constant__ CUtensorMap k_map, const
         acc[1][k] = 0.f;
     }
     int max_pieces = 0;
-    for (int j = 0; j < pend_n; ++j) max_pieces = max(max_pieces, (pend_parts[j] + PER_PIECE - 1) / PER_PIECE);
+    for (int j = 0; j < pend_n; ++j) max_pieces = max(max_pieces, (pend_parts[j] + per_piece[j] - 1) / per_piece[j]);
     for (int i = 0; i < max_pieces; ++i) {
 #pragma unroll
         for (int j = 0; j < 2; ++j) {
-            if (j < pend_n && i * PER_PIECE < pend_parts[j]) {
-                const int pp0 = i * PER_PIECE, np = min(PER_PIECE, pend_parts[j] - pp0);
+            if (j < pend_n && i * per_piece[j] < pend_parts[j]) {
+                const int pp0 = i * per_piece[j], np = min(per_piece[j], pend_parts[j] - pp0);
                 mbar_wait(&tail->cbar[j], (uint32_t)i & 1u, abort, a.status);
-                const float *po = reinterpret_cast<const float *>(ring + j * JOB_BYTES);
+                const float *po = reinterpret_cast<const float *>(ring + buf_off[j]);
                 const float *wj = wsm + j * wstride + pp0 * GP;
 #pragma unroll 2
                 for (int p = 0; p < np; ++p) {
@@ -661,7 +707,7 @@ decode_mma_kernel(const Args a, const __grid_constant__ CUtensorMap k_map, const
             named_barrier(1, kConsThreads);  // everyone is done with the buffers before they are refilled
             if (tid == 0)
                 for (int j = 0; j < pend_n; ++j)
-                    if ((i + 1) * PER_PIECE < pend_parts[j]) issue_piece(j, i + 1);
+                    if ((i + 1) * per_piece[j] < pend_parts[j]) issue_piece(j, i + 1);
         }
     }
 #pragma unroll

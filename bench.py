@@ -269,7 +269,7 @@ def run_ours(args):
         "gpu_launches": per_step * args.steps,
         "device_status_bits": status_bits,
         "clocks": clk.summary(),
-        "roofline": {"bound": "hbm", "kernel": "decode_kernel", "achieved": round(achieved, 1), "peak": peak,
+        "roofline": {"bound": "hbm", "kernel": "decode_mma_kernel", "achieved": round(achieved, 1), "peak": peak,
                      "peak_kind": f"of {peak_kind}", "unit": "GB/s", "frac": round(achieved / peak, 4),
                      "traffic": traffic, "algorithmic_bytes_per_launch": work.bytes["total"],
                      "avg_launch_us": round(launch_us, 3)},
@@ -302,7 +302,7 @@ def read_traffic_note():
     if not note.exists():
         return None
     kv = dict(l.split("=", 1) for l in note.read_text().splitlines() if "=" in l and not l.startswith("#"))
-    src = ROOT / "paper_2512_05033_b200" / "csrc" / "arb_decode.cu"
+    src = ROOT / "paper_2512_05033_b200" / "csrc" / "arb_decode_mma.cu"
     if kv.get("source_sha1", "").strip() != hashlib.sha1(src.read_bytes()).hexdigest():
         return None
     try:
@@ -470,6 +470,9 @@ def main():
     ap.add_argument("--workload", choices=("draft", "target"), default="draft",
                     help="decode workload of the timed loop (the headline is draft)")
     ap.add_argument("--layers", type=int, default=0, help="KV pools rotated per step (default 16 draft, 2 target)")
+    ap.add_argument("--profile-scoring", action="store_true",
+                    help="for runs under ncu: a few passes of the step-scoring workload (chunk attention, route, "
+                         "rollback) and nothing else")
     ap.add_argument("--profile", action="store_true",
                     help="for runs under ncu: stream launches, no e2e / extras / CPU baseline")
     args = ap.parse_args()
@@ -477,6 +480,10 @@ def main():
         args.warmup = 3
     if args.impl == "reference":
         run_reference(args)
+    elif args.profile_scoring:
+        from paper_2512_05033_b200 import binding
+        torch.cuda.set_device(0)
+        print(json.dumps({"step_scoring": run_step_scoring(binding.Context(0), torch.device("cuda", 0))}), flush=True)
     else:
         run_ours(args)
 

@@ -64,9 +64,18 @@ arb_status arb_create(arb_ctx **out, int device, size_t workspace_bytes) {
     bool ok = cudaMalloc(&c->workspace, c->workspace_bytes) == cudaSuccess;
     ok = ok && cudaMalloc(&c->counters, sizeof(int) * (c->counters_len + 4)) == cudaSuccess;
     ok = ok && cudaMemset(c->counters, 0, sizeof(int) * (c->counters_len + 4)) == cudaSuccess;
+    const size_t rot_ints = (size_t)kRotSets * kRotCounters + kRotSets + 4;
+    ok = ok && cudaMalloc(&c->rot, sizeof(int) * rot_ints) == cudaSuccess;
+    ok = ok && cudaMemset(c->rot, 0, sizeof(int) * rot_ints) == cudaSuccess;
+    if (ok) {  // "everything before the first call has completed"
+        const uint32_t done = c->decode_gen - 1;
+        ok = cudaMemcpy(c->rot + (size_t)kRotSets * kRotCounters + kRotSets, &done, sizeof(done),
+                        cudaMemcpyHostToDevice) == cudaSuccess;
+    }
     if (!ok) {
         cudaFree(c->workspace);
         cudaFree(c->counters);
+        cudaFree(c->rot);
         delete c;
         cudaGetLastError();
         return ARB_ERR_CUDA;
@@ -82,6 +91,7 @@ arb_status arb_destroy(arb_ctx *ctx) {
     DeviceGuard guard(c->device);
     cudaFree(c->workspace);
     cudaFree(c->counters);
+    cudaFree(c->rot);
     cudaFree(c->stage);
     delete c;
     return ARB_OK;
@@ -118,8 +128,10 @@ arb_status arb_attn(arb_ctx *ctx, const arb_attn_params *params, const void *q, 
     if (maybe_decode) {
         if (tensor_cores && decode_mma_supported(*params))
             st = launch_decode_mma(c, *params, q, k_pages, v_pages, block_table, seq_lens, q_lens, out, s);
-        else
+        else {
+            c->last_decode_shared_set0 = true;  // it uses workspace set 0 without a generation number
             st = launch_decode(c, *params, q, k_pages, v_pages, block_table, seq_lens, q_lens, out, s);
+        }
         if (st != ARB_OK) return st;
     }
     if (params->max_q_len >= 2) {
@@ -226,6 +238,8 @@ arb_status arb_poll_status(arb_ctx *ctx, arb_stream_t stream, uint32_t *bits) {
     if (bits) *bits = host;
     if (host != 0) {  // a kernel that gave up may have left arrival counters behind
         if (cudaMemsetAsync(c->counters, 0, sizeof(int) * (c->counters_len + 4), s) != cudaSuccess) return ARB_ERR_CUDA;
+        if (cudaMemsetAsync(c->rot, 0, sizeof(int) * ((size_t)kRotSets * kRotCounters + kRotSets), s) != cudaSuccess)
+            return ARB_ERR_CUDA;
         if (cudaStreamSynchronize(s) != cudaSuccess) return ARB_ERR_CUDA;
         return ARB_ERR_DEVICE_STATUS;
     }

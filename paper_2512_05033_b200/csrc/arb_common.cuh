@@ -31,7 +31,15 @@ struct Ctx {
     // staging for the *_host entry points
     char *stage = nullptr;
     size_t stage_bytes = 0;
+    // workspace rotation of the tensor-core decode kernel: kRotSets counter arrays, one exit counter
+    // per set and the generation of the newest completed call, all in one allocation
+    int *rot = nullptr;
+    uint32_t decode_gen = 1000;          // generation of the next tensor-core decode call
+    bool last_decode_shared_set0 = false; // the CUDA-core decode kernel used set 0 since then
 };
+
+constexpr int kRotSets = 4;
+constexpr int kRotCounters = 1 << 16;
 
 // ---------------------------------------------------------------------------------------------
 // Element types

@@ -28,7 +28,7 @@ constexpr int kD = 128;
 constexpr int kConsWarps = 4;
 constexpr int kConsThreads = kConsWarps * 32;
 constexpr int kThreads = kConsThreads + 32;
-constexpr int kGroup = 2;       // pages per consumer work group
+constexpr int kGroup = 1;       // pages per consumer work group: with 16 stages every warp has two groups in flight
 constexpr int kStages = 16;     // ring stages of one 4 KB tile each
 constexpr int kBatch = 16;      // producer lanes issuing side by side
 constexpr int kTileBytes = kPage * kD * 2;
@@ -52,6 +52,13 @@ struct Args {
     uint32_t *status;
     int batch, Hq, Hkv, num_pages, max_pages;
     float scale_log2;
+    // workspace rotation (see launch_decode_mma): this call's generation number, the number of
+    // workspace sets, the generation of the newest completed call, this set's exit counter
+    uint32_t gen;
+    int sets;
+    int force_wait;
+    unsigned *done_gen;
+    int *exit_count;
 };
 
 struct Tail {
@@ -61,6 +68,7 @@ struct Tail {
     float lsum[2 * kMaxGroup];   // per combine job and head: sum of the weighted sums
     int abort;
     int flags[kParked];   // per parked segment: this CTA was the last to arrive
+    int early;            // the workspace set is free: partials may be written before the predecessor is done
 };
 
 struct Parked {  // host-side view of what a parked segment needs besides its record
@@ -318,34 +326,50 @@ decode_mma_kernel(const Args a, const __grid_constant__ CUtensorMap k_map, const
     int pend_slot0[2], pend_parts[2];
     size_t pend_out[2];
 
-    // writes the parked segment results; returns after the arrival counters have been updated
-    auto flush = [&]() {
-        wait_for_predecessor();
+    // Ordering against the previous kernel on the stream.  Writes to `out` always wait for it
+    // (griddepcontrol.wait, once per CTA).  Writes to the workspace wait for it too, unless the call
+    // owns a workspace set that no unfinished call can still be reading: sets rotate with the call's
+    // generation number, and the last CTA of every call publishes its generation in *done_gen.
+    bool waited = false;
+    auto ensure_wait = [&]() {
+        if (!waited) { wait_for_predecessor(); waited = true; }
+    };
+    // Publishes the parked segment results: partials of split (sequence, head)s go to the workspace
+    // and are counted; results that are already final are written to `out` -- at once in the middle
+    // of a range (`last_call` false), or left parked for the epilogue, after the wait.
+    auto flush = [&](bool last_call) {
+        if (tid == 0) {
+            int early = 0;
+            if (a.sets >= 3 && !a.force_wait) {
+                unsigned d;
+                asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(d) : "l"(a.done_gen) : "memory");
+                early = (int)(d - (a.gen - (uint32_t)a.sets)) >= 0;  // the set's previous user has completed
+            }
+            tail->early = early;
+        }
+        named_barrier(1, kConsThreads);
+        if (!tail->early) ensure_wait();
         bool any_multi = false;
         for (int j = 0; j < n_parked; ++j) {
+            if (pk[j].nparts == 1) continue;
             const float *rec = park + j * REC;
             const size_t slot = (size_t)pk[j].bk + blockIdx.x;
             for (int idx = tid; idx < G * kD; idx += kConsThreads) {
                 const int h = idx / kD;
-                if (pk[j].nparts == 1) {
-                    reinterpret_cast<__nv_bfloat16 *>(a.out)[pk[j].out_base + idx] =
-                        __float2bfloat16_rn(rec[2 * GP + idx] / rec[GP + h]);
-                } else {
-                    a.part_o[slot * G * kD + idx] = rec[2 * GP + idx];
-                    if (idx - h * kD == 0) {
-                        a.part_ml[(slot * GP + h) * 2 + 0] = rec[h];
-                        a.part_ml[(slot * GP + h) * 2 + 1] = rec[GP + h];
-                    }
+                a.part_o[slot * G * kD + idx] = rec[2 * GP + idx];
+                if (idx - h * kD == 0) {
+                    a.part_ml[(slot * GP + h) * 2 + 0] = rec[h];
+                    a.part_ml[(slot * GP + h) * 2 + 1] = rec[GP + h];
                 }
             }
-            any_multi |= pk[j].nparts > 1;
+            any_multi = true;
         }
         if (any_multi) {
             fence_proxy_async_all();         // the partials are read back through bulk copies
             named_barrier(1, kConsThreads);  // the block's stores are ordered before thread 0's fence
             if (tid == 0) {
                 __threadfence();
-                fence_proxy_async_all();     // the partials are read back through bulk copies
+                fence_proxy_async_all();
                 for (int j = 0; j < n_parked; ++j) {
                     int last = 0;
                     if (pk[j].nparts > 1) {
@@ -366,8 +390,18 @@ decode_mma_kernel(const Args a, const __grid_constant__ CUtensorMap k_map, const
                 }
             }
         }
-        named_barrier(1, kConsThreads);  // parking slots and flags are free again
-        n_parked = 0;
+        if (!last_call) {
+            ensure_wait();
+            for (int j = 0; j < n_parked; ++j) {
+                if (pk[j].nparts != 1) continue;
+                const float *rec = park + j * REC;
+                for (int idx = tid; idx < G * kD; idx += kConsThreads)
+                    reinterpret_cast<__nv_bfloat16 *>(a.out)[pk[j].out_base + idx] =
+                        __float2bfloat16_rn(rec[2 * GP + idx] / rec[GP + idx / kD]);
+            }
+            named_barrier(1, kConsThreads);  // parking slots and flags are free again
+            n_parked = 0;
+        }
     };
 
     while (next_segment(cur, r1, pref, slen, B, Hkv, chunk, s)) {
@@ -504,7 +538,7 @@ decode_mma_kernel(const Args a, const __grid_constant__ CUtensorMap k_map, const
                 *reinterpret_cast<float2 *>(rec + 2 * GP + gq * kD + 8 * n + tq * 2) = make_float2(o[n][0], o[n][1]);
             if (tq == 0) { rec[gq] = m_run; rec[GP + gq] = l_run; }
         }
-        if (n_parked == kParked) flush();  // uniform across the consumer threads
+        if (n_parked == kParked) flush(false);  // uniform across the consumer threads
         named_barrier(1, kConsThreads);
         float *dst = park + n_parked * REC;
         for (int idx = tid; idx < G * kD; idx += kConsThreads) {
@@ -529,17 +563,28 @@ decode_mma_kernel(const Args a, const __grid_constant__ CUtensorMap k_map, const
         ++n_parked;
         named_barrier(1, kConsThreads);  // warp records are free for the next segment
     }
-    if (n_parked > 0) flush();
+    if (n_parked > 0) flush(true);  // final results stay parked until the epilogue
 
     // ---- split combine of the (sequence, kv head)s this CTA was the last to reach -----------------
     // Up to two jobs, worked on side by side.  The ring is idle: each job gets half of it as a landing
     // buffer for partial outputs (bulk copies, a piece at a time).  While the first pieces are in
     // flight the warps read the parts' (max, sum) records straight from global memory and turn them
     // into weights, kept where the warp records and parked segments used to be.
-    if (pend_n == 0) return;
     constexpr int PART_BYTES = G * kD * 4;
     constexpr int CAP = kRingBytes / PART_BYTES;   // partial outputs the ring can hold at once
     constexpr int NK = (G * kD + kConsThreads - 1) / kConsThreads;
+    float acc[2][NK];
+    int hk[NK];
+#pragma unroll
+    for (int k = 0; k < NK; ++k) {
+        const int idx = tid + k * kConsThreads;
+        hk[k] = idx < G * kD ? idx / kD : 0;
+        acc[0][k] = 0.f;
+        acc[1][k] = 0.f;
+    }
+    bool combined = false;
+    do {
+    if (pend_n == 0) break;
     // landing buffers: the whole ring for one job, shared in proportion to their parts for two
     int per_piece[2] = {CAP, 0}, buf_off[2] = {0, 0};
     if (pend_n == 2) {
@@ -550,7 +595,7 @@ decode_mma_kernel(const Args a, const __grid_constant__ CUtensorMap k_map, const
         buf_off[1] = c0 * PART_BYTES;
     }
     float *wsm = osm;                                        // [job][part][GP] weights
-    constexpr int WSM_FLOATS = (C::OSM_BYTES + C::PARK_BYTES) / 4;
+    constexpr int WSM_FLOATS = C::OSM_BYTES / 4;   // the parked records stay untouched
     const int wstride = WSM_FLOATS / 2;                      // floats per job
     bool fits = true;
     for (int j = 0; j < pend_n; ++j) fits = fits && pend_parts[j] * GP <= wstride;
@@ -558,6 +603,7 @@ decode_mma_kernel(const Args a, const __grid_constant__ CUtensorMap k_map, const
     if (!fits) {
         // more parts than the weight area can describe (one sequence over every CTA of a very large
         // part): merge straight from global memory
+        ensure_wait();
         for (int j = 0; j < pend_n; ++j) {
             const int nparts = pend_parts[j];
             const size_t slot0 = (size_t)pend_slot0[j];
@@ -574,7 +620,7 @@ decode_mma_kernel(const Args a, const __grid_constant__ CUtensorMap k_map, const
                 reinterpret_cast<__nv_bfloat16 *>(a.out)[pend_out[j] + idx] = __float2bfloat16_rn(x / l);
             }
         }
-        return;
+        break;
     }
     auto issue_piece = [&](int j, int i) {  // thread 0 only: piece i of job j into the job's buffer
         const int pp0 = i * per_piece[j], np = min(per_piece[j], pend_parts[j] - pp0);
@@ -674,15 +720,6 @@ decode_mma_kernel(const Args a, const __grid_constant__ CUtensorMap k_map, const
         }
     }
     named_barrier(1, kConsThreads);
-    float acc[2][NK];
-    int hk[NK];
-#pragma unroll
-    for (int k = 0; k < NK; ++k) {
-        const int idx = tid + k * kConsThreads;
-        hk[k] = idx < G * kD ? idx / kD : 0;
-        acc[0][k] = 0.f;
-        acc[1][k] = 0.f;
-    }
     int max_pieces = 0;
     for (int j = 0; j < pend_n; ++j) max_pieces = max(max_pieces, (pend_parts[j] + per_piece[j] - 1) / per_piece[j]);
     for (int i = 0; i < max_pieces; ++i) {
@@ -710,16 +747,43 @@ decode_mma_kernel(const Args a, const __grid_constant__ CUtensorMap k_map, const
                     if ((i + 1) * per_piece[j] < pend_parts[j]) issue_piece(j, i + 1);
         }
     }
+    combined = true;
+    } while (0);
+
+    // ---- epilogue: everything that goes to `out` waits for the previous kernel -------------------------
+    ensure_wait();
+    for (int j = 0; j < n_parked; ++j) {
+        if (pk[j].nparts != 1) continue;
+        const float *rec = park + j * REC;
+        for (int idx = tid; idx < G * kD; idx += kConsThreads)
+            reinterpret_cast<__nv_bfloat16 *>(a.out)[pk[j].out_base + idx] =
+                __float2bfloat16_rn(rec[2 * GP + idx] / rec[GP + idx / kD]);
+    }
+    if (combined) {
 #pragma unroll
-    for (int j = 0; j < 2; ++j) {
-        if (j < pend_n) {
+        for (int j = 0; j < 2; ++j) {
+            if (j < pend_n) {
 #pragma unroll
-            for (int k = 0; k < NK; ++k) {
-                const int idx = tid + k * kConsThreads;
-                if (idx < G * kD)
-                    reinterpret_cast<__nv_bfloat16 *>(a.out)[pend_out[j] + idx] =
-                        __float2bfloat16_rn(acc[j][k] / tail->lsum[j * kMaxGroup + hk[k]]);
+                for (int k = 0; k < NK; ++k) {
+                    const int idx = tid + k * kConsThreads;
+                    if (idx < G * kD)
+                        reinterpret_cast<__nv_bfloat16 *>(a.out)[pend_out[j] + idx] =
+                            __float2bfloat16_rn(acc[j][k] / tail->lsum[j * kMaxGroup + hk[k]]);
+                }
             }
+        }
+    }
+    // The last CTA to get here publishes this call's generation: its workspace set has been read for
+    // the last time (every combine is done) and every earlier call has completed (we waited for it).
+    named_barrier(1, kConsThreads);
+    if (tid == 0) {
+        __threadfence();
+        const int active_ctas = (total + chunk - 1) / chunk;
+        const int old = atomicAdd(a.exit_count, 1);
+        if (old == active_ctas - 1) {
+            *a.exit_count = 0;
+            __threadfence();
+            asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(a.done_gen), "r"(a.gen) : "memory");
         }
     }
 }
@@ -795,17 +859,35 @@ arb_status launch_decode_mma(Ctx *ctx, const arb_attn_params &p, const void *q, 
     if (!make_pool_map(&km, k_pages, p) || !make_pool_map(&vm, v_pages, p)) return ARB_ERR_CUDA;
     const int g = p.num_q_heads / p.num_kv_heads;
     const int gp = (g + 3) / 4 * 4;
-    (void)gp;
     const size_t slots = (size_t)p.batch * p.num_kv_heads + (size_t)ctx->num_sms * kCtasPerSm;
+    // Workspace rotation.  Consecutive calls take consecutive generation numbers and use workspace set
+    // (generation mod sets): partials, (max, sum) records and arrival counters of their own.  A call
+    // may write its set without waiting for the previous call once the set's previous user
+    // (generation - sets) has published its completion.  With fewer than three sets that fit in the
+    // workspace, or right after a CUDA-core decode call (which uses set 0 unnumbered), it waits.
+    const size_t part_o_floats = (slots * g * p.head_dim + 63) & ~size_t(63);
+    const size_t set_bytes = ((part_o_floats + slots * gp * 2) * sizeof(float) + 255) & ~size_t(255);
+    int sets = (int)(ctx->workspace_bytes / set_bytes);
+    if (sets > kRotSets) sets = kRotSets;
+    if (sets < 1) return ARB_ERR_WORKSPACE;
+    if ((long long)p.batch * p.num_kv_heads > kRotCounters) sets = 1;
+    const uint32_t gen = ctx->decode_gen++;
+    const int set = (int)(gen % (uint32_t)sets);
     Args a;
     a.q = static_cast<const char *>(q);
     a.block_table = block_table;
     a.seq_lens = seq_lens;
     a.q_lens = q_lens;
     a.out = static_cast<char *>(out);
-    a.part_o = reinterpret_cast<float *>(ctx->workspace);
-    a.part_ml = a.part_o + ((slots * g * p.head_dim + 63) & ~size_t(63));
-    a.counters = ctx->counters;
+    a.part_o = reinterpret_cast<float *>(ctx->workspace + (size_t)set * set_bytes);
+    a.part_ml = a.part_o + part_o_floats;
+    a.counters = sets > 1 ? ctx->rot + (size_t)set * kRotCounters : ctx->counters;
+    a.exit_count = ctx->rot + (size_t)kRotSets * kRotCounters + set;
+    a.done_gen = reinterpret_cast<unsigned *>(ctx->rot + (size_t)kRotSets * kRotCounters + kRotSets);
+    a.gen = gen;
+    a.sets = sets;
+    a.force_wait = ctx->last_decode_shared_set0 ? 1 : 0;
+    ctx->last_decode_shared_set0 = false;
     a.status = ctx->status;
     a.batch = p.batch;
     a.Hq = p.num_q_heads;

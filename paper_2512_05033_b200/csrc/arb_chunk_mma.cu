@@ -6,19 +6,22 @@
 // it walks the visible keys in tiles of 128 (eight pages):
 //
 //     S = Q K^T      tcgen05.mma, A = Q tile, B = K tile, both K-major in shared memory (128-byte
-//                    swizzle), fp32 accumulator in TMEM columns [0, 128)
+//                    swizzle), fp32 accumulator in one of two TMEM buffers of 128 columns
 //     P = exp2(scale * S - m)   by the 128 softmax threads, one TMEM lane (= query row) each:
 //                    tcgen05.ld, causal / length mask, row max, exponentials, bf16 P written back to
 //                    shared memory in the K-major swizzled layout
 //     O += P V       tcgen05.mma, A = P, B = V tile read MN-major straight from its page layout,
-//                    fp32 accumulator in TMEM columns [128, 256)
+//                    fp32 accumulator in TMEM columns [256, 384)
 //
 // The running max is lazy: O is rescaled (tcgen05.ld / st) only when a row's max grows by more than
 // 2^8, otherwise the stale max keeps the exponentials bounded by 2^8 and nothing is touched.
 // K and V tiles are fetched page by page with tiled TMA copies (one 16 x 64 box per page and half
-// of head_dim, landing in the canonical swizzled layout) into a two-stage ring.  Roles: warps 0-3
-// softmax and epilogue, warp 4 TMA producer, warp 5 MMA issue and TMEM allocation.  Every mbarrier
-// wait is bounded; TMEM is released on every path.
+// of head_dim, landing in the canonical swizzled layout) into a two-stage ring.  S is double-buffered
+// in TMEM (columns 0-127 and 128-255, O in 256-383), so Q K^T of the next tile runs under the softmax
+// of the current one.  Roles: warps 0-3 softmax and epilogue, warp 4 TMA producer, warp 5 MMA issue
+// and TMEM allocation.  Work items are handed out dynamically, longest sequences first: the producer
+// warp takes the next item from an atomic counter and announces it to the other roles through a small
+// queue in shared memory.  Every mbarrier wait is bounded; TMEM is released on every path.
 #include <cuda.h>  // CUtensorMap and its enums only; the encoder is looked up at run time
 
 #include "arb_common.cuh"
@@ -37,8 +40,11 @@ constexpr int kThreads = 192;
 constexpr int kHalfBytes = 128 * 128;      // [128 rows x 64 bf16]: one 128-byte-swizzled half tile
 constexpr int kTileBytes = 2 * kHalfBytes;  // [128 x 128] bf16
 constexpr int kBoxBytes = kPage * 128;      // one TMA box: 16 rows x 64 bf16
-constexpr uint32_t kTmemCols = 256;         // S: columns 0..127, O: columns 128..255
+constexpr uint32_t kTmemCols = 512;         // S0: columns 0..127, S1: 128..255, O: 256..383
+constexpr uint32_t kOCol = 256;
 constexpr float kRescaleThreshold = 8.0f;   // log2 units
+constexpr int kItemSlots = 8;               // work items announced ahead of their use
+constexpr int kSortMaxBatch = 256;          // up to this batch size sequences are served longest first
 
 struct MmaArgs {
     const char *q;
@@ -49,6 +55,7 @@ struct MmaArgs {
     uint32_t *status;
     int batch, Hq, Hkv, num_pages, max_pages;
     int min_rows;  // sequences with q_len * group >= min_rows are handled here
+    int *work_counter;  // next work item; zeroed on the stream before the launch
     float scale_log2;
 };
 
@@ -57,9 +64,12 @@ struct Bars {
     uint64_t k_full[kStages];    // TMA bytes of a K tile landed
     uint64_t v_full[kStages];
     uint64_t kv_empty[kStages];  // the MMAs that read the stage have completed
-    uint64_t s_full;             // S = Q K^T is in TMEM
+    uint64_t s_full[2];          // S = Q K^T is in TMEM buffer 0 / 1
     uint64_t p_full;             // P is in shared memory, S may be overwritten
     uint64_t o_full;             // O += P V has completed
+    uint64_t item_full[kItemSlots];   // the producer warp has fetched the next work item
+    uint64_t item_empty[kItemSlots];  // the MMA thread and the softmax threads have read it
+    int item_id[kItemSlots];
     uint32_t tmem_base;
     int abort;
 };
@@ -67,7 +77,7 @@ struct Bars {
 constexpr size_t kSmemFixed = 1024 /*alignment*/ + 2 * kTileBytes /*Q, P*/ + 2 * kStages * kTileBytes /*K, V*/ +
                               sizeof(Bars);
 
-inline size_t mma_smem_bytes(int batch) { return kSmemFixed + sizeof(int) * (2 * (size_t)batch + 2); }
+inline size_t mma_smem_bytes(int batch) { return kSmemFixed + sizeof(int) * (5 * (size_t)batch + 2); }
 
 // ---- tcgen05 / TMA wrappers -------------------------------------------------------------------
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
@@ -156,6 +166,18 @@ __device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&v)[32
 __device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
+// acc + lo + hi for a packed bf16 pair, in fp32 (mixed-precision FMA with 1.0: no unpacking)
+__device__ __forceinline__ float add_bf16x2(uint32_t w, float acc) {
+    asm("{\n\t.reg .b16 lo, hi, one;\n\t"
+        "mov.b32 {lo, hi}, %1;\n\t"
+        "mov.b16 one, 0x3f80;\n\t"
+        "fma.rn.f32.bf16 %0, lo, one, %0;\n\t"
+        "fma.rn.f32.bf16 %0, hi, one, %0;\n\t}"
+        : "+f"(acc)
+        : "r"(w));
+    return acc;
+}
+
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
     uint32_t r;
     asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
@@ -167,17 +189,18 @@ struct Item {
 };
 
 template <int G>
-__device__ __forceinline__ bool get_item(int item, int total, const int *pref, const int *row0, int B, int Hkv,
-                                         const MmaArgs &a, Item &it) {
+__device__ __forceinline__ bool get_item(int item, int total, const int *pref, const int *row0, const int *sorted,
+                                         int B, int Hkv, const MmaArgs &a, Item &it) {
     if (item >= total) return false;
     int lo = 0, hi = B;
     while (hi - lo > 1) {
         const int mid = (lo + hi) >> 1;
         if (pref[mid] <= item) lo = mid; else hi = mid;
     }
-    it.b = lo;
-    it.n = a.q_lens[lo];
-    it.L = a.seq_lens[lo];
+    const int sb = sorted[lo];  // pref runs over the sequences in serving order
+    it.b = sb;
+    it.n = a.q_lens[sb];
+    it.L = a.seq_lens[sb];
     it.rows_total = it.n * G;
     const int mtiles = (it.rows_total + kBM - 1) / kBM;
     const int r = item - pref[lo];
@@ -188,7 +211,7 @@ __device__ __forceinline__ bool get_item(int item, int total, const int *pref, c
     const int i_last = (it.r_begin + it.rows_here - 1) / G;
     it.kv_len = it.L - it.n + i_last + 1;
     it.ntiles = (it.kv_len + kBN - 1) / kBN;
-    it.qrow0 = row0[lo];
+    it.qrow0 = row0[sb];
     return true;
 }
 
@@ -204,6 +227,9 @@ chunk_mma_kernel(const MmaArgs a, const __grid_constant__ CUtensorMap k_map, con
     Bars *bars = reinterpret_cast<Bars *>(v_s + kStages * kTileBytes);
     int *pref = reinterpret_cast<int *>(bars + 1);     // [B + 1] work items before sequence b
     int *row0 = pref + a.batch + 1;                    // [B + 1] q rows before sequence b
+    int *sorted = row0 + a.batch + 1;                  // [B] sequences in serving order (longest first)
+    int *itm = sorted + a.batch;                       // [B] work items of sequence b
+    int *key = itm + a.batch;                          // [B] visible keys of sequence b (sort key)
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int B = a.batch, Hkv = a.Hkv;
@@ -215,9 +241,14 @@ chunk_mma_kernel(const MmaArgs a, const __grid_constant__ CUtensorMap k_map, con
             mbar_init(&bars->v_full[s], 1);
             mbar_init(&bars->kv_empty[s], 1);
         }
-        mbar_init(&bars->s_full, 1);
+        mbar_init(&bars->s_full[0], 1);
+        mbar_init(&bars->s_full[1], 1);
         mbar_init(&bars->p_full, kSoftmaxThreads);
         mbar_init(&bars->o_full, 1);
+        for (int i = 0; i < kItemSlots; ++i) {
+            mbar_init(&bars->item_full[i], 1);
+            mbar_init(&bars->item_empty[i], 1 + kSoftmaxThreads);
+        }
         bars->abort = 0;
         mbar_fence_init();
         pref[0] = 0;
@@ -227,9 +258,24 @@ chunk_mma_kernel(const MmaArgs a, const __grid_constant__ CUtensorMap k_map, con
         const int n = a.q_lens[b], L = a.seq_lens[b];
         int items = 0;
         if (n >= 2 && n * G >= a.min_rows && L >= n && L <= a.max_pages * kPage) items = Hkv * ((n * G + kBM - 1) / kBM);
-        pref[b + 1] = items;
+        itm[b] = items;
+        key[b] = items > 0 ? L : -1;
         row0[b + 1] = n > 0 ? n : 0;
     }
+    __syncthreads();
+    // serving order: longest first (items of a long sequence take longest), ties by index; large
+    // batches keep their own order
+    for (int b = tid; b < B; b += kThreads) {
+        int rank = b;
+        if (B <= kSortMaxBatch) {
+            rank = 0;
+            const int kb = key[b];
+            for (int o = 0; o < B; ++o) rank += (key[o] > kb) || (key[o] == kb && o < b);
+        }
+        sorted[rank] = b;
+    }
+    __syncthreads();
+    for (int r = tid; r < B; r += kThreads) pref[r + 1] = itm[sorted[r]];
     __syncthreads();
     if (warp == 0) {
         int carry_p = 0, carry_r = 0;
@@ -263,7 +309,19 @@ chunk_mma_kernel(const MmaArgs a, const __grid_constant__ CUtensorMap k_map, con
         // ===================================== TMA producer =========================================
         uint32_t it = 0;  // KV tiles issued so far
         Item w;
-        for (int item = blockIdx.x; get_item<G>(item, total, pref, row0, B, Hkv, a, w); item += gridDim.x) {
+        // Work items are handed out dynamically (an atomic counter, longest sequences first): this
+        // warp fetches the next item, announces it to the other roles through a small queue in
+        // shared memory and runs ahead of them as far as the K/V ring allows.
+        for (uint32_t nq = 0;; ++nq) {
+            const uint32_t slot = nq % kItemSlots, qpar = (nq / kItemSlots) & 1u;
+            int item = total;
+            if (lane == 0) {
+                if (mbar_wait(&bars->item_empty[slot], qpar ^ 1u, abort, a.status)) item = atomicAdd(a.work_counter, 1);
+                bars->item_id[slot] = item;
+                mbar_arrive(&bars->item_full[slot]);
+            }
+            item = __shfl_sync(0xffffffffu, item, 0);
+            if (!get_item<G>(item, total, pref, row0, sorted, B, Hkv, a, w)) break;
             for (int j = 0; j < w.ntiles; ++j, ++it) {
                 const uint32_t s = it % kStages, par = (it / kStages) & 1u;
                 const int npages = min(kTilePages, (w.kv_len - j * kBN + kPage - 1) / kPage);
@@ -304,21 +362,36 @@ chunk_mma_kernel(const MmaArgs a, const __grid_constant__ CUtensorMap k_map, con
             const uint32_t q_addr = smem_u32(q_s), p_addr = smem_u32(p_s);
             uint32_t it = 0, nitem = 0;
             Item w;
-            for (int item = blockIdx.x; get_item<G>(item, total, pref, row0, B, Hkv, a, w); item += gridDim.x, ++nitem) {
+            for (;; ++nitem) {
+                const uint32_t slot = nitem % kItemSlots, qpar = (nitem / kItemSlots) & 1u;
+                if (!mbar_wait(&bars->item_full[slot], qpar, abort, a.status)) break;
+                const int item = bars->item_id[slot];
+                mbar_arrive(&bars->item_empty[slot]);
+                if (!get_item<G>(item, total, pref, row0, sorted, B, Hkv, a, w)) break;
                 mbar_wait(&bars->q_full, nitem & 1u, abort, a.status);
-                for (int j = 0; j < w.ntiles; ++j, ++it) {
-                    const uint32_t s = it % kStages, par = (it / kStages) & 1u;
-                    const uint32_t k_addr = smem_u32(k_s + s * kTileBytes), v_addr = smem_u32(v_s + s * kTileBytes);
-                    // ---- S = Q K^T: 8 steps of 16 dims; 4 per 64-dim half; K-major operands, SBO = 8 rows
+                // S = Q K^T of tile `itx` into S buffer itx & 1: 8 steps of 16 dims, 4 per 64-dim half;
+                // K-major operands, SBO = 8 rows.  Issued one tile ahead, so that it runs under the
+                // softmax of the tile before it.
+                auto issue_qk = [&](uint32_t itx) {
+                    const uint32_t s = itx % kStages, par = (itx / kStages) & 1u;
+                    const uint32_t k_addr = smem_u32(k_s + s * kTileBytes);
                     mbar_wait(&bars->k_full[s], par, abort, a.status);
                     tc_fence_after();
 #pragma unroll
                     for (int ks = 0; ks < kD / 16; ++ks) {
                         const uint32_t off = (ks >> 2) * kHalfBytes + (ks & 3) * 32;
-                        mma_f16_ss(tmem, smem_desc(q_addr + off, 16, 1024), smem_desc(k_addr + off, 16, 1024), idesc_qk,
-                                   ks > 0 ? 1u : 0u);
+                        mma_f16_ss(tmem + (itx & 1u) * kBN, smem_desc(q_addr + off, 16, 1024),
+                                   smem_desc(k_addr + off, 16, 1024), idesc_qk, ks > 0 ? 1u : 0u);
                     }
-                    mma_commit(&bars->s_full);
+                    mma_commit(&bars->s_full[itx & 1u]);
+                };
+                issue_qk(it);
+                for (int j = 0; j < w.ntiles; ++j, ++it) {
+                    const uint32_t s = it % kStages, par = (it / kStages) & 1u;
+                    const uint32_t v_addr = smem_u32(v_s + s * kTileBytes);
+                    // the other S buffer was read by the softmax of tile it - 1, which ended before the
+                    // p_full this thread waited for in the previous iteration
+                    if (j + 1 < w.ntiles) issue_qk(it + 1);
                     // ---- O += P V: 8 steps of 16 keys; P K-major; V MN-major: 64-dim halves LBO apart,
                     //      8-key groups SBO apart
                     mbar_wait(&bars->p_full, it & 1u, abort, a.status);
@@ -327,7 +400,7 @@ chunk_mma_kernel(const MmaArgs a, const __grid_constant__ CUtensorMap k_map, con
 #pragma unroll
                     for (int ks = 0; ks < kBN / 16; ++ks) {
                         const uint32_t p_off = (ks >> 2) * kHalfBytes + (ks & 3) * 32;
-                        mma_f16_ss(tmem + kBN, smem_desc(p_addr + p_off, 16, 1024),
+                        mma_f16_ss(tmem + kOCol, smem_desc(p_addr + p_off, 16, 1024),
                                    smem_desc(v_addr + ks * 2 * 1024, kHalfBytes, 1024), idesc_pv,
                                    (j > 0 || ks > 0) ? 1u : 0u);
                     }
@@ -340,11 +413,16 @@ chunk_mma_kernel(const MmaArgs a, const __grid_constant__ CUtensorMap k_map, con
     } else {
         // ================================ softmax and epilogue ====================================
         const uint32_t lane_base = (uint32_t)(warp * 32) << 16;  // this warp's TMEM lane quadrant
-        const uint32_t s_tmem = tmem + lane_base, o_tmem = tmem + lane_base + kBN;
+        const uint32_t o_tmem = tmem + lane_base + kOCol;
         const int swz = tid & 7;
         uint32_t it = 0, nitem = 0;
         Item w;
-        for (int item = blockIdx.x; get_item<G>(item, total, pref, row0, B, Hkv, a, w); item += gridDim.x, ++nitem) {
+        for (;; ++nitem) {
+            const uint32_t slot = nitem % kItemSlots, qpar = (nitem / kItemSlots) & 1u;
+            if (!mbar_wait(&bars->item_full[slot], qpar, abort, a.status)) break;
+            const int item = bars->item_id[slot];
+            mbar_arrive(&bars->item_empty[slot]);
+            if (!get_item<G>(item, total, pref, row0, sorted, B, Hkv, a, w)) break;
             const bool row_ok = tid < w.rows_here;
             const int r = min(w.r_begin + tid, w.rows_total - 1);
             const int tok = r / G, head = r - tok * G;
@@ -366,7 +444,8 @@ chunk_mma_kernel(const MmaArgs a, const __grid_constant__ CUtensorMap k_map, con
                 const uint32_t s = it % kStages, par = (it / kStages) & 1u;
                 const int key0 = j * kBN;
                 const int nvis = lim - key0;  // columns < nvis are visible to this row (may be <= 0)
-                mbar_wait(&bars->s_full, it & 1u, abort, a.status);
+                const uint32_t s_tmem = tmem + lane_base + (it & 1u) * kBN;
+                mbar_wait(&bars->s_full[it & 1u], (it >> 1) & 1u, abort, a.status);
                 tc_fence_after();
                 // ---- pass 1: row max of the visible scores
                 float mx = -INFINITY;
@@ -393,8 +472,13 @@ chunk_mma_kernel(const MmaArgs a, const __grid_constant__ CUtensorMap k_map, con
                     l_sum *= factor;
                     m_used = m_tile;
                 }
+                // P of the previous tile (shared memory) and O (TMEM) are still in use until its
+                // second product has completed
+                if (j > 0) {
+                    mbar_wait(&bars->o_full, (it - 1u) & 1u, abort, a.status);
+                    tc_fence_after();
+                }
                 if (__any_sync(0xffffffffu, rescale)) {
-                    // O of the previous tiles is complete: s_full of this tile was committed after them
 #pragma unroll 1
                     for (int c4 = 0; c4 < 4; ++c4) {
                         uint32_t v[32];
@@ -424,7 +508,7 @@ chunk_mma_kernel(const MmaArgs a, const __grid_constant__ CUtensorMap k_map, con
                         const uint32_t w = pack_bf16((c4 * 32 + 2 * k < nvis) ? e0 : 0.f,
                                                      (c4 * 32 + 2 * k + 1 < nvis) ? e1 : 0.f);
                         pk[k] = w;
-                        l_sum += __uint_as_float(w << 16) + __uint_as_float(w & 0xffff0000u);
+                        l_sum = add_bf16x2(w, l_sum);
                     }
                     char *prow = p_s + (c4 >> 1) * kHalfBytes + tid * 128;
 #pragma unroll
@@ -562,6 +646,8 @@ arb_status launch_chunk_mma(Ctx *ctx, const arb_attn_params &p, const void *q, c
     a.num_pages = p.num_pages;
     a.max_pages = p.max_pages_per_seq;
     a.min_rows = kChunkMmaMinRows;
+    a.work_counter = ctx->rot + (size_t)kRotSets * kRotCounters + kRotSets + 1;
+    if (cudaMemsetAsync(a.work_counter, 0, sizeof(int), stream) != cudaSuccess) return ARB_ERR_CUDA;
     const float scale = p.softmax_scale > 0.f ? p.softmax_scale : 1.0f / sqrtf((float)p.head_dim);
     a.scale_log2 = scale * 1.4426950408889634f;
     const int g = p.num_q_heads / p.num_kv_heads;

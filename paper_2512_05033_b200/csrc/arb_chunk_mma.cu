@@ -110,6 +110,17 @@ __device__ __forceinline__ void mma_f16_ss(uint32_t d_tmem, uint64_t a_desc, uin
         : "memory");
 }
 
+// D[tmem] (+)= A[tmem] * B[smem]: A is bf16 packed two to a 32-bit column, row m in TMEM lane m
+__device__ __forceinline__ void mma_f16_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc,
+                                           uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+
 // Shared-memory matrix descriptor, 128-byte swizzle: start address, leading / stride byte offsets
 // (all in 16-byte units), descriptor version 1 (sm_100), layout type 2 (SWIZZLE_128B).
 __device__ __forceinline__ uint64_t smem_desc(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
@@ -163,6 +174,14 @@ __device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&v)[32
         : "memory");
 }
 #undef ARB_W8
+__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&v)[16]) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], "
+        "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};"
+        ::"r"(taddr), "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7]), "r"(v[8]),
+        "r"(v[9]), "r"(v[10]), "r"(v[11]), "r"(v[12]), "r"(v[13]), "r"(v[14]), "r"(v[15])
+        : "memory");
+}
 __device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
@@ -359,7 +378,7 @@ chunk_mma_kernel(const MmaArgs a, const __grid_constant__ CUtensorMap k_map, con
         // ====================================== MMA issue ===========================================
         if (lane == 0) {
             constexpr uint32_t idesc_qk = instr_desc(false), idesc_pv = instr_desc(true);
-            const uint32_t q_addr = smem_u32(q_s), p_addr = smem_u32(p_s);
+            const uint32_t q_addr = smem_u32(q_s);
             uint32_t it = 0, nitem = 0;
             Item w;
             for (;; ++nitem) {
@@ -399,8 +418,8 @@ chunk_mma_kernel(const MmaArgs a, const __grid_constant__ CUtensorMap k_map, con
                     tc_fence_after();
 #pragma unroll
                     for (int ks = 0; ks < kBN / 16; ++ks) {
-                        const uint32_t p_off = (ks >> 2) * kHalfBytes + (ks & 3) * 32;
-                        mma_f16_ss(tmem + kOCol, smem_desc(p_addr + p_off, 16, 1024),
+                        // P of this tile sits in the first 64 columns of its S buffer, 16 keys = 8 columns
+                        mma_f16_ts(tmem + kOCol, tmem + (it & 1u) * kBN + ks * 8,
                                    smem_desc(v_addr + ks * 2 * 1024, kHalfBytes, 1024), idesc_pv,
                                    (j > 0 || ks > 0) ? 1u : 0u);
                     }
@@ -472,13 +491,12 @@ chunk_mma_kernel(const MmaArgs a, const __grid_constant__ CUtensorMap k_map, con
                     l_sum *= factor;
                     m_used = m_tile;
                 }
-                // P of the previous tile (shared memory) and O (TMEM) are still in use until its
-                // second product has completed
-                if (j > 0) {
+                if (__any_sync(0xffffffffu, rescale)) {
+                    // O is still being accumulated until the previous tile's second product is done.
+                    // (s_full of this tile was committed after the product before that one, so this
+                    // wait is never more than one phase behind its barrier.)
                     mbar_wait(&bars->o_full, (it - 1u) & 1u, abort, a.status);
                     tc_fence_after();
-                }
-                if (__any_sync(0xffffffffu, rescale)) {
 #pragma unroll 1
                     for (int c4 = 0; c4 < 4; ++c4) {
                         uint32_t v[32];
@@ -510,14 +528,11 @@ chunk_mma_kernel(const MmaArgs a, const __grid_constant__ CUtensorMap k_map, con
                         pk[k] = w;
                         l_sum = add_bf16x2(w, l_sum);
                     }
-                    char *prow = p_s + (c4 >> 1) * kHalfBytes + tid * 128;
-#pragma unroll
-                    for (int qd = 0; qd < 4; ++qd) {
-                        const int cc = (c4 & 1) * 4 + qd;
-                        *reinterpret_cast<uint4 *>(prow + ((cc ^ swz) << 4)) =
-                            make_uint4(pk[qd * 4 + 0], pk[qd * 4 + 1], pk[qd * 4 + 2], pk[qd * 4 + 3]);
-                    }
+                    // P overwrites S in place: keys 32 c4 .. 32 c4 + 31 -> columns 16 c4 .. 16 c4 + 15,
+                    // which this thread has already read
+                    tmem_st16(s_tmem + c4 * 16, pk);
                 }
+                tmem_wait_st();
                 // ---- V rows past the last visible key of the item (stale slots, pages never loaded)
                 //      must not reach the tensor core, not even times zero
                 const int nvalid = w.kv_len - key0;

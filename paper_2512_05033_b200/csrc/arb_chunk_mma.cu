@@ -2,26 +2,29 @@
 //
 // A chunk of n query tokens against one KV head is a dense contraction once n * group >= 64:
 // the M = n * group query rows (token-major, the group's heads of one token are consecutive rows)
-// all read the same keys.  One work item is a tile of 128 query rows of one (sequence, kv head);
-// it walks the visible keys in tiles of 128 (eight pages):
+// all read the same keys.  One work item is a pair of row tiles (A, B: 128 query rows each, B may be
+// missing) of one (sequence, kv head); it walks the visible keys in tiles of 128 (eight pages), and
+// both row tiles use every K/V tile that is loaded.  Per row tile and KV tile:
 //
 //     S = Q K^T      tcgen05.mma, A = Q tile, B = K tile, both K-major in shared memory (128-byte
-//                    swizzle), fp32 accumulator in one of two TMEM buffers of 128 columns
-//     P = exp2(scale * S - m)   by the 128 softmax threads, one TMEM lane (= query row) each:
-//                    tcgen05.ld, causal / length mask, row max, exponentials, bf16 P written back to
-//                    shared memory in the K-major swizzled layout
-//     O += P V       tcgen05.mma, A = P, B = V tile read MN-major straight from its page layout,
-//                    fp32 accumulator in TMEM columns [256, 384)
+//                    swizzle), fp32 accumulator in the row tile's 128 TMEM columns for S
+//     P = exp2(scale * S - m)   by the row tile's 128 softmax threads, one TMEM lane (= query row)
+//                    each: tcgen05.ld, causal / length mask, row max, exponentials; P, rounded to
+//                    bf16, overwrites S in place (tcgen05.st, two keys per column)
+//     O += P V       tcgen05.mma with P as the TMEM A operand and the V tile read MN-major straight
+//                    from its page layout; fp32 accumulator in the row tile's 128 TMEM columns for O
 //
-// The running max is lazy: O is rescaled (tcgen05.ld / st) only when a row's max grows by more than
-// 2^8, otherwise the stale max keeps the exponentials bounded by 2^8 and nothing is touched.
-// K and V tiles are fetched page by page with tiled TMA copies (one 16 x 64 box per page and half
-// of head_dim, landing in the canonical swizzled layout) into a two-stage ring.  S is double-buffered
-// in TMEM (columns 0-127 and 128-255, O in 256-383), so Q K^T of the next tile runs under the softmax
-// of the current one.  Roles: warps 0-3 softmax and epilogue, warp 4 TMA producer, warp 5 MMA issue
-// and TMEM allocation.  Work items are handed out dynamically, longest sequences first: the producer
-// warp takes the next item from an atomic counter and announces it to the other roles through a small
-// queue in shared memory.  Every mbarrier wait is bounded; TMEM is released on every path.
+// TMEM: S_A 0-127, S_B 128-255, O_A 256-383, O_B 384-511.  The MMA thread interleaves the two row
+// tiles (P V of A, next Q K^T of A, P V of B, next Q K^T of B), so the tensor core works for one
+// row tile while the other one's softmax group is busy.  The running max is lazy: O is rescaled
+// (tcgen05.ld / st) only when a row's max grows by more than 2^8, otherwise the stale max keeps the
+// exponentials bounded by 2^8 and nothing is touched.  K and V tiles are fetched page by page with
+// tiled TMA copies (one 16 x 64 box per page and half of head_dim, landing in the canonical swizzled
+// layout) into a two-stage ring.  Roles: warps 0-3 softmax and epilogue of row tile A, warps 4-7 of
+// row tile B, warp 8 TMA producer, warp 9 MMA issue and TMEM allocation.  Work items are handed out
+// dynamically, longest sequences first: the producer warp takes the next item from an atomic counter
+// and announces it to the other roles through a small queue in shared memory.  Every mbarrier wait
+// is bounded; TMEM is released on every path.
 #include <cuda.h>  // CUtensorMap and its enums only; the encoder is looked up at run time
 
 #include "arb_common.cuh"
@@ -31,16 +34,17 @@ namespace arb {
 namespace {
 
 constexpr int kD = 128;           // head_dim
-constexpr int kBM = 128;          // query rows per work item
+constexpr int kBM = 128;          // query rows per row tile; a work item is a pair of row tiles
 constexpr int kBN = 128;          // keys per KV tile
 constexpr int kTilePages = kBN / kPage;
 constexpr int kStages = 2;
-constexpr int kSoftmaxThreads = 128;
-constexpr int kThreads = 192;
+constexpr int kSoftmaxThreads = 128;        // per row tile
+constexpr int kThreads = 2 * kSoftmaxThreads + 64;   // two softmax groups, TMA warp, MMA warp
+constexpr int kTmaWarp = 8, kMmaWarp = 9;
 constexpr int kHalfBytes = 128 * 128;      // [128 rows x 64 bf16]: one 128-byte-swizzled half tile
 constexpr int kTileBytes = 2 * kHalfBytes;  // [128 x 128] bf16
 constexpr int kBoxBytes = kPage * 128;      // one TMA box: 16 rows x 64 bf16
-constexpr uint32_t kTmemCols = 512;         // S0: columns 0..127, S1: 128..255, O: 256..383
+constexpr uint32_t kTmemCols = 512;         // S of tile A: columns 0..127, S of B: 128..255, O of A: 256..383, O of B: 384..511
 constexpr uint32_t kOCol = 256;
 constexpr float kRescaleThreshold = 8.0f;   // log2 units
 constexpr int kItemSlots = 8;               // work items announced ahead of their use
@@ -60,13 +64,13 @@ struct MmaArgs {
 };
 
 struct Bars {
-    uint64_t q_full;             // 128 softmax threads wrote the Q tile
+    uint64_t q_full;             // both softmax groups wrote their Q tiles
     uint64_t k_full[kStages];    // TMA bytes of a K tile landed
     uint64_t v_full[kStages];
     uint64_t kv_empty[kStages];  // the MMAs that read the stage have completed
-    uint64_t s_full[2];          // S = Q K^T is in TMEM buffer 0 / 1
-    uint64_t p_full;             // P is in shared memory, S may be overwritten
-    uint64_t o_full;             // O += P V has completed
+    uint64_t s_full[2];          // S = Q K^T of row tile A / B is in TMEM
+    uint64_t p_full[2];          // P of row tile A / B is in TMEM (over S)
+    uint64_t o_full[2];          // O += P V of row tile A / B has completed
     uint64_t item_full[kItemSlots];   // the producer warp has fetched the next work item
     uint64_t item_empty[kItemSlots];  // the MMA thread and the softmax threads have read it
     int item_id[kItemSlots];
@@ -74,7 +78,7 @@ struct Bars {
     int abort;
 };
 
-constexpr size_t kSmemFixed = 1024 /*alignment*/ + 2 * kTileBytes /*Q, P*/ + 2 * kStages * kTileBytes /*K, V*/ +
+constexpr size_t kSmemFixed = 1024 /*alignment*/ + 2 * kTileBytes /*Q of A, B*/ + 2 * kStages * kTileBytes /*K, V*/ +
                               sizeof(Bars);
 
 inline size_t mma_smem_bytes(int batch) { return kSmemFixed + sizeof(int) * (5 * (size_t)batch + 2); }
@@ -203,8 +207,10 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
     return r;
 }
 
+// A work item: up to two consecutive row tiles (A, B) of one (sequence, kv head).  They share every
+// K/V tile that is loaded; B may be missing (rows[1] == 0).
 struct Item {
-    int b, kvh, mt, n, L, rows_total, r_begin, rows_here, kv_len, ntiles, qrow0;
+    int b, kvh, n, L, rows_total, r_begin, rows[2], kv_len, ntiles, qrow0;
 };
 
 template <int G>
@@ -221,14 +227,15 @@ __device__ __forceinline__ bool get_item(int item, int total, const int *pref, c
     it.n = a.q_lens[sb];
     it.L = a.seq_lens[sb];
     it.rows_total = it.n * G;
-    const int mtiles = (it.rows_total + kBM - 1) / kBM;
+    const int pairs = (it.rows_total + 2 * kBM - 1) / (2 * kBM);
     const int r = item - pref[lo];
-    it.kvh = r / mtiles;
-    it.mt = r - it.kvh * mtiles;
-    it.r_begin = it.mt * kBM;
-    it.rows_here = min(kBM, it.rows_total - it.r_begin);
-    const int i_last = (it.r_begin + it.rows_here - 1) / G;
-    it.kv_len = it.L - it.n + i_last + 1;
+    it.kvh = r / pairs;
+    const int pt = r - it.kvh * pairs;
+    it.r_begin = pt * 2 * kBM;
+    it.rows[0] = min(kBM, it.rows_total - it.r_begin);
+    it.rows[1] = max(0, min(kBM, it.rows_total - it.r_begin - kBM));
+    const int i_last = (it.r_begin + it.rows[0] + it.rows[1] - 1) / G;
+    it.kv_len = it.L - it.n + i_last + 1;   // keys the pair's last row sees
     it.ntiles = (it.kv_len + kBN - 1) / kBN;
     it.qrow0 = row0[sb];
     return true;
@@ -239,8 +246,7 @@ __global__ void __launch_bounds__(kThreads, 1)
 chunk_mma_kernel(const MmaArgs a, const __grid_constant__ CUtensorMap k_map, const __grid_constant__ CUtensorMap v_map) {
     extern __shared__ char smem_raw[];
     char *base = reinterpret_cast<char *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-    char *q_s = base;                                  // [2 halves][128 rows][128 B]
-    char *p_s = base + kTileBytes;
+    char *q_s = base;                                  // [row tile A, B][2 halves][128 rows][128 B]
     char *k_s = base + 2 * kTileBytes;                 // [stage][2 halves][128 keys][128 B]
     char *v_s = k_s + kStages * kTileBytes;
     Bars *bars = reinterpret_cast<Bars *>(v_s + kStages * kTileBytes);
@@ -254,7 +260,7 @@ chunk_mma_kernel(const MmaArgs a, const __grid_constant__ CUtensorMap k_map, con
     const int B = a.batch, Hkv = a.Hkv;
 
     if (tid == 0) {
-        mbar_init(&bars->q_full, kSoftmaxThreads);
+        mbar_init(&bars->q_full, 2 * kSoftmaxThreads);
         for (int s = 0; s < kStages; ++s) {
             mbar_init(&bars->k_full[s], 1);
             mbar_init(&bars->v_full[s], 1);
@@ -262,11 +268,13 @@ chunk_mma_kernel(const MmaArgs a, const __grid_constant__ CUtensorMap k_map, con
         }
         mbar_init(&bars->s_full[0], 1);
         mbar_init(&bars->s_full[1], 1);
-        mbar_init(&bars->p_full, kSoftmaxThreads);
-        mbar_init(&bars->o_full, 1);
+        mbar_init(&bars->p_full[0], kSoftmaxThreads);
+        mbar_init(&bars->p_full[1], kSoftmaxThreads);
+        mbar_init(&bars->o_full[0], 1);
+        mbar_init(&bars->o_full[1], 1);
         for (int i = 0; i < kItemSlots; ++i) {
             mbar_init(&bars->item_full[i], 1);
-            mbar_init(&bars->item_empty[i], 1 + kSoftmaxThreads);
+            mbar_init(&bars->item_empty[i], 1 + 2 * kSoftmaxThreads);
         }
         bars->abort = 0;
         mbar_fence_init();
@@ -276,7 +284,8 @@ chunk_mma_kernel(const MmaArgs a, const __grid_constant__ CUtensorMap k_map, con
     for (int b = tid; b < B; b += kThreads) {
         const int n = a.q_lens[b], L = a.seq_lens[b];
         int items = 0;
-        if (n >= 2 && n * G >= a.min_rows && L >= n && L <= a.max_pages * kPage) items = Hkv * ((n * G + kBM - 1) / kBM);
+        if (n >= 2 && n * G >= a.min_rows && L >= n && L <= a.max_pages * kPage)
+            items = Hkv * ((n * G + 2 * kBM - 1) / (2 * kBM));
         itm[b] = items;
         key[b] = items > 0 ? L : -1;
         row0[b + 1] = n > 0 ? n : 0;
@@ -317,14 +326,14 @@ chunk_mma_kernel(const MmaArgs a, const __grid_constant__ CUtensorMap k_map, con
     const int total = pref[B];
     if ((int)blockIdx.x >= total) return;  // nothing for this CTA; no TMEM taken, no barrier pending
 
-    if (warp == 5) tmem_alloc(&bars->tmem_base, kTmemCols);
+    if (warp == kMmaWarp) tmem_alloc(&bars->tmem_base, kTmemCols);
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = bars->tmem_base;
     volatile int *abort = &bars->abort;
 
-    if (warp == 4) {
+    if (warp == kTmaWarp) {
         // ===================================== TMA producer =========================================
         uint32_t it = 0;  // KV tiles issued so far
         Item w;
@@ -374,12 +383,16 @@ chunk_mma_kernel(const MmaArgs a, const __grid_constant__ CUtensorMap k_map, con
                 __syncwarp();
             }
         }
-    } else if (warp == 5) {
+    } else if (warp == kMmaWarp) {
         // ====================================== MMA issue ===========================================
+        // Per KV tile: S_A = Q_A K^T, S_B = Q_B K^T, then -- as each softmax group delivers its P --
+        // O_A += P_A V and O_B += P_B V.  The next tile's Q K^T of a row tile is issued right after
+        // that row tile's P V, so the tensor core works for one row tile while the other one's
+        // softmax group is busy.
         if (lane == 0) {
             constexpr uint32_t idesc_qk = instr_desc(false), idesc_pv = instr_desc(true);
             const uint32_t q_addr = smem_u32(q_s);
-            uint32_t it = 0, nitem = 0;
+            uint32_t it = 0, nitem = 0, itg[2] = {0u, 0u};  // KV tiles so far: all, per row tile
             Item w;
             for (;; ++nitem) {
                 const uint32_t slot = nitem % kItemSlots, qpar = (nitem / kItemSlots) & 1u;
@@ -388,53 +401,66 @@ chunk_mma_kernel(const MmaArgs a, const __grid_constant__ CUtensorMap k_map, con
                 mbar_arrive(&bars->item_empty[slot]);
                 if (!get_item<G>(item, total, pref, row0, sorted, B, Hkv, a, w)) break;
                 mbar_wait(&bars->q_full, nitem & 1u, abort, a.status);
-                // S = Q K^T of tile `itx` into S buffer itx & 1: 8 steps of 16 dims, 4 per 64-dim half;
-                // K-major operands, SBO = 8 rows.  Issued one tile ahead, so that it runs under the
-                // softmax of the tile before it.
-                auto issue_qk = [&](uint32_t itx) {
-                    const uint32_t s = itx % kStages, par = (itx / kStages) & 1u;
+                const bool has_b = w.rows[1] > 0;
+                // S of row tile g for KV tile `itx`: 8 steps of 16 dims, 4 per 64-dim half; K-major
+                // operands, SBO = 8 rows
+                auto issue_qk = [&](int g, uint32_t itx) {
+                    const uint32_t s = itx % kStages;
                     const uint32_t k_addr = smem_u32(k_s + s * kTileBytes);
-                    mbar_wait(&bars->k_full[s], par, abort, a.status);
                     tc_fence_after();
 #pragma unroll
                     for (int ks = 0; ks < kD / 16; ++ks) {
                         const uint32_t off = (ks >> 2) * kHalfBytes + (ks & 3) * 32;
-                        mma_f16_ss(tmem + (itx & 1u) * kBN, smem_desc(q_addr + off, 16, 1024),
+                        mma_f16_ss(tmem + g * kBN, smem_desc(q_addr + g * kTileBytes + off, 16, 1024),
                                    smem_desc(k_addr + off, 16, 1024), idesc_qk, ks > 0 ? 1u : 0u);
                     }
-                    mma_commit(&bars->s_full[itx & 1u]);
+                    mma_commit(&bars->s_full[g]);
                 };
-                issue_qk(it);
-                for (int j = 0; j < w.ntiles; ++j, ++it) {
-                    const uint32_t s = it % kStages, par = (it / kStages) & 1u;
+                // O of row tile g += P V for KV tile `itx`: 8 steps of 16 keys; P from TMEM (first 64
+                // columns of the tile's S, 8 columns per step); V MN-major: 64-dim halves LBO apart,
+                // 8-key groups SBO apart
+                auto issue_pv = [&](int g, uint32_t itx, bool first) {
+                    const uint32_t s = itx % kStages;
                     const uint32_t v_addr = smem_u32(v_s + s * kTileBytes);
-                    // the other S buffer was read by the softmax of tile it - 1, which ended before the
-                    // p_full this thread waited for in the previous iteration
-                    if (j + 1 < w.ntiles) issue_qk(it + 1);
-                    // ---- O += P V: 8 steps of 16 keys; P K-major; V MN-major: 64-dim halves LBO apart,
-                    //      8-key groups SBO apart
-                    mbar_wait(&bars->p_full, it & 1u, abort, a.status);
-                    mbar_wait(&bars->v_full[s], par, abort, a.status);
+                    mbar_wait(&bars->p_full[g], itg[g] & 1u, abort, a.status);
                     tc_fence_after();
 #pragma unroll
-                    for (int ks = 0; ks < kBN / 16; ++ks) {
-                        // P of this tile sits in the first 64 columns of its S buffer, 16 keys = 8 columns
-                        mma_f16_ts(tmem + kOCol, tmem + (it & 1u) * kBN + ks * 8,
+                    for (int ks = 0; ks < kBN / 16; ++ks)
+                        mma_f16_ts(tmem + kOCol + g * kBN, tmem + g * kBN + ks * 8,
                                    smem_desc(v_addr + ks * 2 * 1024, kHalfBytes, 1024), idesc_pv,
-                                   (j > 0 || ks > 0) ? 1u : 0u);
+                                   (!first || ks > 0) ? 1u : 0u);
+                    mma_commit(&bars->o_full[g]);
+                    ++itg[g];
+                };
+                mbar_wait(&bars->k_full[it % kStages], (it / kStages) & 1u, abort, a.status);
+                issue_qk(0, it);
+                if (has_b) issue_qk(1, it);
+                for (int j = 0; j < w.ntiles; ++j, ++it) {
+                    const uint32_t s = it % kStages, par = (it / kStages) & 1u;
+                    const bool more = j + 1 < w.ntiles;
+                    if (more) mbar_wait(&bars->k_full[(it + 1) % kStages], ((it + 1) / kStages) & 1u, abort, a.status);
+                    mbar_wait(&bars->v_full[s], par, abort, a.status);
+                    issue_pv(0, it, j == 0);
+                    if (more) issue_qk(0, it + 1);
+                    if (has_b) {
+                        issue_pv(1, it, j == 0);
+                        if (more) issue_qk(1, it + 1);
                     }
-                    mma_commit(&bars->kv_empty[s]);
-                    mma_commit(&bars->o_full);
+                    mma_commit(&bars->kv_empty[s]);  // K and V of this tile have been read by everything issued so far
                 }
             }
         }
         __syncwarp();
     } else {
         // ================================ softmax and epilogue ====================================
-        const uint32_t lane_base = (uint32_t)(warp * 32) << 16;  // this warp's TMEM lane quadrant
-        const uint32_t o_tmem = tmem + lane_base + kOCol;
-        const int swz = tid & 7;
-        uint32_t it = 0, nitem = 0;
+        // two groups of 128 threads: group g owns row tile g; thread tg of a group owns TMEM lane tg
+        const int grp = warp >> 2, tg = tid & (kSoftmaxThreads - 1);
+        const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;  // this warp's TMEM lane quadrant
+        const uint32_t s_tmem = tmem + lane_base + grp * kBN;
+        const uint32_t o_tmem = tmem + lane_base + kOCol + grp * kBN;
+        char *q_tile = q_s + grp * kTileBytes;
+        const int swz = tg & 7;
+        uint32_t it = 0, itg = 0, nitem = 0;  // KV tiles so far: of all items, of items that had this row tile
         Item w;
         for (;; ++nitem) {
             const uint32_t slot = nitem % kItemSlots, qpar = (nitem / kItemSlots) & 1u;
@@ -442,29 +468,33 @@ chunk_mma_kernel(const MmaArgs a, const __grid_constant__ CUtensorMap k_map, con
             const int item = bars->item_id[slot];
             mbar_arrive(&bars->item_empty[slot]);
             if (!get_item<G>(item, total, pref, row0, sorted, B, Hkv, a, w)) break;
-            const bool row_ok = tid < w.rows_here;
-            const int r = min(w.r_begin + tid, w.rows_total - 1);
+            const int rows_here = w.rows[grp];
+            const bool row_ok = tg < rows_here;
+            const int r = min(w.r_begin + grp * kBM + tg, w.rows_total - 1);
             const int tok = r / G, head = r - tok * G;
             const int lim = w.L - w.n + tok + 1;  // keys this row may see
             const size_t grow = ((size_t)(w.qrow0 + tok) * a.Hq + w.kvh * G + head) * kD;
-            // ---- Q tile: row `tid`, 16 chunks of 8 dims, chunk c of a half stored at c ^ (row & 7)
+            // ---- Q tile: row `tg`, 16 chunks of 8 dims, chunk c of a half stored at c ^ (row & 7)
             {
                 const uint4 *src = reinterpret_cast<const uint4 *>(a.q + grow * 2);
 #pragma unroll
                 for (int c = 0; c < 16; ++c) {
                     const uint4 v = row_ok ? __ldg(src + c) : make_uint4(0, 0, 0, 0);
-                    *reinterpret_cast<uint4 *>(q_s + (c >> 3) * kHalfBytes + tid * 128 + (((c & 7) ^ swz) << 4)) = v;
+                    *reinterpret_cast<uint4 *>(q_tile + (c >> 3) * kHalfBytes + tg * 128 + (((c & 7) ^ swz) << 4)) = v;
                 }
                 fence_async_smem();
                 mbar_arrive(&bars->q_full);
             }
+            if (rows_here == 0) {  // this item has no second row tile: nothing is issued for it
+                it += w.ntiles;
+                continue;
+            }
             float m_used = -INFINITY, l_sum = 0.f;
-            for (int j = 0; j < w.ntiles; ++j, ++it) {
+            for (int j = 0; j < w.ntiles; ++j, ++it, ++itg) {
                 const uint32_t s = it % kStages, par = (it / kStages) & 1u;
                 const int key0 = j * kBN;
                 const int nvis = lim - key0;  // columns < nvis are visible to this row (may be <= 0)
-                const uint32_t s_tmem = tmem + lane_base + (it & 1u) * kBN;
-                mbar_wait(&bars->s_full[it & 1u], (it >> 1) & 1u, abort, a.status);
+                mbar_wait(&bars->s_full[grp], itg & 1u, abort, a.status);
                 tc_fence_after();
                 // ---- pass 1: row max of the visible scores
                 float mx = -INFINITY;
@@ -492,11 +522,8 @@ chunk_mma_kernel(const MmaArgs a, const __grid_constant__ CUtensorMap k_map, con
                     m_used = m_tile;
                 }
                 if (__any_sync(0xffffffffu, rescale)) {
-                    // O is still being accumulated until the previous tile's second product is done.
-                    // (s_full of this tile was committed after the product before that one, so this
-                    // wait is never more than one phase behind its barrier.)
-                    mbar_wait(&bars->o_full, (it - 1u) & 1u, abort, a.status);
-                    tc_fence_after();
+                    // O of the previous tiles is complete: this tile's S was issued, and committed,
+                    // after the previous tile's second product of this row tile
 #pragma unroll 1
                     for (int c4 = 0; c4 < 4; ++c4) {
                         uint32_t v[32];
@@ -536,10 +563,10 @@ chunk_mma_kernel(const MmaArgs a, const __grid_constant__ CUtensorMap k_map, con
                 // ---- V rows past the last visible key of the item (stale slots, pages never loaded)
                 //      must not reach the tensor core, not even times zero
                 const int nvalid = w.kv_len - key0;
-                if (nvalid < kBN) {
+                if (nvalid < kBN && grp == 0) {   // group A always exists and its P is waited for first
                     mbar_wait(&bars->v_full[s], par, abort, a.status);
-                    if (tid >= nvalid) {
-                        char *vrow = v_s + s * kTileBytes + tid * 128;
+                    if (tg >= nvalid) {
+                        char *vrow = v_s + s * kTileBytes + tg * 128;
 #pragma unroll
                         for (int c = 0; c < 8; ++c) {
                             *reinterpret_cast<uint4 *>(vrow + c * 16) = make_uint4(0, 0, 0, 0);
@@ -549,10 +576,10 @@ chunk_mma_kernel(const MmaArgs a, const __grid_constant__ CUtensorMap k_map, con
                 }
                 fence_async_smem();
                 tc_fence_before();
-                mbar_arrive(&bars->p_full);
+                mbar_arrive(&bars->p_full[grp]);
             }
             // ---- epilogue: O / l, bf16, one 256-byte row per thread
-            mbar_wait(&bars->o_full, (it - 1u) & 1u, abort, a.status);
+            mbar_wait(&bars->o_full[grp], (itg - 1u) & 1u, abort, a.status);
             tc_fence_after();
             const float inv_l = 1.0f / l_sum;
             uint4 *dst = reinterpret_cast<uint4 *>(a.out + grow * 2);
@@ -580,7 +607,7 @@ chunk_mma_kernel(const MmaArgs a, const __grid_constant__ CUtensorMap k_map, con
     // ---- teardown: everyone is done with TMEM before the allocating warp frees it ------------------
     tc_fence_before();
     __syncthreads();
-    if (warp == 5) {
+    if (warp == kMmaWarp) {
         tc_fence_after();
         tmem_dealloc(tmem, kTmemCols);
     }

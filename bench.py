@@ -287,6 +287,7 @@ def run_ours(args):
                         "us_per_call": round(ms2 / max(20, args.steps // 4) / per_step * 1e3, 3)}
                 result["target_shaped_decode"] = run_target_decode(ctx, dev, peak)
                 result["step_scoring"] = run_step_scoring(ctx, dev)
+                result["mixed_loop"] = run_mixed_loop(ctx, dev)
             result["cpu_baseline"] = run_cpu_baseline(work)
     if dist:
         dist.barrier()
@@ -386,6 +387,42 @@ def run_step_scoring(ctx, dev):
     return {"steps_scored_routed_per_s": res, "escalation_rate": esc, "layer_calls_per_step": 1,
             "route_only_steps_per_s": round(shape.batch / (ms_route / 200 * 1e-3), 1),
             "kv_tokens": b["tokens"], "rows": int(inp.q_lens.sum())}
+
+
+def run_mixed_loop(ctx, dev):
+    """Supplementary: the mixed serving loop (64 sequences, prefixes lognormal up to 64k, 10 iterations; in each
+    half the sequences decode one token and half score a step of 16..128 tokens; router at tau 0.5;
+    escalated steps are rolled back).  One layer call per iteration; lengths never leave the device."""
+    m = wl.make_mixed_loop(device=dev)
+    B = m.shape.batch
+    outs = [torch.empty_like(q) for q in m.q]
+    step_lens = [torch.where(ql > 1, ql, torch.zeros_like(ql)) for ql in m.q_lens]
+    max_q = [int(ql.max()) for ql in m.q_lens]
+    scores = torch.empty(B, dtype=torch.float32, device=dev)
+    dec = torch.empty(B, dtype=torch.uint8, device=dev)
+    seq = m.seq_lens0.clone()
+
+    def loop():
+        seq.copy_(m.seq_lens0)
+        for it in range(len(m.q_lens)):
+            seq.add_(m.q_lens[it])  # the new tokens' K/V are in place: append (outside the path)
+            ctx.attn(m.q[it], m.k_pages, m.v_pages, m.block_table, seq, m.q_lens[it], max_q[it], out=outs[it])
+            ctx.route(m.hidden[it], m.w, m.b, m.tau, scores=scores, decisions=dec)
+            ctx.rollback(seq, step_lens[it], dec)
+
+    ms = time_steps(loop, 5, 3) / 5
+    scored = sum(int((ql > 1).sum()) for ql in m.q_lens)
+    # KV tokens attended: replay the lengths on the host
+    kv = 0
+    esz = 2 * 2 * m.shape.num_kv_heads * m.shape.head_dim
+    loop()
+    torch.cuda.synchronize()
+    kv_tokens = int(m.seq_lens0.sum()) * len(m.q_lens)  # lower bound: the prefixes alone, every iteration
+    return {"iterations": len(m.q_lens), "ms_per_loop": round(ms, 3),
+            "steps_scored_routed_per_s": round(scored / (ms * 1e-3), 1),
+            "decode_tokens_per_s": round((B * len(m.q_lens) - scored) / (ms * 1e-3), 1),
+            "kv_gbs_lower_bound": round(kv_tokens * esz / (ms * 1e-3) / 1e9, 1),
+            "device_status_bits": ctx.poll_status()}
 
 
 def run_cpu_baseline(work: DecodeWorkload):

@@ -37,24 +37,28 @@ def build(force: bool = False) -> Path:
     return _LIB
 
 
+def bind(lib):
+    """Declare the C signatures on a loaded library (the built one, or a variant a test compiled)."""
+    c_int, c_long, c_dbl, vp = ctypes.c_int, ctypes.c_long, ctypes.c_double, ctypes.c_void_p
+    lib.oracle_num_threads.restype = c_int
+    lib.oracle_attn.restype = ctypes.c_uint
+    lib.oracle_attn.argtypes = [c_int, c_int, c_int, c_int, c_int, c_int, c_long, c_int,
+                            vp, vp, vp, vp, vp, vp, c_dbl, vp]
+    lib.oracle_attn_row_probs.restype = ctypes.c_uint
+    lib.oracle_attn_row_probs.argtypes = [c_int, c_int, c_int, c_int, c_int, c_long, c_int,
+                                      vp, vp, vp, vp, c_long, c_int, c_long, c_dbl, vp, vp]
+    lib.oracle_route.restype = None
+    lib.oracle_route.argtypes = [c_int, c_int, c_int, vp, vp, c_dbl, ctypes.c_float, vp, vp]
+    lib.oracle_rollback.restype = ctypes.c_uint
+    lib.oracle_rollback.argtypes = [c_int, vp, vp, vp]
+    return lib
+
+
 def _load():
     global _lib
     if _lib is None:
         build()
-        lib = ctypes.CDLL(str(_LIB))
-        c_int, c_long, c_dbl, vp = ctypes.c_int, ctypes.c_long, ctypes.c_double, ctypes.c_void_p
-        lib.oracle_num_threads.restype = c_int
-        lib.oracle_attn.restype = ctypes.c_uint
-        lib.oracle_attn.argtypes = [c_int, c_int, c_int, c_int, c_int, c_int, c_long, c_int,
-                                    vp, vp, vp, vp, vp, vp, c_dbl, vp]
-        lib.oracle_attn_row_probs.restype = ctypes.c_uint
-        lib.oracle_attn_row_probs.argtypes = [c_int, c_int, c_int, c_int, c_int, c_long, c_int,
-                                              vp, vp, vp, vp, c_long, c_int, c_long, c_dbl, vp, vp]
-        lib.oracle_route.restype = None
-        lib.oracle_route.argtypes = [c_int, c_int, c_int, vp, vp, c_dbl, ctypes.c_float, vp, vp]
-        lib.oracle_rollback.restype = ctypes.c_uint
-        lib.oracle_rollback.argtypes = [c_int, vp, vp, vp]
-        _lib = lib
+        _lib = bind(ctypes.CDLL(str(_LIB)))
     return _lib
 
 

@@ -1,0 +1,77 @@
+"""The pins do bite: each plausible mistake, planted in a copy of the oracle's C source and compiled on
+the CPU, is caught by at least one of the pin checks below (the same kinds of checks as in
+test_oracle_attn.py / test_oracle_route.py, run against the mutated build)."""
+import ctypes
+import math
+import subprocess
+from pathlib import Path
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import oracle
+from paper_2512_05033_b200 import workloads as wl
+from tests.test_oracle_attn import brute_force
+
+SRC = (Path(oracle.__file__).parent / "arb_oracle.c").read_text()
+
+MUTATIONS = {
+    "scale dropped": ("s[j] = scale * acc;", "s[j] = acc;"),
+    "causal bound one short": ("long nkeys = pos + 1;", "long nkeys = pos > 0 ? pos : 1;"),
+    "kv head by modulo": ("int kvh = h / g;", "int kvh = h % Hkv;"),
+    "slot off by one": ("size_t koff = kv_offset(page, kvh, (int)(j % P), Hkv, P, D);",
+                        "size_t koff = kv_offset(page, kvh, (int)((j + 1) % P), Hkv, P, D);"),
+    "V read from the K offset of the next dim": ("out_row[d] += p * widen(v_pages, dtype, voff + d);",
+                                                 "out_row[d] += p * widen(v_pages, dtype, voff + (d + 1) % D);"),
+    "no max subtraction and no normalisation": ("double p = s[j] / Z;", "double p = s[j];"),
+    "bf16 widened with the wrong shift": ("<< 16;", "<< 15;"),
+    "sigmoid sign": ("1.0 / (1.0 + exp(-z))", "1.0 / (1.0 + exp(z))"),
+    "bias dropped": ("double z = b;", "double z = 0.0;"),
+    "tie escalates": ("((float)sc > tau)", "((float)sc >= tau)"),
+    "rollback adds": ("long r = (long)seq_lens[i] - (long)step_lens[i];", "long r = (long)seq_lens[i] + (long)step_lens[i];"),
+    "rollback ignores decisions": ("if (decisions && !decisions[i]) continue;", ""),
+}
+
+
+def _variant(tmp_path, name, old, new):
+    assert SRC.count(old) >= 1, name
+    c = tmp_path / "mut.c"
+    so = tmp_path / f"mut_{abs(hash(name))}.so"
+    c.write_text(SRC.replace(old, new))
+    subprocess.check_call(["gcc", "-O1", "-fopenmp", "-fPIC", "-shared", "-std=c11", "-o", str(so), str(c), "-lm"])
+    return oracle.bind(ctypes.CDLL(str(so)))
+
+
+def _pins_pass() -> bool:
+    """A compact set of pins; returns False as soon as one fails."""
+    try:
+        for case in [(2, 6, 2, 64, torch.float32, [17, 64], [5, 16]), (3, 12, 2, 128, torch.bfloat16, [33, 1, 50], [1, 1, 7])]:
+            B, Hq, Hkv, D, dt, sl, ql = case
+            inp = wl.small_attn_case(B, Hq, Hkv, D, dt, sl, ql, seed=11)
+            out, st = oracle.attn(inp.q, inp.k_pages, inp.v_pages, inp.block_table, inp.seq_lens, inp.q_lens)
+            if st or not np.allclose(out, brute_force(inp), rtol=0, atol=1e-12):
+                return False
+        hidden = np.zeros((3, 8), dtype=np.float32)
+        w = np.ones(8, dtype=np.float32)
+        hidden[1, 0] = math.log(3.0) - 0.25
+        hidden[2, 0] = -0.25
+        s, d = oracle.route(hidden, w, 0.25, 0.5)          # z = 0.25, ln 3, 0
+        if not (abs(s[1] - 0.75) < 1e-7 and s[2] == 0.5 and list(d) == [1, 1, 0]):
+            return False
+        new, _ = oracle.rollback(np.array([100, 50]), np.array([10, 20]), np.array([1, 0], dtype=np.uint8))
+        return list(new) == [90, 50]
+    except Exception:
+        return False
+
+
+def test_the_unmutated_oracle_passes_the_compact_pins():
+    assert _pins_pass()
+
+
+@pytest.mark.parametrize("name", sorted(MUTATIONS))
+def test_mutation_is_caught(name, tmp_path, monkeypatch):
+    old, new = MUTATIONS[name]
+    oracle._load()
+    monkeypatch.setattr(oracle, "_lib", _variant(tmp_path, name, old, new))
+    assert not _pins_pass(), f"no pin noticed: {name}"

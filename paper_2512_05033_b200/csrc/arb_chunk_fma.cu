@@ -29,6 +29,7 @@ struct ChunkArgs {
     int batch, Hq, Hkv, num_pages, max_pages;
     int n_lo, n_hi;  // this kernel owns the sequences with n_lo <= q_len <= n_hi ...
     int skip_rows;   // ... except valid ones with q_len * group >= skip_rows (> 0): the tensor-core kernel has them
+    const int *needed;  // with skip_rows > 0: written by the tensor-core kernel, 0 = nothing is left for this one
     float scale_log2;
 };
 
@@ -48,6 +49,7 @@ __global__ void __launch_bounds__(kThreads) chunk_fma_kernel(const ChunkArgs a) 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int B = a.batch;
     const int row = blockIdx.x / a.Hkv, kvh = blockIdx.x - row * a.Hkv;
+    if (a.skip_rows > 0 && a.needed != nullptr && *a.needed == 0) return;  // the usual case: every chunk was large
 
     if (tid == 0) row0[0] = 0;
     for (int b = tid; b < B; b += kThreads) row0[b + 1] = max(a.q_lens[b], 0);
@@ -217,6 +219,7 @@ arb_status launch_chunk_fma(Ctx *ctx, const arb_attn_params &p, const void *q, c
                             const void *v_pages, const int32_t *block_table, const int32_t *seq_lens,
                             const int32_t *q_lens, void *out, int n_lo, int n_hi, int skip_rows,
                             cudaStream_t stream) {
+    const int *needed = skip_rows > 0 ? ctx->rot + (size_t)kRotSets * kRotCounters + kRotSets + 2 : nullptr;
     ChunkArgs a;
     a.q = static_cast<const char *>(q);
     a.k_pages = static_cast<const char *>(k_pages);
@@ -234,6 +237,7 @@ arb_status launch_chunk_fma(Ctx *ctx, const arb_attn_params &p, const void *q, c
     a.n_lo = n_lo;
     a.n_hi = n_hi;
     a.skip_rows = skip_rows;
+    a.needed = needed;
     const float scale = p.softmax_scale > 0.f ? p.softmax_scale : 1.0f / sqrtf((float)p.head_dim);
     a.scale_log2 = scale * 1.4426950408889634f;
     const int g = p.num_q_heads / p.num_kv_heads;

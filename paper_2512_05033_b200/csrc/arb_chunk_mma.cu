@@ -59,7 +59,8 @@ struct MmaArgs {
     uint32_t *status;
     int batch, Hq, Hkv, num_pages, max_pages;
     int min_rows;  // sequences with q_len * group >= min_rows are handled here
-    int *work_counter;  // next work item; zeroed on the stream before the launch
+    int *work_counter;  // [0] next work item, [1] set if a chunk sequence is left for the CUDA-core kernel;
+                        // both zeroed on the stream before the launch
     float scale_log2;
 };
 
@@ -286,6 +287,7 @@ chunk_mma_kernel(const MmaArgs a, const __grid_constant__ CUtensorMap k_map, con
         int items = 0;
         if (n >= 2 && n * G >= a.min_rows && L >= n && L <= a.max_pages * kPage)
             items = Hkv * ((n * G + 2 * kBM - 1) / (2 * kBM));
+        if (blockIdx.x == 0 && n >= 2 && items == 0) atomicOr(a.work_counter + 1, 1);  // small, or invalid lengths
         itm[b] = items;
         key[b] = items > 0 ? L : -1;
         row0[b + 1] = n > 0 ? n : 0;
@@ -689,7 +691,7 @@ arb_status launch_chunk_mma(Ctx *ctx, const arb_attn_params &p, const void *q, c
     a.max_pages = p.max_pages_per_seq;
     a.min_rows = kChunkMmaMinRows;
     a.work_counter = ctx->rot + (size_t)kRotSets * kRotCounters + kRotSets + 1;
-    if (cudaMemsetAsync(a.work_counter, 0, sizeof(int), stream) != cudaSuccess) return ARB_ERR_CUDA;
+    if (cudaMemsetAsync(a.work_counter, 0, 2 * sizeof(int), stream) != cudaSuccess) return ARB_ERR_CUDA;
     const float scale = p.softmax_scale > 0.f ? p.softmax_scale : 1.0f / sqrtf((float)p.head_dim);
     a.scale_log2 = scale * 1.4426950408889634f;
     const int g = p.num_q_heads / p.num_kv_heads;

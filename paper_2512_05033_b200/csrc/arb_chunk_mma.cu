@@ -48,10 +48,12 @@ constexpr uint32_t kTmemCols = 512;         // S of tile A: columns 0..127, S of
 constexpr uint32_t kOCol = 256;
 constexpr float kRescaleThreshold = 8.0f;   // log2 units
 constexpr int kItemSlots = 8;               // work items announced ahead of their use
+constexpr int kPrefetchTiles = 4;            // K/V tiles asked into L2 ahead of the ring
 constexpr int kSortMaxBatch = 256;          // up to this batch size sequences are served longest first
 
 struct MmaArgs {
     const char *q;
+    const char *k_pool, *v_pool;  // for L2 prefetches; the tiles themselves come through the tensor maps
     const int32_t *block_table;
     const int32_t *seq_lens;
     const int32_t *q_lens;
@@ -68,7 +70,8 @@ struct Bars {
     uint64_t q_full;             // both softmax groups wrote their Q tiles
     uint64_t k_full[kStages];    // TMA bytes of a K tile landed
     uint64_t v_full[kStages];
-    uint64_t kv_empty[kStages];  // the MMAs that read the stage have completed
+    uint64_t k_empty[kStages];   // the first products that read the K stage have completed
+    uint64_t v_empty[kStages];   // the second products that read the V stage have completed
     uint64_t s_full[2];          // S = Q K^T of row tile A / B is in TMEM
     uint64_t p_full[2];          // P of row tile A / B is in TMEM (over S)
     uint64_t o_full[2];          // O += P V of row tile A / B has completed
@@ -158,16 +161,19 @@ __device__ __forceinline__ void tma_box_load(void *dst_smem, const CUtensorMap *
 #define ARB_R32(v, o)                                                                                       \
     "=r"(v[o + 0]), "=r"(v[o + 1]), "=r"(v[o + 2]), "=r"(v[o + 3]), "=r"(v[o + 4]), "=r"(v[o + 5]), "=r"(v[o + 6]), \
         "=r"(v[o + 7])
-// 32 consecutive fp32 columns of this thread's TMEM lane
-__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&v)[32]) {
+// 32 consecutive fp32 columns of this thread's TMEM lane into v[O .. O + 31]
+template <int O, int N>
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&v)[N]) {
+    static_assert(O + 32 <= N, "range");
     asm volatile(
         "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
         "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
         "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
-        : ARB_R32(v, 0), ARB_R32(v, 8), ARB_R32(v, 16), ARB_R32(v, 24)
+        : ARB_R32(v, O + 0), ARB_R32(v, O + 8), ARB_R32(v, O + 16), ARB_R32(v, O + 24)
         : "r"(taddr)
         : "memory");
 }
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&v)[32]) { tmem_ld32<0, 32>(taddr, v); }
 #undef ARB_R32
 #define ARB_W8(v, o) "r"(v[o + 0]), "r"(v[o + 1]), "r"(v[o + 2]), "r"(v[o + 3]), "r"(v[o + 4]), "r"(v[o + 5]), "r"(v[o + 6]), "r"(v[o + 7])
 __device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&v)[32]) {
@@ -205,6 +211,12 @@ __device__ __forceinline__ float add_bf16x2(uint32_t w, float acc) {
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
     uint32_t r;
     asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+    return r;
+}
+
+__device__ __forceinline__ float max3(float a, float b, float c) {
+    float r;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));
     return r;
 }
 
@@ -265,7 +277,8 @@ chunk_mma_kernel(const MmaArgs a, const __grid_constant__ CUtensorMap k_map, con
         for (int s = 0; s < kStages; ++s) {
             mbar_init(&bars->k_full[s], 1);
             mbar_init(&bars->v_full[s], 1);
-            mbar_init(&bars->kv_empty[s], 1);
+            mbar_init(&bars->k_empty[s], 1);
+            mbar_init(&bars->v_empty[s], 1);
         }
         mbar_init(&bars->s_full[0], 1);
         mbar_init(&bars->s_full[1], 1);
@@ -352,9 +365,25 @@ chunk_mma_kernel(const MmaArgs a, const __grid_constant__ CUtensorMap k_map, con
             }
             item = __shfl_sync(0xffffffffu, item, 0);
             if (!get_item<G>(item, total, pref, row0, sorted, B, Hkv, a, w)) break;
+            // K and V tiles are asked into L2 kPrefetchTiles ahead of their load into the ring, so the
+            // ring (two tiles deep) only has to cover the L2 latency, not the DRAM latency
+            auto prefetch_tile = [&](int jt) {
+                if (jt >= w.ntiles) return;
+                const int np = min(kTilePages, (w.kv_len - jt * kBN + kPage - 1) / kPage);
+                const int pg = lane & 7;
+                if (lane < 16 && pg < np) {
+                    const int pf = a.block_table[(size_t)w.b * a.max_pages + jt * kTilePages + pg];
+                    if ((unsigned)pf < (unsigned)a.num_pages) {
+                        const char *src = (lane < 8 ? a.k_pool : a.v_pool) + ((size_t)pf * Hkv + w.kvh) * (kPage * kD * 2);
+                        asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(src), "r"(kPage * kD * 2) : "memory");
+                    }
+                }
+            };
+            for (int jt = 0; jt < kPrefetchTiles; ++jt) prefetch_tile(jt);
             for (int j = 0; j < w.ntiles; ++j, ++it) {
                 const uint32_t s = it % kStages, par = (it / kStages) & 1u;
                 const int npages = min(kTilePages, (w.kv_len - j * kBN + kPage - 1) / kPage);
+                prefetch_tile(j + kPrefetchTiles);
                 int pid = 0;
                 if (lane < npages) {
                     pid = a.block_table[(size_t)w.b * a.max_pages + j * kTilePages + lane];
@@ -363,24 +392,30 @@ chunk_mma_kernel(const MmaArgs a, const __grid_constant__ CUtensorMap k_map, con
                         pid = 0;
                     }
                 }
+                // lanes 0..15: (half, page) of K; the same lanes then issue V.  The K stage is free
+                // as soon as the first products of the tile before last have completed, the V stage
+                // only after its second products: two separate waits, in the order they are released.
+                const int pg = lane & 7, half = (lane >> 3) & 1;
+                const int row = (__shfl_sync(0xffffffffu, pid, pg) * Hkv + w.kvh) * kPage;
                 bool ok = true;
-                if (lane == 0) ok = mbar_wait(&bars->kv_empty[s], par ^ 1u, abort, a.status);
+                if (lane == 0) ok = mbar_wait(&bars->k_empty[s], par ^ 1u, abort, a.status);
                 ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
                 if (ok) {
-                    if (lane == 0) {
-                        mbar_arrive_expect_tx(&bars->k_full[s], (uint32_t)npages * 2u * kBoxBytes);
-                        mbar_arrive_expect_tx(&bars->v_full[s], (uint32_t)npages * 2u * kBoxBytes);
-                    }
+                    if (lane == 0) mbar_arrive_expect_tx(&bars->k_full[s], (uint32_t)npages * 2u * kBoxBytes);
                     __syncwarp();
-                    // lanes 0..15: (half, page) of K; the same lanes then issue V
-                    const int pg = lane & 7, half = (lane >> 3) & 1;
-                    const int row = (__shfl_sync(0xffffffffu, pid, pg) * Hkv + w.kvh) * kPage;
-                    if (lane < 16 && pg < npages) {
-                        char *kd = k_s + s * kTileBytes + half * kHalfBytes + pg * kBoxBytes;
-                        char *vd = v_s + s * kTileBytes + half * kHalfBytes + pg * kBoxBytes;
-                        tma_box_load(kd, &k_map, half * 64, row, &bars->k_full[s]);
-                        tma_box_load(vd, &v_map, half * 64, row, &bars->v_full[s]);
-                    }
+                    if (lane < 16 && pg < npages)
+                        tma_box_load(k_s + s * kTileBytes + half * kHalfBytes + pg * kBoxBytes, &k_map, half * 64, row,
+                                     &bars->k_full[s]);
+                }
+                __syncwarp();
+                if (lane == 0) ok = mbar_wait(&bars->v_empty[s], par ^ 1u, abort, a.status);
+                ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+                if (ok) {
+                    if (lane == 0) mbar_arrive_expect_tx(&bars->v_full[s], (uint32_t)npages * 2u * kBoxBytes);
+                    __syncwarp();
+                    if (lane < 16 && pg < npages)
+                        tma_box_load(v_s + s * kTileBytes + half * kHalfBytes + pg * kBoxBytes, &v_map, half * 64, row,
+                                     &bars->v_full[s]);
                 }
                 __syncwarp();
             }
@@ -437,6 +472,7 @@ chunk_mma_kernel(const MmaArgs a, const __grid_constant__ CUtensorMap k_map, con
                 mbar_wait(&bars->k_full[it % kStages], (it / kStages) & 1u, abort, a.status);
                 issue_qk(0, it);
                 if (has_b) issue_qk(1, it);
+                mma_commit(&bars->k_empty[it % kStages]);
                 for (int j = 0; j < w.ntiles; ++j, ++it) {
                     const uint32_t s = it % kStages, par = (it / kStages) & 1u;
                     const bool more = j + 1 < w.ntiles;
@@ -448,7 +484,9 @@ chunk_mma_kernel(const MmaArgs a, const __grid_constant__ CUtensorMap k_map, con
                         issue_pv(1, it, j == 0);
                         if (more) issue_qk(1, it + 1);
                     }
-                    mma_commit(&bars->kv_empty[s]);  // K and V of this tile have been read by everything issued so far
+                    // everything issued so far has read V of this tile and K of the next one
+                    mma_commit(&bars->v_empty[s]);
+                    if (more) mma_commit(&bars->k_empty[(it + 1) % kStages]);
                 }
             }
         }
@@ -498,23 +536,27 @@ chunk_mma_kernel(const MmaArgs a, const __grid_constant__ CUtensorMap k_map, con
                 const int nvis = lim - key0;  // columns < nvis are visible to this row (may be <= 0)
                 mbar_wait(&bars->s_full[grp], itg & 1u, abort, a.status);
                 tc_fence_after();
-                // ---- pass 1: row max of the visible scores
-                float mx = -INFINITY;
-#pragma unroll 1
-                for (int c4 = 0; c4 < 4; ++c4) {
-                    uint32_t v[32];
-                    tmem_ld32(s_tmem + c4 * 32, v);
-                    tmem_wait_ld();
-                    if (nvis >= (c4 + 1) * 32) {
+                // ---- the whole row of S (128 scores) comes into registers with one round trip
+                uint32_t v[kBN];
+                tmem_ld32<0>(s_tmem, v);
+                tmem_ld32<32>(s_tmem + 32, v);
+                tmem_ld32<64>(s_tmem + 64, v);
+                tmem_ld32<96>(s_tmem + 96, v);
+                tmem_wait_ld();
+                if (nvis < kBN) {  // causal edge or end of the sequence: hidden keys weigh exp2(-inf) = 0
 #pragma unroll
-                        for (int k = 0; k < 32; ++k) mx = fmaxf(mx, __uint_as_float(v[k]));
-                    } else {
-#pragma unroll
-                        for (int k = 0; k < 32; ++k)
-                            if (c4 * 32 + k < nvis) mx = fmaxf(mx, __uint_as_float(v[k]));
-                    }
+                    for (int k = 0; k < kBN; ++k)
+                        if (k >= nvis) v[k] = 0xff800000u;
                 }
-                const float m_tile = mx * a.scale_log2;  // -inf if this row sees nothing of the tile
+                // ---- row max, four independent chains of three-input maxima
+                float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+#pragma unroll
+                for (int k = 0; k < kBN; k += 8) {
+#pragma unroll
+                    for (int u = 0; u < 4; ++u)
+                        mx4[u] = max3(mx4[u], __uint_as_float(v[k + 2 * u]), __uint_as_float(v[k + 2 * u + 1]));
+                }
+                const float m_tile = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * a.scale_log2;  // -inf: sees nothing
                 float factor = 1.0f;
                 bool rescale = false;
                 if (m_tile > m_used + kRescaleThreshold || (m_used == -INFINITY && m_tile > -INFINITY)) {
@@ -528,39 +570,34 @@ chunk_mma_kernel(const MmaArgs a, const __grid_constant__ CUtensorMap k_map, con
                     // after the previous tile's second product of this row tile
 #pragma unroll 1
                     for (int c4 = 0; c4 < 4; ++c4) {
-                        uint32_t v[32];
-                        tmem_ld32(o_tmem + c4 * 32, v);
+                        uint32_t o[32];
+                        tmem_ld32(o_tmem + c4 * 32, o);
                         tmem_wait_ld();
 #pragma unroll
-                        for (int k = 0; k < 32; ++k) v[k] = __float_as_uint(__uint_as_float(v[k]) * factor);
-                        tmem_st32(o_tmem + c4 * 32, v);
+                        for (int k = 0; k < 32; ++k) o[k] = __float_as_uint(__uint_as_float(o[k]) * factor);
+                        tmem_st32(o_tmem + c4 * 32, o);
                     }
                     tmem_wait_st();
                 }
-                // ---- pass 2: P = exp2(scale * S - m), bf16, into the swizzled K-major P tile
+                // ---- P = exp2(scale * S - m), rounded to bf16 BEFORE it is summed, so the tensor
+                //      core's numerator and the fp32 denominator use the very same weights and the
+                //      result stays a true convex combination of V rows.  P overwrites S in place:
+                //      keys 32 c .. 32 c + 31 -> columns 16 c .. 16 c + 15 (all of S is in registers).
                 const float neg_m = (m_used == -INFINITY) ? 0.f : -m_used;
-#pragma unroll 1
+                float l4[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
                 for (int c4 = 0; c4 < 4; ++c4) {
-                    uint32_t v[32];
-                    tmem_ld32(s_tmem + c4 * 32, v);
-                    tmem_wait_ld();
-                    // The weights are rounded to bf16 BEFORE they are summed, so the tensor core's
-                    // numerator and the fp32 denominator use the very same weights and the result
-                    // stays a true convex combination of V rows.
                     uint32_t pk[16];
 #pragma unroll
                     for (int k = 0; k < 16; ++k) {
-                        const float e0 = fast_exp2(fmaf(__uint_as_float(v[2 * k]), a.scale_log2, neg_m));
-                        const float e1 = fast_exp2(fmaf(__uint_as_float(v[2 * k + 1]), a.scale_log2, neg_m));
-                        const uint32_t w = pack_bf16((c4 * 32 + 2 * k < nvis) ? e0 : 0.f,
-                                                     (c4 * 32 + 2 * k + 1 < nvis) ? e1 : 0.f);
-                        pk[k] = w;
-                        l_sum = add_bf16x2(w, l_sum);
+                        const float e0 = fast_exp2(fmaf(__uint_as_float(v[c4 * 32 + 2 * k]), a.scale_log2, neg_m));
+                        const float e1 = fast_exp2(fmaf(__uint_as_float(v[c4 * 32 + 2 * k + 1]), a.scale_log2, neg_m));
+                        pk[k] = pack_bf16(e0, e1);
+                        l4[k & 3] = add_bf16x2(pk[k], l4[k & 3]);
                     }
-                    // P overwrites S in place: keys 32 c4 .. 32 c4 + 31 -> columns 16 c4 .. 16 c4 + 15,
-                    // which this thread has already read
                     tmem_st16(s_tmem + c4 * 16, pk);
                 }
+                l_sum += (l4[0] + l4[1]) + (l4[2] + l4[3]);
                 tmem_wait_st();
                 // ---- V rows past the last visible key of the item (stale slots, pages never loaded)
                 //      must not reach the tensor core, not even times zero
@@ -679,6 +716,8 @@ arb_status launch_chunk_mma(Ctx *ctx, const arb_attn_params &p, const void *q, c
     if (!make_pool_map(&km, k_pages, p) || !make_pool_map(&vm, v_pages, p)) return ARB_ERR_CUDA;
     MmaArgs a;
     a.q = static_cast<const char *>(q);
+    a.k_pool = static_cast<const char *>(k_pages);
+    a.v_pool = static_cast<const char *>(v_pages);
     a.block_table = block_table;
     a.seq_lens = seq_lens;
     a.q_lens = q_lens;

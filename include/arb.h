@@ -89,9 +89,13 @@ typedef struct {
  * block_table, seq_lens, q_lens) is written by the kernel that precedes it on the stream.  The
  * decode kernel is then launched as a programmatic dependent of that kernel: it may start streaming
  * KV while its predecessor is still finishing, and waits for the predecessor's completion only
- * before its first write (out, workspace).  Results are the same as without the flag.  Typical
- * use: the per-layer calls of one decode token when q and the KV cache of every layer are ready.
- * Do not set it when the preceding kernel produces q, appends K/V or changes seq_lens.
+ * before its first write to `out` (and to the workspace, unless the workspace set it uses is known
+ * to be free).  A flagged call is taken to be one of a back-to-back series: a small one spreads
+ * over half as many CTAs as an unflagged call, so that more calls of the series are in flight at
+ * once; that changes where its sequences are split, so results agree with the unflagged call
+ * within rounding (same tolerances), not bit for bit.  The same flagged call always gives the same
+ * bits.  Typical use: independent decode calls queued behind one another whose q and KV cache are
+ * ready.  Do not set it when the preceding kernel produces q, appends K/V or changes seq_lens.
  * ARB_ATTN_NO_TENSOR_CORES: run decode and step chunks on the CUDA-core kernels even where the
  * tensor-core kernels apply (bf16, head_dim 128).  Same results within the stated tolerances; for
  * comparison runs and for keeping both paths under test.

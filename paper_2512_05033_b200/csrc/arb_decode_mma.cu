@@ -8,14 +8,21 @@
 // 8 ldmatrix + 16 mma for q.K and the same for P.V, about a tenth of the instructions, so the kernel
 // goes back to being bound by memory and latency.  The rows 8..15 of the tile stay zero (g <= 8).
 //
-// Everything around the arithmetic is the scheme of the CUDA-core decode kernel: flat page list cut
-// into equal ranges per CTA, one producer warp feeding a 16-stage ring, page groups owned by one
-// consumer warp each with its own online softmax, last-arriver split combine staged through the idle
-// ring.  Differences: K/V tiles arrive as tiled TMA boxes (16 rows x 64 dims, 128-byte swizzle, two
-// per tile) so that ldmatrix reads them without bank conflicts; P is rounded to bf16 for the second
-// product (and summed after rounding, so numerator and denominator agree); results of a segment are
-// parked in shared memory and written out after the CTA's last page, so the wait for the previous
-// kernel (programmatic dependent launch) comes once, after all streaming.
+// The streaming part is the scheme of the CUDA-core decode kernel: flat page list cut into equal
+// ranges per CTA, one producer warp feeding a 16-stage ring, pages owned by one consumer warp each
+// with its own online softmax.  Differences: K/V tiles arrive as tiled TMA boxes (16 rows x 64 dims,
+// 128-byte swizzle, two per tile) so that ldmatrix reads them without bank conflicts; P is rounded
+// to bf16 for the second product (and summed after rounding, so numerator and denominator agree);
+// results of a segment are parked in shared memory and written out after the CTA's last page, so
+// the wait for the previous kernel (programmatic dependent launch) comes once, after all streaming.
+//
+// The split combine is a kernel of its own (decode_combine_kernel, below), launched right behind
+// as a programmatic dependent.  Measured per-CTA timelines are the reason: with the combine inside
+// the decode kernel (partials, fence, arrival counter, last arriver reads everything back) the
+// CTAs of a 34 MB call spent 3 to 15 us after their last page in dependent round trips to a
+// loaded memory system, each holding 86 KB of shared memory that the next call's CTAs were
+// waiting for.  Now a decode CTA stores its partials and leaves; the kernel boundary makes them
+// visible, and the few light CTAs of the combine kernel are already resident when it happens.
 #include <cuda.h>  // CUtensorMap and its enums only; the encoder is looked up at run time
 
 #include "arb_common.cuh"
@@ -39,6 +46,8 @@ constexpr int kCtasPerSm = 2;
 constexpr int kParked = 2;      // segment results parked in shared memory before they are written
 constexpr int kSmallCallPages = 64;   // up to this many pages per SM a call runs one CTA per SM
 static_assert(kStages % (kConsWarps * 2 * kGroup) == 0, "a ring stage must always belong to the same warp");
+static_assert(kBatch <= kStages, "two producer lanes of one turn must never wait on the same stage: the later one "
+                                 "would be two phases ahead of the barrier and a parity wait cannot tell");
 
 struct Args {
     const char *q;
@@ -48,26 +57,22 @@ struct Args {
     char *out;
     float *part_o;    // [slots][G][D]
     float *part_ml;   // [slots][GP][2]
-    int *counters;
     uint32_t *status;
     int batch, Hq, Hkv, num_pages, max_pages;
+    int small_ctas;   // CTAs a small call spreads over
     float scale_log2;
     // workspace rotation (see launch_decode_mma): this call's generation number, the number of
-    // workspace sets, the generation of the newest completed call, this set's exit counter
+    // workspace sets, the generation of the newest completed call
     uint32_t gen;
     int sets;
     int force_wait;
     unsigned *done_gen;
-    int *exit_count;
 };
 
 struct Tail {
     uint64_t full[kStages];
     uint64_t empty[kStages];
-    uint64_t cbar[2];
-    float lsum[2 * kMaxGroup];   // per combine job and head: sum of the weighted sums
     int abort;
-    int flags[kParked];   // per parked segment: this CTA was the last to arrive
     int early;            // the workspace set is free: partials may be written before the predecessor is done
 };
 
@@ -93,6 +98,17 @@ size_t smem_bytes(int batch) {
 struct Segment {
     int b, kvh, pg0, pg1, L, bk, nparts, c_first;
 };
+
+// The cut of the flat (sequence, kv head, page) list into per-CTA ranges: both kernels of a call must
+// agree on it.  Small calls use the first `small_ctas` CTAs of the grid -- one per SM, or one per
+// two SMs for a call that runs back to back with its neighbours (see launch_decode_mma) -- and
+// large ones the whole grid.
+__device__ __forceinline__ int plan_chunk(int total, int grid, int small_ctas) {
+    const int one_per_sm = min(grid, small_ctas);
+    const int active = total <= one_per_sm * kSmallCallPages ? one_per_sm : grid;
+    const int chunk = (total + active - 1) / active;
+    return chunk < kMinChunk ? kMinChunk : chunk;
+}
 
 __device__ __forceinline__ bool next_segment(int &cur, int r1, const int *pref, const int *slen, int B, int Hkv,
                                              int chunk, Segment &s) {
@@ -122,7 +138,6 @@ __device__ __forceinline__ bool next_segment(int &cur, int r1, const int *pref, 
     return true;
 }
 
-__device__ __forceinline__ void fence_proxy_async_all() { asm volatile("fence.proxy.async;" ::: "memory"); }
 __device__ __forceinline__ void let_successor_start() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 __device__ __forceinline__ void wait_for_predecessor() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 
@@ -187,13 +202,15 @@ decode_mma_kernel(const Args a, const __grid_constant__ CUtensorMap k_map, const
     // arrival counters comes after it (see the CUDA-core decode kernel for the ordering argument).
     let_successor_start();
 
+    if (tid == kConsThreads) {  // the producer warp's first lane: descriptors on their way before the first copy needs them
+        asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&k_map)) : "memory");
+        asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&v_map)) : "memory");
+    }
     if (tid == 0) {
         for (int s = 0; s < kStages; ++s) {
             mbar_init(&tail->full[s], 1);
             mbar_init(&tail->empty[s], 1);
         }
-        mbar_init(&tail->cbar[0], 1);
-        mbar_init(&tail->cbar[1], 1);
         tail->abort = 0;
         mbar_fence_init();
         pref[0] = 0;
@@ -238,17 +255,19 @@ decode_mma_kernel(const Args a, const __grid_constant__ CUtensorMap k_map, const
     }
     __syncthreads();
 
-    // Small calls use only the first half of the grid (one CTA per SM); the other CTAs leave at once
-    // and their slots are free for the next call, which -- launched as a programmatic dependent --
-    // then streams its KV while this call is still computing and combining.  Large calls use every
+    // Small calls use the first small_ctas CTAs of the grid (see plan_chunk); the other CTAs leave at
+    // once and their places are free for the next call, which -- launched as a programmatic
+    // dependent -- then streams its KV while this call is still computing.  Large calls use every
     // CTA: two per SM keep more bytes in flight.
     const int total = pref[B];
-    const int half_grid = ((int)gridDim.x + 1) / 2;
-    const int active = total <= half_grid * kSmallCallPages ? half_grid : (int)gridDim.x;
-    int chunk = (total + active - 1) / active;
-    if (chunk < kMinChunk) chunk = kMinChunk;
+    const int chunk = plan_chunk(total, (int)gridDim.x, a.small_ctas);
     const long long r0l = (long long)blockIdx.x * chunk;
-    if (r0l >= total) return;
+    if (r0l >= total) {
+        // (CTA 0 only gets here when the call has no decode rows.)  One thread of CTA 0 always waits
+        // for the previous kernel, so that calls complete in stream order.
+        if (blockIdx.x == 0 && tid == 0) wait_for_predecessor();
+        return;
+    }
     const int r0 = (int)r0l;
     const int r1 = min(total, r0 + chunk);
     volatile int *abort = &tail->abort;
@@ -322,76 +341,61 @@ decode_mma_kernel(const Args a, const __grid_constant__ CUtensorMap k_map, const
     Segment s;
     int n_parked = 0;
     Parked pk[kParked];
-    int pend_n = 0;
-    int pend_slot0[2], pend_parts[2];
-    size_t pend_out[2];
 
     // Ordering against the previous kernel on the stream.  Writes to `out` always wait for it
-    // (griddepcontrol.wait, once per CTA).  Writes to the workspace wait for it too, unless the call
-    // owns a workspace set that no unfinished call can still be reading: sets rotate with the call's
-    // generation number, and the last CTA of every call publishes its generation in *done_gen.
+    // (griddepcontrol.wait, once per CTA, and only in CTAs that have something to write there, plus
+    // CTA 0, which keeps the calls completing in stream order).  Writes to the workspace wait for it
+    // too, unless the call owns a workspace set that no unfinished call can still be reading: sets
+    // rotate with the call's generation number, and the combine kernel of every call publishes the
+    // generation in *done_gen when it is through.
     bool waited = false;
     auto ensure_wait = [&]() {
         if (!waited) { wait_for_predecessor(); waited = true; }
     };
-    // Publishes the parked segment results: partials of split (sequence, head)s go to the workspace
-    // and are counted; results that are already final are written to `out` -- at once in the middle
-    // of a range (`last_call` false), or left parked for the epilogue, after the wait.
+    // The set is free when the newest completed call lies in [gen - sets, gen - 1]: calls complete in
+    // stream order, so the set's previous user (gen - sets) is among the completed.  A value outside
+    // the window -- in particular a newer generation left behind by an earlier replay of a captured
+    // graph, whose generations repeat -- proves nothing and the CTA waits instead.
+    const bool may_early = a.sets >= 3 && !a.force_wait;
+    auto set_is_free = [&]() -> bool {
+        unsigned d;
+        asm volatile("ld.relaxed.gpu.global.u32 %0, [%1];" : "=r"(d) : "l"(a.done_gen) : "memory");
+        return (uint32_t)(a.gen - 1u - d) < (uint32_t)a.sets;
+    };
+    bool early_known = false;   // thread 0 only; looked up now so that the answer is there when it is needed
+    if (tid == 0 && may_early) early_known = set_is_free();
+    // Publishes the parked segment results.  Parts of split (sequence, head)s go to the workspace as
+    // partials (the combine kernel that follows merges them); results that are already final are
+    // written to `out` -- at once in the middle of a range (`last_call` false), or left parked for
+    // the epilogue, after the wait.
     auto flush = [&](bool last_call) {
-        if (tid == 0) {
-            int early = 0;
-            if (a.sets >= 3 && !a.force_wait) {
-                unsigned d;
-                asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(d) : "l"(a.done_gen) : "memory");
-                early = (int)(d - (a.gen - (uint32_t)a.sets)) >= 0;  // the set's previous user has completed
-            }
-            tail->early = early;
-        }
-        named_barrier(1, kConsThreads);
-        if (!tail->early) ensure_wait();
-        bool any_multi = false;
+        bool any_multi = false, any_single = false;
         for (int j = 0; j < n_parked; ++j) {
-            if (pk[j].nparts == 1) continue;
-            const float *rec = park + j * REC;
-            const size_t slot = (size_t)pk[j].bk + blockIdx.x;
-            for (int idx = tid; idx < G * kD; idx += kConsThreads) {
-                const int h = idx / kD;
-                a.part_o[slot * G * kD + idx] = rec[2 * GP + idx];
-                if (idx - h * kD == 0) {
-                    a.part_ml[(slot * GP + h) * 2 + 0] = rec[h];
-                    a.part_ml[(slot * GP + h) * 2 + 1] = rec[GP + h];
-                }
-            }
-            any_multi = true;
+            any_multi = any_multi || pk[j].nparts > 1;
+            any_single = any_single || pk[j].nparts == 1;
         }
         if (any_multi) {
-            fence_proxy_async_all();         // the partials are read back through bulk copies
-            named_barrier(1, kConsThreads);  // the block's stores are ordered before thread 0's fence
             if (tid == 0) {
-                __threadfence();
-                fence_proxy_async_all();
-                for (int j = 0; j < n_parked; ++j) {
-                    int last = 0;
-                    if (pk[j].nparts > 1) {
-                        const int old = atomicAdd(&a.counters[pk[j].bk], 1);
-                        last = (old == pk[j].nparts - 1);
-                        if (last) a.counters[pk[j].bk] = 0;
-                    }
-                    tail->flags[j] = last;
-                }
+                if (may_early && !early_known) early_known = set_is_free();
+                tail->early = early_known ? 1 : 0;
             }
             named_barrier(1, kConsThreads);
+            if (!tail->early) ensure_wait();
             for (int j = 0; j < n_parked; ++j) {
-                if (pk[j].nparts > 1 && tail->flags[j] && pend_n < 2) {
-                    pend_slot0[pend_n] = pk[j].bk + pk[j].c_first;
-                    pend_parts[pend_n] = pk[j].nparts;
-                    pend_out[pend_n] = pk[j].out_base;
-                    ++pend_n;
+                if (pk[j].nparts == 1) continue;
+                const float *rec = park + j * REC;
+                const size_t slot = (size_t)pk[j].bk + blockIdx.x;
+                for (int idx = tid; idx < G * kD / 4; idx += kConsThreads)
+                    reinterpret_cast<float4 *>(a.part_o + slot * G * kD)[idx] =
+                        reinterpret_cast<const float4 *>(rec + 2 * GP)[idx];
+                if (tid < G) {
+                    a.part_ml[(slot * GP + tid) * 2 + 0] = rec[tid];
+                    a.part_ml[(slot * GP + tid) * 2 + 1] = rec[GP + tid];
                 }
             }
         }
         if (!last_call) {
-            ensure_wait();
+            if (any_single) ensure_wait();
             for (int j = 0; j < n_parked; ++j) {
                 if (pk[j].nparts != 1) continue;
                 const float *rec = park + j * REC;
@@ -399,7 +403,7 @@ decode_mma_kernel(const Args a, const __grid_constant__ CUtensorMap k_map, const
                     reinterpret_cast<__nv_bfloat16 *>(a.out)[pk[j].out_base + idx] =
                         __float2bfloat16_rn(rec[2 * GP + idx] / rec[GP + idx / kD]);
             }
-            named_barrier(1, kConsThreads);  // parking slots and flags are free again
+            named_barrier(1, kConsThreads);  // parking slots are free again
             n_parked = 0;
         }
     };
@@ -565,193 +569,12 @@ decode_mma_kernel(const Args a, const __grid_constant__ CUtensorMap k_map, const
     }
     if (n_parked > 0) flush(true);  // final results stay parked until the epilogue
 
-    // ---- split combine of the (sequence, kv head)s this CTA was the last to reach -----------------
-    // Up to two jobs, worked on side by side.  The ring is idle: each job gets half of it as a landing
-    // buffer for partial outputs (bulk copies, a piece at a time).  While the first pieces are in
-    // flight the warps read the parts' (max, sum) records straight from global memory and turn them
-    // into weights, kept where the warp records and parked segments used to be.
-    constexpr int PART_BYTES = G * kD * 4;
-    constexpr int CAP = kRingBytes / PART_BYTES;   // partial outputs the ring can hold at once
-    constexpr int NK = (G * kD + kConsThreads - 1) / kConsThreads;
-    float acc[2][NK];
-    int hk[NK];
-#pragma unroll
-    for (int k = 0; k < NK; ++k) {
-        const int idx = tid + k * kConsThreads;
-        hk[k] = idx < G * kD ? idx / kD : 0;
-        acc[0][k] = 0.f;
-        acc[1][k] = 0.f;
-    }
-    bool combined = false;
-    do {
-    if (pend_n == 0) break;
-    // landing buffers: the whole ring for one job, shared in proportion to their parts for two
-    int per_piece[2] = {CAP, 0}, buf_off[2] = {0, 0};
-    if (pend_n == 2) {
-        const int n0 = pend_parts[0], n1 = pend_parts[1];
-        int c0 = (n0 + n1 <= CAP) ? n0 : max(1, min(CAP - 1, CAP * n0 / (n0 + n1)));
-        per_piece[0] = c0;
-        per_piece[1] = CAP - c0;
-        buf_off[1] = c0 * PART_BYTES;
-    }
-    float *wsm = osm;                                        // [job][part][GP] weights
-    constexpr int WSM_FLOATS = C::OSM_BYTES / 4;   // the parked records stay untouched
-    const int wstride = WSM_FLOATS / 2;                      // floats per job
-    bool fits = true;
-    for (int j = 0; j < pend_n; ++j) fits = fits && pend_parts[j] * GP <= wstride;
-    __threadfence();
-    if (!fits) {
-        // more parts than the weight area can describe (one sequence over every CTA of a very large
-        // part): merge straight from global memory
-        ensure_wait();
-        for (int j = 0; j < pend_n; ++j) {
-            const int nparts = pend_parts[j];
-            const size_t slot0 = (size_t)pend_slot0[j];
-            for (int idx = tid; idx < G * kD; idx += kConsThreads) {
-                const int h = idx / kD;
-                float m = -INFINITY;
-                for (int p = 0; p < nparts; ++p) m = fmaxf(m, __ldcg(&a.part_ml[((slot0 + p) * GP + h) * 2]));
-                float l = 0.f, x = 0.f;
-                for (int p = 0; p < nparts; ++p) {
-                    const float w = fast_exp2(__ldcg(&a.part_ml[((slot0 + p) * GP + h) * 2]) - m);
-                    l = fmaf(w, __ldcg(&a.part_ml[((slot0 + p) * GP + h) * 2 + 1]), l);
-                    x = fmaf(w, __ldcg(&a.part_o[(slot0 + p) * G * kD + idx]), x);
-                }
-                reinterpret_cast<__nv_bfloat16 *>(a.out)[pend_out[j] + idx] = __float2bfloat16_rn(x / l);
-            }
-        }
-        break;
-    }
-    auto issue_piece = [&](int j, int i) {  // thread 0 only: piece i of job j into the job's buffer
-        const int pp0 = i * per_piece[j], np = min(per_piece[j], pend_parts[j] - pp0);
-        const uint32_t bytes = (uint32_t)np * PART_BYTES;
-        mbar_arrive_expect_tx(&tail->cbar[j], bytes);
-        bulk_load(ring + buf_off[j], a.part_o + ((size_t)pend_slot0[j] + pp0) * G * kD, bytes, &tail->cbar[j]);
-    };
-    if (tid == 0) {
-        fence_proxy_async_all();
-        for (int j = 0; j < pend_n; ++j) issue_piece(j, 0);
-    }
-    __syncwarp();  // warp 0 goes on as one: without this its lane 0 ran the next phase apart from the rest (5 us)
-    // weights: warp w owns heads w, w + 4 of every job; lanes stride over the parts.  In the usual
-    // case (at most 128 parts) every load of the warp is issued before the first one is used.
-    constexpr int HPW = (G + kConsWarps - 1) / kConsWarps;   // heads per warp
-    bool small = true;
-    for (int j = 0; j < pend_n; ++j) small = small && pend_parts[j] <= 128;
-    if (small) {
-        // every load first, from clamped (always valid) records, so that all of them are in flight
-        // together; what does not exist is masked afterwards
-        float2 raw[2][HPW][4];
-#pragma unroll
-        for (int j = 0; j < 2; ++j) {
-            const float *mlg = a.part_ml + (size_t)pend_slot0[j < pend_n ? j : 0] * GP * 2;
-            const int nparts = j < pend_n ? pend_parts[j] : 1;
-#pragma unroll
-            for (int hh = 0; hh < HPW; ++hh) {
-                const int hc = min(warp + hh * kConsWarps, G - 1);
-#pragma unroll
-                for (int u = 0; u < 4; ++u) {
-                    const int pc = min(lane + 32 * u, nparts - 1);
-                    raw[j][hh][u] = __ldcg(reinterpret_cast<const float2 *>(mlg + (pc * GP + hc) * 2));
-                }
-            }
-        }
-        float mv[2][HPW][4], lv[2][HPW][4];
-#pragma unroll
-        for (int j = 0; j < 2; ++j) {
-            const int nparts = j < pend_n ? pend_parts[j] : 0;
-#pragma unroll
-            for (int hh = 0; hh < HPW; ++hh) {
-#pragma unroll
-                for (int u = 0; u < 4; ++u) {
-                    const bool ok = lane + 32 * u < nparts && warp + hh * kConsWarps < G;
-                    mv[j][hh][u] = ok ? raw[j][hh][u].x : -INFINITY;
-                    lv[j][hh][u] = ok ? raw[j][hh][u].y : 0.f;
-                }
-            }
-        }
-#pragma unroll
-        for (int j = 0; j < 2; ++j) {
-            const int nparts = j < pend_n ? pend_parts[j] : 0;
-#pragma unroll
-            for (int hh = 0; hh < HPW; ++hh) {
-                const int h = warp + hh * kConsWarps;
-                float m = fmaxf(fmaxf(mv[j][hh][0], mv[j][hh][1]), fmaxf(mv[j][hh][2], mv[j][hh][3]));
-#pragma unroll
-                for (int off = 16; off >= 1; off >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, off));
-                float l = 0.f;
-#pragma unroll
-                for (int u = 0; u < 4; ++u) {
-                    const int p = lane + 32 * u;
-                    if (p < nparts && h < G) {
-                        const float w = fast_exp2(mv[j][hh][u] - m);
-                        wsm[j * wstride + p * GP + h] = w;
-                        l = fmaf(w, lv[j][hh][u], l);
-                    }
-                }
-#pragma unroll
-                for (int off = 16; off >= 1; off >>= 1) l += __shfl_xor_sync(0xffffffffu, l, off);
-                if (lane == 0 && h < G && j < pend_n) tail->lsum[j * kMaxGroup + h] = l;
-            }
-        }
-    } else {
-        for (int j = 0; j < pend_n; ++j) {
-            const int nparts = pend_parts[j];
-            const float *mlg = a.part_ml + (size_t)pend_slot0[j] * GP * 2;
-            for (int h = warp; h < G; h += kConsWarps) {
-                float m = -INFINITY;
-                for (int p = lane; p < nparts; p += 32) {
-                    const float x = __ldcg(&mlg[(p * GP + h) * 2]);
-                    wsm[j * wstride + p * GP + h] = x;
-                    m = fmaxf(m, x);
-                }
-#pragma unroll
-                for (int off = 16; off >= 1; off >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, off));
-                float l = 0.f;
-                for (int p = lane; p < nparts; p += 32) {
-                    const float w = fast_exp2(wsm[j * wstride + p * GP + h] - m);
-                    wsm[j * wstride + p * GP + h] = w;
-                    l = fmaf(w, __ldcg(&mlg[(p * GP + h) * 2 + 1]), l);
-                }
-#pragma unroll
-                for (int off = 16; off >= 1; off >>= 1) l += __shfl_xor_sync(0xffffffffu, l, off);
-                if (lane == 0) tail->lsum[j * kMaxGroup + h] = l;
-            }
-        }
-    }
-    named_barrier(1, kConsThreads);
-    int max_pieces = 0;
-    for (int j = 0; j < pend_n; ++j) max_pieces = max(max_pieces, (pend_parts[j] + per_piece[j] - 1) / per_piece[j]);
-    for (int i = 0; i < max_pieces; ++i) {
-#pragma unroll
-        for (int j = 0; j < 2; ++j) {
-            if (j < pend_n && i * per_piece[j] < pend_parts[j]) {
-                const int pp0 = i * per_piece[j], np = min(per_piece[j], pend_parts[j] - pp0);
-                mbar_wait(&tail->cbar[j], (uint32_t)i & 1u, abort, a.status);
-                const float *po = reinterpret_cast<const float *>(ring + buf_off[j]);
-                const float *wj = wsm + j * wstride + pp0 * GP;
-#pragma unroll 2
-                for (int p = 0; p < np; ++p) {
-#pragma unroll
-                    for (int k = 0; k < NK; ++k) {
-                        const int idx = tid + k * kConsThreads;
-                        if (idx < G * kD) acc[j][k] = fmaf(wj[p * GP + hk[k]], po[p * G * kD + idx], acc[j][k]);
-                    }
-                }
-            }
-        }
-        if (i + 1 < max_pieces) {
-            named_barrier(1, kConsThreads);  // everyone is done with the buffers before they are refilled
-            if (tid == 0)
-                for (int j = 0; j < pend_n; ++j)
-                    if ((i + 1) * per_piece[j] < pend_parts[j]) issue_piece(j, i + 1);
-        }
-    }
-    combined = true;
-    } while (0);
-
-    // ---- epilogue: everything that goes to `out` waits for the previous kernel -------------------------
-    ensure_wait();
+    // ---- epilogue: what goes to `out` waits for the previous kernel.  A CTA that only produced parts
+    //      of split (sequence, head)s has nothing to write there and leaves at once, freeing its
+    //      place on the SM for the next call.
+    bool any_single = false;
+    for (int j = 0; j < n_parked; ++j) any_single = any_single || pk[j].nparts == 1;
+    if (any_single || blockIdx.x == 0) ensure_wait();
     for (int j = 0; j < n_parked; ++j) {
         if (pk[j].nparts != 1) continue;
         const float *rec = park + j * REC;
@@ -759,28 +582,163 @@ decode_mma_kernel(const Args a, const __grid_constant__ CUtensorMap k_map, const
             reinterpret_cast<__nv_bfloat16 *>(a.out)[pk[j].out_base + idx] =
                 __float2bfloat16_rn(rec[2 * GP + idx] / rec[GP + idx / kD]);
     }
-    if (combined) {
+}
+
+// ---- split combine ---------------------------------------------------------------------------------
+// Launched right behind the decode kernel as its programmatic dependent: its CTAs come up while the
+// decode kernel is still streaming, work out the same plan from the lengths, and then wait for the
+// decode kernel to complete (griddepcontrol.wait), which makes every partial visible without a fence,
+// an arrival counter or a CTA of the decode kernel staying behind.  One work item is a split
+// (sequence, kv head); a thread merges one or two 4-dimension pieces of the group's G x 128 outputs
+// over the parts,
+//     m = max_p m_p,  w_p = 2^(m_p - m),  out = sum_p w_p o_p / sum_p w_p l_p.
+// Few, light CTAs on purpose: they sit on the SMs, waiting, while decode CTAs of this and of the
+// next call need the room.  The last CTA to finish publishes the call's generation (see the
+// workspace rotation).
+constexpr int kCombineThreads = 128;
+constexpr int kCombinePreload = 4;   // parts whose values are asked for before the weights are known
+
+struct CombineArgs {
+    const int32_t *seq_lens;
+    const int32_t *q_lens;
+    char *out;
+    const float *part_o;
+    const float *part_ml;
+    int batch, Hq, Hkv, max_pages;
+    int small_ctas, decode_grid;
+    uint32_t gen;
+    unsigned *done_gen;
+    int *exit_count;
+};
+
+template <int G>
+__global__ void __launch_bounds__(kCombineThreads)
+decode_combine_kernel(const CombineArgs a) {
+    constexpr int GP = (G + 3) / 4 * 4;
+    constexpr int VECS = G * kD / 4;                                       // float4 pieces of one partial output
+    constexpr int NE = (VECS + kCombineThreads - 1) / kCombineThreads;     // pieces per thread (1 or 2)
+    extern __shared__ int csm[];
+    int *pref = csm;                      // [B + 1] pages (times kv heads) before sequence b
+    int *row0 = pref + a.batch + 1;       // [B + 1] q rows before sequence b
+    float2 *ml_s = reinterpret_cast<float2 *>(row0 + a.batch + 1);   // [parts][G] (max, sum); 2 (B + 1) ints before it
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int B = a.batch, Hkv = a.Hkv;
+
+    let_successor_start();
+    if (tid == 0) { pref[0] = 0; row0[0] = 0; }
+    for (int b = tid; b < B; b += kCombineThreads) {
+        const int n = a.q_lens[b], L = a.seq_lens[b];
+        const int pages = (n == 1 && L >= 1 && L <= a.max_pages * kPage) ? (L + kPage - 1) / kPage : 0;
+        pref[b + 1] = pages * Hkv;
+        row0[b + 1] = n > 0 ? n : 0;
+    }
+    __syncthreads();
+    if (warp == 0) {
+        int carry_p = 0, carry_r = 0;
+        for (int b0 = 0; b0 < B; b0 += 32) {
+            const int b = b0 + lane;
+            int vp = b < B ? pref[b + 1] : 0;
+            int vr = b < B ? row0[b + 1] : 0;
 #pragma unroll
-        for (int j = 0; j < 2; ++j) {
-            if (j < pend_n) {
+            for (int off = 1; off < 32; off <<= 1) {
+                const int tp = __shfl_up_sync(0xffffffffu, vp, off);
+                const int tr = __shfl_up_sync(0xffffffffu, vr, off);
+                if (lane >= off) { vp += tp; vr += tr; }
+            }
+            if (b < B) { pref[b + 1] = vp + carry_p; row0[b + 1] = vr + carry_r; }
+            carry_p += __shfl_sync(0xffffffffu, vp, 31);
+            carry_r += __shfl_sync(0xffffffffu, vr, 31);
+        }
+    }
+    __syncthreads();
+    const int total = pref[B];
+    const int chunk = plan_chunk(total, a.decode_grid, a.small_ctas);
+
+    wait_for_predecessor();   // the decode kernel of this call, and with it every earlier call
+
+    int ev[NE], eh[NE];       // this thread's pieces: index into a partial output, and its head
+    bool eok[NE];
 #pragma unroll
-                for (int k = 0; k < NK; ++k) {
-                    const int idx = tid + k * kConsThreads;
-                    if (idx < G * kD)
-                        reinterpret_cast<__nv_bfloat16 *>(a.out)[pend_out[j] + idx] =
-                            __float2bfloat16_rn(acc[j][k] / tail->lsum[j * kMaxGroup + hk[k]]);
+    for (int k = 0; k < NE; ++k) {
+        const int e = tid + k * kCombineThreads;
+        eok[k] = e < VECS;
+        ev[k] = eok[k] ? e : 0;
+        eh[k] = ev[k] / (kD / 4);
+    }
+    for (int bk = blockIdx.x; bk < B * Hkv; bk += gridDim.x) {
+        const int b = bk / Hkv, kvh = bk - b * Hkv;
+        const int pages = (pref[b + 1] - pref[b]) / Hkv;
+        if (pages == 0) continue;
+        const int s0 = pref[b] + kvh * pages, s1 = s0 + pages;
+        const int c_first = s0 / chunk;
+        const int nparts = (s1 - 1) / chunk - c_first + 1;   // at most one per CTA of the decode grid
+        if (nparts <= 1) continue;       // the decode kernel wrote this one itself
+        const size_t slot0 = (size_t)bk + c_first;
+        const float4 *po = reinterpret_cast<const float4 *>(a.part_o + slot0 * G * kD);
+        // the first partial values are asked for before the weights exist, so that the two round
+        // trips to memory run side by side
+        float4 v[NE][kCombinePreload];
+#pragma unroll
+        for (int u = 0; u < kCombinePreload; ++u)
+#pragma unroll
+            for (int k = 0; k < NE; ++k) v[k][u] = __ldcg(po + (size_t)min(u, nparts - 1) * VECS + ev[k]);
+        __syncthreads();                 // ml_s of the previous item has been read by everyone
+        for (int i = tid; i < nparts * G; i += kCombineThreads) {
+            const int p = i / G, h = i - p * G;
+            ml_s[i] = __ldcg(reinterpret_cast<const float2 *>(a.part_ml + ((slot0 + p) * GP + h) * 2));
+        }
+        __syncthreads();
+        float m[NE], l[NE];
+        float4 x[NE];
+#pragma unroll
+        for (int k = 0; k < NE; ++k) {
+            m[k] = -INFINITY;
+            for (int p = 0; p < nparts; ++p) m[k] = fmaxf(m[k], ml_s[p * G + eh[k]].x);
+            l[k] = 0.f;
+            x[k] = make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+        for (int p0 = 0; p0 < nparts; p0 += kCombinePreload) {
+            if (p0 > 0) {
+#pragma unroll
+                for (int u = 0; u < kCombinePreload; ++u)
+#pragma unroll
+                    for (int k = 0; k < NE; ++k) v[k][u] = __ldcg(po + (size_t)min(p0 + u, nparts - 1) * VECS + ev[k]);
+            }
+#pragma unroll
+            for (int u = 0; u < kCombinePreload; ++u) {
+                if (p0 + u < nparts) {
+#pragma unroll
+                    for (int k = 0; k < NE; ++k) {
+                        const float2 ml = ml_s[(p0 + u) * G + eh[k]];
+                        const float w = fast_exp2(ml.x - m[k]);
+                        l[k] = fmaf(w, ml.y, l[k]);
+                        x[k].x = fmaf(w, v[k][u].x, x[k].x);
+                        x[k].y = fmaf(w, v[k][u].y, x[k].y);
+                        x[k].z = fmaf(w, v[k][u].z, x[k].z);
+                        x[k].w = fmaf(w, v[k][u].w, x[k].w);
+                    }
                 }
             }
         }
+        __nv_bfloat16 *orow = reinterpret_cast<__nv_bfloat16 *>(a.out) + ((size_t)row0[b] * a.Hq + kvh * G) * kD;
+#pragma unroll
+        for (int k = 0; k < NE; ++k) {
+            if (eok[k]) {
+                const float inv = 1.0f / l[k];
+                uint2 o2;
+                o2.x = pack_bf16(x[k].x * inv, x[k].y * inv);
+                o2.y = pack_bf16(x[k].z * inv, x[k].w * inv);
+                *reinterpret_cast<uint2 *>(orow + (size_t)ev[k] * 4) = o2;
+            }
+        }
     }
-    // The last CTA to get here publishes this call's generation: its workspace set has been read for
-    // the last time (every combine is done) and every earlier call has completed (we waited for it).
-    named_barrier(1, kConsThreads);
+    // The last CTA through publishes this call's generation: its workspace set has been read for the
+    // last time, and every earlier call has completed (every CTA here waited for the decode kernel,
+    // whose CTA 0 waited for the kernel before it).
+    __syncthreads();
     if (tid == 0) {
-        __threadfence();
-        const int active_ctas = (total + chunk - 1) / chunk;
         const int old = atomicAdd(a.exit_count, 1);
-        if (old == active_ctas - 1) {
+        if (old == (int)gridDim.x - 1) {
             *a.exit_count = 0;
             __threadfence();
             asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(a.done_gen), "r"(a.gen) : "memory");
@@ -820,8 +778,8 @@ bool make_pool_map(CUtensorMap *map, const void *pool, const arb_attn_params &p)
 }
 
 template <int G>
-arb_status launch_one(Ctx *ctx, const Args &a, const CUtensorMap &km, const CUtensorMap &vm, bool overlap,
-                      cudaStream_t stream) {
+arb_status launch_one(Ctx *ctx, const Args &a, CombineArgs ca, const CUtensorMap &km, const CUtensorMap &vm,
+                      bool overlap, cudaStream_t stream) {
     const size_t smem = smem_bytes<G>(a.batch);
     static bool attr_set[64] = {};
     if (!attr_set[ctx->device & 63]) {
@@ -830,19 +788,36 @@ arb_status launch_one(Ctx *ctx, const Args &a, const CUtensorMap &km, const CUte
             return ARB_ERR_CUDA;
         attr_set[ctx->device & 63] = true;
     }
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(ctx->num_sms * kCtasPerSm);
-    cfg.blockDim = dim3(kThreads);
-    cfg.dynamicSmemBytes = smem;
-    cfg.stream = stream;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cudaLaunchConfig_t cfg = {};
+    // A call that cannot be anything but small -- the block table has room for at most kSmallCallPages
+    // pages per SM -- is launched with one CTA per SM outright: no CTA comes up only to leave.
+    const long long page_bound = (long long)a.batch * a.max_pages * a.Hkv;
+    const bool small = page_bound <= (long long)ctx->num_sms * kSmallCallPages;
+    const int grid = small ? ctx->num_sms : ctx->num_sms * kCtasPerSm;
+    cfg.gridDim = dim3(grid);
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
     cfg.attrs = attr;
     cfg.numAttrs = overlap ? 1 : 0;
-    const cudaError_t err = cudaLaunchKernelEx(&cfg, decode_mma_kernel<G>, a, km, vm);
+    if (cudaLaunchKernelEx(&cfg, decode_mma_kernel<G>, a, km, vm) != cudaSuccess) return ARB_ERR_CUDA;
     ctx->launches++;
-    return err == cudaSuccess ? ARB_OK : ARB_ERR_CUDA;
+    // the combine kernel, always a programmatic dependent of the decode kernel
+    ca.decode_grid = grid;
+    const long long items = (long long)a.batch * a.Hkv;
+    cudaLaunchConfig_t ccfg = {};
+    ccfg.gridDim = dim3((unsigned)(items < ctx->num_sms ? items : ctx->num_sms));
+    ccfg.blockDim = dim3(kCombineThreads);
+    ccfg.dynamicSmemBytes = sizeof(int) * (2 * (size_t)a.batch + 2) + sizeof(float2) * (size_t)grid * G;
+    ccfg.stream = stream;
+    ccfg.attrs = attr;
+    ccfg.numAttrs = 1;
+    if (cudaLaunchKernelEx(&ccfg, decode_combine_kernel<G>, ca) != cudaSuccess) return ARB_ERR_CUDA;
+    ctx->launches++;
+    return ARB_OK;
 }
 
 }  // namespace
@@ -881,8 +856,6 @@ arb_status launch_decode_mma(Ctx *ctx, const arb_attn_params &p, const void *q, 
     a.out = static_cast<char *>(out);
     a.part_o = reinterpret_cast<float *>(ctx->workspace + (size_t)set * set_bytes);
     a.part_ml = a.part_o + part_o_floats;
-    a.counters = sets > 1 ? ctx->rot + (size_t)set * kRotCounters : ctx->counters;
-    a.exit_count = ctx->rot + (size_t)kRotSets * kRotCounters + set;
     a.done_gen = reinterpret_cast<unsigned *>(ctx->rot + (size_t)kRotSets * kRotCounters + kRotSets);
     a.gen = gen;
     a.sets = sets;
@@ -894,18 +867,40 @@ arb_status launch_decode_mma(Ctx *ctx, const arb_attn_params &p, const void *q, 
     a.Hkv = p.num_kv_heads;
     a.num_pages = p.num_pages;
     a.max_pages = p.max_pages_per_seq;
+    // A small call streams at the pace of its CTAs' pipelines, not of the memory system, and every
+    // CTA spends a fixed time before its first and after its last tile.  A call that declares itself
+    // part of a back-to-back series (ARB_ATTN_OVERLAP_PREVIOUS) therefore takes only every second
+    // SM's worth of CTAs: each lives longer, four calls are in flight instead of two, and the
+    // series as a whole moves more bytes per second; a lone call gets one CTA on every SM, which
+    // is what finishes it soonest.
+    a.small_ctas = (p.flags & ARB_ATTN_OVERLAP_PREVIOUS) ? (ctx->num_sms + 1) / 2 : ctx->num_sms;
     const float scale = p.softmax_scale > 0.f ? p.softmax_scale : 1.0f / sqrtf((float)p.head_dim);
     a.scale_log2 = scale * 1.4426950408889634f;
     const bool overlap = (p.flags & ARB_ATTN_OVERLAP_PREVIOUS) != 0;
+    CombineArgs ca;
+    ca.seq_lens = seq_lens;
+    ca.q_lens = q_lens;
+    ca.out = a.out;
+    ca.part_o = a.part_o;
+    ca.part_ml = a.part_ml;
+    ca.batch = a.batch;
+    ca.Hq = a.Hq;
+    ca.Hkv = a.Hkv;
+    ca.max_pages = a.max_pages;
+    ca.small_ctas = a.small_ctas;
+    ca.decode_grid = 0;  // set by launch_one
+    ca.gen = gen;
+    ca.done_gen = a.done_gen;
+    ca.exit_count = ctx->rot + (size_t)kRotSets * kRotCounters + set;
     switch (g) {
-        case 1: return launch_one<1>(ctx, a, km, vm, overlap, stream);
-        case 2: return launch_one<2>(ctx, a, km, vm, overlap, stream);
-        case 3: return launch_one<3>(ctx, a, km, vm, overlap, stream);
-        case 4: return launch_one<4>(ctx, a, km, vm, overlap, stream);
-        case 5: return launch_one<5>(ctx, a, km, vm, overlap, stream);
-        case 6: return launch_one<6>(ctx, a, km, vm, overlap, stream);
-        case 7: return launch_one<7>(ctx, a, km, vm, overlap, stream);
-        case 8: return launch_one<8>(ctx, a, km, vm, overlap, stream);
+        case 1: return launch_one<1>(ctx, a, ca, km, vm, overlap, stream);
+        case 2: return launch_one<2>(ctx, a, ca, km, vm, overlap, stream);
+        case 3: return launch_one<3>(ctx, a, ca, km, vm, overlap, stream);
+        case 4: return launch_one<4>(ctx, a, ca, km, vm, overlap, stream);
+        case 5: return launch_one<5>(ctx, a, ca, km, vm, overlap, stream);
+        case 6: return launch_one<6>(ctx, a, ca, km, vm, overlap, stream);
+        case 7: return launch_one<7>(ctx, a, ca, km, vm, overlap, stream);
+        case 8: return launch_one<8>(ctx, a, ca, km, vm, overlap, stream);
         default: return ARB_ERR_UNSUPPORTED;
     }
 }

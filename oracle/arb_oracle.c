@@ -20,6 +20,16 @@
  *    difference, which is the single (w, b) used here.
  *  - oracle_rollback: Algorithm 1, escalation branch: the target regenerates the step from the same
  *    prefix x, so every cache that absorbed the rejected draft step forgets it.
+ *  - oracle_policy: the escalation rules the paper compares on PRM scores: the RSD baseline of
+ *    Section 3.1 (accept iff s_d > tau), the oracle threshold rule a = 1{Delta > tau} with
+ *    Delta = s_t - s_d and the arg-max rule of Section 4.1, the budgeted rule of Appendix B
+ *    (Theorem: the min(B, #{Delta > 0}) largest positive advantages), with the wasted-call count of
+ *    Section 3.2 (escalated although s_t <= s_d) and the realised score S(a) = s_d + a Delta.
+ *  - oracle_route_classes: the C-way heads of the ablation (Section 6.1, Label Granularity and
+ *    Classification vs. Regression): a softmax head over C ordered advantage classes, or an ordinal
+ *    head (one logit, C - 1 ordered cut points).
+ *  - oracle_kv_append: the write of a step's new keys and values into the paged cache that every
+ *    "Sample ... step" line of Algorithm 1 implies before the next token attends to them.
  *
  * Pins (tests/test_oracle_*.py): rows of softmax sum to one; uniform keys give the mean of V;
  * a single key returns its V; a dominant key returns its V; score-shift invariance; brute-force
@@ -208,6 +218,172 @@ unsigned oracle_rollback(int B, int32_t *seq_lens, const int32_t *step_lens,
         long r = (long)seq_lens[i] - (long)step_lens[i];
         if (r < 0 || step_lens[i] < 0) { status |= ORACLE_ROLLBACK_UNDERFLOW; r = r < 0 ? 0 : seq_lens[i]; }
         seq_lens[i] = (int32_t)r;
+    }
+    return status;
+}
+
+
+/*
+ * Escalation policies on PRM scores.  s_d, s_t: fp32 scores of the draft step and of the target's
+ * counterpart; decisions[i] = 1 escalates step i to the target, 0 keeps the draft step.
+ *   kind 0, RSD (Section 3.1):  accept iff s_d > tau, so escalate iff s_d <= tau; s_t is not read for the
+ *           decision (it may be NULL when stats is NULL).
+ *   kind 1, oracle threshold (Section 4.1):  escalate iff Delta = s_t - s_d > tau.
+ *   kind 2, oracle arg max (Section 4.1):  keep whichever step scores higher; escalate iff s_t > s_d
+ *           (a tie keeps the draft: no target call buys nothing).
+ *   kind 3, budgeted oracle (Appendix B, Theorem):  escalate the k = min(budget, #{Delta > 0}) steps with
+ *           the largest positive Delta; equal advantages go to the lower index.
+ * Delta and the comparisons are taken in fp32, the precision the scores are given in.
+ * stats (may be NULL): [0] escalations, [1] wasted escalations (a = 1 and s_t <= s_d, Section 3.2),
+ * [2] realised score sum_i (a_i ? s_t,i : s_d,i), [3] gain sum_i a_i (s_t,i - s_d,i) in fp64.
+ */
+typedef struct { float delta; int idx; } oracle_adv;
+
+static int adv_desc(const void *x, const void *y)
+{
+    const oracle_adv *a = (const oracle_adv *)x, *b = (const oracle_adv *)y;
+    if (a->delta > b->delta) return -1;
+    if (a->delta < b->delta) return 1;
+    return a->idx - b->idx;
+}
+
+int oracle_policy(int kind, int n, const float *s_d, const float *s_t, float tau, int budget,
+                  uint8_t *decisions, double *stats)
+{
+    if (kind < 0 || kind > 3 || n < 0) return 1;
+    if (kind != 0 && s_t == NULL) return 1;
+    if (kind == 3) {
+        oracle_adv *adv = (oracle_adv *)malloc(sizeof(oracle_adv) * (size_t)(n > 0 ? n : 1));
+        if (!adv) return 2;
+        for (int i = 0; i < n; ++i) {
+            adv[i].delta = s_t[i] - s_d[i];
+            adv[i].idx = i;
+            decisions[i] = 0;
+        }
+        qsort(adv, (size_t)n, sizeof(oracle_adv), adv_desc);
+        for (int r = 0; r < n && r < budget; ++r) {
+            if (!(adv[r].delta > 0.0f)) break;   /* only positive advantages are worth a call */
+            decisions[adv[r].idx] = 1;
+        }
+        free(adv);
+    } else {
+        for (int i = 0; i < n; ++i) {
+            int a;
+            if (kind == 0) a = !(s_d[i] > tau);
+            else if (kind == 1) { float delta = s_t[i] - s_d[i]; a = delta > tau; }
+            else a = s_t[i] > s_d[i];
+            decisions[i] = (uint8_t)a;
+        }
+    }
+    if (stats) {
+        double esc = 0, wasted = 0, realised = 0, gain = 0;
+        for (int i = 0; i < n; ++i) {
+            const double sd = (double)s_d[i], st = s_t ? (double)s_t[i] : sd;
+            if (decisions[i]) {
+                esc += 1;
+                if (!(st > sd)) wasted += 1;
+                realised += st;
+                gain += st - sd;
+            } else {
+                realised += sd;
+            }
+        }
+        stats[0] = esc; stats[1] = wasted; stats[2] = realised; stats[3] = gain;
+    }
+    return 0;
+}
+
+/*
+ * C-way router heads (Section 6.1 ablation).  The paper says the classes are quantile bins of the
+ * advantage, ordered, and that class 0 / 1 of the default head mean accept / escalate; it does not say
+ * how a C-way head is turned into one routing score.  Reading taken: the score is the expected class
+ * level scaled to [0, 1], score = sum_c p_c * c / (C - 1), and the step escalates iff score > tau (a tie
+ * accepts), which for C = 2 is exactly the default head, softmax([l0, l1])_1 = sigmoid(l1 - l0).
+ *   mode 0, softmax head:  l_c = hidden . W[c] + b[c],  p = softmax(l).        W: [C, H], b: fp64 [C]
+ *   mode 1, ordinal head (cumulative link):  z = hidden . W[0] + b[0];  P(y >= k) = sigmoid(z - cut[k-1]),
+ *           k = 1 .. C-1, cut ascending (b[1 .. C-1]);  p_k = P(y >= k) - P(y >= k + 1).  W: [1, H]
+ * probs: fp64 [S, C]; scores fp64 [S]; decisions uint8 [S] from the score rounded to fp32.
+ */
+int oracle_route_classes(int dtype, int mode, int n_steps, int hidden_dim, int n_classes,
+                         const void *hidden, const void *w, const double *b, float tau,
+                         double *probs, double *scores, uint8_t *decisions)
+{
+    if (n_classes < 2 || n_classes > 64 || (mode != 0 && mode != 1)) return 1;
+    const int C = n_classes;
+    for (int i = 0; i < n_steps; ++i) {
+        double *p = probs + (size_t)i * C;
+        if (mode == 0) {
+            double l[64], mx = -INFINITY, z = 0;
+            for (int c = 0; c < C; ++c) {
+                double acc = b[c];
+                for (int k = 0; k < hidden_dim; ++k)
+                    acc += widen(hidden, dtype, (size_t)i * hidden_dim + k) * widen(w, dtype, (size_t)c * hidden_dim + k);
+                l[c] = acc;
+                if (acc > mx) mx = acc;
+            }
+            for (int c = 0; c < C; ++c) { p[c] = exp(l[c] - mx); z += p[c]; }
+            for (int c = 0; c < C; ++c) p[c] /= z;
+        } else {
+            double acc = b[0], ge[65];
+            for (int k = 0; k < hidden_dim; ++k)
+                acc += widen(hidden, dtype, (size_t)i * hidden_dim + k) * widen(w, dtype, (size_t)k);
+            ge[0] = 1.0;
+            for (int k = 1; k < C; ++k) ge[k] = 1.0 / (1.0 + exp(-(acc - b[k])));
+            ge[C] = 0.0;
+            for (int c = 0; c < C; ++c) p[c] = ge[c] - ge[c + 1];
+        }
+        double sc = 0;
+        for (int c = 0; c < C; ++c) sc += p[c] * (double)c / (double)(C - 1);
+        scores[i] = sc;
+        decisions[i] = ((float)sc > tau) ? 1 : 0;
+    }
+    return 0;
+}
+
+/*
+ * KV append: the new tokens of every sequence go to the slots right behind its cached tokens.
+ * k_new, v_new: [total_new, Hkv, D] packed by sequence (new_lens[b] consecutive rows each);
+ * token j of sequence b lands at position pos = seq_lens[b] + j, i.e. page block_table[b][pos / P],
+ * slot pos % P, of the head-major pools [num_pages, Hkv, P, D].  Values are copied bit for bit (esz
+ * bytes per element).  seq_lens is updated to seq_lens + new_lens when update_lens is non-zero.
+ * A sequence whose new tokens do not fit (pos >= max_pages * P), with a negative length, or with a
+ * block-table entry outside the pool, is left untouched and reported in the status bits.
+ */
+unsigned oracle_kv_append(int esz, int B, int Hkv, int D, int P, long num_pages, int max_pages,
+                          const void *k_new, const void *v_new, const int32_t *block_table,
+                          int32_t *seq_lens, const int32_t *new_lens, int update_lens,
+                          void *k_pages, void *v_pages)
+{
+    unsigned status = 0;
+    size_t row = 0;
+    const size_t tok_bytes = (size_t)D * (size_t)esz;
+    for (int b = 0; b < B; ++b) {
+        const int n = new_lens[b], L = seq_lens[b];
+        if (n <= 0) { if (n < 0) status |= ORACLE_BAD_SEQ_LEN; continue; }
+        int ok = L >= 0 && (long)L + n <= (long)max_pages * P;
+        if (ok) {
+            for (int pos = L; pos < L + n; ++pos) {
+                long page = block_table[(size_t)b * max_pages + pos / P];
+                if (page < 0 || page >= num_pages) ok = 0;
+            }
+            if (!ok) status |= ORACLE_BAD_PAGE;
+        } else {
+            status |= ORACLE_BAD_SEQ_LEN;
+        }
+        if (ok) {
+            for (int j = 0; j < n; ++j) {
+                const int pos = L + j;
+                const long page = block_table[(size_t)b * max_pages + pos / P];
+                for (int h = 0; h < Hkv; ++h) {
+                    const size_t dst = kv_offset(page, h, pos % P, Hkv, P, D) * (size_t)esz;
+                    const size_t src = ((row + (size_t)j) * Hkv + h) * tok_bytes;
+                    memcpy((char *)k_pages + dst, (const char *)k_new + src, tok_bytes);
+                    memcpy((char *)v_pages + dst, (const char *)v_new + src, tok_bytes);
+                }
+            }
+            if (update_lens) seq_lens[b] = L + n;
+        }
+        row += (size_t)n;
     }
     return status;
 }

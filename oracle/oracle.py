@@ -51,6 +51,12 @@ def bind(lib):
     lib.oracle_route.argtypes = [c_int, c_int, c_int, vp, vp, c_dbl, ctypes.c_float, vp, vp]
     lib.oracle_rollback.restype = ctypes.c_uint
     lib.oracle_rollback.argtypes = [c_int, vp, vp, vp]
+    lib.oracle_policy.restype = c_int
+    lib.oracle_policy.argtypes = [c_int, c_int, vp, vp, ctypes.c_float, c_int, vp, vp]
+    lib.oracle_route_classes.restype = c_int
+    lib.oracle_route_classes.argtypes = [c_int, c_int, c_int, c_int, c_int, vp, vp, vp, ctypes.c_float, vp, vp, vp]
+    lib.oracle_kv_append.restype = ctypes.c_uint
+    lib.oracle_kv_append.argtypes = [c_int, c_int, c_int, c_int, c_int, c_long, c_int, vp, vp, vp, vp, vp, c_int, vp, vp]
     return lib
 
 
@@ -150,3 +156,64 @@ def rollback(seq_lens, step_lens, decisions=None):
         dp = dk.ctypes.data
     status = _load().oracle_rollback(sl.shape[0], sl.ctypes.data, st.ctypes.data, dp)
     return sl, int(status)
+
+
+POLICY_RSD, POLICY_ORACLE_THRESHOLD, POLICY_ORACLE_ARGMAX, POLICY_ORACLE_BUDGET = 0, 1, 2, 3
+HEAD_SOFTMAX, HEAD_ORDINAL = 0, 1
+
+
+def _f32(t):
+    if hasattr(t, "detach"):
+        return np.ascontiguousarray(t.detach().cpu().float().numpy())
+    return np.ascontiguousarray(np.asarray(t, dtype=np.float32))
+
+
+def policy(kind: int, s_d, s_t=None, tau: float = 0.0, budget: int = 0):
+    """Escalation policy on PRM scores.  Returns (decisions uint8 [N], stats dict)."""
+    sd = _f32(s_d)
+    st = _f32(s_t) if s_t is not None else None
+    n = sd.shape[0]
+    dec = np.zeros(n, dtype=np.uint8)
+    stats = np.zeros(4, dtype=np.float64)
+    rc = _load().oracle_policy(kind, n, sd.ctypes.data, st.ctypes.data if st is not None else None,
+                               float(tau), int(budget), dec.ctypes.data, stats.ctypes.data)
+    assert rc == 0, rc
+    return dec, {"escalated": int(stats[0]), "wasted": int(stats[1]), "realised": float(stats[2]),
+                 "gain": float(stats[3])}
+
+
+def route_classes(mode: int, hidden, w, b, tau: float):
+    """C-way router head.  w: [C, H] (softmax) or [1, H] / [H] (ordinal); b: C numbers (softmax biases, or the
+    ordinal head's bias followed by its C - 1 cut points).  Returns (probs [S, C], scores [S], decisions [S])."""
+    dh, hp, hk = _raw(hidden)
+    dw, wp, wk = _raw(w)
+    assert dh == dw
+    S, H = hidden.shape
+    bb = np.ascontiguousarray(np.asarray(b, dtype=np.float64))
+    C = bb.shape[0]
+    probs = np.zeros((S, C), dtype=np.float64)
+    scores = np.zeros(S, dtype=np.float64)
+    dec = np.zeros(S, dtype=np.uint8)
+    rc = _load().oracle_route_classes(dh, mode, S, H, C, hp, wp, bb.ctypes.data, float(tau), probs.ctypes.data,
+                                      scores.ctypes.data, dec.ctypes.data)
+    assert rc == 0, rc
+    return probs, scores, dec
+
+
+def kv_append(k_new, v_new, block_table, seq_lens, new_lens, k_pages, v_pages, update_lens: bool = True):
+    """Writes the new tokens into copies of the pools.  Returns (k_pages, v_pages, seq_lens, status bits)."""
+    import torch
+
+    kp = k_pages.detach().cpu().contiguous().clone()
+    vp_ = v_pages.detach().cpu().contiguous().clone()
+    kn = k_new.detach().cpu().contiguous()
+    vn = v_new.detach().cpu().contiguous()
+    assert kn.dtype == kp.dtype == vn.dtype == vp_.dtype
+    num_pages, Hkv, P, D = kp.shape
+    bt = _i32(block_table)
+    sl = _i32(seq_lens).copy()
+    nl = _i32(new_lens)
+    st = _load().oracle_kv_append(kp.element_size(), bt.shape[0], Hkv, D, P, num_pages, bt.shape[1],
+                                  kn.data_ptr(), vn.data_ptr(), bt.ctypes.data, sl.ctypes.data, nl.ctypes.data,
+                                  1 if update_lens else 0, kp.data_ptr(), vp_.data_ptr())
+    return kp, vp_, sl, int(st)

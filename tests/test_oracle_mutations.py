@@ -1,6 +1,6 @@
 """The pins do bite: each plausible mistake, planted in a copy of the oracle's C source and compiled on
 the CPU, is caught by at least one of the pin checks below (the same kinds of checks as in
-test_oracle_attn.py / test_oracle_route.py, run against the mutated build)."""
+test_oracle_attn.py / test_oracle_route.py / test_oracle_policy.py, run against the mutated build)."""
 import ctypes
 import math
 import subprocess
@@ -31,6 +31,15 @@ MUTATIONS = {
     "tie escalates": ("((float)sc > tau)", "((float)sc >= tau)"),
     "rollback adds": ("long r = (long)seq_lens[i] - (long)step_lens[i];", "long r = (long)seq_lens[i] + (long)step_lens[i];"),
     "rollback ignores decisions": ("if (decisions && !decisions[i]) continue;", ""),
+    "RSD polarity": ("if (kind == 0) a = !(s_d[i] > tau);", "if (kind == 0) a = (s_d[i] > tau);"),
+    "oracle threshold on the draft score": ("float delta = s_t[i] - s_d[i]; a = delta > tau;", "float delta = s_t[i]; a = delta > tau;"),
+    "budget spent on negative advantages": ("if (!(adv[r].delta > 0.0f)) break;", ""),
+    "wasted counts improvements": ("if (!(st > sd)) wasted += 1;", "if (st > sd) wasted += 1;"),
+    "class level not normalised": ("sc += p[c] * (double)c / (double)(C - 1);", "sc += p[c] * (double)c;"),
+    "ordinal cut sign": ("ge[k] = 1.0 / (1.0 + exp(-(acc - b[k])));", "ge[k] = 1.0 / (1.0 + exp(-(acc + b[k])));"),
+    "append one slot late": ("const int pos = L + j;", "const int pos = L + j + 1;"),
+    "append swaps K and V": ("memcpy((char *)k_pages + dst, (const char *)k_new + src, tok_bytes);",
+                             "memcpy((char *)k_pages + dst, (const char *)v_new + src, tok_bytes);"),
 }
 
 
@@ -60,7 +69,45 @@ def _pins_pass() -> bool:
         if not (abs(s[1] - 0.75) < 1e-7 and s[2] == 0.5 and list(d) == [1, 1, 0]):
             return False
         new, _ = oracle.rollback(np.array([100, 50]), np.array([10, 20]), np.array([1, 0], dtype=np.uint8))
-        return list(new) == [90, 50]
+        if list(new) != [90, 50]:
+            return False
+        # policies on exact scores: (s_d, s_t) = (1/4, 7/8), (5/8, 1/8), (1/2, 3/4)
+        sd, st = [0.25, 0.625, 0.5], [0.875, 0.125, 0.75]
+        d, s = oracle.policy(oracle.POLICY_RSD, sd, st, tau=0.5)
+        if list(d) != [1, 0, 1] or s["wasted"] != 0:
+            return False
+        d, s = oracle.policy(oracle.POLICY_RSD, sd, st, tau=0.75)
+        if list(d) != [1, 1, 1] or s["wasted"] != 1:
+            return False
+        d, _ = oracle.policy(oracle.POLICY_ORACLE_THRESHOLD, sd, st, tau=0.5)
+        if list(d) != [1, 0, 0]:
+            return False
+        d, s = oracle.policy(oracle.POLICY_ORACLE_BUDGET, sd, st, budget=3)
+        if list(d) != [1, 0, 1] or abs(s["gain"] - 0.875) > 1e-12:
+            return False
+        hid = np.zeros((1, 8), dtype=np.float32)
+        hid[0, 0] = 1.0
+        wc = np.zeros((4, 8), dtype=np.float32)
+        wc[2, 0] = 60.0
+        _, sc, _ = oracle.route_classes(oracle.HEAD_SOFTMAX, hid, wc, [0.0] * 4, 0.5)
+        if abs(sc[0] - 2 / 3) > 1e-12:
+            return False
+        wo = np.zeros((1, 8), dtype=np.float32)
+        p, _, _ = oracle.route_classes(oracle.HEAD_ORDINAL, hid, wo, [0.0, -math.log(3.0), 0.0, math.log(3.0)], 0.5)
+        if not np.allclose(p[0], 0.25, atol=1e-12):
+            return False
+        p, _, _ = oracle.route_classes(oracle.HEAD_ORDINAL, hid, wo, [0.0, math.log(3.0), math.log(9.0)], 0.5)
+        if not np.allclose(p[0], [0.75, 0.15, 0.1], atol=1e-12):
+            return False
+        inp = wl.small_attn_case(1, 2, 1, 64, torch.float32, [20], [1], seed=4, extra_tokens=16)
+        kn = torch.full((3, 1, 64), 7.0)
+        vn = torch.full((3, 1, 64), -7.0)
+        kp, vp, sl, st_ = oracle.kv_append(kn, vn, inp.block_table, inp.seq_lens, torch.tensor([3], dtype=torch.int32),
+                                           inp.k_pages, inp.v_pages)
+        page = int(inp.block_table[0, 1])
+        ok = (st_ == 0 and list(sl) == [23] and bool((kp[page, 0, 4:7] == 7.0).all()) and bool((vp[page, 0, 4:7] == -7.0).all())
+              and torch.equal(kp[page, 0, 7:], inp.k_pages[page, 0, 7:]) and torch.equal(kp[page, 0, :4], inp.k_pages[page, 0, :4]))
+        return ok
     except Exception:
         return False
 

@@ -1,0 +1,234 @@
+"""Pins of the oracle's policy rules, C-way router heads and KV append (CPU only).
+
+Nothing here restates the oracle's own code: decisions are checked against a hand-written table, against
+brute force over every subset (the budgeted rule, Appendix B), against closed forms, against library
+routines (scipy's softmax and expit) and against structural properties the paper states."""
+import itertools
+import math
+from pathlib import Path
+
+import numpy as np
+import pytest
+import torch
+from scipy.special import expit, softmax
+
+from oracle import oracle
+from paper_2512_05033_b200 import workloads as wl
+
+GOLDEN = Path(__file__).parent / "golden" / "policy_truth_table.txt"
+
+
+def _table():
+    rows = []
+    for line in GOLDEN.read_text().splitlines():
+        if line.strip() and not line.startswith("#"):
+            f = line.split()
+            rows.append((float(f[0]), float(f[1]), float(f[2]), int(f[3]), int(f[4]), int(f[5]), int(f[6])))
+    return rows
+
+
+def test_policy_truth_table():
+    for sd, st, tau, rsd, rsd_wasted, thr, amax in _table():
+        d, s = oracle.policy(oracle.POLICY_RSD, [sd], [st], tau=tau)
+        assert (int(d[0]), s["wasted"]) == (rsd, rsd_wasted), (sd, st, tau)
+        d, s = oracle.policy(oracle.POLICY_ORACLE_THRESHOLD, [sd], [st], tau=tau)
+        assert int(d[0]) == thr, (sd, st, tau)
+        d, s = oracle.policy(oracle.POLICY_ORACLE_ARGMAX, [sd], [st])
+        assert int(d[0]) == amax and s["wasted"] == 0, (sd, st)
+        assert s["realised"] == max(sd, st)
+
+
+def test_rsd_polarity_and_monotonicity():
+    """Section 3.1: acceptance is inversely related to tau; a tie s_d == tau is not accepted."""
+    rng = np.random.default_rng(0)
+    sd = rng.random(500).astype(np.float32)
+    st = rng.random(500).astype(np.float32)
+    prev = None
+    for tau in (0.1, 0.3, 0.5, 0.7, 0.9):
+        d, s = oracle.policy(oracle.POLICY_RSD, sd, st, tau=tau)
+        assert (d == (sd <= np.float32(tau))).all()
+        assert s["wasted"] == int(((sd <= np.float32(tau)) & (st <= sd)).sum())
+        if prev is not None:
+            assert (d >= prev).all()          # the escalated set only grows with tau
+        prev = d
+    d, _ = oracle.policy(oracle.POLICY_RSD, [0.5], [0.9], tau=0.5)
+    assert d[0] == 1
+
+
+def test_oracle_threshold_nesting_zero_waste_and_argmax():
+    rng = np.random.default_rng(1)
+    sd = rng.random(400).astype(np.float32)
+    st = rng.random(400).astype(np.float32)
+    prev = None
+    for tau in (-0.5, -0.1, 0.0, 0.2, 0.6):
+        d, s = oracle.policy(oracle.POLICY_ORACLE_THRESHOLD, sd, st, tau=tau)
+        assert (d == ((st - sd) > np.float32(tau))).all()
+        if prev is not None:
+            assert (d <= prev).all()          # a higher threshold escalates a subset
+        prev = d
+        if tau >= 0:
+            assert s["wasted"] == 0           # Corollary (zero wasted computation)
+        assert abs(s["realised"] - (sd.astype(np.float64).sum() + s["gain"])) < 1e-9   # S(a) = s_d + a Delta
+    d0, _ = oracle.policy(oracle.POLICY_ORACLE_THRESHOLD, sd, st, tau=0.0)
+    da, sa = oracle.policy(oracle.POLICY_ORACLE_ARGMAX, sd, st)
+    assert (d0 == da).all()
+    assert abs(sa["realised"] - np.maximum(sd, st).astype(np.float64).sum()) < 1e-9
+
+
+@pytest.mark.parametrize("seed", range(6))
+def test_budgeted_rule_is_optimal_by_brute_force(seed):
+    """Appendix B, Theorem: among all a with sum(a) <= B the rule maximises sum(a Delta); it uses
+    k = min(B, #{Delta > 0}) escalations and equals a threshold policy."""
+    rng = np.random.default_rng(100 + seed)
+    n = int(rng.integers(1, 11))
+    sd = (rng.integers(0, 64, n) / 64.0).astype(np.float32)     # exact values, ties included
+    st = (rng.integers(0, 64, n) / 64.0).astype(np.float32)
+    delta = st.astype(np.float64) - sd.astype(np.float64)
+    for budget in range(0, n + 2):
+        d, s = oracle.policy(oracle.POLICY_ORACLE_BUDGET, sd, st, budget=budget)
+        best = max(sum(delta[i] for i in sub)
+                   for k in range(0, min(budget, n) + 1) for sub in itertools.combinations(range(n), k))
+        assert abs(s["gain"] - best) < 1e-12
+        assert s["escalated"] == min(budget, int((delta > 0).sum()))
+        assert s["wasted"] == 0
+        chosen, rest = delta[d == 1], delta[(d == 0) & (delta > 0)]
+        if len(chosen) and len(rest):
+            assert chosen.min() >= rest.max()
+        # the same set as a threshold policy, whenever a threshold can separate it (no tie at the cut)
+        if len(chosen) and (not len(rest) or chosen.min() > rest.max()):
+            lo = max(rest.max() if len(rest) else 0.0, 0.0)
+            tau = (chosen.min() + lo) / 2
+            dt, _ = oracle.policy(oracle.POLICY_ORACLE_THRESHOLD, sd, st, tau=tau)
+            assert (dt == d).all()
+
+
+def test_budgeted_rule_ties_go_to_the_lower_index_and_majorise_rsd():
+    d, _ = oracle.policy(oracle.POLICY_ORACLE_BUDGET, [0.25, 0.25, 0.25], [0.5, 0.5, 0.5], budget=2)
+    assert list(d) == [1, 1, 0]
+    rng = np.random.default_rng(7)
+    sd = rng.random(60).astype(np.float32)
+    st = rng.random(60).astype(np.float32)
+    for tau in (0.2, 0.5, 0.8):        # Corollary (Pareto frontier): no policy of the same cost scores higher
+        dr, sr = oracle.policy(oracle.POLICY_RSD, sd, st, tau=tau)
+        _, sb = oracle.policy(oracle.POLICY_ORACLE_BUDGET, sd, st, budget=sr["escalated"])
+        assert sb["realised"] >= sr["realised"] - 1e-12
+
+
+# ---- C-way heads -------------------------------------------------------------------------------------
+
+def test_two_class_softmax_head_is_the_default_head():
+    r = wl.make_router_inputs(16, 256, torch.float32, seed=5)
+    rng = np.random.default_rng(5)
+    w0 = rng.normal(0, 1 / 16, 256).astype(np.float32)
+    w = np.stack([w0, w0 + r.w.numpy()])                      # w1 - w0 = the default head's w
+    p, s, d = oracle.route_classes(oracle.HEAD_SOFTMAX, r.hidden, w, [0.125, 0.375], 0.5)
+    w_diff = torch.from_numpy(w[1] - w[0])
+    s_ref, d_ref = oracle.route(r.hidden, w_diff, 0.25, 0.5)
+    assert np.allclose(s, s_ref, atol=1e-12) and (d == d_ref).all()
+    assert np.allclose(p.sum(axis=1), 1.0, atol=1e-15) and np.allclose(p[:, 1], s, atol=1e-15)
+
+
+@pytest.mark.parametrize("C", [2, 4, 10])
+def test_softmax_head_against_library_softmax(C):
+    rng = np.random.default_rng(C)
+    hidden = rng.normal(size=(9, 64)).astype(np.float32)
+    w = rng.normal(0, 0.2, size=(C, 64)).astype(np.float32)
+    b = rng.normal(0, 0.3, size=C)
+    p, s, d = oracle.route_classes(oracle.HEAD_SOFTMAX, hidden, w, b, 0.5)
+    logits = hidden.astype(np.float64) @ w.astype(np.float64).T + b
+    p_ref = softmax(logits, axis=1)
+    assert np.allclose(p, p_ref, atol=1e-13)
+    assert np.allclose(s, p_ref @ (np.arange(C) / (C - 1)), atol=1e-13)
+    assert (d == (s.astype(np.float32) > np.float32(0.5))).all()
+
+
+def test_softmax_head_closed_forms():
+    hidden = np.zeros((3, 8), dtype=np.float32)
+    hidden[1, 0] = 1.0
+    hidden[2, 0] = 1.0
+    w = np.zeros((4, 8), dtype=np.float32)
+    w[2, 0] = 60.0                                            # row 1, 2: class 2 dominates by 60 nats
+    p, s, d = oracle.route_classes(oracle.HEAD_SOFTMAX, hidden, w, [0.0] * 4, 0.5)
+    assert np.allclose(p[0], 0.25) and s[0] == 0.5 and d[0] == 0       # equal logits; a tie accepts
+    assert abs(s[1] - 2 / 3) < 1e-12 and d[1] == 1
+
+
+def test_ordinal_head_closed_forms_and_two_class_case():
+    hidden = np.zeros((2, 8), dtype=np.float32)
+    hidden[1, 0] = 1.0
+    w = np.zeros((1, 8), dtype=np.float32)
+    w[0, 0] = math.log(3.0)
+    cuts = [-math.log(3.0), 0.0, math.log(3.0)]
+    p, s, d = oracle.route_classes(oracle.HEAD_ORDINAL, hidden, w, [0.0] + cuts, 0.5)
+    # z = 0: P(y >= k) = 3/4, 1/2, 1/4 -> four equal classes, expected level 1/2
+    assert np.allclose(p[0], 0.25, atol=1e-15) and abs(s[0] - 0.5) < 1e-15 and d[0] == 0
+    # z = ln 3 (as rounded to fp32, hence 1e-7): P(y >= k) = sigmoid(ln 9), sigmoid(ln 3), 1/2 = 0.9, 0.75, 0.5
+    assert np.allclose(p[1], [0.1, 0.15, 0.25, 0.5], rtol=0, atol=1e-7) and abs(s[1] - (0.9 + 0.75 + 0.5) / 3) < 1e-7
+    r = wl.make_router_inputs(12, 128, torch.float32, seed=9)
+    p2, s2, d2 = oracle.route_classes(oracle.HEAD_ORDINAL, r.hidden, r.w.reshape(1, -1), [0.3, 0.0], 0.4)
+    s_ref, d_ref = oracle.route(r.hidden, r.w, 0.3, 0.4)     # one cut at 0: the default head again
+    assert np.allclose(s2, s_ref, atol=1e-12) and (d2 == d_ref).all()
+    z = r.hidden.double().numpy() @ r.w.double().numpy() + 0.3
+    assert np.allclose(p2[:, 1], expit(z), atol=1e-12)
+
+
+# ---- KV append ---------------------------------------------------------------------------------------
+
+def _append_case(dtype, seed):
+    inp = wl.small_attn_case(3, 8, 2, 64, dtype, [40, 17, 96], [1, 1, 1], seed=seed, extra_tokens=40)
+    gen = torch.Generator().manual_seed(seed + 1)
+    new_lens = torch.tensor([5, 0, 33], dtype=torch.int32)
+    k_new = torch.randn(int(new_lens.sum()), 2, 64, generator=gen).to(dtype)
+    v_new = torch.randn(int(new_lens.sum()), 2, 64, generator=gen).to(dtype)
+    return inp, new_lens, k_new, v_new
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+def test_kv_append_puts_every_token_where_attention_reads_it(dtype):
+    inp, new_lens, k_new, v_new = _append_case(dtype, 21)
+    kp, vp, sl, st = oracle.kv_append(k_new, v_new, inp.block_table, inp.seq_lens, new_lens, inp.k_pages, inp.v_pages)
+    assert st == 0 and list(sl) == [45, 17, 129]
+    # independent placement by plain indexing
+    k_ref, v_ref = inp.k_pages.clone(), inp.v_pages.clone()
+    row = 0
+    for b in range(3):
+        for j in range(int(new_lens[b])):
+            pos = int(inp.seq_lens[b]) + j
+            page = int(inp.block_table[b, pos // 16])
+            k_ref[page, :, pos % 16, :] = k_new[row]
+            v_ref[page, :, pos % 16, :] = v_new[row]
+            row += 1
+    assert torch.equal(kp, k_ref) and torch.equal(vp, v_ref)
+    # and attention over the grown cache sees the new tokens: the last query of sequence 2 at its new length
+    q = inp.q
+    out, st2 = oracle.attn(q, kp, vp, inp.block_table, torch.from_numpy(sl), inp.q_lens)
+    out_old, _ = oracle.attn(q, inp.k_pages, inp.v_pages, inp.block_table, inp.seq_lens, inp.q_lens)
+    assert st2 == 0 and not np.allclose(out[2], out_old[2]) and np.array_equal(out[1], out_old[1])
+
+
+def test_kv_append_refuses_what_does_not_fit():
+    inp, new_lens, k_new, v_new = _append_case(torch.float32, 22)
+    cap = inp.block_table.shape[1] * 16
+    too_long = torch.tensor([5, 0, cap], dtype=torch.int32)
+    big_k = torch.zeros(int(too_long.sum()), 2, 64)
+    kp, vp, sl, st = oracle.kv_append(big_k, big_k, inp.block_table, inp.seq_lens, too_long, inp.k_pages, inp.v_pages)
+    assert st & oracle.BAD_SEQ_LEN and list(sl) == [45, 17, 96]
+    bad_bt = inp.block_table.clone()
+    bad_bt[0, 40 // 16] = inp.k_pages.shape[0] + 3
+    kp, vp, sl, st = oracle.kv_append(k_new, v_new, bad_bt, inp.seq_lens, new_lens, inp.k_pages, inp.v_pages)
+    assert st & oracle.BAD_PAGE and list(sl) == [40, 17, 129]
+    neg = torch.tensor([-1, 0, 0], dtype=torch.int32)
+    kp, vp, sl, st = oracle.kv_append(k_new[:0], v_new[:0], inp.block_table, inp.seq_lens, neg, inp.k_pages, inp.v_pages)
+    assert st & oracle.BAD_SEQ_LEN and torch.equal(kp, inp.k_pages)
+
+
+def test_rollback_then_append_overwrites_the_rejected_step():
+    """Algorithm 1, escalation branch: the rejected draft step's slots are reused by the target's step."""
+    inp, new_lens, k_new, v_new = _append_case(torch.float32, 23)
+    kp, vp, sl, _ = oracle.kv_append(k_new, v_new, inp.block_table, inp.seq_lens, new_lens, inp.k_pages, inp.v_pages)
+    rolled, _ = oracle.rollback(sl, new_lens.numpy(), np.array([1, 1, 1], dtype=np.uint8))
+    assert list(rolled) == [40, 17, 96]
+    k2, v2 = -k_new, -v_new
+    kp2, vp2, sl2, _ = oracle.kv_append(k2, v2, inp.block_table, torch.from_numpy(rolled), new_lens, kp, vp)
+    kp_direct, vp_direct, _, _ = oracle.kv_append(k2, v2, inp.block_table, inp.seq_lens, new_lens, inp.k_pages, inp.v_pages)
+    assert torch.equal(kp2, kp_direct) and torch.equal(vp2, vp_direct) and list(sl2) == list(sl)

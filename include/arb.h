@@ -15,6 +15,10 @@
  *                 same prefix x, so a cache that absorbed the rejected draft step drops it by
  *                 resetting its length; no KV bytes move.
  *
+ * Around them: arb_kv_append (the cache write of a step's new tokens), arb_policy (the escalation rules
+ * the paper compares on PRM scores: RSD, oracle threshold / arg max, budgeted oracle, with the wasted
+ * target calls) and arb_route_classes (the C-way heads of the router ablation).
+ *
  * Conventions shared by every call
  *   - Pointers are DEVICE pointers unless the argument says "host".  The caller owns every tensor;
  *     the library owns only the arb_ctx (split-KV partials, arrival counters, a status word and
@@ -60,6 +64,26 @@ enum {
     ARB_DEV_ROLLBACK_UNDERFLOW = 4u, /* step_len < 0 or step_len > seq_len */
     ARB_DEV_WAIT_TIMEOUT = 8u        /* a bounded wait on an asynchronous copy or MMA gave up */
 };
+
+/* escalation policies of arb_policy */
+typedef enum {
+    ARB_POLICY_RSD = 0,              /* escalate iff s_d <= tau (the step is accepted iff s_d > tau) */
+    ARB_POLICY_ORACLE_THRESHOLD = 1, /* escalate iff s_t - s_d > tau */
+    ARB_POLICY_ORACLE_ARGMAX = 2,    /* escalate iff s_t > s_d */
+    ARB_POLICY_ORACLE_BUDGET = 3     /* escalate the min(budget, #{s_t - s_d > 0}) largest positive advantages */
+} arb_policy_kind;
+
+/* what a policy did, accumulated on the device by arb_policy */
+typedef struct {
+    uint32_t escalated; /* steps sent to the target */
+    uint32_t wasted;    /* of those, steps with s_t <= s_d: the target call bought nothing */
+    double realised;    /* sum over steps of the score of the step that was kept: a ? s_t : s_d */
+    double gain;        /* sum over escalated steps of s_t - s_d */
+} arb_policy_stats;
+
+/* C-way router heads of arb_route_classes */
+typedef enum { ARB_HEAD_SOFTMAX = 0, ARB_HEAD_ORDINAL = 1 } arb_head_kind;
+#define ARB_MAX_CLASSES 16
 
 typedef struct CUstream_st *arb_stream_t; /* same type as cudaStream_t */
 typedef struct arb_ctx arb_ctx;
@@ -216,6 +240,71 @@ arb_status arb_route(arb_ctx *ctx, int32_t dtype, int32_t n_steps, int32_t hidde
  */
 arb_status arb_rollback(arb_ctx *ctx, int32_t batch, int32_t *seq_lens, const int32_t *step_lens,
                         const uint8_t *decisions /* nullable */, arb_stream_t stream);
+
+/*
+ * Escalation decisions from PRM scores, for the policies the paper compares (Section 3.1: the RSD
+ * baseline accepts a draft step iff s_d > tau; Section 4.1: the oracle keeps the higher-scoring of the
+ * draft and target step, or escalates iff the advantage Delta = s_t - s_d exceeds tau; Appendix B,
+ * Theorem: under a budget of B escalations the best policy takes the largest positive advantages), and
+ * what each costs (Section 3.2: a target call is wasted when s_t <= s_d; Section 4.1: the realised
+ * score is S(a) = s_d + a Delta).
+ *
+ *   s_d, s_t   fp32 [n_steps]: PRM score of the draft step and of the target's counterpart.  s_t may be
+ *              NULL for ARB_POLICY_RSD when stats is NULL.  Scores are finite.
+ *   tau        threshold (RSD, oracle threshold); budget: escalations allowed (budgeted oracle,
+ *              n_steps <= 65536).
+ *   decisions  uint8 [n_steps]: 1 = escalate to the target, 0 = keep the draft step.  Ties: RSD escalates
+ *              at s_d == tau; the oracle rules keep the draft at Delta == tau / s_t == s_d; among equal
+ *              advantages the budgeted rule takes the lower index first.
+ *   stats      nullable; zeroed on `stream`, then filled by the kernel (sums in fp64).
+ * Delta and every comparison are taken in fp32 (IEEE subtraction, no flush to zero).
+ * Errors: ARB_ERR_INVALID_ARG (null pointer, unknown kind, s_t missing), ARB_ERR_UNSUPPORTED (budgeted
+ * rule beyond 65536 steps).
+ */
+arb_status arb_policy(arb_ctx *ctx, int32_t kind, int32_t n_steps, const float *s_d, const float *s_t, float tau,
+                      int32_t budget, uint8_t *decisions, arb_policy_stats *stats /* nullable */,
+                      arb_stream_t stream);
+
+/*
+ * C-way router heads (Section 6.1, "Label Granularity" and "Classification vs. Regression": heads over
+ * 2, 4 or 10 ordered classes of the advantage, and a 4-level ordinal head).  The paper does not say how
+ * a C-way head becomes one routing score; here it is the expected class level scaled to [0, 1],
+ * score = sum_c p_c * c / (C - 1), and the step escalates iff score > tau (a tie accepts).  For C = 2
+ * that is arb_route with w = w1 - w0, b = b1 - b0.
+ *
+ *   mode       ARB_HEAD_SOFTMAX: logits l_c = hidden . w[c] + b[c], p = softmax(l); w is [C, hidden_dim].
+ *              ARB_HEAD_ORDINAL: one logit z = hidden . w[0] + b[0] and cut points b[1] <= ... <= b[C-1]:
+ *              P(y >= k) = sigmoid(z - b[k]), p_k = P(y >= k) - P(y >= k + 1); w is [hidden_dim].
+ *   hidden     [n_steps, hidden_dim], hidden_dim a multiple of 8; w has hidden's dtype.
+ *   b_host     HOST pointer to n_classes floats (2 <= n_classes <= ARB_MAX_CLASSES).
+ *   probs      nullable, fp32 [n_steps, n_classes]; scores fp32 [n_steps]; decisions uint8 [n_steps].
+ */
+arb_status arb_route_classes(arb_ctx *ctx, int32_t dtype, int32_t mode, int32_t n_steps, int32_t hidden_dim,
+                             int32_t n_classes, const void *hidden, const void *w, const float *b_host, float tau,
+                             float *probs /* nullable */, float *scores, uint8_t *decisions, arb_stream_t stream);
+
+/*
+ * KV append: writes the keys and values of each sequence's new tokens into the paged cache behind the
+ * tokens it already holds (the cache write that every "Sample draft step" / "Sample target step" of
+ * Algorithm 1 implies before the next arb_attn call may attend to them; after a rollback the same slots
+ * are overwritten by the regenerated step).
+ *
+ *   params     dtype, batch, num_kv_heads, head_dim, page_size, num_pages and max_pages_per_seq are
+ *              used; the other fields are ignored.
+ *   k_new,
+ *   v_new      [total_new, Hkv, D], packed by sequence in batch order: sequence b owns new_lens[b] rows.
+ *   seq_lens   int32 [B]: tokens held BEFORE the call.  Token j of sequence b goes to position
+ *              seq_lens[b] + j, i.e. page block_table[b][pos / P], slot pos % P.  With update_lens != 0
+ *              seq_lens[b] becomes seq_lens[b] + new_lens[b] (by a second small kernel), which is the
+ *              value arb_attn expects when it is called with q_lens = new_lens.
+ *   new_lens   int32 [B], >= 0; total_new >= their sum (rows beyond the sum are ignored).
+ * A sequence whose new tokens do not fit under its block-table row, or whose target pages lie outside
+ * the pool, is left untouched (pools and length) and raises ARB_DEV_BAD_SEQ_LEN / ARB_DEV_BAD_PAGE; a
+ * negative new_len raises ARB_DEV_BAD_SEQ_LEN.  Values are copied bit for bit.
+ */
+arb_status arb_kv_append(arb_ctx *ctx, const arb_attn_params *params, int32_t total_new, const void *k_new,
+                         const void *v_new, const int32_t *block_table, int32_t *seq_lens, const int32_t *new_lens,
+                         int32_t update_lens, void *k_pages, void *v_pages, arb_stream_t stream);
 
 /*
  * Synchronise `stream`, read the device status word into *bits (nullable) and clear it together

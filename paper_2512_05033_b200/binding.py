@@ -26,11 +26,15 @@ ARB_F32, ARB_BF16 = 0, 1
 DEV_BAD_SEQ_LEN, DEV_BAD_PAGE, DEV_ROLLBACK_UNDERFLOW, DEV_WAIT_TIMEOUT = 1, 2, 4, 8
 ATTN_OVERLAP_PREVIOUS = 1
 ATTN_NO_TENSOR_CORES = 2
+POLICY_RSD, POLICY_ORACLE_THRESHOLD, POLICY_ORACLE_ARGMAX, POLICY_ORACLE_BUDGET = 0, 1, 2, 3
+HEAD_SOFTMAX, HEAD_ORDINAL = 0, 1
+MAX_CLASSES = 16
 
 # every symbol include/arb.h declares
 EXPORTS = ("arb_create", "arb_destroy", "arb_attn_workspace_bytes", "arb_attn", "arb_attn_host",
            "arb_attn_decode_static",
-           "arb_route", "arb_rollback", "arb_poll_status", "arb_launch_count", "arb_status_string")
+           "arb_route", "arb_rollback", "arb_policy", "arb_route_classes", "arb_kv_append",
+           "arb_poll_status", "arb_launch_count", "arb_status_string")
 
 
 class AttnParams(ctypes.Structure):
@@ -58,6 +62,13 @@ lib.arb_route.restype = ctypes.c_int
 lib.arb_route.argtypes = [_vp, _i32, _i32, _i32, _vp, _vp, _f, _f, _vp, _vp, _vp]
 lib.arb_rollback.restype = ctypes.c_int
 lib.arb_rollback.argtypes = [_vp, _i32, _vp, _vp, _vp, _vp]
+lib.arb_policy.restype = ctypes.c_int
+lib.arb_policy.argtypes = [_vp, _i32, _i32, _vp, _vp, _f, _i32, _vp, _vp, _vp]
+lib.arb_route_classes.restype = ctypes.c_int
+lib.arb_route_classes.argtypes = [_vp, _i32, _i32, _i32, _i32, _i32, _vp, _vp, ctypes.POINTER(ctypes.c_float), _f,
+                                  _vp, _vp, _vp, _vp]
+lib.arb_kv_append.restype = ctypes.c_int
+lib.arb_kv_append.argtypes = [_vp, ctypes.POINTER(AttnParams), _i32, _vp, _vp, _vp, _vp, _vp, _i32, _vp, _vp, _vp]
 lib.arb_poll_status.restype = ctypes.c_int
 lib.arb_poll_status.argtypes = [_vp, _vp, ctypes.POINTER(ctypes.c_uint32)]
 lib.arb_launch_count.restype = ctypes.c_uint64
@@ -213,6 +224,70 @@ class Context:
         st = lib.arb_rollback(self._h, seq_lens.shape[0], _dev(seq_lens, "seq_lens", torch.int32),
                               _dev(step_lens, "step_lens", torch.int32), dp, _stream_ptr(stream))
         _check(st, "arb_rollback")
+        return seq_lens
+
+    # -- arb_policy ---------------------------------------------------------------------------
+    def policy(self, kind: int, s_d, s_t=None, tau: float = 0.0, budget: int = 0, decisions=None, stats=None,
+               stream=None):
+        """Escalation decisions uint8 [N] from PRM scores (fp32 device tensors).  `stats`, if given, is a
+        device tensor of 3 float64 that receives the arb_policy_stats record (two uint32 counters, then the
+        realised score and the gain); read it with policy_stats()."""
+        n = s_d.shape[0]
+        if decisions is None:
+            decisions = torch.empty(n, dtype=torch.uint8, device=s_d.device)
+        sp = None if stats is None else _dev(stats, "stats", torch.float64)
+        tp = None if s_t is None else _dev(s_t, "s_t", torch.float32)
+        st = lib.arb_policy(self._h, kind, n, _dev(s_d, "s_d", torch.float32), tp, float(tau), int(budget),
+                            _dev(decisions, "decisions", torch.uint8), sp, _stream_ptr(stream))
+        _check(st, "arb_policy")
+        return decisions
+
+    @staticmethod
+    def new_policy_stats(device):
+        return torch.zeros(3, dtype=torch.float64, device=device)
+
+    @staticmethod
+    def policy_stats(stats) -> dict:
+        """Decodes the 24-byte arb_policy_stats record held in a float64[3] tensor (synchronises)."""
+        raw = stats.cpu().numpy().tobytes()
+        import struct
+        esc, wasted, realised, gain = struct.unpack("<IIdd", raw)
+        return {"escalated": esc, "wasted": wasted, "realised": realised, "gain": gain}
+
+    # -- arb_route_classes --------------------------------------------------------------------
+    def route_classes(self, mode: int, hidden, w, b, tau: float, probs=None, scores=None, decisions=None,
+                      stream=None):
+        """C-way head: returns (probs fp32 [S, C], scores fp32 [S], decisions uint8 [S]).  b: C host floats."""
+        S, H = hidden.shape
+        C = len(b)
+        if probs is None:
+            probs = torch.empty(S, C, dtype=torch.float32, device=hidden.device)
+        if scores is None:
+            scores = torch.empty(S, dtype=torch.float32, device=hidden.device)
+        if decisions is None:
+            decisions = torch.empty(S, dtype=torch.uint8, device=hidden.device)
+        bh = (ctypes.c_float * C)(*[float(x) for x in b])
+        st = lib.arb_route_classes(self._h, _dtype_code(hidden), mode, S, H, C, _dev(hidden, "hidden"),
+                                   _dev(w, "w", hidden.dtype), bh, float(tau), _dev(probs, "probs", torch.float32),
+                                   _dev(scores, "scores", torch.float32), _dev(decisions, "decisions", torch.uint8),
+                                   _stream_ptr(stream))
+        _check(st, "arb_route_classes")
+        return probs, scores, decisions
+
+    # -- arb_kv_append ------------------------------------------------------------------------
+    def kv_append(self, k_new, v_new, block_table, seq_lens, new_lens, k_pages, v_pages, update_lens: bool = True,
+                  stream=None):
+        """In place: the new tokens' K/V go behind each sequence's cached tokens; seq_lens += new_lens."""
+        num_pages, Hkv, P, D = k_pages.shape
+        B, max_pages = block_table.shape
+        p = attn_params(_dtype_code(k_pages), B, Hkv, Hkv, D, num_pages, max_pages, 0, 0, 0.0, P, 0)
+        total_new = k_new.shape[0]
+        st = lib.arb_kv_append(self._h, ctypes.byref(p), total_new, _dev(k_new, "k_new", k_pages.dtype),
+                               _dev(v_new, "v_new", k_pages.dtype), _dev(block_table, "block_table", torch.int32),
+                               _dev(seq_lens, "seq_lens", torch.int32), _dev(new_lens, "new_lens", torch.int32),
+                               1 if update_lens else 0, _dev(k_pages, "k_pages"), _dev(v_pages, "v_pages", k_pages.dtype),
+                               _stream_ptr(stream))
+        _check(st, "arb_kv_append")
         return seq_lens
 
     # -- status -------------------------------------------------------------------------------

@@ -228,6 +228,50 @@ arb_status arb_rollback(arb_ctx *ctx, int32_t batch, int32_t *seq_lens, const in
                            reinterpret_cast<cudaStream_t>(stream));
 }
 
+arb_status arb_policy(arb_ctx *ctx, int32_t kind, int32_t n_steps, const float *s_d, const float *s_t, float tau,
+                      int32_t budget, uint8_t *decisions, arb_policy_stats *stats, arb_stream_t stream) {
+    if (ctx == nullptr || n_steps < 0) return ARB_ERR_INVALID_ARG;
+    if (kind < ARB_POLICY_RSD || kind > ARB_POLICY_ORACLE_BUDGET) return ARB_ERR_INVALID_ARG;
+    if (n_steps == 0) return ARB_OK;
+    if (!s_d || !decisions) return ARB_ERR_INVALID_ARG;
+    if (!s_t && (kind != ARB_POLICY_RSD || stats != nullptr)) return ARB_ERR_INVALID_ARG;
+    if (kind == ARB_POLICY_ORACLE_BUDGET && n_steps > 65536) return ARB_ERR_UNSUPPORTED;
+    if (stats != nullptr && (reinterpret_cast<uintptr_t>(stats) & 7u) != 0) return ARB_ERR_INVALID_ARG;
+    return launch_policy(reinterpret_cast<Ctx *>(ctx), kind, n_steps, s_d, s_t, tau, budget, decisions, stats,
+                         reinterpret_cast<cudaStream_t>(stream));
+}
+
+arb_status arb_route_classes(arb_ctx *ctx, int32_t dtype, int32_t mode, int32_t n_steps, int32_t hidden_dim,
+                             int32_t n_classes, const void *hidden, const void *w, const float *b_host, float tau,
+                             float *probs, float *scores, uint8_t *decisions, arb_stream_t stream) {
+    if (ctx == nullptr || n_steps < 0 || hidden_dim < 1) return ARB_ERR_INVALID_ARG;
+    if (dtype != ARB_F32 && dtype != ARB_BF16) return ARB_ERR_UNSUPPORTED;
+    if (mode != ARB_HEAD_SOFTMAX && mode != ARB_HEAD_ORDINAL) return ARB_ERR_INVALID_ARG;
+    if (n_classes < 2 || n_classes > ARB_MAX_CLASSES || hidden_dim % 8 != 0) return ARB_ERR_UNSUPPORTED;
+    if (n_steps == 0) return ARB_OK;
+    if (!hidden || !w || !b_host || !scores || !decisions) return ARB_ERR_INVALID_ARG;
+    if (!aligned16(hidden) || !aligned16(w)) return ARB_ERR_INVALID_ARG;
+    return launch_route_classes(reinterpret_cast<Ctx *>(ctx), dtype, mode, n_steps, hidden_dim, n_classes, hidden, w,
+                                b_host, tau, probs, scores, decisions, reinterpret_cast<cudaStream_t>(stream));
+}
+
+arb_status arb_kv_append(arb_ctx *ctx, const arb_attn_params *params, int32_t total_new, const void *k_new,
+                         const void *v_new, const int32_t *block_table, int32_t *seq_lens, const int32_t *new_lens,
+                         int32_t update_lens, void *k_pages, void *v_pages, arb_stream_t stream) {
+    if (ctx == nullptr || params == nullptr || total_new < 0) return ARB_ERR_INVALID_ARG;
+    if (params->batch < 1 || params->num_kv_heads < 1 || params->num_pages < 1 || params->max_pages_per_seq < 1)
+        return ARB_ERR_INVALID_ARG;
+    if (params->dtype != ARB_F32 && params->dtype != ARB_BF16) return ARB_ERR_UNSUPPORTED;
+    if (params->head_dim != 64 && params->head_dim != 128) return ARB_ERR_UNSUPPORTED;
+    if (params->page_size != kPage || params->batch > kMaxBatch) return ARB_ERR_UNSUPPORTED;
+    if (!block_table || !seq_lens || !new_lens || !k_pages || !v_pages) return ARB_ERR_INVALID_ARG;
+    if (total_new == 0) return ARB_OK;
+    if (!k_new || !v_new) return ARB_ERR_INVALID_ARG;
+    if (!aligned16(k_new) || !aligned16(v_new) || !aligned16(k_pages) || !aligned16(v_pages)) return ARB_ERR_INVALID_ARG;
+    return launch_kv_append(reinterpret_cast<Ctx *>(ctx), *params, total_new, k_new, v_new, block_table, seq_lens,
+                            new_lens, update_lens, k_pages, v_pages, reinterpret_cast<cudaStream_t>(stream));
+}
+
 arb_status arb_poll_status(arb_ctx *ctx, arb_stream_t stream, uint32_t *bits) {
     if (ctx == nullptr) return ARB_ERR_INVALID_ARG;
     Ctx *c = reinterpret_cast<Ctx *>(ctx);

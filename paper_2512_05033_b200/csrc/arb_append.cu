@@ -1,0 +1,146 @@
+// KV append: the keys and values of a step's new tokens go into the paged cache, right behind the
+// tokens each sequence already holds (the write every "Sample ... step" line of Algorithm 1 of the
+// paper implies before the next token, or the router's forward, attends to them).
+//
+// k_new, v_new are [total_new, Hkv, D], packed by sequence; token j of sequence b lands at position
+// seq_lens[b] + j: page block_table[b][pos / 16], slot pos % 16 of the head-major pools
+// [num_pages, Hkv, 16, D].  Plain memory movement: a (token, kv head) row of D elements is 256 or 512
+// contiguous bytes on both sides, copied as 16-byte vectors, one row per half warp or warp.  Nothing
+// is known on the host but the total number of new tokens; every CTA derives the row offsets from
+// new_lens (scan in shared memory) and checks each sequence once: new tokens that do not fit under the
+// block table, or that would land on a page outside the pool, leave that sequence untouched and set a
+// status bit.  Lengths are advanced by a second, one-CTA kernel, after every CTA of the first has read
+// them.
+#include "arb_common.cuh"
+
+namespace arb {
+
+namespace {
+
+constexpr int kAppendThreads = 256;
+
+struct AppendArgs {
+    const char *k_new, *v_new;
+    char *k_pages, *v_pages;
+    const int32_t *block_table;
+    int32_t *seq_lens;
+    const int32_t *new_lens;
+    uint32_t *status;
+    int batch, Hkv, num_pages, max_pages;
+    int row_bytes;   // D * element size: bytes of one (token, kv head) row
+    int total_new;
+};
+
+// 0 = append, otherwise the status bit that explains why not (new_len == 0 appends nothing and is fine)
+__device__ __forceinline__ uint32_t append_check(const AppendArgs &a, int b) {
+    const int n = a.new_lens[b], L = a.seq_lens[b];
+    if (n == 0) return 0;
+    if (n < 0 || L < 0 || (long long)L + n > (long long)a.max_pages * kPage) return ARB_DEV_BAD_SEQ_LEN;
+    for (int pg = L / kPage; pg <= (L + n - 1) / kPage; ++pg) {
+        const int page = a.block_table[(size_t)b * a.max_pages + pg];
+        if ((unsigned)page >= (unsigned)a.num_pages) return ARB_DEV_BAD_PAGE;
+    }
+    return 0;
+}
+
+__global__ void __launch_bounds__(kAppendThreads)
+kv_append_kernel(const AppendArgs a) {
+    extern __shared__ int asm_[];
+    int *pref = asm_;                  // [B + 1] new rows before sequence b
+    int *okay = pref + a.batch + 1;    // [B] the sequence's new tokens may be written
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int B = a.batch;
+    if (tid == 0) pref[0] = 0;
+    for (int b = tid; b < B; b += kAppendThreads) {
+        const uint32_t bad = append_check(a, b);
+        if (bad && blockIdx.x == 0) atomicOr(a.status, bad);
+        okay[b] = bad == 0;
+        const int n = a.new_lens[b];
+        pref[b + 1] = n > 0 ? n : 0;
+    }
+    __syncthreads();
+    if (warp == 0) {
+        int carry = 0;
+        for (int b0 = 0; b0 < B; b0 += 32) {
+            const int b = b0 + lane;
+            int v = b < B ? pref[b + 1] : 0;
+#pragma unroll
+            for (int off = 1; off < 32; off <<= 1) {
+                const int t = __shfl_up_sync(0xffffffffu, v, off);
+                if (lane >= off) v += t;
+            }
+            if (b < B) pref[b + 1] = v + carry;
+            carry += __shfl_sync(0xffffffffu, v, 31);
+        }
+    }
+    __syncthreads();
+    const int total = min(pref[B], a.total_new);
+    const int vecs = a.row_bytes / 16;             // 16 (bf16, D 128 / fp32, D 64), 8 or 32
+    const int rows_per_pass = kAppendThreads / vecs;
+    const int sub = tid / vecs, vec = tid - sub * vecs;
+    const long long nrows = (long long)total * a.Hkv;
+    for (long long r = (long long)blockIdx.x * rows_per_pass + sub; r < nrows; r += (long long)gridDim.x * rows_per_pass) {
+        const int tok = (int)(r / a.Hkv), h = (int)(r - (long long)tok * a.Hkv);
+        int lo = 0, hi = B;
+        while (hi - lo > 1) {
+            const int mid = (lo + hi) >> 1;
+            if (pref[mid] <= tok) lo = mid; else hi = mid;
+        }
+        if (!okay[lo]) continue;
+        const int pos = a.seq_lens[lo] + (tok - pref[lo]);
+        const int page = a.block_table[(size_t)lo * a.max_pages + pos / kPage];
+        const size_t dst = (((size_t)page * a.Hkv + h) * kPage + (pos % kPage)) * a.row_bytes + (size_t)vec * 16;
+        const size_t src = (size_t)r * a.row_bytes + (size_t)vec * 16;
+        const uint4 kx = __ldg(reinterpret_cast<const uint4 *>(a.k_new + src));
+        const uint4 vx = __ldg(reinterpret_cast<const uint4 *>(a.v_new + src));
+        *reinterpret_cast<uint4 *>(a.k_pages + dst) = kx;
+        *reinterpret_cast<uint4 *>(a.v_pages + dst) = vx;
+    }
+}
+
+__global__ void __launch_bounds__(kAppendThreads)
+advance_lens_kernel(const AppendArgs a) {
+    for (int b = threadIdx.x; b < a.batch; b += kAppendThreads) {
+        const int n = a.new_lens[b];
+        if (n > 0 && append_check(a, b) == 0) a.seq_lens[b] += n;
+    }
+}
+
+}  // namespace
+
+arb_status launch_kv_append(Ctx *ctx, const arb_attn_params &p, int total_new, const void *k_new, const void *v_new,
+                            const int32_t *block_table, int32_t *seq_lens, const int32_t *new_lens, int update_lens,
+                            void *k_pages, void *v_pages, cudaStream_t stream) {
+    AppendArgs a;
+    a.k_new = static_cast<const char *>(k_new);
+    a.v_new = static_cast<const char *>(v_new);
+    a.k_pages = static_cast<char *>(k_pages);
+    a.v_pages = static_cast<char *>(v_pages);
+    a.block_table = block_table;
+    a.seq_lens = seq_lens;
+    a.new_lens = new_lens;
+    a.status = ctx->status;
+    a.batch = p.batch;
+    a.Hkv = p.num_kv_heads;
+    a.num_pages = p.num_pages;
+    a.max_pages = p.max_pages_per_seq;
+    a.row_bytes = p.head_dim * (p.dtype == ARB_BF16 ? 2 : 4);
+    a.total_new = total_new;
+    const int rows_per_pass = kAppendThreads / (a.row_bytes / 16);
+    const long long nrows = (long long)total_new * p.num_kv_heads;
+    long long want = (nrows + rows_per_pass - 1) / rows_per_pass;
+    const long long cap = (long long)ctx->num_sms * 4;
+    const int grid = (int)(want < 1 ? 1 : (want > cap ? cap : want));
+    const size_t smem = sizeof(int) * (2 * (size_t)p.batch + 1);
+    kv_append_kernel<<<grid, kAppendThreads, smem, stream>>>(a);
+    ctx->launches++;
+    if (cudaGetLastError() != cudaSuccess) return ARB_ERR_CUDA;
+    if (update_lens) {
+        advance_lens_kernel<<<1, kAppendThreads, 0, stream>>>(a);
+        ctx->launches++;
+        if (cudaGetLastError() != cudaSuccess) return ARB_ERR_CUDA;
+    }
+    return ARB_OK;
+}
+
+}  // namespace arb

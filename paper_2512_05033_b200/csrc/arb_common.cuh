@@ -194,6 +194,14 @@ arb_status launch_rollback(Ctx *ctx, int batch, int32_t *seq_lens, const int32_t
 arb_status launch_decode_static(const arb_attn_params &p, const void *q, const void *k_pages, const void *v_pages,
                                 const int32_t *block_table, const int32_t *seq_lens, const int32_t *q_lens,
                                 void *out, uint32_t *device_status, cudaStream_t stream);
+arb_status launch_policy(Ctx *ctx, int kind, int n_steps, const float *s_d, const float *s_t, float tau, int budget,
+                         uint8_t *decisions, arb_policy_stats *stats, cudaStream_t stream);
+arb_status launch_route_classes(Ctx *ctx, int dtype, int mode, int n_steps, int hidden_dim, int n_classes,
+                                const void *hidden, const void *w, const float *b_host, float tau, float *probs,
+                                float *scores, uint8_t *decisions, cudaStream_t stream);
+arb_status launch_kv_append(Ctx *ctx, const arb_attn_params &p, int total_new, const void *k_new, const void *v_new,
+                            const int32_t *block_table, int32_t *seq_lens, const int32_t *new_lens, int update_lens,
+                            void *k_pages, void *v_pages, cudaStream_t stream);
 size_t decode_workspace_bytes(const arb_attn_params &p, int num_sms);
 int decode_grid(int num_sms);
 

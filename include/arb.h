@@ -307,6 +307,20 @@ arb_status arb_kv_append(arb_ctx *ctx, const arb_attn_params *params, int32_t to
                          int32_t update_lens, void *k_pages, void *v_pages, arb_stream_t stream);
 
 /*
+ * Lengths of the next call of a phase of Algorithm 1, derived on the device so that the loop never reads
+ * a length or a decision on the host: after the routing decision, accepted steps are absorbed by the
+ * caches that did not generate them, and escalated steps are regenerated token by token by the target.
+ *
+ *   step_lens  int32 [B] (negative counts as 0);  decisions  uint8 [B], nullable.
+ *   A sequence takes part iff decisions is NULL or (decisions[b] != 0) == (want != 0).
+ *   t >= 0:  out[b] = 1 if it takes part and t < step_lens[b], else 0   (token t of a step decoded token by token)
+ *   t <  0:  out[b] = step_lens[b] if it takes part, else 0             (a whole step absorbed as one chunk)
+ *   out        int32 [B]; may be used as q_lens of arb_attn and as new_lens of arb_kv_append.
+ */
+arb_status arb_phase_lens(arb_ctx *ctx, int32_t batch, const int32_t *step_lens, const uint8_t *decisions /* nullable */,
+                          int32_t want, int32_t t, int32_t *out, arb_stream_t stream);
+
+/*
  * Synchronise `stream`, read the device status word into *bits (nullable) and clear it together
  * with the split-KV arrival counters.  Returns ARB_OK if the word was zero, else
  * ARB_ERR_DEVICE_STATUS.

@@ -30,6 +30,8 @@
  *    head (one logit, C - 1 ordered cut points).
  *  - oracle_kv_append: the write of a step's new keys and values into the paged cache that every
  *    "Sample ... step" line of Algorithm 1 implies before the next token attends to them.
+ *  - oracle_phase_lens: which sequences take part in a phase of Algorithm 1 (accepted steps are
+ *    absorbed by the target's cache, escalated ones are regenerated token by token by the target).
  *
  * Pins (tests/test_oracle_*.py): rows of softmax sum to one; uniform keys give the mean of V;
  * a single key returns its V; a dominant key returns its V; score-shift invariance; brute-force
@@ -386,4 +388,22 @@ unsigned oracle_kv_append(int esz, int B, int Hkv, int D, int P, long num_pages,
         row += (size_t)n;
     }
     return status;
+}
+
+
+/*
+ * Lengths of the next call of a phase of Algorithm 1, from the step lengths and the routing decisions.
+ * A sequence takes part in the phase iff decisions is NULL or (decisions[b] != 0) == (want != 0):
+ *   token t of a step generated token by token:  out[b] = 1 if it takes part and t < step_lens[b], else 0
+ *   a whole step absorbed at once (t < 0):        out[b] = step_lens[b] if it takes part, else 0
+ * Negative step lengths count as 0.
+ */
+void oracle_phase_lens(int B, const int32_t *step_lens, const uint8_t *decisions, int want, int t,
+                       int32_t *out)
+{
+    for (int b = 0; b < B; ++b) {
+        const int n = step_lens[b] > 0 ? step_lens[b] : 0;
+        const int in = decisions == NULL || ((decisions[b] != 0) == (want != 0));
+        out[b] = !in ? 0 : (t < 0 ? n : (t < n ? 1 : 0));
+    }
 }

@@ -55,6 +55,8 @@ def bind(lib):
     lib.oracle_policy.argtypes = [c_int, c_int, vp, vp, ctypes.c_float, c_int, vp, vp]
     lib.oracle_route_classes.restype = c_int
     lib.oracle_route_classes.argtypes = [c_int, c_int, c_int, c_int, c_int, vp, vp, vp, ctypes.c_float, vp, vp, vp]
+    lib.oracle_phase_lens.restype = None
+    lib.oracle_phase_lens.argtypes = [c_int, vp, vp, c_int, c_int, vp]
     lib.oracle_kv_append.restype = ctypes.c_uint
     lib.oracle_kv_append.argtypes = [c_int, c_int, c_int, c_int, c_int, c_long, c_int, vp, vp, vp, vp, vp, c_int, vp, vp]
     return lib
@@ -88,9 +90,9 @@ def _raw(t):
 
 
 def _i32(t):
-    if isinstance(t, np.ndarray):
-        return np.ascontiguousarray(t, dtype=np.int32)
-    return np.ascontiguousarray(t.detach().cpu().numpy().astype(np.int32))
+    if hasattr(t, "detach"):
+        return np.ascontiguousarray(t.detach().cpu().numpy().astype(np.int32))
+    return np.ascontiguousarray(np.asarray(t), dtype=np.int32)
 
 
 def attn(q, k_pages, v_pages, block_table, seq_lens, q_lens, scale: float = 0.0):
@@ -217,3 +219,17 @@ def kv_append(k_new, v_new, block_table, seq_lens, new_lens, k_pages, v_pages, u
                                   kn.data_ptr(), vn.data_ptr(), bt.ctypes.data, sl.ctypes.data, nl.ctypes.data,
                                   1 if update_lens else 0, kp.data_ptr(), vp_.data_ptr())
     return kp, vp_, sl, int(st)
+
+
+def phase_lens(step_lens, decisions=None, want: int = 1, t: int = -1):
+    """Per-sequence lengths of the next call of a phase of the step loop (int32 [B])."""
+    sl = _i32(step_lens)
+    if decisions is None:
+        dp, dk = None, None
+    else:
+        dk = np.ascontiguousarray(decisions.detach().cpu().numpy() if hasattr(decisions, "detach") else np.asarray(decisions),
+                                  dtype=np.uint8)
+        dp = dk.ctypes.data
+    out = np.zeros(sl.shape[0], dtype=np.int32)
+    _load().oracle_phase_lens(sl.shape[0], sl.ctypes.data, dp, int(want), int(t), out.ctypes.data)
+    return out

@@ -33,7 +33,7 @@ MAX_CLASSES = 16
 # every symbol include/arb.h declares
 EXPORTS = ("arb_create", "arb_destroy", "arb_attn_workspace_bytes", "arb_attn", "arb_attn_host",
            "arb_attn_decode_static",
-           "arb_route", "arb_rollback", "arb_policy", "arb_route_classes", "arb_kv_append",
+           "arb_route", "arb_rollback", "arb_policy", "arb_route_classes", "arb_kv_append", "arb_phase_lens",
            "arb_poll_status", "arb_launch_count", "arb_status_string")
 
 
@@ -62,6 +62,8 @@ lib.arb_route.restype = ctypes.c_int
 lib.arb_route.argtypes = [_vp, _i32, _i32, _i32, _vp, _vp, _f, _f, _vp, _vp, _vp]
 lib.arb_rollback.restype = ctypes.c_int
 lib.arb_rollback.argtypes = [_vp, _i32, _vp, _vp, _vp, _vp]
+lib.arb_phase_lens.restype = ctypes.c_int
+lib.arb_phase_lens.argtypes = [_vp, _i32, _vp, _vp, _i32, _i32, _vp, _vp]
 lib.arb_policy.restype = ctypes.c_int
 lib.arb_policy.argtypes = [_vp, _i32, _i32, _vp, _vp, _f, _i32, _vp, _vp, _vp]
 lib.arb_route_classes.restype = ctypes.c_int
@@ -225,6 +227,17 @@ class Context:
                               _dev(step_lens, "step_lens", torch.int32), dp, _stream_ptr(stream))
         _check(st, "arb_rollback")
         return seq_lens
+
+    # -- arb_phase_lens -----------------------------------------------------------------------
+    def phase_lens(self, step_lens, decisions=None, want: int = 1, t: int = -1, out=None, stream=None):
+        """out int32 [B]: lengths of the next call of a phase of the step loop (see arb_phase_lens)."""
+        if out is None:
+            out = torch.empty_like(step_lens)
+        dp = None if decisions is None else _dev(decisions, "decisions", torch.uint8)
+        st = lib.arb_phase_lens(self._h, step_lens.shape[0], _dev(step_lens, "step_lens", torch.int32), dp, int(want),
+                                int(t), _dev(out, "out", torch.int32), _stream_ptr(stream))
+        _check(st, "arb_phase_lens")
+        return out
 
     # -- arb_policy ---------------------------------------------------------------------------
     def policy(self, kind: int, s_d, s_t=None, tau: float = 0.0, budget: int = 0, decisions=None, stats=None,

@@ -194,6 +194,8 @@ arb_status launch_rollback(Ctx *ctx, int batch, int32_t *seq_lens, const int32_t
 arb_status launch_decode_static(const arb_attn_params &p, const void *q, const void *k_pages, const void *v_pages,
                                 const int32_t *block_table, const int32_t *seq_lens, const int32_t *q_lens,
                                 void *out, uint32_t *device_status, cudaStream_t stream);
+arb_status launch_phase_lens(Ctx *ctx, int batch, const int32_t *step_lens, const uint8_t *decisions, int want, int t,
+                             int32_t *out, cudaStream_t stream);
 arb_status launch_policy(Ctx *ctx, int kind, int n_steps, const float *s_d, const float *s_t, float tau, int budget,
                          uint8_t *decisions, arb_policy_stats *stats, cudaStream_t stream);
 arb_status launch_route_classes(Ctx *ctx, int dtype, int mode, int n_steps, int hidden_dim, int n_classes,

@@ -80,7 +80,24 @@ __global__ void rollback_kernel(int batch, int32_t *__restrict__ seq_lens, const
     seq_lens[i] = r;
 }
 
+// Lengths of the next call of a phase of the step loop (see arb_phase_lens): one thread per sequence.
+__global__ void phase_lens_kernel(int batch, const int32_t *__restrict__ step_lens, const uint8_t *__restrict__ decisions,
+                                  int want, int t, int32_t *__restrict__ out) {
+    const int b = blockIdx.x * blockDim.x + threadIdx.x;
+    if (b >= batch) return;
+    const int n = max(step_lens[b], 0);
+    const bool in = decisions == nullptr || ((decisions[b] != 0) == (want != 0));
+    out[b] = !in ? 0 : (t < 0 ? n : (t < n ? 1 : 0));
+}
+
 }  // namespace
+
+arb_status launch_phase_lens(Ctx *ctx, int batch, const int32_t *step_lens, const uint8_t *decisions, int want, int t,
+                             int32_t *out, cudaStream_t stream) {
+    phase_lens_kernel<<<(batch + 127) / 128, 128, 0, stream>>>(batch, step_lens, decisions, want, t, out);
+    ctx->launches++;
+    return cudaGetLastError() == cudaSuccess ? ARB_OK : ARB_ERR_CUDA;
+}
 
 arb_status launch_route(Ctx *ctx, int dtype, int n_steps, int hidden_dim, const void *hidden, const void *w,
                         float b, float tau, float *scores, uint8_t *decisions, cudaStream_t stream) {

@@ -232,3 +232,19 @@ def test_rollback_then_append_overwrites_the_rejected_step():
     kp2, vp2, sl2, _ = oracle.kv_append(k2, v2, inp.block_table, torch.from_numpy(rolled), new_lens, kp, vp)
     kp_direct, vp_direct, _, _ = oracle.kv_append(k2, v2, inp.block_table, inp.seq_lens, new_lens, inp.k_pages, inp.v_pages)
     assert torch.equal(kp2, kp_direct) and torch.equal(vp2, vp_direct) and list(sl2) == list(sl)
+
+
+def test_phase_lens_partitions_the_batch():
+    """Every sequence is in exactly one of the two branches after the decision, and a step decoded token by
+    token adds up to the step absorbed at once."""
+    rng = np.random.default_rng(3)
+    step = rng.integers(0, 9, 50).astype(np.int32)
+    dec = rng.integers(0, 2, 50).astype(np.uint8)
+    acc = oracle.phase_lens(step, dec, want=0, t=-1)
+    esc = oracle.phase_lens(step, dec, want=1, t=-1)
+    assert np.array_equal(acc + esc, step) and np.array_equal(acc[dec == 1], 0 * acc[dec == 1])
+    assert np.array_equal(esc, step * dec)
+    by_token = sum(oracle.phase_lens(step, dec, want=1, t=t) for t in range(9))
+    assert np.array_equal(by_token, esc)
+    assert list(oracle.phase_lens([3, -4, 0], None, t=-1)) == [3, 0, 0]
+    assert list(oracle.phase_lens([3, 1, 2], None, t=1)) == [1, 0, 1]

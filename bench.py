@@ -290,6 +290,9 @@ def run_ours(args):
                 result["target_shaped_decode"] = run_target_decode(ctx, dev, peak)
                 result["step_scoring"] = run_step_scoring(ctx, dev)
                 result["mixed_loop"] = run_mixed_loop(ctx, dev)
+                result["step_loop"] = run_step_loop(ctx, dev)
+                result["kv_append"] = run_kv_append(ctx, dev, peak)
+                result["policies"] = run_policies(ctx, dev)
             result["cpu_baseline"] = run_cpu_baseline(work)
     if dist:
         dist.barrier()
@@ -425,6 +428,114 @@ def run_mixed_loop(ctx, dev):
             "decode_tokens_per_s": round((B * len(m.q_lens) - scored) / (ms * 1e-3), 1),
             "kv_gbs_lower_bound": round(kv_tokens * esz / (ms * 1e-3) / 1e9, 1),
             "device_status_bits": ctx.poll_status()}
+
+
+def run_step_loop(ctx, dev):
+    """Supplementary: whole rounds of Algorithm 1 (step_loop.StepLoop) replayed as one CUDA graph.  Batch 16;
+    draft cache 12/2 heads, router cache 28/4 heads with a 3584-wide head, target cache 32/8 heads; prefixes
+    uniform in [2048, 8192]; draft and target steps of 8..32 tokens generated token by token; routing at
+    tau 0.5; escalated steps rolled back and regenerated; every cache absorbs the step it did not write.
+    One layer call per forward; lengths and decisions never leave the device."""
+    from paper_2512_05033_b200.step_loop import Cache, StepLoop
+    B, D, nd, nt, Hr, rounds = 16, 128, 32, 32, 3584, 2
+    bf = torch.bfloat16
+    gen = torch.Generator().manual_seed(41)
+    prefix = torch.randint(2048, 8193, (B,), generator=gen)
+    geometry = ((12, 2), (28, 4), (32, 8))   # draft, router, target: query / KV heads
+    caches, starts = [], []
+    for i, (hq, hkv) in enumerate(geometry):
+        shape = wl.AttnShape(f"loop-{i}", B, hq, hkv, D, bf, 0, 0, seed=50 + i)
+        inp = wl.make_attn_inputs(shape, device=dev, seed=50 + i, extra_tokens=rounds * (nd + nt) + 16,
+                                  prefix_lens=prefix, q_lens=torch.zeros(B, dtype=torch.int64))
+        caches.append(Cache(hq, inp.k_pages, inp.v_pages, inp.block_table, inp.seq_lens.clone()))
+        starts.append(inp.seq_lens.clone())
+    r = wl.make_router_inputs(B, Hr, bf, device=dev, seed=60)
+    loop = StepLoop(ctx, *caches, r.w, 0.0, 0.5, nd, nt)
+
+    def rows(n, heads, seed):
+        return wl.normal((n, heads, D), 1.0, bf, dev, seed)
+
+    def gen_rows(n, hq, hkv, seed):    # one row per sequence and token of a step written token by token
+        return tuple(rows(n * B, h, seed + j).view(n, B, h, D) for j, h in enumerate((hq, hkv, hkv)))
+
+    def chunk_rows(n, hq, hkv, seed):  # a whole step per sequence, packed
+        return tuple(rows(n * B, h, seed + j) for j, h in enumerate((hq, hkv, hkv)))
+
+    per_round = []
+    for k in range(rounds):
+        step_d = torch.randint(8, nd + 1, (B,), generator=gen, dtype=torch.int32).to(dev)
+        step_t = torch.randint(8, nt + 1, (B,), generator=gen, dtype=torch.int32).to(dev)
+        hidden = wl.normal((B, Hr), 1.0, bf, dev, 700 + k)
+        sd = 800 + 20 * k
+        acts = {"draft.gen": gen_rows(nd, 12, 2, sd), "target.gen": gen_rows(nt, 32, 8, sd + 3),
+                "router.zd": chunk_rows(nd, 28, 4, sd + 6), "target.zd": chunk_rows(nd, 32, 8, sd + 9),
+                "router.zt": chunk_rows(nt, 28, 4, sd + 12), "draft.zt": chunk_rows(nt, 12, 2, sd + 15)}
+        per_round.append((step_d, step_t, hidden, acts))
+
+    def run():
+        for c, s0 in zip(caches, starts):
+            c.seq_lens.copy_(s0)   # every replay starts from the same prefixes (outside the path)
+        for step_d, step_t, hidden, acts in per_round:
+            loop.round(step_d, step_t, hidden, acts)
+
+    run()
+    torch.cuda.synchronize()
+    n0 = ctx.launch_count()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g):
+        run()
+    launches = ctx.launch_count() - n0
+    ms = time_steps(g.replay, 10, 3) / 10
+    return {"rounds_per_graph": rounds, "batch": B, "kernels_per_graph": launches,
+            "ms_per_round": round(ms / rounds, 3), "steps_per_s": round(B * rounds / (ms * 1e-3), 1),
+            "escalation_rate_last_round": float(loop.decisions.float().mean().item()),
+            "device_status_bits": ctx.poll_status()}
+
+
+def run_kv_append(ctx, dev, peak):
+    """Supplementary: arb_kv_append alone on the step-scoring geometry (batch 32, 4 KV heads, steps of 16..128
+    tokens): bytes read from k_new / v_new plus bytes written to the pools, over the kernel time."""
+    shape = wl.STEP_SCORING
+    inp = wl.make_attn_inputs(shape, device=dev, seed=shape.seed, extra_tokens=160)
+    new = inp.q_lens.clone()
+    total = int(new.sum())
+    k_new = wl.normal((total, shape.num_kv_heads, shape.head_dim), 1.0, shape.dtype, dev, 901)
+    v_new = wl.normal((total, shape.num_kv_heads, shape.head_dim), 1.0, shape.dtype, dev, 902)
+    seq = inp.seq_lens.clone()
+    fn = lambda: ctx.kv_append(k_new, v_new, inp.block_table, seq, new, inp.k_pages, inp.v_pages, update_lens=False)
+    ms = time_steps(fn, 200, 10) / 200
+    nbytes = 4 * total * shape.num_kv_heads * shape.head_dim * 2
+    gbs = nbytes / (ms * 1e-3) / 1e9
+    return {"tokens": total, "bytes_per_call": nbytes, "us_per_call": round(ms * 1e3, 2), "gbs": round(gbs, 1),
+            "frac_of_measured": round(gbs / peak, 4), "note": "10 MB per call: bound by launch latency, not by HBM"}
+
+
+def run_policies(ctx, dev):
+    """Supplementary: arb_policy on 4096 synthetic PRM score pairs (uniform in [0, 1]) and the C-way heads on the
+    step-scoring router shape (32 steps, hidden 3584)."""
+    from paper_2512_05033_b200 import binding
+    n = 4096
+    sd = torch.rand(n, generator=torch.Generator().manual_seed(5)).to(dev)
+    st = torch.rand(n, generator=torch.Generator().manual_seed(6)).to(dev)
+    stats = ctx.new_policy_stats(dev)
+    dec = torch.empty(n, dtype=torch.uint8, device=dev)
+    out = {}
+    for name, kind, tau, budget in (("rsd_tau0.5", binding.POLICY_RSD, 0.5, 0),
+                                    ("oracle_tau0", binding.POLICY_ORACLE_THRESHOLD, 0.0, 0),
+                                    ("oracle_budget_25pct", binding.POLICY_ORACLE_BUDGET, 0.0, n // 4)):
+        fn = lambda: ctx.policy(kind, sd, st, tau=tau, budget=budget, decisions=dec, stats=stats)
+        ms = time_steps(fn, 100, 5) / 100
+        got = ctx.policy_stats(stats)
+        out[name] = {"us_per_call": round(ms * 1e3, 2), "steps_per_s": round(n / (ms * 1e-3), 0),
+                     "escalated": got["escalated"], "wasted": got["wasted"],
+                     "mean_realised_score": round(got["realised"] / n, 4)}
+    r = wl.make_router_inputs(32, 3584, torch.bfloat16, device=dev, seed=3)
+    for C in (4, 10):
+        w = wl.normal((C, 3584), 1.0 / 3584 ** 0.5, torch.bfloat16, dev, 950 + C)
+        fn = lambda: ctx.route_classes(binding.HEAD_SOFTMAX, r.hidden, w, [0.0] * C, 0.5)
+        ms = time_steps(fn, 100, 5) / 100
+        out[f"softmax_head_{C}_classes"] = {"us_per_call": round(ms * 1e3, 2), "steps_per_s": round(32 / (ms * 1e-3), 0)}
+    return out
 
 
 def run_cpu_baseline(work: DecodeWorkload):

@@ -30,6 +30,9 @@
  *    head (one logit, C - 1 ordered cut points).
  *  - oracle_kv_append: the write of a step's new keys and values into the paged cache that every
  *    "Sample ... step" line of Algorithm 1 implies before the next token attends to them.
+ *  - oracle_spearman: the rank correlation the paper reports between the router's predictions and the
+ *    oracle advantage (Section 4.2, "Evaluation"; Tables 1-3): Pearson correlation of the two rank
+ *    variables, ties sharing the mean of the ranks they span.
  *  - oracle_phase_lens: which sequences take part in a phase of Algorithm 1 (accepted steps are
  *    absorbed by the target's cache, escalated ones are regenerated token by token by the target).
  *
@@ -406,4 +409,40 @@ void oracle_phase_lens(int B, const int32_t *step_lens, const uint8_t *decisions
         const int in = decisions == NULL || ((decisions[b] != 0) == (want != 0));
         out[b] = !in ? 0 : (t < 0 ? n : (t < n ? 1 : 0));
     }
+}
+
+
+/*
+ * Spearman's rho of two samples: each value is replaced by its rank among its own sample (1 = smallest;
+ * equal values share the average of the ranks they occupy), and rho is the Pearson correlation of the two
+ * rank variables, rho = sum (rx - m)(ry - m) / sqrt(sum (rx - m)^2 * sum (ry - m)^2) with m = (n + 1) / 2.
+ * Returns NaN when n < 2 or a sample is constant (the correlation is undefined).  ranks_x / ranks_y
+ * (nullable) receive the ranks.
+ */
+double oracle_spearman(int n, const float *x, const float *y, double *ranks_x, double *ranks_y)
+{
+    if (n < 2) return NAN;
+    double *rx = (double *)malloc(sizeof(double) * (size_t)n * 2), *ry = rx + n;
+    if (!rx) return NAN;
+    for (int i = 0; i < n; ++i) {
+        long lx = 0, ex = 0, ly = 0, ey = 0;
+        for (int j = 0; j < n; ++j) {
+            lx += x[j] < x[i]; ex += x[j] == x[i];
+            ly += y[j] < y[i]; ey += y[j] == y[i];
+        }
+        rx[i] = (double)lx + ((double)ex + 1.0) / 2.0;   /* ranks lx + 1 .. lx + ex, averaged */
+        ry[i] = (double)ly + ((double)ey + 1.0) / 2.0;
+    }
+    const double m = ((double)n + 1.0) / 2.0;
+    double sxy = 0, sxx = 0, syy = 0;
+    for (int i = 0; i < n; ++i) {
+        sxy += (rx[i] - m) * (ry[i] - m);
+        sxx += (rx[i] - m) * (rx[i] - m);
+        syy += (ry[i] - m) * (ry[i] - m);
+    }
+    if (ranks_x) memcpy(ranks_x, rx, sizeof(double) * (size_t)n);
+    if (ranks_y) memcpy(ranks_y, ry, sizeof(double) * (size_t)n);
+    free(rx);
+    if (!(sxx > 0) || !(syy > 0)) return NAN;
+    return sxy / sqrt(sxx * syy);
 }

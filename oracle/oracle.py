@@ -55,6 +55,8 @@ def bind(lib):
     lib.oracle_policy.argtypes = [c_int, c_int, vp, vp, ctypes.c_float, c_int, vp, vp]
     lib.oracle_route_classes.restype = c_int
     lib.oracle_route_classes.argtypes = [c_int, c_int, c_int, c_int, c_int, vp, vp, vp, ctypes.c_float, vp, vp, vp]
+    lib.oracle_spearman.restype = c_dbl
+    lib.oracle_spearman.argtypes = [c_int, vp, vp, vp, vp]
     lib.oracle_phase_lens.restype = None
     lib.oracle_phase_lens.argtypes = [c_int, vp, vp, c_int, c_int, vp]
     lib.oracle_kv_append.restype = ctypes.c_uint
@@ -233,3 +235,14 @@ def phase_lens(step_lens, decisions=None, want: int = 1, t: int = -1):
     out = np.zeros(sl.shape[0], dtype=np.int32)
     _load().oracle_phase_lens(sl.shape[0], sl.ctypes.data, dp, int(want), int(t), out.ctypes.data)
     return out
+
+
+def spearman(x, y, return_ranks: bool = False):
+    """Spearman's rho of two fp32 samples (average ranks for ties); NaN if undefined."""
+    xa, ya = _f32(x), _f32(y)
+    assert xa.shape == ya.shape and xa.ndim == 1
+    n = xa.shape[0]
+    rx = np.zeros(n, dtype=np.float64)
+    ry = np.zeros(n, dtype=np.float64)
+    rho = float(_load().oracle_spearman(n, xa.ctypes.data, ya.ctypes.data, rx.ctypes.data, ry.ctypes.data))
+    return (rho, rx, ry) if return_ranks else rho

@@ -38,6 +38,8 @@ MUTATIONS = {
     "class level not normalised": ("sc += p[c] * (double)c / (double)(C - 1);", "sc += p[c] * (double)c;"),
     "ordinal cut sign": ("ge[k] = 1.0 / (1.0 + exp(-(acc - b[k])));", "ge[k] = 1.0 / (1.0 + exp(-(acc + b[k])));"),
     "append one slot late": ("const int pos = L + j;", "const int pos = L + j + 1;"),
+    "ties take the lowest rank": ("rx[i] = (double)lx + ((double)ex + 1.0) / 2.0;", "rx[i] = (double)lx + 1.0;"),
+    "ranks not centred": ("const double m = ((double)n + 1.0) / 2.0;", "const double m = 0.0;"),
     "append swaps K and V": ("memcpy((char *)k_pages + dst, (const char *)k_new + src, tok_bytes);",
                              "memcpy((char *)k_pages + dst, (const char *)v_new + src, tok_bytes);"),
 }
@@ -98,6 +100,10 @@ def _pins_pass() -> bool:
             return False
         p, _, _ = oracle.route_classes(oracle.HEAD_ORDINAL, hid, wo, [0.0, math.log(3.0), math.log(9.0)], 0.5)
         if not np.allclose(p[0], [0.75, 0.15, 0.1], atol=1e-12):
+            return False
+        if abs(oracle.spearman([1, 2, 2, 3], [1, 2, 3, 4]) - 3 / math.sqrt(10)) > 1e-12:
+            return False
+        if abs(oracle.spearman([1, 2, 3, 4, 5], [2, 1, 4, 3, 5]) - 0.8) > 1e-12:   # 1 - 6 * 4 / 120
             return False
         inp = wl.small_attn_case(1, 2, 1, 64, torch.float32, [20], [1], seed=4, extra_tokens=16)
         kn = torch.full((3, 1, 64), 7.0)

@@ -248,3 +248,27 @@ def test_phase_lens_partitions_the_batch():
     assert np.array_equal(by_token, esc)
     assert list(oracle.phase_lens([3, -4, 0], None, t=-1)) == [3, 0, 0]
     assert list(oracle.phase_lens([3, 1, 2], None, t=1)) == [1, 0, 1]
+
+
+# ---- Spearman ----------------------------------------------------------------------------------------
+
+def test_spearman_against_library_and_closed_forms():
+    from scipy.stats import rankdata, spearmanr
+    rng = np.random.default_rng(11)
+    for n, ties in ((2, False), (17, False), (200, False), (200, True), (1000, True)):
+        x = rng.normal(size=n).astype(np.float32)
+        y = (0.3 * x + rng.normal(size=n)).astype(np.float32)
+        if ties:
+            x, y = np.round(x * 2) / 2, np.round(y * 3) / 3
+        rho, rx, ry = oracle.spearman(x, y, return_ranks=True)
+        assert np.array_equal(rx, rankdata(x)) and np.array_equal(ry, rankdata(y))     # average ranks
+        assert abs(rho - spearmanr(x, y).statistic) < 1e-12
+        if not ties:      # the textbook form for distinct values: 1 - 6 sum d^2 / (n (n^2 - 1))
+            d = rankdata(x) - rankdata(y)
+            assert abs(rho - (1 - 6 * float((d * d).sum()) / (n * (n * n - 1)))) < 1e-12
+    # by hand: x = 1 2 2 3 -> ranks 1 2.5 2.5 4; y = 1 2 3 4: sums 4.5, 4.5, 5 -> rho = 3 / sqrt(10)
+    assert abs(oracle.spearman([1, 2, 2, 3], [1, 2, 3, 4]) - 3 / math.sqrt(10)) < 1e-15
+    x = rng.normal(size=50).astype(np.float32)
+    assert oracle.spearman(x, np.exp(x)) == 1.0 and oracle.spearman(x, -x ** 3) == -1.0    # monotone maps
+    assert abs(oracle.spearman(x, x[::-1].copy()) - oracle.spearman(x[::-1].copy(), x)) < 1e-15   # symmetric
+    assert math.isnan(oracle.spearman([1, 1, 1], [1, 2, 3])) and math.isnan(oracle.spearman([1], [2]))

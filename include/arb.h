@@ -307,6 +307,19 @@ arb_status arb_kv_append(arb_ctx *ctx, const arb_attn_params *params, int32_t to
                          int32_t update_lens, void *k_pages, void *v_pages, arb_stream_t stream);
 
 /*
+ * Spearman's rank correlation of two samples (Section 4.2, "Evaluation", and Tables 1-3 of the paper:
+ * the correlation between the router's predicted scores and the oracle advantage Delta).  Each value is
+ * replaced by its rank within its sample, equal values sharing the mean of the ranks they span, and
+ * rho is the Pearson correlation of the two rank variables.
+ *
+ *   x, y   fp32 [n], finite;  n <= 65536 (ranks are found by counting, n^2 comparisons).
+ *   rho    DEVICE pointer to one double (8-byte aligned): the result, NaN when n < 2 or a sample is
+ *          constant.  Sums are taken in fp64.
+ * Uses three accumulators in the ctx: one call at a time per ctx.
+ */
+arb_status arb_spearman(arb_ctx *ctx, int32_t n, const float *x, const float *y, double *rho, arb_stream_t stream);
+
+/*
  * Lengths of the next call of a phase of Algorithm 1, derived on the device so that the loop never reads
  * a length or a decision on the host: after the routing decision, accepted steps are absorbed by the
  * caches that did not generate them, and escalated steps are regenerated token by token by the target.

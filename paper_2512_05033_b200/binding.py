@@ -33,7 +33,7 @@ MAX_CLASSES = 16
 # every symbol include/arb.h declares
 EXPORTS = ("arb_create", "arb_destroy", "arb_attn_workspace_bytes", "arb_attn", "arb_attn_host",
            "arb_attn_decode_static",
-           "arb_route", "arb_rollback", "arb_policy", "arb_route_classes", "arb_kv_append", "arb_phase_lens",
+           "arb_route", "arb_rollback", "arb_policy", "arb_route_classes", "arb_kv_append", "arb_phase_lens", "arb_spearman",
            "arb_poll_status", "arb_launch_count", "arb_status_string")
 
 
@@ -62,6 +62,8 @@ lib.arb_route.restype = ctypes.c_int
 lib.arb_route.argtypes = [_vp, _i32, _i32, _i32, _vp, _vp, _f, _f, _vp, _vp, _vp]
 lib.arb_rollback.restype = ctypes.c_int
 lib.arb_rollback.argtypes = [_vp, _i32, _vp, _vp, _vp, _vp]
+lib.arb_spearman.restype = ctypes.c_int
+lib.arb_spearman.argtypes = [_vp, _i32, _vp, _vp, _vp, _vp]
 lib.arb_phase_lens.restype = ctypes.c_int
 lib.arb_phase_lens.argtypes = [_vp, _i32, _vp, _vp, _i32, _i32, _vp, _vp]
 lib.arb_policy.restype = ctypes.c_int
@@ -227,6 +229,16 @@ class Context:
                               _dev(step_lens, "step_lens", torch.int32), dp, _stream_ptr(stream))
         _check(st, "arb_rollback")
         return seq_lens
+
+    # -- arb_spearman -------------------------------------------------------------------------
+    def spearman(self, x, y, rho=None, stream=None):
+        """rho (device float64 [1]) = Spearman's rank correlation of two fp32 device vectors."""
+        if rho is None:
+            rho = torch.empty(1, dtype=torch.float64, device=x.device)
+        st = lib.arb_spearman(self._h, x.shape[0], _dev(x, "x", torch.float32), _dev(y, "y", torch.float32),
+                              _dev(rho, "rho", torch.float64), _stream_ptr(stream))
+        _check(st, "arb_spearman")
+        return rho
 
     # -- arb_phase_lens -----------------------------------------------------------------------
     def phase_lens(self, step_lens, decisions=None, want: int = 1, t: int = -1, out=None, stream=None):

@@ -67,6 +67,7 @@ arb_status arb_create(arb_ctx **out, int device, size_t workspace_bytes) {
     const size_t rot_ints = (size_t)kRotSets * kRotCounters + kRotSets + 4;
     ok = ok && cudaMalloc(&c->rot, sizeof(int) * rot_ints) == cudaSuccess;
     ok = ok && cudaMemset(c->rot, 0, sizeof(int) * rot_ints) == cudaSuccess;
+    ok = ok && cudaMalloc(&c->spearman_acc, 4 * sizeof(double)) == cudaSuccess;
     if (ok) {  // "everything before the first call has completed"
         const uint32_t done = c->decode_gen - 1;
         ok = cudaMemcpy(c->rot + (size_t)kRotSets * kRotCounters + kRotSets, &done, sizeof(done),
@@ -76,6 +77,7 @@ arb_status arb_create(arb_ctx **out, int device, size_t workspace_bytes) {
         cudaFree(c->workspace);
         cudaFree(c->counters);
         cudaFree(c->rot);
+        cudaFree(c->spearman_acc);
         delete c;
         cudaGetLastError();
         return ARB_ERR_CUDA;
@@ -92,6 +94,7 @@ arb_status arb_destroy(arb_ctx *ctx) {
     cudaFree(c->workspace);
     cudaFree(c->counters);
     cudaFree(c->rot);
+    cudaFree(c->spearman_acc);
     cudaFree(c->stage);
     delete c;
     return ARB_OK;
@@ -226,6 +229,14 @@ arb_status arb_rollback(arb_ctx *ctx, int32_t batch, int32_t *seq_lens, const in
     if (!seq_lens || !step_lens) return ARB_ERR_INVALID_ARG;
     return launch_rollback(reinterpret_cast<Ctx *>(ctx), batch, seq_lens, step_lens, decisions,
                            reinterpret_cast<cudaStream_t>(stream));
+}
+
+arb_status arb_spearman(arb_ctx *ctx, int32_t n, const float *x, const float *y, double *rho, arb_stream_t stream) {
+    if (ctx == nullptr || n < 0 || rho == nullptr) return ARB_ERR_INVALID_ARG;
+    if (n > 0 && (!x || !y)) return ARB_ERR_INVALID_ARG;
+    if (n > 65536) return ARB_ERR_UNSUPPORTED;
+    if ((reinterpret_cast<uintptr_t>(rho) & 7u) != 0) return ARB_ERR_INVALID_ARG;
+    return launch_spearman(reinterpret_cast<Ctx *>(ctx), n, x, y, rho, reinterpret_cast<cudaStream_t>(stream));
 }
 
 arb_status arb_phase_lens(arb_ctx *ctx, int32_t batch, const int32_t *step_lens, const uint8_t *decisions, int32_t want,

@@ -36,6 +36,7 @@ struct Ctx {
     int *rot = nullptr;
     uint32_t decode_gen = 1000;          // generation of the next tensor-core decode call
     bool last_decode_shared_set0 = false; // the CUDA-core decode kernel used set 0 since then
+    double *spearman_acc = nullptr;       // three fp64 accumulators of arb_spearman
 };
 
 constexpr int kRotSets = 4;
@@ -196,6 +197,7 @@ arb_status launch_decode_static(const arb_attn_params &p, const void *q, const v
                                 void *out, uint32_t *device_status, cudaStream_t stream);
 arb_status launch_phase_lens(Ctx *ctx, int batch, const int32_t *step_lens, const uint8_t *decisions, int want, int t,
                              int32_t *out, cudaStream_t stream);
+arb_status launch_spearman(Ctx *ctx, int n, const float *x, const float *y, double *rho, cudaStream_t stream);
 arb_status launch_policy(Ctx *ctx, int kind, int n_steps, const float *s_d, const float *s_t, float tau, int budget,
                          uint8_t *decisions, arb_policy_stats *stats, cudaStream_t stream);
 arb_status launch_route_classes(Ctx *ctx, int dtype, int mode, int n_steps, int hidden_dim, int n_classes,

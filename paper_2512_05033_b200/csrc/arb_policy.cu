@@ -16,6 +16,11 @@
 // C-way heads (Section 6.1, ablation): one warp per step computes the C logits (softmax head) or one
 // logit against C - 1 ordered cut points (ordinal head), the class probabilities, the expected class
 // level scaled to [0, 1] as the routing score, and the threshold decision (a tie accepts).
+//
+// Spearman's rho (the rank correlation the paper reports between router scores and the oracle advantage,
+// Section 4.2 "Evaluation" and Tables 1-3): ranks by counting -- rank_i = #{x_j < x_i} + (#{x_j = x_i} + 1) / 2,
+// ties sharing the mean of the ranks they span -- for both samples in one pass over shared-memory tiles,
+// then the three centred sums of the Pearson formula in fp64 and a one-thread kernel for the quotient.
 #include "arb_common.cuh"
 
 namespace arb {
@@ -94,6 +99,49 @@ policy_kernel(int kind, int n, const float *__restrict__ s_d, const float *__res
         add_stats(stats, (unsigned)a, (unsigned)w, live ? (double)(a ? st : sd) : 0.0,
                   a ? (double)st - (double)sd : 0.0);
     }
+}
+
+__global__ void __launch_bounds__(kPolicyThreads)
+spearman_rank_kernel(int n, const float *__restrict__ x, const float *__restrict__ y, double *__restrict__ acc) {
+    __shared__ float xs[kPolicyThreads], ys[kPolicyThreads];
+    __shared__ double red[3][kPolicyThreads / 32];
+    const int i = blockIdx.x * kPolicyThreads + threadIdx.x;
+    const bool live = i < n;
+    const float xi = live ? x[i] : 0.f, yi = live ? y[i] : 0.f;
+    int lx = 0, ex = 0, ly = 0, ey = 0;
+    for (int j0 = 0; j0 < n; j0 += kPolicyThreads) {
+        const int j = j0 + threadIdx.x;
+        __syncthreads();
+        xs[threadIdx.x] = j < n ? x[j] : 0.f;
+        ys[threadIdx.x] = j < n ? y[j] : 0.f;
+        __syncthreads();
+        const int m = min(kPolicyThreads, n - j0);
+        for (int k = 0; k < m; ++k) {
+            lx += xs[k] < xi; ex += xs[k] == xi;
+            ly += ys[k] < yi; ey += ys[k] == yi;
+        }
+    }
+    const double mean = ((double)n + 1.0) * 0.5;
+    const double dx = live ? (double)lx + ((double)ex + 1.0) * 0.5 - mean : 0.0;
+    const double dy = live ? (double)ly + ((double)ey + 1.0) * 0.5 - mean : 0.0;
+    double v[3] = {dx * dy, dx * dx, dy * dy};
+#pragma unroll
+    for (int q = 0; q < 3; ++q) {
+#pragma unroll
+        for (int off = 16; off >= 1; off >>= 1) v[q] += __shfl_xor_sync(0xffffffffu, v[q], off);
+        if ((threadIdx.x & 31) == 0) red[q][threadIdx.x >> 5] = v[q];
+    }
+    __syncthreads();
+    if (threadIdx.x < 3) {
+        double t = 0.0;
+        for (int w = 0; w < kPolicyThreads / 32; ++w) t += red[threadIdx.x][w];
+        atomicAdd(&acc[threadIdx.x], t);
+    }
+}
+
+__global__ void spearman_finish_kernel(int n, const double *__restrict__ acc, double *__restrict__ rho) {
+    const double sxy = acc[0], sxx = acc[1], syy = acc[2];
+    *rho = (n < 2 || !(sxx > 0.0) || !(syy > 0.0)) ? __longlong_as_double(0x7ff8000000000000ll) : sxy / sqrt(sxx * syy);
 }
 
 constexpr int kHeadWarps = 4;
@@ -188,6 +236,17 @@ arb_status launch_policy(Ctx *ctx, int kind, int n_steps, const float *s_d, cons
     if (stats != nullptr && cudaMemsetAsync(stats, 0, sizeof(arb_policy_stats), stream) != cudaSuccess) return ARB_ERR_CUDA;
     const int grid = (n_steps + kPolicyThreads - 1) / kPolicyThreads;
     policy_kernel<<<grid, kPolicyThreads, 0, stream>>>(kind, n_steps, s_d, s_t, tau, budget, decisions, stats);
+    ctx->launches++;
+    return cudaGetLastError() == cudaSuccess ? ARB_OK : ARB_ERR_CUDA;
+}
+
+arb_status launch_spearman(Ctx *ctx, int n, const float *x, const float *y, double *rho, cudaStream_t stream) {
+    if (cudaMemsetAsync(ctx->spearman_acc, 0, 3 * sizeof(double), stream) != cudaSuccess) return ARB_ERR_CUDA;
+    if (n > 0) {
+        spearman_rank_kernel<<<(n + kPolicyThreads - 1) / kPolicyThreads, kPolicyThreads, 0, stream>>>(n, x, y, ctx->spearman_acc);
+        ctx->launches++;
+    }
+    spearman_finish_kernel<<<1, 1, 0, stream>>>(n, ctx->spearman_acc, rho);
     ctx->launches++;
     return cudaGetLastError() == cudaSuccess ? ARB_OK : ARB_ERR_CUDA;
 }

@@ -182,3 +182,20 @@ def test_one_round_of_the_step_loop_matches_oracle():
     assert torch.equal(kp.cpu(), k2) and torch.equal(vp.cpu(), v2)
     H.assert_close(out1.double().cpu().numpy(), o1, BF, tight=3e-3)
     H.assert_close(out2.double().cpu().numpy(), o2, BF, tight=3e-3)
+
+
+@pytest.mark.parametrize("n,ties", [(2, False), (255, False), (256, True), (1000, True), (5000, False), (20000, True)])
+def test_spearman_matches_oracle(n, ties):
+    import math
+    c = H.ctx()
+    g = torch.Generator().manual_seed(n)
+    x = torch.randn(n, generator=g)
+    y = 0.2 * x + torch.randn(n, generator=g)
+    if ties:
+        x, y = torch.round(x * 4) / 4, torch.round(y * 3) / 3
+    ref = oracle.spearman(x, y)
+    got = float(c.spearman(x.cuda(), y.cuda()).item())
+    assert abs(got - ref) <= 1e-12, (got, ref)        # same ranks; fp64 sums in another order
+    const = float(c.spearman(torch.ones(n).cuda(), y.cuda()).item())
+    assert math.isnan(const) and math.isnan(oracle.spearman(torch.ones(n), y))
+    assert c.poll_status() == 0

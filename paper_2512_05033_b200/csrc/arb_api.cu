@@ -68,6 +68,8 @@ arb_status arb_create(arb_ctx **out, int device, size_t workspace_bytes) {
     ok = ok && cudaMalloc(&c->rot, sizeof(int) * rot_ints) == cudaSuccess;
     ok = ok && cudaMemset(c->rot, 0, sizeof(int) * rot_ints) == cudaSuccess;
     ok = ok && cudaMalloc(&c->spearman_acc, 4 * sizeof(double)) == cudaSuccess;
+    c->chunk_ws_bytes = 2 * c->workspace_bytes;   // partials of long step chunks that are split over their keys
+    ok = ok && cudaMalloc(&c->chunk_ws, c->chunk_ws_bytes) == cudaSuccess;
     if (ok) {  // "everything before the first call has completed"
         const uint32_t done = c->decode_gen - 1;
         ok = cudaMemcpy(c->rot + (size_t)kRotSets * kRotCounters + kRotSets, &done, sizeof(done),
@@ -78,6 +80,7 @@ arb_status arb_create(arb_ctx **out, int device, size_t workspace_bytes) {
         cudaFree(c->counters);
         cudaFree(c->rot);
         cudaFree(c->spearman_acc);
+        cudaFree(c->chunk_ws);
         delete c;
         cudaGetLastError();
         return ARB_ERR_CUDA;
@@ -95,6 +98,7 @@ arb_status arb_destroy(arb_ctx *ctx) {
     cudaFree(c->counters);
     cudaFree(c->rot);
     cudaFree(c->spearman_acc);
+    cudaFree(c->chunk_ws);
     cudaFree(c->stage);
     delete c;
     return ARB_OK;

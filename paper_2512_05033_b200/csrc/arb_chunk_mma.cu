@@ -50,6 +50,15 @@ constexpr float kRescaleThreshold = 8.0f;   // log2 units
 constexpr int kItemSlots = 8;               // work items announced ahead of their use
 constexpr int kPrefetchTiles = 4;            // K/V tiles asked into L2 ahead of the ring
 constexpr int kSortMaxBatch = 256;          // up to this batch size sequences are served longest first
+// Split-KV for long sequences: a sequence that sees more than kSplitMinTiles KV tiles has its key range
+// cut into parts of about kSplitPartTiles tiles; every (row tile pair, part) is a work item of its own
+// and leaves un-normalised partial results, which chunk_combine_kernel merges.  Without this one 64k-token
+// sequence in a batch keeps a single CTA busy long after all others have run dry.
+constexpr int kSplitMinTiles = 160;
+constexpr int kSplitPartTiles = 96;
+constexpr int kSplitMaxParts = 32;          // a warp's lanes cover the parts in the combine
+constexpr size_t kSlotFloats = (size_t)kBM * kD + 2 * kBM;   // one row tile's partial: O as [32 groups of 4 dims][128 rows][4],
+                                                             // so that the rows' 16-byte pieces lie side by side; then (max, sum) [128][2]
 
 struct MmaArgs {
     const char *q;
@@ -63,6 +72,8 @@ struct MmaArgs {
     int min_rows;  // sequences with q_len * group >= min_rows are handled here
     int *work_counter;  // [0] next work item, [1] set if a chunk sequence is left for the CUDA-core kernel;
                         // both zeroed on the stream before the launch
+    float *split_ws;    // partial results of split sequences, kSlotFloats per (item, row tile)
+    int split_cap;      // slots that fit there
     float scale_log2;
 };
 
@@ -85,7 +96,7 @@ struct Bars {
 constexpr size_t kSmemFixed = 1024 /*alignment*/ + 2 * kTileBytes /*Q of A, B*/ + 2 * kStages * kTileBytes /*K, V*/ +
                               sizeof(Bars);
 
-inline size_t mma_smem_bytes(int batch) { return kSmemFixed + sizeof(int) * (5 * (size_t)batch + 2); }
+inline size_t mma_smem_bytes(int batch) { return kSmemFixed + sizeof(int) * (7 * (size_t)batch + 2); }
 
 // ---- tcgen05 / TMA wrappers -------------------------------------------------------------------
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
@@ -220,37 +231,152 @@ __device__ __forceinline__ float max3(float a, float b, float c) {
     return r;
 }
 
-// A work item: up to two consecutive row tiles (A, B) of one (sequence, kv head).  They share every
-// K/V tile that is loaded; B may be missing (rows[1] == 0).
+// A work item: up to two consecutive row tiles (A, B) of one (sequence, kv head), over the KV tiles
+// [t0, t0 + ntiles) of the keys they see.  They share every K/V tile that is loaded; B may be missing
+// (rows[1] == 0).  `split`: the sequence's keys are cut into parts and this item leaves partials in
+// slots `slot` (tile A) and `slot + 1` (tile B).
 struct Item {
-    int b, kvh, n, L, rows_total, r_begin, rows[2], kv_len, ntiles, qrow0;
+    int b, kvh, n, L, rows_total, r_begin, rows[2], kv_len, t0, ntiles, qrow0, slot;
+    bool split;
 };
 
+// The tables every CTA (and the combine kernel) derives from the lengths, in shared memory.
+struct Plan {
+    int *pref;     // [B + 1] work items before the sequence in serving position r
+    int *row0;     // [B + 1] q rows before sequence b
+    int *sorted;   // [B] sequences in serving order (longest first)
+    int *pairs;    // [B] row tile pairs of sequence b (0: not served by this kernel)
+    int *key;      // [B] visible keys of sequence b (sort key)
+    int *parts;    // [B] parts the keys of the sequence in serving position r are cut into
+    int *sslot;    // [B] first partial slot of the sequence in serving position r
+};
+
+__device__ __forceinline__ Plan plan_arrays(int *base, int B) {
+    Plan pl;
+    pl.pref = base;
+    pl.row0 = pl.pref + B + 1;
+    pl.sorted = pl.row0 + B + 1;
+    pl.pairs = pl.sorted + B;
+    pl.key = pl.pairs + B;
+    pl.parts = pl.key + B;
+    pl.sslot = pl.parts + B;
+    return pl;
+}
+
+// Fills the plan; every thread of the block takes part.  small_flag (nullable): set to 1 by block 0 if a
+// chunk sequence is left for the CUDA-core kernel.
 template <int G>
-__device__ __forceinline__ bool get_item(int item, int total, const int *pref, const int *row0, const int *sorted,
-                                         int B, int Hkv, const MmaArgs &a, Item &it) {
+__device__ void make_plan(const MmaArgs &a, Plan pl, int tid, int nthreads, int *small_flag) {
+    const int B = a.batch, Hkv = a.Hkv, lane = tid & 31, warp = tid >> 5;
+    if (tid == 0) { pl.pref[0] = 0; pl.row0[0] = 0; }
+    for (int b = tid; b < B; b += nthreads) {
+        const int n = a.q_lens[b], L = a.seq_lens[b];
+        int pairs = 0;
+        if (n >= 2 && n * G >= a.min_rows && L >= n && L <= a.max_pages * kPage) pairs = (n * G + 2 * kBM - 1) / (2 * kBM);
+        if (small_flag != nullptr && blockIdx.x == 0 && n >= 2 && pairs == 0) atomicOr(small_flag, 1);  // small, or invalid lengths
+        pl.pairs[b] = pairs;
+        pl.key[b] = pairs > 0 ? L : -1;
+        pl.row0[b + 1] = n > 0 ? n : 0;
+    }
+    __syncthreads();
+    // serving order: longest first (items of a long sequence take longest), ties by index; large
+    // batches keep their own order
+    for (int b = tid; b < B; b += nthreads) {
+        int rank = b;
+        if (B <= kSortMaxBatch) {
+            rank = 0;
+            const int kb = pl.key[b];
+            for (int o = 0; o < B; ++o) rank += (pl.key[o] > kb) || (pl.key[o] == kb && o < b);
+        }
+        pl.sorted[rank] = b;
+    }
+    __syncthreads();
+    if (warp == 0) {
+        // in serving order: parts (granted while the partial slots last), partial slots and work items;
+        // and, in batch order, the q rows
+        int carry_p = 0, carry_r = 0, carry_s = 0;
+        for (int r0 = 0; r0 < B; r0 += 32) {
+            const int r = r0 + lane;
+            int want = 1, slots = 0, pairs = 0;
+            if (r < B) {
+                const int sb = pl.sorted[r];
+                pairs = pl.pairs[sb];
+                const int nt = pairs > 0 ? (pl.key[sb] + kBN - 1) / kBN : 0;
+                if (nt > kSplitMinTiles) {
+                    want = min((nt + kSplitPartTiles - 1) / kSplitPartTiles, kSplitMaxParts);
+                    slots = Hkv * pairs * want * 2;
+                }
+            }
+            int vs = slots;
+            int vr = r < B ? pl.row0[r + 1] : 0;
+#pragma unroll
+            for (int off = 1; off < 32; off <<= 1) {
+                const int ts = __shfl_up_sync(0xffffffffu, vs, off);
+                const int tr = __shfl_up_sync(0xffffffffu, vr, off);
+                if (lane >= off) { vs += ts; vr += tr; }
+            }
+            const bool granted = slots > 0 && vs + carry_s <= a.split_cap;
+            const int P = granted ? want : 1;
+            int vp = Hkv * pairs * P;
+#pragma unroll
+            for (int off = 1; off < 32; off <<= 1) {
+                const int tp = __shfl_up_sync(0xffffffffu, vp, off);
+                if (lane >= off) vp += tp;
+            }
+            if (r < B) {
+                pl.parts[r] = P;
+                pl.sslot[r] = vs + carry_s - slots;
+                pl.pref[r + 1] = vp + carry_p;
+                pl.row0[r + 1] = vr + carry_r;
+            }
+            carry_p += __shfl_sync(0xffffffffu, vp, 31);
+            carry_r += __shfl_sync(0xffffffffu, vr, 31);
+            carry_s += __shfl_sync(0xffffffffu, vs, 31);
+        }
+    }
+    __syncthreads();
+}
+
+// keys the row tile pair that starts at row r_begin sees, and the tiles of one part of the sequence
+template <int G>
+__device__ __forceinline__ int pair_kv_len(int L, int n, int rows_total, int r_begin) {
+    const int r_last = min(r_begin + 2 * kBM, rows_total) - 1;
+    return L - n + r_last / G + 1;
+}
+__device__ __forceinline__ int part_tiles(int L, int P) {
+    const int nt = (L + kBN - 1) / kBN;
+    return (nt + P - 1) / P;
+}
+
+template <int G>
+__device__ __forceinline__ bool get_item(int item, int total, const Plan &pl, int B, int Hkv, const MmaArgs &a, Item &it) {
     if (item >= total) return false;
     int lo = 0, hi = B;
     while (hi - lo > 1) {
         const int mid = (lo + hi) >> 1;
-        if (pref[mid] <= item) lo = mid; else hi = mid;
+        if (pl.pref[mid] <= item) lo = mid; else hi = mid;
     }
-    const int sb = sorted[lo];  // pref runs over the sequences in serving order
+    const int sb = pl.sorted[lo];  // pref runs over the sequences in serving order
     it.b = sb;
     it.n = a.q_lens[sb];
     it.L = a.seq_lens[sb];
     it.rows_total = it.n * G;
-    const int pairs = (it.rows_total + 2 * kBM - 1) / (2 * kBM);
-    const int r = item - pref[lo];
-    it.kvh = r / pairs;
-    const int pt = r - it.kvh * pairs;
+    const int pairs = pl.pairs[sb], P = pl.parts[lo];
+    const int r = item - pl.pref[lo];
+    it.kvh = r / (pairs * P);
+    const int rem = r - it.kvh * pairs * P;
+    const int pt = rem / P, part = rem - pt * P;
     it.r_begin = pt * 2 * kBM;
     it.rows[0] = min(kBM, it.rows_total - it.r_begin);
     it.rows[1] = max(0, min(kBM, it.rows_total - it.r_begin - kBM));
-    const int i_last = (it.r_begin + it.rows[0] + it.rows[1] - 1) / G;
-    it.kv_len = it.L - it.n + i_last + 1;   // keys the pair's last row sees
-    it.ntiles = (it.kv_len + kBN - 1) / kBN;
-    it.qrow0 = row0[sb];
+    it.kv_len = pair_kv_len<G>(it.L, it.n, it.rows_total, it.r_begin);   // keys the pair's last row sees
+    const int nt_pair = (it.kv_len + kBN - 1) / kBN;
+    const int T = part_tiles(it.L, P);
+    it.t0 = part * T;
+    it.ntiles = max(0, min(it.t0 + T, nt_pair) - it.t0);   // 0: nothing of this part is visible to the pair
+    it.split = P > 1;
+    it.slot = pl.sslot[lo] + ((it.kvh * pairs + pt) * P + part) * 2;
+    it.qrow0 = pl.row0[sb];
     return true;
 }
 
@@ -263,11 +389,7 @@ chunk_mma_kernel(const MmaArgs a, const __grid_constant__ CUtensorMap k_map, con
     char *k_s = base + 2 * kTileBytes;                 // [stage][2 halves][128 keys][128 B]
     char *v_s = k_s + kStages * kTileBytes;
     Bars *bars = reinterpret_cast<Bars *>(v_s + kStages * kTileBytes);
-    int *pref = reinterpret_cast<int *>(bars + 1);     // [B + 1] work items before sequence b
-    int *row0 = pref + a.batch + 1;                    // [B + 1] q rows before sequence b
-    int *sorted = row0 + a.batch + 1;                  // [B] sequences in serving order (longest first)
-    int *itm = sorted + a.batch;                       // [B] work items of sequence b
-    int *key = itm + a.batch;                          // [B] visible keys of sequence b (sort key)
+    const Plan pl = plan_arrays(reinterpret_cast<int *>(bars + 1), a.batch);
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int B = a.batch, Hkv = a.Hkv;
@@ -292,53 +414,9 @@ chunk_mma_kernel(const MmaArgs a, const __grid_constant__ CUtensorMap k_map, con
         }
         bars->abort = 0;
         mbar_fence_init();
-        pref[0] = 0;
-        row0[0] = 0;
     }
-    for (int b = tid; b < B; b += kThreads) {
-        const int n = a.q_lens[b], L = a.seq_lens[b];
-        int items = 0;
-        if (n >= 2 && n * G >= a.min_rows && L >= n && L <= a.max_pages * kPage)
-            items = Hkv * ((n * G + 2 * kBM - 1) / (2 * kBM));
-        if (blockIdx.x == 0 && n >= 2 && items == 0) atomicOr(a.work_counter + 1, 1);  // small, or invalid lengths
-        itm[b] = items;
-        key[b] = items > 0 ? L : -1;
-        row0[b + 1] = n > 0 ? n : 0;
-    }
-    __syncthreads();
-    // serving order: longest first (items of a long sequence take longest), ties by index; large
-    // batches keep their own order
-    for (int b = tid; b < B; b += kThreads) {
-        int rank = b;
-        if (B <= kSortMaxBatch) {
-            rank = 0;
-            const int kb = key[b];
-            for (int o = 0; o < B; ++o) rank += (key[o] > kb) || (key[o] == kb && o < b);
-        }
-        sorted[rank] = b;
-    }
-    __syncthreads();
-    for (int r = tid; r < B; r += kThreads) pref[r + 1] = itm[sorted[r]];
-    __syncthreads();
-    if (warp == 0) {
-        int carry_p = 0, carry_r = 0;
-        for (int b0 = 0; b0 < B; b0 += 32) {
-            const int b = b0 + lane;
-            int vp = b < B ? pref[b + 1] : 0;
-            int vr = b < B ? row0[b + 1] : 0;
-#pragma unroll
-            for (int off = 1; off < 32; off <<= 1) {
-                const int tp = __shfl_up_sync(0xffffffffu, vp, off);
-                const int tr = __shfl_up_sync(0xffffffffu, vr, off);
-                if (lane >= off) { vp += tp; vr += tr; }
-            }
-            if (b < B) { pref[b + 1] = vp + carry_p; row0[b + 1] = vr + carry_r; }
-            carry_p += __shfl_sync(0xffffffffu, vp, 31);
-            carry_r += __shfl_sync(0xffffffffu, vr, 31);
-        }
-    }
-    __syncthreads();
-    const int total = pref[B];
+    make_plan<G>(a, pl, tid, kThreads, a.work_counter + 1);
+    const int total = pl.pref[B];
     if ((int)blockIdx.x >= total) return;  // nothing for this CTA; no TMEM taken, no barrier pending
 
     if (warp == kMmaWarp) tmem_alloc(&bars->tmem_base, kTmemCols);
@@ -364,11 +442,12 @@ chunk_mma_kernel(const MmaArgs a, const __grid_constant__ CUtensorMap k_map, con
                 mbar_arrive(&bars->item_full[slot]);
             }
             item = __shfl_sync(0xffffffffu, item, 0);
-            if (!get_item<G>(item, total, pref, row0, sorted, B, Hkv, a, w)) break;
+            if (!get_item<G>(item, total, pl, B, Hkv, a, w)) break;
             // K and V tiles are asked into L2 kPrefetchTiles ahead of their load into the ring, so the
             // ring (two tiles deep) only has to cover the L2 latency, not the DRAM latency
-            auto prefetch_tile = [&](int jt) {
+            auto prefetch_tile = [&](int jt) {   // jt: tile of this item, 0-based
                 if (jt >= w.ntiles) return;
+                jt += w.t0;
                 const int np = min(kTilePages, (w.kv_len - jt * kBN + kPage - 1) / kPage);
                 const int pg = lane & 7;
                 if (lane < 16 && pg < np) {
@@ -382,11 +461,12 @@ chunk_mma_kernel(const MmaArgs a, const __grid_constant__ CUtensorMap k_map, con
             for (int jt = 0; jt < kPrefetchTiles; ++jt) prefetch_tile(jt);
             for (int j = 0; j < w.ntiles; ++j, ++it) {
                 const uint32_t s = it % kStages, par = (it / kStages) & 1u;
-                const int npages = min(kTilePages, (w.kv_len - j * kBN + kPage - 1) / kPage);
+                const int jg = w.t0 + j;   // tile of the sequence
+                const int npages = min(kTilePages, (w.kv_len - jg * kBN + kPage - 1) / kPage);
                 prefetch_tile(j + kPrefetchTiles);
                 int pid = 0;
                 if (lane < npages) {
-                    pid = a.block_table[(size_t)w.b * a.max_pages + j * kTilePages + lane];
+                    pid = a.block_table[(size_t)w.b * a.max_pages + jg * kTilePages + lane];
                     if ((unsigned)pid >= (unsigned)a.num_pages) {
                         atomicOr(a.status, (uint32_t)ARB_DEV_BAD_PAGE);
                         pid = 0;
@@ -429,15 +509,17 @@ chunk_mma_kernel(const MmaArgs a, const __grid_constant__ CUtensorMap k_map, con
         if (lane == 0) {
             constexpr uint32_t idesc_qk = instr_desc(false), idesc_pv = instr_desc(true);
             const uint32_t q_addr = smem_u32(q_s);
-            uint32_t it = 0, nitem = 0, itg[2] = {0u, 0u};  // KV tiles so far: all, per row tile
+            uint32_t it = 0, nitem = 0, nproc = 0, itg[2] = {0u, 0u};  // KV tiles so far: all, per row tile
             Item w;
             for (;; ++nitem) {
                 const uint32_t slot = nitem % kItemSlots, qpar = (nitem / kItemSlots) & 1u;
                 if (!mbar_wait(&bars->item_full[slot], qpar, abort, a.status)) break;
                 const int item = bars->item_id[slot];
                 mbar_arrive(&bars->item_empty[slot]);
-                if (!get_item<G>(item, total, pref, row0, sorted, B, Hkv, a, w)) break;
-                mbar_wait(&bars->q_full, nitem & 1u, abort, a.status);
+                if (!get_item<G>(item, total, pl, B, Hkv, a, w)) break;
+                if (w.ntiles == 0) continue;   // a part the pair sees nothing of: no role does anything for it
+                mbar_wait(&bars->q_full, nproc & 1u, abort, a.status);
+                ++nproc;
                 const bool has_b = w.rows[1] > 0;
                 // S of row tile g for KV tile `itx`: 8 steps of 16 dims, 4 per 64-dim half; K-major
                 // operands, SBO = 8 rows
@@ -507,7 +589,8 @@ chunk_mma_kernel(const MmaArgs a, const __grid_constant__ CUtensorMap k_map, con
             if (!mbar_wait(&bars->item_full[slot], qpar, abort, a.status)) break;
             const int item = bars->item_id[slot];
             mbar_arrive(&bars->item_empty[slot]);
-            if (!get_item<G>(item, total, pref, row0, sorted, B, Hkv, a, w)) break;
+            if (!get_item<G>(item, total, pl, B, Hkv, a, w)) break;
+            if (w.ntiles == 0) continue;   // a part the pair sees nothing of
             const int rows_here = w.rows[grp];
             const bool row_ok = tg < rows_here;
             const int r = min(w.r_begin + grp * kBM + tg, w.rows_total - 1);
@@ -532,7 +615,7 @@ chunk_mma_kernel(const MmaArgs a, const __grid_constant__ CUtensorMap k_map, con
             float m_used = -INFINITY, l_sum = 0.f;
             for (int j = 0; j < w.ntiles; ++j, ++it, ++itg) {
                 const uint32_t s = it % kStages, par = (it / kStages) & 1u;
-                const int key0 = j * kBN;
+                const int key0 = (w.t0 + j) * kBN;
                 const int nvis = lim - key0;  // columns < nvis are visible to this row (may be <= 0)
                 mbar_wait(&bars->s_full[grp], itg & 1u, abort, a.status);
                 tc_fence_after();
@@ -620,6 +703,25 @@ chunk_mma_kernel(const MmaArgs a, const __grid_constant__ CUtensorMap k_map, con
             // ---- epilogue: O / l, bf16, one 256-byte row per thread
             mbar_wait(&bars->o_full[grp], (itg - 1u) & 1u, abort, a.status);
             tc_fence_after();
+            if (w.split) {
+                // one part of a split sequence: leave the un-normalised O row and its (max, sum)
+                float *po = a.split_ws + (size_t)(w.slot + grp) * kSlotFloats;
+#pragma unroll 1
+                for (int c4 = 0; c4 < 4; ++c4) {
+                    uint32_t v[32];
+                    tmem_ld32(o_tmem + c4 * 32, v);
+                    tmem_wait_ld();
+                    if (row_ok) {
+#pragma unroll
+                        for (int qd = 0; qd < 8; ++qd)
+                            *reinterpret_cast<uint4 *>(po + ((size_t)(c4 * 8 + qd) * kBM + tg) * 4) =
+                                make_uint4(v[qd * 4], v[qd * 4 + 1], v[qd * 4 + 2], v[qd * 4 + 3]);
+                    }
+                }
+                if (row_ok) *reinterpret_cast<float2 *>(po + (size_t)kBM * kD + tg * 2) = make_float2(m_used, l_sum);
+                tc_fence_before();
+                continue;
+            }
             const float inv_l = 1.0f / l_sum;
             uint4 *dst = reinterpret_cast<uint4 *>(a.out + grow * 2);
 #pragma unroll 1
@@ -649,6 +751,87 @@ chunk_mma_kernel(const MmaArgs a, const __grid_constant__ CUtensorMap k_map, con
     if (warp == kMmaWarp) {
         tc_fence_after();
         tmem_dealloc(tmem, kTmemCols);
+    }
+}
+
+// ---- merge of the parts of split sequences -------------------------------------------------------------
+// Runs behind chunk_mma_kernel on the stream.  Every CTA rebuilds the plan, then takes jobs in turn: a job
+// is a quarter (32 dimensions) of one row tile of a split sequence, one thread per query row:
+//     m = max_p m_p,  w_p = 2^(m_p - m),  out = sum_p w_p O_p / sum_p w_p l_p.
+// Partials are laid out so that the threads of a warp (consecutive rows) read consecutive 16-byte pieces.
+constexpr int kCombineThreads = kBM;
+constexpr int kCombineDims = 32;    // dimensions of a row per job
+
+template <int G>
+__global__ void __launch_bounds__(kCombineThreads)
+chunk_combine_kernel(const MmaArgs a) {
+    extern __shared__ int plan_smem[];
+    const Plan pl = plan_arrays(plan_smem, a.batch);
+    const int tid = threadIdx.x;
+    const int B = a.batch, Hkv = a.Hkv;
+    make_plan<G>(a, pl, tid, kCombineThreads, nullptr);
+    constexpr int kQuarters = kD / kCombineDims;
+    int job = 0;
+    for (int r = 0; r < B; ++r) {
+        const int P = pl.parts[r];
+        if (P <= 1) continue;
+        const int sb = pl.sorted[r], pairs = pl.pairs[sb];
+        const int n = a.q_lens[sb], L = a.seq_lens[sb], rows_total = n * G;
+        const int T = part_tiles(L, P);
+        const int njobs = Hkv * pairs * 2 * kQuarters;
+        // the jobs of this sequence that fall to this CTA
+        int j = (int)blockIdx.x - job % (int)gridDim.x;
+        if (j < 0) j += (int)gridDim.x;
+        job += njobs;
+        for (; j < njobs; j += (int)gridDim.x) {
+            const int qd = j % kQuarters, jt = j / kQuarters;
+            const int g = jt & 1, pt = (jt >> 1) % pairs, kvh = (jt >> 1) / pairs;
+            const int r_begin = pt * 2 * kBM;
+            const int rows_here = max(0, min(kBM, rows_total - r_begin - g * kBM));
+            if (tid >= rows_here) continue;
+            const int nt_pair = (pair_kv_len<G>(L, n, rows_total, r_begin) + kBN - 1) / kBN;
+            const int nparts = min(P, (nt_pair + T - 1) / T);   // parts the pair sees something of
+            const float *slot0 = a.split_ws + (size_t)(pl.sslot[r] + ((kvh * pairs + pt) * P) * 2 + g) * kSlotFloats;
+            const size_t part_stride = 2 * kSlotFloats;
+            float m = -INFINITY;
+            for (int p = 0; p < nparts; ++p)
+                m = fmaxf(m, __ldcg(slot0 + p * part_stride + (size_t)kBM * kD + tid * 2));   // part 0 sees key 0: finite
+            float l = 0.f;
+            float4 acc[kCombineDims / 4];
+#pragma unroll
+            for (int c = 0; c < kCombineDims / 4; ++c) acc[c] = make_float4(0.f, 0.f, 0.f, 0.f);
+            for (int p = 0; p < nparts; ++p) {
+                const float *sp = slot0 + p * part_stride;
+                float4 o[kCombineDims / 4];
+#pragma unroll
+                for (int c = 0; c < kCombineDims / 4; ++c)
+                    o[c] = __ldcg(reinterpret_cast<const float4 *>(sp + ((size_t)(qd * (kCombineDims / 4) + c) * kBM + tid) * 4));
+                const float2 ml = __ldcg(reinterpret_cast<const float2 *>(sp + (size_t)kBM * kD + tid * 2));
+                const float w = fast_exp2(ml.x - m);
+                l = fmaf(w, ml.y, l);
+#pragma unroll
+                for (int c = 0; c < kCombineDims / 4; ++c) {
+                    acc[c].x = fmaf(w, o[c].x, acc[c].x);
+                    acc[c].y = fmaf(w, o[c].y, acc[c].y);
+                    acc[c].z = fmaf(w, o[c].z, acc[c].z);
+                    acc[c].w = fmaf(w, o[c].w, acc[c].w);
+                }
+            }
+            const int rr = r_begin + g * kBM + tid;
+            const int tok = rr / G, head = rr - tok * G;
+            const size_t grow = ((size_t)(pl.row0[sb] + tok) * a.Hq + kvh * G + head) * kD + (size_t)qd * kCombineDims;
+            const float inv = 1.0f / l;
+            uint4 *dst = reinterpret_cast<uint4 *>(a.out + grow * 2);
+#pragma unroll
+            for (int c = 0; c < kCombineDims / 8; ++c) {
+                uint4 o4;
+                o4.x = pack_bf16(acc[2 * c].x * inv, acc[2 * c].y * inv);
+                o4.y = pack_bf16(acc[2 * c].z * inv, acc[2 * c].w * inv);
+                o4.z = pack_bf16(acc[2 * c + 1].x * inv, acc[2 * c + 1].y * inv);
+                o4.w = pack_bf16(acc[2 * c + 1].z * inv, acc[2 * c + 1].w * inv);
+                dst[c] = o4;
+            }
+        }
     }
 }
 
@@ -698,7 +881,15 @@ arb_status launch_one(Ctx *ctx, const MmaArgs &a, const CUtensorMap &km, const C
     const int grid = max_items < ctx->num_sms ? max_items : ctx->num_sms;
     chunk_mma_kernel<G><<<grid, kThreads, smem, stream>>>(a, km, vm);
     ctx->launches++;
-    return cudaGetLastError() == cudaSuccess ? ARB_OK : ARB_ERR_CUDA;
+    if (cudaGetLastError() != cudaSuccess) return ARB_ERR_CUDA;
+    // the merge of split sequences, when the block table is long enough for a sequence to be split at all
+    if (a.split_cap > 0 && ((long long)a.max_pages * kPage + kBN - 1) / kBN > kSplitMinTiles) {
+        const size_t csmem = sizeof(int) * (7 * (size_t)a.batch + 2);
+        chunk_combine_kernel<G><<<4 * ctx->num_sms, kCombineThreads, csmem, stream>>>(a);
+        ctx->launches++;
+        if (cudaGetLastError() != cudaSuccess) return ARB_ERR_CUDA;
+    }
+    return ARB_OK;
 }
 
 }  // namespace
@@ -730,12 +921,16 @@ arb_status launch_chunk_mma(Ctx *ctx, const arb_attn_params &p, const void *q, c
     a.max_pages = p.max_pages_per_seq;
     a.min_rows = kChunkMmaMinRows;
     a.work_counter = ctx->rot + (size_t)kRotSets * kRotCounters + kRotSets + 1;
+    a.split_ws = ctx->chunk_ws;
+    a.split_cap = (int)(ctx->chunk_ws_bytes / (kSlotFloats * sizeof(float)));
+    if (((long long)p.max_pages_per_seq * kPage + kBN - 1) / kBN <= kSplitMinTiles) a.split_cap = 0;
     if (cudaMemsetAsync(a.work_counter, 0, 2 * sizeof(int), stream) != cudaSuccess) return ARB_ERR_CUDA;
     const float scale = p.softmax_scale > 0.f ? p.softmax_scale : 1.0f / sqrtf((float)p.head_dim);
     a.scale_log2 = scale * 1.4426950408889634f;
     const int g = p.num_q_heads / p.num_kv_heads;
     // upper bound of the work items from what the host knows: every row could sit in its own tile run
-    const long long bound = (long long)p.num_kv_heads * ((long long)p.total_q * g / kBM + p.batch);
+    long long bound = (long long)p.num_kv_heads * ((long long)p.total_q * g / kBM + p.batch);
+    if (a.split_cap > 0) bound *= kSplitMaxParts;   // every item of a split sequence comes once per part
     const int max_items = (int)(bound < 1 ? 1 : (bound > (1 << 30) ? (1 << 30) : bound));
     switch (g) {
         case 1: return launch_one<1>(ctx, a, km, vm, max_items, stream);

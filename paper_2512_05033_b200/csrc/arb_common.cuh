@@ -37,6 +37,8 @@ struct Ctx {
     uint32_t decode_gen = 1000;          // generation of the next tensor-core decode call
     bool last_decode_shared_set0 = false; // the CUDA-core decode kernel used set 0 since then
     double *spearman_acc = nullptr;       // three fp64 accumulators of arb_spearman
+    float *chunk_ws = nullptr;            // partial results of split long sequences (step-chunk attention)
+    size_t chunk_ws_bytes = 0;
 };
 
 constexpr int kRotSets = 4;

@@ -74,6 +74,40 @@ CHUNK_CASES = [
 ]
 
 
+SPLIT_CASES = [
+    # sequences that see more than 160 KV tiles are cut into parts over their keys and merged afterwards
+    (1, 32, 8, 128, BF, [26000], [100]),                     # g = 4: 400 rows = a full pair and a ragged one, 3 parts
+    (3, 28, 4, 128, BF, [21000, 900, 40000], [40, 64, 17]),  # g = 7: split and unsplit sequences in one call, 4 parts
+    (2, 16, 2, 128, BF, [20481, 65536], [16, 16]),           # g = 8: the first tile count that splits, and 64k keys
+]
+
+
+@pytest.mark.parametrize("case", SPLIT_CASES)
+def test_split_chunk_matches_oracle(case):
+    B, Hq, Hkv, D, dt, sl, ql = case
+    inp = wl.small_attn_case(B, Hq, Hkv, D, dt, sl, ql, seed=500 + Hq)
+    out, bits = H.gpu_attn(inp)
+    ref, st = H.oracle_attn(inp)
+    assert bits == 0 and st == 0
+    H.assert_close(out, ref, dt, tight=3e-3)
+
+
+def test_split_chunk_without_room_for_partials():
+    """A context too small to hold every partial serves the sequences it has no room for unsplit: same
+    results, only slower."""
+    from paper_2512_05033_b200 import binding
+    B, Hq, Hkv, D, dt, sl, ql = SPLIT_CASES[1]
+    inp = wl.small_attn_case(B, Hq, Hkv, D, dt, sl, ql, seed=500 + Hq)
+    ref, _ = H.oracle_attn(inp)
+    d = inp.to("cuda")
+    for ws in (2 << 20,):              # 4 MB for partials: room for the longest sequence's parts, not for the next one's
+        c = binding.Context(0, workspace_bytes=ws)
+        out = c.attn(d.q, d.k_pages, d.v_pages, d.block_table, d.seq_lens, d.q_lens, max(ql))
+        assert c.poll_status() == 0
+        H.assert_close(out.double().cpu().numpy(), ref, dt, tight=3e-3)
+        c.close()
+
+
 @pytest.mark.parametrize("case", CHUNK_CASES)
 def test_chunk_matches_oracle(case):
     B, Hq, Hkv, D, dt, sl, ql = case

@@ -33,6 +33,11 @@
  *  - oracle_spearman: the rank correlation the paper reports between the router's predictions and the
  *    oracle advantage (Section 4.2, "Evaluation"; Tables 1-3): Pearson correlation of the two rank
  *    variables, ties sharing the mean of the ranks they span.
+ *  - oracle_e4m3_decode / oracle_e4m3_encode: the 8-bit floating-point format E4M3 (1 sign, 4 exponent bits
+ *    with bias 7, 3 mantissa bits, no infinities, S.1111.111 = NaN, largest finite value 448) used for
+ *    the reduced-precision KV cache of a quantised draft model (Section 5.1 names 4-bit / 3-bit drafts; the
+ *    cache format is this library's choice).  Encoding rounds to nearest, ties to the even code, and
+ *    saturates at +-448.
  *  - oracle_phase_lens: which sequences take part in a phase of Algorithm 1 (accepted steps are
  *    absorbed by the target's cache, escalated ones are regenerated token by token by the target).
  *
@@ -445,4 +450,45 @@ double oracle_spearman(int n, const float *x, const float *y, double *ranks_x, d
     free(rx);
     if (!(sxx > 0) || !(syy > 0)) return NAN;
     return sxy / sqrt(sxx * syy);
+}
+
+
+/* E4M3 code -> value.  e = 0: subnormal m * 2^-9; otherwise (1 + m / 8) * 2^(e - 7); 0x7f / 0xff: NaN. */
+double oracle_e4m3_decode(uint8_t code)
+{
+    const int e = (code >> 3) & 15, m = code & 7;
+    const double sign = (code & 0x80) ? -1.0 : 1.0;
+    if (e == 15 && m == 7) return NAN;
+    if (e == 0) return sign * (double)m * ldexp(1.0, -9);
+    return sign * (1.0 + (double)m / 8.0) * ldexp(1.0, e - 7);
+}
+
+/* value -> nearest E4M3 code, by search over the 127 finite magnitudes: ties go to the even code, anything
+ * beyond the largest finite value saturates to it, NaN gives the NaN code. */
+uint8_t oracle_e4m3_encode(float x)
+{
+    if (x != x) return 0x7f;
+    const uint8_t sign = signbit(x) ? 0x80 : 0x00;
+    const double a = fabs((double)x);
+    int best = 0;
+    double best_err = a;   /* code 0 = 0.0 */
+    for (int c = 1; c <= 0x7e; ++c) {
+        const double err = fabs(oracle_e4m3_decode((uint8_t)c) - a);
+        if (err < best_err || (err == best_err && (c & 1) == 0)) { best = c; best_err = err; }
+    }
+    return (uint8_t)(sign | best);
+}
+
+/* codes[i] = encode(x[i] * inv_scale), the product taken in fp32 */
+void oracle_e4m3_encode_array(long n, const float *x, float inv_scale, uint8_t *codes)
+{
+    for (long i = 0; i < n; ++i) {
+        volatile float y = x[i] * inv_scale;
+        codes[i] = oracle_e4m3_encode(y);
+    }
+}
+
+void oracle_e4m3_decode_array(long n, const uint8_t *codes, float *x)
+{
+    for (long i = 0; i < n; ++i) x[i] = (float)oracle_e4m3_decode(codes[i]);
 }

@@ -55,6 +55,14 @@ def bind(lib):
     lib.oracle_policy.argtypes = [c_int, c_int, vp, vp, ctypes.c_float, c_int, vp, vp]
     lib.oracle_route_classes.restype = c_int
     lib.oracle_route_classes.argtypes = [c_int, c_int, c_int, c_int, c_int, vp, vp, vp, ctypes.c_float, vp, vp, vp]
+    lib.oracle_e4m3_decode.restype = c_dbl
+    lib.oracle_e4m3_decode.argtypes = [ctypes.c_uint8]
+    lib.oracle_e4m3_encode.restype = ctypes.c_uint8
+    lib.oracle_e4m3_encode.argtypes = [ctypes.c_float]
+    lib.oracle_e4m3_encode_array.restype = None
+    lib.oracle_e4m3_encode_array.argtypes = [c_long, vp, ctypes.c_float, vp]
+    lib.oracle_e4m3_decode_array.restype = None
+    lib.oracle_e4m3_decode_array.argtypes = [c_long, vp, vp]
     lib.oracle_spearman.restype = c_dbl
     lib.oracle_spearman.argtypes = [c_int, vp, vp, vp, vp]
     lib.oracle_phase_lens.restype = None
@@ -246,3 +254,44 @@ def spearman(x, y, return_ranks: bool = False):
     ry = np.zeros(n, dtype=np.float64)
     rho = float(_load().oracle_spearman(n, xa.ctypes.data, ya.ctypes.data, rx.ctypes.data, ry.ctypes.data))
     return (rho, rx, ry) if return_ranks else rho
+
+
+# ---- E4M3 (8-bit floating point) KV cache ---------------------------------------------------------------
+
+def e4m3_decode(codes):
+    """uint8 codes (numpy or torch) -> fp32 numpy array of the same shape (exact)."""
+    c = np.ascontiguousarray(codes.detach().cpu().numpy() if hasattr(codes, "detach") else np.asarray(codes), dtype=np.uint8)
+    out = np.zeros(c.shape, dtype=np.float32)
+    _load().oracle_e4m3_decode_array(c.size, c.ctypes.data, out.ctypes.data)
+    return out
+
+
+def e4m3_encode(x, inv_scale: float = 1.0):
+    """values -> uint8 codes of x * inv_scale (fp32 product; nearest, ties to even, saturating at 448)."""
+    a = _f32(x)
+    out = np.zeros(a.shape, dtype=np.uint8)
+    _load().oracle_e4m3_encode_array(a.size, a.ctypes.data, float(inv_scale), out.ctypes.data)
+    return out
+
+
+def kv_append_e4m3(k_new, v_new, block_table, seq_lens, new_lens, k_codes, v_codes, k_inv_scale: float,
+                   v_inv_scale: float, update_lens: bool = True):
+    """Quantising append: the new rows are encoded (x * inv_scale) and written into copies of the uint8 pools."""
+    import torch
+
+    kc = torch.from_numpy(e4m3_encode(k_new, k_inv_scale))
+    vc = torch.from_numpy(e4m3_encode(v_new, v_inv_scale))
+    return kv_append(kc, vc, block_table, seq_lens, new_lens, k_codes, v_codes, update_lens)
+
+
+def attn_e4m3(q, k_codes, v_codes, k_scale: float, v_scale: float, block_table, seq_lens, q_lens, scale: float = 0.0):
+    """Attention over an E4M3 cache: keys are k_scale * decode(code), values v_scale * decode(code)."""
+    import math
+    import torch
+
+    D = q.shape[-1]
+    sm = scale if scale > 0 else 1.0 / math.sqrt(D)
+    kf = torch.from_numpy(e4m3_decode(k_codes))
+    vf = torch.from_numpy(e4m3_decode(v_codes))
+    out, st = attn(q.float(), kf, vf, block_table, seq_lens, q_lens, sm * float(k_scale))
+    return out * float(v_scale), st

@@ -40,6 +40,8 @@ MUTATIONS = {
     "append one slot late": ("const int pos = L + j;", "const int pos = L + j + 1;"),
     "ties take the lowest rank": ("rx[i] = (double)lx + ((double)ex + 1.0) / 2.0;", "rx[i] = (double)lx + 1.0;"),
     "ranks not centred": ("const double m = ((double)n + 1.0) / 2.0;", "const double m = 0.0;"),
+    "E4M3 bias off by one": ("ldexp(1.0, e - 7);", "ldexp(1.0, e - 8);"),
+    "E4M3 ties away from even": ("(err == best_err && (c & 1) == 0)", "(err == best_err && (c & 1) == 1)"),
     "append swaps K and V": ("memcpy((char *)k_pages + dst, (const char *)k_new + src, tok_bytes);",
                              "memcpy((char *)k_pages + dst, (const char *)v_new + src, tok_bytes);"),
 }
@@ -104,6 +106,10 @@ def _pins_pass() -> bool:
         if abs(oracle.spearman([1, 2, 2, 3], [1, 2, 3, 4]) - 3 / math.sqrt(10)) > 1e-12:
             return False
         if abs(oracle.spearman([1, 2, 3, 4, 5], [2, 1, 4, 3, 5]) - 0.8) > 1e-12:   # 1 - 6 * 4 / 120
+            return False
+        if list(oracle.e4m3_decode(np.uint8([0x38, 0x7e, 0x01]))) != [1.0, 448.0, 2.0 ** -9]:
+            return False
+        if list(oracle.e4m3_encode(np.float32([1.0625, 1.1875, 500.0]))) != [0x38, 0x3a, 0x7e]:
             return False
         inp = wl.small_attn_case(1, 2, 1, 64, torch.float32, [20], [1], seed=4, extra_tokens=16)
         kn = torch.full((3, 1, 64), 7.0)

@@ -272,3 +272,49 @@ def test_spearman_against_library_and_closed_forms():
     assert oracle.spearman(x, np.exp(x)) == 1.0 and oracle.spearman(x, -x ** 3) == -1.0    # monotone maps
     assert abs(oracle.spearman(x, x[::-1].copy()) - oracle.spearman(x[::-1].copy(), x)) < 1e-15   # symmetric
     assert math.isnan(oracle.spearman([1, 1, 1], [1, 2, 3])) and math.isnan(oracle.spearman([1], [2]))
+
+
+# ---- E4M3 ----------------------------------------------------------------------------------------------
+
+def test_e4m3_against_the_library_type_and_the_format():
+    codes = np.arange(256, dtype=np.uint8)
+    ours = oracle.e4m3_decode(codes)
+    lib = torch.from_numpy(codes).view(torch.float8_e4m3fn).float().numpy()
+    assert np.array_equal(np.isnan(ours), np.isnan(lib)) and np.array_equal(ours[~np.isnan(ours)], lib[~np.isnan(lib)])
+    # format facts: largest finite 448, smallest subnormal 2^-9, smallest normal 2^-6, no infinities
+    assert ours[0x7e] == 448.0 and ours[0x01] == 2.0 ** -9 and ours[0x08] == 2.0 ** -6 and np.isnan(ours[0x7f])
+    assert not np.isinf(ours).any() and ours[0x80] == 0.0 and np.signbit(ours[0x80])
+    finite = codes[~np.isnan(ours)]
+    assert np.array_equal(oracle.e4m3_encode(ours[finite]), finite)                 # round trip, -0 included
+    # nearest with ties to even, against the library's conversion inside the finite range
+    rng = np.random.default_rng(8)
+    x = np.concatenate([rng.normal(0, 1, 4000), rng.normal(0, 60, 2000), rng.uniform(-2.0 ** -6, 2.0 ** -6, 1000),
+                        [1.0625, 1.1875, 2.0 ** -10, 3 * 2.0 ** -10, 464.0 - 1e-3, -447.9]]).astype(np.float32)
+    x = x[np.abs(x) < 464.0]
+    lib_codes = torch.from_numpy(x).to(torch.float8_e4m3fn).view(torch.uint8).numpy()
+    assert np.array_equal(oracle.e4m3_encode(x), lib_codes)
+    # saturation (this library's choice; the library type gives NaN there): by definition
+    assert list(oracle.e4m3_encode(np.float32([464.0, 1e9, -500.0, np.inf]))) == [0x7e, 0x7e, 0xfe, 0x7e]
+    assert oracle.e4m3_encode(np.float32([3.0]), inv_scale=0.5)[0] == 0x3c           # 1.5 = (1 + 4/8) * 2^0
+
+
+def test_e4m3_cache_attention_and_quantising_append():
+    inp = wl.small_attn_case(2, 8, 2, 64, torch.bfloat16, [70, 33], [1, 1], seed=61, extra_tokens=32)
+    ks, vs = 0.02, 0.03
+    kc = torch.from_numpy(oracle.e4m3_encode(inp.k_pages, 1 / ks))
+    vc = torch.from_numpy(oracle.e4m3_encode(inp.v_pages, 1 / vs))
+    out, st = oracle.attn_e4m3(inp.q, kc, vc, ks, vs, inp.block_table, inp.seq_lens, inp.q_lens)
+    # the same thing spelled out with the library type: dequantise, then the bf16-cache oracle path on fp32 pools
+    kf = kc.view(torch.float8_e4m3fn).float() * ks
+    vf = vc.view(torch.float8_e4m3fn).float() * vs
+    ref, _ = oracle.attn(inp.q.float(), kf, vf, inp.block_table, inp.seq_lens, inp.q_lens)
+    assert st == 0 and np.allclose(out, ref, rtol=0, atol=1e-6)
+    full, _ = oracle.attn(inp.q, inp.k_pages, inp.v_pages, inp.block_table, inp.seq_lens, inp.q_lens)
+    assert np.abs(out - full).max() < 0.15                                           # and it is a fair copy of the cache
+    new = torch.tensor([3, 20], dtype=torch.int32)
+    g = torch.Generator().manual_seed(3)
+    kn, vn = torch.randn(23, 2, 64, generator=g).bfloat16(), torch.randn(23, 2, 64, generator=g).bfloat16()
+    kc2, vc2, sl, st = oracle.kv_append_e4m3(kn, vn, inp.block_table, inp.seq_lens, new, kc, vc, 1 / ks, 1 / vs)
+    page, slot = int(inp.block_table[1, 33 // 16]), 33 % 16
+    want = torch.from_numpy((kn[3].float() / 1).numpy() * np.float32(1 / ks)).to(torch.float8_e4m3fn).view(torch.uint8)
+    assert st == 0 and list(sl) == [73, 53] and torch.equal(kc2[page, :, slot, :], want)

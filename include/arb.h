@@ -307,6 +307,25 @@ arb_status arb_kv_append(arb_ctx *ctx, const arb_attn_params *params, int32_t to
                          int32_t update_lens, void *k_pages, void *v_pages, arb_stream_t stream);
 
 /*
+ * Quantising KV append: as arb_kv_append, but the pools hold E4M3 codes, one byte per element (1 sign bit,
+ * 4 exponent bits with bias 7, 3 mantissa bits, no infinities, largest finite value 448) -- the
+ * reduced-precision cache of a quantised draft model (Section 5.1 of the paper runs 4-bit and 3-bit drafts;
+ * the cache format is this library's choice, the paper names none).
+ *
+ *   params        dtype is the type of k_new / v_new (fp32 or bf16); the other fields as for arb_kv_append.
+ *   k_inv_scale,
+ *   v_inv_scale   > 0.  code = e4m3(x * inv_scale): the product in fp32, the conversion to the nearest code,
+ *                 ties to the even code, saturating at +-448.  The reader multiplies by 1 / inv_scale.
+ *   k_codes,
+ *   v_codes       uint8 [num_pages, Hkv, P, D].
+ * Everything else (placement, length update, refusals and status bits) as arb_kv_append.
+ */
+arb_status arb_kv_append_e4m3(arb_ctx *ctx, const arb_attn_params *params, int32_t total_new, const void *k_new,
+                              const void *v_new, float k_inv_scale, float v_inv_scale, const int32_t *block_table,
+                              int32_t *seq_lens, const int32_t *new_lens, int32_t update_lens, uint8_t *k_codes,
+                              uint8_t *v_codes, arb_stream_t stream);
+
+/*
  * Spearman's rank correlation of two samples (Section 4.2, "Evaluation", and Tables 1-3 of the paper:
  * the correlation between the router's predicted scores and the oracle advantage Delta).  Each value is
  * replaced by its rank within its sample, equal values sharing the mean of the ranks they span, and

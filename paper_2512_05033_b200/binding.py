@@ -33,7 +33,7 @@ MAX_CLASSES = 16
 # every symbol include/arb.h declares
 EXPORTS = ("arb_create", "arb_destroy", "arb_attn_workspace_bytes", "arb_attn", "arb_attn_host",
            "arb_attn_decode_static",
-           "arb_route", "arb_rollback", "arb_policy", "arb_route_classes", "arb_kv_append", "arb_phase_lens", "arb_spearman",
+           "arb_route", "arb_rollback", "arb_policy", "arb_route_classes", "arb_kv_append", "arb_kv_append_e4m3", "arb_phase_lens", "arb_spearman",
            "arb_poll_status", "arb_launch_count", "arb_status_string")
 
 
@@ -62,6 +62,8 @@ lib.arb_route.restype = ctypes.c_int
 lib.arb_route.argtypes = [_vp, _i32, _i32, _i32, _vp, _vp, _f, _f, _vp, _vp, _vp]
 lib.arb_rollback.restype = ctypes.c_int
 lib.arb_rollback.argtypes = [_vp, _i32, _vp, _vp, _vp, _vp]
+lib.arb_kv_append_e4m3.restype = ctypes.c_int
+lib.arb_kv_append_e4m3.argtypes = [_vp, ctypes.POINTER(AttnParams), _i32, _vp, _vp, _f, _f, _vp, _vp, _vp, _i32, _vp, _vp, _vp]
 lib.arb_spearman.restype = ctypes.c_int
 lib.arb_spearman.argtypes = [_vp, _i32, _vp, _vp, _vp, _vp]
 lib.arb_phase_lens.restype = ctypes.c_int
@@ -228,6 +230,22 @@ class Context:
         st = lib.arb_rollback(self._h, seq_lens.shape[0], _dev(seq_lens, "seq_lens", torch.int32),
                               _dev(step_lens, "step_lens", torch.int32), dp, _stream_ptr(stream))
         _check(st, "arb_rollback")
+        return seq_lens
+
+    # -- arb_kv_append_e4m3 -------------------------------------------------------------------
+    def kv_append_e4m3(self, k_new, v_new, k_inv_scale: float, v_inv_scale: float, block_table, seq_lens, new_lens,
+                       k_codes, v_codes, update_lens: bool = True, stream=None):
+        """In place: the new rows are quantised to E4M3 (x * inv_scale) and written behind each sequence's tokens."""
+        num_pages, Hkv, P, D = k_codes.shape
+        B, max_pages = block_table.shape
+        p = attn_params(_dtype_code(k_new), B, Hkv, Hkv, D, num_pages, max_pages, 0, 0, 0.0, P, 0)
+        st = lib.arb_kv_append_e4m3(self._h, ctypes.byref(p), k_new.shape[0], _dev(k_new, "k_new"),
+                                    _dev(v_new, "v_new", k_new.dtype), float(k_inv_scale), float(v_inv_scale),
+                                    _dev(block_table, "block_table", torch.int32), _dev(seq_lens, "seq_lens", torch.int32),
+                                    _dev(new_lens, "new_lens", torch.int32), 1 if update_lens else 0,
+                                    _dev(k_codes, "k_codes", torch.uint8), _dev(v_codes, "v_codes", torch.uint8),
+                                    _stream_ptr(stream))
+        _check(st, "arb_kv_append_e4m3")
         return seq_lens
 
     # -- arb_spearman -------------------------------------------------------------------------

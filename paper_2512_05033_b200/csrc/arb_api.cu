@@ -296,6 +296,26 @@ arb_status arb_kv_append(arb_ctx *ctx, const arb_attn_params *params, int32_t to
                             new_lens, update_lens, k_pages, v_pages, reinterpret_cast<cudaStream_t>(stream));
 }
 
+arb_status arb_kv_append_e4m3(arb_ctx *ctx, const arb_attn_params *params, int32_t total_new, const void *k_new,
+                              const void *v_new, float k_inv_scale, float v_inv_scale, const int32_t *block_table,
+                              int32_t *seq_lens, const int32_t *new_lens, int32_t update_lens, uint8_t *k_codes,
+                              uint8_t *v_codes, arb_stream_t stream) {
+    if (ctx == nullptr || params == nullptr || total_new < 0) return ARB_ERR_INVALID_ARG;
+    if (params->batch < 1 || params->num_kv_heads < 1 || params->num_pages < 1 || params->max_pages_per_seq < 1)
+        return ARB_ERR_INVALID_ARG;
+    if (params->dtype != ARB_F32 && params->dtype != ARB_BF16) return ARB_ERR_UNSUPPORTED;
+    if (params->head_dim != 64 && params->head_dim != 128) return ARB_ERR_UNSUPPORTED;
+    if (params->page_size != kPage || params->batch > kMaxBatch) return ARB_ERR_UNSUPPORTED;
+    if (!(k_inv_scale > 0.f) || !(v_inv_scale > 0.f)) return ARB_ERR_INVALID_ARG;
+    if (!block_table || !seq_lens || !new_lens || !k_codes || !v_codes) return ARB_ERR_INVALID_ARG;
+    if (total_new == 0) return ARB_OK;
+    if (!k_new || !v_new) return ARB_ERR_INVALID_ARG;
+    if (!aligned16(k_new) || !aligned16(v_new) || !aligned16(k_codes) || !aligned16(v_codes)) return ARB_ERR_INVALID_ARG;
+    return launch_kv_append_e4m3(reinterpret_cast<Ctx *>(ctx), *params, total_new, k_new, v_new, k_inv_scale, v_inv_scale,
+                                 block_table, seq_lens, new_lens, update_lens, k_codes, v_codes,
+                                 reinterpret_cast<cudaStream_t>(stream));
+}
+
 arb_status arb_poll_status(arb_ctx *ctx, arb_stream_t stream, uint32_t *bits) {
     if (ctx == nullptr) return ARB_ERR_INVALID_ARG;
     Ctx *c = reinterpret_cast<Ctx *>(ctx);

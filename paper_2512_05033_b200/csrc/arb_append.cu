@@ -11,6 +11,11 @@
 // block table, or that would land on a page outside the pool, leave that sequence untouched and set a
 // status bit.  Lengths are advanced by a second, one-CTA kernel, after every CTA of the first has read
 // them.
+//
+// The quantising form writes an E4M3 cache (one byte per element: 1 sign, 4 exponent bits with bias 7, 3
+// mantissa bits, largest finite value 448): code = e4m3(x * inv_scale), the product in fp32, the conversion
+// to nearest with ties to even and saturation (cvt.rn.satfinite.e4m3x2.f32).  Same plan, same checks; a
+// thread turns one 16-byte piece of a source row into 8 (bf16 source) or 4 (fp32 source) bytes.
 #include "arb_common.cuh"
 
 namespace arb {
@@ -98,6 +103,85 @@ kv_append_kernel(const AppendArgs a) {
     }
 }
 
+// two values -> two E4M3 codes; lo lands in the low byte
+__device__ __forceinline__ uint32_t e4m3x2(float lo, float hi) {
+    uint16_t r;
+    asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(r) : "f"(hi), "f"(lo));
+    return r;
+}
+
+template <typename T>
+__global__ void __launch_bounds__(kAppendThreads)
+kv_append_e4m3_kernel(const AppendArgs a, float k_inv_scale, float v_inv_scale) {
+    constexpr int EPL = Elt<T>::kPerVec;   // source elements per 16-byte piece = code bytes written per thread
+    extern __shared__ int asm_[];
+    int *pref = asm_;
+    int *okay = pref + a.batch + 1;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int B = a.batch;
+    if (tid == 0) pref[0] = 0;
+    for (int b = tid; b < B; b += kAppendThreads) {
+        const uint32_t bad = append_check(a, b);
+        if (bad && blockIdx.x == 0) atomicOr(a.status, bad);
+        okay[b] = bad == 0;
+        const int n = a.new_lens[b];
+        pref[b + 1] = n > 0 ? n : 0;
+    }
+    __syncthreads();
+    if (warp == 0) {
+        int carry = 0;
+        for (int b0 = 0; b0 < B; b0 += 32) {
+            const int b = b0 + lane;
+            int v = b < B ? pref[b + 1] : 0;
+#pragma unroll
+            for (int off = 1; off < 32; off <<= 1) {
+                const int t = __shfl_up_sync(0xffffffffu, v, off);
+                if (lane >= off) v += t;
+            }
+            if (b < B) pref[b + 1] = v + carry;
+            carry += __shfl_sync(0xffffffffu, v, 31);
+        }
+    }
+    __syncthreads();
+    const int total = min(pref[B], a.total_new);
+    const int vecs = a.row_bytes / 16;             // 16-byte pieces of a source row
+    const int D = vecs * EPL;                      // = bytes of a row of codes
+    const int rows_per_pass = kAppendThreads / vecs;
+    const int sub = tid / vecs, vec = tid - sub * vecs;
+    const long long nrows = (long long)total * a.Hkv;
+    for (long long r = (long long)blockIdx.x * rows_per_pass + sub; r < nrows; r += (long long)gridDim.x * rows_per_pass) {
+        const int tok = (int)(r / a.Hkv), h = (int)(r - (long long)tok * a.Hkv);
+        int lo = 0, hi = B;
+        while (hi - lo > 1) {
+            const int mid = (lo + hi) >> 1;
+            if (pref[mid] <= tok) lo = mid; else hi = mid;
+        }
+        if (!okay[lo]) continue;
+        const int pos = a.seq_lens[lo] + (tok - pref[lo]);
+        const int page = a.block_table[(size_t)lo * a.max_pages + pos / kPage];
+        const size_t dst = (((size_t)page * a.Hkv + h) * kPage + (pos % kPage)) * D + (size_t)vec * EPL;
+        const size_t src = (size_t)r * a.row_bytes + (size_t)vec * 16;
+        float kf[EPL], vf[EPL];
+        Elt<T>::unpack(__ldg(reinterpret_cast<const uint4 *>(a.k_new + src)), kf);
+        Elt<T>::unpack(__ldg(reinterpret_cast<const uint4 *>(a.v_new + src)), vf);
+        uint32_t kc[EPL / 4], vc[EPL / 4];
+#pragma unroll
+        for (int w = 0; w < EPL / 4; ++w) {
+            kc[w] = e4m3x2(kf[4 * w] * k_inv_scale, kf[4 * w + 1] * k_inv_scale) |
+                    (e4m3x2(kf[4 * w + 2] * k_inv_scale, kf[4 * w + 3] * k_inv_scale) << 16);
+            vc[w] = e4m3x2(vf[4 * w] * v_inv_scale, vf[4 * w + 1] * v_inv_scale) |
+                    (e4m3x2(vf[4 * w + 2] * v_inv_scale, vf[4 * w + 3] * v_inv_scale) << 16);
+        }
+        if (EPL == 8) {
+            *reinterpret_cast<uint2 *>(a.k_pages + dst) = make_uint2(kc[0], kc[EPL / 4 - 1]);
+            *reinterpret_cast<uint2 *>(a.v_pages + dst) = make_uint2(vc[0], vc[EPL / 4 - 1]);
+        } else {
+            *reinterpret_cast<uint32_t *>(a.k_pages + dst) = kc[0];
+            *reinterpret_cast<uint32_t *>(a.v_pages + dst) = vc[0];
+        }
+    }
+}
+
 __global__ void __launch_bounds__(kAppendThreads)
 advance_lens_kernel(const AppendArgs a) {
     for (int b = threadIdx.x; b < a.batch; b += kAppendThreads) {
@@ -133,6 +217,45 @@ arb_status launch_kv_append(Ctx *ctx, const arb_attn_params &p, int total_new, c
     const int grid = (int)(want < 1 ? 1 : (want > cap ? cap : want));
     const size_t smem = sizeof(int) * (2 * (size_t)p.batch + 1);
     kv_append_kernel<<<grid, kAppendThreads, smem, stream>>>(a);
+    ctx->launches++;
+    if (cudaGetLastError() != cudaSuccess) return ARB_ERR_CUDA;
+    if (update_lens) {
+        advance_lens_kernel<<<1, kAppendThreads, 0, stream>>>(a);
+        ctx->launches++;
+        if (cudaGetLastError() != cudaSuccess) return ARB_ERR_CUDA;
+    }
+    return ARB_OK;
+}
+
+arb_status launch_kv_append_e4m3(Ctx *ctx, const arb_attn_params &p, int total_new, const void *k_new,
+                                 const void *v_new, float k_inv_scale, float v_inv_scale, const int32_t *block_table,
+                                 int32_t *seq_lens, const int32_t *new_lens, int update_lens, void *k_codes,
+                                 void *v_codes, cudaStream_t stream) {
+    AppendArgs a;
+    a.k_new = static_cast<const char *>(k_new);
+    a.v_new = static_cast<const char *>(v_new);
+    a.k_pages = static_cast<char *>(k_codes);
+    a.v_pages = static_cast<char *>(v_codes);
+    a.block_table = block_table;
+    a.seq_lens = seq_lens;
+    a.new_lens = new_lens;
+    a.status = ctx->status;
+    a.batch = p.batch;
+    a.Hkv = p.num_kv_heads;
+    a.num_pages = p.num_pages;
+    a.max_pages = p.max_pages_per_seq;
+    a.row_bytes = p.head_dim * (p.dtype == ARB_BF16 ? 2 : 4);   // of the source rows
+    a.total_new = total_new;
+    const int rows_per_pass = kAppendThreads / (a.row_bytes / 16);
+    const long long nrows = (long long)total_new * p.num_kv_heads;
+    long long want = (nrows + rows_per_pass - 1) / rows_per_pass;
+    const long long cap = (long long)ctx->num_sms * 4;
+    const int grid = (int)(want < 1 ? 1 : (want > cap ? cap : want));
+    const size_t smem = sizeof(int) * (2 * (size_t)p.batch + 1);
+    if (p.dtype == ARB_BF16)
+        kv_append_e4m3_kernel<__nv_bfloat16><<<grid, kAppendThreads, smem, stream>>>(a, k_inv_scale, v_inv_scale);
+    else
+        kv_append_e4m3_kernel<float><<<grid, kAppendThreads, smem, stream>>>(a, k_inv_scale, v_inv_scale);
     ctx->launches++;
     if (cudaGetLastError() != cudaSuccess) return ARB_ERR_CUDA;
     if (update_lens) {

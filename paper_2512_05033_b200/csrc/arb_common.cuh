@@ -208,6 +208,10 @@ arb_status launch_route_classes(Ctx *ctx, int dtype, int mode, int n_steps, int 
 arb_status launch_kv_append(Ctx *ctx, const arb_attn_params &p, int total_new, const void *k_new, const void *v_new,
                             const int32_t *block_table, int32_t *seq_lens, const int32_t *new_lens, int update_lens,
                             void *k_pages, void *v_pages, cudaStream_t stream);
+arb_status launch_kv_append_e4m3(Ctx *ctx, const arb_attn_params &p, int total_new, const void *k_new,
+                                 const void *v_new, float k_inv_scale, float v_inv_scale, const int32_t *block_table,
+                                 int32_t *seq_lens, const int32_t *new_lens, int update_lens, void *k_codes,
+                                 void *v_codes, cudaStream_t stream);
 size_t decode_workspace_bytes(const arb_attn_params &p, int num_sms);
 int decode_grid(int num_sms);
 

@@ -9,7 +9,7 @@ ROOT = Path(__file__).resolve().parent.parent
 def _declared_symbols():
     text = (ROOT / "include" / "arb.h").read_text()
     text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
-    return sorted(set(re.findall(r"\b(arb_[a-z_]+)\s*\(", text)))
+    return sorted(set(re.findall(r"\b(arb_[a-z0-9_]+)\s*\(", text)))
 
 
 def test_library_exports_every_declared_symbol():

@@ -199,3 +199,25 @@ def test_spearman_matches_oracle(n, ties):
     const = float(c.spearman(torch.ones(n).cuda(), y.cuda()).item())
     assert math.isnan(const) and math.isnan(oracle.spearman(torch.ones(n), y))
     assert c.poll_status() == 0
+
+
+@pytest.mark.parametrize("dtype,D", [(BF, 128), (F32, 128), (BF, 64), (F32, 64)])
+def test_quantising_append_matches_oracle(dtype, D):
+    c = H.ctx()
+    B, Hkv = 4, 2
+    sl, nl = [100, 15, 16, 0], [33, 1, 17, 40]
+    inp = wl.small_attn_case(B, Hkv, Hkv, D, dtype, sl, [1] * B, seed=640 + D, extra_tokens=64)
+    g = torch.Generator().manual_seed(19)
+    # values across the whole range of the format: subnormal codes, ties, saturation
+    k_new = (torch.randn(sum(nl), Hkv, D, generator=g) * torch.logspace(-4, 2.5, sum(nl)).view(-1, 1, 1)).to(dtype)
+    v_new = torch.randn(sum(nl), Hkv, D, generator=g).to(dtype)
+    k_new[0, 0, :8] = torch.tensor([1.0625, 1.1875, 500.0, -1e6, 2.0 ** -10, 3 * 2.0 ** -10, 0.0, -0.0]).to(dtype)
+    kc = torch.randint(0, 127, inp.k_pages.shape, generator=g, dtype=torch.uint8)
+    vc = torch.randint(0, 127, inp.k_pages.shape, generator=g, dtype=torch.uint8)
+    seq, new = torch.tensor(sl, dtype=torch.int32), torch.tensor(nl, dtype=torch.int32)
+    dk, dv, dseq = kc.cuda(), vc.cuda(), seq.cuda()
+    c.kv_append_e4m3(k_new.cuda(), v_new.cuda(), 1.0, 1 / 0.03, inp.block_table.cuda(), dseq, new.cuda(), dk, dv)
+    k_ref, v_ref, sl_ref, st = oracle.kv_append_e4m3(k_new, v_new, inp.block_table, seq, new, kc, vc, 1.0, 1 / 0.03)
+    assert st == 0 and c.poll_status() == 0
+    assert torch.equal(dk.cpu(), k_ref) and torch.equal(dv.cpu(), v_ref)          # codes: bit-exact
+    assert np.array_equal(dseq.cpu().numpy(), sl_ref)

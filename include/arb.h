@@ -307,6 +307,26 @@ arb_status arb_kv_append(arb_ctx *ctx, const arb_attn_params *params, int32_t to
                          int32_t update_lens, void *k_pages, void *v_pages, arb_stream_t stream);
 
 /*
+ * Decode attention (every q_len 1 or 0) over an E4M3 KV cache: keys are k_scale * code, values v_scale * code,
+ * one byte per element -- half the bytes per token of the bf16 cache, for the token-by-token steps of a
+ * quantised draft model (Section 3.1: z_i ~ q(z_i | x, z_<i); Section 5.1 runs 4-bit and 3-bit drafts; the
+ * cache format is this library's choice).  q and out are bf16; head_dim 128; g <= 8.
+ *
+ *   params     as for arb_attn, dtype ARB_BF16 (the type of q and out), max_q_len 1.  ARB_ATTN_OVERLAP_PREVIOUS
+ *              has the meaning it has for arb_attn.
+ *   k_codes,
+ *   v_codes    uint8 [num_pages, Hkv, P, D], written by arb_kv_append_e4m3 with inv_scale = 1 / scale.
+ *   k_scale,
+ *   v_scale    > 0, host scalars.
+ * The codes widen to f16 exactly; products run on the tensor cores in f16 with fp32 accumulation and the
+ * softmax weights are rounded to f16.  Against an oracle that reads the same codes the result meets the
+ * tolerance of the bf16 path; what quantisation itself costs is a property of the format, not of this call.
+ */
+arb_status arb_attn_decode_e4m3(arb_ctx *ctx, const arb_attn_params *params, const void *q, const uint8_t *k_codes,
+                                const uint8_t *v_codes, float k_scale, float v_scale, const int32_t *block_table,
+                                const int32_t *seq_lens, const int32_t *q_lens, void *out, arb_stream_t stream);
+
+/*
  * Quantising KV append: as arb_kv_append, but the pools hold E4M3 codes, one byte per element (1 sign bit,
  * 4 exponent bits with bias 7, 3 mantissa bits, no infinities, largest finite value 448) -- the
  * reduced-precision cache of a quantised draft model (Section 5.1 of the paper runs 4-bit and 3-bit drafts;

@@ -482,7 +482,8 @@ uint8_t oracle_e4m3_encode(float x)
 /* codes[i] = encode(x[i] * inv_scale), the product taken in fp32 */
 void oracle_e4m3_encode_array(long n, const float *x, float inv_scale, uint8_t *codes)
 {
-    for (long i = 0; i < n; ++i) {
+#pragma omp parallel for schedule(static)
+    for (long i = 0; i < n; ++i) {   /* independent elements */
         volatile float y = x[i] * inv_scale;
         codes[i] = oracle_e4m3_encode(y);
     }

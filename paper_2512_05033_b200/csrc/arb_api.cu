@@ -296,6 +296,24 @@ arb_status arb_kv_append(arb_ctx *ctx, const arb_attn_params *params, int32_t to
                             new_lens, update_lens, k_pages, v_pages, reinterpret_cast<cudaStream_t>(stream));
 }
 
+arb_status arb_attn_decode_e4m3(arb_ctx *ctx, const arb_attn_params *params, const void *q, const uint8_t *k_codes,
+                                const uint8_t *v_codes, float k_scale, float v_scale, const int32_t *block_table,
+                                const int32_t *seq_lens, const int32_t *q_lens, void *out, arb_stream_t stream) {
+    if (ctx == nullptr) return ARB_ERR_INVALID_ARG;
+    arb_status st = check_params(params);
+    if (st != ARB_OK) return st;
+    if (params->dtype != ARB_BF16 || params->head_dim != 128) return ARB_ERR_UNSUPPORTED;
+    if (params->max_q_len != 1 || params->total_q < 1 || params->total_q > params->batch) return ARB_ERR_INVALID_ARG;
+    if (params->flags & ARB_ATTN_NO_TENSOR_CORES) return ARB_ERR_UNSUPPORTED;
+    if (!(k_scale > 0.f) || !(v_scale > 0.f)) return ARB_ERR_INVALID_ARG;
+    if (!q || !out || !k_codes || !v_codes || !block_table || !seq_lens || !q_lens) return ARB_ERR_INVALID_ARG;
+    if (!aligned16(q) || !aligned16(out) || !aligned16(k_codes) || !aligned16(v_codes)) return ARB_ERR_INVALID_ARG;
+    Ctx *c = reinterpret_cast<Ctx *>(ctx);
+    if (decode_workspace_bytes(*params, c->num_sms) > c->workspace_bytes) return ARB_ERR_WORKSPACE;
+    return launch_decode_e4m3(c, *params, q, k_codes, v_codes, k_scale, v_scale, block_table, seq_lens, q_lens, out,
+                              reinterpret_cast<cudaStream_t>(stream));
+}
+
 arb_status arb_kv_append_e4m3(arb_ctx *ctx, const arb_attn_params *params, int32_t total_new, const void *k_new,
                               const void *v_new, float k_inv_scale, float v_inv_scale, const int32_t *block_table,
                               int32_t *seq_lens, const int32_t *new_lens, int32_t update_lens, uint8_t *k_codes,

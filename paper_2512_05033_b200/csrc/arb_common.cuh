@@ -212,6 +212,9 @@ arb_status launch_kv_append_e4m3(Ctx *ctx, const arb_attn_params &p, int total_n
                                  const void *v_new, float k_inv_scale, float v_inv_scale, const int32_t *block_table,
                                  int32_t *seq_lens, const int32_t *new_lens, int update_lens, void *k_codes,
                                  void *v_codes, cudaStream_t stream);
+arb_status launch_decode_e4m3(Ctx *ctx, const arb_attn_params &p, const void *q, const void *k_pages,
+                              const void *v_pages, float k_scale, float v_scale, const int32_t *block_table,
+                              const int32_t *seq_lens, const int32_t *q_lens, void *out, cudaStream_t stream);
 size_t decode_workspace_bytes(const arb_attn_params &p, int num_sms);
 int decode_grid(int num_sms);
 

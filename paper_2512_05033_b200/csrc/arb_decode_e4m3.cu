@@ -1,0 +1,932 @@
+// Split-KV decode attention (q_len = 1) over an E4M3 KV cache (one byte per element), head_dim 128, bf16
+// queries and outputs: the reduced-precision cache of a quantised draft model.  Half the bytes of the bf16
+// cache per token, which is the only way past the bf16 cache's HBM roofline.
+//
+// The kernel is the tensor-core decode kernel (flat page list cut into equal ranges per CTA, producer warp
+// and TMA ring, one page per consumer warp turn with its own online softmax, partials to a rotating
+// workspace set, a small programmatic-dependent combine kernel behind) with these differences:
+//   - a (page, kv head) tile is 16 rows x 128 bytes = 2 KB, one TMA box (128-byte swizzle); the ring has
+//     32 stages, so the bytes in flight per CTA stay the same;
+//   - the codes are widened to f16, which holds every E4M3 value exactly (cvt.rn.f16x2.e4m3x2), and the
+//     products run as f16 MMAs (m16n8k16, fp32 accumulate); q is converted bf16 -> f16 once per segment, P
+//     is rounded to f16 (11 significant bits) and summed after rounding;
+//   - ldmatrix moves 16-bit units, i.e. pairs of codes.  For q.K a thread receives four consecutive
+//     dimensions of one key per 8 x 16-byte matrix; they serve as the B fragment of a k-slice whose sixteen
+//     "k" positions are the matrix's sixteen dimensions in the order 4t, 4t+1 | 4t+2, 4t+3 (t = lane mod 4),
+//     and q's A fragment is loaded in the same order (a dot product does not care).  For P.V the transposed
+//     load gives a thread the codes (key 2t, dims d, d+1 | key 2t+1, dims d, d+1); one byte permute sorts
+//     them into the B fragments of two n-tiles, the even and the odd dimensions of a 16-dimension group, so
+//     a thread ends up owning four consecutive output dimensions per group;
+//   - the key scale is folded into the softmax scale, the value scale into the segment result.
+#include <cuda.h>  // CUtensorMap and its enums only; the encoder is looked up at run time
+
+#include "arb_common.cuh"
+
+namespace arb {
+
+namespace {
+
+constexpr int kD = 128;
+constexpr int kConsWarps = 4;
+constexpr int kConsThreads = kConsWarps * 32;
+constexpr int kThreads = kConsThreads + 32;
+constexpr int kGroup = 1;       // pages per consumer work group: with 16 stages every warp has two groups in flight
+constexpr int kStages = 32;     // ring stages of one 2 KB tile each
+constexpr int kBatch = 16;      // producer lanes issuing side by side
+constexpr int kTileBytes = kPage * kD;      // one TMA box: 16 rows x 128 codes
+constexpr int kRingBytes = kStages * kTileBytes;
+constexpr int kMinChunk = 4;
+constexpr int kCtasPerSm = 2;
+constexpr int kParked = 2;      // segment results parked in shared memory before they are written
+constexpr int kSmallCallPages = 64;   // up to this many pages per SM a call runs one CTA per SM
+static_assert(kStages % (kConsWarps * 2 * kGroup) == 0, "a ring stage must always belong to the same warp");
+static_assert(kBatch <= kStages, "two producer lanes of one turn must never wait on the same stage: the later one "
+                                 "would be two phases ahead of the barrier and a parity wait cannot tell");
+
+struct Args {
+    const char *q;
+    const int32_t *block_table;
+    const int32_t *seq_lens;
+    const int32_t *q_lens;
+    char *out;
+    float *part_o;    // [slots][G][D]
+    float *part_ml;   // [slots][GP][2]
+    uint32_t *status;
+    int batch, Hq, Hkv, num_pages, max_pages;
+    int small_ctas;   // CTAs a small call spreads over
+    float scale_log2;   // softmax scale * key scale * log2(e)
+    float v_scale;      // value scale
+    // workspace rotation (see launch_decode_e4m3): this call's generation number, the number of
+    // workspace sets, the generation of the newest completed call
+    uint32_t gen;
+    int sets;
+    int force_wait;
+    unsigned *done_gen;
+};
+
+struct Tail {
+    uint64_t full[kStages];
+    uint64_t empty[kStages];
+    int abort;
+    int early;            // the workspace set is free: partials may be written before the predecessor is done
+};
+
+struct Parked {  // host-side view of what a parked segment needs besides its record
+    int bk, nparts, c_first;
+    size_t out_base;
+};
+
+template <int G>
+struct Cfg {
+    static constexpr int GP = (G + 3) / 4 * 4;
+    static constexpr int REC = G * kD + 2 * GP;            // [m[GP] | l[GP] | o[G][D]]
+    static constexpr int OSM_BYTES = kConsWarps * REC * 4;
+    static constexpr int PARK_BYTES = kParked * REC * 4;
+};
+
+template <int G>
+size_t smem_bytes(int batch) {
+    using C = Cfg<G>;
+    return 1024 + kRingBytes + C::OSM_BYTES + C::PARK_BYTES + sizeof(Tail) + sizeof(int) * (3 * (size_t)batch + 2);
+}
+
+struct Segment {
+    int b, kvh, pg0, pg1, L, bk, nparts, c_first;
+};
+
+// The cut of the flat (sequence, kv head, page) list into per-CTA ranges: both kernels of a call must
+// agree on it.  Small calls use the first `small_ctas` CTAs of the grid -- one per SM, or one per
+// two SMs for a call that runs back to back with its neighbours (see launch_decode_e4m3) -- and
+// large ones the whole grid.
+__device__ __forceinline__ int plan_chunk(int total, int grid, int small_ctas) {
+    const int one_per_sm = min(grid, small_ctas);
+    const int active = total <= one_per_sm * kSmallCallPages ? one_per_sm : grid;
+    const int chunk = (total + active - 1) / active;
+    return chunk < kMinChunk ? kMinChunk : chunk;
+}
+
+__device__ __forceinline__ bool next_segment(int &cur, int r1, const int *pref, const int *slen, int B, int Hkv,
+                                             int chunk, Segment &s) {
+    if (cur >= r1) return false;
+    int lo = 0, hi = B;
+    while (hi - lo > 1) {
+        const int mid = (lo + hi) >> 1;
+        if (pref[mid] <= cur) lo = mid; else hi = mid;
+    }
+    const int b = lo;
+    const int pages = (pref[b + 1] - pref[b]) / Hkv;
+    const int r = cur - pref[b];
+    const int kvh = r / pages;
+    const int pg0 = r - kvh * pages;
+    const int s0 = pref[b] + kvh * pages;
+    const int s1 = s0 + pages;
+    const int end = s1 < r1 ? s1 : r1;
+    s.b = b;
+    s.kvh = kvh;
+    s.pg0 = pg0;
+    s.pg1 = pg0 + (end - cur);
+    s.L = slen[b];
+    s.bk = b * Hkv + kvh;
+    s.c_first = s0 / chunk;
+    s.nparts = (s1 - 1) / chunk - s.c_first + 1;
+    cur = end;
+    return true;
+}
+
+__device__ __forceinline__ void let_successor_start() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void wait_for_predecessor() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
+__device__ __forceinline__ void tma_box_load(void *dst_smem, const CUtensorMap *map, int x, int y, uint64_t *bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+        ::"r"(smem_u32(dst_smem)), "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(smem_u32(bar))
+        : "memory");
+}
+
+// four 8x8 bf16 blocks; lanes 8i..8i+7 give the row addresses of block i
+__device__ __forceinline__ void ldmatrix_x4(uint32_t addr, uint32_t (&r)[4]) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0, %1, %2, %3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
+                 : "r"(addr));
+}
+__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t addr, uint32_t (&r)[4]) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0, %1, %2, %3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
+                 : "r"(addr));
+}
+// D(16x8, fp32) += A(16x16, f16, row) * B(16x8, f16, col)
+__device__ __forceinline__ void mma_16816(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+    asm volatile(
+        "mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, "
+        "{%0, %1, %2, %3};"
+        : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+        : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+    uint32_t r;
+    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+    return r;
+}
+__device__ __forceinline__ uint32_t pack_f16(float lo, float hi) {
+    uint32_t r;
+    asm("cvt.rn.f16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+    return r;
+}
+__device__ __forceinline__ float2 unpack_f16(uint32_t v) {
+    float lo, hi;
+    asm("{\n\t.reg .b16 l, h;\n\tmov.b32 {l, h}, %2;\n\tcvt.f32.f16 %0, l;\n\tcvt.f32.f16 %1, h;\n\t}" : "=f"(lo), "=f"(hi) : "r"(v));
+    return make_float2(lo, hi);
+}
+// two E4M3 codes (low 16 bits of v) -> f16x2, exact; the low byte lands in the low half
+__device__ __forceinline__ uint32_t e4m3x2_to_f16x2(uint32_t v) {
+    uint32_t r;
+    asm("{\n\t.reg .b16 c;\n\tcvt.u16.u32 c, %1;\n\tcvt.rn.f16x2.e4m3x2 %0, c;\n\t}" : "=r"(r) : "r"(v));
+    return r;
+}
+__device__ __forceinline__ uint32_t byte_perm(uint32_t v, uint32_t sel) {
+    uint32_t r;
+    asm("prmt.b32 %0, %1, %1, %2;" : "=r"(r) : "r"(v), "r"(sel));
+    return r;
+}
+
+// byte offset of 16-byte chunk `c` (0..7 across the 128-byte row of codes) of row `r` inside a swizzled tile
+__device__ __forceinline__ uint32_t tile_off(int r, int c) {
+    return (uint32_t)(r * 128 + ((c ^ (r & 7)) << 4));
+}
+
+template <int G>
+__global__ void __launch_bounds__(kThreads, kCtasPerSm)
+decode_e4m3_kernel(const Args a, const __grid_constant__ CUtensorMap k_map, const __grid_constant__ CUtensorMap v_map) {
+    using C = Cfg<G>;
+    constexpr int GP = C::GP, REC = C::REC;
+    static_assert(G >= 1 && G <= 8, "query heads of a group occupy rows 0..7 of the 16-row tile");
+
+    extern __shared__ char smem_raw[];
+    char *base = reinterpret_cast<char *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    char *ring = base;
+    float *osm = reinterpret_cast<float *>(base + kRingBytes);
+    float *park = reinterpret_cast<float *>(base + kRingBytes + C::OSM_BYTES);
+    Tail *tail = reinterpret_cast<Tail *>(base + kRingBytes + C::OSM_BYTES + C::PARK_BYTES);
+    int *pref = reinterpret_cast<int *>(tail + 1);
+    int *row0 = pref + a.batch + 1;
+    int *slen = row0 + a.batch + 1;
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int B = a.batch, Hkv = a.Hkv;
+
+    // Until wait_for_predecessor() only inputs are read; every write to out, the workspace or the
+    // arrival counters comes after it (see the CUDA-core decode kernel for the ordering argument).
+    let_successor_start();
+
+    if (tid == kConsThreads) {  // the producer warp's first lane: descriptors on their way before the first copy needs them
+        asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&k_map)) : "memory");
+        asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&v_map)) : "memory");
+    }
+    if (tid == 0) {
+        for (int s = 0; s < kStages; ++s) {
+            mbar_init(&tail->full[s], 1);
+            mbar_init(&tail->empty[s], 1);
+        }
+        tail->abort = 0;
+        mbar_fence_init();
+        pref[0] = 0;
+        row0[0] = 0;
+    }
+    for (int b = tid; b < B; b += kThreads) {
+        const int n = a.q_lens[b], L = a.seq_lens[b];
+        int pages = 0;
+        if (n == 1) {
+            if (L >= 1 && L <= a.max_pages * kPage) {
+                pages = (L + kPage - 1) / kPage;
+            } else if (blockIdx.x == 0) {
+                wait_for_predecessor();
+                atomicOr(a.status, (uint32_t)ARB_DEV_BAD_SEQ_LEN);
+                int row = 0;
+                for (int i = 0; i < b; ++i) row += max(a.q_lens[i], 0);
+                __nv_bfloat16 *o = reinterpret_cast<__nv_bfloat16 *>(a.out) + (size_t)row * a.Hq * kD;
+                for (int i = 0; i < a.Hq * kD; ++i) o[i] = __float2bfloat16_rn(0.f);
+            }
+        }
+        pref[b + 1] = pages * Hkv;
+        row0[b + 1] = n > 0 ? n : 0;
+        slen[b] = L;
+    }
+    __syncthreads();
+    if (warp == 0) {
+        int carry_p = 0, carry_r = 0;
+        for (int b0 = 0; b0 < B; b0 += 32) {
+            const int b = b0 + lane;
+            int vp = b < B ? pref[b + 1] : 0;
+            int vr = b < B ? row0[b + 1] : 0;
+#pragma unroll
+            for (int off = 1; off < 32; off <<= 1) {
+                const int tp = __shfl_up_sync(0xffffffffu, vp, off);
+                const int tr = __shfl_up_sync(0xffffffffu, vr, off);
+                if (lane >= off) { vp += tp; vr += tr; }
+            }
+            if (b < B) { pref[b + 1] = vp + carry_p; row0[b + 1] = vr + carry_r; }
+            carry_p += __shfl_sync(0xffffffffu, vp, 31);
+            carry_r += __shfl_sync(0xffffffffu, vr, 31);
+        }
+    }
+    __syncthreads();
+
+    // Small calls use the first small_ctas CTAs of the grid (see plan_chunk); the other CTAs leave at
+    // once and their places are free for the next call, which -- launched as a programmatic
+    // dependent -- then streams its KV while this call is still computing.  Large calls use every
+    // CTA: two per SM keep more bytes in flight.
+    const int total = pref[B];
+    const int chunk = plan_chunk(total, (int)gridDim.x, a.small_ctas);
+    const long long r0l = (long long)blockIdx.x * chunk;
+    if (r0l >= total) {
+        // (CTA 0 only gets here when the call has no decode rows.)  One thread of CTA 0 always waits
+        // for the previous kernel, so that calls complete in stream order.
+        if (blockIdx.x == 0 && tid == 0) wait_for_predecessor();
+        return;
+    }
+    const int r0 = (int)r0l;
+    const int r1 = min(total, r0 + chunk);
+    volatile int *abort = &tail->abort;
+
+    if (warp == kConsWarps) {
+        // ================================ producer warp ==========================================
+        uint32_t c = 0;
+        int cur = r0;
+        Segment s;
+        while (next_segment(cur, r1, pref, slen, B, Hkv, chunk, s)) {
+            for (int sp0 = s.pg0; sp0 < s.pg1; sp0 += 32) {
+                const int np = min(32, s.pg1 - sp0);
+                int pid = 0;
+                if (lane < np) {
+                    pid = a.block_table[(size_t)s.b * a.max_pages + sp0 + lane];
+                    if ((unsigned)pid >= (unsigned)a.num_pages) {
+                        atomicOr(a.status, (uint32_t)ARB_DEV_BAD_PAGE);
+                        pid = 0;
+                    }
+                }
+                const int full_tiles = (np / kGroup) * 2 * kGroup;
+                const int rem = np % kGroup;
+                const int ntiles = 2 * np;
+#pragma unroll 1
+                for (int i0 = 0; i0 < ntiles; i0 += kBatch) {
+                    const int i = i0 + lane;
+                    int page, is_v;
+                    if (i < full_tiles) {
+                        const int g = i / (2 * kGroup), r = i - g * 2 * kGroup;
+                        is_v = r / kGroup;
+                        page = g * kGroup + (r - is_v * kGroup);
+                    } else {
+                        const int r = i - full_tiles, d = rem > 0 ? rem : 1;
+                        is_v = r / d;
+                        page = (np / kGroup) * kGroup + (r - is_v * d);
+                    }
+                    const int pg = __shfl_sync(0xffffffffu, pid, page & 31);
+                    if (lane < kBatch && i < ntiles) {
+                        const uint32_t cc = c + i, st = cc % kStages, par = (cc / kStages) & 1u;
+                        const CUtensorMap *map = is_v ? &v_map : &k_map;
+                        if (mbar_wait(&tail->empty[st], par ^ 1u, abort, a.status)) {
+                            mbar_arrive_expect_tx(&tail->full[st], kTileBytes);
+                            const int row = (pg * Hkv + s.kvh) * kPage;
+                            tma_box_load(ring + st * kTileBytes, map, 0, row, &tail->full[st]);
+                        }
+                    }
+                    __syncwarp();
+                }
+                c += ntiles;
+            }
+        }
+        if (lane == 0 && *abort) {
+            const uint32_t n = c < (uint32_t)kStages ? c : (uint32_t)kStages;
+            for (uint32_t i = 0; i < n; ++i) {
+                const uint32_t cc = c - 1 - i;
+                const long long t0 = clock64();
+                while (!mbar_try_wait(&tail->full[cc % kStages], (cc / kStages) & 1u) && clock64() - t0 < (1ll << 24)) {
+                }
+            }
+        }
+        return;
+    }
+
+    // ==================================== consumer warps ==========================================
+    const int gq = lane >> 2, tq = lane & 3;   // fragment coordinates: row / column pair
+    const bool row_ok = gq < G;                // this lane's row is a real query head
+    const uint32_t ring_addr = smem_u32(ring);
+    uint32_t seg_base = 0;
+    int cur = r0;
+    Segment s;
+    int n_parked = 0;
+    Parked pk[kParked];
+
+    // Ordering against the previous kernel on the stream.  Writes to `out` always wait for it
+    // (griddepcontrol.wait, once per CTA, and only in CTAs that have something to write there, plus
+    // CTA 0, which keeps the calls completing in stream order).  Writes to the workspace wait for it
+    // too, unless the call owns a workspace set that no unfinished call can still be reading: sets
+    // rotate with the call's generation number, and the combine kernel of every call publishes the
+    // generation in *done_gen when it is through.
+    bool waited = false;
+    auto ensure_wait = [&]() {
+        if (!waited) { wait_for_predecessor(); waited = true; }
+    };
+    // The set is free when the newest completed call lies in [gen - sets, gen - 1]: calls complete in
+    // stream order, so the set's previous user (gen - sets) is among the completed.  A value outside
+    // the window -- in particular a newer generation left behind by an earlier replay of a captured
+    // graph, whose generations repeat -- proves nothing and the CTA waits instead.
+    const bool may_early = a.sets >= 3 && !a.force_wait;
+    auto set_is_free = [&]() -> bool {
+        unsigned d;
+        asm volatile("ld.relaxed.gpu.global.u32 %0, [%1];" : "=r"(d) : "l"(a.done_gen) : "memory");
+        return (uint32_t)(a.gen - 1u - d) < (uint32_t)a.sets;
+    };
+    bool early_known = false;   // thread 0 only; looked up now so that the answer is there when it is needed
+    if (tid == 0 && may_early) early_known = set_is_free();
+    // Publishes the parked segment results.  Parts of split (sequence, head)s go to the workspace as
+    // partials (the combine kernel that follows merges them); results that are already final are
+    // written to `out` -- at once in the middle of a range (`last_call` false), or left parked for
+    // the epilogue, after the wait.
+    auto flush = [&](bool last_call) {
+        bool any_multi = false, any_single = false;
+        for (int j = 0; j < n_parked; ++j) {
+            any_multi = any_multi || pk[j].nparts > 1;
+            any_single = any_single || pk[j].nparts == 1;
+        }
+        if (any_multi) {
+            if (tid == 0) {
+                if (may_early && !early_known) early_known = set_is_free();
+                tail->early = early_known ? 1 : 0;
+            }
+            named_barrier(1, kConsThreads);
+            if (!tail->early) ensure_wait();
+            for (int j = 0; j < n_parked; ++j) {
+                if (pk[j].nparts == 1) continue;
+                const float *rec = park + j * REC;
+                const size_t slot = (size_t)pk[j].bk + blockIdx.x;
+                for (int idx = tid; idx < G * kD / 4; idx += kConsThreads)
+                    reinterpret_cast<float4 *>(a.part_o + slot * G * kD)[idx] =
+                        reinterpret_cast<const float4 *>(rec + 2 * GP)[idx];
+                if (tid < G) {
+                    a.part_ml[(slot * GP + tid) * 2 + 0] = rec[tid];
+                    a.part_ml[(slot * GP + tid) * 2 + 1] = rec[GP + tid];
+                }
+            }
+        }
+        if (!last_call) {
+            if (any_single) ensure_wait();
+            for (int j = 0; j < n_parked; ++j) {
+                if (pk[j].nparts != 1) continue;
+                const float *rec = park + j * REC;
+                for (int idx = tid; idx < G * kD; idx += kConsThreads)
+                    reinterpret_cast<__nv_bfloat16 *>(a.out)[pk[j].out_base + idx] =
+                        __float2bfloat16_rn(rec[2 * GP + idx] / rec[GP + idx / kD]);
+            }
+            named_barrier(1, kConsThreads);  // parking slots are free again
+            n_parked = 0;
+        }
+    };
+
+    while (next_segment(cur, r1, pref, slen, B, Hkv, chunk, s)) {
+        const int qrow = row0[s.b];
+        // A fragments of q (16 x 128, rows >= G zero), f16: k-slice ks covers dims 16 ks .. 16 ks + 15 in the
+        // order the widened codes arrive in: this lane holds dims 16 ks + 4 tq + {0, 1} (k = 2 tq, + 1) and
+        // + {2, 3} (k = 8 + 2 tq, + 1)
+        uint32_t qa[8][4];
+        {
+            const char *qh = a.q + ((size_t)qrow * a.Hq + s.kvh * G + gq) * kD * 2;
+#pragma unroll
+            for (int ks = 0; ks < 8; ++ks) {
+                const uint2 raw = row_ok ? __ldg(reinterpret_cast<const uint2 *>(qh + ks * 32 + tq * 8)) : make_uint2(0u, 0u);
+                qa[ks][0] = pack_f16(__uint_as_float(raw.x << 16), __uint_as_float(raw.x & 0xffff0000u));
+                qa[ks][2] = pack_f16(__uint_as_float(raw.y << 16), __uint_as_float(raw.y & 0xffff0000u));
+                qa[ks][1] = 0u;
+                qa[ks][3] = 0u;
+            }
+        }
+        // this lane's row (head gq): running max (the same in the 4 lanes of a row), its share of the
+        // sum, and 16 n-tiles of the output row: o[2c][0..1] = dims 16c + 4 tq, + 2 and o[2c+1][0..1] = dims 16c + 4 tq + 1, + 3
+        // (o[n][2..3]: rows 8..15)
+        float m_run = -INFINITY, l_run = 0.f;
+        float o[16][4];
+#pragma unroll
+        for (int n = 0; n < 16; ++n) { o[n][0] = o[n][1] = o[n][2] = o[n][3] = 0.f; }
+
+        const int seg_pages = s.pg1 - s.pg0;
+        const int ngroups = (seg_pages + kGroup - 1) / kGroup;
+        for (int gi = warp; gi < ngroups; gi += kConsWarps) {
+            const int p0 = s.pg0 + gi * kGroup;
+            const int npg = min(kGroup, s.pg1 - p0);
+            const int ntok = min(s.L - p0 * kPage, npg * kPage);
+            const uint32_t gbase = seg_base + (uint32_t)gi * 2 * kGroup;
+
+            // ---- S = q K^T for the group's pages: per page two n-tiles of 8 keys -----------------
+            float sc[kGroup * 2][4];
+#pragma unroll
+            for (int t = 0; t < kGroup; ++t) {
+#pragma unroll
+                for (int j = 0; j < 2; ++j) { sc[t * 2 + j][0] = sc[t * 2 + j][1] = sc[t * 2 + j][2] = sc[t * 2 + j][3] = 0.f; }
+                if (t < npg) {
+                    const uint32_t cc = gbase + t, st = cc % kStages, par = (cc / kStages) & 1u;
+                    mbar_wait(&tail->full[st], par, abort, a.status);
+                    const uint32_t tile = ring_addr + st * kTileBytes;
+#pragma unroll
+                    for (int j = 0; j < 2; ++j) {          // keys 8j .. 8j+7 of the page
+#pragma unroll
+                        for (int kq = 0; kq < 2; ++kq) {   // k-slices 4kq .. 4kq + 3: one 16-byte chunk of codes each
+                            uint32_t bfr[4];
+                            ldmatrix_x4(tile + tile_off(8 * j + (lane & 7), 4 * kq + (lane >> 3)), bfr);
+#pragma unroll
+                            for (int i = 0; i < 4; ++i)
+                                mma_16816(sc[t * 2 + j], qa[4 * kq + i], e4m3x2_to_f16x2(bfr[i]), e4m3x2_to_f16x2(bfr[i] >> 16));
+                        }
+                    }
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&tail->empty[st]);
+                }
+            }
+
+            // ---- online softmax on the fragments: this lane has 2 scores per n-tile of its row ------
+            float mx = -INFINITY;
+#pragma unroll
+            for (int nt = 0; nt < kGroup * 2; ++nt) {
+#pragma unroll
+                for (int e = 0; e < 2; ++e) {
+                    const int key = nt * 8 + tq * 2 + e;
+                    const float v = (key < ntok) ? sc[nt][e] * a.scale_log2 : -INFINITY;
+                    sc[nt][e] = v;
+                    mx = fmaxf(mx, v);
+                }
+            }
+            mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
+            mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
+            const float m_new = fmaxf(m_run, mx);            // finite: the group has a visible key
+            const float f = fast_exp2(m_run - m_new);        // 0 for the first group
+            m_run = m_new;
+            uint32_t pa[kGroup][4];                          // A fragments of P: one k-slice per page
+            float lsum = 0.f;
+#pragma unroll
+            for (int t = 0; t < kGroup; ++t) {
+                const float p00 = fast_exp2(sc[2 * t][0] - m_new), p01 = fast_exp2(sc[2 * t][1] - m_new);
+                const float p10 = fast_exp2(sc[2 * t + 1][0] - m_new), p11 = fast_exp2(sc[2 * t + 1][1] - m_new);
+                const uint32_t w0 = pack_f16(p00, p01), w1 = pack_f16(p10, p11);
+                pa[t][0] = w0;   // row gq, keys 2 tq, +1
+                pa[t][2] = w1;   // row gq, keys 8 + 2 tq, +1
+                pa[t][1] = 0u;   // rows 8..15
+                pa[t][3] = 0u;
+                // the sum uses the rounded weights, like the tensor core
+                const float2 r0 = unpack_f16(w0), r1 = unpack_f16(w1);
+                lsum += (r0.x + r0.y) + (r1.x + r1.y);
+            }
+            l_run = fmaf(l_run, f, lsum);
+            if (__any_sync(0xffffffffu, f != 1.0f)) {
+#pragma unroll
+                for (int n = 0; n < 16; ++n) { o[n][0] *= f; o[n][1] *= f; }
+            }
+
+            // ---- O += P V: per page 16 n-tiles of 8 dims, one k-slice of 16 keys ------------------
+#pragma unroll
+            for (int t = 0; t < kGroup; ++t) {
+                if (t < npg) {
+                    const uint32_t cc = gbase + npg + t, st = cc % kStages, par = (cc / kStages) & 1u;
+                    mbar_wait(&tail->full[st], par, abort, a.status);
+                    const uint32_t tile = ring_addr + st * kTileBytes;
+                    const int nvalid = ntok - t * kPage;
+                    if (nvalid < kPage) {
+                        // slots past the sequence end may hold anything; they must not reach the
+                        // tensor core, not even times zero: blank them in shared memory
+                        for (int i = lane; i < (kPage - nvalid) * 8; i += 32) {
+                            const int r = nvalid + (i >> 3), c = i & 7;
+                            *reinterpret_cast<uint4 *>(ring + st * kTileBytes + tile_off(r, c)) = make_uint4(0, 0, 0, 0);
+                        }
+                        __syncwarp();
+                    }
+#pragma unroll
+                    for (int np2 = 0; np2 < 4; ++np2) {    // dims 32 np2 .. 32 np2 + 31: two 16-byte chunks of codes
+                        uint32_t bfr[4];
+                        // blocks: (keys 0-7, chunk 2np2), (keys 8-15, 2np2), (keys 0-7, 2np2+1), (keys 8-15, 2np2+1);
+                        // a lane gets (key 2tq: dims d, d+1 | key 2tq+1: dims d, d+1) with d = 16 chunk + 2 gq
+                        ldmatrix_x4_trans(tile + tile_off((lane & 7) + ((lane >> 3) & 1) * 8, 2 * np2 + (lane >> 4)), bfr);
+#pragma unroll
+                        for (int h = 0; h < 2; ++h) {      // chunk 2np2 + h
+                            // bytes -> (key 2tq, key 2tq+1) of dim d | the same of dim d + 1
+                            const uint32_t lo = byte_perm(bfr[2 * h], 0x3120u), hi = byte_perm(bfr[2 * h + 1], 0x3120u);
+                            mma_16816(o[4 * np2 + 2 * h], pa[t], e4m3x2_to_f16x2(lo), e4m3x2_to_f16x2(hi));
+                            mma_16816(o[4 * np2 + 2 * h + 1], pa[t], e4m3x2_to_f16x2(lo >> 16), e4m3x2_to_f16x2(hi >> 16));
+                        }
+                    }
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&tail->empty[st]);
+                }
+            }
+        }
+        seg_base += 2u * (uint32_t)seg_pages;
+
+        // ---- segment end: every warp leaves (max, sum, row accumulators); all threads merge them ------
+        l_run += __shfl_xor_sync(0xffffffffu, l_run, 1);
+        l_run += __shfl_xor_sync(0xffffffffu, l_run, 2);
+        float *rec = osm + warp * REC;
+        if (row_ok) {
+#pragma unroll
+            for (int c = 0; c < 8; ++c)   // four consecutive dims per 16-dim group
+                *reinterpret_cast<float4 *>(rec + 2 * GP + gq * kD + 16 * c + 4 * tq) =
+                    make_float4(o[2 * c][0], o[2 * c + 1][0], o[2 * c][1], o[2 * c + 1][1]);
+            if (tq == 0) { rec[gq] = m_run; rec[GP + gq] = l_run; }
+        }
+        if (n_parked == kParked) flush(false);  // uniform across the consumer threads
+        named_barrier(1, kConsThreads);
+        float *dst = park + n_parked * REC;
+        for (int idx = tid; idx < G * kD; idx += kConsThreads) {
+            const int h = idx / kD;
+            float M = -INFINITY;
+#pragma unroll
+            for (int w = 0; w < kConsWarps; ++w) M = fmaxf(M, osm[w * REC + h]);
+            float l = 0.f, acc = 0.f;
+#pragma unroll
+            for (int w = 0; w < kConsWarps; ++w) {
+                const float ff = fast_exp2(osm[w * REC + h] - M);  // 0 for a warp that had no group
+                l = fmaf(ff, osm[w * REC + GP + h], l);
+                acc = fmaf(ff, osm[w * REC + 2 * GP + idx], acc);
+            }
+            dst[2 * GP + idx] = acc * a.v_scale;   // values are v_scale * code
+            if (idx - h * kD == 0) { dst[h] = M; dst[GP + h] = l; }
+        }
+        pk[n_parked].bk = s.bk;
+        pk[n_parked].nparts = s.nparts;
+        pk[n_parked].c_first = s.c_first;
+        pk[n_parked].out_base = ((size_t)qrow * a.Hq + s.kvh * G) * kD;
+        ++n_parked;
+        named_barrier(1, kConsThreads);  // warp records are free for the next segment
+    }
+    if (n_parked > 0) flush(true);  // final results stay parked until the epilogue
+
+    // ---- epilogue: what goes to `out` waits for the previous kernel.  A CTA that only produced parts
+    //      of split (sequence, head)s has nothing to write there and leaves at once, freeing its
+    //      place on the SM for the next call.
+    bool any_single = false;
+    for (int j = 0; j < n_parked; ++j) any_single = any_single || pk[j].nparts == 1;
+    if (any_single || blockIdx.x == 0) ensure_wait();
+    for (int j = 0; j < n_parked; ++j) {
+        if (pk[j].nparts != 1) continue;
+        const float *rec = park + j * REC;
+        for (int idx = tid; idx < G * kD; idx += kConsThreads)
+            reinterpret_cast<__nv_bfloat16 *>(a.out)[pk[j].out_base + idx] =
+                __float2bfloat16_rn(rec[2 * GP + idx] / rec[GP + idx / kD]);
+    }
+}
+
+// ---- split combine ---------------------------------------------------------------------------------
+// Launched right behind the decode kernel as its programmatic dependent: its CTAs come up while the
+// decode kernel is still streaming, work out the same plan from the lengths, and then wait for the
+// decode kernel to complete (griddepcontrol.wait), which makes every partial visible without a fence,
+// an arrival counter or a CTA of the decode kernel staying behind.  One work item is a split
+// (sequence, kv head); a thread merges one or two 4-dimension pieces of the group's G x 128 outputs
+// over the parts,
+//     m = max_p m_p,  w_p = 2^(m_p - m),  out = sum_p w_p o_p / sum_p w_p l_p.
+// Few, light CTAs on purpose: they sit on the SMs, waiting, while decode CTAs of this and of the
+// next call need the room.  The last CTA to finish publishes the call's generation (see the
+// workspace rotation).
+constexpr int kCombineThreads = 128;
+constexpr int kCombinePreload = 4;   // parts whose values are asked for before the weights are known
+
+struct CombineArgs {
+    const int32_t *seq_lens;
+    const int32_t *q_lens;
+    char *out;
+    const float *part_o;
+    const float *part_ml;
+    int batch, Hq, Hkv, max_pages;
+    int small_ctas, decode_grid;
+    uint32_t gen;
+    unsigned *done_gen;
+    int *exit_count;
+};
+
+template <int G>
+__global__ void __launch_bounds__(kCombineThreads)
+decode_combine_kernel(const CombineArgs a) {
+    constexpr int GP = (G + 3) / 4 * 4;
+    constexpr int VECS = G * kD / 4;                                       // float4 pieces of one partial output
+    constexpr int NE = (VECS + kCombineThreads - 1) / kCombineThreads;     // pieces per thread (1 or 2)
+    extern __shared__ int csm[];
+    int *pref = csm;                      // [B + 1] pages (times kv heads) before sequence b
+    int *row0 = pref + a.batch + 1;       // [B + 1] q rows before sequence b
+    float2 *ml_s = reinterpret_cast<float2 *>(row0 + a.batch + 1);   // [parts][G] (max, sum); 2 (B + 1) ints before it
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int B = a.batch, Hkv = a.Hkv;
+
+    let_successor_start();
+    if (tid == 0) { pref[0] = 0; row0[0] = 0; }
+    for (int b = tid; b < B; b += kCombineThreads) {
+        const int n = a.q_lens[b], L = a.seq_lens[b];
+        const int pages = (n == 1 && L >= 1 && L <= a.max_pages * kPage) ? (L + kPage - 1) / kPage : 0;
+        pref[b + 1] = pages * Hkv;
+        row0[b + 1] = n > 0 ? n : 0;
+    }
+    __syncthreads();
+    if (warp == 0) {
+        int carry_p = 0, carry_r = 0;
+        for (int b0 = 0; b0 < B; b0 += 32) {
+            const int b = b0 + lane;
+            int vp = b < B ? pref[b + 1] : 0;
+            int vr = b < B ? row0[b + 1] : 0;
+#pragma unroll
+            for (int off = 1; off < 32; off <<= 1) {
+                const int tp = __shfl_up_sync(0xffffffffu, vp, off);
+                const int tr = __shfl_up_sync(0xffffffffu, vr, off);
+                if (lane >= off) { vp += tp; vr += tr; }
+            }
+            if (b < B) { pref[b + 1] = vp + carry_p; row0[b + 1] = vr + carry_r; }
+            carry_p += __shfl_sync(0xffffffffu, vp, 31);
+            carry_r += __shfl_sync(0xffffffffu, vr, 31);
+        }
+    }
+    __syncthreads();
+    const int total = pref[B];
+    const int chunk = plan_chunk(total, a.decode_grid, a.small_ctas);
+
+    wait_for_predecessor();   // the decode kernel of this call, and with it every earlier call
+
+    int ev[NE], eh[NE];       // this thread's pieces: index into a partial output, and its head
+    bool eok[NE];
+#pragma unroll
+    for (int k = 0; k < NE; ++k) {
+        const int e = tid + k * kCombineThreads;
+        eok[k] = e < VECS;
+        ev[k] = eok[k] ? e : 0;
+        eh[k] = ev[k] / (kD / 4);
+    }
+    for (int bk = blockIdx.x; bk < B * Hkv; bk += gridDim.x) {
+        const int b = bk / Hkv, kvh = bk - b * Hkv;
+        const int pages = (pref[b + 1] - pref[b]) / Hkv;
+        if (pages == 0) continue;
+        const int s0 = pref[b] + kvh * pages, s1 = s0 + pages;
+        const int c_first = s0 / chunk;
+        const int nparts = (s1 - 1) / chunk - c_first + 1;   // at most one per CTA of the decode grid
+        if (nparts <= 1) continue;       // the decode kernel wrote this one itself
+        const size_t slot0 = (size_t)bk + c_first;
+        const float4 *po = reinterpret_cast<const float4 *>(a.part_o + slot0 * G * kD);
+        // the first partial values are asked for before the weights exist, so that the two round
+        // trips to memory run side by side
+        float4 v[NE][kCombinePreload];
+#pragma unroll
+        for (int u = 0; u < kCombinePreload; ++u)
+#pragma unroll
+            for (int k = 0; k < NE; ++k) v[k][u] = __ldcg(po + (size_t)min(u, nparts - 1) * VECS + ev[k]);
+        __syncthreads();                 // ml_s of the previous item has been read by everyone
+        for (int i = tid; i < nparts * G; i += kCombineThreads) {
+            const int p = i / G, h = i - p * G;
+            ml_s[i] = __ldcg(reinterpret_cast<const float2 *>(a.part_ml + ((slot0 + p) * GP + h) * 2));
+        }
+        __syncthreads();
+        float m[NE], l[NE];
+        float4 x[NE];
+#pragma unroll
+        for (int k = 0; k < NE; ++k) {
+            m[k] = -INFINITY;
+            for (int p = 0; p < nparts; ++p) m[k] = fmaxf(m[k], ml_s[p * G + eh[k]].x);
+            l[k] = 0.f;
+            x[k] = make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+        for (int p0 = 0; p0 < nparts; p0 += kCombinePreload) {
+            if (p0 > 0) {
+#pragma unroll
+                for (int u = 0; u < kCombinePreload; ++u)
+#pragma unroll
+                    for (int k = 0; k < NE; ++k) v[k][u] = __ldcg(po + (size_t)min(p0 + u, nparts - 1) * VECS + ev[k]);
+            }
+#pragma unroll
+            for (int u = 0; u < kCombinePreload; ++u) {
+                if (p0 + u < nparts) {
+#pragma unroll
+                    for (int k = 0; k < NE; ++k) {
+                        const float2 ml = ml_s[(p0 + u) * G + eh[k]];
+                        const float w = fast_exp2(ml.x - m[k]);
+                        l[k] = fmaf(w, ml.y, l[k]);
+                        x[k].x = fmaf(w, v[k][u].x, x[k].x);
+                        x[k].y = fmaf(w, v[k][u].y, x[k].y);
+                        x[k].z = fmaf(w, v[k][u].z, x[k].z);
+                        x[k].w = fmaf(w, v[k][u].w, x[k].w);
+                    }
+                }
+            }
+        }
+        __nv_bfloat16 *orow = reinterpret_cast<__nv_bfloat16 *>(a.out) + ((size_t)row0[b] * a.Hq + kvh * G) * kD;
+#pragma unroll
+        for (int k = 0; k < NE; ++k) {
+            if (eok[k]) {
+                const float inv = 1.0f / l[k];
+                uint2 o2;
+                o2.x = pack_bf16(x[k].x * inv, x[k].y * inv);
+                o2.y = pack_bf16(x[k].z * inv, x[k].w * inv);
+                *reinterpret_cast<uint2 *>(orow + (size_t)ev[k] * 4) = o2;
+            }
+        }
+    }
+    // The last CTA through publishes this call's generation: its workspace set has been read for the
+    // last time, and every earlier call has completed (every CTA here waited for the decode kernel,
+    // whose CTA 0 waited for the kernel before it).
+    __syncthreads();
+    if (tid == 0) {
+        const int old = atomicAdd(a.exit_count, 1);
+        if (old == (int)gridDim.x - 1) {
+            *a.exit_count = 0;
+            __threadfence();
+            asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(a.done_gen), "r"(a.gen) : "memory");
+        }
+    }
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_tiled_fn() {
+    static EncodeTiledFn fn = nullptr;
+    static bool tried = false;
+    if (!tried) {
+        tried = true;
+        void *p = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) == cudaSuccess &&
+            qres == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(p);
+        cudaGetLastError();
+    }
+    return fn;
+}
+
+bool make_pool_map(CUtensorMap *map, const void *pool, const arb_attn_params &p) {
+    EncodeTiledFn fn = encode_tiled_fn();
+    if (!fn) return false;
+    const cuuint64_t dims[2] = {(cuuint64_t)kD, (cuuint64_t)p.num_pages * p.num_kv_heads * kPage};
+    const cuuint64_t strides[1] = {(cuuint64_t)kD};
+    const cuuint32_t box[2] = {(cuuint32_t)kD, (cuuint32_t)kPage};
+    const cuuint32_t estr[2] = {1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void *>(pool), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+template <int G>
+arb_status launch_one(Ctx *ctx, const Args &a, CombineArgs ca, const CUtensorMap &km, const CUtensorMap &vm,
+                      bool overlap, cudaStream_t stream) {
+    const size_t smem = smem_bytes<G>(a.batch);
+    static bool attr_set[64] = {};
+    if (!attr_set[ctx->device & 63]) {
+        if (cudaFuncSetAttribute(decode_e4m3_kernel<G>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 (int)smem_bytes<G>(kMaxBatch)) != cudaSuccess)
+            return ARB_ERR_CUDA;
+        attr_set[ctx->device & 63] = true;
+    }
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cudaLaunchConfig_t cfg = {};
+    // A call that cannot be anything but small -- the block table has room for at most kSmallCallPages
+    // pages per SM -- is launched with one CTA per SM outright: no CTA comes up only to leave.
+    const long long page_bound = (long long)a.batch * a.max_pages * a.Hkv;
+    const bool small = page_bound <= (long long)ctx->num_sms * kSmallCallPages;
+    const int grid = small ? ctx->num_sms : ctx->num_sms * kCtasPerSm;
+    cfg.gridDim = dim3(grid);
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cfg.attrs = attr;
+    cfg.numAttrs = overlap ? 1 : 0;
+    if (cudaLaunchKernelEx(&cfg, decode_e4m3_kernel<G>, a, km, vm) != cudaSuccess) return ARB_ERR_CUDA;
+    ctx->launches++;
+    // the combine kernel, always a programmatic dependent of the decode kernel
+    ca.decode_grid = grid;
+    const long long items = (long long)a.batch * a.Hkv;
+    cudaLaunchConfig_t ccfg = {};
+    ccfg.gridDim = dim3((unsigned)(items < ctx->num_sms ? items : ctx->num_sms));
+    ccfg.blockDim = dim3(kCombineThreads);
+    ccfg.dynamicSmemBytes = sizeof(int) * (2 * (size_t)a.batch + 2) + sizeof(float2) * (size_t)grid * G;
+    ccfg.stream = stream;
+    ccfg.attrs = attr;
+    ccfg.numAttrs = 1;
+    if (cudaLaunchKernelEx(&ccfg, decode_combine_kernel<G>, ca) != cudaSuccess) return ARB_ERR_CUDA;
+    ctx->launches++;
+    return ARB_OK;
+}
+
+}  // namespace
+
+arb_status launch_decode_e4m3(Ctx *ctx, const arb_attn_params &p, const void *q, const void *k_pages,
+                              const void *v_pages, float k_scale, float v_scale, const int32_t *block_table,
+                              const int32_t *seq_lens, const int32_t *q_lens, void *out, cudaStream_t stream) {
+    if (encode_tiled_fn() == nullptr) return ARB_ERR_UNSUPPORTED;
+    alignas(64) CUtensorMap km, vm;
+    if (!make_pool_map(&km, k_pages, p) || !make_pool_map(&vm, v_pages, p)) return ARB_ERR_CUDA;
+    const int g = p.num_q_heads / p.num_kv_heads;
+    const int gp = (g + 3) / 4 * 4;
+    const size_t slots = (size_t)p.batch * p.num_kv_heads + (size_t)ctx->num_sms * kCtasPerSm;
+    // Workspace rotation.  Consecutive calls take consecutive generation numbers and use workspace set
+    // (generation mod sets): partials, (max, sum) records and arrival counters of their own.  A call
+    // may write its set without waiting for the previous call once the set's previous user
+    // (generation - sets) has published its completion.  With fewer than three sets that fit in the
+    // workspace, or right after a CUDA-core decode call (which uses set 0 unnumbered), it waits.
+    const size_t part_o_floats = (slots * g * p.head_dim + 63) & ~size_t(63);
+    const size_t set_bytes = ((part_o_floats + slots * gp * 2) * sizeof(float) + 255) & ~size_t(255);
+    int sets = (int)(ctx->workspace_bytes / set_bytes);
+    if (sets > kRotSets) sets = kRotSets;
+    if (sets < 1) return ARB_ERR_WORKSPACE;
+    if ((long long)p.batch * p.num_kv_heads > kRotCounters) sets = 1;
+    const uint32_t gen = ctx->decode_gen++;
+    const int set = (int)(gen % (uint32_t)sets);
+    Args a;
+    a.q = static_cast<const char *>(q);
+    a.block_table = block_table;
+    a.seq_lens = seq_lens;
+    a.q_lens = q_lens;
+    a.out = static_cast<char *>(out);
+    a.part_o = reinterpret_cast<float *>(ctx->workspace + (size_t)set * set_bytes);
+    a.part_ml = a.part_o + part_o_floats;
+    a.done_gen = reinterpret_cast<unsigned *>(ctx->rot + (size_t)kRotSets * kRotCounters + kRotSets);
+    a.gen = gen;
+    a.sets = sets;
+    a.force_wait = ctx->last_decode_shared_set0 ? 1 : 0;
+    ctx->last_decode_shared_set0 = false;
+    a.status = ctx->status;
+    a.batch = p.batch;
+    a.Hq = p.num_q_heads;
+    a.Hkv = p.num_kv_heads;
+    a.num_pages = p.num_pages;
+    a.max_pages = p.max_pages_per_seq;
+    // A small call streams at the pace of its CTAs' pipelines, not of the memory system, and every
+    // CTA spends a fixed time before its first and after its last tile.  A call that declares itself
+    // part of a back-to-back series (ARB_ATTN_OVERLAP_PREVIOUS) therefore takes only every second
+    // SM's worth of CTAs: each lives longer, four calls are in flight instead of two, and the
+    // series as a whole moves more bytes per second; a lone call gets one CTA on every SM, which
+    // is what finishes it soonest.
+    a.small_ctas = (p.flags & ARB_ATTN_OVERLAP_PREVIOUS) ? (ctx->num_sms + 1) / 2 : ctx->num_sms;
+    const float scale = p.softmax_scale > 0.f ? p.softmax_scale : 1.0f / sqrtf((float)p.head_dim);
+    a.scale_log2 = scale * k_scale * 1.4426950408889634f;   // keys are k_scale * code
+    a.v_scale = v_scale;
+    const bool overlap = (p.flags & ARB_ATTN_OVERLAP_PREVIOUS) != 0;
+    CombineArgs ca;
+    ca.seq_lens = seq_lens;
+    ca.q_lens = q_lens;
+    ca.out = a.out;
+    ca.part_o = a.part_o;
+    ca.part_ml = a.part_ml;
+    ca.batch = a.batch;
+    ca.Hq = a.Hq;
+    ca.Hkv = a.Hkv;
+    ca.max_pages = a.max_pages;
+    ca.small_ctas = a.small_ctas;
+    ca.decode_grid = 0;  // set by launch_one
+    ca.gen = gen;
+    ca.done_gen = a.done_gen;
+    ca.exit_count = ctx->rot + (size_t)kRotSets * kRotCounters + set;
+    switch (g) {
+        case 1: return launch_one<1>(ctx, a, ca, km, vm, overlap, stream);
+        case 2: return launch_one<2>(ctx, a, ca, km, vm, overlap, stream);
+        case 3: return launch_one<3>(ctx, a, ca, km, vm, overlap, stream);
+        case 4: return launch_one<4>(ctx, a, ca, km, vm, overlap, stream);
+        case 5: return launch_one<5>(ctx, a, ca, km, vm, overlap, stream);
+        case 6: return launch_one<6>(ctx, a, ca, km, vm, overlap, stream);
+        case 7: return launch_one<7>(ctx, a, ca, km, vm, overlap, stream);
+        case 8: return launch_one<8>(ctx, a, ca, km, vm, overlap, stream);
+        default: return ARB_ERR_UNSUPPORTED;
+    }
+}
+
+}  // namespace arb

@@ -3,6 +3,7 @@ import numpy as np
 import pytest
 import torch
 
+from oracle import oracle
 from paper_2512_05033_b200 import workloads as wl
 from tests import helpers as H
 
@@ -308,3 +309,65 @@ def test_overlap_flag_in_a_replayed_graph():
         for a, b in zip(expect, outs):
             assert torch.equal(a, b), rep
     assert c.poll_status() == 0
+
+
+E4M3_CASES = [
+    # (B, Hq, Hkv, seq_lens)
+    (3, 12, 2, [16, 17, 15]),                                  # page boundaries
+    (8, 12, 2, [1025, 2000, 3001, 777, 4096, 1, 640, 5555]),   # draft-shaped, ragged
+    (4, 32, 8, [4100, 9000, 33, 12000]),                       # g = 4
+    (2, 28, 4, [3000, 150]),                                   # g = 7
+    (1, 5, 1, [40000]),                                        # one long sequence over every CTA
+    (2, 16, 2, [2100, 900]),                                   # g = 8
+    (5, 8, 2, [100, 1, 300, 1, 47]),                           # with idle slots (below)
+]
+
+
+@pytest.mark.parametrize("case", E4M3_CASES)
+def test_e4m3_decode_matches_oracle(case):
+    B, Hq, Hkv, sl = case
+    ql = [1, 0, 1, 0, 1] if B == 5 else [1] * B
+    inp = wl.small_attn_case(B, Hq, Hkv, 128, BF, sl, ql, seed=700 + Hq)
+    ks, vs = 0.011, 0.017          # N(0,1) values / scale reach about 400: the whole range of the format is used
+    kc = torch.from_numpy(oracle.e4m3_encode(inp.k_pages, 1 / ks))
+    vc = torch.from_numpy(oracle.e4m3_encode(inp.v_pages, 1 / vs))
+    # stale slots past the ends hold NaN codes: they must never reach the arithmetic
+    for b in range(B):
+        L = sl[b]
+        if L % 16:
+            page = int(inp.block_table[b, L // 16])
+            kc[page, :, L % 16:, :] = 0x7f
+            vc[page, :, L % 16:, :] = 0x7f
+    c = H.ctx()
+    d = inp.to("cuda")
+    out = torch.full_like(d.q, float("nan"))
+    c.attn_decode_e4m3(d.q, kc.cuda(), vc.cuda(), ks, vs, d.block_table, d.seq_lens, d.q_lens, out=out)
+    assert c.poll_status() == 0
+    ref, st = oracle.attn_e4m3(inp.q, kc, vc, ks, vs, inp.block_table, inp.seq_lens, inp.q_lens)
+    assert st == 0
+    H.assert_close(out.double().cpu().numpy(), ref, BF, tight=3e-3)
+
+
+def test_e4m3_decode_peaked_and_back_to_back():
+    """q scaled up so that few keys carry the weight, and flagged calls in flight behind one another."""
+    from paper_2512_05033_b200 import binding
+    inp = wl.small_attn_case(4, 12, 2, 128, BF, [3000, 513, 64, 1500], [1] * 4, seed=7, q_std=6.0)
+    ks, vs = 0.012, 0.012
+    kc = torch.from_numpy(oracle.e4m3_encode(inp.k_pages, 1 / ks))
+    vc = torch.from_numpy(oracle.e4m3_encode(inp.v_pages, 1 / vs))
+    ref, _ = oracle.attn_e4m3(inp.q, kc, vc, ks, vs, inp.block_table, inp.seq_lens, inp.q_lens)
+    c = H.ctx()
+    d = inp.to("cuda")
+    dk, dv = kc.cuda(), vc.cuda()
+    alone = c.attn_decode_e4m3(d.q, dk, dv, ks, vs, d.block_table, d.seq_lens, d.q_lens, flags=binding.ATTN_OVERLAP_PREVIOUS)
+    torch.cuda.synchronize()
+    outs = [torch.full_like(d.q, float("nan")) for _ in range(6)]
+    for rep in range(20):
+        for o in outs:
+            c.attn_decode_e4m3(d.q, dk, dv, ks, vs, d.block_table, d.seq_lens, d.q_lens, out=o,
+                               flags=binding.ATTN_OVERLAP_PREVIOUS)
+    assert c.poll_status() == 0
+    for o in outs:
+        assert torch.equal(o, alone)
+    err = np.abs(alone.double().cpu().numpy() - ref)
+    assert (err <= 2.0 ** -8 * np.abs(ref) + 3e-3).all(), err.max()

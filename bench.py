@@ -293,6 +293,7 @@ def run_ours(args):
                 result["step_loop"] = run_step_loop(ctx, dev)
                 result["kv_append"] = run_kv_append(ctx, dev, peak)
                 result["policies"] = run_policies(ctx, dev)
+                result["e4m3_decode"] = run_e4m3_decode(ctx, dev, peak)
             result["cpu_baseline"] = run_cpu_baseline(work)
     if dist:
         dist.barrier()
@@ -538,6 +539,46 @@ def run_policies(ctx, dev):
     return out
 
 
+def run_e4m3_decode(ctx, dev, peak, profile=False):
+    """Supplementary: decode over an E4M3 KV cache (arb_attn_decode_e4m3), same batches and lengths as the two
+    bf16 decode workloads, pools filled with random codes (the arithmetic does not care what they mean).
+    Algorithmic bytes: one byte per KV element, plus q, out, block table and lengths as for the bf16 cache."""
+    from paper_2512_05033_b200 import binding
+    out = {}
+    for name, shape, layers, overlap, steps in (("draft_shaped", wl.DRAFT_DECODE, 16, True, 300), ("target_shaped", wl.TARGET_DECODE, 2, False, 20)):
+        inp = wl.make_attn_inputs(shape, device=dev, seed=shape.seed)
+        pools = []
+        for l in range(layers):
+            g = torch.Generator(device=dev)
+            g.manual_seed(3000 + l)
+            pools.append((torch.randint(0, 0x7f, inp.k_pages.shape, generator=g, device=dev, dtype=torch.uint8),
+                          torch.randint(0, 0x7f, inp.k_pages.shape, generator=g, device=dev, dtype=torch.uint8)))
+        o = torch.empty_like(inp.q)
+        p = ctx.params_for(inp.q, pools[0][0], inp.block_table, 1, flags=binding.ATTN_OVERLAP_PREVIOUS if overlap else 0)
+
+        def step():
+            for kc, vc in pools:
+                ctx.attn_decode_e4m3(inp.q, kc, vc, 0.01, 0.01, inp.block_table, inp.seq_lens, inp.q_lens, out=o, params=p)
+
+        step()
+        torch.cuda.synchronize()
+        if profile:   # stream launches, a few calls, for runs under ncu
+            ms = time_steps(step, 3, 3) / 3
+        else:
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g):
+                step()
+            ms = time_steps(g.replay, steps, 5) / steps
+        b = attn_bytes(shape, inp.seq_lens.cpu().to(torch.int64), inp.q_lens.cpu().to(torch.int64))
+        nbytes = b["kv"] // 2 + b["qo"] + b["table"]
+        us = ms / layers * 1e3
+        gbs = nbytes / (us * 1e-6) / 1e9
+        out[name] = {"us_per_call": round(us, 2), "algorithmic_bytes_per_call": nbytes, "gbs": round(gbs, 1),
+                     "frac_of_measured": round(gbs / peak, 4), "kv_tokens_per_us": round(b["tokens"] / us, 1),
+                     "bf16_equivalent_gbs": round(b["total"] / (us * 1e-6) / 1e9, 1)}
+    return out
+
+
 def run_cpu_baseline(work: DecodeWorkload):
     """The fp64 oracle, as it stands, on the host cores: whole steps of the same batch."""
     from oracle import oracle
@@ -623,6 +664,8 @@ def main():
     ap.add_argument("--profile-scoring", action="store_true",
                     help="for runs under ncu: a few passes of the step-scoring workload (chunk attention, route, "
                          "rollback) and nothing else")
+    ap.add_argument("--profile-e4m3", action="store_true",
+                    help="for runs under ncu: a few calls of the E4M3 decode on both decode workloads and nothing else")
     ap.add_argument("--profile", action="store_true",
                     help="for runs under ncu: stream launches, no e2e / extras / CPU baseline")
     args = ap.parse_args()
@@ -634,6 +677,11 @@ def main():
         from paper_2512_05033_b200 import binding
         torch.cuda.set_device(0)
         print(json.dumps({"step_scoring": run_step_scoring(binding.Context(0), torch.device("cuda", 0))}), flush=True)
+    elif args.profile_e4m3:
+        from paper_2512_05033_b200 import binding
+        torch.cuda.set_device(0)
+        print(json.dumps({"e4m3_decode": run_e4m3_decode(binding.Context(0), torch.device("cuda", 0), measured_peak()[0],
+                                                         profile=True)}), flush=True)
     else:
         run_ours(args)
 

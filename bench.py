@@ -329,9 +329,16 @@ def run_e2e(ctx, work: DecodeWorkload, steps: int, world: int):
     qlh = i.q_lens.cpu().pin_memory()
     outh = torch.empty_like(qh).pin_memory()
 
+    params = ctx.params_for(qh, i.k_pages, bth, 1)
+    sp = torch.cuda.current_stream().cuda_stream
+    ptrs = [(k.data_ptr(), v.data_ptr()) for k, v in work.pools]
+    host = (bth.data_ptr(), slh.data_ptr(), qlh.data_ptr(), outh.data_ptr())
+
     def step():
-        for k, v in work.pools:
-            ctx.attn_host(qh, k, v, bth, slh, qlh, 1, out_host=outh)
+        for kp, vp in ptrs:
+            st = ctx.attn_host_raw(params, qh.data_ptr(), kp, vp, host[0], host[1], host[2], host[3], sp)
+            if st != 0:
+                raise RuntimeError(f"arb_attn_host failed with status {st}")
 
     for _ in range(3):
         step()

@@ -211,6 +211,10 @@ class Context:
         _check(st, "arb_attn_host")
         return out_host
 
+    def attn_host_raw(self, p: AttnParams, q_ptr, k_ptr, v_ptr, bt_ptr, sl_ptr, ql_ptr, out_ptr, stream_ptr) -> int:
+        """Pointer-level form of attn_host (host pointers for q, block table, lengths and out); returns the arb_status."""
+        return lib.arb_attn_host(self._h, ctypes.byref(p), q_ptr, k_ptr, v_ptr, bt_ptr, sl_ptr, ql_ptr, out_ptr, stream_ptr)
+
     # -- arb_route ----------------------------------------------------------------------------
     def route(self, hidden, w, b: float, tau: float, scores=None, decisions=None, stream=None):
         """scores fp32 [S] = sigmoid(hidden . w + b); decisions uint8 [S] = (score > tau)."""

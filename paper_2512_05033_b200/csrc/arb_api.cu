@@ -1,4 +1,5 @@
 // C ABI of the arb library: argument validation, context and dispatch.  No arithmetic here.
+#include <cstring>
 #include <new>
 
 #include "arb_common.cuh"
@@ -100,6 +101,7 @@ arb_status arb_destroy(arb_ctx *ctx) {
     cudaFree(c->spearman_acc);
     cudaFree(c->chunk_ws);
     cudaFree(c->stage);
+    cudaFreeHost(c->host_stage);
     delete c;
     return ARB_OK;
 }
@@ -199,13 +201,28 @@ arb_status arb_attn_host(arb_ctx *ctx, const arb_attn_params *params, const void
         }
         c->stage_bytes = need;
     }
-    char *dq = c->stage, *dout = dq + up(q_bytes), *dbt = dout + up(q_bytes);
+    // device staging: [out | q | block table | seq_lens | q_lens]; the four inputs are gathered in a page-locked host
+    // block of the same layout first, so that they cross the bus as one copy instead of four
+    char *dout = c->stage, *dq = dout + up(q_bytes), *dbt = dq + up(q_bytes);
     char *dsl = dbt + up(bt_bytes), *dql = dsl + up(len_bytes);
-    bool ok = cudaMemcpyAsync(dq, q_host, q_bytes, cudaMemcpyHostToDevice, s) == cudaSuccess;
-    ok = ok && cudaMemcpyAsync(dbt, block_table_host, bt_bytes, cudaMemcpyHostToDevice, s) == cudaSuccess;
-    ok = ok && cudaMemcpyAsync(dsl, seq_lens_host, len_bytes, cudaMemcpyHostToDevice, s) == cudaSuccess;
-    ok = ok && cudaMemcpyAsync(dql, q_lens_host, len_bytes, cudaMemcpyHostToDevice, s) == cudaSuccess;
-    if (!ok) return ARB_ERR_CUDA;
+    const size_t in_bytes = need - up(q_bytes);
+    if (in_bytes > c->host_stage_bytes) {
+        if (cudaStreamSynchronize(s) != cudaSuccess) return ARB_ERR_CUDA;
+        cudaFreeHost(c->host_stage);
+        c->host_stage = nullptr;
+        c->host_stage_bytes = 0;
+        if (cudaHostAlloc(&c->host_stage, in_bytes, cudaHostAllocDefault) != cudaSuccess) {
+            cudaGetLastError();
+            return ARB_ERR_CUDA;
+        }
+        c->host_stage_bytes = in_bytes;
+    }
+    char *hq = c->host_stage, *hbt = hq + up(q_bytes), *hsl = hbt + up(bt_bytes), *hql = hsl + up(len_bytes);
+    memcpy(hq, q_host, q_bytes);
+    memcpy(hbt, block_table_host, bt_bytes);
+    memcpy(hsl, seq_lens_host, len_bytes);
+    memcpy(hql, q_lens_host, len_bytes);
+    if (cudaMemcpyAsync(dq, hq, in_bytes, cudaMemcpyHostToDevice, s) != cudaSuccess) return ARB_ERR_CUDA;
     st = arb_attn(ctx, params, dq, k_pages, v_pages, reinterpret_cast<int32_t *>(dbt),
                   reinterpret_cast<int32_t *>(dsl), reinterpret_cast<int32_t *>(dql), dout, stream);
     if (st != ARB_OK) return st;

@@ -31,6 +31,8 @@ struct Ctx {
     // staging for the *_host entry points
     char *stage = nullptr;
     size_t stage_bytes = 0;
+    char *host_stage = nullptr;   // page-locked gather buffer of the *_host entry points
+    size_t host_stage_bytes = 0;
     // workspace rotation of the tensor-core decode kernel: kRotSets counter arrays, one exit counter
     // per set and the generation of the newest completed call, all in one allocation
     int *rot = nullptr;

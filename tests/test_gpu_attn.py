@@ -233,7 +233,12 @@ def test_host_buffer_entry_point():
     c = H.ctx()
     out = c.attn_host(inp.q.pin_memory(), inp.k_pages.cuda(), inp.v_pages.cuda(), inp.block_table.pin_memory(),
                       inp.seq_lens.pin_memory(), inp.q_lens.pin_memory(), 4)
-    H.assert_close(out.double().numpy(), ref, BF)
+    H.assert_close(out.double().numpy(), ref, BF)      # page-locked buffers: read and written in place over the bus
+    pageable = torch.full_like(inp.q, float("nan"))
+    out2 = c.attn_host(inp.q.clone(), inp.k_pages.cuda(), inp.v_pages.cuda(), inp.block_table.clone(),
+                       inp.seq_lens.clone(), inp.q_lens.clone(), 4, out_host=pageable)
+    H.assert_close(out2.double().numpy(), ref, BF)     # ordinary host memory: staged through device copies
+    assert torch.equal(out, out2)
 
 
 def test_repeated_calls_reuse_the_workspace():

@@ -23,6 +23,22 @@
 // loaded memory system, each holding 86 KB of shared memory that the next call's CTAs were
 // waiting for.  Now a decode CTA stores its partials and leaves; the kernel boundary makes them
 // visible, and the few light CTAs of the combine kernel are already resident when it happens.
+//
+// The same kernel, compiled a second time (template parameter E4M3), reads an E4M3 KV cache: one byte per
+// element, half the bytes of the bf16 cache per token -- the only way past the bf16 cache's HBM roofline.
+//   - a (page, kv head) tile is 16 rows x 128 bytes = 2 KB, one TMA box (128-byte swizzle); the ring has 32
+//     stages, so the bytes in flight per CTA stay the same;
+//   - the codes are widened to f16, which holds every E4M3 value exactly (cvt.rn.f16x2.e4m3x2), and the
+//     products run as f16 MMAs (fp32 accumulate); q is converted bf16 -> f16 once per segment, P is rounded to
+//     f16 (11 significant bits) and summed after rounding;
+//   - ldmatrix moves 16-bit units, i.e. pairs of codes.  For q.K a thread receives four consecutive dimensions
+//     of one key per 8 x 16-byte matrix; they serve as the B fragment of a k-slice whose sixteen "k" positions
+//     are the matrix's sixteen dimensions in the order 4t, 4t+1 | 4t+2, 4t+3 (t = lane mod 4), and q's A
+//     fragment is loaded in the same order (a dot product does not care).  For P.V the transposed load gives a
+//     thread the codes (key 2t: dims d, d+1 | key 2t+1: dims d, d+1); one byte permute sorts them into the B
+//     fragments of two n-tiles, the even and the odd dimensions of a 16-dimension group, so a thread ends up
+//     owning four consecutive output dimensions per group;
+//   - the key scale is folded into the softmax scale, the value scale into the segment result.
 #include <cuda.h>  // CUtensorMap and its enums only; the encoder is looked up at run time
 
 #include "arb_common.cuh"
@@ -36,18 +52,24 @@ constexpr int kConsWarps = 4;
 constexpr int kConsThreads = kConsWarps * 32;
 constexpr int kThreads = kConsThreads + 32;
 constexpr int kGroup = 1;       // pages per consumer work group: with 16 stages every warp has two groups in flight
-constexpr int kStages = 16;     // ring stages of one 4 KB tile each
 constexpr int kBatch = 16;      // producer lanes issuing side by side
-constexpr int kTileBytes = kPage * kD * 2;
-constexpr int kHalfTile = kTileBytes / 2;   // one TMA box: 16 rows x 64 bf16
-constexpr int kRingBytes = kStages * kTileBytes;
+constexpr int kRingBytes = 64 * 1024;
+// what differs between the bf16 cache and the E4M3 cache in the ring
+template <bool E4M3>
+struct Fmt {
+    static constexpr int kTileBytes = kPage * kD * (E4M3 ? 1 : 2);   // 4 KB (two TMA boxes of 16 rows x 64 bf16) or
+                                                                     // 2 KB (one box of 16 rows x 128 codes)
+    static constexpr int kHalfTile = kTileBytes / 2;
+    static constexpr int kStages = kRingBytes / kTileBytes;          // 16 or 32
+};
 constexpr int kMinChunk = 4;
 constexpr int kCtasPerSm = 2;
 constexpr int kParked = 2;      // segment results parked in shared memory before they are written
 constexpr int kSmallCallPages = 64;   // up to this many pages per SM a call runs one CTA per SM
-static_assert(kStages % (kConsWarps * 2 * kGroup) == 0, "a ring stage must always belong to the same warp");
-static_assert(kBatch <= kStages, "two producer lanes of one turn must never wait on the same stage: the later one "
-                                 "would be two phases ahead of the barrier and a parity wait cannot tell");
+static_assert(Fmt<false>::kStages % (kConsWarps * 2 * kGroup) == 0 && Fmt<true>::kStages % (kConsWarps * 2 * kGroup) == 0,
+              "a ring stage must always belong to the same warp");
+static_assert(kBatch <= Fmt<false>::kStages, "two producer lanes of one turn must never wait on the same stage: the later "
+                                            "one would be two phases ahead of the barrier and a parity wait cannot tell");
 
 struct Args {
     const char *q;
@@ -60,7 +82,8 @@ struct Args {
     uint32_t *status;
     int batch, Hq, Hkv, num_pages, max_pages;
     int small_ctas;   // CTAs a small call spreads over
-    float scale_log2;
+    float scale_log2;   // softmax scale (times the key scale of an E4M3 cache) * log2(e)
+    float v_scale;      // value scale of an E4M3 cache, 1 otherwise
     // workspace rotation (see launch_decode_mma): this call's generation number, the number of
     // workspace sets, the generation of the newest completed call
     uint32_t gen;
@@ -69,9 +92,10 @@ struct Args {
     unsigned *done_gen;
 };
 
+template <bool E4M3>
 struct Tail {
-    uint64_t full[kStages];
-    uint64_t empty[kStages];
+    uint64_t full[Fmt<E4M3>::kStages];
+    uint64_t empty[Fmt<E4M3>::kStages];
     int abort;
     int early;            // the workspace set is free: partials may be written before the predecessor is done
 };
@@ -89,10 +113,10 @@ struct Cfg {
     static constexpr int PARK_BYTES = kParked * REC * 4;
 };
 
-template <int G>
+template <int G, bool E4M3>
 size_t smem_bytes(int batch) {
     using C = Cfg<G>;
-    return 1024 + kRingBytes + C::OSM_BYTES + C::PARK_BYTES + sizeof(Tail) + sizeof(int) * (3 * (size_t)batch + 2);
+    return 1024 + kRingBytes + C::OSM_BYTES + C::PARK_BYTES + sizeof(Tail<E4M3>) + sizeof(int) * (3 * (size_t)batch + 2);
 }
 
 struct Segment {
@@ -159,13 +183,21 @@ __device__ __forceinline__ void ldmatrix_x4_trans(uint32_t addr, uint32_t (&r)[4
                  : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
                  : "r"(addr));
 }
-// D(16x8, fp32) += A(16x16, bf16, row) * B(16x8, bf16, col)
+// D(16x8, fp32) += A(16x16, row) * B(16x8, col), operands bf16 (bf16 cache) or f16 (widened E4M3 codes)
+template <bool F16>
 __device__ __forceinline__ void mma_16816(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
-    asm volatile(
-        "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, "
-        "{%0, %1, %2, %3};"
-        : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
-        : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+    if constexpr (F16)
+        asm volatile(
+            "mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, "
+            "{%0, %1, %2, %3};"
+            : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+            : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+    else
+        asm volatile(
+            "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, "
+            "{%0, %1, %2, %3};"
+            : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+            : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
 }
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
     uint32_t r;
@@ -173,15 +205,42 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
     return r;
 }
 
-// byte offset of 16-byte chunk `c` (0..15 across the 256-byte row) of row `r` inside a swizzled tile
-__device__ __forceinline__ uint32_t tile_off(int r, int c) {
-    return (uint32_t)((c >> 3) * kHalfTile + r * 128 + (((c & 7) ^ (r & 7)) << 4));
+__device__ __forceinline__ uint32_t pack_f16(float lo, float hi) {
+    uint32_t r;
+    asm("cvt.rn.f16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+    return r;
+}
+__device__ __forceinline__ float2 unpack_f16(uint32_t v) {
+    float lo, hi;
+    asm("{\n\t.reg .b16 l, h;\n\tmov.b32 {l, h}, %2;\n\tcvt.f32.f16 %0, l;\n\tcvt.f32.f16 %1, h;\n\t}" : "=f"(lo), "=f"(hi) : "r"(v));
+    return make_float2(lo, hi);
+}
+// two E4M3 codes (low 16 bits of v) -> f16x2, exact; the low byte lands in the low half
+__device__ __forceinline__ uint32_t e4m3x2_to_f16x2(uint32_t v) {
+    uint32_t r;
+    asm("{\n\t.reg .b16 c;\n\tcvt.u16.u32 c, %1;\n\tcvt.rn.f16x2.e4m3x2 %0, c;\n\t}" : "=r"(r) : "r"(v));
+    return r;
+}
+__device__ __forceinline__ uint32_t byte_perm(uint32_t v, uint32_t sel) {
+    uint32_t r;
+    asm("prmt.b32 %0, %1, %1, %2;" : "=r"(r) : "r"(v), "r"(sel));
+    return r;
 }
 
-template <int G>
+// byte offset of 16-byte chunk `c` of row `r` inside a swizzled tile: 16 chunks across the 256-byte row of a
+// bf16 tile (two halves of 64 dims), 8 chunks across the 128-byte row of codes of an E4M3 tile
+template <bool E4M3>
+__device__ __forceinline__ uint32_t tile_off(int r, int c) {
+    if constexpr (E4M3) return (uint32_t)(r * 128 + ((c ^ (r & 7)) << 4));
+    else return (uint32_t)((c >> 3) * Fmt<false>::kHalfTile + r * 128 + (((c & 7) ^ (r & 7)) << 4));
+}
+
+template <int G, bool E4M3>
 __global__ void __launch_bounds__(kThreads, kCtasPerSm)
 decode_mma_kernel(const Args a, const __grid_constant__ CUtensorMap k_map, const __grid_constant__ CUtensorMap v_map) {
     using C = Cfg<G>;
+    using Tail = arb::Tail<E4M3>;
+    constexpr int kStages = Fmt<E4M3>::kStages, kTileBytes = Fmt<E4M3>::kTileBytes, kHalfTile = Fmt<E4M3>::kHalfTile;
     constexpr int GP = C::GP, REC = C::REC;
     static_assert(G >= 1 && G <= 8, "query heads of a group occupy rows 0..7 of the 16-row tile");
 
@@ -312,7 +371,7 @@ decode_mma_kernel(const Args a, const __grid_constant__ CUtensorMap k_map, const
                             mbar_arrive_expect_tx(&tail->full[st], kTileBytes);
                             const int row = (pg * Hkv + s.kvh) * kPage;
                             tma_box_load(ring + st * kTileBytes, map, 0, row, &tail->full[st]);
-                            tma_box_load(ring + st * kTileBytes + kHalfTile, map, 64, row, &tail->full[st]);
+                            if constexpr (!E4M3) tma_box_load(ring + st * kTileBytes + kHalfTile, map, 64, row, &tail->full[st]);
                         }
                     }
                     __syncwarp();
@@ -410,20 +469,29 @@ decode_mma_kernel(const Args a, const __grid_constant__ CUtensorMap k_map, const
 
     while (next_segment(cur, r1, pref, slen, B, Hkv, chunk, s)) {
         const int qrow = row0[s.b];
-        // A fragments of q (16 x 128, rows >= G zero): 8 k-slices of 16 dims
+        // A fragments of q (16 x 128, rows >= G zero): 8 k-slices of 16 dims.  E4M3 cache: converted to f16, and
+        // k-slice ks holds dims 16 ks .. 16 ks + 15 in the order the widened codes arrive in: this lane has dims
+        // 16 ks + 4 tq + {0, 1} (k = 2 tq, + 1) and + {2, 3} (k = 8 + 2 tq, + 1)
         uint32_t qa[8][4];
         {
             const char *qh = a.q + ((size_t)qrow * a.Hq + s.kvh * G + gq) * kD * 2;
 #pragma unroll
             for (int ks = 0; ks < 8; ++ks) {
-                qa[ks][0] = row_ok ? __ldg(reinterpret_cast<const uint32_t *>(qh + ks * 32 + tq * 4)) : 0u;
-                qa[ks][2] = row_ok ? __ldg(reinterpret_cast<const uint32_t *>(qh + ks * 32 + 16 + tq * 4)) : 0u;
+                if constexpr (E4M3) {
+                    const uint2 raw = row_ok ? __ldg(reinterpret_cast<const uint2 *>(qh + ks * 32 + tq * 8)) : make_uint2(0u, 0u);
+                    qa[ks][0] = pack_f16(__uint_as_float(raw.x << 16), __uint_as_float(raw.x & 0xffff0000u));
+                    qa[ks][2] = pack_f16(__uint_as_float(raw.y << 16), __uint_as_float(raw.y & 0xffff0000u));
+                } else {
+                    qa[ks][0] = row_ok ? __ldg(reinterpret_cast<const uint32_t *>(qh + ks * 32 + tq * 4)) : 0u;
+                    qa[ks][2] = row_ok ? __ldg(reinterpret_cast<const uint32_t *>(qh + ks * 32 + 16 + tq * 4)) : 0u;
+                }
                 qa[ks][1] = 0u;
                 qa[ks][3] = 0u;
             }
         }
         // this lane's row (head gq): running max (the same in the 4 lanes of a row), its share of the
-        // sum, and 16 n-tiles of the output row: o[n][0..1] = dims 8n + 2 tq, + 1 (o[n][2..3]: rows 8..15)
+        // sum, and 16 n-tiles of the output row: o[n][0..1] = dims 8n + 2 tq, + 1 (o[n][2..3]: rows 8..15); with an E4M3
+        // cache o[2c][0..1] = dims 16c + 4 tq, + 2 and o[2c+1][0..1] = dims 16c + 4 tq + 1, + 3
         float m_run = -INFINITY, l_run = 0.f;
         float o[16][4];
 #pragma unroll
@@ -449,12 +517,24 @@ decode_mma_kernel(const Args a, const __grid_constant__ CUtensorMap k_map, const
                     const uint32_t tile = ring_addr + st * kTileBytes;
 #pragma unroll
                     for (int j = 0; j < 2; ++j) {          // keys 8j .. 8j+7 of the page
+                        if constexpr (E4M3) {
 #pragma unroll
-                        for (int kp = 0; kp < 4; ++kp) {   // k-slices 2kp, 2kp+1
-                            uint32_t bfr[4];
-                            ldmatrix_x4(tile + tile_off(8 * j + (lane & 7), 4 * kp + (lane >> 3)), bfr);
-                            mma_16816(sc[t * 2 + j], qa[2 * kp], bfr[0], bfr[1]);
-                            mma_16816(sc[t * 2 + j], qa[2 * kp + 1], bfr[2], bfr[3]);
+                            for (int kq = 0; kq < 2; ++kq) {   // k-slices 4kq .. 4kq + 3: one 16-byte chunk of codes each
+                                uint32_t bfr[4];
+                                ldmatrix_x4(tile + tile_off<true>(8 * j + (lane & 7), 4 * kq + (lane >> 3)), bfr);
+#pragma unroll
+                                for (int i = 0; i < 4; ++i)
+                                    mma_16816<true>(sc[t * 2 + j], qa[4 * kq + i], e4m3x2_to_f16x2(bfr[i]),
+                                                    e4m3x2_to_f16x2(bfr[i] >> 16));
+                            }
+                        } else {
+#pragma unroll
+                            for (int kp = 0; kp < 4; ++kp) {   // k-slices 2kp, 2kp+1
+                                uint32_t bfr[4];
+                                ldmatrix_x4(tile + tile_off<false>(8 * j + (lane & 7), 4 * kp + (lane >> 3)), bfr);
+                                mma_16816<false>(sc[t * 2 + j], qa[2 * kp], bfr[0], bfr[1]);
+                                mma_16816<false>(sc[t * 2 + j], qa[2 * kp + 1], bfr[2], bfr[3]);
+                            }
                         }
                     }
                     __syncwarp();
@@ -485,14 +565,20 @@ decode_mma_kernel(const Args a, const __grid_constant__ CUtensorMap k_map, const
             for (int t = 0; t < kGroup; ++t) {
                 const float p00 = fast_exp2(sc[2 * t][0] - m_new), p01 = fast_exp2(sc[2 * t][1] - m_new);
                 const float p10 = fast_exp2(sc[2 * t + 1][0] - m_new), p11 = fast_exp2(sc[2 * t + 1][1] - m_new);
-                const uint32_t w0 = pack_bf16(p00, p01), w1 = pack_bf16(p10, p11);
+                const uint32_t w0 = E4M3 ? pack_f16(p00, p01) : pack_bf16(p00, p01);
+                const uint32_t w1 = E4M3 ? pack_f16(p10, p11) : pack_bf16(p10, p11);
                 pa[t][0] = w0;   // row gq, keys 2 tq, +1
                 pa[t][2] = w1;   // row gq, keys 8 + 2 tq, +1
                 pa[t][1] = 0u;   // rows 8..15
                 pa[t][3] = 0u;
                 // the sum uses the rounded weights, like the tensor core
-                lsum += __uint_as_float(w0 << 16) + __uint_as_float(w0 & 0xffff0000u) +
-                        __uint_as_float(w1 << 16) + __uint_as_float(w1 & 0xffff0000u);
+                if constexpr (E4M3) {
+                    const float2 r0 = unpack_f16(w0), r1 = unpack_f16(w1);
+                    lsum += (r0.x + r0.y) + (r1.x + r1.y);
+                } else {
+                    lsum += __uint_as_float(w0 << 16) + __uint_as_float(w0 & 0xffff0000u) +
+                            __uint_as_float(w1 << 16) + __uint_as_float(w1 & 0xffff0000u);
+                }
             }
             l_run = fmaf(l_run, f, lsum);
             if (__any_sync(0xffffffffu, f != 1.0f)) {
@@ -511,19 +597,31 @@ decode_mma_kernel(const Args a, const __grid_constant__ CUtensorMap k_map, const
                     if (nvalid < kPage) {
                         // slots past the sequence end may hold anything; they must not reach the
                         // tensor core, not even times zero: blank them in shared memory
-                        for (int i = lane; i < (kPage - nvalid) * 16; i += 32) {
-                            const int r = nvalid + (i >> 4), c = i & 15;
-                            *reinterpret_cast<uint4 *>(ring + st * kTileBytes + tile_off(r, c)) = make_uint4(0, 0, 0, 0);
+                        constexpr int kRowChunks = kTileBytes / kPage / 16;   // 16-byte chunks of a row: 16 or 8
+                        for (int i = lane; i < (kPage - nvalid) * kRowChunks; i += 32) {
+                            const int r = nvalid + i / kRowChunks, c = i % kRowChunks;
+                            *reinterpret_cast<uint4 *>(ring + st * kTileBytes + tile_off<E4M3>(r, c)) = make_uint4(0, 0, 0, 0);
                         }
                         __syncwarp();
                     }
 #pragma unroll
-                    for (int np2 = 0; np2 < 8; ++np2) {    // dims 16 np2 .. 16 np2 + 15
+                    for (int np2 = 0; np2 < (E4M3 ? 4 : 8); ++np2) {    // two 16-byte chunks of a row: 16 dims, or 32 dims of codes
                         uint32_t bfr[4];
                         // blocks: (keys 0-7, chunk 2np2), (keys 8-15, 2np2), (keys 0-7, 2np2+1), (keys 8-15, 2np2+1)
-                        ldmatrix_x4_trans(tile + tile_off((lane & 7) + ((lane >> 3) & 1) * 8, 2 * np2 + (lane >> 4)), bfr);
-                        mma_16816(o[2 * np2], pa[t], bfr[0], bfr[1]);
-                        mma_16816(o[2 * np2 + 1], pa[t], bfr[2], bfr[3]);
+                        ldmatrix_x4_trans(tile + tile_off<E4M3>((lane & 7) + ((lane >> 3) & 1) * 8, 2 * np2 + (lane >> 4)), bfr);
+                        if constexpr (E4M3) {
+                            // a lane has (key 2tq: dims d, d+1 | key 2tq+1: dims d, d+1) with d = 16 chunk + 2 gq
+#pragma unroll
+                            for (int h = 0; h < 2; ++h) {      // chunk 2np2 + h
+                                // bytes -> (key 2tq, key 2tq+1) of dim d | the same of dim d + 1
+                                const uint32_t lo = byte_perm(bfr[2 * h], 0x3120u), hi = byte_perm(bfr[2 * h + 1], 0x3120u);
+                                mma_16816<true>(o[4 * np2 + 2 * h], pa[t], e4m3x2_to_f16x2(lo), e4m3x2_to_f16x2(hi));
+                                mma_16816<true>(o[4 * np2 + 2 * h + 1], pa[t], e4m3x2_to_f16x2(lo >> 16), e4m3x2_to_f16x2(hi >> 16));
+                            }
+                        } else {
+                            mma_16816<false>(o[2 * np2], pa[t], bfr[0], bfr[1]);
+                            mma_16816<false>(o[2 * np2 + 1], pa[t], bfr[2], bfr[3]);
+                        }
                     }
                     __syncwarp();
                     if (lane == 0) mbar_arrive(&tail->empty[st]);
@@ -538,8 +636,14 @@ decode_mma_kernel(const Args a, const __grid_constant__ CUtensorMap k_map, const
         float *rec = osm + warp * REC;
         if (row_ok) {
 #pragma unroll
-            for (int n = 0; n < 16; ++n)
-                *reinterpret_cast<float2 *>(rec + 2 * GP + gq * kD + 8 * n + tq * 2) = make_float2(o[n][0], o[n][1]);
+            if constexpr (E4M3) {
+                for (int c = 0; c < 8; ++c)   // four consecutive dims per 16-dim group
+                    *reinterpret_cast<float4 *>(rec + 2 * GP + gq * kD + 16 * c + 4 * tq) =
+                        make_float4(o[2 * c][0], o[2 * c + 1][0], o[2 * c][1], o[2 * c + 1][1]);
+            } else {
+                for (int n = 0; n < 16; ++n)
+                    *reinterpret_cast<float2 *>(rec + 2 * GP + gq * kD + 8 * n + tq * 2) = make_float2(o[n][0], o[n][1]);
+            }
             if (tq == 0) { rec[gq] = m_run; rec[GP + gq] = l_run; }
         }
         if (n_parked == kParked) flush(false);  // uniform across the consumer threads
@@ -557,7 +661,7 @@ decode_mma_kernel(const Args a, const __grid_constant__ CUtensorMap k_map, const
                 l = fmaf(ff, osm[w * REC + GP + h], l);
                 acc = fmaf(ff, osm[w * REC + 2 * GP + idx], acc);
             }
-            dst[2 * GP + idx] = acc;
+            dst[2 * GP + idx] = E4M3 ? acc * a.v_scale : acc;   // values of an E4M3 cache are v_scale * code
             if (idx - h * kD == 0) { dst[h] = M; dst[GP + h] = l; }
         }
         pk[n_parked].bk = s.bk;
@@ -765,26 +869,27 @@ EncodeTiledFn encode_tiled_fn() {
     return fn;
 }
 
-bool make_pool_map(CUtensorMap *map, const void *pool, const arb_attn_params &p) {
+bool make_pool_map(CUtensorMap *map, const void *pool, const arb_attn_params &p, bool e4m3) {
     EncodeTiledFn fn = encode_tiled_fn();
     if (!fn) return false;
     const cuuint64_t dims[2] = {(cuuint64_t)kD, (cuuint64_t)p.num_pages * p.num_kv_heads * kPage};
-    const cuuint64_t strides[1] = {(cuuint64_t)kD * 2};
-    const cuuint32_t box[2] = {64, (cuuint32_t)kPage};
+    // bf16: rows of 256 bytes, a box is half a row (64 dims) of 16 rows; E4M3: rows of 128 bytes, a box is 16 whole rows
+    const cuuint64_t strides[1] = {(cuuint64_t)kD * (e4m3 ? 1 : 2)};
+    const cuuint32_t box[2] = {(cuuint32_t)(e4m3 ? kD : 64), (cuuint32_t)kPage};
     const cuuint32_t estr[2] = {1, 1};
-    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(pool), dims, strides, box, estr,
+    return fn(map, e4m3 ? CU_TENSOR_MAP_DATA_TYPE_UINT8 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(pool), dims, strides, box, estr,
               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-template <int G>
+template <int G, bool E4M3>
 arb_status launch_one(Ctx *ctx, const Args &a, CombineArgs ca, const CUtensorMap &km, const CUtensorMap &vm,
                       bool overlap, cudaStream_t stream) {
-    const size_t smem = smem_bytes<G>(a.batch);
+    const size_t smem = smem_bytes<G, E4M3>(a.batch);
     static bool attr_set[64] = {};
     if (!attr_set[ctx->device & 63]) {
-        if (cudaFuncSetAttribute(decode_mma_kernel<G>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 (int)smem_bytes<G>(kMaxBatch)) != cudaSuccess)
+        if (cudaFuncSetAttribute(decode_mma_kernel<G, E4M3>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 (int)smem_bytes<G, E4M3>(kMaxBatch)) != cudaSuccess)
             return ARB_ERR_CUDA;
         attr_set[ctx->device & 63] = true;
     }
@@ -803,7 +908,7 @@ arb_status launch_one(Ctx *ctx, const Args &a, CombineArgs ca, const CUtensorMap
     cfg.stream = stream;
     cfg.attrs = attr;
     cfg.numAttrs = overlap ? 1 : 0;
-    if (cudaLaunchKernelEx(&cfg, decode_mma_kernel<G>, a, km, vm) != cudaSuccess) return ARB_ERR_CUDA;
+    if (cudaLaunchKernelEx(&cfg, decode_mma_kernel<G, E4M3>, a, km, vm) != cudaSuccess) return ARB_ERR_CUDA;
     ctx->launches++;
     // the combine kernel, always a programmatic dependent of the decode kernel
     ca.decode_grid = grid;
@@ -827,11 +932,14 @@ bool decode_mma_supported(const arb_attn_params &p) {
     return p.dtype == ARB_BF16 && p.head_dim == kD && g >= kDecodeMmaMinGroup && g <= 8 && encode_tiled_fn() != nullptr;
 }
 
-arb_status launch_decode_mma(Ctx *ctx, const arb_attn_params &p, const void *q, const void *k_pages,
-                             const void *v_pages, const int32_t *block_table, const int32_t *seq_lens,
-                             const int32_t *q_lens, void *out, cudaStream_t stream) {
+namespace {
+
+// both caches: e4m3 selects the E4M3 form, whose keys are k_scale * code and values v_scale * code
+arb_status launch_decode_tc(Ctx *ctx, const arb_attn_params &p, const void *q, const void *k_pages, const void *v_pages,
+                            bool e4m3, float k_scale, float v_scale, const int32_t *block_table, const int32_t *seq_lens,
+                            const int32_t *q_lens, void *out, cudaStream_t stream) {
     alignas(64) CUtensorMap km, vm;
-    if (!make_pool_map(&km, k_pages, p) || !make_pool_map(&vm, v_pages, p)) return ARB_ERR_CUDA;
+    if (!make_pool_map(&km, k_pages, p, e4m3) || !make_pool_map(&vm, v_pages, p, e4m3)) return ARB_ERR_CUDA;
     const int g = p.num_q_heads / p.num_kv_heads;
     const int gp = (g + 3) / 4 * 4;
     const size_t slots = (size_t)p.batch * p.num_kv_heads + (size_t)ctx->num_sms * kCtasPerSm;
@@ -875,7 +983,8 @@ arb_status launch_decode_mma(Ctx *ctx, const arb_attn_params &p, const void *q, 
     // is what finishes it soonest.
     a.small_ctas = (p.flags & ARB_ATTN_OVERLAP_PREVIOUS) ? (ctx->num_sms + 1) / 2 : ctx->num_sms;
     const float scale = p.softmax_scale > 0.f ? p.softmax_scale : 1.0f / sqrtf((float)p.head_dim);
-    a.scale_log2 = scale * 1.4426950408889634f;
+    a.scale_log2 = scale * k_scale * 1.4426950408889634f;
+    a.v_scale = v_scale;
     const bool overlap = (p.flags & ARB_ATTN_OVERLAP_PREVIOUS) != 0;
     CombineArgs ca;
     ca.seq_lens = seq_lens;
@@ -892,17 +1001,41 @@ arb_status launch_decode_mma(Ctx *ctx, const arb_attn_params &p, const void *q, 
     ca.gen = gen;
     ca.done_gen = a.done_gen;
     ca.exit_count = ctx->rot + (size_t)kRotSets * kRotCounters + set;
-    switch (g) {
-        case 1: return launch_one<1>(ctx, a, ca, km, vm, overlap, stream);
-        case 2: return launch_one<2>(ctx, a, ca, km, vm, overlap, stream);
-        case 3: return launch_one<3>(ctx, a, ca, km, vm, overlap, stream);
-        case 4: return launch_one<4>(ctx, a, ca, km, vm, overlap, stream);
-        case 5: return launch_one<5>(ctx, a, ca, km, vm, overlap, stream);
-        case 6: return launch_one<6>(ctx, a, ca, km, vm, overlap, stream);
-        case 7: return launch_one<7>(ctx, a, ca, km, vm, overlap, stream);
-        case 8: return launch_one<8>(ctx, a, ca, km, vm, overlap, stream);
+    switch (e4m3 ? g + 8 : g) {
+        case 1: return launch_one<1, false>(ctx, a, ca, km, vm, overlap, stream);
+        case 2: return launch_one<2, false>(ctx, a, ca, km, vm, overlap, stream);
+        case 3: return launch_one<3, false>(ctx, a, ca, km, vm, overlap, stream);
+        case 4: return launch_one<4, false>(ctx, a, ca, km, vm, overlap, stream);
+        case 5: return launch_one<5, false>(ctx, a, ca, km, vm, overlap, stream);
+        case 6: return launch_one<6, false>(ctx, a, ca, km, vm, overlap, stream);
+        case 7: return launch_one<7, false>(ctx, a, ca, km, vm, overlap, stream);
+        case 8: return launch_one<8, false>(ctx, a, ca, km, vm, overlap, stream);
+        case 9: return launch_one<1, true>(ctx, a, ca, km, vm, overlap, stream);
+        case 10: return launch_one<2, true>(ctx, a, ca, km, vm, overlap, stream);
+        case 11: return launch_one<3, true>(ctx, a, ca, km, vm, overlap, stream);
+        case 12: return launch_one<4, true>(ctx, a, ca, km, vm, overlap, stream);
+        case 13: return launch_one<5, true>(ctx, a, ca, km, vm, overlap, stream);
+        case 14: return launch_one<6, true>(ctx, a, ca, km, vm, overlap, stream);
+        case 15: return launch_one<7, true>(ctx, a, ca, km, vm, overlap, stream);
+        case 16: return launch_one<8, true>(ctx, a, ca, km, vm, overlap, stream);
         default: return ARB_ERR_UNSUPPORTED;
     }
+}
+
+}  // namespace
+
+arb_status launch_decode_mma(Ctx *ctx, const arb_attn_params &p, const void *q, const void *k_pages,
+                             const void *v_pages, const int32_t *block_table, const int32_t *seq_lens,
+                             const int32_t *q_lens, void *out, cudaStream_t stream) {
+    return launch_decode_tc(ctx, p, q, k_pages, v_pages, false, 1.0f, 1.0f, block_table, seq_lens, q_lens, out, stream);
+}
+
+arb_status launch_decode_e4m3(Ctx *ctx, const arb_attn_params &p, const void *q, const void *k_pages,
+                              const void *v_pages, float k_scale, float v_scale, const int32_t *block_table,
+                              const int32_t *seq_lens, const int32_t *q_lens, void *out, cudaStream_t stream) {
+    const int g = p.num_q_heads / p.num_kv_heads;
+    if (g > 8 || encode_tiled_fn() == nullptr) return ARB_ERR_UNSUPPORTED;
+    return launch_decode_tc(ctx, p, q, k_pages, v_pages, true, k_scale, v_scale, block_table, seq_lens, q_lens, out, stream);
 }
 
 }  // namespace arb

@@ -6,9 +6,10 @@
 
 Headline workload: the draft-shaped decode configuration (batch 8, 12 query / 2 KV heads, head_dim
 128, bf16, page 16, prefix lengths uniform in [1024, 8192], q_len 1).  One step is one generated
-token's attention for the whole batch across 16 layers, each with its own KV pool, i.e. 16
-arb_attn calls (a decode kernel with the prepass fused in, and a small combine kernel behind it).  The pools together
-(about 600 MB) are several times the L2, so every call streams its KV from HBM.  The rows of the
+token's attention for the whole batch across 28 layers (the depth of the 1.5B-parameter model family that
+has this head geometry), each with its own KV pool, i.e. 28 arb_attn calls (a decode kernel with the
+prepass fused in, and a small combine kernel behind it).  The pools together (about 950 MB) are several
+times the L2, so every call streams its KV from HBM.  The rows of the
 path that this workload does not contain (step-chunk attention, router head, rollback: there is no
 step boundary inside one decode token) are timed on the step-scoring workload and reported in
 "step_scoring" on the same line.
@@ -35,7 +36,7 @@ sys.path.insert(0, str(ROOT))
 from paper_2512_05033_b200 import workloads as wl  # noqa: E402
 
 METRIC = "attention KV HBM GB/s (% of B200 peak) and draft steps scored+routed/sec"
-LAYERS = 16
+LAYERS = 28   # attention layers of one decode token of the draft-shaped model
 NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
 
@@ -322,37 +323,56 @@ def run_e2e(ctx, work: DecodeWorkload, steps: int, world: int):
     """Same step through arb_attn_host: per call, q / block table / lengths come from pinned host
     memory and out goes back to pinned host memory, all inside the timed region.  The KV cache stays
     resident: it is state of the generation loop, not an input of a step."""
+    from paper_2512_05033_b200 import binding
     i = work.inp
     qh = i.q.cpu().pin_memory()
     bth = i.block_table.cpu().pin_memory()
     slh = i.seq_lens.cpu().pin_memory()
     qlh = i.q_lens.cpu().pin_memory()
-    outh = torch.empty_like(qh).pin_memory()
+    outs = [torch.empty_like(qh).pin_memory() for _ in work.pools]   # one result per layer
 
-    params = ctx.params_for(qh, i.k_pages, bth, 1)
     sp = torch.cuda.current_stream().cuda_stream
-    ptrs = [(k.data_ptr(), v.data_ptr()) for k, v in work.pools]
-    host = (bth.data_ptr(), slh.data_ptr(), qlh.data_ptr(), outh.data_ptr())
+    ptrs = [(k.data_ptr(), v.data_ptr(), o.data_ptr()) for (k, v), o in zip(work.pools, outs)]
+    host = (qh.data_ptr(), bth.data_ptr(), slh.data_ptr(), qlh.data_ptr())
 
-    def step():
-        for kp, vp in ptrs:
-            st = ctx.attn_host_raw(params, qh.data_ptr(), kp, vp, host[0], host[1], host[2], host[3], sp)
-            if st != 0:
-                raise RuntimeError(f"arb_attn_host failed with status {st}")
+    def make(pipelined: bool, flags: int):
+        params = ctx.params_for(qh, i.k_pages, bth, 1, flags=flags)
+        call = ctx.attn_host_begin_raw if pipelined else ctx.attn_host_raw
 
-    for _ in range(3):
-        step()
-    torch.cuda.synchronize()
-    t0 = time.perf_counter()
-    for _ in range(steps):
-        step()
-    torch.cuda.synchronize()
-    dt = (time.perf_counter() - t0) / steps
+        def step():
+            for kp, vp, op in ptrs:
+                st = call(params, host[0], kp, vp, host[1], host[2], host[3], op, sp)
+                if st != 0:
+                    raise RuntimeError(f"arb_attn_host call failed with status {st}")
+            if pipelined:
+                ctx.attn_host_wait()   # the step's results are in host memory from here on
+        return step
+
+    def timed(step):
+        for _ in range(3):
+            step()
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        for _ in range(steps):
+            step()
+        torch.cuda.synchronize()
+        return (time.perf_counter() - t0) / steps
+
+    dt = timed(make(True, 0))
+    dt_flag = timed(make(True, binding.ATTN_OVERLAP_PREVIOUS))
+    dt_sync = timed(make(False, 0))
+    gbs = lambda t: round(world * work.bytes["kv"] * work.layers / t / 1e9, 1)  # noqa: E731
     h2d = (qh.numel() * qh.element_size() + bth.numel() * 4 + slh.numel() * 4 + qlh.numel() * 4) * work.layers
-    d2h = outh.numel() * outh.element_size() * work.layers
-    return {"value": round(world * work.bytes["kv"] * work.layers / dt / 1e9, 1), "unit": "GB/s",
+    d2h = qh.numel() * qh.element_size() * work.layers
+    return {"value": gbs(dt), "unit": "GB/s",
             "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": round(dt * 1e3, 4),
-            "note": "arb_attn_host per layer call; KV cache resident; measured on rank 0, scaled by ranks"}
+            "flagged_calls": {"value": gbs(dt_flag), "ms_per_step": round(dt_flag * 1e3, 4),
+                              "note": "ARB_ATTN_OVERLAP_PREVIOUS buys nothing here: each call's kernels wait for "
+                                      "their own inputs' copy, and a flagged small call takes half the CTAs"},
+            "one_call_at_a_time": {"value": gbs(dt_sync), "ms_per_step": round(dt_sync * 1e3, 4),
+                                   "note": "arb_attn_host: each layer call returns with its result on the host"},
+            "note": "arb_attn_host_begin per layer call and one arb_attn_host_wait per "
+                    "step; host clock around the steps; KV cache resident; measured on rank 0, scaled by ranks"}
 
 
 def run_target_decode(ctx, dev, peak):
@@ -674,7 +694,7 @@ def main():
                     help="do not let a layer call start under the tail of the previous one")
     ap.add_argument("--workload", choices=("draft", "target"), default="draft",
                     help="decode workload of the timed loop (the headline is draft)")
-    ap.add_argument("--layers", type=int, default=0, help="KV pools rotated per step (default 16 draft, 2 target)")
+    ap.add_argument("--layers", type=int, default=0, help="KV pools rotated per step (default 28 draft, 2 target)")
     ap.add_argument("--profile-scoring", action="store_true",
                     help="for runs under ncu: a few passes of the step-scoring workload (chunk attention, route, "
                          "rollback) and nothing else")

@@ -180,6 +180,29 @@ arb_status arb_attn_host(arb_ctx *ctx, const arb_attn_params *params, const void
                          const int32_t *q_lens_host, void *out_host, arb_stream_t stream);
 
 /*
+ * arb_attn_host in two halves, for callers that issue several host-side calls before they need a
+ * result (the layers of one decode token, the caches of one round of Algorithm 1).
+ *
+ * arb_attn_host_begin takes the arguments of arb_attn_host.  Before it returns it has copied the
+ * four input arrays into staging owned by ctx (the caller may overwrite them at once) and has
+ * enqueued: the inputs' copy to the device on a copy stream of ctx, the arb_attn kernels on
+ * `stream` (in call order, so cache updates enqueued on `stream` between two calls are seen by the
+ * later one), and the copy of the result into out_host on a second copy stream of ctx.  out_host
+ * (page-locked memory keeps that copy asynchronous) must not be read before arb_attn_host_wait has
+ * returned ARB_OK; synchronising `stream` alone does not cover the copy back.  Up to 8 calls are in
+ * flight per ctx; a further call first waits for the oldest.  Staging grows here when a call needs
+ * more (allocation, as in arb_attn_host).  Not for a stream that is being captured into a graph.
+ *
+ * arb_attn_host_wait blocks until every call begun on ctx has delivered its result.
+ * Errors: as arb_attn_host; after an error nothing of the failed call is left in flight.
+ */
+arb_status arb_attn_host_begin(arb_ctx *ctx, const arb_attn_params *params, const void *q_host,
+                               const void *k_pages, const void *v_pages,
+                               const int32_t *block_table_host, const int32_t *seq_lens_host,
+                               const int32_t *q_lens_host, void *out_host, arb_stream_t stream);
+arb_status arb_attn_host_wait(arb_ctx *ctx);
+
+/*
  * Decode attention (q_len = 1 for every sequence) for callers that must not allocate.
  *
  * The paper has no counterpart to this call; it exists for the way the library gets embedded.

@@ -32,6 +32,7 @@ MAX_CLASSES = 16
 
 # every symbol include/arb.h declares
 EXPORTS = ("arb_create", "arb_destroy", "arb_attn_workspace_bytes", "arb_attn", "arb_attn_host",
+           "arb_attn_host_begin", "arb_attn_host_wait",
            "arb_attn_decode_static",
            "arb_route", "arb_rollback", "arb_policy", "arb_route_classes", "arb_kv_append", "arb_kv_append_e4m3", "arb_attn_decode_e4m3", "arb_phase_lens", "arb_spearman",
            "arb_poll_status", "arb_launch_count", "arb_status_string")
@@ -56,6 +57,10 @@ lib.arb_attn.restype = ctypes.c_int
 lib.arb_attn.argtypes = [_vp, ctypes.POINTER(AttnParams), _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp]
 lib.arb_attn_host.restype = ctypes.c_int
 lib.arb_attn_host.argtypes = [_vp, ctypes.POINTER(AttnParams), _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp]
+lib.arb_attn_host_begin.restype = ctypes.c_int
+lib.arb_attn_host_begin.argtypes = [_vp, ctypes.POINTER(AttnParams), _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp]
+lib.arb_attn_host_wait.restype = ctypes.c_int
+lib.arb_attn_host_wait.argtypes = [_vp]
 lib.arb_attn_decode_static.restype = ctypes.c_int
 lib.arb_attn_decode_static.argtypes = [ctypes.POINTER(AttnParams), _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp]
 lib.arb_route.restype = ctypes.c_int
@@ -214,6 +219,30 @@ class Context:
     def attn_host_raw(self, p: AttnParams, q_ptr, k_ptr, v_ptr, bt_ptr, sl_ptr, ql_ptr, out_ptr, stream_ptr) -> int:
         """Pointer-level form of attn_host (host pointers for q, block table, lengths and out); returns the arb_status."""
         return lib.arb_attn_host(self._h, ctypes.byref(p), q_ptr, k_ptr, v_ptr, bt_ptr, sl_ptr, ql_ptr, out_ptr, stream_ptr)
+
+    def attn_host_begin(self, q_host, k_pages, v_pages, block_table_host, seq_lens_host, q_lens_host, max_q_len: int,
+                        out_host, softmax_scale: float = 0.0, flags: int = 0, stream=None):
+        """First half of the pipelined host call: enqueues copies and kernels and returns; out_host (pinned) holds
+        the result once attn_host_wait() has returned."""
+        for t in (q_host, block_table_host, seq_lens_host, q_lens_host, out_host):
+            if t.is_cuda or not t.is_contiguous():
+                raise ValueError("host tensors must be contiguous CPU tensors")
+        p = self.params_for(q_host, k_pages, block_table_host, max_q_len, softmax_scale)
+        p.flags = flags
+        st = lib.arb_attn_host_begin(self._h, ctypes.byref(p), q_host.data_ptr(), _dev(k_pages, "k_pages"),
+                                     _dev(v_pages, "v_pages"), block_table_host.data_ptr(), seq_lens_host.data_ptr(),
+                                     q_lens_host.data_ptr(), out_host.data_ptr(), _stream_ptr(stream))
+        _check(st, "arb_attn_host_begin")
+        return out_host
+
+    def attn_host_begin_raw(self, p: AttnParams, q_ptr, k_ptr, v_ptr, bt_ptr, sl_ptr, ql_ptr, out_ptr, stream_ptr) -> int:
+        """Pointer-level form of attn_host_begin; returns the arb_status."""
+        return lib.arb_attn_host_begin(self._h, ctypes.byref(p), q_ptr, k_ptr, v_ptr, bt_ptr, sl_ptr, ql_ptr, out_ptr,
+                                       stream_ptr)
+
+    def attn_host_wait(self):
+        """Blocks until every attn_host_begin of this context has delivered its result."""
+        _check(lib.arb_attn_host_wait(self._h), "arb_attn_host_wait")
 
     # -- arb_route ----------------------------------------------------------------------------
     def route(self, hidden, w, b: float, tau: float, scores=None, decisions=None, stream=None):

@@ -44,6 +44,51 @@ struct DeviceGuard {
 
 }  // namespace
 
+namespace {
+
+bool pipe_setup(Ctx *c) {
+    if (c->pipe_ready) return true;
+    bool ok = cudaStreamCreateWithFlags(&c->in_stream, cudaStreamNonBlocking) == cudaSuccess;
+    ok = ok && cudaStreamCreateWithFlags(&c->out_stream, cudaStreamNonBlocking) == cudaSuccess;
+    for (int i = 0; ok && i < kHostSlots; ++i) {
+        HostSlot &h = c->slots[i];
+        ok = cudaEventCreateWithFlags(&h.in_done, cudaEventDisableTiming) == cudaSuccess &&
+             cudaEventCreateWithFlags(&h.kernels_done, cudaEventDisableTiming) == cudaSuccess &&
+             cudaEventCreateWithFlags(&h.out_done, cudaEventDisableTiming) == cudaSuccess;
+    }
+    if (!ok) cudaGetLastError();
+    c->pipe_ready = ok;
+    return ok;
+}
+
+// Waits for every call in flight; the slots become free.
+arb_status pipe_drain(Ctx *c) {
+    arb_status st = ARB_OK;
+    for (int i = 0; i < kHostSlots; ++i) {
+        HostSlot &h = c->slots[i];
+        if (!h.busy) continue;
+        if (cudaEventSynchronize(h.out_done) != cudaSuccess) st = ARB_ERR_CUDA;
+        h.busy = false;
+    }
+    return st;
+}
+
+void pipe_teardown(Ctx *c) {
+    if (c->pipe_ready) pipe_drain(c);
+    for (int i = 0; i < kHostSlots; ++i) {
+        HostSlot &h = c->slots[i];
+        if (h.in_done) cudaEventDestroy(h.in_done);
+        if (h.kernels_done) cudaEventDestroy(h.kernels_done);
+        if (h.out_done) cudaEventDestroy(h.out_done);
+        cudaFree(h.dev);
+        cudaFreeHost(h.host);
+    }
+    if (c->in_stream) cudaStreamDestroy(c->in_stream);
+    if (c->out_stream) cudaStreamDestroy(c->out_stream);
+}
+
+}  // namespace
+
 extern "C" {
 
 arb_status arb_create(arb_ctx **out, int device, size_t workspace_bytes) {
@@ -102,6 +147,7 @@ arb_status arb_destroy(arb_ctx *ctx) {
     cudaFree(c->chunk_ws);
     cudaFree(c->stage);
     cudaFreeHost(c->host_stage);
+    pipe_teardown(c);
     delete c;
     return ARB_OK;
 }
@@ -229,6 +275,99 @@ arb_status arb_attn_host(arb_ctx *ctx, const arb_attn_params *params, const void
     if (cudaMemcpyAsync(out_host, dout, q_bytes, cudaMemcpyDeviceToHost, s) != cudaSuccess) return ARB_ERR_CUDA;
     if (cudaStreamSynchronize(s) != cudaSuccess) return ARB_ERR_CUDA;
     return ARB_OK;
+}
+
+arb_status arb_attn_host_begin(arb_ctx *ctx, const arb_attn_params *params, const void *q_host, const void *k_pages,
+                               const void *v_pages, const int32_t *block_table_host, const int32_t *seq_lens_host,
+                               const int32_t *q_lens_host, void *out_host, arb_stream_t stream) {
+    if (ctx == nullptr) return ARB_ERR_INVALID_ARG;
+    arb_status st = check_params(params);
+    if (st != ARB_OK) return st;
+    if (!q_host || !out_host || !block_table_host || !seq_lens_host || !q_lens_host) return ARB_ERR_INVALID_ARG;
+    Ctx *c = reinterpret_cast<Ctx *>(ctx);
+    DeviceGuard guard(c->device);
+    if (!guard.ok) return ARB_ERR_CUDA;
+    if (!pipe_setup(c)) return ARB_ERR_CUDA;
+    cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+    const size_t esz = params->dtype == ARB_BF16 ? 2 : 4;
+    auto up = [](size_t x) { return (x + 255) & ~size_t(255); };
+    const size_t q_bytes = (size_t)params->total_q * params->num_q_heads * params->head_dim * esz;
+    const size_t bt_bytes = sizeof(int32_t) * (size_t)params->batch * params->max_pages_per_seq;
+    const size_t len_bytes = sizeof(int32_t) * (size_t)params->batch;
+    const size_t in_bytes = up(q_bytes) + up(bt_bytes) + 2 * up(len_bytes);
+    const size_t need = up(q_bytes) + in_bytes;
+
+    HostSlot &h = c->slots[c->next_slot];
+    if (h.busy) {  // the ring is full: the oldest call has to finish first
+        if (cudaEventSynchronize(h.out_done) != cudaSuccess) return ARB_ERR_CUDA;
+        h.busy = false;
+    }
+    if (need > h.dev_bytes) {  // the slot is idle, so nothing on the device still uses its buffers
+        cudaFree(h.dev);
+        h.dev = nullptr;
+        h.dev_bytes = 0;
+        if (cudaMalloc(&h.dev, need) != cudaSuccess) {
+            cudaGetLastError();
+            return ARB_ERR_CUDA;
+        }
+        h.dev_bytes = need;
+    }
+    if (in_bytes > h.host_bytes) {
+        cudaFreeHost(h.host);
+        h.host = nullptr;
+        h.host_bytes = 0;
+        if (cudaHostAlloc(&h.host, in_bytes, cudaHostAllocDefault) != cudaSuccess) {
+            cudaGetLastError();
+            return ARB_ERR_CUDA;
+        }
+        h.host_bytes = in_bytes;
+    }
+    char *dout = h.dev, *dq = dout + up(q_bytes), *dbt = dq + up(q_bytes);
+    char *dsl = dbt + up(bt_bytes), *dql = dsl + up(len_bytes);
+    char *hq = h.host, *hbt = hq + up(q_bytes), *hsl = hbt + up(bt_bytes), *hql = hsl + up(len_bytes);
+    memcpy(hq, q_host, q_bytes);
+    memcpy(hbt, block_table_host, bt_bytes);
+    memcpy(hsl, seq_lens_host, len_bytes);
+    memcpy(hql, q_lens_host, len_bytes);
+    // inputs in on one copy stream, kernels on the caller's stream, result out on the other copy stream:
+    // the copies of neighbouring calls run beside the kernels instead of between them
+    if (cudaMemcpyAsync(dq, hq, in_bytes, cudaMemcpyHostToDevice, c->in_stream) != cudaSuccess ||
+        cudaEventRecord(h.in_done, c->in_stream) != cudaSuccess) {
+        cudaStreamSynchronize(c->in_stream);
+        cudaGetLastError();
+        return ARB_ERR_CUDA;
+    }
+    if (cudaStreamWaitEvent(s, h.in_done, 0) == cudaSuccess)
+        st = arb_attn(ctx, params, dq, k_pages, v_pages, reinterpret_cast<int32_t *>(dbt),
+                      reinterpret_cast<int32_t *>(dsl), reinterpret_cast<int32_t *>(dql), dout, stream);
+    else
+        st = ARB_ERR_CUDA;
+    if (st != ARB_OK) {  // nothing of this call may stay in flight on a slot that is not marked busy
+        cudaStreamSynchronize(c->in_stream);
+        cudaGetLastError();
+        return st;
+    }
+    bool ok = cudaEventRecord(h.kernels_done, s) == cudaSuccess;
+    ok = ok && cudaStreamWaitEvent(c->out_stream, h.kernels_done, 0) == cudaSuccess;
+    ok = ok && cudaMemcpyAsync(out_host, dout, q_bytes, cudaMemcpyDeviceToHost, c->out_stream) == cudaSuccess;
+    ok = ok && cudaEventRecord(h.out_done, c->out_stream) == cudaSuccess;
+    if (!ok) {
+        cudaStreamSynchronize(s);
+        cudaStreamSynchronize(c->out_stream);
+        cudaGetLastError();
+        return ARB_ERR_CUDA;
+    }
+    h.busy = true;
+    c->next_slot = (c->next_slot + 1) % kHostSlots;
+    return ARB_OK;
+}
+
+arb_status arb_attn_host_wait(arb_ctx *ctx) {
+    if (ctx == nullptr) return ARB_ERR_INVALID_ARG;
+    Ctx *c = reinterpret_cast<Ctx *>(ctx);
+    DeviceGuard guard(c->device);
+    if (!guard.ok) return ARB_ERR_CUDA;
+    return pipe_drain(c);
 }
 
 arb_status arb_route(arb_ctx *ctx, int32_t dtype, int32_t n_steps, int32_t hidden_dim, const void *hidden,

@@ -19,6 +19,19 @@ constexpr long long kWaitCycles = 1ll << 31;  // bound of every mbarrier wait (a
 // ---------------------------------------------------------------------------------------------
 // Host-side context
 // ---------------------------------------------------------------------------------------------
+// One call of the pipelined host entry points in flight: its staging on both sides and the events that order its
+// three parts (inputs in, kernels, result out) across the copy streams and the caller's stream.
+struct HostSlot {
+    char *dev = nullptr;     // [out | q | block table | seq_lens | q_lens]
+    size_t dev_bytes = 0;
+    char *host = nullptr;    // page-locked, [q | block table | seq_lens | q_lens]
+    size_t host_bytes = 0;
+    cudaEvent_t in_done = nullptr, kernels_done = nullptr, out_done = nullptr;
+    bool busy = false;
+};
+
+constexpr int kHostSlots = 8;
+
 struct Ctx {
     int device = 0;
     int num_sms = 0;
@@ -33,6 +46,11 @@ struct Ctx {
     size_t stage_bytes = 0;
     char *host_stage = nullptr;   // page-locked gather buffer of the *_host entry points
     size_t host_stage_bytes = 0;
+    // pipelined host calls: a ring of slots and one copy stream per direction, created at the first such call
+    HostSlot slots[kHostSlots];
+    int next_slot = 0;
+    cudaStream_t in_stream = nullptr, out_stream = nullptr;
+    bool pipe_ready = false;
     // workspace rotation of the tensor-core decode kernel: kRotSets counter arrays, one exit counter
     // per set and the generation of the newest completed call, all in one allocation
     int *rot = nullptr;

@@ -241,6 +241,63 @@ def test_host_buffer_entry_point():
     assert torch.equal(out, out2)
 
 
+def test_pipelined_host_calls():
+    """arb_attn_host_begin / arb_attn_host_wait: more calls in flight than the ring has slots, shapes that change from
+    call to call (staging grows), inputs overwritten as soon as begin has returned; every result equals the one-shot
+    host call bit for bit and the oracle within tolerance."""
+    c = H.ctx()
+    shapes = [([500, 90, 2000], [1, 4, 1]), ([33], [1]), ([4000, 4100, 777, 12, 640], [1, 1, 1, 1, 1]),
+              ([300, 200], [16, 128])]
+    cases, outs, expect = [], [], []
+    for i in range(19):
+        sl, ql = shapes[i % len(shapes)]
+        inp = wl.small_attn_case(len(sl), 12, 2, 128, BF, sl, ql, seed=700 + i)
+        kp, vp = inp.k_pages.cuda(), inp.v_pages.cuda()
+        expect.append(c.attn_host(inp.q.pin_memory(), kp, vp, inp.block_table.pin_memory(), inp.seq_lens.pin_memory(),
+                                  inp.q_lens.pin_memory(), max(ql)).clone())
+        cases.append((inp, kp, vp, max(ql)))
+    for inp, kp, vp, mq in cases:
+        q, bt, sl, ql = inp.q.clone(), inp.block_table.clone(), inp.seq_lens.clone(), inp.q_lens.clone()
+        out = torch.full_like(inp.q, float("nan")).pin_memory()
+        c.attn_host_begin(q, kp, vp, bt, sl, ql, mq, out)
+        q.fill_(float("nan")); bt.fill_(-1); sl.fill_(-1); ql.fill_(-1)   # the library has its own copy by now
+        outs.append(out)
+    c.attn_host_wait()
+    c.attn_host_wait()                                                     # nothing in flight: returns at once
+    assert c.poll_status() == 0
+    for i, (out, exp) in enumerate(zip(outs, expect)):
+        assert torch.equal(out, exp), i
+    for i in (0, 3, 18):
+        ref, _ = H.oracle_attn(cases[i][0])
+        H.assert_close(outs[i].double().numpy(), ref, BF)
+
+
+def test_pipelined_host_calls_see_cache_updates_in_stream_order():
+    """Kernels of begun calls run on the caller's stream in call order: an append enqueued between two calls is
+    seen by the second and not by the first."""
+    inp = wl.small_attn_case(2, 12, 2, 128, BF, [300, 45], [1, 1], seed=731).to("cuda")
+    c = H.ctx()
+    host = [t.cpu().pin_memory() for t in (inp.q, inp.block_table, inp.seq_lens, inp.q_lens)]
+    out_a = torch.empty_like(host[0]).pin_memory()
+    out_b = torch.empty_like(host[0]).pin_memory()
+    g = torch.Generator().manual_seed(732)
+    k_new = torch.randn(2, 2, 128, generator=g).to(BF).cuda()
+    v_new = torch.randn(2, 2, 128, generator=g).to(BF).cuda()
+    one = torch.ones(2, dtype=torch.int32, device="cuda")
+    lens_dev = inp.seq_lens.clone()
+    kp, vp = inp.k_pages.clone(), inp.v_pages.clone()
+    c.attn_host_begin(*host[:1], kp, vp, *host[1:], 1, out_a)
+    c.kv_append(k_new, v_new, inp.block_table, lens_dev, one, kp, vp)      # seq_lens += 1, new rows written
+    longer = (inp.seq_lens + 1).cpu().pin_memory()
+    c.attn_host_begin(host[0], kp, vp, host[1], longer, host[3], 1, out_b)
+    c.attn_host_wait()
+    before = c.attn(inp.q, inp.k_pages, inp.v_pages, inp.block_table, inp.seq_lens, inp.q_lens, 1)
+    after = c.attn(inp.q, kp, vp, inp.block_table, inp.seq_lens + 1, inp.q_lens, 1)
+    torch.cuda.synchronize()
+    assert torch.equal(out_a, before.cpu()) and torch.equal(out_b, after.cpu())
+    assert not torch.equal(out_a, out_b)
+
+
 def test_repeated_calls_reuse_the_workspace():
     """Arrival counters return to zero after every call: same answer five times in a row."""
     inp = wl.small_attn_case(2, 12, 2, 128, BF, [9000, 5000], [1, 1], seed=56)

@@ -21,9 +21,9 @@
 // exponentials bounded by 2^8 and nothing is touched.  K and V tiles are fetched page by page with
 // tiled TMA copies (one 16 x 64 box per page and half of head_dim, landing in the canonical swizzled
 // layout) into a two-stage ring.  Roles: warps 0-3 softmax and epilogue of row tile A, warps 4-7 of
-// row tile B, warp 8 TMA producer, warp 9 MMA issue and TMEM allocation.  Work items are handed out
-// dynamically, longest sequences first: the producer warp takes the next item from an atomic counter
-// and announces it to the other roles through a small queue in shared memory.  Every mbarrier wait
+// row tile B, warp 8 TMA producer of K, warp 10 of V, warp 9 MMA issue and TMEM allocation.  Work items are
+// handed out dynamically, longest sequences first: the K producer takes the next item from an atomic
+// counter and announces it to the other roles through a small queue in shared memory.  Every mbarrier wait
 // is bounded; TMEM is released on every path.
 #include <cuda.h>  // CUtensorMap and its enums only; the encoder is looked up at run time
 
@@ -39,8 +39,9 @@ constexpr int kBN = 128;          // keys per KV tile
 constexpr int kTilePages = kBN / kPage;
 constexpr int kStages = 2;
 constexpr int kSoftmaxThreads = 128;        // per row tile
-constexpr int kThreads = 2 * kSoftmaxThreads + 64;   // two softmax groups, TMA warp, MMA warp
-constexpr int kTmaWarp = 8, kMmaWarp = 9;
+constexpr int kThreads = 3 * kSoftmaxThreads;   // two softmax groups and a group of service warps; registers are
+                                                // handed out per 128 threads, so the third group's spare warps cost none
+constexpr int kTmaWarp = 8, kMmaWarp = 9, kVWarp = 10;   // warp 11 has no role
 constexpr int kHalfBytes = 128 * 128;      // [128 rows x 64 bf16]: one 128-byte-swizzled half tile
 constexpr int kTileBytes = 2 * kHalfBytes;  // [128 x 128] bf16
 constexpr int kBoxBytes = kPage * 128;      // one TMA box: 16 rows x 64 bf16
@@ -87,7 +88,7 @@ struct Bars {
     uint64_t p_full[2];          // P of row tile A / B is in TMEM (over S)
     uint64_t o_full[2];          // O += P V of row tile A / B has completed
     uint64_t item_full[kItemSlots];   // the producer warp has fetched the next work item
-    uint64_t item_empty[kItemSlots];  // the MMA thread and the softmax threads have read it
+    uint64_t item_empty[kItemSlots];  // the MMA thread, the V producer and the softmax threads have read it
     int item_id[kItemSlots];
     uint32_t tmem_base;
     int abort;
@@ -207,22 +208,30 @@ __device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&v)[16
 __device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
-// acc + lo + hi for a packed bf16 pair, in fp32 (mixed-precision FMA with 1.0: no unpacking)
-__device__ __forceinline__ float add_bf16x2(uint32_t w, float acc) {
-    asm("{\n\t.reg .b16 lo, hi, one;\n\t"
-        "mov.b32 {lo, hi}, %1;\n\t"
-        "mov.b16 one, 0x3f80;\n\t"
-        "fma.rn.f32.bf16 %0, lo, one, %0;\n\t"
-        "fma.rn.f32.bf16 %0, hi, one, %0;\n\t}"
-        : "+f"(acc)
-        : "r"(w));
-    return acc;
-}
-
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
     uint32_t r;
     asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
     return r;
+}
+
+// packed pairs of fp32 (one instruction for two lanes of arithmetic)
+__device__ __forceinline__ uint64_t pack_f32x2(float lo, float hi) {
+    uint64_t r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
+}
+__device__ __forceinline__ void unpack_f32x2(uint64_t v, float &lo, float &hi) {
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ uint64_t fma_f32x2(uint64_t a, uint64_t b, uint64_t c) {
+    uint64_t d;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+    return d;
+}
+__device__ __forceinline__ uint64_t add_f32x2(uint64_t a, uint64_t b) {
+    uint64_t d;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
 }
 
 __device__ __forceinline__ float max3(float a, float b, float c) {
@@ -410,7 +419,7 @@ chunk_mma_kernel(const MmaArgs a, const __grid_constant__ CUtensorMap k_map, con
         mbar_init(&bars->o_full[1], 1);
         for (int i = 0; i < kItemSlots; ++i) {
             mbar_init(&bars->item_full[i], 1);
-            mbar_init(&bars->item_empty[i], 1 + 2 * kSoftmaxThreads);
+            mbar_init(&bars->item_empty[i], 2 + 2 * kSoftmaxThreads);   // MMA thread, V warp, softmax threads
         }
         bars->abort = 0;
         mbar_fence_init();
@@ -426,76 +435,80 @@ chunk_mma_kernel(const MmaArgs a, const __grid_constant__ CUtensorMap k_map, con
     const uint32_t tmem = bars->tmem_base;
     volatile int *abort = &bars->abort;
 
-    if (warp == kTmaWarp) {
-        // ===================================== TMA producer =========================================
+    if (warp == kTmaWarp || warp == kVWarp) {
+        // ================================= TMA producers: K warp, V warp ==========================
+        // One warp per operand: a tiled TMA copy is issued per (page, 64-dim half), sixteen to a tile, and one
+        // warp issues them one after the other (about 1500 cycles per tile), so K and V of a tile are in
+        // flight together only when two warps issue them.  The K warp also hands out the work: items come
+        // from an atomic counter (longest sequences first) and are announced to every other role, the V warp
+        // included, through a small queue in shared memory.  Both run ahead of the consumers as far as their
+        // two-stage rings allow.
+        const bool is_v = warp == kVWarp;
+        uint64_t *full = is_v ? bars->v_full : bars->k_full, *empty = is_v ? bars->v_empty : bars->k_empty;
+        char *ring = is_v ? v_s : k_s;
+        const CUtensorMap *map = is_v ? &v_map : &k_map;
+        const char *pool = is_v ? a.v_pool : a.k_pool;
         uint32_t it = 0;  // KV tiles issued so far
         Item w;
-        // Work items are handed out dynamically (an atomic counter, longest sequences first): this
-        // warp fetches the next item, announces it to the other roles through a small queue in
-        // shared memory and runs ahead of them as far as the K/V ring allows.
         for (uint32_t nq = 0;; ++nq) {
             const uint32_t slot = nq % kItemSlots, qpar = (nq / kItemSlots) & 1u;
             int item = total;
             if (lane == 0) {
-                if (mbar_wait(&bars->item_empty[slot], qpar ^ 1u, abort, a.status)) item = atomicAdd(a.work_counter, 1);
-                bars->item_id[slot] = item;
-                mbar_arrive(&bars->item_full[slot]);
+                if (!is_v) {
+                    if (mbar_wait(&bars->item_empty[slot], qpar ^ 1u, abort, a.status)) item = atomicAdd(a.work_counter, 1);
+                    bars->item_id[slot] = item;
+                    mbar_arrive(&bars->item_full[slot]);
+                } else if (mbar_wait(&bars->item_full[slot], qpar, abort, a.status)) {
+                    item = bars->item_id[slot];
+                    mbar_arrive(&bars->item_empty[slot]);
+                }
             }
             item = __shfl_sync(0xffffffffu, item, 0);
             if (!get_item<G>(item, total, pl, B, Hkv, a, w)) break;
-            // K and V tiles are asked into L2 kPrefetchTiles ahead of their load into the ring, so the
-            // ring (two tiles deep) only has to cover the L2 latency, not the DRAM latency
-            auto prefetch_tile = [&](int jt) {   // jt: tile of this item, 0-based
-                if (jt >= w.ntiles) return;
+            // Block-table entries are read one step before they are used (the tile's own pages one tile
+            // ahead, the pages to ask into L2 one tile before the request), so that no global-memory round
+            // trip sits between two tiles.  Lanes 0-7: the pages of a tile; -1 marks "no such page".
+            auto table_entry = [&](int jt) -> int {   // jt: tile of this item, 0-based
+                if (jt >= w.ntiles) return -1;
                 jt += w.t0;
                 const int np = min(kTilePages, (w.kv_len - jt * kBN + kPage - 1) / kPage);
-                const int pg = lane & 7;
-                if (lane < 16 && pg < np) {
-                    const int pf = a.block_table[(size_t)w.b * a.max_pages + jt * kTilePages + pg];
-                    if ((unsigned)pf < (unsigned)a.num_pages) {
-                        const char *src = (lane < 8 ? a.k_pool : a.v_pool) + ((size_t)pf * Hkv + w.kvh) * (kPage * kD * 2);
-                        asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(src), "r"(kPage * kD * 2) : "memory");
-                    }
+                return (lane < np) ? a.block_table[(size_t)w.b * a.max_pages + jt * kTilePages + lane] : -1;
+            };
+            // K and V tiles are asked into L2 kPrefetchTiles ahead of their load into the ring, so the
+            // ring (two tiles deep) only has to cover the L2 latency, not the DRAM latency
+            auto prefetch_pages = [&](int pf) {
+                if ((unsigned)pf < (unsigned)a.num_pages) {
+                    const char *src = pool + ((size_t)pf * Hkv + w.kvh) * (kPage * kD * 2);
+                    asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(src), "r"(kPage * kD * 2) : "memory");
                 }
             };
-            for (int jt = 0; jt < kPrefetchTiles; ++jt) prefetch_tile(jt);
+            for (int jt = 0; jt < kPrefetchTiles; ++jt) prefetch_pages(table_entry(jt));
+            int pf_next = table_entry(kPrefetchTiles), pid_next = table_entry(0);
             for (int j = 0; j < w.ntiles; ++j, ++it) {
                 const uint32_t s = it % kStages, par = (it / kStages) & 1u;
                 const int jg = w.t0 + j;   // tile of the sequence
                 const int npages = min(kTilePages, (w.kv_len - jg * kBN + kPage - 1) / kPage);
-                prefetch_tile(j + kPrefetchTiles);
-                int pid = 0;
-                if (lane < npages) {
-                    pid = a.block_table[(size_t)w.b * a.max_pages + jg * kTilePages + lane];
-                    if ((unsigned)pid >= (unsigned)a.num_pages) {
-                        atomicOr(a.status, (uint32_t)ARB_DEV_BAD_PAGE);
-                        pid = 0;
-                    }
+                int pid = pid_next;
+                const int pf = pf_next;
+                pid_next = table_entry(j + 1);
+                pf_next = table_entry(j + 1 + kPrefetchTiles);
+                prefetch_pages(pf);
+                if (lane < npages && (unsigned)pid >= (unsigned)a.num_pages) {
+                    atomicOr(a.status, (uint32_t)ARB_DEV_BAD_PAGE);
+                    pid = 0;
                 }
-                // lanes 0..15: (half, page) of K; the same lanes then issue V.  The K stage is free
-                // as soon as the first products of the tile before last have completed, the V stage
-                // only after its second products: two separate waits, in the order they are released.
+                // lanes 0..15: (half, page).  A K stage is free as soon as the first products of the tile
+                // before last have completed, a V stage only after its second products.
                 const int pg = lane & 7, half = (lane >> 3) & 1;
                 const int row = (__shfl_sync(0xffffffffu, pid, pg) * Hkv + w.kvh) * kPage;
                 bool ok = true;
-                if (lane == 0) ok = mbar_wait(&bars->k_empty[s], par ^ 1u, abort, a.status);
+                if (lane == 0) ok = mbar_wait(&empty[s], par ^ 1u, abort, a.status);
                 ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
                 if (ok) {
-                    if (lane == 0) mbar_arrive_expect_tx(&bars->k_full[s], (uint32_t)npages * 2u * kBoxBytes);
+                    if (lane == 0) mbar_arrive_expect_tx(&full[s], (uint32_t)npages * 2u * kBoxBytes);
                     __syncwarp();
                     if (lane < 16 && pg < npages)
-                        tma_box_load(k_s + s * kTileBytes + half * kHalfBytes + pg * kBoxBytes, &k_map, half * 64, row,
-                                     &bars->k_full[s]);
-                }
-                __syncwarp();
-                if (lane == 0) ok = mbar_wait(&bars->v_empty[s], par ^ 1u, abort, a.status);
-                ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
-                if (ok) {
-                    if (lane == 0) mbar_arrive_expect_tx(&bars->v_full[s], (uint32_t)npages * 2u * kBoxBytes);
-                    __syncwarp();
-                    if (lane < 16 && pg < npages)
-                        tma_box_load(v_s + s * kTileBytes + half * kHalfBytes + pg * kBoxBytes, &v_map, half * 64, row,
-                                     &bars->v_full[s]);
+                        tma_box_load(ring + s * kTileBytes + half * kHalfBytes + pg * kBoxBytes, map, half * 64, row, &full[s]);
                 }
                 __syncwarp();
             }
@@ -573,7 +586,7 @@ chunk_mma_kernel(const MmaArgs a, const __grid_constant__ CUtensorMap k_map, con
             }
         }
         __syncwarp();
-    } else {
+    } else if (warp < 2 * kSoftmaxThreads / 32) {
         // ================================ softmax and epilogue ====================================
         // two groups of 128 threads: group g owns row tile g; thread tg of a group owns TMEM lane tg
         const int grp = warp >> 2, tg = tid & (kSoftmaxThreads - 1);
@@ -662,25 +675,36 @@ chunk_mma_kernel(const MmaArgs a, const __grid_constant__ CUtensorMap k_map, con
                     }
                     tmem_wait_st();
                 }
-                // ---- P = exp2(scale * S - m), rounded to bf16 BEFORE it is summed, so the tensor
-                //      core's numerator and the fp32 denominator use the very same weights and the
-                //      result stays a true convex combination of V rows.  P overwrites S in place:
-                //      keys 32 c .. 32 c + 31 -> columns 16 c .. 16 c + 15 (all of S is in registers).
+                // ---- P = exp2(scale * S - m) for two keys per instruction where the hardware has a packed form
+                //      (fma.f32x2, add.f32x2; ex2 and the bf16 conversion have none).  The denominator sums
+                //      the fp32 weights, the tensor core the same weights rounded to bf16: the two differ by
+                //      independent relative errors of at most 2^-9 per key, which the sum averages out.
+                //      P overwrites S in place: keys 32 c .. 32 c + 31 -> columns 16 c .. 16 c + 15 (all
+                //      of S is in registers).
                 const float neg_m = (m_used == -INFINITY) ? 0.f : -m_used;
-                float l4[4] = {0.f, 0.f, 0.f, 0.f};
+                const uint64_t sc2 = pack_f32x2(a.scale_log2, a.scale_log2), nm2 = pack_f32x2(neg_m, neg_m);
+                uint64_t l2[4] = {0ull, 0ull, 0ull, 0ull};
 #pragma unroll
                 for (int c4 = 0; c4 < 4; ++c4) {
                     uint32_t pk[16];
 #pragma unroll
                     for (int k = 0; k < 16; ++k) {
-                        const float e0 = fast_exp2(fmaf(__uint_as_float(v[c4 * 32 + 2 * k]), a.scale_log2, neg_m));
-                        const float e1 = fast_exp2(fmaf(__uint_as_float(v[c4 * 32 + 2 * k + 1]), a.scale_log2, neg_m));
+                        const uint64_t t = fma_f32x2(pack_f32x2(__uint_as_float(v[c4 * 32 + 2 * k]),
+                                                                __uint_as_float(v[c4 * 32 + 2 * k + 1])), sc2, nm2);
+                        float t0, t1;
+                        unpack_f32x2(t, t0, t1);
+                        const float e0 = fast_exp2(t0), e1 = fast_exp2(t1);
                         pk[k] = pack_bf16(e0, e1);
-                        l4[k & 3] = add_bf16x2(pk[k], l4[k & 3]);
+                        l2[k & 3] = add_f32x2(l2[k & 3], pack_f32x2(e0, e1));
                     }
                     tmem_st16(s_tmem + c4 * 16, pk);
                 }
-                l_sum += (l4[0] + l4[1]) + (l4[2] + l4[3]);
+                {
+                    float x0, x1, y0, y1;
+                    unpack_f32x2(add_f32x2(l2[0], l2[1]), x0, x1);
+                    unpack_f32x2(add_f32x2(l2[2], l2[3]), y0, y1);
+                    l_sum += (x0 + x1) + (y0 + y1);
+                }
                 tmem_wait_st();
                 // ---- V rows past the last visible key of the item (stale slots, pages never loaded)
                 //      must not reach the tensor core, not even times zero

@@ -128,8 +128,9 @@ def test_large_chunk_peaked_and_stale_slots():
     assert bits == 0
     ref, _ = H.oracle_attn(inp)
     err = np.abs(clean - ref)
-    # The softmax weights enter the second product rounded to bf16 (relative 2^-9 each), the output is
-    # rounded to bf16 once more.  Gross bound for every element, exact bound on sampled rows.
+    # The softmax weights enter the second product rounded to bf16 (relative 2^-9 each) while the denominator
+    # sums them in fp32, and the output is rounded to bf16 once more.  Gross bound for every element, the bound
+    # that follows from this arithmetic on sampled rows.
     vmax = float(inp.v_pages.abs().max())
     assert (err <= 2.0 ** -8 * np.abs(ref) + 2.0 ** -9 * 2 * vmax).all(), err.max()
     from oracle import oracle
@@ -142,7 +143,7 @@ def test_large_chunk_peaked_and_stale_slots():
         o, p, _ = oracle.attn_row_probs(inp.q, inp.k_pages, inp.v_pages, inp.block_table[b], row, h, pos)
         bt = inp.block_table[b].numpy()
         v = np.stack([Vd[bt[j // wl.PAGE], h // 7, j % wl.PAGE] for j in range(pos + 1)])      # [keys, D]
-        bound = 2.0 ** -9 * (p[:, None] * np.abs(v - o[None, :])).sum(axis=0) + 2.0 ** -8 * np.abs(o) + 1e-3
+        bound = 2.0 ** -9 * (p[:, None] * np.abs(v)).sum(axis=0) + 2.0 ** -8 * np.abs(o) + 1e-3
         assert (np.abs(clean[row, h] - o) <= bound).all(), (b, i, h)
     k2, v2 = inp.k_pages.clone(), inp.v_pages.clone()
     for b in range(2):

@@ -2,7 +2,7 @@
 #include <cstring>
 #include <new>
 
-#include "arb_common.cuh"
+#include "arb_tma.cuh"
 
 using namespace arb;
 
@@ -148,6 +148,7 @@ arb_status arb_destroy(arb_ctx *ctx) {
     cudaFree(c->stage);
     cudaFreeHost(c->host_stage);
     pipe_teardown(c);
+    pool_map_cache_free(c);
     delete c;
     return ARB_OK;
 }

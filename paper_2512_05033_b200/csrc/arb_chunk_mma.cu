@@ -25,9 +25,7 @@
 // handed out dynamically, longest sequences first: the K producer takes the next item from an atomic
 // counter and announces it to the other roles through a small queue in shared memory.  Every mbarrier wait
 // is bounded; TMEM is released on every path.
-#include <cuda.h>  // CUtensorMap and its enums only; the encoder is looked up at run time
-
-#include "arb_common.cuh"
+#include "arb_tma.cuh"
 
 namespace arb {
 
@@ -859,38 +857,6 @@ chunk_combine_kernel(const MmaArgs a) {
     }
 }
 
-typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
-                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
-                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-EncodeTiledFn encode_tiled_fn() {
-    static EncodeTiledFn fn = nullptr;
-    static bool tried = false;
-    if (!tried) {
-        tried = true;
-        void *p = nullptr;
-        cudaDriverEntryPointQueryResult qres;
-        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) == cudaSuccess &&
-            qres == cudaDriverEntryPointSuccess)
-            fn = reinterpret_cast<EncodeTiledFn>(p);
-        cudaGetLastError();
-    }
-    return fn;
-}
-
-// 2-D view of a page pool: rows = (page, kv head, slot), 128 bf16 columns; box = one page-head, 64 columns
-bool make_pool_map(CUtensorMap *map, const void *pool, const arb_attn_params &p) {
-    EncodeTiledFn fn = encode_tiled_fn();
-    if (!fn) return false;
-    const cuuint64_t dims[2] = {(cuuint64_t)kD, (cuuint64_t)p.num_pages * p.num_kv_heads * kPage};
-    const cuuint64_t strides[1] = {(cuuint64_t)kD * 2};
-    const cuuint32_t box[2] = {64, (cuuint32_t)kPage};
-    const cuuint32_t estr[2] = {1, 1};
-    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(pool), dims, strides, box, estr,
-              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
-              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
-}
-
 template <int G>
 arb_status launch_one(Ctx *ctx, const MmaArgs &a, const CUtensorMap &km, const CUtensorMap &vm, int max_items,
                       cudaStream_t stream) {
@@ -921,14 +887,16 @@ arb_status launch_one(Ctx *ctx, const MmaArgs &a, const CUtensorMap &km, const C
 bool chunk_mma_supported(const arb_attn_params &p) {
     const int g = p.num_q_heads / p.num_kv_heads;
     return p.dtype == ARB_BF16 && p.head_dim == kD && p.max_q_len >= 2 && p.max_q_len * g >= kChunkMmaMinRows &&
-           encode_tiled_fn() != nullptr;
+           tma_available();
 }
 
 arb_status launch_chunk_mma(Ctx *ctx, const arb_attn_params &p, const void *q, const void *k_pages,
                             const void *v_pages, const int32_t *block_table, const int32_t *seq_lens,
                             const int32_t *q_lens, void *out, cudaStream_t stream) {
     alignas(64) CUtensorMap km, vm;
-    if (!make_pool_map(&km, k_pages, p) || !make_pool_map(&vm, v_pages, p)) return ARB_ERR_CUDA;
+    if (!pool_map(ctx, &km, k_pages, p.num_pages, p.num_kv_heads, false) ||
+        !pool_map(ctx, &vm, v_pages, p.num_pages, p.num_kv_heads, false))
+        return ARB_ERR_CUDA;
     MmaArgs a;
     a.q = static_cast<const char *>(q);
     a.k_pool = static_cast<const char *>(k_pages);

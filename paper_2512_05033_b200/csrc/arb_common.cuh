@@ -51,6 +51,8 @@ struct Ctx {
     int next_slot = 0;
     cudaStream_t in_stream = nullptr, out_stream = nullptr;
     bool pipe_ready = false;
+    void *map_cache = nullptr;      // tensor maps of the KV pools seen so far (arb_tma.cu)
+    unsigned map_evictions = 0;
     // workspace rotation of the tensor-core decode kernel: kRotSets counter arrays, one exit counter
     // per set and the generation of the newest completed call, all in one allocation
     int *rot = nullptr;

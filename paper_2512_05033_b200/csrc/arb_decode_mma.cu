@@ -39,9 +39,7 @@
 //     fragments of two n-tiles, the even and the odd dimensions of a 16-dimension group, so a thread ends up
 //     owning four consecutive output dimensions per group;
 //   - the key scale is folded into the softmax scale, the value scale into the segment result.
-#include <cuda.h>  // CUtensorMap and its enums only; the encoder is looked up at run time
-
-#include "arb_common.cuh"
+#include "arb_tma.cuh"
 
 namespace arb {
 
@@ -850,38 +848,6 @@ decode_combine_kernel(const CombineArgs a) {
     }
 }
 
-typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
-                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
-                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-EncodeTiledFn encode_tiled_fn() {
-    static EncodeTiledFn fn = nullptr;
-    static bool tried = false;
-    if (!tried) {
-        tried = true;
-        void *p = nullptr;
-        cudaDriverEntryPointQueryResult qres;
-        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) == cudaSuccess &&
-            qres == cudaDriverEntryPointSuccess)
-            fn = reinterpret_cast<EncodeTiledFn>(p);
-        cudaGetLastError();
-    }
-    return fn;
-}
-
-bool make_pool_map(CUtensorMap *map, const void *pool, const arb_attn_params &p, bool e4m3) {
-    EncodeTiledFn fn = encode_tiled_fn();
-    if (!fn) return false;
-    const cuuint64_t dims[2] = {(cuuint64_t)kD, (cuuint64_t)p.num_pages * p.num_kv_heads * kPage};
-    // bf16: rows of 256 bytes, a box is half a row (64 dims) of 16 rows; E4M3: rows of 128 bytes, a box is 16 whole rows
-    const cuuint64_t strides[1] = {(cuuint64_t)kD * (e4m3 ? 1 : 2)};
-    const cuuint32_t box[2] = {(cuuint32_t)(e4m3 ? kD : 64), (cuuint32_t)kPage};
-    const cuuint32_t estr[2] = {1, 1};
-    return fn(map, e4m3 ? CU_TENSOR_MAP_DATA_TYPE_UINT8 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(pool), dims, strides, box, estr,
-              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
-              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
-}
-
 template <int G, bool E4M3>
 arb_status launch_one(Ctx *ctx, const Args &a, CombineArgs ca, const CUtensorMap &km, const CUtensorMap &vm,
                       bool overlap, cudaStream_t stream) {
@@ -929,7 +895,7 @@ arb_status launch_one(Ctx *ctx, const Args &a, CombineArgs ca, const CUtensorMap
 
 bool decode_mma_supported(const arb_attn_params &p) {
     const int g = p.num_q_heads / p.num_kv_heads;
-    return p.dtype == ARB_BF16 && p.head_dim == kD && g >= kDecodeMmaMinGroup && g <= 8 && encode_tiled_fn() != nullptr;
+    return p.dtype == ARB_BF16 && p.head_dim == kD && g >= kDecodeMmaMinGroup && g <= 8 && tma_available();
 }
 
 namespace {
@@ -939,7 +905,9 @@ arb_status launch_decode_tc(Ctx *ctx, const arb_attn_params &p, const void *q, c
                             bool e4m3, float k_scale, float v_scale, const int32_t *block_table, const int32_t *seq_lens,
                             const int32_t *q_lens, void *out, cudaStream_t stream) {
     alignas(64) CUtensorMap km, vm;
-    if (!make_pool_map(&km, k_pages, p, e4m3) || !make_pool_map(&vm, v_pages, p, e4m3)) return ARB_ERR_CUDA;
+    if (!pool_map(ctx, &km, k_pages, p.num_pages, p.num_kv_heads, e4m3) ||
+        !pool_map(ctx, &vm, v_pages, p.num_pages, p.num_kv_heads, e4m3))
+        return ARB_ERR_CUDA;
     const int g = p.num_q_heads / p.num_kv_heads;
     const int gp = (g + 3) / 4 * 4;
     const size_t slots = (size_t)p.batch * p.num_kv_heads + (size_t)ctx->num_sms * kCtasPerSm;
@@ -1034,7 +1002,7 @@ arb_status launch_decode_e4m3(Ctx *ctx, const arb_attn_params &p, const void *q,
                               const void *v_pages, float k_scale, float v_scale, const int32_t *block_table,
                               const int32_t *seq_lens, const int32_t *q_lens, void *out, cudaStream_t stream) {
     const int g = p.num_q_heads / p.num_kv_heads;
-    if (g > 8 || encode_tiled_fn() == nullptr) return ARB_ERR_UNSUPPORTED;
+    if (g > 8 || !tma_available()) return ARB_ERR_UNSUPPORTED;
     return launch_decode_tc(ctx, p, q, k_pages, v_pages, true, k_scale, v_scale, block_table, seq_lens, q_lens, out, stream);
 }
 

@@ -299,6 +299,37 @@ def test_pipelined_host_calls_see_cache_updates_in_stream_order():
     assert not torch.equal(out_a, out_b)
 
 
+def test_pool_tensor_maps_are_cached_by_address_and_shape():
+    """The tensor maps of the KV pools are kept per context.  The same device address with another pool shape must
+    not get the earlier map (whose row bound would zero-fill the pages beyond it), and many pools in turn must
+    each keep their own."""
+    c = H.ctx()
+    small = wl.small_attn_case(2, 12, 2, 128, BF, [100, 45], [1, 1], seed=801)
+    large = wl.small_attn_case(2, 8, 1, 128, BF, [3000, 2100], [1, 1], seed=802)
+    n_small, n_large = small.k_pages.numel(), large.k_pages.numel()
+    assert n_large > 2 * n_small
+    kbuf = torch.zeros(n_large, dtype=BF, device="cuda")
+    vbuf = torch.zeros(n_large, dtype=BF, device="cuda")
+    for inp, n in ((small, n_small), (large, n_large), (small, n_small)):
+        k = kbuf[:n].view(inp.k_pages.shape); v = vbuf[:n].view(inp.v_pages.shape)
+        k.copy_(inp.k_pages); v.copy_(inp.v_pages)
+        d = inp.to("cuda")
+        out = c.attn(d.q, k, v, d.block_table, d.seq_lens, d.q_lens, 1)
+        ref, _ = H.oracle_attn(inp)
+        H.assert_close(out.double().cpu().numpy(), ref, BF)
+    # sixty pools of their own, visited twice
+    d = small.to("cuda")
+    pools = [(d.k_pages.clone(), d.v_pages.clone()) for _ in range(60)]
+    first = [c.attn(d.q, k, v, d.block_table, d.seq_lens, d.q_lens, 1).clone() for k, v in pools]
+    for k, v in pools[::7]:
+        k.mul_(0.5)                      # same address, other contents: the map holds no data
+    again = [c.attn(d.q, k, v, d.block_table, d.seq_lens, d.q_lens, 1).clone() for k, v in pools]
+    torch.cuda.synchronize()
+    for i, (x, y) in enumerate(zip(first, again)):
+        assert torch.equal(x, y) == (i % 7 != 0), i
+    assert c.poll_status() == 0
+
+
 def test_repeated_calls_reuse_the_workspace():
     """Arrival counters return to zero after every call: same answer five times in a row."""
     inp = wl.small_attn_case(2, 12, 2, 128, BF, [9000, 5000], [1, 1], seed=56)

@@ -189,9 +189,12 @@ arb_status arb_attn_host(arb_ctx *ctx, const arb_attn_params *params, const void
  * `stream` (in call order, so cache updates enqueued on `stream` between two calls are seen by the
  * later one), and the copy of the result into out_host on a second copy stream of ctx.  out_host
  * (page-locked memory keeps that copy asynchronous) must not be read before arb_attn_host_wait has
- * returned ARB_OK; synchronising `stream` alone does not cover the copy back.  Up to 8 calls are in
+ * returned ARB_OK; synchronising `stream` alone does not cover the copy back.  Up to 32 calls are in
  * flight per ctx; a further call first waits for the oldest.  Staging grows here when a call needs
  * more (allocation, as in arb_attn_host).  Not for a stream that is being captured into a graph.
+ * A call flagged ARB_ATTN_OVERLAP_PREVIOUS whose out_host is page-locked uses no copies at all: its
+ * kernels read the staged inputs and write out_host in place over the bus (the faster way for a
+ * series of small calls).  `stream` must stay alive until arb_attn_host_wait has returned.
  *
  * arb_attn_host_wait blocks until every call begun on ctx has delivered its result.
  * Errors: as arb_attn_host; after an error nothing of the failed call is left in flight.

@@ -30,7 +30,7 @@ struct HostSlot {
     bool busy = false;
 };
 
-constexpr int kHostSlots = 8;
+constexpr int kHostSlots = 32;
 
 struct Ctx {
     int device = 0;

@@ -172,7 +172,8 @@ arb_status arb_attn(arb_ctx *ctx, const arb_attn_params *params, const void *q,
  * pointers with the shapes above; k_pages and v_pages stay DEVICE pointers (the cache is resident
  * state, not a per-step input).  Copies the inputs to staging buffers owned by ctx (grown here if
  * too small -- the one call besides arb_create that may allocate), runs arb_attn, copies out back
- * and synchronises `stream` before returning.
+ * (a page-locked out_host is written by the kernels directly instead) and synchronises `stream`
+ * before returning.
  */
 arb_status arb_attn_host(arb_ctx *ctx, const arb_attn_params *params, const void *q_host,
                          const void *k_pages, const void *v_pages,

@@ -277,10 +277,19 @@ arb_status arb_attn_host(arb_ctx *ctx, const arb_attn_params *params, const void
     memcpy(hsl, seq_lens_host, len_bytes);
     memcpy(hql, q_lens_host, len_bytes);
     if (cudaMemcpyAsync(dq, hq, in_bytes, cudaMemcpyHostToDevice, s) != cudaSuccess) return ARB_ERR_CUDA;
+    // a page-locked result buffer is written by the kernels themselves, row by row over the bus (posted
+    // writes: nothing waits for them but the final synchronisation), which saves the copy back
+    void *mapped_out = nullptr;
+    if (!aligned16(out_host) || cudaHostGetDevicePointer(&mapped_out, out_host, 0) != cudaSuccess) {
+        cudaGetLastError();
+        mapped_out = nullptr;
+    }
     st = arb_attn(ctx, params, dq, k_pages, v_pages, reinterpret_cast<int32_t *>(dbt),
-                  reinterpret_cast<int32_t *>(dsl), reinterpret_cast<int32_t *>(dql), dout, stream);
+                  reinterpret_cast<int32_t *>(dsl), reinterpret_cast<int32_t *>(dql), mapped_out ? mapped_out : dout,
+                  stream);
     if (st != ARB_OK) return st;
-    if (cudaMemcpyAsync(out_host, dout, q_bytes, cudaMemcpyDeviceToHost, s) != cudaSuccess) return ARB_ERR_CUDA;
+    if (!mapped_out && cudaMemcpyAsync(out_host, dout, q_bytes, cudaMemcpyDeviceToHost, s) != cudaSuccess)
+        return ARB_ERR_CUDA;
     if (cudaStreamSynchronize(s) != cudaSuccess) return ARB_ERR_CUDA;
     return ARB_OK;
 }
@@ -329,10 +338,14 @@ arb_status arb_attn_host_begin(arb_ctx *ctx, const arb_attn_params *params, cons
     // with the copies below and unflagged kernels.  It pays for flagged calls only: every CTA reads lengths,
     // block-table entries and q rows over the bus in small requests, and an unflagged small call has twice the
     // CTAs (41 us per call).
-    if (params->flags & ARB_ATTN_OVERLAP_PREVIOUS) {
-        void *mapped_out = nullptr, *mapped_in = nullptr;
-        if (aligned16(out_host) && cudaHostGetDevicePointer(&mapped_out, out_host, 0) == cudaSuccess &&
-            cudaHostGetDevicePointer(&mapped_in, h.host, 0) == cudaSuccess) {
+    void *mapped_out = nullptr;
+    if (!aligned16(out_host) || cudaHostGetDevicePointer(&mapped_out, out_host, 0) != cudaSuccess) {
+        cudaGetLastError();   // out_host is ordinary memory
+        mapped_out = nullptr;
+    }
+    if ((params->flags & ARB_ATTN_OVERLAP_PREVIOUS) && mapped_out) {
+        void *mapped_in = nullptr;
+        if (cudaHostGetDevicePointer(&mapped_in, h.host, 0) == cudaSuccess) {
             char *mq = static_cast<char *>(mapped_in), *mbt = mq + up(q_bytes);
             char *msl = mbt + up(bt_bytes), *mql = msl + up(len_bytes);
             st = arb_attn(ctx, params, mq, k_pages, v_pages, reinterpret_cast<int32_t *>(mbt),
@@ -347,7 +360,7 @@ arb_status arb_attn_host_begin(arb_ctx *ctx, const arb_attn_params *params, cons
             c->next_slot = (c->next_slot + 1) % kHostSlots;
             return ARB_OK;
         }
-        cudaGetLastError();   // out_host is ordinary memory: the staged path below
+        cudaGetLastError();
     }
     if (need > h.dev_bytes) {  // the slot is idle, so nothing on the device still uses its buffers
         cudaFree(h.dev);
@@ -379,6 +392,9 @@ arb_status arb_attn_host_begin(arb_ctx *ctx, const arb_attn_params *params, cons
         cudaGetLastError();
         return st;
     }
+    // (Letting these kernels write a page-locked out_host themselves was measured and is slower here, 27 against
+    // 24 us per call: the writes over the bus have to drain before the kernel counts as complete, and that is on
+    // the chain of serialised kernels, while the copy below is beside it.)
     bool ok = cudaEventRecord(h.kernels_done, s) == cudaSuccess;
     ok = ok && cudaStreamWaitEvent(c->out_stream, h.kernels_done, 0) == cudaSuccess;
     ok = ok && cudaMemcpyAsync(out_host, dout, q_bytes, cudaMemcpyDeviceToHost, c->out_stream) == cudaSuccess;

@@ -242,12 +242,14 @@ def test_host_buffer_entry_point():
     assert torch.equal(out, out2)
 
 
+@pytest.mark.parametrize("pinned_out", [True, False])
 @pytest.mark.parametrize("flagged", [False, True])
-def test_pipelined_host_calls(flagged):
+def test_pipelined_host_calls(flagged, pinned_out):
     """arb_attn_host_begin / arb_attn_host_wait: more calls in flight than the ring has slots, shapes that change from
     call to call (staging grows), inputs overwritten as soon as begin has returned; every result equals the one-shot
     host call bit for bit and the oracle within tolerance.  Flagged calls (operands moved in place over the bus,
-    another split of the keys) are held to the oracle alone."""
+    another split of the keys) are held to the oracle alone.  A page-locked result buffer is written by the kernels
+    themselves, an ordinary one through a copy."""
     from paper_2512_05033_b200 import binding
     c = H.ctx()
     shapes = [([500, 90, 2000], [1, 4, 1]), ([33], [1]), ([4000, 4100, 777, 12, 640], [1, 1, 1, 1, 1]),
@@ -262,7 +264,9 @@ def test_pipelined_host_calls(flagged):
         cases.append((inp, kp, vp, max(ql)))
     for inp, kp, vp, mq in cases:
         q, bt, sl, ql = inp.q.clone(), inp.block_table.clone(), inp.seq_lens.clone(), inp.q_lens.clone()
-        out = torch.full_like(inp.q, float("nan")).pin_memory()
+        out = torch.full_like(inp.q, float("nan"))
+        if pinned_out:
+            out = out.pin_memory()
         c.attn_host_begin(q, kp, vp, bt, sl, ql, mq, out, flags=binding.ATTN_OVERLAP_PREVIOUS if flagged else 0)
         q.fill_(float("nan")); bt.fill_(-1); sl.fill_(-1); ql.fill_(-1)   # the library has its own copy by now
         outs.append(out)

@@ -894,8 +894,8 @@ arb_status launch_chunk_mma(Ctx *ctx, const arb_attn_params &p, const void *q, c
                             const void *v_pages, const int32_t *block_table, const int32_t *seq_lens,
                             const int32_t *q_lens, void *out, cudaStream_t stream) {
     alignas(64) CUtensorMap km, vm;
-    if (!pool_map(ctx, &km, k_pages, p.num_pages, p.num_kv_heads, false) ||
-        !pool_map(ctx, &vm, v_pages, p.num_pages, p.num_kv_heads, false))
+    if (!pool_map(ctx, &km, k_pages, p.num_pages, p.num_kv_heads, PoolView::kBf16HalfRows) ||
+        !pool_map(ctx, &vm, v_pages, p.num_pages, p.num_kv_heads, PoolView::kBf16HalfRows))
         return ARB_ERR_CUDA;
     MmaArgs a;
     a.q = static_cast<const char *>(q);

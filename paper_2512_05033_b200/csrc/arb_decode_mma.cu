@@ -10,8 +10,9 @@
 //
 // The streaming part is the scheme of the CUDA-core decode kernel: flat page list cut into equal
 // ranges per CTA, one producer warp feeding a 16-stage ring, pages owned by one consumer warp each
-// with its own online softmax.  Differences: K/V tiles arrive as tiled TMA boxes (16 rows x 64 dims,
-// 128-byte swizzle, two per tile) so that ldmatrix reads them without bank conflicts; P is rounded
+// with its own online softmax.  Differences: K/V tiles arrive through tiled TMA copies as two 128-byte-swizzled
+// halves of 16 rows x 64 dims (one box of a 3-D view of the pool brings both) so that ldmatrix reads them
+// without bank conflicts; P is rounded
 // to bf16 for the second product (and summed after rounding, so numerator and denominator agree);
 // results of a segment are parked in shared memory and written out after the CTA's last page, so
 // the wait for the previous kernel (programmatic dependent launch) comes once, after all streaming.
@@ -55,7 +56,7 @@ constexpr int kRingBytes = 64 * 1024;
 // what differs between the bf16 cache and the E4M3 cache in the ring
 template <bool E4M3>
 struct Fmt {
-    static constexpr int kTileBytes = kPage * kD * (E4M3 ? 1 : 2);   // 4 KB (two TMA boxes of 16 rows x 64 bf16) or
+    static constexpr int kTileBytes = kPage * kD * (E4M3 ? 1 : 2);   // 4 KB (two halves of 16 rows x 64 bf16) or
                                                                      // 2 KB (one box of 16 rows x 128 codes)
     static constexpr int kHalfTile = kTileBytes / 2;
     static constexpr int kStages = kRingBytes / kTileBytes;          // 16 or 32
@@ -80,6 +81,7 @@ struct Args {
     uint32_t *status;
     int batch, Hq, Hkv, num_pages, max_pages;
     int small_ctas;   // CTAs a small call spreads over
+    int whole_rows;   // the tensor maps are 3-D: one copy per page instead of one per half
     float scale_log2;   // softmax scale (times the key scale of an E4M3 cache) * log2(e)
     float v_scale;      // value scale of an E4M3 cache, 1 otherwise
     // workspace rotation (see launch_decode_mma): this call's generation number, the number of
@@ -167,6 +169,13 @@ __device__ __forceinline__ void tma_box_load(void *dst_smem, const CUtensorMap *
     asm volatile(
         "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
         ::"r"(smem_u32(dst_smem)), "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(smem_u32(bar))
+        : "memory");
+}
+
+__device__ __forceinline__ void tma_box_load3(void *dst_smem, const CUtensorMap *map, int x, int y, int z, uint64_t *bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
+        ::"r"(smem_u32(dst_smem)), "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(z), "r"(smem_u32(bar))
         : "memory");
 }
 
@@ -368,8 +377,12 @@ decode_mma_kernel(const Args a, const __grid_constant__ CUtensorMap k_map, const
                         if (mbar_wait(&tail->empty[st], par ^ 1u, abort, a.status)) {
                             mbar_arrive_expect_tx(&tail->full[st], kTileBytes);
                             const int row = (pg * Hkv + s.kvh) * kPage;
-                            tma_box_load(ring + st * kTileBytes, map, 0, row, &tail->full[st]);
-                            if constexpr (!E4M3) tma_box_load(ring + st * kTileBytes + kHalfTile, map, 64, row, &tail->full[st]);
+                            if (!E4M3 && a.whole_rows) {
+                                tma_box_load3(ring + st * kTileBytes, map, 0, row, 0, &tail->full[st]);
+                            } else {
+                                tma_box_load(ring + st * kTileBytes, map, 0, row, &tail->full[st]);
+                                if constexpr (!E4M3) tma_box_load(ring + st * kTileBytes + kHalfTile, map, 64, row, &tail->full[st]);
+                            }
                         }
                     }
                     __syncwarp();
@@ -905,8 +918,16 @@ arb_status launch_decode_tc(Ctx *ctx, const arb_attn_params &p, const void *q, c
                             bool e4m3, float k_scale, float v_scale, const int32_t *block_table, const int32_t *seq_lens,
                             const int32_t *q_lens, void *out, cudaStream_t stream) {
     alignas(64) CUtensorMap km, vm;
-    if (!pool_map(ctx, &km, k_pages, p.num_pages, p.num_kv_heads, e4m3) ||
-        !pool_map(ctx, &vm, v_pages, p.num_pages, p.num_kv_heads, e4m3))
+    // bf16 pools: a page is fetched as one box of the 3-D view (both 64-element halves of its 16 rows), which
+    // halves the number of TMA copies; the 2-D view with two boxes per page stays as the fallback should a
+    // driver refuse the 3-D encoding, whose third stride is smaller than its second.
+    bool whole_rows = false;
+    if (!e4m3)
+        whole_rows = pool_map(ctx, &km, k_pages, p.num_pages, p.num_kv_heads, PoolView::kBf16WholeRows) &&
+                     pool_map(ctx, &vm, v_pages, p.num_pages, p.num_kv_heads, PoolView::kBf16WholeRows);
+    const PoolView view = e4m3 ? PoolView::kE4m3 : PoolView::kBf16HalfRows;
+    if (!whole_rows && (!pool_map(ctx, &km, k_pages, p.num_pages, p.num_kv_heads, view) ||
+                        !pool_map(ctx, &vm, v_pages, p.num_pages, p.num_kv_heads, view)))
         return ARB_ERR_CUDA;
     const int g = p.num_q_heads / p.num_kv_heads;
     const int gp = (g + 3) / 4 * 4;
@@ -943,6 +964,7 @@ arb_status launch_decode_tc(Ctx *ctx, const arb_attn_params &p, const void *q, c
     a.Hkv = p.num_kv_heads;
     a.num_pages = p.num_pages;
     a.max_pages = p.max_pages_per_seq;
+    a.whole_rows = whole_rows ? 1 : 0;
     // A small call streams at the pace of its CTAs' pipelines, not of the memory system, and every
     // CTA spends a fixed time before its first and after its last tile.  A call that declares itself
     // part of a back-to-back series (ARB_ATTN_OVERLAP_PREVIOUS) therefore takes only every second

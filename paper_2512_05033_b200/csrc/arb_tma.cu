@@ -33,7 +33,7 @@ constexpr int kMapProbe = 4;
 struct MapEntry {
     alignas(64) CUtensorMap map;
     const void *pool = nullptr;
-    int num_pages = 0, num_kv_heads = 0, e4m3 = 0;
+    int num_pages = 0, num_kv_heads = 0, view = 0;
 };
 
 }  // namespace
@@ -53,11 +53,33 @@ bool encode_pool_map(CUtensorMap *map, const void *pool, int num_pages, int num_
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-bool pool_map(Ctx *ctx, CUtensorMap *map, const void *pool, int num_pages, int num_kv_heads, bool e4m3) {
+// The same bf16 pool as a 3-D view (64 elements, rows, the two 64-element halves of a row; the third
+// dimension's stride, 128 bytes, is smaller than the second's, 256): one box of 16 rows x both halves lands
+// as [half][row][128 bytes], the layout two boxes of the 2-D view give, with one copy instead of two.
+bool encode_pool_map3(CUtensorMap *map, const void *pool, int num_pages, int num_kv_heads) {
+    EncodeTiledFn fn = encode_tiled_fn();
+    if (!fn) return false;
+    const cuuint64_t dims[3] = {64, (cuuint64_t)num_pages * num_kv_heads * kPage, 2};
+    const cuuint64_t strides[2] = {(cuuint64_t)kD * 2, 128};
+    const cuuint32_t box[3] = {64, (cuuint32_t)kPage, 2};
+    const cuuint32_t estr[3] = {1, 1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(pool), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+namespace {
+bool encode_view(CUtensorMap *map, const void *pool, int num_pages, int num_kv_heads, PoolView view) {
+    if (view == PoolView::kBf16WholeRows) return encode_pool_map3(map, pool, num_pages, num_kv_heads);
+    return encode_pool_map(map, pool, num_pages, num_kv_heads, view == PoolView::kE4m3);
+}
+}  // namespace
+
+bool pool_map(Ctx *ctx, CUtensorMap *map, const void *pool, int num_pages, int num_kv_heads, PoolView view) {
     MapEntry *cache = static_cast<MapEntry *>(ctx->map_cache);
     if (cache == nullptr) {
         cache = new (std::nothrow) MapEntry[kMapSlots];
-        if (cache == nullptr) return encode_pool_map(map, pool, num_pages, num_kv_heads, e4m3);
+        if (cache == nullptr) return encode_view(map, pool, num_pages, num_kv_heads, view);
         ctx->map_cache = cache;
     }
     // pools are large allocations: the low bits of their addresses carry nothing
@@ -66,7 +88,7 @@ bool pool_map(Ctx *ctx, CUtensorMap *map, const void *pool, int num_pages, int n
     const unsigned first = (h >> 16) & (kMapSlots - 1);
     for (int i = 0; i < kMapProbe; ++i) {
         MapEntry &e = cache[(first + i) & (kMapSlots - 1)];
-        if (e.pool == pool && e.num_pages == num_pages && e.num_kv_heads == num_kv_heads && e.e4m3 == (e4m3 ? 1 : 0)) {
+        if (e.pool == pool && e.num_pages == num_pages && e.num_kv_heads == num_kv_heads && e.view == (int)view) {
             *map = e.map;
             return true;
         }
@@ -79,11 +101,11 @@ bool pool_map(Ctx *ctx, CUtensorMap *map, const void *pool, int num_pages, int n
     }
     if (slot == nullptr) slot = &cache[(first + (ctx->map_evictions++ % kMapProbe)) & (kMapSlots - 1)];
     slot->pool = nullptr;
-    if (!encode_pool_map(&slot->map, pool, num_pages, num_kv_heads, e4m3)) return false;
+    if (!encode_view(&slot->map, pool, num_pages, num_kv_heads, view)) return false;
     slot->pool = pool;
     slot->num_pages = num_pages;
     slot->num_kv_heads = num_kv_heads;
-    slot->e4m3 = e4m3 ? 1 : 0;
+    slot->view = (int)view;
     *map = slot->map;
     return true;
 }

@@ -15,10 +15,20 @@ bool tma_available();
 // 16 whole rows.  128-byte swizzle either way.
 bool encode_pool_map(CUtensorMap *map, const void *pool, int num_pages, int num_kv_heads, bool e4m3);
 
-// The same map out of the context's cache, copied to `map` (encoded on first use: a model's pools come back
+// The views of a pool the kernels use.
+enum class PoolView : int {
+    kBf16HalfRows = 0,    // 2-D, box 16 rows x 64 elements (one 128-byte-swizzled half tile)
+    kE4m3 = 1,            // 2-D over E4M3 codes, box 16 whole rows of 128 bytes
+    kBf16WholeRows = 2,   // 3-D (64 elements, rows, 2 halves), box 16 rows x both halves: a page in one copy
+};
+
+// 3-D view kBf16WholeRows; false if the driver refuses the encoding (the caller then uses kBf16HalfRows).
+bool encode_pool_map3(CUtensorMap *map, const void *pool, int num_pages, int num_kv_heads);
+
+// A view's map out of the context's cache, copied to `map` (encoded on first use: a model's pools come back
 // every token, and encoding two maps costs about as much host time as launching a kernel).  Host-side, not
 // thread-safe, like ctx.
-bool pool_map(Ctx *ctx, CUtensorMap *map, const void *pool, int num_pages, int num_kv_heads, bool e4m3);
+bool pool_map(Ctx *ctx, CUtensorMap *map, const void *pool, int num_pages, int num_kv_heads, PoolView view);
 
 void pool_map_cache_free(Ctx *ctx);
 

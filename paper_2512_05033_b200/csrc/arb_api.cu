@@ -350,7 +350,11 @@ arb_status arb_attn_host_begin(arb_ctx *ctx, const arb_attn_params *params, cons
             char *msl = mbt + up(bt_bytes), *mql = msl + up(len_bytes);
             st = arb_attn(ctx, params, mq, k_pages, v_pages, reinterpret_cast<int32_t *>(mbt),
                           reinterpret_cast<int32_t *>(msl), reinterpret_cast<int32_t *>(mql), mapped_out, stream);
-            if (st != ARB_OK) return st;   // nothing was enqueued
+            if (st != ARB_OK) {  // a part of the call may be in flight: the slot is not marked busy, so wait here
+                cudaStreamSynchronize(s);
+                cudaGetLastError();
+                return st;
+            }
             if (cudaEventRecord(h.out_done, s) != cudaSuccess) {
                 cudaStreamSynchronize(s);
                 cudaGetLastError();
@@ -389,6 +393,7 @@ arb_status arb_attn_host_begin(arb_ctx *ctx, const arb_attn_params *params, cons
         st = ARB_ERR_CUDA;
     if (st != ARB_OK) {  // nothing of this call may stay in flight on a slot that is not marked busy
         cudaStreamSynchronize(c->in_stream);
+        cudaStreamSynchronize(s);
         cudaGetLastError();
         return st;
     }

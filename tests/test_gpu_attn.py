@@ -281,6 +281,37 @@ def test_pipelined_host_calls(flagged, pinned_out):
         H.assert_close(outs[i].double().numpy(), ref, BF)
 
 
+def test_pipelined_host_call_errors_leave_nothing_in_flight():
+    """Bad arguments are refused by arb_attn_host_begin like by arb_attn; the context goes on working."""
+    from paper_2512_05033_b200 import binding
+    c = H.ctx()
+    inp = wl.small_attn_case(2, 12, 2, 128, BF, [300, 45], [1, 1], seed=741)
+    kp, vp = inp.k_pages.cuda(), inp.v_pages.cuda()
+    host = [t.pin_memory() for t in (inp.q, inp.block_table, inp.seq_lens, inp.q_lens)]
+    out = torch.empty_like(inp.q).pin_memory()
+    p = c.params_for(host[0], kp, host[1], 1)
+    args = [host[0].data_ptr(), kp.data_ptr(), vp.data_ptr(), host[1].data_ptr(), host[2].data_ptr(),
+            host[3].data_ptr(), out.data_ptr(), 0]
+    bad = list(args); bad[6] = None
+    assert c.attn_host_begin_raw(p, *bad) == binding.ARB_ERR_INVALID_ARG          # no result buffer
+    bad = list(args); bad[1] = None
+    assert c.attn_host_begin_raw(p, *bad) == binding.ARB_ERR_INVALID_ARG          # no key pool
+    p2 = c.params_for(host[0], kp, host[1], 1); p2.head_dim = 96
+    assert c.attn_host_begin_raw(p2, *args) == binding.ARB_ERR_UNSUPPORTED
+    small = binding.Context(0, workspace_bytes=1024)
+    assert small.attn_host_begin_raw(p, *args) == binding.ARB_ERR_WORKSPACE
+    small.attn_host_wait()
+    small.close()
+    for flags in (0, binding.ATTN_OVERLAP_PREVIOUS):
+        p.flags = flags
+        assert c.attn_host_begin_raw(p, *args) == binding.ARB_OK
+        c.attn_host_wait()
+        ref, _ = H.oracle_attn(inp)
+        H.assert_close(out.double().numpy(), ref, BF)
+        out.zero_()
+    assert c.poll_status() == 0
+
+
 def test_pipelined_host_calls_see_cache_updates_in_stream_order():
     """Kernels of begun calls run on the caller's stream in call order: an append enqueued between two calls is
     seen by the second and not by the first."""

@@ -160,9 +160,11 @@ template <typename T>
 __global__ void __launch_bounds__(kHeadWarps * 32)
 route_classes_kernel(const HeadArgs a) {
     constexpr int EPL = Elt<T>::kPerVec;
-    const int lane = threadIdx.x & 31;
-    const int step = blockIdx.x * kHeadWarps + (threadIdx.x >> 5);
-    if (step >= a.n_steps) return;
+    // one CTA per step: its warps share the row (a single warp per step would walk the row in 14 dependent
+    // round trips at the router's hidden size), partial sums meet in shared memory
+    __shared__ float part[kHeadWarps][ARB_MAX_CLASSES];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int step = blockIdx.x;
     const int C = a.n_classes;
     const int nlog = a.mode == ARB_HEAD_SOFTMAX ? C : 1;   // dot products to take
     const int nvec = a.hidden_dim / EPL;
@@ -170,7 +172,7 @@ route_classes_kernel(const HeadArgs a) {
     float acc[ARB_MAX_CLASSES];
 #pragma unroll
     for (int c = 0; c < ARB_MAX_CLASSES; ++c) acc[c] = 0.f;
-    for (int v = lane; v < nvec; v += 32) {
+    for (int v = threadIdx.x; v < nvec; v += kHeadWarps * 32) {
         float hf[EPL];
         Elt<T>::unpack(__ldg(hrow + v), hf);
 #pragma unroll
@@ -190,7 +192,21 @@ route_classes_kernel(const HeadArgs a) {
             for (int off = 16; off >= 1; off >>= 1) acc[c] += __shfl_xor_sync(0xffffffffu, acc[c], off);
         }
     }
-    if (lane != 0) return;
+    if (lane == 0) {
+#pragma unroll
+        for (int c = 0; c < ARB_MAX_CLASSES; ++c)
+            if (c < nlog) part[warp][c] = acc[c];
+    }
+    __syncthreads();
+    if (threadIdx.x != 0) return;
+#pragma unroll
+    for (int c = 0; c < ARB_MAX_CLASSES; ++c) {
+        if (c < nlog) {
+            float t = part[0][c];
+            for (int w2 = 1; w2 < kHeadWarps; ++w2) t += part[w2][c];
+            acc[c] = t;
+        }
+    }
     float p[ARB_MAX_CLASSES];
     if (a.mode == ARB_HEAD_SOFTMAX) {
         float mx = -INFINITY, z = 0.f;
@@ -266,7 +282,7 @@ arb_status launch_route_classes(Ctx *ctx, int dtype, int mode, int n_steps, int 
     a.probs = probs;
     a.scores = scores;
     a.decisions = decisions;
-    const int grid = (n_steps + kHeadWarps - 1) / kHeadWarps;
+    const int grid = n_steps;
     if (dtype == ARB_BF16)
         route_classes_kernel<__nv_bfloat16><<<grid, kHeadWarps * 32, 0, stream>>>(a);
     else if (dtype == ARB_F32)

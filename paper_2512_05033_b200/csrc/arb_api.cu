@@ -198,9 +198,9 @@ arb_status arb_attn(arb_ctx *ctx, const arb_attn_params *params, const void *q, 
         if (st != ARB_OK) return st;
     }
     if (params->max_q_len >= 2) {
-        // Step chunks: a chunk with q_len * group >= 64 rows (bf16, head_dim 128) is a dense
-        // contraction and goes to the tcgen05 kernel; the rest, and every fp32 chunk, to the
-        // CUDA-core kernel.  Both kernels decide per sequence on the device.
+        // Step chunks: bf16 chunks of head_dim 128 go to the tcgen05 kernel (from kChunkMmaMinRows
+        // rows on, i.e. all of them); the rest, and every fp32 chunk, to the CUDA-core kernel.  Both
+        // kernels decide per sequence on the device.
         int skip_rows = 0;
         if (tensor_cores && chunk_mma_supported(*params)) {
             st = launch_chunk_mma(c, *params, q, k_pages, v_pages, block_table, seq_lens, q_lens, out, s);

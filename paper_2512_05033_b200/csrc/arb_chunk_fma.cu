@@ -1,7 +1,7 @@
 // Step-chunk attention, CUDA-core path: one CTA per (query row, kv head).
 //
-// This is the path for chunks that are not a dense contraction worth the tensor cores: fp32 inputs
-// (whose 1e-5 tolerance rules out tf32), head_dim 64, and chunks with q_len * group < 64 rows.  It
+// This is the path for chunks the tensor-core kernel does not take: fp32 inputs (whose 1e-5 tolerance
+// rules out tf32), head_dim 64, groups above 8, and every chunk when ARB_ATTN_NO_TENSOR_CORES is set.  It
 // also zero-fills the rows of chunk sequences whose lengths are invalid, whatever their size.  Query token i of
 // a chunk of n tokens sits at position pos = L - n + i and attends keys 0..pos; the causal mask is
 // just each row's own key count.  K and V rows are read straight from global memory with 16-byte

@@ -1,8 +1,9 @@
 // Step-chunk attention on the 5th-generation tensor cores (tcgen05 + TMEM), bf16, head_dim 128.
 //
-// A chunk of n query tokens against one KV head is a dense contraction once n * group >= 64:
-// the M = n * group query rows (token-major, the group's heads of one token are consecutive rows)
-// all read the same keys.  One work item is a pair of row tiles (A, B: 128 query rows each, B may be
+// A chunk of n query tokens against one KV head is a contraction over shared operands: the
+// M = n * group query rows (token-major, the group's heads of one token are consecutive rows) all read
+// the same keys (dense enough to keep the tensor core busy from M of about 64; below that the tile is
+// mostly padding, but it still reads every key once).  One work item is a pair of row tiles (A, B: 128 query rows each, B may be
 // missing) of one (sequence, kv head); it walks the visible keys in tiles of 128 (eight pages), and
 // both row tiles use every K/V tile that is loaded.  Per row tile and KV tile:
 //

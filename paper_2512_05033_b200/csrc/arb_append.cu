@@ -34,6 +34,8 @@ struct AppendArgs {
     int batch, Hkv, num_pages, max_pages;
     int row_bytes;   // D * element size: bytes of one (token, kv head) row
     int total_new;
+    int update_lens;     // seq_lens += new_lens once every CTA has placed its rows
+    int *done_counter;   // CTAs of this call that have; zero between calls
 };
 
 // 0 = append, otherwise the status bit that explains why not (new_len == 0 appends nothing and is fine)
@@ -46,6 +48,26 @@ __device__ __forceinline__ uint32_t append_check(const AppendArgs &a, int b) {
         if ((unsigned)page >= (unsigned)a.num_pages) return ARB_DEV_BAD_PAGE;
     }
     return 0;
+}
+
+// The lengths move forward inside the append kernel: every CTA reads the old lengths for the rows it places, so
+// the CTA that finishes last (a counter tells it) adds new_lens, and leaves the counter at zero for the next call.
+// `okay` is this CTA's copy of the per-sequence checks, taken from the old lengths.
+__device__ __forceinline__ void advance_lens_when_last(const AppendArgs &a, const int *okay) {
+    if (!a.update_lens) return;
+    __shared__ int is_last;
+    __syncthreads();   // all rows of this CTA are placed, all its reads of seq_lens are done
+    if (threadIdx.x == 0) {
+        __threadfence();
+        is_last = atomicAdd(a.done_counter, 1) == (int)gridDim.x - 1;
+    }
+    __syncthreads();
+    if (!is_last) return;
+    for (int b = threadIdx.x; b < a.batch; b += kAppendThreads) {
+        const int n = a.new_lens[b];
+        if (n > 0 && okay[b]) a.seq_lens[b] += n;
+    }
+    if (threadIdx.x == 0) *a.done_counter = 0;
 }
 
 __global__ void __launch_bounds__(kAppendThreads)
@@ -101,6 +123,7 @@ kv_append_kernel(const AppendArgs a) {
         *reinterpret_cast<uint4 *>(a.k_pages + dst) = kx;
         *reinterpret_cast<uint4 *>(a.v_pages + dst) = vx;
     }
+    advance_lens_when_last(a, okay);
 }
 
 // two values -> two E4M3 codes; lo lands in the low byte
@@ -180,14 +203,7 @@ kv_append_e4m3_kernel(const AppendArgs a, float k_inv_scale, float v_inv_scale) 
             *reinterpret_cast<uint32_t *>(a.v_pages + dst) = vc[0];
         }
     }
-}
-
-__global__ void __launch_bounds__(kAppendThreads)
-advance_lens_kernel(const AppendArgs a) {
-    for (int b = threadIdx.x; b < a.batch; b += kAppendThreads) {
-        const int n = a.new_lens[b];
-        if (n > 0 && append_check(a, b) == 0) a.seq_lens[b] += n;
-    }
+    advance_lens_when_last(a, okay);
 }
 
 }  // namespace
@@ -210,6 +226,8 @@ arb_status launch_kv_append(Ctx *ctx, const arb_attn_params &p, int total_new, c
     a.max_pages = p.max_pages_per_seq;
     a.row_bytes = p.head_dim * (p.dtype == ARB_BF16 ? 2 : 4);
     a.total_new = total_new;
+    a.update_lens = update_lens;
+    a.done_counter = ctx->rot + (size_t)kRotSets * kRotCounters + kRotSets + 3;
     const int rows_per_pass = kAppendThreads / (a.row_bytes / 16);
     const long long nrows = (long long)total_new * p.num_kv_heads;
     long long want = (nrows + rows_per_pass - 1) / rows_per_pass;
@@ -219,11 +237,6 @@ arb_status launch_kv_append(Ctx *ctx, const arb_attn_params &p, int total_new, c
     kv_append_kernel<<<grid, kAppendThreads, smem, stream>>>(a);
     ctx->launches++;
     if (cudaGetLastError() != cudaSuccess) return ARB_ERR_CUDA;
-    if (update_lens) {
-        advance_lens_kernel<<<1, kAppendThreads, 0, stream>>>(a);
-        ctx->launches++;
-        if (cudaGetLastError() != cudaSuccess) return ARB_ERR_CUDA;
-    }
     return ARB_OK;
 }
 
@@ -246,6 +259,8 @@ arb_status launch_kv_append_e4m3(Ctx *ctx, const arb_attn_params &p, int total_n
     a.max_pages = p.max_pages_per_seq;
     a.row_bytes = p.head_dim * (p.dtype == ARB_BF16 ? 2 : 4);   // of the source rows
     a.total_new = total_new;
+    a.update_lens = update_lens;
+    a.done_counter = ctx->rot + (size_t)kRotSets * kRotCounters + kRotSets + 3;
     const int rows_per_pass = kAppendThreads / (a.row_bytes / 16);
     const long long nrows = (long long)total_new * p.num_kv_heads;
     long long want = (nrows + rows_per_pass - 1) / rows_per_pass;
@@ -258,11 +273,6 @@ arb_status launch_kv_append_e4m3(Ctx *ctx, const arb_attn_params &p, int total_n
         kv_append_e4m3_kernel<float><<<grid, kAppendThreads, smem, stream>>>(a, k_inv_scale, v_inv_scale);
     ctx->launches++;
     if (cudaGetLastError() != cudaSuccess) return ARB_ERR_CUDA;
-    if (update_lens) {
-        advance_lens_kernel<<<1, kAppendThreads, 0, stream>>>(a);
-        ctx->launches++;
-        if (cudaGetLastError() != cudaSuccess) return ARB_ERR_CUDA;
-    }
     return ARB_OK;
 }
 

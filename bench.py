@@ -372,22 +372,30 @@ def run_e2e(ctx, work: DecodeWorkload, steps: int, world: int):
         torch.cuda.synchronize()
         return (time.perf_counter() - t0) / steps
 
-    dt = timed(make(True, binding.ATTN_OVERLAP_PREVIOUS))
+    dt_flag = timed(make(True, binding.ATTN_OVERLAP_PREVIOUS))
     dt_staged = timed(make(True, 0))
     dt_sync = timed(make(False, 0))
     gbs = lambda t: round(world * work.bytes["kv"] * work.layers / t / 1e9, 1)  # noqa: E731
     h2d = (qh.numel() * qh.element_size() + bth.numel() * 4 + slh.numel() * 4 + qlh.numel() * 4) * work.layers
     d2h = qh.numel() * qh.element_size() * work.layers
+    # Two ways of issuing the same pipelined calls.  Which is faster depends on the box: the flagged calls read their
+    # inputs over the bus from page-locked host memory, and that has been seen at 17 and at 29 us per call on
+    # different hosts, while the staged copies are steady at 24.  The headline is the better of the two, named.
+    flagged_wins = dt_flag <= dt_staged
+    dt = min(dt_flag, dt_staged)
     return {"value": gbs(dt), "unit": "GB/s",
             "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": round(dt * 1e3, 4),
+            "mode": "flagged_calls" if flagged_wins else "unflagged_calls",
+            "flagged_calls": {"value": gbs(dt_flag), "ms_per_step": round(dt_flag * 1e3, 4),
+                              "note": "ARB_ATTN_OVERLAP_PREVIOUS: the kernels read the inputs from page-locked host "
+                                      "memory and write out into it over the bus, no copies"},
             "unflagged_calls": {"value": gbs(dt_staged), "ms_per_step": round(dt_staged * 1e3, 4),
                                 "note": "operands staged by copies on two copy streams beside the kernels"},
             "one_call_at_a_time": {"value": gbs(dt_sync), "ms_per_step": round(dt_sync * 1e3, 4),
                                    "note": "arb_attn_host: each layer call returns with its result on the host"},
-            "note": "arb_attn_host_begin per layer call, flagged ARB_ATTN_OVERLAP_PREVIOUS (the kernels read the inputs "
-                    "from page-locked host memory and write out into it over the bus, no copies), and one "
-                    "arb_attn_host_wait per step; host clock around the steps; KV cache resident; measured on rank 0, "
-                    "scaled by ranks"}
+            "note": "arb_attn_host_begin per layer call and one arb_attn_host_wait per step, issued both ways (mode = the "
+                    "faster one, whose figure is the value); host clock around the steps; KV cache resident; measured "
+                    "on rank 0, scaled by ranks"}
 
 
 def run_target_decode(ctx, dev, peak):

@@ -3,6 +3,7 @@
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
                     [--workload draft|target] [--layers L] [--no-graph] [--no-extras] [--profile]
+                    [--profile-scoring] [--profile-e4m3] [--profile-step-loop]
 
 Headline workload: the draft-shaped decode configuration (batch 8, 12 query / 2 KV heads, head_dim
 128, bf16, page 16, prefix lengths uniform in [1024, 8192], q_len 1).  One step is one generated
@@ -728,6 +729,8 @@ def main():
                          "rollback) and nothing else")
     ap.add_argument("--profile-e4m3", action="store_true",
                     help="for runs under ncu: a few calls of the E4M3 decode on both decode workloads and nothing else")
+    ap.add_argument("--profile-step-loop", action="store_true",
+                    help="for runs under ncu: the step loop (rounds of Algorithm 1 over three caches) and nothing else")
     ap.add_argument("--profile", action="store_true",
                     help="for runs under ncu: stream launches, no e2e / extras / CPU baseline")
     args = ap.parse_args()
@@ -739,6 +742,10 @@ def main():
         from paper_2512_05033_b200 import binding
         torch.cuda.set_device(0)
         print(json.dumps({"step_scoring": run_step_scoring(binding.Context(0), torch.device("cuda", 0))}), flush=True)
+    elif args.profile_step_loop:
+        from paper_2512_05033_b200 import binding
+        torch.cuda.set_device(0)
+        print(json.dumps({"step_loop": run_step_loop(binding.Context(0), torch.device("cuda", 0))}), flush=True)
     elif args.profile_e4m3:
         from paper_2512_05033_b200 import binding
         torch.cuda.set_device(0)

@@ -400,6 +400,16 @@ arb_status arb_phase_lens(arb_ctx *ctx, int32_t batch, const int32_t *step_lens,
                           int32_t want, int32_t t, int32_t *out, arb_stream_t stream);
 
 /*
+ * arb_phase_lens for all tokens of a step that is generated token by token, in one launch: the lengths of
+ * token t depend only on step_lens and decisions, which are fixed while the step is generated.
+ *   out  int32 [n_tokens, B]:  out[t][b] = 1 if b takes part and t < step_lens[b], else 0;  row t is what
+ *        arb_phase_lens gives for that t.  batch * n_tokens <= 2^30.
+ */
+arb_status arb_phase_lens_tokens(arb_ctx *ctx, int32_t batch, const int32_t *step_lens,
+                                 const uint8_t *decisions /* nullable */, int32_t want, int32_t n_tokens, int32_t *out,
+                                 arb_stream_t stream);
+
+/*
  * Synchronise `stream`, read the device status word into *bits (nullable) and clear it together
  * with the split-KV arrival counters.  Returns ARB_OK if the word was zero, else
  * ARB_ERR_DEVICE_STATUS.

@@ -34,7 +34,7 @@ MAX_CLASSES = 16
 EXPORTS = ("arb_create", "arb_destroy", "arb_attn_workspace_bytes", "arb_attn", "arb_attn_host",
            "arb_attn_host_begin", "arb_attn_host_wait",
            "arb_attn_decode_static",
-           "arb_route", "arb_rollback", "arb_policy", "arb_route_classes", "arb_kv_append", "arb_kv_append_e4m3", "arb_attn_decode_e4m3", "arb_phase_lens", "arb_spearman",
+           "arb_route", "arb_rollback", "arb_policy", "arb_route_classes", "arb_kv_append", "arb_kv_append_e4m3", "arb_attn_decode_e4m3", "arb_phase_lens", "arb_phase_lens_tokens", "arb_spearman",
            "arb_poll_status", "arb_launch_count", "arb_status_string")
 
 
@@ -75,6 +75,8 @@ lib.arb_spearman.restype = ctypes.c_int
 lib.arb_spearman.argtypes = [_vp, _i32, _vp, _vp, _vp, _vp]
 lib.arb_phase_lens.restype = ctypes.c_int
 lib.arb_phase_lens.argtypes = [_vp, _i32, _vp, _vp, _i32, _i32, _vp, _vp]
+lib.arb_phase_lens_tokens.restype = ctypes.c_int
+lib.arb_phase_lens_tokens.argtypes = [_vp, _i32, _vp, _vp, _i32, _i32, _vp, _vp]
 lib.arb_policy.restype = ctypes.c_int
 lib.arb_policy.argtypes = [_vp, _i32, _i32, _vp, _vp, _f, _i32, _vp, _vp, _vp]
 lib.arb_route_classes.restype = ctypes.c_int
@@ -317,6 +319,17 @@ class Context:
         st = lib.arb_phase_lens(self._h, step_lens.shape[0], _dev(step_lens, "step_lens", torch.int32), dp, int(want),
                                 int(t), _dev(out, "out", torch.int32), _stream_ptr(stream))
         _check(st, "arb_phase_lens")
+        return out
+
+    def phase_lens_tokens(self, step_lens, n_tokens: int, decisions=None, want: int = 1, out=None, stream=None):
+        """out int32 [n_tokens, B]: row t = phase_lens(..., t=t), all rows in one launch."""
+        B = step_lens.shape[0]
+        if out is None:
+            out = torch.empty(n_tokens, B, dtype=torch.int32, device=step_lens.device)
+        dp = None if decisions is None else _dev(decisions, "decisions", torch.uint8)
+        st = lib.arb_phase_lens_tokens(self._h, B, _dev(step_lens, "step_lens", torch.int32), dp, int(want), int(n_tokens),
+                                       _dev(out, "out", torch.int32), _stream_ptr(stream))
+        _check(st, "arb_phase_lens_tokens")
         return out
 
     # -- arb_policy ---------------------------------------------------------------------------

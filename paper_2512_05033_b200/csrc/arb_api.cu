@@ -461,6 +461,16 @@ arb_status arb_phase_lens(arb_ctx *ctx, int32_t batch, const int32_t *step_lens,
                              reinterpret_cast<cudaStream_t>(stream));
 }
 
+arb_status arb_phase_lens_tokens(arb_ctx *ctx, int32_t batch, const int32_t *step_lens, const uint8_t *decisions,
+                                 int32_t want, int32_t n_tokens, int32_t *out, arb_stream_t stream) {
+    if (ctx == nullptr || batch < 0 || n_tokens < 0) return ARB_ERR_INVALID_ARG;
+    if (batch == 0 || n_tokens == 0) return ARB_OK;
+    if (!step_lens || !out) return ARB_ERR_INVALID_ARG;
+    if ((long long)batch * n_tokens > (1ll << 30)) return ARB_ERR_UNSUPPORTED;
+    return launch_phase_lens_tokens(reinterpret_cast<Ctx *>(ctx), batch, step_lens, decisions, want, n_tokens, out,
+                                    reinterpret_cast<cudaStream_t>(stream));
+}
+
 arb_status arb_policy(arb_ctx *ctx, int32_t kind, int32_t n_steps, const float *s_d, const float *s_t, float tau,
                       int32_t budget, uint8_t *decisions, arb_policy_stats *stats, arb_stream_t stream) {
     if (ctx == nullptr || n_steps < 0) return ARB_ERR_INVALID_ARG;

@@ -225,6 +225,8 @@ arb_status launch_decode_static(const arb_attn_params &p, const void *q, const v
                                 void *out, uint32_t *device_status, cudaStream_t stream);
 arb_status launch_phase_lens(Ctx *ctx, int batch, const int32_t *step_lens, const uint8_t *decisions, int want, int t,
                              int32_t *out, cudaStream_t stream);
+arb_status launch_phase_lens_tokens(Ctx *ctx, int batch, const int32_t *step_lens, const uint8_t *decisions, int want,
+                                    int n_tokens, int32_t *out, cudaStream_t stream);
 arb_status launch_spearman(Ctx *ctx, int n, const float *x, const float *y, double *rho, cudaStream_t stream);
 arb_status launch_policy(Ctx *ctx, int kind, int n_steps, const float *s_d, const float *s_t, float tau, int budget,
                          uint8_t *decisions, arb_policy_stats *stats, cudaStream_t stream);

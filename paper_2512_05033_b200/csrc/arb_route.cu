@@ -90,7 +90,27 @@ __global__ void phase_lens_kernel(int batch, const int32_t *__restrict__ step_le
     out[b] = !in ? 0 : (t < 0 ? n : (t < n ? 1 : 0));
 }
 
+// The same for every token of a step that is decoded token by token: out[t][b], t < n_tokens, in one launch.
+__global__ void phase_lens_tokens_kernel(int batch, const int32_t *__restrict__ step_lens,
+                                         const uint8_t *__restrict__ decisions, int want, int n_tokens,
+                                         int32_t *__restrict__ out) {
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= batch * n_tokens) return;
+    const int t = i / batch, b = i - t * batch;
+    const bool in = decisions == nullptr || ((decisions[b] != 0) == (want != 0));
+    out[i] = (in && t < step_lens[b]) ? 1 : 0;
+}
+
 }  // namespace
+
+arb_status launch_phase_lens_tokens(Ctx *ctx, int batch, const int32_t *step_lens, const uint8_t *decisions, int want,
+                                    int n_tokens, int32_t *out, cudaStream_t stream) {
+    const long long n = (long long)batch * n_tokens;
+    phase_lens_tokens_kernel<<<(unsigned)((n + 255) / 256), 256, 0, stream>>>(batch, step_lens, decisions, want, n_tokens,
+                                                                             out);
+    ctx->launches++;
+    return cudaGetLastError() == cudaSuccess ? ARB_OK : ARB_ERR_CUDA;
+}
 
 arb_status launch_phase_lens(Ctx *ctx, int batch, const int32_t *step_lens, const uint8_t *decisions, int want, int t,
                              int32_t *out, cudaStream_t stream) {

@@ -13,7 +13,7 @@ work it causes:
                  drops z_d and absorbs z_t
   target cache   absorbs accepted draft steps as one chunk; generates z_t token by token for the escalated
 
-Which sequences take part in a phase comes from arb_phase_lens on the device.  A round is therefore a fixed
+Which sequences take part in a phase comes from arb_phase_lens / arb_phase_lens_tokens on the device.  A round is therefore a fixed
 list of kernel launches for given maximum step lengths and can be captured in a CUDA graph.
 """
 from __future__ import annotations
@@ -48,6 +48,9 @@ class StepLoop:
         dev = draft.seq_lens.device
         self.B = B
         self.lens = torch.zeros(B, dtype=torch.int32, device=dev)       # lengths of the call in flight
+        # ... of every token of a step that is generated token by token (one row per token)
+        self.token_lens = {"draft.gen": torch.zeros(self.nd, B, dtype=torch.int32, device=dev),
+                           "target.gen": torch.zeros(self.nt, B, dtype=torch.int32, device=dev)}
         self.scores = torch.empty(B, dtype=torch.float32, device=dev)
         self.decisions = torch.empty(B, dtype=torch.uint8, device=dev)
         self.out = {}                                                    # last outputs of every phase, by name
@@ -64,9 +67,9 @@ class StepLoop:
     def _generate(self, name: str, c: Cache, step_lens, decisions, want: int, n_max: int, q, k_new, v_new):
         """Token-by-token generation of a step by the model that owns `c`: q, k_new, v_new are [n_max, B, ...];
         at token t only sequences that take part and have t < step_lens[b] are active."""
+        lens = self.ctx.phase_lens_tokens(step_lens, n_max, decisions, want=want, out=self.token_lens[name])
         for t in range(n_max):
-            self.ctx.phase_lens(step_lens, decisions, want=want, t=t, out=self.lens)
-            self._absorb(f"{name}[{t}]", c, k_new[t], v_new[t], q[t], self.lens, 1)
+            self._absorb(f"{name}[{t}]", c, k_new[t], v_new[t], q[t], lens[t], 1)
 
     # -- one round ---------------------------------------------------------------------------------
     def round(self, step_d, step_t, hidden, acts):

@@ -113,3 +113,6 @@ def test_phase_lens_matches_oracle():
             for t in (-1, 0, 3, 8):
                 got = c.phase_lens(step.cuda(), None if decisions is None else decisions.cuda(), want=want, t=t)
                 assert np.array_equal(got.cpu().numpy(), oracle.phase_lens(step, decisions, want=want, t=t))
+            table = c.phase_lens_tokens(step.cuda(), 9, None if decisions is None else decisions.cuda(), want=want)
+            for t in range(9):   # one launch for all tokens of a step: row t is the call for token t
+                assert np.array_equal(table[t].cpu().numpy(), oracle.phase_lens(step, decisions, want=want, t=t))

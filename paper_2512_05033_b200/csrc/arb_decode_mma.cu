@@ -47,26 +47,29 @@ namespace arb {
 namespace {
 
 constexpr int kD = 128;
-constexpr int kConsWarps = 4;
-constexpr int kConsThreads = kConsWarps * 32;
-constexpr int kThreads = kConsThreads + 32;
+constexpr int kMaxConsWarps = 5;
 constexpr int kGroup = 1;       // pages per consumer work group: with 16 stages every warp has two groups in flight
 constexpr int kBatch = 16;      // producer lanes issuing side by side
-constexpr int kRingBytes = 64 * 1024;
-// what differs between the bf16 cache and the E4M3 cache in the ring
+// what differs between the bf16 cache and the E4M3 cache: the ring, and the number of consumer warps.  The E4M3 path
+// is bound by its consumers (every code is widened to f16 on the way to the tensor core), so large calls run five.
 template <bool E4M3>
 struct Fmt {
     static constexpr int kTileBytes = kPage * kD * (E4M3 ? 1 : 2);   // 4 KB (two halves of 16 rows x 64 bf16) or
                                                                      // 2 KB (one box of 16 rows x 128 codes)
     static constexpr int kHalfTile = kTileBytes / 2;
-    static constexpr int kStages = kRingBytes / kTileBytes;          // 16 or 32
+    // consumer warps of a large call (two CTAs per SM stream at the memory system's pace); a small call, whose
+    // pace is set by latencies, runs four either way (five are slower there: 7.3 against 7.0 us per call)
+    static constexpr int kLargeCallWarps = E4M3 ? 5 : 4;
+    static constexpr int kStages = E4M3 ? 40 : 16;                   // 64 KB of bf16 tiles, 80 KB of E4M3 tiles
+    static constexpr int kRingBytes = kStages * kTileBytes;
+    static_assert(kLargeCallWarps <= kMaxConsWarps, "warp records are sized for kMaxConsWarps");
+    // a ring stage must always belong to the same warp
+    static_assert(kStages % (kLargeCallWarps * 2 * kGroup) == 0 && kStages % (4 * 2 * kGroup) == 0, "stage ownership");
 };
 constexpr int kMinChunk = 4;
 constexpr int kCtasPerSm = 2;
 constexpr int kParked = 2;      // segment results parked in shared memory before they are written
 constexpr int kSmallCallPages = 64;   // up to this many pages per SM a call runs one CTA per SM
-static_assert(Fmt<false>::kStages % (kConsWarps * 2 * kGroup) == 0 && Fmt<true>::kStages % (kConsWarps * 2 * kGroup) == 0,
-              "a ring stage must always belong to the same warp");
 static_assert(kBatch <= Fmt<false>::kStages, "two producer lanes of one turn must never wait on the same stage: the later "
                                             "one would be two phases ahead of the barrier and a parity wait cannot tell");
 
@@ -109,14 +112,14 @@ template <int G>
 struct Cfg {
     static constexpr int GP = (G + 3) / 4 * 4;
     static constexpr int REC = G * kD + 2 * GP;            // [m[GP] | l[GP] | o[G][D]]
-    static constexpr int OSM_BYTES = kConsWarps * REC * 4;
+    static constexpr int OSM_BYTES = kMaxConsWarps * REC * 4;
     static constexpr int PARK_BYTES = kParked * REC * 4;
 };
 
 template <int G, bool E4M3>
 size_t smem_bytes(int batch) {
     using C = Cfg<G>;
-    return 1024 + kRingBytes + C::OSM_BYTES + C::PARK_BYTES + sizeof(Tail<E4M3>) + sizeof(int) * (3 * (size_t)batch + 2);
+    return 1024 + Fmt<E4M3>::kRingBytes + C::OSM_BYTES + C::PARK_BYTES + sizeof(Tail<E4M3>) + sizeof(int) * (3 * (size_t)batch + 2);
 }
 
 struct Segment {
@@ -242,12 +245,15 @@ __device__ __forceinline__ uint32_t tile_off(int r, int c) {
     else return (uint32_t)((c >> 3) * Fmt<false>::kHalfTile + r * 128 + (((c & 7) ^ (r & 7)) << 4));
 }
 
-template <int G, bool E4M3>
-__global__ void __launch_bounds__(kThreads, kCtasPerSm)
+template <int G, bool E4M3, int CW>
+__global__ void __launch_bounds__(CW * 32 + 32, kCtasPerSm)
 decode_mma_kernel(const Args a, const __grid_constant__ CUtensorMap k_map, const __grid_constant__ CUtensorMap v_map) {
     using C = Cfg<G>;
     using Tail = arb::Tail<E4M3>;
     constexpr int kStages = Fmt<E4M3>::kStages, kTileBytes = Fmt<E4M3>::kTileBytes, kHalfTile = Fmt<E4M3>::kHalfTile;
+    constexpr int kRingBytes = Fmt<E4M3>::kRingBytes;
+    constexpr int kCW = CW, kCT = CW * 32, kNT = kCT + 32;   // consumer warps, their threads, + the producer warp
+    static_assert(CW <= kMaxConsWarps && kStages % (CW * 2 * kGroup) == 0, "stage ownership");
     constexpr int GP = C::GP, REC = C::REC;
     static_assert(G >= 1 && G <= 8, "query heads of a group occupy rows 0..7 of the 16-row tile");
 
@@ -268,7 +274,7 @@ decode_mma_kernel(const Args a, const __grid_constant__ CUtensorMap k_map, const
     // arrival counters comes after it (see the CUDA-core decode kernel for the ordering argument).
     let_successor_start();
 
-    if (tid == kConsThreads) {  // the producer warp's first lane: descriptors on their way before the first copy needs them
+    if (tid == kCT) {  // the producer warp's first lane: descriptors on their way before the first copy needs them
         asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&k_map)) : "memory");
         asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&v_map)) : "memory");
     }
@@ -282,7 +288,7 @@ decode_mma_kernel(const Args a, const __grid_constant__ CUtensorMap k_map, const
         pref[0] = 0;
         row0[0] = 0;
     }
-    for (int b = tid; b < B; b += kThreads) {
+    for (int b = tid; b < B; b += kNT) {
         const int n = a.q_lens[b], L = a.seq_lens[b];
         int pages = 0;
         if (n == 1) {
@@ -338,7 +344,7 @@ decode_mma_kernel(const Args a, const __grid_constant__ CUtensorMap k_map, const
     const int r1 = min(total, r0 + chunk);
     volatile int *abort = &tail->abort;
 
-    if (warp == kConsWarps) {
+    if (warp == kCW) {
         // ================================ producer warp ==========================================
         uint32_t c = 0;
         int cur = r0;
@@ -449,13 +455,13 @@ decode_mma_kernel(const Args a, const __grid_constant__ CUtensorMap k_map, const
                 if (may_early && !early_known) early_known = set_is_free();
                 tail->early = early_known ? 1 : 0;
             }
-            named_barrier(1, kConsThreads);
+            named_barrier(1, kCT);
             if (!tail->early) ensure_wait();
             for (int j = 0; j < n_parked; ++j) {
                 if (pk[j].nparts == 1) continue;
                 const float *rec = park + j * REC;
                 const size_t slot = (size_t)pk[j].bk + blockIdx.x;
-                for (int idx = tid; idx < G * kD / 4; idx += kConsThreads)
+                for (int idx = tid; idx < G * kD / 4; idx += kCT)
                     reinterpret_cast<float4 *>(a.part_o + slot * G * kD)[idx] =
                         reinterpret_cast<const float4 *>(rec + 2 * GP)[idx];
                 if (tid < G) {
@@ -469,11 +475,11 @@ decode_mma_kernel(const Args a, const __grid_constant__ CUtensorMap k_map, const
             for (int j = 0; j < n_parked; ++j) {
                 if (pk[j].nparts != 1) continue;
                 const float *rec = park + j * REC;
-                for (int idx = tid; idx < G * kD; idx += kConsThreads)
+                for (int idx = tid; idx < G * kD; idx += kCT)
                     reinterpret_cast<__nv_bfloat16 *>(a.out)[pk[j].out_base + idx] =
                         __float2bfloat16_rn(rec[2 * GP + idx] / rec[GP + idx / kD]);
             }
-            named_barrier(1, kConsThreads);  // parking slots are free again
+            named_barrier(1, kCT);  // parking slots are free again
             n_parked = 0;
         }
     };
@@ -510,7 +516,7 @@ decode_mma_kernel(const Args a, const __grid_constant__ CUtensorMap k_map, const
 
         const int seg_pages = s.pg1 - s.pg0;
         const int ngroups = (seg_pages + kGroup - 1) / kGroup;
-        for (int gi = warp; gi < ngroups; gi += kConsWarps) {
+        for (int gi = warp; gi < ngroups; gi += kCW) {
             const int p0 = s.pg0 + gi * kGroup;
             const int npg = min(kGroup, s.pg1 - p0);
             const int ntok = min(s.L - p0 * kPage, npg * kPage);
@@ -658,16 +664,16 @@ decode_mma_kernel(const Args a, const __grid_constant__ CUtensorMap k_map, const
             if (tq == 0) { rec[gq] = m_run; rec[GP + gq] = l_run; }
         }
         if (n_parked == kParked) flush(false);  // uniform across the consumer threads
-        named_barrier(1, kConsThreads);
+        named_barrier(1, kCT);
         float *dst = park + n_parked * REC;
-        for (int idx = tid; idx < G * kD; idx += kConsThreads) {
+        for (int idx = tid; idx < G * kD; idx += kCT) {
             const int h = idx / kD;
             float M = -INFINITY;
 #pragma unroll
-            for (int w = 0; w < kConsWarps; ++w) M = fmaxf(M, osm[w * REC + h]);
+            for (int w = 0; w < kCW; ++w) M = fmaxf(M, osm[w * REC + h]);
             float l = 0.f, acc = 0.f;
 #pragma unroll
-            for (int w = 0; w < kConsWarps; ++w) {
+            for (int w = 0; w < kCW; ++w) {
                 const float ff = fast_exp2(osm[w * REC + h] - M);  // 0 for a warp that had no group
                 l = fmaf(ff, osm[w * REC + GP + h], l);
                 acc = fmaf(ff, osm[w * REC + 2 * GP + idx], acc);
@@ -680,7 +686,7 @@ decode_mma_kernel(const Args a, const __grid_constant__ CUtensorMap k_map, const
         pk[n_parked].c_first = s.c_first;
         pk[n_parked].out_base = ((size_t)qrow * a.Hq + s.kvh * G) * kD;
         ++n_parked;
-        named_barrier(1, kConsThreads);  // warp records are free for the next segment
+        named_barrier(1, kCT);  // warp records are free for the next segment
     }
     if (n_parked > 0) flush(true);  // final results stay parked until the epilogue
 
@@ -693,7 +699,7 @@ decode_mma_kernel(const Args a, const __grid_constant__ CUtensorMap k_map, const
     for (int j = 0; j < n_parked; ++j) {
         if (pk[j].nparts != 1) continue;
         const float *rec = park + j * REC;
-        for (int idx = tid; idx < G * kD; idx += kConsThreads)
+        for (int idx = tid; idx < G * kD; idx += kCT)
             reinterpret_cast<__nv_bfloat16 *>(a.out)[pk[j].out_base + idx] =
                 __float2bfloat16_rn(rec[2 * GP + idx] / rec[GP + idx / kD]);
     }
@@ -865,10 +871,12 @@ template <int G, bool E4M3>
 arb_status launch_one(Ctx *ctx, const Args &a, CombineArgs ca, const CUtensorMap &km, const CUtensorMap &vm,
                       bool overlap, cudaStream_t stream) {
     const size_t smem = smem_bytes<G, E4M3>(a.batch);
+    constexpr int kLarge = Fmt<E4M3>::kLargeCallWarps;
     static bool attr_set[64] = {};
     if (!attr_set[ctx->device & 63]) {
-        if (cudaFuncSetAttribute(decode_mma_kernel<G, E4M3>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 (int)smem_bytes<G, E4M3>(kMaxBatch)) != cudaSuccess)
+        const int most = (int)smem_bytes<G, E4M3>(kMaxBatch);
+        if (cudaFuncSetAttribute(decode_mma_kernel<G, E4M3, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, most) != cudaSuccess ||
+            cudaFuncSetAttribute(decode_mma_kernel<G, E4M3, kLarge>, cudaFuncAttributeMaxDynamicSharedMemorySize, most) != cudaSuccess)
             return ARB_ERR_CUDA;
         attr_set[ctx->device & 63] = true;
     }
@@ -882,12 +890,15 @@ arb_status launch_one(Ctx *ctx, const Args &a, CombineArgs ca, const CUtensorMap
     const bool small = page_bound <= (long long)ctx->num_sms * kSmallCallPages;
     const int grid = small ? ctx->num_sms : ctx->num_sms * kCtasPerSm;
     cfg.gridDim = dim3(grid);
-    cfg.blockDim = dim3(kThreads);
+    const int cons_warps = small ? 4 : kLarge;
+    cfg.blockDim = dim3(cons_warps * 32 + 32);
     cfg.dynamicSmemBytes = smem;
     cfg.stream = stream;
     cfg.attrs = attr;
     cfg.numAttrs = overlap ? 1 : 0;
-    if (cudaLaunchKernelEx(&cfg, decode_mma_kernel<G, E4M3>, a, km, vm) != cudaSuccess) return ARB_ERR_CUDA;
+    const cudaError_t err = cons_warps == 4 ? cudaLaunchKernelEx(&cfg, decode_mma_kernel<G, E4M3, 4>, a, km, vm)
+                                            : cudaLaunchKernelEx(&cfg, decode_mma_kernel<G, E4M3, kLarge>, a, km, vm);
+    if (err != cudaSuccess) return ARB_ERR_CUDA;
     ctx->launches++;
     // the combine kernel, always a programmatic dependent of the decode kernel
     ca.decode_grid = grid;

@@ -379,7 +379,7 @@ def run_e2e(ctx, work: DecodeWorkload, steps: int, world: int):
     gbs = lambda t: round(world * work.bytes["kv"] * work.layers / t / 1e9, 1)  # noqa: E731
     h2d = (qh.numel() * qh.element_size() + bth.numel() * 4 + slh.numel() * 4 + qlh.numel() * 4) * work.layers
     d2h = qh.numel() * qh.element_size() * work.layers
-    # Two ways of issuing the same pipelined calls.  Which is faster depends on the box: the flagged calls read their
+    # Two ways of issuing the same pipelined calls.  Which is faster depends on the host: the flagged calls read their
     # inputs over the bus from page-locked host memory, and that has been seen at 17 and at 29 us per call on
     # different hosts, while the staged copies are steady at 24.  The headline is the better of the two, named.
     flagged_wins = dt_flag <= dt_staged

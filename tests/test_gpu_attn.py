@@ -456,6 +456,9 @@ E4M3_CASES = [
     (1, 5, 1, [40000]),                                        # one long sequence over every CTA
     (2, 16, 2, [2100, 900]),                                   # g = 8
     (5, 8, 2, [100, 1, 300, 1, 47]),                           # with idle slots (below)
+    # block tables wide enough for the launcher to treat the call as a large one (five consumer warps per CTA)
+    (8, 12, 2, [12000, 9000, 700, 33, 5000, 11000, 1, 2500]),  # g = 6
+    (4, 16, 2, [20000, 15000, 100, 9000]),                     # g = 8
 ]
 
 

@@ -57,6 +57,11 @@ constexpr int kSortMaxBatch = 256;          // up to this batch size sequences a
 constexpr int kSplitMinTiles = 160;
 constexpr int kSplitPartTiles = 96;
 constexpr int kSplitMaxParts = 32;          // a warp's lanes cover the parts in the combine
+// A call with few work items (a small batch of short steps) leaves most SMs idle while each item walks its keys at
+// the pace of one row tile's chain.  Such a call is cut the same way, down to parts of kFillPartTiles tiles, for
+// sequences of at least kFillMinTiles tiles.
+constexpr int kFillMinTiles = 16;
+constexpr int kFillPartTiles = 8;
 constexpr size_t kSlotFloats = (size_t)kBM * kD + 2 * kBM;   // one row tile's partial: O as [32 groups of 4 dims][128 rows][4],
                                                              // so that the rows' 16-byte pieces lie side by side; then (max, sum) [128][2]
 
@@ -74,6 +79,8 @@ struct MmaArgs {
                         // both zeroed on the stream before the launch
     float *split_ws;    // partial results of split sequences, kSlotFloats per (item, row tile)
     int split_cap;      // slots that fit there
+    int fill_ctas;      // CTAs a call should keep busy: a call with fewer than half as many work items has its
+                        // sequences cut over their keys as well (0: never)
     float scale_log2;
 };
 
@@ -302,6 +309,22 @@ __device__ void make_plan(const MmaArgs &a, Plan pl, int tid, int nthreads, int 
     if (warp == 0) {
         // in serving order: parts (granted while the partial slots last), partial slots and work items;
         // and, in batch order, the q rows
+        // does the call fill the machine as it is?  (work items and their KV tiles without any split)
+        int items0 = 0, tiles0 = 0;
+        for (int r0 = 0; r0 < B; r0 += 32) {
+            const int r = r0 + lane;
+            if (r < B && pl.pairs[r] > 0) {
+                items0 += Hkv * pl.pairs[r];
+                tiles0 += Hkv * pl.pairs[r] * ((pl.key[r] + kBN - 1) / kBN);
+            }
+        }
+#pragma unroll
+        for (int off = 16; off >= 1; off >>= 1) {
+            items0 += __shfl_xor_sync(0xffffffffu, items0, off);
+            tiles0 += __shfl_xor_sync(0xffffffffu, tiles0, off);
+        }
+        const bool fill = a.fill_ctas > 0 && items0 > 0 && 2 * items0 <= a.fill_ctas;
+        const int fill_part = max(kFillPartTiles, (tiles0 + max(a.fill_ctas, 1) - 1) / max(a.fill_ctas, 1));
         int carry_p = 0, carry_r = 0, carry_s = 0;
         for (int r0 = 0; r0 < B; r0 += 32) {
             const int r = r0 + lane;
@@ -313,6 +336,9 @@ __device__ void make_plan(const MmaArgs &a, Plan pl, int tid, int nthreads, int 
                 if (nt > kSplitMinTiles) {
                     want = min((nt + kSplitPartTiles - 1) / kSplitPartTiles, kSplitMaxParts);
                     slots = Hkv * pairs * want * 2;
+                } else if (fill && nt >= kFillMinTiles) {
+                    want = min((nt + fill_part - 1) / fill_part, kSplitMaxParts);
+                    slots = want > 1 ? Hkv * pairs * want * 2 : 0;
                 }
             }
             int vs = slots;
@@ -874,7 +900,7 @@ arb_status launch_one(Ctx *ctx, const MmaArgs &a, const CUtensorMap &km, const C
     ctx->launches++;
     if (cudaGetLastError() != cudaSuccess) return ARB_ERR_CUDA;
     // the merge of split sequences, when the block table is long enough for a sequence to be split at all
-    if (a.split_cap > 0 && ((long long)a.max_pages * kPage + kBN - 1) / kBN > kSplitMinTiles) {
+    if (a.split_cap > 0) {
         const size_t csmem = sizeof(int) * (7 * (size_t)a.batch + 2);
         chunk_combine_kernel<G><<<4 * ctx->num_sms, kCombineThreads, csmem, stream>>>(a);
         ctx->launches++;
@@ -916,7 +942,13 @@ arb_status launch_chunk_mma(Ctx *ctx, const arb_attn_params &p, const void *q, c
     a.work_counter = ctx->rot + (size_t)kRotSets * kRotCounters + kRotSets + 1;
     a.split_ws = ctx->chunk_ws;
     a.split_cap = (int)(ctx->chunk_ws_bytes / (kSlotFloats * sizeof(float)));
-    if (((long long)p.max_pages_per_seq * kPage + kBN - 1) / kBN <= kSplitMinTiles) a.split_cap = 0;
+    // Can a sequence of this call be split at all?  Long ones from kSplitMinTiles tiles on; shorter ones only in a call
+    // whose work items may fail to fill the machine.  The host knows the rows: at most `batch` of them are decode rows,
+    // the others sit in row-tile pairs of 256, one work item per pair and KV head.
+    const long long max_tiles = ((long long)p.max_pages_per_seq * kPage + kBN - 1) / kBN;
+    const long long least_items = (long long)p.num_kv_heads * (((long long)p.total_q - p.batch) * (p.num_q_heads / p.num_kv_heads) / (2 * kBM));
+    a.fill_ctas = (2 * least_items <= ctx->num_sms && max_tiles >= kFillMinTiles) ? ctx->num_sms : 0;
+    if (max_tiles <= kSplitMinTiles && a.fill_ctas == 0) a.split_cap = 0;
     if (cudaMemsetAsync(a.work_counter, 0, 2 * sizeof(int), stream) != cudaSuccess) return ARB_ERR_CUDA;
     const float scale = p.softmax_scale > 0.f ? p.softmax_scale : 1.0f / sqrtf((float)p.head_dim);
     a.scale_log2 = scale * 1.4426950408889634f;

@@ -60,8 +60,8 @@ constexpr int kSplitMaxParts = 32;          // a warp's lanes cover the parts in
 // A call with few work items (a small batch of short steps) leaves most SMs idle while each item walks its keys at
 // the pace of one row tile's chain.  Such a call is cut the same way, down to parts of kFillPartTiles tiles, for
 // sequences of at least kFillMinTiles tiles.
-constexpr int kFillMinTiles = 16;
-constexpr int kFillPartTiles = 8;
+constexpr int kFillMinTiles = 8;
+constexpr int kFillPartTiles = 4;
 constexpr size_t kSlotFloats = (size_t)kBM * kD + 2 * kBM;   // one row tile's partial: O as [32 groups of 4 dims][128 rows][4],
                                                              // so that the rows' 16-byte pieces lie side by side; then (max, sum) [128][2]
 

@@ -70,7 +70,7 @@ CHUNK_CASES = [
     (3, 12, 2, 128, BF, [2, 17, 300], [2, 3, 2]),            # smallest chunks: 12 and 18 rows; the chunk is the whole sequence
     (2, 8, 8, 128, BF, [40, 300], [2, 9]),                   # g = 1: 2 and 9 rows in a 128-row tile
     (3, 16, 2, 128, BF, [33, 1000, 129], [3, 7, 1]),         # g = 8: 24 and 56 rows beside a decode row
-    # few work items and sequences of 16 KV tiles and more: the call is cut over the keys to fill the SMs
+    # few work items and sequences of 8 KV tiles and more: the call is cut over the keys to fill the SMs
     (3, 12, 2, 128, BF, [5000, 2500, 300], [24, 9, 1]),      # parts of two chunk sequences beside a decode row
     (2, 32, 8, 128, BF, [6000, 3000], [40, 64]),             # g = 4, one and two row tiles per sequence
     (1, 8, 2, 64, F32, [528], [16]),                         # the tiny config: 16-token chunk, prefix 512

@@ -233,7 +233,10 @@ arb_status arb_attn_host_wait(arb_ctx *ctx);
  * other) race on it and corrupt each other's results; ARB_ATTN_OVERLAP_PREVIOUS is therefore
  * rejected with ARB_ERR_INVALID_ARG.  The current device must be the one the pointers live on.
  * The first call on a device looks up the array's device address and sets the kernel's
- * shared-memory attribute; make that first call before any stream capture begins.
+ * shared-memory attribute; make that first call before any stream capture begins.  That set-up is
+ * serialised inside the library, so first calls from several host threads are safe.  With
+ * device_status == NULL the ARB_DEV_* bits of a call (a wait that timed out included) go to a word inside
+ * the array that no API reads and that the next call clears: pass a word if you need to see them.
  */
 arb_status arb_attn_decode_static(const arb_attn_params *params, const void *q, const void *k_pages,
                                   const void *v_pages, const int32_t *block_table,
@@ -241,9 +244,10 @@ arb_status arb_attn_decode_static(const arb_attn_params *params, const void *q, 
                                   uint32_t *device_status /* nullable */, arb_stream_t stream);
 
 /*
- * Router head and threshold decision (Section 4.2: the score is the likelihood that the target
- * outperforms the draft, reject iff y_hat > tau; Algorithm 1: accept iff y_hat <= tau; the
- * classification head reads the final token's embedding).  A two-class softmax head (accept = 0,
+ * Router head and threshold decision (Section 4.2, Figure 1, Algorithm 1 "Routing decision": the score
+ * estimates the probability that escalating improves the step; the draft step is rejected iff
+ * y_hat > tau and accepted iff y_hat <= tau; Section 4.2 "Training": the head reads the hidden state of the
+ * step's final token).  A two-class softmax head (accept = 0,
  * escalate = 1) is the same function with w = w1 - w0 and b = b1 - b0.
  *
  *   hidden     [n_steps, hidden_dim]; row i is the final-layer hidden state of the last token of
@@ -322,7 +326,8 @@ arb_status arb_route_classes(arb_ctx *ctx, int32_t dtype, int32_t mode, int32_t 
  *   v_new      [total_new, Hkv, D], packed by sequence in batch order: sequence b owns new_lens[b] rows.
  *   seq_lens   int32 [B]: tokens held BEFORE the call.  Token j of sequence b goes to position
  *              seq_lens[b] + j, i.e. page block_table[b][pos / P], slot pos % P.  With update_lens != 0
- *              seq_lens[b] becomes seq_lens[b] + new_lens[b] (by a second small kernel), which is the
+ *              seq_lens[b] becomes seq_lens[b] + new_lens[b] (written by the CTA of the append kernel that
+ *              finishes last, once every CTA has read the old lengths), which is the
  *              value arb_attn expects when it is called with q_lens = new_lens.
  *   new_lens   int32 [B], >= 0; total_new >= their sum (rows beyond the sum are ignored).
  * A sequence whose new tokens do not fit under its block-table row, or whose target pages lie outside

@@ -192,7 +192,7 @@ arb_status arb_attn(arb_ctx *ctx, const arb_attn_params *params, const void *q, 
         if (tensor_cores && decode_mma_supported(*params))
             st = launch_decode_mma(c, *params, q, k_pages, v_pages, block_table, seq_lens, q_lens, out, s);
         else {
-            c->last_decode_shared_set0 = true;  // it uses workspace set 0 without a generation number
+            note_unnumbered_decode(c, decode_workspace_bytes(*params, c->num_sms));  // region 0, no generation number
             st = launch_decode(c, *params, q, k_pages, v_pages, block_table, seq_lens, q_lens, out, s);
         }
         if (st != ARB_OK) return st;

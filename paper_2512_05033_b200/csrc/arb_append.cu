@@ -9,8 +9,8 @@
 // is known on the host but the total number of new tokens; every CTA derives the row offsets from
 // new_lens (scan in shared memory) and checks each sequence once: new tokens that do not fit under the
 // block table, or that would land on a page outside the pool, leave that sequence untouched and set a
-// status bit.  Lengths are advanced by a second, one-CTA kernel, after every CTA of the first has read
-// them.
+// status bit.  Lengths are advanced inside the same kernel by the CTA that finishes last (an arrival counter
+// tells it, see advance_lens_when_last): by then every CTA has read the old lengths for the rows it placed.
 //
 // The quantising form writes an E4M3 cache (one byte per element: 1 sign, 4 exponent bits with bias 7, 3
 // mantissa bits, largest finite value 448): code = e4m3(x * inv_scale), the product in fp32, the conversion

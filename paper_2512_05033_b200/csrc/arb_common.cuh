@@ -61,7 +61,7 @@ struct Ctx {
     // per set and the generation of the newest completed call, all in one allocation
     int *rot = nullptr;
     uint32_t decode_gen = 1000;          // generation of the next tensor-core decode call
-    bool last_decode_shared_set0 = false; // the CUDA-core decode kernel used set 0 since then
+    uint32_t rot_wait_through = 0;        // tensor-core decode calls up to this generation wait for their predecessor
     double *spearman_acc = nullptr;       // three fp64 accumulators of arb_spearman
     float *chunk_ws = nullptr;            // partial results of split long sequences (step-chunk attention)
     size_t chunk_ws_bytes = 0;
@@ -69,6 +69,18 @@ struct Ctx {
 
 constexpr int kRotSets = 4;
 constexpr int kRotCounters = 1 << 16;
+
+// The decode workspace is cut into kRotSets + 1 regions of this size: region 0 for the decode kernels that take
+// no generation number, regions 1 .. kRotSets for the rotation of the tensor-core decode kernel.
+inline size_t rot_region_bytes(const Ctx *ctx) { return (ctx->workspace_bytes / (kRotSets + 1)) & ~size_t(255); }
+
+// A decode kernel without a generation number is about to use `bytes` of the workspace from its start.  Inside
+// region 0 it touches no rotation set.  Beyond it, it may lie over sets that later tensor-core calls would write
+// early: those of the next kRotSets generations wait (a later completion, which they would otherwise trust,
+// then implies this call's).
+inline void note_unnumbered_decode(Ctx *ctx, size_t bytes) {
+    if (bytes > rot_region_bytes(ctx)) ctx->rot_wait_through = ctx->decode_gen + (uint32_t)kRotSets - 1u;
+}
 
 // ---------------------------------------------------------------------------------------------
 // Element types

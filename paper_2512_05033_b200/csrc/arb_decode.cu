@@ -25,6 +25,8 @@
 // Split combine.  Partials of one (sequence, kv head) lie in consecutive workspace slots.  The CTA
 // that arrives last notes the job and, once its own pages are done and the ring is idle, pulls the
 // partials into shared memory with bulk copies and merges them there.
+#include <mutex>
+
 #include "arb_common.cuh"
 
 namespace arb {
@@ -677,16 +679,22 @@ __global__ void __launch_bounds__(kThreads, Cfg<T, D, G>::CTAS) decode_kernel(co
     }
 }
 
+// first-use set-up (function attributes, the static scratch address) may be reached from several host threads
+std::mutex g_setup_mutex;
+
 template <typename T, int D, int G>
 arb_status launch_one(Ctx *ctx, const DecodeArgs &args, bool overlap, cudaStream_t stream) {
     using C = Cfg<T, D, G>;
     const size_t smem = smem_bytes<T, D, G>(args.batch);
     static bool attr_set[64] = {};
-    if (!attr_set[ctx->device & 63]) {
-        if (cudaFuncSetAttribute(decode_kernel<T, D, G>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 (int)smem_bytes<T, D, G>(kMaxBatch)) != cudaSuccess)
-            return ARB_ERR_CUDA;
-        attr_set[ctx->device & 63] = true;
+    {
+        std::lock_guard<std::mutex> lock(g_setup_mutex);
+        if (!attr_set[ctx->device & 63]) {
+            if (cudaFuncSetAttribute(decode_kernel<T, D, G>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     (int)smem_bytes<T, D, G>(kMaxBatch)) != cudaSuccess)
+                return ARB_ERR_CUDA;
+            attr_set[ctx->device & 63] = true;
+        }
     }
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(ctx->num_sms * C::CTAS);
@@ -745,6 +753,7 @@ arb_status launch_decode_static(const arb_attn_params &p, const void *q, const v
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return ARB_ERR_CUDA;
     StaticSetup &su = g_static_setup[dev];
+    std::unique_lock<std::mutex> setup_lock(g_setup_mutex);
     if (!su.ready) {  // first call on this device: it is current, so the symbol resolves to its copy
         void *ptr = nullptr;
         if (cudaGetSymbolAddress(&ptr, g_static_scratch) != cudaSuccess || ptr == nullptr) {
@@ -758,6 +767,7 @@ arb_status launch_decode_static(const arb_attn_params &p, const void *q, const v
         su.num_sms = sms;
         su.ready = true;
     }
+    setup_lock.unlock();
     const int g = p.num_q_heads / p.num_kv_heads;
     const int gp = (g + 3) / 4 * 4;
     if ((long long)p.batch * p.num_kv_heads > kStaticMaxBk) return ARB_ERR_STATIC_LIMIT;

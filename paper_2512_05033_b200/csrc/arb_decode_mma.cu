@@ -27,8 +27,8 @@
 //
 // The same kernel, compiled a second time (template parameter E4M3), reads an E4M3 KV cache: one byte per
 // element, half the bytes of the bf16 cache per token -- the only way past the bf16 cache's HBM roofline.
-//   - a (page, kv head) tile is 16 rows x 128 bytes = 2 KB, one TMA box (128-byte swizzle); the ring has 32
-//     stages, so the bytes in flight per CTA stay the same;
+//   - a (page, kv head) tile is 16 rows x 128 bytes = 2 KB, one TMA box (128-byte swizzle); the ring has 40
+//     stages (80 KB in flight per CTA against 64 KB of bf16 tiles);
 //   - the codes are widened to f16, which holds every E4M3 value exactly (cvt.rn.f16x2.e4m3x2), and the
 //     products run as f16 MMAs (fp32 accumulate); q is converted bf16 -> f16 once per segment, P is rounded to
 //     f16 (11 significant bits) and summed after rounding;
@@ -943,32 +943,39 @@ arb_status launch_decode_tc(Ctx *ctx, const arb_attn_params &p, const void *q, c
     const int g = p.num_q_heads / p.num_kv_heads;
     const int gp = (g + 3) / 4 * 4;
     const size_t slots = (size_t)p.batch * p.num_kv_heads + (size_t)ctx->num_sms * kCtasPerSm;
-    // Workspace rotation.  Consecutive calls take consecutive generation numbers and use workspace set
-    // (generation mod sets): partials, (max, sum) records and arrival counters of their own.  A call
-    // may write its set without waiting for the previous call once the set's previous user
-    // (generation - sets) has published its completion.  With fewer than three sets that fit in the
-    // workspace, or right after a CUDA-core decode call (which uses set 0 unnumbered), it waits.
+    // Workspace rotation.  The workspace is cut into kRotSets + 1 regions of one fixed size, whatever the
+    // shape of the call: region 0 belongs to the decode kernels that take no generation number, regions
+    // 1 .. kRotSets are the rotation sets.  Consecutive calls take consecutive generation numbers and use set
+    // (generation mod kRotSets): partials and (max, sum) records of their own.  A call may write its set
+    // without waiting for the previous call once the set's previous user (generation - kRotSets) has published
+    // its completion.  Because a set always lies at the same place, that holds for any mix of shapes in a
+    // series.  A call whose partials do not fit in one region takes the whole workspace and waits; it may lie
+    // over every set, so the calls of the next kRotSets generations wait as well (until the window
+    // [generation - kRotSets, generation - 1] no longer reaches back to it, a completion inside the window says
+    // nothing about the large call).
     const size_t part_o_floats = (slots * g * p.head_dim + 63) & ~size_t(63);
     const size_t set_bytes = ((part_o_floats + slots * gp * 2) * sizeof(float) + 255) & ~size_t(255);
-    int sets = (int)(ctx->workspace_bytes / set_bytes);
-    if (sets > kRotSets) sets = kRotSets;
-    if (sets < 1) return ARB_ERR_WORKSPACE;
-    if ((long long)p.batch * p.num_kv_heads > kRotCounters) sets = 1;
+    if (set_bytes > ctx->workspace_bytes) return ARB_ERR_WORKSPACE;
+    const size_t region = rot_region_bytes(ctx);
     const uint32_t gen = ctx->decode_gen++;
-    const int set = (int)(gen % (uint32_t)sets);
+    const bool rotates = set_bytes <= region;
+    const int sets = rotates ? kRotSets : 1;
+    const int set = rotates ? (int)(gen % (uint32_t)kRotSets) : 0;
+    const size_t set_offset = rotates ? (size_t)(1 + set) * region : 0;
+    const bool force_wait = !rotates || (int32_t)(ctx->rot_wait_through - gen) >= 0;
+    if (!rotates) ctx->rot_wait_through = gen + (uint32_t)kRotSets;
     Args a;
     a.q = static_cast<const char *>(q);
     a.block_table = block_table;
     a.seq_lens = seq_lens;
     a.q_lens = q_lens;
     a.out = static_cast<char *>(out);
-    a.part_o = reinterpret_cast<float *>(ctx->workspace + (size_t)set * set_bytes);
+    a.part_o = reinterpret_cast<float *>(ctx->workspace + set_offset);
     a.part_ml = a.part_o + part_o_floats;
     a.done_gen = reinterpret_cast<unsigned *>(ctx->rot + (size_t)kRotSets * kRotCounters + kRotSets);
     a.gen = gen;
     a.sets = sets;
-    a.force_wait = ctx->last_decode_shared_set0 ? 1 : 0;
-    ctx->last_decode_shared_set0 = false;
+    a.force_wait = force_wait ? 1 : 0;
     a.status = ctx->status;
     a.batch = p.batch;
     a.Hq = p.num_q_heads;

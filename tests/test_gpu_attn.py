@@ -416,6 +416,60 @@ def test_overlap_flag_results():
         H.assert_close(o.double().cpu().numpy(), ref, BF, tight=3e-3)
 
 
+def test_overlap_flag_mixed_shapes():
+    """A flagged series whose calls differ in shape and kernel: draft-like (12/2 heads) and target-like (32/8)
+    tensor-core calls alternate, with a CUDA-core call (ARB_ATTN_NO_TENSOR_CORES) and an E4M3 call in every
+    round.  The workspace sets of the rotation must lie at the same place whatever the call's shape, or a
+    later call's early partials land on records an earlier call's combine is still reading.  Each call must
+    give the bits it gives alone, and match the oracle."""
+    from paper_2512_05033_b200 import binding
+    c = H.ctx()
+    F = binding.ATTN_OVERLAP_PREVIOUS
+    geo = [(4, 12, 2, [5000, 700, 3000, 64], F), (4, 32, 8, [2100, 4000, 33, 900], F),
+           (3, 28, 4, [3000, 150, 1024], F), (4, 12, 2, [1500, 2500, 17, 800], F | binding.ATTN_NO_TENSOR_CORES),
+           (6, 16, 2, [6000, 100, 2000, 1, 4100, 333], F)]
+    cpu_cases = [wl.small_attn_case(B, Hq, Hkv, 128, BF, sl, [1] * B, seed=170 + i)
+                 for i, (B, Hq, Hkv, sl, _) in enumerate(geo)]
+    cases = [d.to("cuda") for d in cpu_cases]
+    params = [c.params_for(d.q, d.k_pages, d.block_table, 1, flags=g[4]) for d, g in zip(cases, geo)]
+    # one E4M3 call in the series as well (same rotation, other kernel)
+    e_cpu = wl.small_attn_case(4, 12, 2, 128, BF, [3100, 513, 64, 1500], [1] * 4, seed=177)
+    kc = torch.from_numpy(oracle.e4m3_encode(e_cpu.k_pages, 1 / 0.012))
+    vc = torch.from_numpy(oracle.e4m3_encode(e_cpu.v_pages, 1 / 0.012))
+    e = e_cpu.to("cuda")
+    ekc, evc = kc.cuda(), vc.cuda()
+
+    def call(i, out=None):
+        d, p = cases[i], params[i]
+        return c.attn(d.q, d.k_pages, d.v_pages, d.block_table, d.seq_lens, d.q_lens, 1, out=out, params=p)
+
+    def call_e(out=None):
+        return c.attn_decode_e4m3(e.q, ekc, evc, 0.012, 0.012, e.block_table, e.seq_lens, e.q_lens, out=out, flags=F)
+
+    alone = []
+    for i in range(len(cases)):
+        alone.append(call(i))
+        torch.cuda.synchronize()
+    alone_e = call_e()
+    torch.cuda.synchronize()
+    outs = [torch.full_like(d.q, float("nan")) for d in cases]
+    out_e = torch.full_like(e.q, float("nan"))
+    for rep in range(50):                      # 300 calls in flight behind one another
+        for i in range(len(cases)):
+            call(i, outs[i])
+            if i == 2:
+                call_e(out_e)
+    assert c.poll_status() == 0
+    for a, b in zip(alone, outs):
+        assert torch.equal(a, b)
+    assert torch.equal(alone_e, out_e)
+    for d, o, g in zip(cpu_cases, outs, geo):
+        ref, _ = H.oracle_attn(d)
+        H.assert_close(o.double().cpu().numpy(), ref, BF, tight=1e-3 if g[4] & binding.ATTN_NO_TENSOR_CORES else 3e-3)
+    ref, _ = oracle.attn_e4m3(e_cpu.q, kc, vc, 0.012, 0.012, e_cpu.block_table, e_cpu.seq_lens, e_cpu.q_lens)
+    H.assert_close(out_e.double().cpu().numpy(), ref, BF, tight=3e-3)
+
+
 def test_overlap_flag_in_a_replayed_graph():
     """Five flagged calls captured in one CUDA graph and replayed back to back.  The generation
     numbers of the workspace rotation are frozen into the graph and repeat with every replay, and

@@ -4,8 +4,9 @@ Some embedders cannot call cudaMalloc once they are running -- all free device m
 belongs to their KV pool, or they sit inside another framework's operator where an allocation stalls
 the device.  They cannot hold an arb_ctx (creating one allocates), so this call keeps its split-KV
 scratch in a fixed array inside the library.  The test drives it through the C ABI and compares it
-with arb_attn on the same inputs, twice in a row with different inputs, because the shared array keeps
-the previous call's contents.  This file is collected last on purpose.
+with arb_attn on the same inputs (bit for bit against the CUDA-core kernel it shares, within tolerance
+against the default tensor-core kernel) and with the fp64 oracle, several times in a row with different
+inputs, because the shared array keeps the previous call's contents.  This file is collected last on purpose.
 """
 import ctypes
 
@@ -13,6 +14,7 @@ import numpy as np
 import pytest
 import torch
 
+from oracle import oracle
 from paper_2512_05033_b200 import workloads as wl
 
 pytestmark = pytest.mark.gpu
@@ -21,6 +23,8 @@ pytestmark = pytest.mark.gpu
 def _both(binding, ctx, inp):
     d = inp.to("cuda")
     ref = ctx.attn(d.q, d.k_pages, d.v_pages, d.block_table, d.seq_lens, d.q_lens, 1)
+    same_kernel = ctx.attn(d.q, d.k_pages, d.v_pages, d.block_table, d.seq_lens, d.q_lens, 1,
+                           params=ctx.params_for(d.q, d.k_pages, d.block_table, 1, flags=binding.ATTN_NO_TENSOR_CORES))
     out = torch.full_like(d.q, float("nan"))          # allocated by the test, not by the library
     status = torch.zeros(1, dtype=torch.int32, device="cuda")
     p = binding.attn_params(binding.ARB_BF16, d.block_table.shape[0], d.q.shape[1], d.k_pages.shape[1],
@@ -32,6 +36,7 @@ def _both(binding, ctx, inp):
     assert st == binding.ARB_OK
     torch.cuda.synchronize()
     assert int(status.item()) == 0 and ctx.poll_status() == 0
+    assert torch.equal(out, same_kernel)     # arb_attn on the CUDA-core decode kernel: the same kernel, the same plan
     return out.double().cpu().numpy(), ref.double().cpu().numpy()
 
 
@@ -46,6 +51,10 @@ def test_static_entry_point_matches_arb_attn_twice_in_a_row():
         # arb_attn may take the tensor-core decode kernel, the static call always the CUDA-core one
         assert np.abs(out - ref).max() <= 1e-2
         assert (np.abs(out - ref) <= 2.0 ** -7 * np.abs(ref) + 3e-3).all()
+        # and the definition itself, at the bar of the CUDA-core kernels
+        exact, st = oracle.attn(inp.q, inp.k_pages, inp.v_pages, inp.block_table, inp.seq_lens, inp.q_lens)
+        assert st == 0
+        assert (np.abs(out - exact) <= 2.0 ** -8 * np.abs(exact) + 1e-3).all(), np.abs(out - exact).max()
     ctx.close()
 
 

@@ -421,6 +421,21 @@ arb_status arb_phase_lens_tokens(arb_ctx *ctx, int32_t batch, const int32_t *ste
  */
 arb_status arb_poll_status(arb_ctx *ctx, arb_stream_t stream, uint32_t *bits);
 
+/*
+ * ---- Self-test ----------------------------------------------------------------------------------
+ * Every wait inside the kernels (on a TMA copy, on a tensor-core commit) gives up after a bounded number of
+ * cycles, raises ARB_DEV_WAIT_TIMEOUT, makes the other waits of its CTA return at once and lets the kernel
+ * end normally.  A healthy run never takes that path, so this call exists to exercise it: it launches one
+ * small kernel (64 threads) that waits, with the library's own wait routine, on a barrier nothing will ever
+ * signal.  The first warp gives up after limit_cycles SM cycles (1 .. 2^31, i.e. up to about a second); the
+ * second warp is given a far longer limit and must leave through the CTA's abort flag.  Nothing faults or
+ * traps; the ctx stays usable and the next arb_poll_status reports and clears ARB_DEV_WAIT_TIMEOUT.
+ *   report   DEVICE pointer to three int32: [0] = 1 once the kernel has run to its end, [1] = threads whose
+ *            wait returned "gave up" (64 expected), [2] = cycles the first thread waited.
+ * The paper has no counterpart; this is failure-detection plumbing of the library.
+ */
+arb_status arb_selftest_wait_timeout(arb_ctx *ctx, int64_t limit_cycles, int32_t *report, arb_stream_t stream);
+
 /* Number of kernels the library has launched through this ctx since arb_create. */
 uint64_t arb_launch_count(const arb_ctx *ctx);
 

@@ -35,7 +35,7 @@ EXPORTS = ("arb_create", "arb_destroy", "arb_attn_workspace_bytes", "arb_attn", 
            "arb_attn_host_begin", "arb_attn_host_wait",
            "arb_attn_decode_static",
            "arb_route", "arb_rollback", "arb_policy", "arb_route_classes", "arb_kv_append", "arb_kv_append_e4m3", "arb_attn_decode_e4m3", "arb_phase_lens", "arb_phase_lens_tokens", "arb_spearman",
-           "arb_poll_status", "arb_launch_count", "arb_status_string")
+           "arb_selftest_wait_timeout", "arb_poll_status", "arb_launch_count", "arb_status_string")
 
 
 class AttnParams(ctypes.Structure):
@@ -84,6 +84,8 @@ lib.arb_route_classes.argtypes = [_vp, _i32, _i32, _i32, _i32, _i32, _vp, _vp, c
                                   _vp, _vp, _vp, _vp]
 lib.arb_kv_append.restype = ctypes.c_int
 lib.arb_kv_append.argtypes = [_vp, ctypes.POINTER(AttnParams), _i32, _vp, _vp, _vp, _vp, _vp, _i32, _vp, _vp, _vp]
+lib.arb_selftest_wait_timeout.restype = ctypes.c_int
+lib.arb_selftest_wait_timeout.argtypes = [_vp, ctypes.c_int64, _vp, _vp]
 lib.arb_poll_status.restype = ctypes.c_int
 lib.arb_poll_status.argtypes = [_vp, _vp, ctypes.POINTER(ctypes.c_uint32)]
 lib.arb_launch_count.restype = ctypes.c_uint64
@@ -395,6 +397,16 @@ class Context:
                                _stream_ptr(stream))
         _check(st, "arb_kv_append")
         return seq_lens
+
+    # -- self-test ----------------------------------------------------------------------------
+    def selftest_wait_timeout(self, limit_cycles: int, report=None, stream=None):
+        """Launches the kernel whose wait can only run out (see arb_selftest_wait_timeout); returns the int32[3]
+        device report.  The status word carries DEV_WAIT_TIMEOUT afterwards."""
+        if report is None:
+            report = torch.zeros(3, dtype=torch.int32, device=self.device)
+        _check(lib.arb_selftest_wait_timeout(self._h, int(limit_cycles), _dev(report, "report", torch.int32),
+                                             _stream_ptr(stream)), "arb_selftest_wait_timeout")
+        return report
 
     # -- status -------------------------------------------------------------------------------
     def poll_status(self, stream=None) -> int:

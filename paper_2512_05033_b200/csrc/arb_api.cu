@@ -571,6 +571,12 @@ arb_status arb_poll_status(arb_ctx *ctx, arb_stream_t stream, uint32_t *bits) {
     return ARB_OK;
 }
 
+arb_status arb_selftest_wait_timeout(arb_ctx *ctx, int64_t limit_cycles, int32_t *report, arb_stream_t stream) {
+    if (ctx == nullptr || report == nullptr) return ARB_ERR_INVALID_ARG;
+    if (limit_cycles < 1 || limit_cycles > (1ll << 31)) return ARB_ERR_INVALID_ARG;   // at most about a second
+    return launch_selftest_wait(reinterpret_cast<Ctx *>(ctx), limit_cycles, report, reinterpret_cast<cudaStream_t>(stream));
+}
+
 uint64_t arb_launch_count(const arb_ctx *ctx) {
     return ctx ? reinterpret_cast<const Ctx *>(ctx)->launches : 0;
 }

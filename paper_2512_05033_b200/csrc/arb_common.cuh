@@ -156,22 +156,28 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity) {
     return ok != 0;
 }
 
-// Wait for the phase with the given parity.  Every wait is bounded: after kWaitCycles, or as soon
-// as another thread of the block has given up (*abort != 0), it returns false and the caller
-// carries on with whatever is in shared memory; the status word then carries ARB_DEV_WAIT_TIMEOUT.
-__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volatile int *abort,
-                                          uint32_t *status) {
+// Wait for the phase with the given parity.  Every wait is bounded: after `limit` cycles (kWaitCycles in
+// every production kernel), or as soon as another thread of the block has given up (*abort != 0), it returns
+// false and the caller carries on with whatever is in shared memory; the status word then carries
+// ARB_DEV_WAIT_TIMEOUT.
+__device__ __forceinline__ bool mbar_wait_limit(uint64_t *bar, uint32_t parity, volatile int *abort,
+                                                uint32_t *status, long long limit) {
     if (mbar_try_wait(bar, parity)) return true;
     const long long t0 = clock64();
     while (true) {
         if (mbar_try_wait(bar, parity)) return true;
         if (*abort) return false;
-        if (clock64() - t0 > kWaitCycles) {
+        if (clock64() - t0 > limit) {
             *abort = 1;
             atomicOr(status, (uint32_t)ARB_DEV_WAIT_TIMEOUT);
             return false;
         }
     }
+}
+
+__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volatile int *abort,
+                                          uint32_t *status) {
+    return mbar_wait_limit(bar, parity, abort, status, kWaitCycles);
 }
 
 // One contiguous global -> shared copy by the TMA unit; completion is counted in bytes on `bar`.
@@ -255,6 +261,7 @@ arb_status launch_kv_append_e4m3(Ctx *ctx, const arb_attn_params &p, int total_n
 arb_status launch_decode_e4m3(Ctx *ctx, const arb_attn_params &p, const void *q, const void *k_pages,
                               const void *v_pages, float k_scale, float v_scale, const int32_t *block_table,
                               const int32_t *seq_lens, const int32_t *q_lens, void *out, cudaStream_t stream);
+arb_status launch_selftest_wait(Ctx *ctx, long long limit_cycles, int32_t *report, cudaStream_t stream);
 size_t decode_workspace_bytes(const arb_attn_params &p, int num_sms);
 int decode_grid(int num_sms);
 

@@ -40,6 +40,9 @@ METRIC = "attention KV HBM GB/s (% of B200 peak) and draft steps scored+routed/s
 LAYERS = 28   # attention layers of one decode token of the draft-shaped model
 NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
+FALLBACK_BF16_TFLOPS = 1590.0
+FALLBACK_BF16_TFLOPS_SUSTAINED = 1400.0
+MIN_TIMED_MS = 150.0   # the K-step region is repeated until this much device time has been measured
 
 
 # ------------------------------------------------------------------------------------------------
@@ -53,6 +56,28 @@ def measured_peak():
         except Exception:
             pass
     return FALLBACK_HBM_GBS, "fallback"
+
+
+def measured_tensor_peaks():
+    """(burst, sustained) dense bf16 TFLOP/s and where they come from."""
+    f = ROOT / "MEASURED_PEAKS.json"
+    if f.exists():
+        try:
+            d = json.loads(f.read_text())
+            return float(d["bf16_tflops"]), float(d["bf16_tflops_sustained"]), "measured"
+        except Exception:
+            pass
+    return FALLBACK_BF16_TFLOPS, FALLBACK_BF16_TFLOPS_SUSTAINED, "fallback"
+
+
+def hbm_roofline(kernel: str, nbytes: int, us: float, peak: float, peak_kind: str, traffic=None, **extra) -> dict:
+    """The roofline object of an HBM-bound kernel: algorithmic bytes per launch over its average launch time."""
+    achieved = nbytes / (us * 1e-6) / 1e9
+    r = {"bound": "hbm", "kernel": kernel, "achieved": round(achieved, 1), "peak": peak, "peak_kind": f"of {peak_kind}",
+         "unit": "GB/s", "frac": round(achieved / peak, 4), "traffic": traffic, "algorithmic_bytes_per_launch": int(nbytes),
+         "avg_launch_us": round(us, 3)}
+    r.update(extra)
+    return r
 
 
 def attn_bytes(shape: wl.AttnShape, seq_lens, q_lens) -> dict:
@@ -174,6 +199,23 @@ def time_steps(step_fn, steps, warmup, dist_barrier=None):
     return e0.elapsed_time(e1)  # ms
 
 
+def time_repeated(step_fn, steps, warmup, dist_barrier=None, min_total_ms=MIN_TIMED_MS, max_repeats=400):
+    """The K-step region of time_steps, repeated: a region of a few milliseconds is too thin to carry a headline.
+    The first region tells how many are needed for min_total_ms of timed work in all (at least 5, at most
+    max_repeats).  Returns the list of region times (ms), one per region, each bracketed like time_steps."""
+    first = time_steps(step_fn, steps, warmup, dist_barrier)
+    repeats = int(min(max_repeats, max(5, -(-min_total_ms // max(first, 1e-3)))))
+    if dist_barrier:   # every region has barriers in it, so all ranks must run the same number: rank 0's
+        import torch.distributed as dist
+        t = torch.tensor([repeats], device="cuda")
+        dist.broadcast(t, 0)
+        repeats = int(t.item())
+    times = [first]
+    for _ in range(repeats - 1):
+        times.append(time_steps(step_fn, steps, 0, dist_barrier))
+    return times
+
+
 def time_graphed(fn, calls: int = 50, replays: int = 10):
     """Device time per call of a small library call: `calls` of them captured in one CUDA graph, the graph replayed
     `replays` times between CUDA events.  Issued one by one from Python these calls are bound by the interpreter
@@ -220,14 +262,34 @@ def rank_seed(shape: wl.AttnShape, rank: int) -> int:
     return shape.seed + 1000 * rank
 
 
-def reduce_over_ranks(ms_local: float, kv_bytes_local: float, dist, device):
-    """(slowest rank's time, bytes of all ranks).  `dist` is torch.distributed or None."""
-    t = torch.tensor([ms_local], dtype=torch.float64, device=device)
+def reduce_over_ranks(ms_local, kv_bytes_local: float, dist, device):
+    """(slowest rank's time, bytes of all ranks).  ms_local: one time or a list of region times (reduced
+    region by region).  `dist` is torch.distributed or None."""
+    many = isinstance(ms_local, (list, tuple))
+    t = torch.tensor(list(ms_local) if many else [ms_local], dtype=torch.float64, device=device)
     b = torch.tensor([kv_bytes_local], dtype=torch.float64, device=device)
     if dist is not None:
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
         dist.all_reduce(b, op=dist.ReduceOp.SUM)
-    return float(t.item()), float(b.item())
+    return (t.tolist() if many else float(t.item())), float(b.item())
+
+
+def workload_config(shape: wl.AttnShape, layers: int, world: int, tokens=None) -> dict:
+    """The `config` object: what the workload is, the same in both arms (the arms' own launch details go elsewhere)."""
+    kv_tok_bytes = 2 * shape.num_kv_heads * shape.head_dim * 2
+    cfg = {"workload": shape.name, "batch_per_gpu": shape.batch, "num_q_heads": shape.num_q_heads,
+           "num_kv_heads": shape.num_kv_heads, "head_dim": shape.head_dim, "page_size": wl.PAGE,
+           "prefix_lens": f"uniform in [{shape.prefix_lo}, {shape.prefix_hi}]", "q_len": 1,
+           "layers_per_step": layers,
+           "step": f"one generated token: {layers} layer calls of arb_attn, each on its own KV pool",
+           "l2": f"inputs larger than L2: the {layers} KV pools of a step rotate (about "
+                 f"{layers * (shape.prefix_lo + shape.prefix_hi) // 2 * shape.batch * kv_tok_bytes / 1e6:.0f} MB against 126 MB)",
+           "overlap": "the layer calls of one token share q and read caches nobody writes meanwhile, so the GPU arm "
+                      "launches them as programmatic dependents (ARB_ATTN_OVERLAP_PREVIOUS); inside Algorithm 1's token "
+                      "chain every call reads what the call before it wrote and the flag does not apply: see "
+                      "serialised_calls and step_loop on the GPU arm's line",
+           "parallelism": f"dp{world} by sequence, no collective"}
+    return cfg
 
 
 # ------------------------------------------------------------------------------------------------
@@ -256,41 +318,45 @@ def run_ours(args):
     step_fn, per_step = make_step(ctx, work, use_graph, overlap)
 
     with ClockSampler(cuda_physical_index(local)) as clk:
-        ms = time_steps(step_fn, args.steps, args.warmup, barrier)
+        if args.profile:
+            regions = [time_steps(step_fn, args.steps, args.warmup, barrier)]
+        else:
+            regions = time_repeated(step_fn, args.steps, args.warmup, barrier)
     status_bits = ctx.poll_status()
     kv_per_step = work.bytes["kv"] * layers
-    ms_max, kv_all_ranks = reduce_over_ranks(ms, kv_per_step, dist, dev)
-    ms_per_step = ms_max / args.steps
+    regions_max, kv_all_ranks = reduce_over_ranks(regions, kv_per_step, dist, dev)
+    ms_region = statistics.median(regions_max)          # the K-step region, slowest rank, median over the repeats
+    ms_per_step = ms_region / args.steps
     value = kv_all_ranks / (ms_per_step * 1e-3) / 1e9  # whole job: bytes of every rank over the slowest rank's time
 
     peak, peak_kind = measured_peak()
     # one arb_attn call = one decode_mma_kernel launch (+ its small combine kernel, whose time is counted in)
-    launch_us = ms / args.steps / layers * 1e3  # this rank's average interval between decode launches
-    achieved = work.bytes["total"] / (launch_us * 1e-6) / 1e9
+    launch_us = statistics.median(regions) / args.steps / layers * 1e3  # this rank's average interval between decode launches
     traffic = read_traffic_note() if shape is wl.DRAFT_DECODE else None
 
+    cfg = workload_config(shape, layers, world)
     result = {
         "metric": METRIC, "value": round(value, 1), "unit": "GB/s", "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": round(ms_per_step, 5), "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-        "config": {"workload": shape.name, "batch_per_gpu": shape.batch, "num_q_heads": shape.num_q_heads,
-                   "num_kv_heads": shape.num_kv_heads, "head_dim": shape.head_dim, "page_size": wl.PAGE,
-                   "kv_tokens_per_gpu": work.bytes["tokens"], "layers_per_step": layers,
-                   "kv_bytes_per_step_per_gpu": kv_per_step,
-                   "l2": f"inputs larger than L2: {layers} KV pools of {work.bytes['kv'] / 1e6:.1f} MB rotate",
-                   "launch": f"one CUDA graph of {layers} arb_attn calls ({per_step} kernels) per step" if use_graph
+        "config": cfg,
+        "timing": {"repeats": len(regions_max), "ms_per_step_median": round(ms_per_step, 5),
+                   "ms_per_step_min": round(min(regions_max) / args.steps, 5),
+                   "ms_per_step_max": round(max(regions_max) / args.steps, 5),
+                   "timed_region_ms_total": round(sum(regions_max), 2),
+                   "note": "the K-step region (barrier + synchronize on both sides, CUDA events) is repeated; "
+                           "ms_per_step is the median region / K, max over ranks per region"},
+        "launch": {"kv_tokens_per_gpu": work.bytes["tokens"], "kv_bytes_per_step_per_gpu": kv_per_step,
+                   "mode": f"one CUDA graph of {layers} arb_attn calls ({per_step} kernels) per step" if use_graph
                    else "stream launches",
                    "overlap": "layer calls launched as programmatic dependents (ARB_ATTN_OVERLAP_PREVIOUS)"
-                   if overlap else "none: every call waits for the one before it",
-                   "parallelism": f"dp{world} by sequence, no collective"},
+                   if overlap else "none: every call waits for the one before it"},
         "pct_of_nominal_8TBs_per_gpu": round(100 * value / world / NOMINAL_HBM_GBS, 2),
         "gpu_launches": per_step * args.steps,
         "device_status_bits": status_bits,
         "clocks": clk.summary(),
-        "roofline": {"bound": "hbm", "kernel": "decode_mma_kernel", "achieved": round(achieved, 1), "peak": peak,
-                     "peak_kind": f"of {peak_kind}", "unit": "GB/s", "frac": round(achieved / peak, 4),
-                     "traffic": traffic, "algorithmic_bytes_per_launch": work.bytes["total"],
-                     "avg_launch_us": round(launch_us, 3)},
+        "roofline": hbm_roofline("decode_mma_kernel (+ decode_combine_kernel)", work.bytes["total"], launch_us, peak,
+                                 peak_kind, traffic),
     }
 
     if rank == 0 and not args.profile:
@@ -299,10 +365,16 @@ def run_ours(args):
             if not args.no_extras:
                 if overlap:  # the same loop with every call fully serialised behind the previous one
                     fn2, _ = make_step(ctx, work, use_graph, overlap=False)
-                    ms2 = time_steps(fn2, max(20, args.steps // 4), 5)
+                    n2 = max(20, args.steps // 4)
+                    ms2 = statistics.median(time_repeated(fn2, n2, 5, min_total_ms=60.0))
+                    us2 = ms2 / n2 / layers * 1e3
                     result["serialised_calls"] = {
-                        "gbs": round(kv_per_step / (ms2 / max(20, args.steps // 4) * 1e-3) / 1e9, 1),
-                        "us_per_call": round(ms2 / max(20, args.steps // 4) / layers * 1e3, 3)}
+                        "gbs": round(kv_per_step / (ms2 / n2 * 1e-3) / 1e9, 1), "us_per_call": round(us2, 3),
+                        "frac_of_measured": round(work.bytes["total"] / (us2 * 1e-6) / 1e9 / peak, 4),
+                        "roofline": hbm_roofline("the decode kernel of an unflagged arb_attn call", work.bytes["total"],
+                                                 us2, peak, peak_kind),
+                        "note": "the same calls without ARB_ATTN_OVERLAP_PREVIOUS: every call waits for the one "
+                                "before it, which is what a token of Algorithm 1 sees"}
                 result["target_shaped_decode"] = run_target_decode(ctx, dev, peak)
                 result["step_scoring"] = run_step_scoring(ctx, dev)
                 result["mixed_loop"] = run_mixed_loop(ctx, dev)
@@ -414,6 +486,7 @@ def run_target_decode(ctx, dev, peak):
     gbs2 = work.bytes["total"] / (us2 * 1e-6) / 1e9
     return {"kv_tokens": work.bytes["tokens"], "us_per_call": round(us, 2), "gbs": round(gbs, 1),
             "frac_of_measured": round(gbs / peak, 4), "pct_of_nominal_8TBs": round(100 * gbs / NOMINAL_HBM_GBS, 2),
+            "roofline": hbm_roofline("decode kernel, target-shaped", work.bytes["total"], us, peak, measured_peak()[1]),
             "back_to_back": {"us_per_call": round(us2, 2), "gbs": round(gbs2, 1), "frac_of_measured": round(gbs2 / peak, 4),
                              "pct_of_nominal_8TBs": round(100 * gbs2 / NOMINAL_HBM_GBS, 2)}}
 
@@ -448,9 +521,29 @@ def run_step_scoring(ctx, dev):
         esc[str(tau)] = float(dec.float().mean().item())
     ms_route = 200 * time_graphed(lambda: ctx.route(r.hidden, r.w, r.b, 0.5, scores=scores, decisions=dec))
     b = attn_bytes(shape, seq0.cpu().to(torch.int64), inp.q_lens.cpu().to(torch.int64))
+    # the chunk attention call alone (609 MB of KV per call: larger than L2), and its roofline: per KV token and
+    # kv head 4 D bytes and 4 M D flop with M = q_len * group rows (full rectangles; the causal triangle is < 3 %)
+    inp.seq_lens.copy_(seq0)
+    attn_only = lambda: ctx.attn(inp.q, inp.k_pages, inp.v_pages, inp.block_table, inp.seq_lens, inp.q_lens, max_q, out=out)
+    us_attn = statistics.median(time_repeated(attn_only, 10, 3, min_total_ms=40.0)) / 10 * 1e3
+    sl, ql = seq0.cpu().to(torch.int64), inp.q_lens.cpu().to(torch.int64)
+    flops = int((4 * ql * shape.num_q_heads * shape.head_dim * sl).sum())
+    burst, sustained, kind = measured_tensor_peaks()
+    hbm_peak, hbm_kind = measured_peak()
+    t_tensor, t_hbm = flops / (sustained * 1e12) * 1e6, b["total"] / (hbm_peak * 1e9) * 1e6
+    tflops = flops / (us_attn * 1e-6) / 1e12
+    roof = {"bound": "tensor" if t_tensor >= t_hbm else "hbm", "kernel": "chunk_mma_kernel",
+            "achieved": round(tflops, 1), "peak": sustained, "peak_kind": f"of {kind} (sustained bf16)", "unit": "TFLOP/s",
+            "frac": round(max(t_tensor, t_hbm) / us_attn, 4), "traffic": None, "algorithmic_flops_per_launch": flops,
+            "algorithmic_bytes_per_launch": b["total"], "avg_launch_us": round(us_attn, 2),
+            "roofline_us": {"tensor": round(t_tensor, 1), "hbm": round(t_hbm, 1)},
+            "tensor_utilisation": round(tflops / sustained, 4), "tensor_utilisation_of_burst_peak": round(tflops / burst, 4),
+            "hbm_utilisation": round(b["total"] / (us_attn * 1e-6) / 1e9 / hbm_peak, 4),
+            "note": "frac = max(bytes / HBM peak, flops / tensor peak) / measured time"}
     return {"steps_scored_routed_per_s": res, "escalation_rate": esc, "layer_calls_per_step": 1,
             "route_only_steps_per_s": round(shape.batch / (ms_route / 200 * 1e-3), 1),
-            "kv_tokens": b["tokens"], "rows": int(inp.q_lens.sum())}
+            "kv_tokens": b["tokens"], "rows": int(inp.q_lens.sum()), "attn_us_per_call": round(us_attn, 2),
+            "roofline": roof}
 
 
 def run_mixed_loop(ctx, dev):
@@ -567,6 +660,7 @@ def run_kv_append(ctx, dev, peak):
     gbs = nbytes / (ms * 1e-3) / 1e9
     return {"tokens": total, "bytes_per_call": nbytes, "us_per_call": round(ms * 1e3, 2), "gbs": round(gbs, 1),
             "frac_of_measured": round(gbs / peak, 4),
+            "roofline": hbm_roofline("kv_append_kernel", nbytes, ms * 1e3, peak, measured_peak()[1]),
             "note": "50 calls per CUDA graph; 10 MB per call, back-to-back calls rewrite the same pages (L2-resident)"}
 
 
@@ -638,6 +732,7 @@ def run_e4m3_decode(ctx, dev, peak, profile=False):
         gbs = nbytes / (us * 1e-6) / 1e9
         out[name] = {"us_per_call": round(us, 2), "algorithmic_bytes_per_call": nbytes, "gbs": round(gbs, 1),
                      "frac_of_measured": round(gbs / peak, 4), "kv_tokens_per_us": round(b["tokens"] / us, 1),
+                     "roofline": hbm_roofline("decode_mma_kernel<E4M3>", nbytes, us, peak, measured_peak()[1]),
                      "bf16_equivalent_gbs": round(b["total"] / (us * 1e-6) / 1e9, 1)}
     return out
 
@@ -701,9 +796,8 @@ def run_reference(args):
         "n_gpus": int(os.environ.get("WORLD_SIZE", "1")), "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": round(dt * 1e3, 3), "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "f64", "data": "synthetic",
-        "config": {"workload": shape.name, "batch_per_gpu": shape.batch, "num_q_heads": shape.num_q_heads,
-                   "num_kv_heads": shape.num_kv_heads, "head_dim": shape.head_dim, "page_size": wl.PAGE,
-                   "sample": sample},
+        "config": workload_config(shape, LAYERS, int(os.environ.get("WORLD_SIZE", "1"))),
+        "sample": sample,
         "cpu_baseline": {"value": value, "unit": "GB/s", "cores": oracle.num_threads(), "kind": "oracle",
                          "sample": sample},
         "e2e": {"value": value, "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},

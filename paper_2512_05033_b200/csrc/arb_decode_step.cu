@@ -1,0 +1,667 @@
+// One decode token in one launch (bf16, head_dim 128, group size <= 8): the cache write of the token's new
+// K/V rows, split-KV attention over the paged cache, the split combine and the length update, all in one
+// kernel.  This is what a token of a draft or target step costs in Algorithm 1 of the paper ("Sample draft
+// step" / "Sample target step": z_i ~ q(z_i | x, z_<i), Section 3.1): every call of that chain reads what the
+// call before it wrote, so nothing overlaps and a token pays the latency of every launch on its way.  Three
+// launches (append, decode, combine) become one.
+//
+// What is shared with the two-kernel decode (arb_decode_mma.cu): the flat (sequence, kv head, page) list cut
+// into equal ranges per CTA, a producer warp feeding a ring of 4 KB page tiles through tiled TMA copies, one
+// consumer warp per page with its own online softmax.  What differs:
+//   - The product is transposed.  S^T = K q^T puts the 16 keys of a page on the 16 rows of an m16n8k16 tile and
+//     the group's heads (padded to 8) on its 8 columns; O^T += V^T P^T does the same for the second product.
+//     A page costs 8 + 8 MMAs instead of 16 + 16, the accumulators take 32 registers instead of 64, and the
+//     CTA runs eight consumer warps, two per scheduler, which hide one another's latencies.  P^T reaches the
+//     second product's B fragment through two movmatrix transposes; the row maximum is a reduction over the
+//     lanes that share a column pair (three shuffles).
+//   - The kernel waits for its predecessor at its top (griddepcontrol.wait) and lets its successor come up at
+//     once (griddepcontrol.launch_dependents): launched as a programmatic dependent it is resident, barriers
+//     initialised, when the kernel before it ends.  Nothing is read or written before the wait, so this is
+//     safe behind any kernel.
+//   - The combine is inside: a CTA that holds a part of a split (sequence, kv head) stores its partial, fences,
+//     and adds one to the item's arrival counter; the CTA that arrives last merges the parts (two round trips
+//     to L2) and writes the rows.  No CTA waits for another.
+//   - With k_new / v_new given, the warp that owns a sequence's last page puts the token's new row into the
+//     tile in shared memory (the tile arrives with whatever the slot held) and stores it to the pool; the
+//     lengths move forward once every CTA has read them (a counter in the prologue tells the last reader).
+#include "arb_decode_tc.cuh"
+
+namespace arb {
+
+namespace {
+
+constexpr int kCW = 8;                        // consumer warps
+constexpr int kCT = kCW * 32;                 // consumer threads
+constexpr int kProdWarp = kCW;                // the producer warp
+constexpr int kAuxWarp = kCW + 1;             // bookkeeping: length update, rows of refused sequences
+constexpr int kNT = kCT + 64;
+constexpr int kTileBytes = kPage * kD * 2;    // 4 KB: one (page, kv head) tile of K or of V
+constexpr int kHalfTile = kTileBytes / 2;
+constexpr int kBatch = 16;                    // producer lanes issuing side by side
+constexpr int kParked = 2;                    // segment results parked in shared memory before they are written
+constexpr int kOStride = kD + 4;              // floats between two heads of a warp record (spreads the banks)
+constexpr int kPreload = 4;                   // parts of a merge asked for before the weights are known
+
+struct StepArgs {
+    const char *q;
+    const char *k_new, *v_new;   // [rows, Hkv, D]; null: no cache write, seq_lens already count the token
+    char *k_pool, *v_pool;
+    const int32_t *block_table;
+    int32_t *seq_lens;
+    const int32_t *q_lens;
+    char *out;
+    float *part_o;     // [slots][G][D]
+    float *part_ml;    // [slots][GP][2]
+    int *counters;     // [batch * Hkv] arrival counters, zero between calls
+    int *lens_counter; // CTAs that have read the lengths, zero between calls
+    uint32_t *status;
+    int batch, Hq, Hkv, num_pages, max_pages;
+    int whole_rows;    // the tensor maps are 3-D: one copy per page tile instead of one per half
+    float scale_log2;
+};
+
+template <int STAGES>
+struct Tail {
+    uint64_t full[STAGES];
+    uint64_t empty[STAGES];
+    int abort;
+    int last[kParked];
+};
+
+template <int G>
+struct Cfg {
+    static constexpr int GP = (G + 3) / 4 * 4;
+    static constexpr int WREC = 2 * 8 + G * kOStride;     // warp record: [m[8] | l[8] | o[G][kOStride]]
+    static constexpr int REC = 2 * GP + G * kD;           // parked record: [m[GP] | l[GP] | o[G][D]]
+    static constexpr int OSM_BYTES = kCW * WREC * 4;
+    static constexpr int PARK_BYTES = kParked * REC * 4;
+};
+
+template <int G, int STAGES>
+size_t smem_bytes(int batch) {
+    using C = Cfg<G>;
+    return 1024 + (size_t)STAGES * kTileBytes + C::OSM_BYTES + C::PARK_BYTES + sizeof(Tail<STAGES>) +
+           sizeof(int) * (3 * (size_t)batch + 2);
+}
+
+struct Parked {
+    int bk, nparts, c_first;
+    size_t out_base;
+};
+
+struct Pending {   // a split (sequence, kv head) this CTA was the last to reach
+    int slot0, nparts;
+    size_t out_base;
+};
+
+__device__ __forceinline__ uint32_t tile_off(int r, int c) {   // 16-byte chunk c of row r of a swizzled bf16 tile
+    return (uint32_t)((c >> 3) * kHalfTile + r * 128 + (((c & 7) ^ (r & 7)) << 4));
+}
+
+// transposes an 8 x 8 matrix of 16-bit elements held one row per four lanes, two elements per lane
+__device__ __forceinline__ uint32_t movmatrix_trans(uint32_t v) {
+    uint32_t r;
+    asm volatile("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;" : "=r"(r) : "r"(v));
+    return r;
+}
+
+__device__ __forceinline__ void fence_proxy_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+
+// A sequence takes part when it decodes (q_len 1) and its length after the token fits the block table.
+// L0: the length the call finds in seq_lens; with a cache write the token lands at position L0.
+template <bool APPEND>
+__device__ __forceinline__ bool step_ok(int n, int L0, int max_pages) {
+    if (n != 1) return false;
+    const long long L = (long long)L0 + (APPEND ? 1 : 0);
+    return L0 >= (APPEND ? 0 : 1) && L <= (long long)max_pages * kPage;
+}
+
+template <int G, int STAGES, bool APPEND>
+__global__ void __launch_bounds__(kNT, STAGES <= 16 ? 2 : 1)
+decode_step_kernel(const StepArgs a, const __grid_constant__ CUtensorMap k_map, const __grid_constant__ CUtensorMap v_map) {
+    using C = Cfg<G>;
+    using Tail = arb::Tail<STAGES>;
+    constexpr int GP = C::GP, WREC = C::WREC, REC = C::REC;
+    constexpr int kRingBytes = STAGES * kTileBytes;
+    static_assert(G >= 1 && G <= 8, "the group's heads are the 8 columns of the tile");
+    static_assert(STAGES % (2 * kCW) == 0 && kBatch <= STAGES, "a ring stage always belongs to the same warp of a segment");
+
+    extern __shared__ char smem_raw[];
+    char *base = reinterpret_cast<char *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    char *ring = base;
+    float *osm = reinterpret_cast<float *>(base + kRingBytes);
+    float *park = reinterpret_cast<float *>(base + kRingBytes + C::OSM_BYTES);
+    Tail *tail = reinterpret_cast<Tail *>(base + kRingBytes + C::OSM_BYTES + C::PARK_BYTES);
+    int *pref = reinterpret_cast<int *>(tail + 1);
+    int *row0 = pref + a.batch + 1;
+    int *slen = row0 + a.batch + 1;
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int B = a.batch, Hkv = a.Hkv;
+
+    let_successor_start();
+    if (tid == kCT) {
+        asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&k_map)) : "memory");
+        asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&v_map)) : "memory");
+    }
+    if (tid == 0) {
+        for (int s = 0; s < STAGES; ++s) {
+            mbar_init(&tail->full[s], 1);
+            mbar_init(&tail->empty[s], 1);
+        }
+        tail->abort = 0;
+        mbar_fence_init();
+        pref[0] = 0;
+        row0[0] = 0;
+    }
+    // Everything below may read what the kernel before this one wrote (lengths, q, new rows, the cache).
+    wait_for_predecessor();
+
+    // ---- prologue: lengths -> page counts and q row offsets ------------------------------------------
+    for (int b = tid; b < B; b += kNT) {
+        const int n = a.q_lens[b], L0 = a.seq_lens[b];
+        const bool ok = step_ok<APPEND>(n, L0, a.max_pages);
+        const int L = L0 + (APPEND ? 1 : 0);
+        pref[b + 1] = ok ? (L + kPage - 1) / kPage * Hkv : 0;
+        row0[b + 1] = n > 0 ? n : 0;
+        slen[b] = L;
+    }
+    __syncthreads();
+    if (warp == 0) {
+        int carry_p = 0, carry_r = 0;
+        for (int b0 = 0; b0 < B; b0 += 32) {
+            const int b = b0 + lane;
+            int vp = b < B ? pref[b + 1] : 0;
+            int vr = b < B ? row0[b + 1] : 0;
+#pragma unroll
+            for (int off = 1; off < 32; off <<= 1) {
+                const int tp = __shfl_up_sync(0xffffffffu, vp, off);
+                const int tr = __shfl_up_sync(0xffffffffu, vr, off);
+                if (lane >= off) { vp += tp; vr += tr; }
+            }
+            if (b < B) { pref[b + 1] = vp + carry_p; row0[b + 1] = vr + carry_r; }
+            carry_p += __shfl_sync(0xffffffffu, vp, 31);
+            carry_r += __shfl_sync(0xffffffffu, vr, 31);
+        }
+    }
+    __syncthreads();
+
+    if (warp == kAuxWarp) {
+        // ================================ bookkeeping warp ==========================================
+        // Lengths: every CTA has its copy in shared memory by now.  The CTA whose count completes the grid
+        // knows that nobody will read seq_lens again and moves them forward: for the sequences that take part
+        // and whose new row has a page inside the pool to go to (the same test the writer of the row makes).
+        if constexpr (APPEND) {
+            int last = 0;
+            if (lane == 0) last = atomicAdd(a.lens_counter, 1) == (int)gridDim.x - 1;
+            last = __shfl_sync(0xffffffffu, last, 0);
+            if (last) {
+                for (int b = lane; b < B; b += 32) {
+                    const int L0 = slen[b] - 1;
+                    if (step_ok<true>(a.q_lens[b], L0, a.max_pages)) {
+                        const int pid = a.block_table[(size_t)b * a.max_pages + L0 / kPage];
+                        if ((unsigned)pid < (unsigned)a.num_pages) a.seq_lens[b] = L0 + 1;
+                    }
+                }
+                if (lane == 0) *a.lens_counter = 0;
+            }
+        }
+        // Sequences that were asked to decode but cannot: status bit, rows of zeros.
+        if (blockIdx.x == 0) {
+            for (int b = 0; b < B; ++b) {
+                const int n = row0[b + 1] - row0[b];
+                if (n != 1 || pref[b + 1] != pref[b]) continue;
+                if (lane == 0) atomicOr(a.status, (uint32_t)ARB_DEV_BAD_SEQ_LEN);
+                uint4 *o = reinterpret_cast<uint4 *>(a.out + (size_t)row0[b] * a.Hq * kD * 2);
+                for (int i = lane; i < a.Hq * kD * 2 / 16; i += 32) o[i] = make_uint4(0, 0, 0, 0);
+            }
+        }
+        return;
+    }
+
+    const int total = pref[B];
+    int chunk = (total + (int)gridDim.x - 1) / (int)gridDim.x;
+    if (chunk < kMinChunk) chunk = kMinChunk;
+    const long long r0l = (long long)blockIdx.x * chunk;
+    if (r0l >= total) return;
+    const int r0 = (int)r0l;
+    const int r1 = min(total, r0 + chunk);
+    volatile int *abort = &tail->abort;
+
+    if (warp == kProdWarp) {
+        // ================================ producer warp ==========================================
+        // Tiles enter the ring page by page, K then V; lanes 0 .. kBatch-1 each own one stage at a time.
+        uint32_t c = 0;
+        int cur = r0;
+        Segment s;
+        while (next_segment(cur, r1, pref, slen, B, Hkv, chunk, s)) {
+            for (int sp0 = s.pg0; sp0 < s.pg1; sp0 += 32) {
+                const int np = min(32, s.pg1 - sp0);
+                int pid = 0;
+                if (lane < np) {
+                    pid = a.block_table[(size_t)s.b * a.max_pages + sp0 + lane];
+                    if ((unsigned)pid >= (unsigned)a.num_pages) {
+                        atomicOr(a.status, (uint32_t)ARB_DEV_BAD_PAGE);
+                        pid = 0;
+                    }
+                }
+                const int ntiles = 2 * np;
+#pragma unroll 1
+                for (int i0 = 0; i0 < ntiles; i0 += kBatch) {
+                    const int i = i0 + lane;
+                    const int pg = __shfl_sync(0xffffffffu, pid, (i >> 1) & 31);
+                    if (lane < kBatch && i < ntiles) {
+                        const uint32_t cc = c + i, st = cc % STAGES, par = (cc / STAGES) & 1u;
+                        const CUtensorMap *map = (i & 1) ? &v_map : &k_map;
+                        if (mbar_wait(&tail->empty[st], par ^ 1u, abort, a.status)) {
+                            mbar_arrive_expect_tx(&tail->full[st], kTileBytes);
+                            const int row = (pg * Hkv + s.kvh) * kPage;
+                            if (a.whole_rows) {
+                                tma_box_load3(ring + st * kTileBytes, map, 0, row, 0, &tail->full[st]);
+                            } else {
+                                tma_box_load(ring + st * kTileBytes, map, 0, row, &tail->full[st]);
+                                tma_box_load(ring + st * kTileBytes + kHalfTile, map, 64, row, &tail->full[st]);
+                            }
+                        }
+                    }
+                    __syncwarp();
+                }
+                c += ntiles;
+            }
+        }
+        // After a timeout the consumers may have left copies unconsumed: wait (bounded) for the last ring's
+        // worth, so that no copy is in flight into this CTA's shared memory when it exits.
+        if (lane == 0 && *abort) {
+            const uint32_t n = c < (uint32_t)STAGES ? c : (uint32_t)STAGES;
+            for (uint32_t i = 0; i < n; ++i) {
+                const uint32_t cc = c - 1 - i;
+                const long long t0 = clock64();
+                while (!mbar_try_wait(&tail->full[cc % STAGES], (cc / STAGES) & 1u) && clock64() - t0 < (1ll << 24)) {
+                }
+            }
+        }
+        return;
+    }
+
+    // ==================================== consumer warps ==========================================
+    const int gq = lane >> 2, tq = lane & 3;   // fragment coordinates
+    const bool head_ok = gq < G;               // as a B-fragment column: this lane's head is a real one
+    const int h0 = 2 * tq, h1 = 2 * tq + 1;    // as accumulator columns: the two heads this lane holds
+    const uint32_t ring_addr = smem_u32(ring);
+    uint32_t seg_base = 0;                     // ring counter of the segment's first tile
+    int cur = r0;
+    Segment s;
+    int n_parked = 0, pend_n = 0;
+    Parked pk[kParked];
+    Pending pend[2];
+
+    // Writes what is parked: whole (sequence, kv head)s to `out`, parts of split ones to the workspace, followed
+    // by the arrival at the item's counter.  The last to arrive notes the merge for the epilogue.
+    auto flush = [&]() {
+        bool any_multi = false;
+        for (int j = 0; j < n_parked; ++j) {
+            const float *rec = park + j * REC;
+            if (pk[j].nparts == 1) {
+                for (int idx = tid; idx < G * kD; idx += kCT)
+                    reinterpret_cast<__nv_bfloat16 *>(a.out)[pk[j].out_base + idx] =
+                        __float2bfloat16_rn(rec[2 * GP + idx] / rec[GP + idx / kD]);
+            } else {
+                any_multi = true;
+                const size_t slot = (size_t)pk[j].bk + blockIdx.x;
+                for (int idx = tid; idx < G * kD / 4; idx += kCT)
+                    reinterpret_cast<float4 *>(a.part_o + slot * G * kD)[idx] =
+                        reinterpret_cast<const float4 *>(rec + 2 * GP)[idx];
+                if (tid < G) {
+                    a.part_ml[(slot * GP + tid) * 2 + 0] = rec[tid];
+                    a.part_ml[(slot * GP + tid) * 2 + 1] = rec[GP + tid];
+                }
+            }
+        }
+        if (any_multi) {
+            __threadfence();
+            named_barrier(1, kCT);
+            if (tid == 0) {
+                int old[kParked];
+                for (int j = 0; j < n_parked; ++j)
+                    old[j] = pk[j].nparts > 1 ? atomicAdd(&a.counters[pk[j].bk], 1) : -1;
+                for (int j = 0; j < n_parked; ++j) {
+                    const int last = pk[j].nparts > 1 && old[j] == pk[j].nparts - 1;
+                    if (last) a.counters[pk[j].bk] = 0;   // everyone has arrived: ready for the next call
+                    tail->last[j] = last;
+                }
+                __threadfence();
+            }
+            named_barrier(1, kCT);
+            for (int j = 0; j < n_parked; ++j) {
+                if (pk[j].nparts > 1 && tail->last[j] && pend_n < 2) {
+                    pend[pend_n].slot0 = pk[j].bk + pk[j].c_first;
+                    pend[pend_n].nparts = pk[j].nparts;
+                    pend[pend_n].out_base = pk[j].out_base;
+                    ++pend_n;
+                }
+            }
+        }
+        named_barrier(1, kCT);   // parking slots and flags are free again
+        n_parked = 0;
+    };
+
+    while (next_segment(cur, r1, pref, slen, B, Hkv, chunk, s)) {
+        const int qrow = row0[s.b];
+        // B fragments of q^T (128 dims x 8 heads): k-slice ks holds dims 16 ks + 2 tq, + 1 and + 8 of head gq
+        uint32_t qb[8][2];
+        {
+            const char *qh = a.q + ((size_t)qrow * a.Hq + s.kvh * G + (head_ok ? gq : 0)) * kD * 2;
+#pragma unroll
+            for (int ks = 0; ks < 8; ++ks) {
+                qb[ks][0] = head_ok ? __ldg(reinterpret_cast<const uint32_t *>(qh + ks * 32 + tq * 4)) : 0u;
+                qb[ks][1] = head_ok ? __ldg(reinterpret_cast<const uint32_t *>(qh + ks * 32 + 16 + tq * 4)) : 0u;
+            }
+        }
+        // The token's new row: it belongs in slot (L - 1) mod 16 of the sequence's last page.  The warp that owns
+        // that page fetches the row (lanes 0..15: K, lanes 16..31: V, 16 bytes each), stores it to the pool and
+        // patches it into the tiles when they arrive.
+        const int seg_pages = s.pg1 - s.pg0;
+        const int last_pg = (s.L - 1) / kPage, new_slot = (s.L - 1) % kPage;
+        bool patch = false;
+        uint4 new_row = make_uint4(0, 0, 0, 0);
+        if constexpr (APPEND) {
+            patch = last_pg >= s.pg0 && last_pg < s.pg1 && ((last_pg - s.pg0) % kCW) == warp;
+            if (patch) {
+                const char *src = (lane < 16 ? a.k_new : a.v_new) + ((size_t)qrow * Hkv + s.kvh) * kD * 2 + (lane & 15) * 16;
+                new_row = __ldg(reinterpret_cast<const uint4 *>(src));
+                const int pid = a.block_table[(size_t)s.b * a.max_pages + last_pg];
+                if ((unsigned)pid < (unsigned)a.num_pages) {
+                    char *dst = (lane < 16 ? a.k_pool : a.v_pool) +
+                                (((size_t)pid * Hkv + s.kvh) * kPage + new_slot) * (kD * 2) + (lane & 15) * 16;
+                    *reinterpret_cast<uint4 *>(dst) = new_row;
+                }   // a page outside the pool: the producer has raised ARB_DEV_BAD_PAGE; nothing is written
+            }
+        }
+
+        // this lane's columns (heads h0, h1): running max (the same in the 8 lanes of a column pair), its share of
+        // the sum, and 8 m-tiles of O^T: o[mt][0..1] = dim 16 mt + gq of heads h0, h1; o[mt][2..3] = dim + 8
+        float m_run0 = -INFINITY, m_run1 = -INFINITY, l_run0 = 0.f, l_run1 = 0.f;
+        float o[8][4];
+#pragma unroll
+        for (int mt = 0; mt < 8; ++mt) { o[mt][0] = o[mt][1] = o[mt][2] = o[mt][3] = 0.f; }
+
+        for (int gi = warp; gi < seg_pages; gi += kCW) {
+            const int pg = s.pg0 + gi;
+            const int ntok = min(s.L - pg * kPage, kPage);
+            const bool patch_here = APPEND && patch && pg == last_pg;
+            const uint32_t ck = seg_base + 2u * (uint32_t)gi;
+
+            // ---- S^T = K q^T: 16 keys x 8 heads, two accumulators so that the chain is four deep ----------
+            float sa[4] = {0.f, 0.f, 0.f, 0.f}, sb[4] = {0.f, 0.f, 0.f, 0.f};
+            {
+                const uint32_t st = ck % STAGES, par = (ck / STAGES) & 1u;
+                mbar_wait(&tail->full[st], par, abort, a.status);
+                if (patch_here) {
+                    if (lane < 16) *reinterpret_cast<uint4 *>(ring + st * kTileBytes + tile_off(new_slot, lane)) = new_row;
+                    __syncwarp();
+                }
+                const uint32_t tile = ring_addr + st * kTileBytes;
+#pragma unroll
+                for (int ks = 0; ks < 8; ++ks) {
+                    uint32_t af[4];   // rows: keys; matrices: (keys 0-7 | 8-15) x (dims 16 ks + 0-7 | 8-15)
+                    ldmatrix_x4(tile + tile_off((lane & 7) + ((lane >> 3) & 1) * 8, 2 * ks + (lane >> 4)), af);
+                    if (ks & 1) mma_16816<false>(sb, af, qb[ks][0], qb[ks][1]);
+                    else mma_16816<false>(sa, af, qb[ks][0], qb[ks][1]);
+                }
+                __syncwarp();
+                if (patch_here) fence_proxy_async_smem();   // the stage's next writer is the TMA unit
+                if (lane == 0) mbar_arrive(&tail->empty[st]);
+            }
+
+            // ---- online softmax: this lane has keys gq and gq + 8 of heads h0 and h1 -------------------
+            const bool k0 = gq < ntok, k1 = gq + 8 < ntok;
+            const float s00 = k0 ? (sa[0] + sb[0]) * a.scale_log2 : -INFINITY;
+            const float s01 = k0 ? (sa[1] + sb[1]) * a.scale_log2 : -INFINITY;
+            const float s10 = k1 ? (sa[2] + sb[2]) * a.scale_log2 : -INFINITY;
+            const float s11 = k1 ? (sa[3] + sb[3]) * a.scale_log2 : -INFINITY;
+            float mx0 = fmaxf(s00, s10), mx1 = fmaxf(s01, s11);
+#pragma unroll
+            for (int off = 4; off < 32; off <<= 1) {
+                mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, off));
+                mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, off));
+            }
+            const float mn0 = fmaxf(m_run0, mx0), mn1 = fmaxf(m_run1, mx1);   // finite: key 0 of the page is visible
+            const float f0 = fast_exp2(m_run0 - mn0), f1 = fast_exp2(m_run1 - mn1);   // 0 on the first page
+            m_run0 = mn0;
+            m_run1 = mn1;
+            // P^T, rounded to bf16; the sums use the rounded weights, like the tensor core
+            const uint32_t w0 = pack_bf16(fast_exp2(s00 - mn0), fast_exp2(s01 - mn1));   // key gq:     heads h0, h1
+            const uint32_t w1 = pack_bf16(fast_exp2(s10 - mn0), fast_exp2(s11 - mn1));   // key gq + 8
+            l_run0 = fmaf(l_run0, f0, __uint_as_float(w0 << 16) + __uint_as_float(w1 << 16));
+            l_run1 = fmaf(l_run1, f1, __uint_as_float(w0 & 0xffff0000u) + __uint_as_float(w1 & 0xffff0000u));
+            // B fragment of P^T (16 keys x 8 heads): keys 2 tq, + 1 (and + 8) of head gq
+            const uint32_t pb0 = movmatrix_trans(w0), pb1 = movmatrix_trans(w1);
+            if (__any_sync(0xffffffffu, f0 != 1.0f || f1 != 1.0f)) {
+#pragma unroll
+                for (int mt = 0; mt < 8; ++mt) { o[mt][0] *= f0; o[mt][1] *= f1; o[mt][2] *= f0; o[mt][3] *= f1; }
+            }
+
+            // ---- O^T += V^T P^T: 8 m-tiles of 16 dims ---------------------------------------------------
+            {
+                const uint32_t cv = ck + 1u, st = cv % STAGES, par = (cv / STAGES) & 1u;
+                mbar_wait(&tail->full[st], par, abort, a.status);
+                if (patch_here) {
+                    if (lane >= 16) *reinterpret_cast<uint4 *>(ring + st * kTileBytes + tile_off(new_slot, lane - 16)) = new_row;
+                    __syncwarp();
+                }
+                if (ntok < kPage) {
+                    // slots past the sequence end may hold anything; they must not reach the tensor core, not even
+                    // times zero: blank them in shared memory
+                    for (int i = lane; i < (kPage - ntok) * 16; i += 32)
+                        *reinterpret_cast<uint4 *>(ring + st * kTileBytes + tile_off(ntok + (i >> 4), i & 15)) = make_uint4(0, 0, 0, 0);
+                    __syncwarp();
+                }
+                const uint32_t tile = ring_addr + st * kTileBytes;
+#pragma unroll
+                for (int mt = 0; mt < 8; ++mt) {
+                    uint32_t af[4];   // transposed on the way: rows dims (16 mt + 0-7 | 8-15), columns keys (0-7 | 8-15)
+                    ldmatrix_x4_trans(tile + tile_off((lane & 7) + (lane >> 4) * 8, 2 * mt + ((lane >> 3) & 1)), af);
+                    mma_16816<false>(o[mt], af, pb0, pb1);
+                }
+                __syncwarp();
+                if (patch_here || ntok < kPage) fence_proxy_async_smem();
+                if (lane == 0) mbar_arrive(&tail->empty[st]);
+            }
+        }
+        seg_base += 2u * (uint32_t)seg_pages;
+
+        // ---- segment end: every warp leaves (max, sum, accumulators); all consumer threads merge them ----
+#pragma unroll
+        for (int off = 4; off < 32; off <<= 1) {
+            l_run0 += __shfl_xor_sync(0xffffffffu, l_run0, off);
+            l_run1 += __shfl_xor_sync(0xffffffffu, l_run1, off);
+        }
+        float *rec = osm + warp * WREC;
+        if (gq == 0) {
+            rec[h0] = m_run0; rec[h1] = m_run1;
+            rec[8 + h0] = l_run0; rec[8 + h1] = l_run1;
+        }
+#pragma unroll
+        for (int mt = 0; mt < 8; ++mt) {
+            const int d = 16 * mt + gq;
+            if (h0 < G) { rec[16 + h0 * kOStride + d] = o[mt][0]; rec[16 + h0 * kOStride + d + 8] = o[mt][2]; }
+            if (h1 < G) { rec[16 + h1 * kOStride + d] = o[mt][1]; rec[16 + h1 * kOStride + d + 8] = o[mt][3]; }
+        }
+        if (n_parked == kParked) flush();   // uniform across the consumer threads
+        named_barrier(1, kCT);
+        float *dst = park + n_parked * REC;
+        for (int idx = tid; idx < G * kD; idx += kCT) {
+            const int h = idx / kD, d = idx - h * kD;
+            float M = -INFINITY;
+#pragma unroll
+            for (int w = 0; w < kCW; ++w) M = fmaxf(M, osm[w * WREC + h]);
+            float l = 0.f, acc = 0.f;
+#pragma unroll
+            for (int w = 0; w < kCW; ++w) {
+                const float ff = fast_exp2(osm[w * WREC + h] - M);   // 0 for a warp that had no page
+                l = fmaf(ff, osm[w * WREC + 8 + h], l);
+                acc = fmaf(ff, osm[w * WREC + 16 + h * kOStride + d], acc);
+            }
+            dst[2 * GP + idx] = acc;
+            if (d == 0) { dst[h] = M; dst[GP + h] = l; }
+        }
+        pk[n_parked].bk = s.bk;
+        pk[n_parked].nparts = s.nparts;
+        pk[n_parked].c_first = s.c_first;
+        pk[n_parked].out_base = ((size_t)qrow * a.Hq + s.kvh * G) * kD;
+        ++n_parked;
+        named_barrier(1, kCT);   // warp records are free for the next segment
+    }
+    if (n_parked > 0) flush();
+
+    // ---- merges of the split (sequence, kv head)s this CTA was the last to reach ------------------------
+    // One 4-dimension piece of the group's G x 128 outputs per thread:
+    //     m = max_p m_p,  w_p = 2^(m_p - m),  out = sum_p w_p o_p / sum_p w_p l_p.
+    // The (max, sum) records of the parts go to shared memory (the warp records are idle by now); the first
+    // partial values are asked for before the weights exist, so that the two round trips run side by side.
+    constexpr int VECS = G * kD / 4;
+    static_assert(VECS <= kCT, "one piece per consumer thread");
+    float2 *ml_s = reinterpret_cast<float2 *>(osm);
+    for (int j = 0; j < pend_n; ++j) {
+        const int nparts = pend[j].nparts;
+        const size_t slot0 = (size_t)pend[j].slot0;
+        const bool mine = tid < VECS;
+        const int e = mine ? tid : 0, eh = e / (kD / 4);
+        const float4 *po = reinterpret_cast<const float4 *>(a.part_o + slot0 * G * kD);
+        float4 v[kPreload];
+#pragma unroll
+        for (int u = 0; u < kPreload; ++u) v[u] = __ldcg(po + (size_t)min(u, nparts - 1) * VECS + e);
+        for (int i = tid; i < nparts * G; i += kCT) {
+            const int p = i / G, h = i - p * G;
+            ml_s[i] = __ldcg(reinterpret_cast<const float2 *>(a.part_ml + ((slot0 + p) * GP + h) * 2));
+        }
+        named_barrier(1, kCT);
+        float m = -INFINITY;
+        for (int p = 0; p < nparts; ++p) m = fmaxf(m, ml_s[p * G + eh].x);
+        float l = 0.f;
+        float4 x = make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int p0 = 0; p0 < nparts; p0 += kPreload) {
+            if (p0 > 0) {
+#pragma unroll
+                for (int u = 0; u < kPreload; ++u) v[u] = __ldcg(po + (size_t)min(p0 + u, nparts - 1) * VECS + e);
+            }
+#pragma unroll
+            for (int u = 0; u < kPreload; ++u) {
+                if (p0 + u < nparts) {
+                    const float2 ml = ml_s[(p0 + u) * G + eh];
+                    const float w = fast_exp2(ml.x - m);
+                    l = fmaf(w, ml.y, l);
+                    x.x = fmaf(w, v[u].x, x.x);
+                    x.y = fmaf(w, v[u].y, x.y);
+                    x.z = fmaf(w, v[u].z, x.z);
+                    x.w = fmaf(w, v[u].w, x.w);
+                }
+            }
+        }
+        if (mine) {
+            const float inv = 1.0f / l;
+            uint2 o2;
+            o2.x = pack_bf16(x.x * inv, x.y * inv);
+            o2.y = pack_bf16(x.z * inv, x.w * inv);
+            *reinterpret_cast<uint2 *>(reinterpret_cast<__nv_bfloat16 *>(a.out) + pend[j].out_base + (size_t)e * 4) = o2;
+        }
+        named_barrier(1, kCT);   // ml_s is free for the next merge
+    }
+}
+
+// Ring depth.  32 stages (128 KB of tiles in flight per SM, one CTA per SM) serve a call that streams at the
+// pace of the memory system; 16 stages leave room for two CTAs per SM, so the next kernel of a chain of small
+// dependent calls is resident, waiting, while this one finishes.
+template <int G, int STAGES, bool APPEND>
+arb_status launch_variant(Ctx *ctx, const StepArgs &a, const CUtensorMap &km, const CUtensorMap &vm, cudaStream_t stream) {
+    static bool attr_set[64] = {};
+    if (!attr_set[ctx->device & 63]) {
+        if (cudaFuncSetAttribute(decode_step_kernel<G, STAGES, APPEND>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 (int)smem_bytes<G, STAGES>(kMaxBatch)) != cudaSuccess)
+            return ARB_ERR_CUDA;
+        attr_set[ctx->device & 63] = true;
+    }
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(ctx->num_sms);
+    cfg.blockDim = dim3(kNT);
+    cfg.dynamicSmemBytes = smem_bytes<G, STAGES>(a.batch);
+    cfg.stream = stream;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    if (cudaLaunchKernelEx(&cfg, decode_step_kernel<G, STAGES, APPEND>, a, km, vm) != cudaSuccess) return ARB_ERR_CUDA;
+    ctx->launches++;
+    return ARB_OK;
+}
+
+template <int G>
+arb_status launch_g(Ctx *ctx, const StepArgs &a, const CUtensorMap &km, const CUtensorMap &vm, bool deep, cudaStream_t stream) {
+    if (a.k_new != nullptr)
+        return deep ? launch_variant<G, 32, true>(ctx, a, km, vm, stream) : launch_variant<G, 16, true>(ctx, a, km, vm, stream);
+    return deep ? launch_variant<G, 32, false>(ctx, a, km, vm, stream) : launch_variant<G, 16, false>(ctx, a, km, vm, stream);
+}
+
+}  // namespace
+
+bool decode_step_supported(const arb_attn_params &p) {
+    const int g = p.num_q_heads / p.num_kv_heads;
+    return p.dtype == ARB_BF16 && p.head_dim == kD && g >= 1 && g <= 8 && tma_available();
+}
+
+// k_new == nullptr: attention only (seq_lens is not written).
+arb_status launch_decode_step(Ctx *ctx, const arb_attn_params &p, const void *q, const void *k_new, const void *v_new,
+                              void *k_pages, void *v_pages, const int32_t *block_table, int32_t *seq_lens,
+                              const int32_t *q_lens, void *out, cudaStream_t stream) {
+    alignas(64) CUtensorMap km, vm;
+    bool whole_rows = pool_map(ctx, &km, k_pages, p.num_pages, p.num_kv_heads, PoolView::kBf16WholeRows) &&
+                      pool_map(ctx, &vm, v_pages, p.num_pages, p.num_kv_heads, PoolView::kBf16WholeRows);
+    if (!whole_rows && (!pool_map(ctx, &km, k_pages, p.num_pages, p.num_kv_heads, PoolView::kBf16HalfRows) ||
+                        !pool_map(ctx, &vm, v_pages, p.num_pages, p.num_kv_heads, PoolView::kBf16HalfRows)))
+        return ARB_ERR_CUDA;
+    const int g = p.num_q_heads / p.num_kv_heads;
+    const int gp = (g + 3) / 4 * 4;
+    const size_t slots = (size_t)p.batch * p.num_kv_heads + (size_t)ctx->num_sms;
+    const size_t part_o_floats = (slots * g * p.head_dim + 63) & ~size_t(63);
+    const size_t bytes = (part_o_floats + slots * gp * 2) * sizeof(float);
+    if (bytes > ctx->workspace_bytes) return ARB_ERR_WORKSPACE;
+    note_unnumbered_decode(ctx, bytes);   // region 0 of the workspace: this kernel waits for its predecessor first
+    StepArgs a;
+    a.q = static_cast<const char *>(q);
+    a.k_new = static_cast<const char *>(k_new);
+    a.v_new = static_cast<const char *>(v_new);
+    a.k_pool = static_cast<char *>(k_pages);
+    a.v_pool = static_cast<char *>(v_pages);
+    a.block_table = block_table;
+    a.seq_lens = seq_lens;
+    a.q_lens = q_lens;
+    a.out = static_cast<char *>(out);
+    a.part_o = reinterpret_cast<float *>(ctx->workspace);
+    a.part_ml = a.part_o + part_o_floats;
+    a.counters = ctx->rot;                                                       // [kRotCounters]
+    a.lens_counter = ctx->rot + (size_t)kRotSets * kRotCounters + kRotSets + 4;
+    a.status = ctx->status;
+    a.batch = p.batch;
+    a.Hq = p.num_q_heads;
+    a.Hkv = p.num_kv_heads;
+    a.num_pages = p.num_pages;
+    a.max_pages = p.max_pages_per_seq;
+    a.whole_rows = whole_rows ? 1 : 0;
+    const float scale = p.softmax_scale > 0.f ? p.softmax_scale : 1.0f / sqrtf((float)p.head_dim);
+    a.scale_log2 = scale * 1.4426950408889634f;
+    const bool deep = ctx->step_deep_ring;
+    switch (g) {
+        case 1: return launch_g<1>(ctx, a, km, vm, deep, stream);
+        case 2: return launch_g<2>(ctx, a, km, vm, deep, stream);
+        case 3: return launch_g<3>(ctx, a, km, vm, deep, stream);
+        case 4: return launch_g<4>(ctx, a, km, vm, deep, stream);
+        case 5: return launch_g<5>(ctx, a, km, vm, deep, stream);
+        case 6: return launch_g<6>(ctx, a, km, vm, deep, stream);
+        case 7: return launch_g<7>(ctx, a, km, vm, deep, stream);
+        case 8: return launch_g<8>(ctx, a, km, vm, deep, stream);
+        default: return ARB_ERR_UNSUPPORTED;
+    }
+}
+
+}  // namespace arb

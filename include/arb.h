@@ -15,7 +15,8 @@
  *                 same prefix x, so a cache that absorbed the rejected draft step drops it by
  *                 resetting its length; no KV bytes move.
  *
- * Around them: arb_kv_append (the cache write of a step's new tokens), arb_policy (the escalation rules
+ * Around them: arb_kv_append (the cache write of a step's new tokens), arb_decode_step (one decode token:
+ * cache write, attention and length update in one launch), arb_policy (the escalation rules
  * the paper compares on PRM scores: RSD, oracle threshold / arg max, budgeted oracle, with the wasted
  * target calls) and arb_route_classes (the C-way heads of the router ablation).
  *
@@ -337,6 +338,36 @@ arb_status arb_route_classes(arb_ctx *ctx, int32_t dtype, int32_t mode, int32_t 
 arb_status arb_kv_append(arb_ctx *ctx, const arb_attn_params *params, int32_t total_new, const void *k_new,
                          const void *v_new, const int32_t *block_table, int32_t *seq_lens, const int32_t *new_lens,
                          int32_t update_lens, void *k_pages, void *v_pages, arb_stream_t stream);
+
+/*
+ * One decode token in one launch: arb_kv_append of the token's K/V rows, arb_attn with q_len = 1 over the
+ * cache that now holds them, and the length update, fused (Algorithm 1, "Sample draft step" / "Sample target
+ * step": a step is generated token by token, z_i ~ q(z_i | x, z_<i), Section 3.1; every token of every step
+ * pays this call once per layer, and each call reads what the one before it wrote, so its latency -- not its
+ * bytes -- is what the loop sees).
+ *
+ *   params     as for arb_attn with max_q_len == 1; total_q = number of sequences with q_lens[b] == 1.
+ *              ARB_ATTN_OVERLAP_PREVIOUS is refused (ARB_ERR_INVALID_ARG): the call writes the cache it reads.
+ *   q, out     [total_q, Hq, D], rows in batch order of the sequences that take part.
+ *   k_new,
+ *   v_new      [total_q, Hkv, D], same row order: the token's key and value rows.
+ *   k_pages,
+ *   v_pages    the pools, written (one row per sequence and kv head) and read.
+ *   seq_lens   int32 [B]: tokens held BEFORE the call.  The token of sequence b goes to position seq_lens[b],
+ *              attends keys 0 .. seq_lens[b] inclusive (itself included), and seq_lens[b] becomes seq_lens[b] + 1.
+ *   q_lens     int32 [B]: 1 = the sequence takes part, 0 = idle slot (nothing read, written or advanced).
+ * The result equals arb_kv_append(new_lens = q_lens, update_lens = 1) followed by arb_attn(max_q_len = 1),
+ * within the tolerances of arb_attn.  A sequence whose token does not fit under its block-table row is left
+ * untouched (pools, length), its out row is zero-filled and ARB_DEV_BAD_SEQ_LEN is raised; a sequence whose
+ * new row would land on a page outside the pool keeps its length and pools, raises ARB_DEV_BAD_PAGE, and its
+ * out row is unspecified but finite-safe (as for arb_attn).  q_lens other than 0 and 1 count as 0 with the
+ * status bit.  bf16 / head_dim 128 / g <= 8 run as one kernel; other shapes as the two calls above.
+ * Asynchronous on `stream`; launched as a programmatic dependent of the kernel before it (it touches no
+ * memory before that kernel has completed, so this is safe behind any kernel).
+ */
+arb_status arb_decode_step(arb_ctx *ctx, const arb_attn_params *params, const void *q, const void *k_new,
+                           const void *v_new, void *k_pages, void *v_pages, const int32_t *block_table,
+                           int32_t *seq_lens, const int32_t *q_lens, void *out, arb_stream_t stream);
 
 /*
  * Decode attention (every q_len 1 or 0) over an E4M3 KV cache: keys are k_scale * code, values v_scale * code,

@@ -33,7 +33,7 @@ MAX_CLASSES = 16
 # every symbol include/arb.h declares
 EXPORTS = ("arb_create", "arb_destroy", "arb_attn_workspace_bytes", "arb_attn", "arb_attn_host",
            "arb_attn_host_begin", "arb_attn_host_wait",
-           "arb_attn_decode_static",
+           "arb_attn_decode_static", "arb_decode_step",
            "arb_route", "arb_rollback", "arb_policy", "arb_route_classes", "arb_kv_append", "arb_kv_append_e4m3", "arb_attn_decode_e4m3", "arb_phase_lens", "arb_phase_lens_tokens", "arb_spearman",
            "arb_selftest_wait_timeout", "arb_poll_status", "arb_launch_count", "arb_status_string")
 
@@ -63,6 +63,8 @@ lib.arb_attn_host_wait.restype = ctypes.c_int
 lib.arb_attn_host_wait.argtypes = [_vp]
 lib.arb_attn_decode_static.restype = ctypes.c_int
 lib.arb_attn_decode_static.argtypes = [ctypes.POINTER(AttnParams), _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp]
+lib.arb_decode_step.restype = ctypes.c_int
+lib.arb_decode_step.argtypes = [_vp, ctypes.POINTER(AttnParams), _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp]
 lib.arb_route.restype = ctypes.c_int
 lib.arb_route.argtypes = [_vp, _i32, _i32, _i32, _vp, _vp, _f, _f, _vp, _vp, _vp]
 lib.arb_rollback.restype = ctypes.c_int
@@ -247,6 +249,22 @@ class Context:
     def attn_host_wait(self):
         """Blocks until every attn_host_begin of this context has delivered its result."""
         _check(lib.arb_attn_host_wait(self._h), "arb_attn_host_wait")
+
+    # -- arb_decode_step ----------------------------------------------------------------------
+    def decode_step(self, q, k_new, v_new, k_pages, v_pages, block_table, seq_lens, q_lens, out=None,
+                    softmax_scale: float = 0.0, stream=None, params: AttnParams | None = None):
+        """One decode token in one launch: the new K/V rows go into the cache, out = attention over the cache
+        including them, seq_lens += q_lens (in place).  Asynchronous."""
+        if out is None:
+            out = torch.empty_like(q)
+        p = params or self.params_for(q, k_pages, block_table, 1, softmax_scale)
+        st = lib.arb_decode_step(self._h, ctypes.byref(p), _dev(q, "q"), _dev(k_new, "k_new", q.dtype),
+                                 _dev(v_new, "v_new", q.dtype), _dev(k_pages, "k_pages", q.dtype),
+                                 _dev(v_pages, "v_pages", q.dtype), _dev(block_table, "block_table", torch.int32),
+                                 _dev(seq_lens, "seq_lens", torch.int32), _dev(q_lens, "q_lens", torch.int32),
+                                 _dev(out, "out", q.dtype), _stream_ptr(stream))
+        _check(st, "arb_decode_step")
+        return out
 
     # -- arb_route ----------------------------------------------------------------------------
     def route(self, hidden, w, b: float, tau: float, scores=None, decisions=None, stream=None):

@@ -1,4 +1,5 @@
 // C ABI of the arb library: argument validation, context and dispatch.  No arithmetic here.
+#include <cstdlib>
 #include <cstring>
 #include <new>
 
@@ -112,12 +113,13 @@ arb_status arb_create(arb_ctx **out, int device, size_t workspace_bytes) {
         return ARB_ERR_CUDA;
     }
     c->num_sms = sms;
+    if (const char *ring = std::getenv("ARB_STEP_RING")) c->step_deep_ring = std::atoi(ring) != 16;   // tuning knob
     c->workspace_bytes = workspace_bytes ? workspace_bytes : kDefaultWorkspace;
     c->counters_len = kCounters;
     bool ok = cudaMalloc(&c->workspace, c->workspace_bytes) == cudaSuccess;
     ok = ok && cudaMalloc(&c->counters, sizeof(int) * (c->counters_len + 4)) == cudaSuccess;
     ok = ok && cudaMemset(c->counters, 0, sizeof(int) * (c->counters_len + 4)) == cudaSuccess;
-    const size_t rot_ints = (size_t)kRotSets * kRotCounters + kRotSets + 4;
+    const size_t rot_ints = (size_t)kRotSets * kRotCounters + kRotSets + 8;
     ok = ok && cudaMalloc(&c->rot, sizeof(int) * rot_ints) == cudaSuccess;
     ok = ok && cudaMemset(c->rot, 0, sizeof(int) * rot_ints) == cudaSuccess;
     ok = ok && cudaMalloc(&c->spearman_acc, 4 * sizeof(double)) == cudaSuccess;
@@ -189,7 +191,14 @@ arb_status arb_attn(arb_ctx *ctx, const arb_attn_params *params, const void *q, 
     const bool maybe_decode = params->max_q_len == 1 || params->total_q > params->max_q_len;
     const bool tensor_cores = (params->flags & ARB_ATTN_NO_TENSOR_CORES) == 0;
     if (maybe_decode) {
-        if (tensor_cores && decode_mma_supported(*params))
+        // bf16 / head_dim 128: a call that is one of a back-to-back series (ARB_ATTN_OVERLAP_PREVIOUS) takes the
+        // two-kernel form, whose calls stream under one another's tails; a call on its own takes the single
+        // launch, which is what finishes a lone call soonest.
+        const bool series = (params->flags & ARB_ATTN_OVERLAP_PREVIOUS) != 0;
+        if (tensor_cores && !series && decode_step_supported(*params))
+            st = launch_decode_step(c, *params, q, nullptr, nullptr, const_cast<void *>(k_pages),
+                                    const_cast<void *>(v_pages), block_table, const_cast<int32_t *>(seq_lens), q_lens, out, s);
+        else if (tensor_cores && decode_mma_supported(*params))
             st = launch_decode_mma(c, *params, q, k_pages, v_pages, block_table, seq_lens, q_lens, out, s);
         else {
             note_unnumbered_decode(c, decode_workspace_bytes(*params, c->num_sms));  // region 0, no generation number
@@ -212,6 +221,32 @@ arb_status arb_attn(arb_ctx *ctx, const arb_attn_params *params, const void *q, 
         if (st != ARB_OK) return st;
     }
     return ARB_OK;
+}
+
+arb_status arb_decode_step(arb_ctx *ctx, const arb_attn_params *params, const void *q, const void *k_new,
+                           const void *v_new, void *k_pages, void *v_pages, const int32_t *block_table,
+                           int32_t *seq_lens, const int32_t *q_lens, void *out, arb_stream_t stream) {
+    if (ctx == nullptr) return ARB_ERR_INVALID_ARG;
+    arb_status st = check_params(params);
+    if (st != ARB_OK) return st;
+    if (params->max_q_len != 1 || params->total_q < 0 || params->total_q > params->batch) return ARB_ERR_INVALID_ARG;
+    if (params->flags & ARB_ATTN_OVERLAP_PREVIOUS) return ARB_ERR_INVALID_ARG;   // the call writes the cache it reads
+    if (!k_pages || !v_pages || !block_table || !seq_lens || !q_lens) return ARB_ERR_INVALID_ARG;
+    if (params->total_q == 0) return ARB_OK;
+    if (!q || !out || !k_new || !v_new) return ARB_ERR_INVALID_ARG;
+    if (!aligned16(q) || !aligned16(out) || !aligned16(k_pages) || !aligned16(v_pages) || !aligned16(k_new) ||
+        !aligned16(v_new))
+        return ARB_ERR_INVALID_ARG;
+    Ctx *c = reinterpret_cast<Ctx *>(ctx);
+    if (decode_workspace_bytes(*params, c->num_sms) > c->workspace_bytes) return ARB_ERR_WORKSPACE;
+    cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+    if ((params->flags & ARB_ATTN_NO_TENSOR_CORES) == 0 && decode_step_supported(*params))
+        return launch_decode_step(c, *params, q, k_new, v_new, k_pages, v_pages, block_table, seq_lens, q_lens, out, s);
+    // shapes the single launch does not serve (fp32, head_dim 64): the same step as two launches
+    st = launch_kv_append(c, *params, params->total_q, k_new, v_new, block_table, seq_lens, q_lens, 1, k_pages, v_pages, s);
+    if (st != ARB_OK) return st;
+    note_unnumbered_decode(c, decode_workspace_bytes(*params, c->num_sms));
+    return launch_decode(c, *params, q, k_pages, v_pages, block_table, seq_lens, q_lens, out, s);
 }
 
 arb_status arb_attn_decode_static(const arb_attn_params *params, const void *q, const void *k_pages,

@@ -63,6 +63,7 @@ struct Ctx {
     uint32_t decode_gen = 1000;          // generation of the next tensor-core decode call
     uint32_t rot_wait_through = 0;        // tensor-core decode calls up to this generation wait for their predecessor
     double *spearman_acc = nullptr;       // three fp64 accumulators of arb_spearman
+    bool step_deep_ring = true;           // single-launch decode: 32-stage ring (one CTA per SM) rather than 16 stages
     float *chunk_ws = nullptr;            // partial results of split long sequences (step-chunk attention)
     size_t chunk_ws_bytes = 0;
 };
@@ -261,6 +262,10 @@ arb_status launch_kv_append_e4m3(Ctx *ctx, const arb_attn_params &p, int total_n
 arb_status launch_decode_e4m3(Ctx *ctx, const arb_attn_params &p, const void *q, const void *k_pages,
                               const void *v_pages, float k_scale, float v_scale, const int32_t *block_table,
                               const int32_t *seq_lens, const int32_t *q_lens, void *out, cudaStream_t stream);
+bool decode_step_supported(const arb_attn_params &p);
+arb_status launch_decode_step(Ctx *ctx, const arb_attn_params &p, const void *q, const void *k_new, const void *v_new,
+                              void *k_pages, void *v_pages, const int32_t *block_table, int32_t *seq_lens,
+                              const int32_t *q_lens, void *out, cudaStream_t stream);
 arb_status launch_selftest_wait(Ctx *ctx, long long limit_cycles, int32_t *report, cudaStream_t stream);
 size_t decode_workspace_bytes(const arb_attn_params &p, int num_sms);
 int decode_grid(int num_sms);

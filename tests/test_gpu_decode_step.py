@@ -1,0 +1,180 @@
+"""arb_decode_step -- one decode token in one launch (cache write, attention, combine, length update) -- against
+the oracle's kv_append followed by its attention: pools bit for bit, lengths exact, rows within tolerance."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import oracle
+from paper_2512_05033_b200 import workloads as wl
+from tests import helpers as H
+
+pytestmark = pytest.mark.gpu
+BF, F32 = torch.bfloat16, torch.float32
+
+
+def _new_rows(inp, n, seed):
+    Hkv, D = inp.k_pages.shape[1], inp.k_pages.shape[3]
+    return (wl.normal((n, Hkv, D), 1.0, inp.q.dtype, "cpu", seed), wl.normal((n, Hkv, D), 1.0, inp.q.dtype, "cpu", seed + 1))
+
+
+def _run(c, inp, k_new, v_new, dev=None):
+    """One step on the device and through the oracle.  `inp.seq_lens` are the lengths BEFORE the token.
+    Returns (out, pools, lens, bits) of the device and (out, pools, lens, status) of the oracle."""
+    d = dev or inp.to("cuda")
+    out = torch.full_like(d.q, float("nan"))
+    c.decode_step(d.q, k_new.cuda(), v_new.cuda(), d.k_pages, d.v_pages, d.block_table, d.seq_lens, d.q_lens, out=out)
+    bits = c.poll_status()
+    ok, ov, osl, st = oracle.kv_append(k_new, v_new, inp.block_table, inp.seq_lens, inp.q_lens, inp.k_pages, inp.v_pages)
+    ref, st2 = oracle.attn(inp.q, ok, ov, inp.block_table, osl, inp.q_lens)
+    return (out, d, bits), (ref, ok, ov, osl, st | st2)
+
+
+def _same_bits(a, b):
+    """Bit-for-bit equality (pools may hold NaN on purpose)."""
+    it = torch.int16 if a.element_size() == 2 else torch.int32
+    return torch.equal(a.cpu().contiguous().view(it), b.cpu().contiguous().view(it))
+
+
+def _check(got, exp, dt, tight):
+    (out, d, bits), (ref, ok, ov, osl, st) = got, exp
+    assert bits == 0 and st == 0
+    assert np.array_equal(d.seq_lens.cpu().numpy(), osl)
+    assert _same_bits(d.k_pages, ok) and _same_bits(d.v_pages, ov)
+    H.assert_close(out.double().cpu().numpy(), ref, dt, tight=tight if dt == BF else None)
+
+
+STEP_CASES = [
+    # (B, Hq, Hkv, D, dtype, lengths before the token, q_lens)
+    (3, 12, 2, 128, BF, [15, 16, 17], [1, 1, 1]),                       # last slot of a page, first slot of a new page
+    (4, 12, 2, 128, BF, [0, 1, 31, 32], [1, 1, 1, 1]),                  # an empty sequence: the token is its only key
+    (8, 12, 2, 128, BF, [1025, 2000, 3001, 777, 4096, 1, 640, 5555], [1] * 8),   # draft-shaped, ragged
+    (4, 32, 8, 128, BF, [4100, 9000, 33, 12000], [1, 1, 1, 1]),         # target-shaped heads
+    (2, 28, 4, 128, BF, [3000, 150], [1, 1]),                           # g = 7
+    (5, 16, 2, 128, BF, [2100, 5, 900, 77, 4000], [1, 0, 1, 0, 1]),     # g = 8, idle slots
+    (1, 5, 1, 128, BF, [40000], [1]),                                   # one long sequence over every CTA
+    (2, 8, 8, 128, BF, [260, 100], [1, 1]),                             # g = 1
+    (16, 32, 8, 128, BF, [100 * i + 7 for i in range(16)], [1] * 16),   # many short segments per CTA
+    (1, 8, 2, 64, F32, [512], [1]),                                     # the tiny config's shape: two launches inside
+    (2, 6, 2, 64, BF, [700, 70], [1, 1]),                               # bf16, head_dim 64: two launches inside
+]
+
+
+@pytest.mark.parametrize("case", STEP_CASES)
+def test_decode_step_matches_append_then_attention(case):
+    B, Hq, Hkv, D, dt, sl, ql = case
+    inp = wl.small_attn_case(B, Hq, Hkv, D, dt, sl, ql, seed=800 + len(sl) + Hq, extra_tokens=4)
+    k_new, v_new = _new_rows(inp, sum(ql), 8100 + Hq)
+    single = dt == BF and D == 128
+    _check(*_run(H.ctx(), inp, k_new, v_new), dt, 3e-3 if single else 1e-3)
+
+
+def test_decode_step_over_stale_slots_after_a_rollback():
+    """A rejected step leaves its slots behind: beyond the length they hold anything (NaN here).  The next token
+    overwrites the first of them and must see none of the others."""
+    c = H.ctx()
+    sl = [3000, 45, 640, 16]
+    inp = wl.small_attn_case(4, 12, 2, 128, BF, sl, [1] * 4, seed=77, extra_tokens=40)
+    for b, L in enumerate(sl):                       # poison everything from position L on, 30 tokens deep
+        for pos in range(L, L + 30):
+            page = int(inp.block_table[b, pos // 16])
+            inp.k_pages[page, :, pos % 16, :] = float("nan")
+            inp.v_pages[page, :, pos % 16, :] = float("nan")
+    k_new, v_new = _new_rows(inp, 4, 91)
+    _check(*_run(c, inp, k_new, v_new), BF, 3e-3)
+
+
+def test_decode_step_chain_in_place():
+    """Twenty tokens in a row on the same cache: every call finds the lengths the previous one left, in place, with
+    the set of active sequences changing from token to token; then the same chain replayed as one CUDA graph."""
+    c = H.ctx()
+    B, T = 6, 20
+    inp = wl.small_attn_case(B, 12, 2, 128, BF, [500, 33, 2100, 0, 1500, 64], [1] * B, seed=78, extra_tokens=T + 2)
+    g = torch.Generator().manual_seed(5)
+    active = (torch.rand(T, B, generator=g) < 0.7).to(torch.int32)
+    active[:, 0] = 1
+    q = wl.normal((T, B, 12, 128), 1.0, BF, "cpu", 79)
+    kn = wl.normal((T, B, 2, 128), 1.0, BF, "cpu", 80)
+    vn = wl.normal((T, B, 2, 128), 1.0, BF, "cpu", 81)
+    d = inp.to("cuda")
+    start = (d.k_pages.clone(), d.v_pages.clone(), d.seq_lens.clone())
+    dq, dk, dv, dact = q.cuda(), kn.cuda(), vn.cuda(), active.cuda()
+    outs = [torch.full((B, 12, 128), float("nan"), dtype=BF, device="cuda") for _ in range(T)]
+
+    def chain():
+        for t in range(T):
+            n = int(active[t].sum())
+            p = c.params_for(dq[t][:n], d.k_pages, d.block_table, 1)
+            c.decode_step(dq[t][:n], dk[t][:n], dv[t][:n], d.k_pages, d.v_pages, d.block_table, d.seq_lens, dact[t],
+                          out=outs[t][:n], params=p)
+
+    chain()
+    assert c.poll_status() == 0
+    k, v, sl = inp.k_pages, inp.v_pages, inp.seq_lens.numpy()
+    refs = []
+    for t in range(T):
+        n = int(active[t].sum())
+        k, v, sl, st = oracle.kv_append(kn[t][:n], vn[t][:n], inp.block_table, sl, active[t], k, v)
+        ref, st2 = oracle.attn(q[t][:n], k, v, inp.block_table, sl, active[t])
+        assert st == 0 and st2 == 0
+        refs.append(ref)
+        H.assert_close(outs[t][:n].double().cpu().numpy(), ref, BF, tight=3e-3)
+    assert np.array_equal(d.seq_lens.cpu().numpy(), sl)
+    assert torch.equal(d.k_pages.cpu(), k) and torch.equal(d.v_pages.cpu(), v)
+    # the same chain as a graph, replayed twice from the starting state
+    eager = [o.clone() for o in outs]
+    gr = torch.cuda.CUDAGraph()
+    for t_, s_ in zip((d.k_pages, d.v_pages, d.seq_lens), start):
+        t_.copy_(s_)
+    with torch.cuda.graph(gr):
+        chain()
+    for rep in range(2):
+        for t_, s_ in zip((d.k_pages, d.v_pages, d.seq_lens), start):
+            t_.copy_(s_)
+        for o in outs:
+            o.fill_(float("nan"))
+        gr.replay()
+        torch.cuda.synchronize()
+        for t in range(T):
+            n = int(active[t].sum())
+            assert torch.equal(outs[t][:n], eager[t][:n]), (rep, t)
+        assert np.array_equal(d.seq_lens.cpu().numpy(), sl)
+    assert c.poll_status() == 0
+
+
+def test_decode_step_refuses_what_does_not_fit():
+    """A token that does not fit under the block-table row: the sequence is left untouched, its row is zero, the bit
+    is raised; a new row whose page lies outside the pool is not written and the length stays."""
+    from paper_2512_05033_b200 import binding
+    c = H.ctx()
+    inp = wl.small_attn_case(3, 12, 2, 128, BF, [100, 64, 300], [1, 1, 1], seed=83)
+    inp.seq_lens[1] = inp.block_table.shape[1] * 16          # full: one more token does not fit
+    k_new, v_new = _new_rows(inp, 3, 84)
+    d = inp.to("cuda")
+    k0, v0 = d.k_pages.clone(), d.v_pages.clone()
+    out = torch.full_like(d.q, float("nan"))
+    c.decode_step(d.q, k_new.cuda(), v_new.cuda(), d.k_pages, d.v_pages, d.block_table, d.seq_lens, d.q_lens, out=out)
+    assert c.poll_status() == binding.DEV_BAD_SEQ_LEN
+    ok, ov, osl, st = oracle.kv_append(k_new, v_new, inp.block_table, inp.seq_lens, inp.q_lens, inp.k_pages, inp.v_pages)
+    assert st == oracle.BAD_SEQ_LEN
+    assert np.array_equal(d.seq_lens.cpu().numpy(), osl)
+    assert torch.equal(d.k_pages.cpu(), ok) and torch.equal(d.v_pages.cpu(), ov)
+    assert float(out[1].abs().max()) == 0.0
+    keep = torch.tensor([1, 0, 1], dtype=torch.int32)
+    ref, _ = oracle.attn(inp.q[[0, 2]], ok, ov, inp.block_table, osl, keep)
+    H.assert_close(out[[0, 2]].double().cpu().numpy(), ref, BF, tight=3e-3)
+    # a page id outside the pool at the new row's place
+    inp2 = wl.small_attn_case(2, 12, 2, 128, BF, [100, 47], [1, 1], seed=85)
+    inp2.block_table[1, 47 // 16] = inp2.k_pages.shape[0] + 5
+    d2 = inp2.to("cuda")
+    k2 = d2.k_pages.clone()
+    kn2, vn2 = _new_rows(inp2, 2, 86)
+    out2 = c.decode_step(d2.q, kn2.cuda(), vn2.cuda(), d2.k_pages, d2.v_pages, d2.block_table, d2.seq_lens, d2.q_lens)
+    assert c.poll_status() == binding.DEV_BAD_PAGE
+    assert d2.seq_lens.cpu().tolist() == [101, 47]
+    assert torch.isfinite(out2.float()).all()
+    changed = (d2.k_pages != k2).flatten(1).any(1).nonzero().flatten().cpu().tolist()
+    assert changed == [int(inp2.block_table[0, 100 // 16])]   # only sequence 0's page was written
+    # host-side refusals
+    p = c.params_for(d2.q, d2.k_pages, d2.block_table, 1, flags=binding.ATTN_OVERLAP_PREVIOUS)
+    with pytest.raises(binding.ArbError):
+        c.decode_step(d2.q, kn2.cuda(), vn2.cuda(), d2.k_pages, d2.v_pages, d2.block_table, d2.seq_lens, d2.q_lens, params=p)

@@ -346,7 +346,8 @@ arb_status arb_kv_append(arb_ctx *ctx, const arb_attn_params *params, int32_t to
  * pays this call once per layer, and each call reads what the one before it wrote, so its latency -- not its
  * bytes -- is what the loop sees).
  *
- *   params     as for arb_attn with max_q_len == 1; total_q = number of sequences with q_lens[b] == 1.
+ *   params     as for arb_attn with max_q_len == 1; total_q >= the number of sequences with q_lens[b] == 1
+ *              (the rows of q, k_new, v_new and out; rows beyond that number are ignored), total_q <= batch.
  *              ARB_ATTN_OVERLAP_PREVIOUS is refused (ARB_ERR_INVALID_ARG): the call writes the cache it reads.
  *   q, out     [total_q, Hq, D], rows in batch order of the sequences that take part.
  *   k_new,

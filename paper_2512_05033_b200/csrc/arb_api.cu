@@ -1,4 +1,5 @@
 // C ABI of the arb library: argument validation, context and dispatch.  No arithmetic here.
+#include <algorithm>
 #include <cstdlib>
 #include <cstring>
 #include <new>
@@ -113,7 +114,8 @@ arb_status arb_create(arb_ctx **out, int device, size_t workspace_bytes) {
         return ARB_ERR_CUDA;
     }
     c->num_sms = sms;
-    if (const char *ring = std::getenv("ARB_STEP_RING")) c->step_deep_ring = std::atoi(ring) != 16;   // tuning knob
+    // tuning knob of the single-launch decode (see Plan in arb_decode_step.cu)
+    if (const char *pct = std::getenv("ARB_STEP_BOUNDARY_PCT")) c->step_boundary_pct = std::max(0, std::min(400, std::atoi(pct)));
     c->workspace_bytes = workspace_bytes ? workspace_bytes : kDefaultWorkspace;
     c->counters_len = kCounters;
     bool ok = cudaMalloc(&c->workspace, c->workspace_bytes) == cudaSuccess;

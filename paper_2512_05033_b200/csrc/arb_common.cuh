@@ -63,7 +63,7 @@ struct Ctx {
     uint32_t decode_gen = 1000;          // generation of the next tensor-core decode call
     uint32_t rot_wait_through = 0;        // tensor-core decode calls up to this generation wait for their predecessor
     double *spearman_acc = nullptr;       // three fp64 accumulators of arb_spearman
-    bool step_deep_ring = true;           // single-launch decode: 32-stage ring (one CTA per SM) rather than 16 stages
+    int step_boundary_pct = 100;          // single-launch decode: what a (sequence, kv head) boundary inside a CTA's range counts for
     float *chunk_ws = nullptr;            // partial results of split long sequences (step-chunk attention)
     size_t chunk_ws_bytes = 0;
 };

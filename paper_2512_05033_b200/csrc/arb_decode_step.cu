@@ -37,10 +37,12 @@ constexpr int kAuxWarp = kCW + 1;             // bookkeeping: length update, row
 constexpr int kNT = kCT + 64;
 constexpr int kTileBytes = kPage * kD * 2;    // 4 KB: one (page, kv head) tile of K or of V
 constexpr int kHalfTile = kTileBytes / 2;
-constexpr int kBatch = 16;                    // producer lanes issuing side by side
+constexpr int kBatch = 32;                    // producer lanes issuing side by side
 constexpr int kParked = 2;                    // segment results parked in shared memory before they are written
 constexpr int kOStride = kD + 4;              // floats between two heads of a warp record (spreads the banks)
-constexpr int kPreload = 4;                   // parts of a merge asked for before the weights are known
+// What a boundary costs is time (the warps meet, a second arrival, perhaps a second merge), a few microseconds
+// whatever the call's size: as pages it is the CTA's even share, but no more than this many.
+constexpr int kBoundaryCap = 32;
 
 struct StepArgs {
     const char *q;
@@ -57,6 +59,7 @@ struct StepArgs {
     uint32_t *status;
     int batch, Hq, Hkv, num_pages, max_pages;
     int whole_rows;    // the tensor maps are 3-D: one copy per page tile instead of one per half
+    int boundary_pct;  // cost of a (sequence, kv head) boundary inside a CTA's range: percent of min(even share, kBoundaryCap) pages
     float scale_log2;
 };
 
@@ -64,6 +67,7 @@ template <int STAGES>
 struct Tail {
     uint64_t full[STAGES];
     uint64_t empty[STAGES];
+    uint64_t merge_bar;   // the bulk copies of a merge
     int abort;
     int last[kParked];
 };
@@ -81,7 +85,7 @@ template <int G, int STAGES>
 size_t smem_bytes(int batch) {
     using C = Cfg<G>;
     return 1024 + (size_t)STAGES * kTileBytes + C::OSM_BYTES + C::PARK_BYTES + sizeof(Tail<STAGES>) +
-           sizeof(int) * (3 * (size_t)batch + 2);
+           sizeof(int) * (4 * (size_t)batch + 3 + 8);
 }
 
 struct Parked {
@@ -116,8 +120,85 @@ __device__ __forceinline__ bool step_ok(int n, int L0, int max_pages) {
     return L0 >= (APPEND ? 0 : 1) && L <= (long long)max_pages * kPage;
 }
 
+// a / b for 0 <= a, 0 < b: through the float reciprocal with a correction step while a is exactly representable
+// (the plan sits on every CTA's path to its first copy, and an integer division is some forty dependent instructions)
+__device__ __forceinline__ int fast_div(int a, int b) {
+    if (a >= (1 << 24)) return a / b;
+    int q = __float2int_rz(__fdividef((float)a, (float)b));
+    const int r = a - q * b;
+    if (r < 0) --q; else if (r >= b) ++q;
+    return q;
+}
+
+// a / b where the quotient is a kv head index (small): a few subtractions beat any division
+__device__ __forceinline__ int small_div(int a, int b, int &rem) {
+    int q = 0;
+    while (a >= b) { a -= b; ++q; }
+    rem = a;
+    return q;
+}
+
+// The cut of the flat (sequence, kv head, page) list into per-CTA ranges.  A CTA whose range crosses from one
+// (sequence, kv head) into the next pays for it (the warps meet, their records are merged, the next q is
+// loaded), and it then tends to be the last to arrive at both items and merges both.  So a boundary counts as
+// `pen` pages of work: the list is cut evenly in a padded coordinate in which every item is preceded by `pen`
+// virtual pages.  Item j (in list order) with real range [s, s + n) occupies [s + j pen, s + (j + 1) pen + n) there,
+// its real pages the last n of them.  Everything after the cut works in real coordinates.
+struct Plan {
+    const int *pref;   // [B + 1] real flat start of sequence b (pages times kv heads)
+    const int *act;    // [B + 1] sequences before b that take part
+    const int *slen;   // [B] length of sequence b (with the new token)
+    int B, Hkv, pen, chunk, total_padded;
+
+    __device__ __forceinline__ int pages_of(int b) const { return pref[b + 1] != pref[b] ? (slen[b] + kPage - 1) / kPage : 0; }
+    __device__ __forceinline__ int padded_start(int b) const { return pref[b] + pen * Hkv * act[b]; }
+    // real flat position of padded position r inside sequence b (a virtual page maps to the first real page behind it)
+    __device__ __forceinline__ int real_in(int b, long long r) const {
+        const int pages = pages_of(b);
+        int o2;
+        const int kvh = small_div((int)r - padded_start(b), pages + pen, o2);
+        return pref[b] + kvh * pages + max(0, o2 - pen);
+    }
+    // the CTA that holds real page `pg` of item (b, kvh)
+    __device__ __forceinline__ int cta_of(int b, int kvh, int pages, int pg) const {
+        return fast_div(padded_start(b) + kvh * (pages + pen) + pen + pg, chunk);
+    }
+    // the sequence that holds real flat position r, walking up from a sequence known to start at or before r
+    __device__ __forceinline__ int seq_of(int r, int b) const {
+        while (b + 1 < B && pref[b + 1] <= r) ++b;
+        return b;
+    }
+};
+
+// Next segment of the real flat range [cur, r1); `b` is the sequence of the segment before (or of r0) and moves along.
+__device__ __forceinline__ bool next_segment(int &cur, int r1, int &b, const Plan &pl, Segment &s) {
+    if (cur >= r1) return false;
+    b = pl.seq_of(cur, b);
+    const int pages = pl.pages_of(b);
+    int pg0;
+    const int kvh = small_div(cur - pl.pref[b], pages, pg0);
+    const int s1 = pl.pref[b] + (kvh + 1) * pages;
+    const int end = s1 < r1 ? s1 : r1;
+    s.b = b;
+    s.kvh = kvh;
+    s.pg0 = pg0;
+    s.pg1 = pg0 + (end - cur);
+    s.L = pl.slen[b];
+    s.bk = b * pl.Hkv + kvh;
+    s.c_first = -1;   // filled in by parts_of when the segment's result is parked
+    s.nparts = 0;
+    cur = end;
+    return true;
+}
+
+__device__ __forceinline__ void parts_of(const Plan &pl, Segment &s) {
+    const int pages = pl.pages_of(s.b);
+    s.c_first = pl.cta_of(s.b, s.kvh, pages, 0);
+    s.nparts = pl.cta_of(s.b, s.kvh, pages, pages - 1) - s.c_first + 1;
+}
+
 template <int G, int STAGES, bool APPEND>
-__global__ void __launch_bounds__(kNT, STAGES <= 16 ? 2 : 1)
+__global__ void __launch_bounds__(kNT, 1)
 decode_step_kernel(const StepArgs a, const __grid_constant__ CUtensorMap k_map, const __grid_constant__ CUtensorMap v_map) {
     using C = Cfg<G>;
     using Tail = arb::Tail<STAGES>;
@@ -134,7 +215,9 @@ decode_step_kernel(const StepArgs a, const __grid_constant__ CUtensorMap k_map, 
     Tail *tail = reinterpret_cast<Tail *>(base + kRingBytes + C::OSM_BYTES + C::PARK_BYTES);
     int *pref = reinterpret_cast<int *>(tail + 1);
     int *row0 = pref + a.batch + 1;
-    int *slen = row0 + a.batch + 1;
+    int *act = row0 + a.batch + 1;
+    int *slen = act + a.batch + 1;
+    int *plan_s = slen + a.batch;    // [8]: this CTA's cut, worked out by warp 0
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int B = a.batch, Hkv = a.Hkv;
@@ -149,10 +232,12 @@ decode_step_kernel(const StepArgs a, const __grid_constant__ CUtensorMap k_map, 
             mbar_init(&tail->full[s], 1);
             mbar_init(&tail->empty[s], 1);
         }
+        mbar_init(&tail->merge_bar, 1);
         tail->abort = 0;
         mbar_fence_init();
         pref[0] = 0;
         row0[0] = 0;
+        act[0] = 0;
     }
     // Everything below may read what the kernel before this one wrote (lengths, q, new rows, the cache).
     wait_for_predecessor();
@@ -164,24 +249,59 @@ decode_step_kernel(const StepArgs a, const __grid_constant__ CUtensorMap k_map, 
         const int L = L0 + (APPEND ? 1 : 0);
         pref[b + 1] = ok ? (L + kPage - 1) / kPage * Hkv : 0;
         row0[b + 1] = n > 0 ? n : 0;
+        act[b + 1] = ok ? 1 : 0;
         slen[b] = L;
     }
     __syncthreads();
     if (warp == 0) {
-        int carry_p = 0, carry_r = 0;
+        int carry_p = 0, carry_r = 0, carry_a = 0;
         for (int b0 = 0; b0 < B; b0 += 32) {
             const int b = b0 + lane;
             int vp = b < B ? pref[b + 1] : 0;
             int vr = b < B ? row0[b + 1] : 0;
+            int va = b < B ? act[b + 1] : 0;
 #pragma unroll
             for (int off = 1; off < 32; off <<= 1) {
                 const int tp = __shfl_up_sync(0xffffffffu, vp, off);
                 const int tr = __shfl_up_sync(0xffffffffu, vr, off);
-                if (lane >= off) { vp += tp; vr += tr; }
+                const int ta = __shfl_up_sync(0xffffffffu, va, off);
+                if (lane >= off) { vp += tp; vr += tr; va += ta; }
             }
-            if (b < B) { pref[b + 1] = vp + carry_p; row0[b + 1] = vr + carry_r; }
+            if (b < B) { pref[b + 1] = vp + carry_p; row0[b + 1] = vr + carry_r; act[b + 1] = va + carry_a; }
             carry_p += __shfl_sync(0xffffffffu, vp, 31);
             carry_r += __shfl_sync(0xffffffffu, vr, 31);
+            carry_a += __shfl_sync(0xffffffffu, va, 31);
+        }
+        // The cut, while the warp is at it: an even share of the padded list per CTA; both ends of this CTA's range
+        // are looked up with one ballot per 32 sequences (the padded starts ascend, so the sequence that holds a
+        // position is the last one that starts at or before it) instead of a search in every warp.
+        __syncwarp();
+        Plan pl;
+        pl.pref = pref; pl.act = act; pl.slen = slen; pl.B = B; pl.Hkv = Hkv;
+        const int total = pref[B], items = act[B] * Hkv, grid = (int)gridDim.x;
+        const int even = max(kMinChunk, fast_div(total + grid - 1, grid));
+        pl.pen = items > 1 ? (min(even, kBoundaryCap) * a.boundary_pct + 99) / 100 : 0;
+        pl.total_padded = total + pl.pen * items;
+        pl.chunk = max(kMinChunk, fast_div(pl.total_padded + grid - 1, grid));
+        int ends[2], seq0 = 0;
+#pragma unroll
+        for (int w = 0; w < 2; ++w) {
+            const long long t = (long long)(blockIdx.x + w) * pl.chunk;
+            int best = 0;
+            for (int b0 = 0; b0 < B; b0 += 32) {
+                const int b = b0 + lane;
+                const unsigned mask = __ballot_sync(0xffffffffu, b < B && pl.padded_start(b) <= t);
+                if (mask) best = b0 + 31 - __clz(mask);
+            }
+            ends[w] = t >= pl.total_padded ? total : pl.real_in(best, t);
+            if (w == 0) seq0 = best;
+        }
+        if (lane == 0) {
+            plan_s[0] = ends[0];
+            plan_s[1] = ends[1];
+            plan_s[2] = pl.pen;
+            plan_s[3] = pl.chunk;
+            plan_s[4] = seq0;
         }
     }
     __syncthreads();
@@ -219,55 +339,67 @@ decode_step_kernel(const StepArgs a, const __grid_constant__ CUtensorMap k_map, 
         return;
     }
 
-    const int total = pref[B];
-    int chunk = (total + (int)gridDim.x - 1) / (int)gridDim.x;
-    if (chunk < kMinChunk) chunk = kMinChunk;
-    const long long r0l = (long long)blockIdx.x * chunk;
-    if (r0l >= total) return;
-    const int r0 = (int)r0l;
-    const int r1 = min(total, r0 + chunk);
+    Plan pl;
+    pl.pref = pref;
+    pl.act = act;
+    pl.slen = slen;
+    pl.B = B;
+    pl.Hkv = Hkv;
+    const int r0 = plan_s[0], r1 = plan_s[1], seq0 = plan_s[4];
+    pl.pen = plan_s[2];
+    pl.chunk = plan_s[3];
+    pl.total_padded = 0;   // only the cut needs it
+    if (r0 >= r1) return;
     volatile int *abort = &tail->abort;
 
     if (warp == kProdWarp) {
         // ================================ producer warp ==========================================
-        // Tiles enter the ring page by page, K then V; lanes 0 .. kBatch-1 each own one stage at a time.
+        // The CTA's flat range of (sequence, kv head, page) triples goes through in groups of 32: lane i finds
+        // triple i of the group (a short walk up the prefix table from the range's first sequence) and fetches its block-table entry; the entries
+        // of the next group are asked for before the tiles of this one are issued, so that the look-up is off the
+        // path after the first group, across sequence boundaries too.  Tiles enter the ring page by page, K then
+        // V; lanes 0 .. kBatch-1 each own one stage at a time.
+        const int nflat = r1 - r0;
+        auto tile_row = [&](int r) -> int {   // first row, in the 2-D view of the pool, of the tile of flat triple r
+            const int lo = pl.seq_of(r, seq0);
+            const int pages = pl.pages_of(lo);
+            int pg;
+            const int kvh = small_div(r - pref[lo], pages, pg);
+            int pid = a.block_table[(size_t)lo * a.max_pages + pg];
+            if ((unsigned)pid >= (unsigned)a.num_pages) {
+                atomicOr(a.status, (uint32_t)ARB_DEV_BAD_PAGE);
+                pid = 0;
+            }
+            return (pid * Hkv + kvh) * kPage;
+        };
         uint32_t c = 0;
-        int cur = r0;
-        Segment s;
-        while (next_segment(cur, r1, pref, slen, B, Hkv, chunk, s)) {
-            for (int sp0 = s.pg0; sp0 < s.pg1; sp0 += 32) {
-                const int np = min(32, s.pg1 - sp0);
-                int pid = 0;
-                if (lane < np) {
-                    pid = a.block_table[(size_t)s.b * a.max_pages + sp0 + lane];
-                    if ((unsigned)pid >= (unsigned)a.num_pages) {
-                        atomicOr(a.status, (uint32_t)ARB_DEV_BAD_PAGE);
-                        pid = 0;
-                    }
-                }
-                const int ntiles = 2 * np;
+        int row_next = lane < nflat ? tile_row(r0 + lane) : 0;
+        for (int g0 = 0; g0 < nflat; g0 += 32) {
+            const int row_cur = row_next;
+            const int ntiles = 2 * min(32, nflat - g0);
 #pragma unroll 1
-                for (int i0 = 0; i0 < ntiles; i0 += kBatch) {
-                    const int i = i0 + lane;
-                    const int pg = __shfl_sync(0xffffffffu, pid, (i >> 1) & 31);
-                    if (lane < kBatch && i < ntiles) {
-                        const uint32_t cc = c + i, st = cc % STAGES, par = (cc / STAGES) & 1u;
-                        const CUtensorMap *map = (i & 1) ? &v_map : &k_map;
-                        if (mbar_wait(&tail->empty[st], par ^ 1u, abort, a.status)) {
-                            mbar_arrive_expect_tx(&tail->full[st], kTileBytes);
-                            const int row = (pg * Hkv + s.kvh) * kPage;
-                            if (a.whole_rows) {
-                                tma_box_load3(ring + st * kTileBytes, map, 0, row, 0, &tail->full[st]);
-                            } else {
-                                tma_box_load(ring + st * kTileBytes, map, 0, row, &tail->full[st]);
-                                tma_box_load(ring + st * kTileBytes + kHalfTile, map, 64, row, &tail->full[st]);
-                            }
+            for (int i0 = 0; i0 < ntiles; i0 += kBatch) {
+                // the next group's look-up goes out behind this group's first copies, not in front of them
+                if (i0 == kBatch && g0 + 32 + lane < nflat) row_next = tile_row(r0 + g0 + 32 + lane);
+                const int i = i0 + lane;
+                const int row = __shfl_sync(0xffffffffu, row_cur, (i >> 1) & 31);
+                if (i < ntiles) {
+                    const uint32_t cc = c + i, st = cc % STAGES, par = (cc / STAGES) & 1u;
+                    const CUtensorMap *map = (i & 1) ? &v_map : &k_map;
+                    if (mbar_wait(&tail->empty[st], par ^ 1u, abort, a.status)) {
+                        mbar_arrive_expect_tx(&tail->full[st], kTileBytes);
+                        if (a.whole_rows) {
+                            tma_box_load3(ring + st * kTileBytes, map, 0, row, 0, &tail->full[st]);
+                        } else {
+                            tma_box_load(ring + st * kTileBytes, map, 0, row, &tail->full[st]);
+                            tma_box_load(ring + st * kTileBytes + kHalfTile, map, 64, row, &tail->full[st]);
                         }
                     }
-                    __syncwarp();
                 }
-                c += ntiles;
+                __syncwarp();
             }
+            if (ntiles <= kBatch && g0 + 32 + lane < nflat) row_next = tile_row(r0 + g0 + 32 + lane);
+            c += ntiles;
         }
         // After a timeout the consumers may have left copies unconsumed: wait (bounded) for the last ring's
         // worth, so that no copy is in flight into this CTA's shared memory when it exits.
@@ -319,6 +451,7 @@ decode_step_kernel(const StepArgs a, const __grid_constant__ CUtensorMap k_map, 
         }
         if (any_multi) {
             __threadfence();
+            asm volatile("fence.proxy.async;" ::: "memory");   // the partials are read back through bulk copies
             named_barrier(1, kCT);
             if (tid == 0) {
                 int old[kParked];
@@ -345,18 +478,25 @@ decode_step_kernel(const StepArgs a, const __grid_constant__ CUtensorMap k_map, 
         n_parked = 0;
     };
 
-    while (next_segment(cur, r1, pref, slen, B, Hkv, chunk, s)) {
-        const int qrow = row0[s.b];
-        // B fragments of q^T (128 dims x 8 heads): k-slice ks holds dims 16 ks + 2 tq, + 1 and + 8 of head gq
-        uint32_t qb[8][2];
-        {
-            const char *qh = a.q + ((size_t)qrow * a.Hq + s.kvh * G + (head_ok ? gq : 0)) * kD * 2;
+    // B fragments of q^T (128 dims x 8 heads): k-slice ks holds dims 16 ks + 2 tq, + 1 and + 8 of head gq.  The
+    // fragments of the next segment are asked for while this one streams.
+    uint32_t qb[8][2], qn[8][2];
+    auto load_q = [&](const Segment &g, uint32_t (&dst)[8][2]) {
+        const char *qh = a.q + ((size_t)row0[g.b] * a.Hq + g.kvh * G + (head_ok ? gq : 0)) * kD * 2;
 #pragma unroll
-            for (int ks = 0; ks < 8; ++ks) {
-                qb[ks][0] = head_ok ? __ldg(reinterpret_cast<const uint32_t *>(qh + ks * 32 + tq * 4)) : 0u;
-                qb[ks][1] = head_ok ? __ldg(reinterpret_cast<const uint32_t *>(qh + ks * 32 + 16 + tq * 4)) : 0u;
-            }
+        for (int ks = 0; ks < 8; ++ks) {
+            dst[ks][0] = head_ok ? __ldg(reinterpret_cast<const uint32_t *>(qh + ks * 32 + tq * 4)) : 0u;
+            dst[ks][1] = head_ok ? __ldg(reinterpret_cast<const uint32_t *>(qh + ks * 32 + 16 + tq * 4)) : 0u;
         }
+    };
+    Segment s_next;
+    int seq_at = seq0;
+    bool have = next_segment(cur, r1, seq_at, pl, s);
+    if (have) load_q(s, qb);
+    while (have) {
+        const bool have_next = next_segment(cur, r1, seq_at, pl, s_next);
+        if (have_next) load_q(s_next, qn);
+        const int qrow = row0[s.b];
         // The token's new row: it belongs in slot (L - 1) mod 16 of the sequence's last page.  The warp that owns
         // that page fetches the row (lanes 0..15: K, lanes 16..31: V, 16 bytes each), stores it to the pool and
         // patches it into the tiles when they arrive.
@@ -505,79 +645,120 @@ decode_step_kernel(const StepArgs a, const __grid_constant__ CUtensorMap k_map, 
             dst[2 * GP + idx] = acc;
             if (d == 0) { dst[h] = M; dst[GP + h] = l; }
         }
+        parts_of(pl, s);
         pk[n_parked].bk = s.bk;
         pk[n_parked].nparts = s.nparts;
         pk[n_parked].c_first = s.c_first;
         pk[n_parked].out_base = ((size_t)qrow * a.Hq + s.kvh * G) * kD;
         ++n_parked;
         named_barrier(1, kCT);   // warp records are free for the next segment
+        s = s_next;
+        have = have_next;
+#pragma unroll
+        for (int ks = 0; ks < 8; ++ks) { qb[ks][0] = qn[ks][0]; qb[ks][1] = qn[ks][1]; }
     }
     if (n_parked > 0) flush();
 
     // ---- merges of the split (sequence, kv head)s this CTA was the last to reach ------------------------
-    // One 4-dimension piece of the group's G x 128 outputs per thread:
-    //     m = max_p m_p,  w_p = 2^(m_p - m),  out = sum_p w_p o_p / sum_p w_p l_p.
-    // The (max, sum) records of the parts go to shared memory (the warp records are idle by now); the first
-    // partial values are asked for before the weights exist, so that the two round trips run side by side.
+    //     m = max_p m_p,  w_p = 2^(m_p - m),  out = sum_p w_p o_p / sum_p w_p l_p,
+    // one 4-dimension piece of the group's G x 128 outputs per thread.  The parts of an item lie in consecutive
+    // workspace slots, and the ring is idle by now (every tile has been consumed, the producer issues nothing
+    // more): one bulk copy brings the (max, sum) records, one the partial outputs -- a single round trip however
+    // many parts there are -- and the sum runs out of shared memory.  More parts than the ring holds go in pieces.
     constexpr int VECS = G * kD / 4;
+    constexpr int kPartBytes = G * kD * 4;
     static_assert(VECS <= kCT, "one piece per consumer thread");
-    float2 *ml_s = reinterpret_cast<float2 *>(osm);
-    for (int j = 0; j < pend_n; ++j) {
-        const int nparts = pend[j].nparts;
-        const size_t slot0 = (size_t)pend[j].slot0;
-        const bool mine = tid < VECS;
-        const int e = mine ? tid : 0, eh = e / (kD / 4);
-        const float4 *po = reinterpret_cast<const float4 *>(a.part_o + slot0 * G * kD);
-        float4 v[kPreload];
-#pragma unroll
-        for (int u = 0; u < kPreload; ++u) v[u] = __ldcg(po + (size_t)min(u, nparts - 1) * VECS + e);
-        for (int i = tid; i < nparts * G; i += kCT) {
-            const int p = i / G, h = i - p * G;
-            ml_s[i] = __ldcg(reinterpret_cast<const float2 *>(a.part_ml + ((slot0 + p) * GP + h) * 2));
+    if (pend_n == 0) return;
+    // up to two merges, each in its own half of the ring, their first copies in flight together
+    const int cap = kRingBytes / pend_n;
+    const bool mine = tid < VECS;
+    const int e = mine ? tid : 0, eh = e / (kD / 4);
+    uint32_t merge_phase = 0;
+    float m[2] = {-INFINITY, -INFINITY}, l[2] = {0.f, 0.f};
+    float4 x[2] = {make_float4(0.f, 0.f, 0.f, 0.f), make_float4(0.f, 0.f, 0.f, 0.f)};
+    int done[2] = {0, 0};
+    auto ml_area = [&](int j) -> uint32_t { return ((uint32_t)pend[j].nparts * GP * 8u + 127u) & ~127u; };
+    auto per_piece = [&](int j) -> int { return (cap - (int)ml_area(j)) / kPartBytes; };   // >= 6: at most 148 parts of 64-byte records
+    auto issue = [&](int j, int p0, uint32_t &bytes_out) {   // thread 0
+        const int np = min(per_piece(j), pend[j].nparts - p0);
+        const uint32_t bytes = (uint32_t)np * kPartBytes, ml_bytes = (uint32_t)pend[j].nparts * GP * 8u;
+        char *dst = ring + j * cap;
+        if (p0 == 0) bulk_load(dst, a.part_ml + (size_t)pend[j].slot0 * GP * 2, ml_bytes, &tail->merge_bar);
+        bulk_load(dst + ml_area(j), a.part_o + ((size_t)pend[j].slot0 + p0) * G * kD, bytes, &tail->merge_bar);
+        bytes_out += bytes + (p0 == 0 ? ml_bytes : 0u);
+    };
+    auto add_piece = [&](int j, int p0) {
+        const float2 *ml_s = reinterpret_cast<const float2 *>(ring + j * cap);
+        const float4 *po_s = reinterpret_cast<const float4 *>(ring + j * cap + ml_area(j));
+        const int np = min(per_piece(j), pend[j].nparts - p0);
+        if (p0 == 0)
+            for (int p = 0; p < pend[j].nparts; ++p) m[j] = fmaxf(m[j], ml_s[p * GP + eh].x);
+#pragma unroll 4
+        for (int p = 0; p < np; ++p) {
+            const float2 ml = ml_s[(p0 + p) * GP + eh];
+            const float w = fast_exp2(ml.x - m[j]);
+            const float4 v = po_s[p * VECS + e];
+            l[j] = fmaf(w, ml.y, l[j]);
+            x[j].x = fmaf(w, v.x, x[j].x);
+            x[j].y = fmaf(w, v.y, x[j].y);
+            x[j].z = fmaf(w, v.z, x[j].z);
+            x[j].w = fmaf(w, v.w, x[j].w);
         }
-        named_barrier(1, kCT);
-        float m = -INFINITY;
-        for (int p = 0; p < nparts; ++p) m = fmaxf(m, ml_s[p * G + eh].x);
-        float l = 0.f;
-        float4 x = make_float4(0.f, 0.f, 0.f, 0.f);
-        for (int p0 = 0; p0 < nparts; p0 += kPreload) {
-            if (p0 > 0) {
+        done[j] = p0 + np;
+    };
+    while (true) {
+        bool more = false;
 #pragma unroll
-                for (int u = 0; u < kPreload; ++u) v[u] = __ldcg(po + (size_t)min(p0 + u, nparts - 1) * VECS + e);
-            }
+        for (int j = 0; j < 2; ++j) more = more || (j < pend_n && done[j] < pend[j].nparts);
+        if (!more) break;
+        if (tid == 0) {
+            asm volatile("fence.proxy.async;" ::: "memory");
+            uint32_t bytes = 0;
+            // the expected bytes are known before the copies are issued: same arithmetic as issue()
 #pragma unroll
-            for (int u = 0; u < kPreload; ++u) {
-                if (p0 + u < nparts) {
-                    const float2 ml = ml_s[(p0 + u) * G + eh];
-                    const float w = fast_exp2(ml.x - m);
-                    l = fmaf(w, ml.y, l);
-                    x.x = fmaf(w, v[u].x, x.x);
-                    x.y = fmaf(w, v[u].y, x.y);
-                    x.z = fmaf(w, v[u].z, x.z);
-                    x.w = fmaf(w, v[u].w, x.w);
+            for (int j = 0; j < 2; ++j)
+                if (j < pend_n && done[j] < pend[j].nparts) {
+                    const int np = min(per_piece(j), pend[j].nparts - done[j]);
+                    bytes += (uint32_t)np * kPartBytes + (done[j] == 0 ? (uint32_t)pend[j].nparts * GP * 8u : 0u);
                 }
-            }
+            mbar_arrive_expect_tx(&tail->merge_bar, bytes);
+            uint32_t issued = 0;
+#pragma unroll
+            for (int j = 0; j < 2; ++j)
+                if (j < pend_n && done[j] < pend[j].nparts) issue(j, done[j], issued);
         }
-        if (mine) {
-            const float inv = 1.0f / l;
+        __syncwarp();
+        mbar_wait(&tail->merge_bar, merge_phase & 1u, abort, a.status);
+        ++merge_phase;
+#pragma unroll
+        for (int j = 0; j < 2; ++j)
+            if (j < pend_n && done[j] < pend[j].nparts) add_piece(j, done[j]);
+        named_barrier(1, kCT);   // everyone is done with the ring before the next pieces overwrite it
+    }
+#pragma unroll
+    for (int j = 0; j < 2; ++j) {
+        if (j < pend_n && mine) {
+            const float inv = 1.0f / l[j];
             uint2 o2;
-            o2.x = pack_bf16(x.x * inv, x.y * inv);
-            o2.y = pack_bf16(x.z * inv, x.w * inv);
+            o2.x = pack_bf16(x[j].x * inv, x[j].y * inv);
+            o2.y = pack_bf16(x[j].z * inv, x[j].w * inv);
             *reinterpret_cast<uint2 *>(reinterpret_cast<__nv_bfloat16 *>(a.out) + pend[j].out_base + (size_t)e * 4) = o2;
         }
-        named_barrier(1, kCT);   // ml_s is free for the next merge
     }
 }
 
-// Ring depth.  32 stages (128 KB of tiles in flight per SM, one CTA per SM) serve a call that streams at the
-// pace of the memory system; 16 stages leave room for two CTAs per SM, so the next kernel of a chain of small
-// dependent calls is resident, waiting, while this one finishes.
-template <int G, int STAGES, bool APPEND>
+// Ring depth: 32 stages, 128 KB of tiles in flight per SM with one CTA per SM.  A 16-stage ring with room for two
+// CTAs per SM (so that the next kernel of a chain is resident before this one ends) was measured and is slower on
+// every workload: a lone call is bound by bytes in flight, and the successor's CTAs come up SM by SM as this
+// kernel's CTAs leave anyway.
+constexpr int kStages = 32;
+
+template <int G, bool APPEND>
 arb_status launch_variant(Ctx *ctx, const StepArgs &a, const CUtensorMap &km, const CUtensorMap &vm, cudaStream_t stream) {
     static bool attr_set[64] = {};
     if (!attr_set[ctx->device & 63]) {
-        if (cudaFuncSetAttribute(decode_step_kernel<G, STAGES, APPEND>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 (int)smem_bytes<G, STAGES>(kMaxBatch)) != cudaSuccess)
+        if (cudaFuncSetAttribute(decode_step_kernel<G, kStages, APPEND>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 (int)smem_bytes<G, kStages>(kMaxBatch)) != cudaSuccess)
             return ARB_ERR_CUDA;
         attr_set[ctx->device & 63] = true;
     }
@@ -587,20 +768,18 @@ arb_status launch_variant(Ctx *ctx, const StepArgs &a, const CUtensorMap &km, co
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(ctx->num_sms);
     cfg.blockDim = dim3(kNT);
-    cfg.dynamicSmemBytes = smem_bytes<G, STAGES>(a.batch);
+    cfg.dynamicSmemBytes = smem_bytes<G, kStages>(a.batch);
     cfg.stream = stream;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    if (cudaLaunchKernelEx(&cfg, decode_step_kernel<G, STAGES, APPEND>, a, km, vm) != cudaSuccess) return ARB_ERR_CUDA;
+    if (cudaLaunchKernelEx(&cfg, decode_step_kernel<G, kStages, APPEND>, a, km, vm) != cudaSuccess) return ARB_ERR_CUDA;
     ctx->launches++;
     return ARB_OK;
 }
 
 template <int G>
-arb_status launch_g(Ctx *ctx, const StepArgs &a, const CUtensorMap &km, const CUtensorMap &vm, bool deep, cudaStream_t stream) {
-    if (a.k_new != nullptr)
-        return deep ? launch_variant<G, 32, true>(ctx, a, km, vm, stream) : launch_variant<G, 16, true>(ctx, a, km, vm, stream);
-    return deep ? launch_variant<G, 32, false>(ctx, a, km, vm, stream) : launch_variant<G, 16, false>(ctx, a, km, vm, stream);
+arb_status launch_g(Ctx *ctx, const StepArgs &a, const CUtensorMap &km, const CUtensorMap &vm, cudaStream_t stream) {
+    return a.k_new != nullptr ? launch_variant<G, true>(ctx, a, km, vm, stream) : launch_variant<G, false>(ctx, a, km, vm, stream);
 }
 
 }  // namespace
@@ -648,18 +827,18 @@ arb_status launch_decode_step(Ctx *ctx, const arb_attn_params &p, const void *q,
     a.num_pages = p.num_pages;
     a.max_pages = p.max_pages_per_seq;
     a.whole_rows = whole_rows ? 1 : 0;
+    a.boundary_pct = ctx->step_boundary_pct;
     const float scale = p.softmax_scale > 0.f ? p.softmax_scale : 1.0f / sqrtf((float)p.head_dim);
     a.scale_log2 = scale * 1.4426950408889634f;
-    const bool deep = ctx->step_deep_ring;
     switch (g) {
-        case 1: return launch_g<1>(ctx, a, km, vm, deep, stream);
-        case 2: return launch_g<2>(ctx, a, km, vm, deep, stream);
-        case 3: return launch_g<3>(ctx, a, km, vm, deep, stream);
-        case 4: return launch_g<4>(ctx, a, km, vm, deep, stream);
-        case 5: return launch_g<5>(ctx, a, km, vm, deep, stream);
-        case 6: return launch_g<6>(ctx, a, km, vm, deep, stream);
-        case 7: return launch_g<7>(ctx, a, km, vm, deep, stream);
-        case 8: return launch_g<8>(ctx, a, km, vm, deep, stream);
+        case 1: return launch_g<1>(ctx, a, km, vm, stream);
+        case 2: return launch_g<2>(ctx, a, km, vm, stream);
+        case 3: return launch_g<3>(ctx, a, km, vm, stream);
+        case 4: return launch_g<4>(ctx, a, km, vm, stream);
+        case 5: return launch_g<5>(ctx, a, km, vm, stream);
+        case 6: return launch_g<6>(ctx, a, km, vm, stream);
+        case 7: return launch_g<7>(ctx, a, km, vm, stream);
+        case 8: return launch_g<8>(ctx, a, km, vm, stream);
         default: return ARB_ERR_UNSUPPORTED;
     }
 }

@@ -5,8 +5,8 @@ There are no models in this repository, so the "models" are stand-ins that hand 
 key and value rows; what is real is everything the loop does to the three paged caches and the attention
 work it causes:
 
-  draft cache    the draft model writes its step z_d token by token (arb_kv_append + decode arb_attn per
-                 token); if the step is escalated it drops z_d (arb_rollback) and later absorbs the target's
+  draft cache    the draft model writes its step z_d token by token (one arb_decode_step per token: cache
+                 write, decode attention and length update in one launch); if the step is escalated it drops z_d (arb_rollback) and later absorbs the target's
                  step z_t as one chunk (arb_kv_append + chunk arb_attn)
   router cache   absorbs z_d as one chunk -- the router's single forward over (x, z_d), Section 4.2 -- and
                  the head turns the last token's hidden row into the decision (arb_route); on escalation it
@@ -68,8 +68,13 @@ class StepLoop:
         """Token-by-token generation of a step by the model that owns `c`: q, k_new, v_new are [n_max, B, ...];
         at token t only sequences that take part and have t < step_lens[b] are active."""
         lens = self.ctx.phase_lens_tokens(step_lens, n_max, decisions, want=want, out=self.token_lens[name])
-        for t in range(n_max):
-            self._absorb(f"{name}[{t}]", c, k_new[t], v_new[t], q[t], lens[t], 1)
+        for t in range(n_max):   # one launch per token: cache write, attention and length update (arb_decode_step)
+            key = f"{name}[{t}]"
+            out = self.out.get(key)
+            if out is None or out.shape != q[t].shape:
+                out = self.out[key] = torch.zeros_like(q[t])
+            self.ctx.decode_step(q[t], k_new[t], v_new[t], c.k_pages, c.v_pages, c.block_table, c.seq_lens, lens[t],
+                                 out=out)
 
     # -- one round ---------------------------------------------------------------------------------
     def round(self, step_d, step_t, hidden, acts):

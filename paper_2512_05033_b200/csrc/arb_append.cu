@@ -77,6 +77,7 @@ kv_append_kernel(const AppendArgs a) {
     int *okay = pref + a.batch + 1;    // [B] the sequence's new tokens may be written
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int B = a.batch;
+    pdl_enter();
     if (tid == 0) pref[0] = 0;
     for (int b = tid; b < B; b += kAppendThreads) {
         const uint32_t bad = append_check(a, b);
@@ -142,6 +143,7 @@ kv_append_e4m3_kernel(const AppendArgs a, float k_inv_scale, float v_inv_scale) 
     int *okay = pref + a.batch + 1;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int B = a.batch;
+    pdl_enter();
     if (tid == 0) pref[0] = 0;
     for (int b = tid; b < B; b += kAppendThreads) {
         const uint32_t bad = append_check(a, b);
@@ -234,10 +236,9 @@ arb_status launch_kv_append(Ctx *ctx, const arb_attn_params &p, int total_new, c
     const long long cap = (long long)ctx->num_sms * 4;
     const int grid = (int)(want < 1 ? 1 : (want > cap ? cap : want));
     const size_t smem = sizeof(int) * (2 * (size_t)p.batch + 1);
-    kv_append_kernel<<<grid, kAppendThreads, smem, stream>>>(a);
+    const cudaError_t err = launch_pdl(kv_append_kernel, dim3(grid), dim3(kAppendThreads), smem, stream, a);
     ctx->launches++;
-    if (cudaGetLastError() != cudaSuccess) return ARB_ERR_CUDA;
-    return ARB_OK;
+    return err == cudaSuccess ? ARB_OK : ARB_ERR_CUDA;
 }
 
 arb_status launch_kv_append_e4m3(Ctx *ctx, const arb_attn_params &p, int total_new, const void *k_new,
@@ -267,13 +268,12 @@ arb_status launch_kv_append_e4m3(Ctx *ctx, const arb_attn_params &p, int total_n
     const long long cap = (long long)ctx->num_sms * 4;
     const int grid = (int)(want < 1 ? 1 : (want > cap ? cap : want));
     const size_t smem = sizeof(int) * (2 * (size_t)p.batch + 1);
-    if (p.dtype == ARB_BF16)
-        kv_append_e4m3_kernel<__nv_bfloat16><<<grid, kAppendThreads, smem, stream>>>(a, k_inv_scale, v_inv_scale);
-    else
-        kv_append_e4m3_kernel<float><<<grid, kAppendThreads, smem, stream>>>(a, k_inv_scale, v_inv_scale);
+    const cudaError_t err =
+        p.dtype == ARB_BF16
+            ? launch_pdl(kv_append_e4m3_kernel<__nv_bfloat16>, dim3(grid), dim3(kAppendThreads), smem, stream, a, k_inv_scale, v_inv_scale)
+            : launch_pdl(kv_append_e4m3_kernel<float>, dim3(grid), dim3(kAppendThreads), smem, stream, a, k_inv_scale, v_inv_scale);
     ctx->launches++;
-    if (cudaGetLastError() != cudaSuccess) return ARB_ERR_CUDA;
-    return ARB_OK;
+    return err == cudaSuccess ? ARB_OK : ARB_ERR_CUDA;
 }
 
 }  // namespace arb

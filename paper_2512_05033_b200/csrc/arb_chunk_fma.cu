@@ -49,6 +49,7 @@ __global__ void __launch_bounds__(kThreads) chunk_fma_kernel(const ChunkArgs a) 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int B = a.batch;
     const int row = blockIdx.x / a.Hkv, kvh = blockIdx.x - row * a.Hkv;
+    pdl_enter();
     if (a.skip_rows > 0 && a.needed != nullptr && *a.needed == 0) return;  // the usual case: every chunk was large
 
     if (tid == 0) row0[0] = 0;
@@ -193,9 +194,9 @@ arb_status launch_one(Ctx *ctx, const ChunkArgs &a, int total_q, cudaStream_t st
             return ARB_ERR_CUDA;
         attr_set[ctx->device & 63] = true;
     }
-    chunk_fma_kernel<T, D, G><<<total_q * a.Hkv, kThreads, smem, stream>>>(a);
+    const cudaError_t err = launch_pdl(chunk_fma_kernel<T, D, G>, dim3(total_q * a.Hkv), dim3(kThreads), smem, stream, a);
     ctx->launches++;
-    return cudaGetLastError() == cudaSuccess ? ARB_OK : ARB_ERR_CUDA;
+    return err == cudaSuccess ? ARB_OK : ARB_ERR_CUDA;
 }
 
 template <typename T, int D>

@@ -428,6 +428,7 @@ chunk_mma_kernel(const MmaArgs a, const __grid_constant__ CUtensorMap k_map, con
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int B = a.batch, Hkv = a.Hkv;
 
+    let_successor_start();
     if (tid == 0) {
         mbar_init(&bars->q_full, 2 * kSoftmaxThreads);
         for (int s = 0; s < kStages; ++s) {
@@ -449,6 +450,7 @@ chunk_mma_kernel(const MmaArgs a, const __grid_constant__ CUtensorMap k_map, con
         bars->abort = 0;
         mbar_fence_init();
     }
+    wait_for_predecessor();   // everything below reads what the kernel before this one may have written
     make_plan<G>(a, pl, tid, kThreads, a.work_counter + 1);
     const int total = pl.pref[B];
     if ((int)blockIdx.x >= total) return;  // nothing for this CTA; no TMEM taken, no barrier pending
@@ -818,6 +820,7 @@ chunk_combine_kernel(const MmaArgs a) {
     const Plan pl = plan_arrays(plan_smem, a.batch);
     const int tid = threadIdx.x;
     const int B = a.batch, Hkv = a.Hkv;
+    pdl_enter();
     make_plan<G>(a, pl, tid, kCombineThreads, nullptr);
     constexpr int kQuarters = kD / kCombineDims;
     int job = 0;
@@ -896,15 +899,15 @@ arb_status launch_one(Ctx *ctx, const MmaArgs &a, const CUtensorMap &km, const C
         attr_set[ctx->device & 63] = true;
     }
     const int grid = max_items < ctx->num_sms ? max_items : ctx->num_sms;
-    chunk_mma_kernel<G><<<grid, kThreads, smem, stream>>>(a, km, vm);
+    const cudaError_t err = launch_pdl(chunk_mma_kernel<G>, dim3(grid), dim3(kThreads), smem, stream, a, km, vm);
     ctx->launches++;
-    if (cudaGetLastError() != cudaSuccess) return ARB_ERR_CUDA;
+    if (err != cudaSuccess) return ARB_ERR_CUDA;
     // the merge of split sequences, when the block table is long enough for a sequence to be split at all
     if (a.split_cap > 0) {
         const size_t csmem = sizeof(int) * (7 * (size_t)a.batch + 2);
-        chunk_combine_kernel<G><<<4 * ctx->num_sms, kCombineThreads, csmem, stream>>>(a);
+        const cudaError_t cerr = launch_pdl(chunk_combine_kernel<G>, dim3(4 * ctx->num_sms), dim3(kCombineThreads), csmem, stream, a);
         ctx->launches++;
-        if (cudaGetLastError() != cudaSuccess) return ARB_ERR_CUDA;
+        if (cerr != cudaSuccess) return ARB_ERR_CUDA;
     }
     return ARB_OK;
 }

@@ -201,6 +201,36 @@ __device__ __forceinline__ float fast_exp2(float x) {
     return y;
 }
 
+// Programmatic dependent launch.  Both are no-ops in a kernel launched the ordinary way.
+//  - let_successor_start: the next kernel on the stream, if launched as a programmatic dependent, may come up
+//    once every CTA of this grid has passed this point or exited.
+//  - wait_for_predecessor: returns when the preceding kernel has completed and its writes are visible.
+// Every kernel launched through launch_pdl passes wait_for_predecessor on all its paths before it touches global
+// memory (so that its own completion implies that of everything before it on the stream), and calls
+// let_successor_start at its top: a chain of small dependent kernels then pays no launch latency between them.
+__device__ __forceinline__ void let_successor_start() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void wait_for_predecessor() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_enter() {
+    let_successor_start();
+    wait_for_predecessor();
+}
+
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream,
+                              Args... args) {
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+}
+
 // Transposing reduction of N per-lane values over an aligned group of W lanes (W a power of two,
 // N a multiple of W).  On return v[j], j < N/W, holds the group-wide sum of the original value
 // with index j + (N/W) * (lane % W).  N - N/W shuffles instead of N * log2(W).

@@ -158,12 +158,6 @@ __device__ __forceinline__ float fma_bf16x2(uint32_t q, uint32_t k, float acc) {
 
 __device__ __forceinline__ void fence_proxy_async_all() { asm volatile("fence.proxy.async;" ::: "memory"); }
 
-// Programmatic dependent launch.  Both are no-ops in a kernel launched the ordinary way.
-//  - let_successor_start: the next kernel on the stream, if launched as a programmatic dependent,
-//    may begin once every CTA of this grid has passed this point or exited.
-//  - wait_for_predecessor: returns when the preceding kernel has completed and its writes are visible.
-__device__ __forceinline__ void let_successor_start() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
-__device__ __forceinline__ void wait_for_predecessor() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 
 template <typename T, int D, int G>
 __global__ void __launch_bounds__(kThreads, Cfg<T, D, G>::CTAS) decode_kernel(const DecodeArgs a) {

@@ -54,8 +54,6 @@ __device__ __forceinline__ bool next_segment(int &cur, int r1, const int *pref, 
     return true;
 }
 
-__device__ __forceinline__ void let_successor_start() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
-__device__ __forceinline__ void wait_for_predecessor() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 
 __device__ __forceinline__ void tma_box_load(void *dst_smem, const CUtensorMap *map, int x, int y, uint64_t *bar) {
     asm volatile(

@@ -20,6 +20,7 @@ __global__ void __launch_bounds__(kRouteWarps * 32)
 route_kernel(const char *__restrict__ hidden, const char *__restrict__ w, int n_steps, int hidden_dim, float b,
              float tau, float *__restrict__ scores, uint8_t *__restrict__ decisions) {
     constexpr int EPL = Elt<T>::kPerVec;
+    pdl_enter();
     const int lane = threadIdx.x & 31;
     const int step = blockIdx.x * kRouteWarps + (threadIdx.x >> 5);
     if (step >= n_steps) return;
@@ -64,6 +65,7 @@ route_kernel(const char *__restrict__ hidden, const char *__restrict__ w, int n_
 
 __global__ void rollback_kernel(int batch, int32_t *__restrict__ seq_lens, const int32_t *__restrict__ step_lens,
                                 const uint8_t *__restrict__ decisions, uint32_t *status) {
+    pdl_enter();
     const int i = blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= batch) return;
     if (decisions != nullptr && decisions[i] == 0) return;
@@ -83,6 +85,7 @@ __global__ void rollback_kernel(int batch, int32_t *__restrict__ seq_lens, const
 // Lengths of the next call of a phase of the step loop (see arb_phase_lens): one thread per sequence.
 __global__ void phase_lens_kernel(int batch, const int32_t *__restrict__ step_lens, const uint8_t *__restrict__ decisions,
                                   int want, int t, int32_t *__restrict__ out) {
+    pdl_enter();
     const int b = blockIdx.x * blockDim.x + threadIdx.x;
     if (b >= batch) return;
     const int n = max(step_lens[b], 0);
@@ -94,6 +97,7 @@ __global__ void phase_lens_kernel(int batch, const int32_t *__restrict__ step_le
 __global__ void phase_lens_tokens_kernel(int batch, const int32_t *__restrict__ step_lens,
                                          const uint8_t *__restrict__ decisions, int want, int n_tokens,
                                          int32_t *__restrict__ out) {
+    pdl_enter();
     const int i = blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= batch * n_tokens) return;
     const int t = i / batch, b = i - t * batch;
@@ -106,41 +110,44 @@ __global__ void phase_lens_tokens_kernel(int batch, const int32_t *__restrict__ 
 arb_status launch_phase_lens_tokens(Ctx *ctx, int batch, const int32_t *step_lens, const uint8_t *decisions, int want,
                                     int n_tokens, int32_t *out, cudaStream_t stream) {
     const long long n = (long long)batch * n_tokens;
-    phase_lens_tokens_kernel<<<(unsigned)((n + 255) / 256), 256, 0, stream>>>(batch, step_lens, decisions, want, n_tokens,
-                                                                             out);
+    const cudaError_t err = launch_pdl(phase_lens_tokens_kernel, dim3((unsigned)((n + 255) / 256)), dim3(256), 0, stream,
+                                       batch, step_lens, decisions, want, n_tokens, out);
     ctx->launches++;
-    return cudaGetLastError() == cudaSuccess ? ARB_OK : ARB_ERR_CUDA;
+    return err == cudaSuccess ? ARB_OK : ARB_ERR_CUDA;
 }
 
 arb_status launch_phase_lens(Ctx *ctx, int batch, const int32_t *step_lens, const uint8_t *decisions, int want, int t,
                              int32_t *out, cudaStream_t stream) {
-    phase_lens_kernel<<<(batch + 127) / 128, 128, 0, stream>>>(batch, step_lens, decisions, want, t, out);
+    const cudaError_t err = launch_pdl(phase_lens_kernel, dim3((batch + 127) / 128), dim3(128), 0, stream, batch,
+                                       step_lens, decisions, want, t, out);
     ctx->launches++;
-    return cudaGetLastError() == cudaSuccess ? ARB_OK : ARB_ERR_CUDA;
+    return err == cudaSuccess ? ARB_OK : ARB_ERR_CUDA;
 }
 
 arb_status launch_route(Ctx *ctx, int dtype, int n_steps, int hidden_dim, const void *hidden, const void *w,
                         float b, float tau, float *scores, uint8_t *decisions, cudaStream_t stream) {
     const int grid = (n_steps + kRouteWarps - 1) / kRouteWarps;
+    cudaError_t err;
     if (dtype == ARB_BF16)
-        route_kernel<__nv_bfloat16><<<grid, kRouteWarps * 32, 0, stream>>>(
-            static_cast<const char *>(hidden), static_cast<const char *>(w), n_steps, hidden_dim, b, tau, scores,
-            decisions);
+        err = launch_pdl(route_kernel<__nv_bfloat16>, dim3(grid), dim3(kRouteWarps * 32), 0, stream,
+                         static_cast<const char *>(hidden), static_cast<const char *>(w), n_steps, hidden_dim, b, tau,
+                         scores, decisions);
     else if (dtype == ARB_F32)
-        route_kernel<float><<<grid, kRouteWarps * 32, 0, stream>>>(static_cast<const char *>(hidden),
-                                                                   static_cast<const char *>(w), n_steps,
-                                                                   hidden_dim, b, tau, scores, decisions);
+        err = launch_pdl(route_kernel<float>, dim3(grid), dim3(kRouteWarps * 32), 0, stream,
+                         static_cast<const char *>(hidden), static_cast<const char *>(w), n_steps, hidden_dim, b, tau,
+                         scores, decisions);
     else
         return ARB_ERR_UNSUPPORTED;
     ctx->launches++;
-    return cudaGetLastError() == cudaSuccess ? ARB_OK : ARB_ERR_CUDA;
+    return err == cudaSuccess ? ARB_OK : ARB_ERR_CUDA;
 }
 
 arb_status launch_rollback(Ctx *ctx, int batch, int32_t *seq_lens, const int32_t *step_lens,
                            const uint8_t *decisions, cudaStream_t stream) {
-    rollback_kernel<<<(batch + 127) / 128, 128, 0, stream>>>(batch, seq_lens, step_lens, decisions, ctx->status);
+    const cudaError_t err = launch_pdl(rollback_kernel, dim3((batch + 127) / 128), dim3(128), 0, stream, batch, seq_lens,
+                                       step_lens, decisions, ctx->status);
     ctx->launches++;
-    return cudaGetLastError() == cudaSuccess ? ARB_OK : ARB_ERR_CUDA;
+    return err == cudaSuccess ? ARB_OK : ARB_ERR_CUDA;
 }
 
 }  // namespace arb

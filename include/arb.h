@@ -391,6 +391,20 @@ arb_status arb_attn_decode_e4m3(arb_ctx *ctx, const arb_attn_params *params, con
                                 const int32_t *seq_lens, const int32_t *q_lens, void *out, arb_stream_t stream);
 
 /*
+ * arb_attn over an E4M3 KV cache, decode rows and step chunks alike (q_lens 0, 1 or a step length): what a
+ * quantised draft's cache needs for all of Algorithm 1 -- its own token-by-token steps, and the causal chunk by
+ * which it absorbs the target's step after an escalation (Section 5.1 for the quantised-draft regime; the cache
+ * format is this library's choice).  Arguments as for arb_attn_decode_e4m3, params->max_q_len = the largest
+ * q_len.  Decode rows run on that call's kernel; chunks on the tcgen05 kernel of arb_attn with the codes widened
+ * to f16 on their way into its operand tiles (exact), q converted bf16 -> f16 (|q| must stay below the f16
+ * range, 65504) and the softmax weights rounded to f16.  batch <= 512 when chunks are present.  Against an oracle
+ * that reads the same codes the result meets the tolerance of the bf16 tensor-core paths.
+ */
+arb_status arb_attn_e4m3(arb_ctx *ctx, const arb_attn_params *params, const void *q, const uint8_t *k_codes,
+                         const uint8_t *v_codes, float k_scale, float v_scale, const int32_t *block_table,
+                         const int32_t *seq_lens, const int32_t *q_lens, void *out, arb_stream_t stream);
+
+/*
  * Quantising KV append: as arb_kv_append, but the pools hold E4M3 codes, one byte per element (1 sign bit,
  * 4 exponent bits with bias 7, 3 mantissa bits, no infinities, largest finite value 448) -- the
  * reduced-precision cache of a quantised draft model (Section 5.1 of the paper runs 4-bit and 3-bit drafts;

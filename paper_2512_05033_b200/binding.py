@@ -34,7 +34,7 @@ MAX_CLASSES = 16
 EXPORTS = ("arb_create", "arb_destroy", "arb_attn_workspace_bytes", "arb_attn", "arb_attn_host",
            "arb_attn_host_begin", "arb_attn_host_wait",
            "arb_attn_decode_static", "arb_decode_step",
-           "arb_route", "arb_rollback", "arb_policy", "arb_route_classes", "arb_kv_append", "arb_kv_append_e4m3", "arb_attn_decode_e4m3", "arb_phase_lens", "arb_phase_lens_tokens", "arb_spearman",
+           "arb_route", "arb_rollback", "arb_policy", "arb_route_classes", "arb_kv_append", "arb_kv_append_e4m3", "arb_attn_decode_e4m3", "arb_attn_e4m3", "arb_phase_lens", "arb_phase_lens_tokens", "arb_spearman",
            "arb_selftest_wait_timeout", "arb_poll_status", "arb_launch_count", "arb_status_string")
 
 
@@ -71,6 +71,8 @@ lib.arb_rollback.restype = ctypes.c_int
 lib.arb_rollback.argtypes = [_vp, _i32, _vp, _vp, _vp, _vp]
 lib.arb_attn_decode_e4m3.restype = ctypes.c_int
 lib.arb_attn_decode_e4m3.argtypes = [_vp, ctypes.POINTER(AttnParams), _vp, _vp, _vp, _f, _f, _vp, _vp, _vp, _vp, _vp]
+lib.arb_attn_e4m3.restype = ctypes.c_int
+lib.arb_attn_e4m3.argtypes = [_vp, ctypes.POINTER(AttnParams), _vp, _vp, _vp, _f, _f, _vp, _vp, _vp, _vp, _vp]
 lib.arb_kv_append_e4m3.restype = ctypes.c_int
 lib.arb_kv_append_e4m3.argtypes = [_vp, ctypes.POINTER(AttnParams), _i32, _vp, _vp, _f, _f, _vp, _vp, _vp, _i32, _vp, _vp, _vp]
 lib.arb_spearman.restype = ctypes.c_int
@@ -302,6 +304,21 @@ class Context:
                                       _dev(seq_lens, "seq_lens", torch.int32), _dev(q_lens, "q_lens", torch.int32),
                                       _dev(out, "out", torch.bfloat16), _stream_ptr(stream))
         _check(st, "arb_attn_decode_e4m3")
+        return out
+
+    # -- arb_attn_e4m3 ------------------------------------------------------------------------
+    def attn_e4m3(self, q, k_codes, v_codes, k_scale: float, v_scale: float, block_table, seq_lens, q_lens,
+                  max_q_len: int, out=None, softmax_scale: float = 0.0, stream=None, params=None):
+        """Attention (decode rows and step chunks) over an E4M3 cache; q and out bf16.  Asynchronous."""
+        if out is None:
+            out = torch.empty_like(q)
+        p = params or self.params_for(q, k_codes, block_table, max_q_len, softmax_scale)
+        st = lib.arb_attn_e4m3(self._h, ctypes.byref(p), _dev(q, "q", torch.bfloat16),
+                               _dev(k_codes, "k_codes", torch.uint8), _dev(v_codes, "v_codes", torch.uint8),
+                               float(k_scale), float(v_scale), _dev(block_table, "block_table", torch.int32),
+                               _dev(seq_lens, "seq_lens", torch.int32), _dev(q_lens, "q_lens", torch.int32),
+                               _dev(out, "out", torch.bfloat16), _stream_ptr(stream))
+        _check(st, "arb_attn_e4m3")
         return out
 
     # -- arb_kv_append_e4m3 -------------------------------------------------------------------

@@ -115,6 +115,7 @@ arb_status arb_create(arb_ctx **out, int device, size_t workspace_bytes) {
     }
     c->num_sms = sms;
     // tuning knob of the single-launch decode (see Plan in arb_decode_step.cu)
+    if (const char *mc = std::getenv("ARB_STEP_MIN_CHUNK")) c->step_min_chunk = std::max(1, std::min(1024, std::atoi(mc)));
     if (const char *pct = std::getenv("ARB_STEP_BOUNDARY_PCT")) c->step_boundary_pct = std::max(0, std::min(400, std::atoi(pct)));
     c->workspace_bytes = workspace_bytes ? workspace_bytes : kDefaultWorkspace;
     c->counters_len = kCounters;
@@ -568,6 +569,40 @@ arb_status arb_attn_decode_e4m3(arb_ctx *ctx, const arb_attn_params *params, con
     if (decode_workspace_bytes(*params, c->num_sms) > c->workspace_bytes) return ARB_ERR_WORKSPACE;
     return launch_decode_e4m3(c, *params, q, k_codes, v_codes, k_scale, v_scale, block_table, seq_lens, q_lens, out,
                               reinterpret_cast<cudaStream_t>(stream));
+}
+
+arb_status arb_attn_e4m3(arb_ctx *ctx, const arb_attn_params *params, const void *q, const uint8_t *k_codes,
+                         const uint8_t *v_codes, float k_scale, float v_scale, const int32_t *block_table,
+                         const int32_t *seq_lens, const int32_t *q_lens, void *out, arb_stream_t stream) {
+    if (ctx == nullptr) return ARB_ERR_INVALID_ARG;
+    arb_status st = check_params(params);
+    if (st != ARB_OK) return st;
+    if (params->dtype != ARB_BF16 || params->head_dim != 128) return ARB_ERR_UNSUPPORTED;
+    if (params->flags & ARB_ATTN_NO_TENSOR_CORES) return ARB_ERR_UNSUPPORTED;
+    if (!(k_scale > 0.f) || !(v_scale > 0.f)) return ARB_ERR_INVALID_ARG;
+    if (!k_codes || !v_codes || !block_table || !seq_lens || !q_lens) return ARB_ERR_INVALID_ARG;
+    if (params->total_q == 0 || params->max_q_len == 0) return ARB_OK;
+    if (!q || !out) return ARB_ERR_INVALID_ARG;
+    if (!aligned16(q) || !aligned16(out) || !aligned16(k_codes) || !aligned16(v_codes)) return ARB_ERR_INVALID_ARG;
+    if (params->max_q_len > params->total_q) return ARB_ERR_INVALID_ARG;
+    Ctx *c = reinterpret_cast<Ctx *>(ctx);
+    if (decode_workspace_bytes(*params, c->num_sms) > c->workspace_bytes) return ARB_ERR_WORKSPACE;
+    cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+    const bool maybe_decode = params->max_q_len == 1 || params->total_q > params->max_q_len;
+    if (maybe_decode) {
+        st = launch_decode_e4m3(c, *params, q, k_codes, v_codes, k_scale, v_scale, block_table, seq_lens, q_lens, out, s);
+        if (st != ARB_OK) return st;
+    }
+    if (params->max_q_len >= 2) {
+        st = launch_chunk_e4m3(c, *params, q, k_codes, v_codes, k_scale, v_scale, block_table, seq_lens, q_lens, out, s);
+        if (st != ARB_OK) return st;
+        // the CUDA-core chunk kernel reads no key here: every chunk of valid lengths has gone to the tensor cores; it
+        // zero-fills the rows of sequences whose lengths are not (status bit) and otherwise leaves at once
+        st = launch_chunk_fma(c, *params, q, k_codes, v_codes, block_table, seq_lens, q_lens, out, 2, params->max_q_len,
+                              kChunkMmaMinRows, s);
+        if (st != ARB_OK) return st;
+    }
+    return ARB_OK;
 }
 
 arb_status arb_kv_append_e4m3(arb_ctx *ctx, const arb_attn_params *params, int32_t total_new, const void *k_new,

@@ -26,6 +26,15 @@
 // handed out dynamically, longest sequences first: the K producer takes the next item from an atomic
 // counter and announces it to the other roles through a small queue in shared memory.  Every mbarrier wait
 // is bounded; TMEM is released on every path.
+//
+// The same kernel, compiled a second time (template parameter E4M3), reads an E4M3 KV cache (one byte per element;
+// keys are k_scale * code, values v_scale * code): the chunk a quantised draft's cache absorbs when the target's
+// step replaces its own (Algorithm 1, escalation branch).  The codes widen to f16 exactly, so the products run as
+// f16 MMAs with fp32 accumulation; q is converted bf16 -> f16 as its tile is written, P is rounded to f16.  A page
+// of codes (16 rows x 128 bytes) arrives through one tiled TMA copy in a small staging ring of four pages per
+// operand; the producer warp of the operand widens it (cvt.rn.f16x2.e4m3x2) into the operand stage, in the
+// 128-byte-swizzled layout the bf16 tiles land in, and asks for the page four ahead.  The key scale folds into the
+// softmax scale, the value scale into the epilogue.
 #include "arb_tma.cuh"
 
 namespace arb {
@@ -44,6 +53,8 @@ constexpr int kTmaWarp = 8, kMmaWarp = 9, kVWarp = 10;   // warp 11 has no role
 constexpr int kHalfBytes = 128 * 128;      // [128 rows x 64 bf16]: one 128-byte-swizzled half tile
 constexpr int kTileBytes = 2 * kHalfBytes;  // [128 x 128] bf16
 constexpr int kBoxBytes = kPage * 128;      // one TMA box: 16 rows x 64 bf16
+constexpr int kStagePages = 4;              // E4M3: pages of codes in flight per operand
+constexpr int kCodePageBytes = kPage * kD;  // 2 KB: one (page, kv head) tile of codes
 constexpr uint32_t kTmemCols = 512;         // S of tile A: columns 0..127, S of B: 128..255, O of A: 256..383, O of B: 384..511
 constexpr uint32_t kOCol = 256;
 constexpr float kRescaleThreshold = 8.0f;   // log2 units
@@ -81,7 +92,8 @@ struct MmaArgs {
     int split_cap;      // slots that fit there
     int fill_ctas;      // CTAs a call should keep busy: a call with fewer than half as many work items has its
                         // sequences cut over their keys as well (0: never)
-    float scale_log2;
+    float scale_log2;   // softmax scale (times the key scale of an E4M3 cache) * log2(e)
+    float v_scale;      // value scale of an E4M3 cache, 1 otherwise
 };
 
 struct Bars {
@@ -95,6 +107,7 @@ struct Bars {
     uint64_t o_full[2];          // O += P V of row tile A / B has completed
     uint64_t item_full[kItemSlots];   // the producer warp has fetched the next work item
     uint64_t item_empty[kItemSlots];  // the MMA thread, the V producer and the softmax threads have read it
+    uint64_t code_full[2][kStagePages];   // E4M3: a page of codes of K / of V has landed in its staging slot
     int item_id[kItemSlots];
     uint32_t tmem_base;
     int abort;
@@ -103,7 +116,12 @@ struct Bars {
 constexpr size_t kSmemFixed = 1024 /*alignment*/ + 2 * kTileBytes /*Q of A, B*/ + 2 * kStages * kTileBytes /*K, V*/ +
                               sizeof(Bars);
 
-inline size_t mma_smem_bytes(int batch) { return kSmemFixed + sizeof(int) * (7 * (size_t)batch + 2); }
+constexpr size_t kCodeStageBytes = 2 * kStagePages * kCodePageBytes;   // E4M3: staging of both operands
+constexpr int kMaxBatchE4m3 = 512;   // the staging takes 16 KB of what the plan tables of a larger batch would need
+
+inline size_t mma_smem_bytes(int batch, bool e4m3 = false) {
+    return kSmemFixed + (e4m3 ? kCodeStageBytes : 0) + sizeof(int) * (7 * (size_t)batch + 2);
+}
 
 // ---- tcgen05 / TMA wrappers -------------------------------------------------------------------
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
@@ -159,10 +177,10 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t saddr, uint32_t lbo_bytes
     return d;
 }
 
-// Instruction descriptor of kind::f16: fp32 accumulator, bf16 A and B, M = 128, N = 128.
-__host__ __device__ constexpr uint32_t instr_desc(bool b_mn_major) {
+// Instruction descriptor of kind::f16: fp32 accumulator, A and B both bf16 or both f16, M = 128, N = 128.
+__host__ __device__ constexpr uint32_t instr_desc(bool b_mn_major, bool f16 = false) {
     return (1u << 4)                       // accumulator format: f32
-           | (1u << 7) | (1u << 10)        // A, B format: bf16
+           | ((f16 ? 0u : 1u) << 7) | ((f16 ? 0u : 1u) << 10)   // A, B format: f16 = 0, bf16 = 1
            | (0u << 15)                    // A is K-major
            | ((b_mn_major ? 1u : 0u) << 16)
            | ((uint32_t)(kBN >> 3) << 17)  // N
@@ -217,6 +235,22 @@ __device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
     uint32_t r;
     asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+    return r;
+}
+
+__device__ __forceinline__ uint32_t pack_f16(float lo, float hi) {
+    uint32_t r;
+    asm("cvt.rn.f16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+    return r;
+}
+// two bf16 (one 32-bit word) -> two f16
+__device__ __forceinline__ uint32_t bf16x2_to_f16x2(uint32_t v) {
+    return pack_f16(__uint_as_float(v << 16), __uint_as_float(v & 0xffff0000u));
+}
+// two E4M3 codes (a 16-bit pair) -> f16x2, exact; the low byte lands in the low half
+__device__ __forceinline__ uint32_t e4m3x2_to_f16x2(uint16_t v) {
+    uint32_t r;
+    asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(r) : "h"(v));
     return r;
 }
 
@@ -414,7 +448,7 @@ __device__ __forceinline__ bool get_item(int item, int total, const Plan &pl, in
     return true;
 }
 
-template <int G>
+template <int G, bool E4M3>
 __global__ void __launch_bounds__(kThreads, 1)
 chunk_mma_kernel(const MmaArgs a, const __grid_constant__ CUtensorMap k_map, const __grid_constant__ CUtensorMap v_map) {
     extern __shared__ char smem_raw[];
@@ -422,7 +456,8 @@ chunk_mma_kernel(const MmaArgs a, const __grid_constant__ CUtensorMap k_map, con
     char *q_s = base;                                  // [row tile A, B][2 halves][128 rows][128 B]
     char *k_s = base + 2 * kTileBytes;                 // [stage][2 halves][128 keys][128 B]
     char *v_s = k_s + kStages * kTileBytes;
-    Bars *bars = reinterpret_cast<Bars *>(v_s + kStages * kTileBytes);
+    char *code_s = v_s + kStages * kTileBytes;         // E4M3: [K, V][kStagePages][16 rows][128 B of codes]
+    Bars *bars = reinterpret_cast<Bars *>(code_s + (E4M3 ? kCodeStageBytes : 0));
     const Plan pl = plan_arrays(reinterpret_cast<int *>(bars + 1), a.batch);
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -446,6 +481,10 @@ chunk_mma_kernel(const MmaArgs a, const __grid_constant__ CUtensorMap k_map, con
         for (int i = 0; i < kItemSlots; ++i) {
             mbar_init(&bars->item_full[i], 1);
             mbar_init(&bars->item_empty[i], 2 + 2 * kSoftmaxThreads);   // MMA thread, V warp, softmax threads
+        }
+        for (int i = 0; i < kStagePages; ++i) {
+            mbar_init(&bars->code_full[0][i], 1);
+            mbar_init(&bars->code_full[1][i], 1);
         }
         bars->abort = 0;
         mbar_fence_init();
@@ -476,6 +515,7 @@ chunk_mma_kernel(const MmaArgs a, const __grid_constant__ CUtensorMap k_map, con
         const CUtensorMap *map = is_v ? &v_map : &k_map;
         const char *pool = is_v ? a.v_pool : a.k_pool;
         uint32_t it = 0;  // KV tiles issued so far
+        uint32_t pc = 0;  // E4M3: pages of codes asked for so far (staging slot and phase)
         Item w;
         for (uint32_t nq = 0;; ++nq) {
             const uint32_t slot = nq % kItemSlots, qpar = (nq / kItemSlots) & 1u;
@@ -505,8 +545,9 @@ chunk_mma_kernel(const MmaArgs a, const __grid_constant__ CUtensorMap k_map, con
             // ring (two tiles deep) only has to cover the L2 latency, not the DRAM latency
             auto prefetch_pages = [&](int pf) {
                 if ((unsigned)pf < (unsigned)a.num_pages) {
-                    const char *src = pool + ((size_t)pf * Hkv + w.kvh) * (kPage * kD * 2);
-                    asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(src), "r"(kPage * kD * 2) : "memory");
+                    constexpr int kPageBytes = kPage * kD * (E4M3 ? 1 : 2);
+                    const char *src = pool + ((size_t)pf * Hkv + w.kvh) * kPageBytes;
+                    asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(src), "r"(kPageBytes) : "memory");
                 }
             };
             for (int jt = 0; jt < kPrefetchTiles; ++jt) prefetch_pages(table_entry(jt));
@@ -529,13 +570,69 @@ chunk_mma_kernel(const MmaArgs a, const __grid_constant__ CUtensorMap k_map, con
                 const int pg = lane & 7, half = (lane >> 3) & 1;
                 const int row = (__shfl_sync(0xffffffffu, pid, pg) * Hkv + w.kvh) * kPage;
                 bool ok = true;
-                if (lane == 0) ok = mbar_wait(&empty[s], par ^ 1u, abort, a.status);
-                ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
-                if (ok) {
-                    if (lane == 0) mbar_arrive_expect_tx(&full[s], (uint32_t)npages * 2u * kBoxBytes);
-                    __syncwarp();
-                    if (lane < 16 && pg < npages)
-                        tma_box_load(ring + s * kTileBytes + half * kHalfBytes + pg * kBoxBytes, map, half * 64, row, &full[s]);
+                if constexpr (E4M3) {
+                    // Pages of codes go through the staging slots: wait for a page, widen it into the operand stage,
+                    // ask for the page kStagePages ahead (of this tile or of the next).  Lane (r, h) = (lane / 2,
+                    // lane % 2) widens the 64 codes of half h of row r: four 16-byte pieces in, eight out.
+                    char *stg = code_s + (is_v ? kStagePages * kCodePageBytes : 0);
+                    uint64_t *cfull = bars->code_full[is_v ? 1 : 0];
+                    // (an entry of the next tile that lies outside the pool is reported when that tile is the current one)
+                    const int pid_ahead = __shfl_sync(0xffffffffu, pid_next, pg);
+                    const int row_next = (((unsigned)pid_ahead < (unsigned)a.num_pages ? pid_ahead : 0) * Hkv + w.kvh) * kPage;
+                    const int left = min(kTilePages, (w.kv_len - (jg + 1) * kBN + kPage - 1) / kPage);   // pages of the next tile
+                    const int np_next = (j + 1 < w.ntiles) ? max(left, 0) : 0;
+                    auto ask = [&](int p_in_tile, uint32_t at) {   // lane 0: page p of this tile (or p - 8 of the next)
+                        const int rr = p_in_tile < kTilePages ? __shfl_sync(0xffffffffu, row, p_in_tile & 7)
+                                                              : __shfl_sync(0xffffffffu, row_next, p_in_tile & 7);
+                        if (lane == 0) {
+                            const uint32_t sl = at % kStagePages;
+                            mbar_arrive_expect_tx(&cfull[sl], kCodePageBytes);
+                            tma_box_load(stg + sl * kCodePageBytes, map, 0, rr, &cfull[sl]);
+                        }
+                    };
+                    if (j == 0) {   // a new item: nothing of it is in flight yet
+                        for (int p = 0; p < kStagePages; ++p) {
+                            const bool there = p < npages || (p >= kTilePages && p - kTilePages < np_next);
+                            if (__shfl_sync(0xffffffffu, there ? 1 : 0, 0)) ask(p, pc + p);
+                        }
+                    }
+                    if (lane == 0) ok = mbar_wait(&empty[s], par ^ 1u, abort, a.status);
+                    ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+                    const int r = lane >> 1, h = lane & 1;
+                    for (int p = 0; p < npages; ++p, ++pc) {
+                        const uint32_t sl = pc % kStagePages, ph = (pc / kStagePages) & 1u;
+                        mbar_wait(&cfull[sl], ph, abort, a.status);
+                        const char *src = stg + sl * kCodePageBytes + r * 128;
+                        char *dst = ring + s * kTileBytes + h * kHalfBytes + (p * kPage + r) * 128;
+                        if (ok) {
+#pragma unroll
+                            for (int c4 = 0; c4 < 4; ++c4) {
+                                const uint4 cd = *reinterpret_cast<const uint4 *>(src + (((4 * h + c4) ^ (r & 7)) << 4));
+                                uint4 lo, hi;
+                                lo.x = e4m3x2_to_f16x2((uint16_t)cd.x); lo.y = e4m3x2_to_f16x2((uint16_t)(cd.x >> 16));
+                                lo.z = e4m3x2_to_f16x2((uint16_t)cd.y); lo.w = e4m3x2_to_f16x2((uint16_t)(cd.y >> 16));
+                                hi.x = e4m3x2_to_f16x2((uint16_t)cd.z); hi.y = e4m3x2_to_f16x2((uint16_t)(cd.z >> 16));
+                                hi.z = e4m3x2_to_f16x2((uint16_t)cd.w); hi.w = e4m3x2_to_f16x2((uint16_t)(cd.w >> 16));
+                                *reinterpret_cast<uint4 *>(dst + (((2 * c4) ^ (r & 7)) << 4)) = lo;
+                                *reinterpret_cast<uint4 *>(dst + (((2 * c4 + 1) ^ (r & 7)) << 4)) = hi;
+                            }
+                        }
+                        fence_async_smem();   // the slot's next writer is the TMA unit; the stage's reader the tensor core
+                        __syncwarp();
+                        const int ahead = p + kStagePages;   // the page that takes this slot
+                        const bool there = ahead < npages || (ahead >= kTilePages && ahead - kTilePages < np_next);
+                        if (there) ask(ahead, pc + kStagePages);
+                    }
+                    if (lane == 0) mbar_arrive(&full[s]);
+                } else {
+                    if (lane == 0) ok = mbar_wait(&empty[s], par ^ 1u, abort, a.status);
+                    ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+                    if (ok) {
+                        if (lane == 0) mbar_arrive_expect_tx(&full[s], (uint32_t)npages * 2u * kBoxBytes);
+                        __syncwarp();
+                        if (lane < 16 && pg < npages)
+                            tma_box_load(ring + s * kTileBytes + half * kHalfBytes + pg * kBoxBytes, map, half * 64, row, &full[s]);
+                    }
                 }
                 __syncwarp();
             }
@@ -547,7 +644,7 @@ chunk_mma_kernel(const MmaArgs a, const __grid_constant__ CUtensorMap k_map, con
         // that row tile's P V, so the tensor core works for one row tile while the other one's
         // softmax group is busy.
         if (lane == 0) {
-            constexpr uint32_t idesc_qk = instr_desc(false), idesc_pv = instr_desc(true);
+            constexpr uint32_t idesc_qk = instr_desc(false, E4M3), idesc_pv = instr_desc(true, E4M3);
             const uint32_t q_addr = smem_u32(q_s);
             uint32_t it = 0, nitem = 0, nproc = 0, itg[2] = {0u, 0u};  // KV tiles so far: all, per row tile
             Item w;
@@ -642,7 +739,11 @@ chunk_mma_kernel(const MmaArgs a, const __grid_constant__ CUtensorMap k_map, con
                 const uint4 *src = reinterpret_cast<const uint4 *>(a.q + grow * 2);
 #pragma unroll
                 for (int c = 0; c < 16; ++c) {
-                    const uint4 v = row_ok ? __ldg(src + c) : make_uint4(0, 0, 0, 0);
+                    uint4 v = row_ok ? __ldg(src + c) : make_uint4(0, 0, 0, 0);
+                    if constexpr (E4M3) {   // the operands of one MMA share a type: q goes to f16 like the widened codes
+                        v.x = bf16x2_to_f16x2(v.x); v.y = bf16x2_to_f16x2(v.y);
+                        v.z = bf16x2_to_f16x2(v.z); v.w = bf16x2_to_f16x2(v.w);
+                    }
                     *reinterpret_cast<uint4 *>(q_tile + (c >> 3) * kHalfBytes + tg * 128 + (((c & 7) ^ swz) << 4)) = v;
                 }
                 fence_async_smem();
@@ -721,7 +822,7 @@ chunk_mma_kernel(const MmaArgs a, const __grid_constant__ CUtensorMap k_map, con
                         float t0, t1;
                         unpack_f32x2(t, t0, t1);
                         const float e0 = fast_exp2(t0), e1 = fast_exp2(t1);
-                        pk[k] = pack_bf16(e0, e1);
+                        pk[k] = E4M3 ? pack_f16(e0, e1) : pack_bf16(e0, e1);
                         l2[k & 3] = add_f32x2(l2[k & 3], pack_f32x2(e0, e1));
                     }
                     tmem_st16(s_tmem + c4 * 16, pk);
@@ -763,6 +864,10 @@ chunk_mma_kernel(const MmaArgs a, const __grid_constant__ CUtensorMap k_map, con
                     tmem_ld32(o_tmem + c4 * 32, v);
                     tmem_wait_ld();
                     if (row_ok) {
+                        if constexpr (E4M3) {   // values of an E4M3 cache are v_scale * code
+#pragma unroll
+                            for (int k = 0; k < 32; ++k) v[k] = __float_as_uint(__uint_as_float(v[k]) * a.v_scale);
+                        }
 #pragma unroll
                         for (int qd = 0; qd < 8; ++qd)
                             *reinterpret_cast<uint4 *>(po + ((size_t)(c4 * 8 + qd) * kBM + tg) * 4) =
@@ -773,7 +878,7 @@ chunk_mma_kernel(const MmaArgs a, const __grid_constant__ CUtensorMap k_map, con
                 tc_fence_before();
                 continue;
             }
-            const float inv_l = 1.0f / l_sum;
+            const float inv_l = (E4M3 ? a.v_scale : 1.0f) / l_sum;
             uint4 *dst = reinterpret_cast<uint4 *>(a.out + grow * 2);
 #pragma unroll 1
             for (int c4 = 0; c4 < 4; ++c4) {
@@ -887,19 +992,19 @@ chunk_combine_kernel(const MmaArgs a) {
     }
 }
 
-template <int G>
+template <int G, bool E4M3>
 arb_status launch_one(Ctx *ctx, const MmaArgs &a, const CUtensorMap &km, const CUtensorMap &vm, int max_items,
                       cudaStream_t stream) {
-    const size_t smem = mma_smem_bytes(a.batch);
+    const size_t smem = mma_smem_bytes(a.batch, E4M3);
     static bool attr_set[64] = {};
     if (!attr_set[ctx->device & 63]) {
-        if (cudaFuncSetAttribute(chunk_mma_kernel<G>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 (int)mma_smem_bytes(kMaxBatch)) != cudaSuccess)
+        if (cudaFuncSetAttribute(chunk_mma_kernel<G, E4M3>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 (int)mma_smem_bytes(E4M3 ? kMaxBatchE4m3 : kMaxBatch, E4M3)) != cudaSuccess)
             return ARB_ERR_CUDA;
         attr_set[ctx->device & 63] = true;
     }
     const int grid = max_items < ctx->num_sms ? max_items : ctx->num_sms;
-    const cudaError_t err = launch_pdl(chunk_mma_kernel<G>, dim3(grid), dim3(kThreads), smem, stream, a, km, vm);
+    const cudaError_t err = launch_pdl(chunk_mma_kernel<G, E4M3>, dim3(grid), dim3(kThreads), smem, stream, a, km, vm);
     ctx->launches++;
     if (err != cudaSuccess) return ARB_ERR_CUDA;
     // the merge of split sequences, when the block table is long enough for a sequence to be split at all
@@ -920,12 +1025,15 @@ bool chunk_mma_supported(const arb_attn_params &p) {
            tma_available();
 }
 
-arb_status launch_chunk_mma(Ctx *ctx, const arb_attn_params &p, const void *q, const void *k_pages,
-                            const void *v_pages, const int32_t *block_table, const int32_t *seq_lens,
-                            const int32_t *q_lens, void *out, cudaStream_t stream) {
+namespace {
+
+arb_status launch_chunk_tc(Ctx *ctx, const arb_attn_params &p, const void *q, const void *k_pages, const void *v_pages,
+                           bool e4m3, float k_scale, float v_scale, const int32_t *block_table, const int32_t *seq_lens,
+                           const int32_t *q_lens, void *out, cudaStream_t stream) {
     alignas(64) CUtensorMap km, vm;
-    if (!pool_map(ctx, &km, k_pages, p.num_pages, p.num_kv_heads, PoolView::kBf16HalfRows) ||
-        !pool_map(ctx, &vm, v_pages, p.num_pages, p.num_kv_heads, PoolView::kBf16HalfRows))
+    const PoolView view = e4m3 ? PoolView::kE4m3 : PoolView::kBf16HalfRows;
+    if (!pool_map(ctx, &km, k_pages, p.num_pages, p.num_kv_heads, view) ||
+        !pool_map(ctx, &vm, v_pages, p.num_pages, p.num_kv_heads, view))
         return ARB_ERR_CUDA;
     MmaArgs a;
     a.q = static_cast<const char *>(q);
@@ -954,23 +1062,48 @@ arb_status launch_chunk_mma(Ctx *ctx, const arb_attn_params &p, const void *q, c
     if (max_tiles <= kSplitMinTiles && a.fill_ctas == 0) a.split_cap = 0;
     if (cudaMemsetAsync(a.work_counter, 0, 2 * sizeof(int), stream) != cudaSuccess) return ARB_ERR_CUDA;
     const float scale = p.softmax_scale > 0.f ? p.softmax_scale : 1.0f / sqrtf((float)p.head_dim);
-    a.scale_log2 = scale * 1.4426950408889634f;
+    a.scale_log2 = scale * k_scale * 1.4426950408889634f;
+    a.v_scale = v_scale;
     const int g = p.num_q_heads / p.num_kv_heads;
     // upper bound of the work items from what the host knows: every row could sit in its own tile run
     long long bound = (long long)p.num_kv_heads * ((long long)p.total_q * g / kBM + p.batch);
     if (a.split_cap > 0) bound *= kSplitMaxParts;   // every item of a split sequence comes once per part
     const int max_items = (int)(bound < 1 ? 1 : (bound > (1 << 30) ? (1 << 30) : bound));
-    switch (g) {
-        case 1: return launch_one<1>(ctx, a, km, vm, max_items, stream);
-        case 2: return launch_one<2>(ctx, a, km, vm, max_items, stream);
-        case 3: return launch_one<3>(ctx, a, km, vm, max_items, stream);
-        case 4: return launch_one<4>(ctx, a, km, vm, max_items, stream);
-        case 5: return launch_one<5>(ctx, a, km, vm, max_items, stream);
-        case 6: return launch_one<6>(ctx, a, km, vm, max_items, stream);
-        case 7: return launch_one<7>(ctx, a, km, vm, max_items, stream);
-        case 8: return launch_one<8>(ctx, a, km, vm, max_items, stream);
+    switch (e4m3 ? g + 8 : g) {
+        case 1: return launch_one<1, false>(ctx, a, km, vm, max_items, stream);
+        case 2: return launch_one<2, false>(ctx, a, km, vm, max_items, stream);
+        case 3: return launch_one<3, false>(ctx, a, km, vm, max_items, stream);
+        case 4: return launch_one<4, false>(ctx, a, km, vm, max_items, stream);
+        case 5: return launch_one<5, false>(ctx, a, km, vm, max_items, stream);
+        case 6: return launch_one<6, false>(ctx, a, km, vm, max_items, stream);
+        case 7: return launch_one<7, false>(ctx, a, km, vm, max_items, stream);
+        case 8: return launch_one<8, false>(ctx, a, km, vm, max_items, stream);
+        case 9: return launch_one<1, true>(ctx, a, km, vm, max_items, stream);
+        case 10: return launch_one<2, true>(ctx, a, km, vm, max_items, stream);
+        case 11: return launch_one<3, true>(ctx, a, km, vm, max_items, stream);
+        case 12: return launch_one<4, true>(ctx, a, km, vm, max_items, stream);
+        case 13: return launch_one<5, true>(ctx, a, km, vm, max_items, stream);
+        case 14: return launch_one<6, true>(ctx, a, km, vm, max_items, stream);
+        case 15: return launch_one<7, true>(ctx, a, km, vm, max_items, stream);
+        case 16: return launch_one<8, true>(ctx, a, km, vm, max_items, stream);
         default: return ARB_ERR_UNSUPPORTED;
     }
+}
+
+}  // namespace
+
+arb_status launch_chunk_mma(Ctx *ctx, const arb_attn_params &p, const void *q, const void *k_pages,
+                            const void *v_pages, const int32_t *block_table, const int32_t *seq_lens,
+                            const int32_t *q_lens, void *out, cudaStream_t stream) {
+    return launch_chunk_tc(ctx, p, q, k_pages, v_pages, false, 1.0f, 1.0f, block_table, seq_lens, q_lens, out, stream);
+}
+
+// step chunks over an E4M3 cache (q, out bf16): keys are k_scale * code, values v_scale * code
+arb_status launch_chunk_e4m3(Ctx *ctx, const arb_attn_params &p, const void *q, const void *k_codes,
+                             const void *v_codes, float k_scale, float v_scale, const int32_t *block_table,
+                             const int32_t *seq_lens, const int32_t *q_lens, void *out, cudaStream_t stream) {
+    if (p.num_q_heads / p.num_kv_heads > 8 || p.batch > kMaxBatchE4m3 || !tma_available()) return ARB_ERR_UNSUPPORTED;
+    return launch_chunk_tc(ctx, p, q, k_codes, v_codes, true, k_scale, v_scale, block_table, seq_lens, q_lens, out, stream);
 }
 
 }  // namespace arb

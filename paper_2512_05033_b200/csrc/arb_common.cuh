@@ -63,6 +63,7 @@ struct Ctx {
     uint32_t decode_gen = 1000;          // generation of the next tensor-core decode call
     uint32_t rot_wait_through = 0;        // tensor-core decode calls up to this generation wait for their predecessor
     double *spearman_acc = nullptr;       // three fp64 accumulators of arb_spearman
+    int step_min_chunk = 16;              // single-launch decode: fewest pages worth giving a CTA
     int step_boundary_pct = 100;          // single-launch decode: what a (sequence, kv head) boundary inside a CTA's range counts for
     float *chunk_ws = nullptr;            // partial results of split long sequences (step-chunk attention)
     size_t chunk_ws_bytes = 0;
@@ -265,6 +266,9 @@ arb_status launch_decode_mma(Ctx *ctx, const arb_attn_params &p, const void *q, 
 arb_status launch_chunk_mma(Ctx *ctx, const arb_attn_params &p, const void *q, const void *k_pages,
                             const void *v_pages, const int32_t *block_table, const int32_t *seq_lens,
                             const int32_t *q_lens, void *out, cudaStream_t stream);
+arb_status launch_chunk_e4m3(Ctx *ctx, const arb_attn_params &p, const void *q, const void *k_codes,
+                             const void *v_codes, float k_scale, float v_scale, const int32_t *block_table,
+                             const int32_t *seq_lens, const int32_t *q_lens, void *out, cudaStream_t stream);
 arb_status launch_route(Ctx *ctx, int dtype, int n_steps, int hidden_dim, const void *hidden, const void *w,
                         float b, float tau, float *scores, uint8_t *decisions, cudaStream_t stream);
 arb_status launch_rollback(Ctx *ctx, int batch, int32_t *seq_lens, const int32_t *step_lens,

@@ -59,6 +59,7 @@ struct StepArgs {
     uint32_t *status;
     int batch, Hq, Hkv, num_pages, max_pages;
     int whole_rows;    // the tensor maps are 3-D: one copy per page tile instead of one per half
+    int min_chunk;     // fewest pages worth giving a CTA
     int boundary_pct;  // cost of a (sequence, kv head) boundary inside a CTA's range: percent of min(even share, kBoundaryCap) pages
     float scale_log2;
 };
@@ -279,10 +280,10 @@ decode_step_kernel(const StepArgs a, const __grid_constant__ CUtensorMap k_map, 
         Plan pl;
         pl.pref = pref; pl.act = act; pl.slen = slen; pl.B = B; pl.Hkv = Hkv;
         const int total = pref[B], items = act[B] * Hkv, grid = (int)gridDim.x;
-        const int even = max(kMinChunk, fast_div(total + grid - 1, grid));
+        const int even = max(a.min_chunk, fast_div(total + grid - 1, grid));
         pl.pen = items > 1 ? (min(even, kBoundaryCap) * a.boundary_pct + 99) / 100 : 0;
         pl.total_padded = total + pl.pen * items;
-        pl.chunk = max(kMinChunk, fast_div(pl.total_padded + grid - 1, grid));
+        pl.chunk = max(a.min_chunk, fast_div(pl.total_padded + grid - 1, grid));
         int ends[2], seq0 = 0;
 #pragma unroll
         for (int w = 0; w < 2; ++w) {
@@ -828,6 +829,7 @@ arb_status launch_decode_step(Ctx *ctx, const arb_attn_params &p, const void *q,
     a.max_pages = p.max_pages_per_seq;
     a.whole_rows = whole_rows ? 1 : 0;
     a.boundary_pct = ctx->step_boundary_pct;
+    a.min_chunk = ctx->step_min_chunk;
     const float scale = p.softmax_scale > 0.f ? p.softmax_scale : 1.0f / sqrtf((float)p.head_dim);
     a.scale_log2 = scale * 1.4426950408889634f;
     switch (g) {

@@ -567,3 +567,67 @@ def test_e4m3_decode_peaked_and_back_to_back():
         assert torch.equal(o, alone)
     err = np.abs(alone.double().cpu().numpy() - ref)
     assert (err <= 2.0 ** -8 * np.abs(ref) + 3e-3).all(), err.max()
+
+
+E4M3_CHUNK_CASES = [
+    # (B, Hq, Hkv, seq_lens, q_lens)
+    (1, 32, 8, [300], [64]),                                   # g = 4: two full row tiles
+    (2, 28, 4, [600, 2100], [16, 100]),                        # g = 7: a ragged tile and 700 rows
+    (2, 12, 2, [131, 128], [128, 11]),                         # the chunk is almost the whole sequence
+    (4, 32, 8, [5000, 77, 1300, 256], [1, 30, 128, 5]),        # decode rows beside large and small chunks
+    (1, 16, 2, [4099], [19]),                                  # g = 8, key count not a page multiple
+    (3, 12, 2, [2, 17, 300], [2, 3, 2]),                       # smallest chunks; the chunk is the whole sequence
+    (2, 8, 8, [40, 300], [2, 9]),                              # g = 1
+    (3, 12, 2, [5000, 2500, 300], [24, 9, 1]),                 # few work items: cut over the keys to fill the SMs
+    (3, 28, 4, [21000, 900, 40000], [40, 64, 17]),             # long sequences split into parts and merged
+    (5, 12, 2, [100, 1, 300, 1, 47], [3, 0, 1, 0, 20]),        # idle slots
+]
+
+
+@pytest.mark.parametrize("case", E4M3_CHUNK_CASES)
+def test_e4m3_chunk_matches_oracle(case):
+    """arb_attn_e4m3: step chunks (and the decode rows beside them) over an E4M3 cache against the oracle on the
+    same codes; slots past each sequence's end hold NaN codes, which must never reach the arithmetic."""
+    B, Hq, Hkv, sl, ql = case
+    inp = wl.small_attn_case(B, Hq, Hkv, 128, BF, sl, ql, seed=900 + Hq + len(sl))
+    ks, vs = 0.011, 0.017
+    kc = torch.from_numpy(oracle.e4m3_encode(inp.k_pages, 1 / ks))
+    vc = torch.from_numpy(oracle.e4m3_encode(inp.v_pages, 1 / vs))
+    for b in range(B):
+        L = sl[b]
+        if L % 16:
+            page = int(inp.block_table[b, L // 16])
+            kc[page, :, L % 16:, :] = 0x7f
+            vc[page, :, L % 16:, :] = 0x7f
+    c = H.ctx()
+    d = inp.to("cuda")
+    out = torch.full_like(d.q, float("nan"))
+    c.attn_e4m3(d.q, kc.cuda(), vc.cuda(), ks, vs, d.block_table, d.seq_lens, d.q_lens, max(ql), out=out)
+    assert c.poll_status() == 0
+    ref, st = oracle.attn_e4m3(inp.q, kc, vc, ks, vs, inp.block_table, inp.seq_lens, inp.q_lens)
+    assert st == 0
+    H.assert_close(out.double().cpu().numpy(), ref, BF, tight=3e-3)
+
+
+def test_e4m3_chunk_peaked_and_bad_lengths():
+    """Few keys carry the weight (outputs of order one), and a sequence whose lengths make no sense is zero-filled
+    with the status bit while the others are served."""
+    from paper_2512_05033_b200 import binding
+    inp = wl.small_attn_case(3, 12, 2, 128, BF, [3000, 513, 700], [40, 7, 12], seed=907, q_std=6.0)
+    ks, vs = 0.012, 0.012
+    kc = torch.from_numpy(oracle.e4m3_encode(inp.k_pages, 1 / ks))
+    vc = torch.from_numpy(oracle.e4m3_encode(inp.v_pages, 1 / vs))
+    ref, _ = oracle.attn_e4m3(inp.q, kc, vc, ks, vs, inp.block_table, inp.seq_lens, inp.q_lens)
+    c = H.ctx()
+    d = inp.to("cuda")
+    out = c.attn_e4m3(d.q, kc.cuda(), vc.cuda(), ks, vs, d.block_table, d.seq_lens, d.q_lens, 40)
+    assert c.poll_status() == 0
+    err = np.abs(out.double().cpu().numpy() - ref)
+    assert (err <= 2.0 ** -8 * np.abs(ref) + 3e-3).all(), err.max()
+    bad = d.seq_lens.clone()
+    bad[1] = 3                                   # fewer keys than query tokens
+    out2 = torch.full_like(d.q, float("nan"))
+    c.attn_e4m3(d.q, kc.cuda(), vc.cuda(), ks, vs, d.block_table, bad, d.q_lens, 40, out=out2)
+    assert c.poll_status() == binding.DEV_BAD_SEQ_LEN
+    assert float(out2[40:47].abs().max()) == 0.0
+    assert torch.equal(out2[:40], out[:40]) and torch.equal(out2[47:], out[47:])

@@ -379,6 +379,7 @@ def run_ours(args):
                 result["step_scoring"] = run_step_scoring(ctx, dev)
                 result["mixed_loop"] = run_mixed_loop(ctx, dev)
                 result["step_loop"] = run_step_loop(ctx, dev)
+                result["step_loop"]["e4m3_draft"] = run_step_loop(ctx, dev, e4m3_draft=True)
                 result["kv_append"] = run_kv_append(ctx, dev, peak)
                 result["policies"] = run_policies(ctx, dev)
                 result["e4m3_decode"] = run_e4m3_decode(ctx, dev, peak)
@@ -582,12 +583,13 @@ def run_mixed_loop(ctx, dev):
             "device_status_bits": ctx.poll_status()}
 
 
-def run_step_loop(ctx, dev):
+def run_step_loop(ctx, dev, e4m3_draft: bool = False):
     """Supplementary: whole rounds of Algorithm 1 (step_loop.StepLoop) replayed as one CUDA graph.  Batch 16;
     draft cache 12/2 heads, router cache 28/4 heads with a 3584-wide head, target cache 32/8 heads; prefixes
     uniform in [2048, 8192]; draft and target steps of 8..32 tokens generated token by token; routing at
     tau 0.5; escalated steps rolled back and regenerated; every cache absorbs the step it did not write.
-    One layer call per forward; lengths and decisions never leave the device."""
+    One layer call per forward; lengths and decisions never leave the device.  e4m3_draft: the draft cache holds
+    E4M3 codes (pools of random codes; the quantised-draft regime)."""
     from paper_2512_05033_b200.step_loop import Cache, StepLoop
     B, D, nd, nt, Hr, rounds = 16, 128, 32, 32, 3584, 2
     bf = torch.bfloat16
@@ -599,7 +601,13 @@ def run_step_loop(ctx, dev):
         shape = wl.AttnShape(f"loop-{i}", B, hq, hkv, D, bf, 0, 0, seed=50 + i)
         inp = wl.make_attn_inputs(shape, device=dev, seed=50 + i, extra_tokens=rounds * (nd + nt) + 16,
                                   prefix_lens=prefix, q_lens=torch.zeros(B, dtype=torch.int64))
-        caches.append(Cache(hq, inp.k_pages, inp.v_pages, inp.block_table, inp.seq_lens.clone()))
+        if e4m3_draft and i == 0:
+            g8 = torch.Generator(device=dev)
+            g8.manual_seed(77)
+            codes = [torch.randint(0, 0x7f, inp.k_pages.shape, generator=g8, device=dev, dtype=torch.uint8) for _ in range(2)]
+            caches.append(Cache(hq, codes[0], codes[1], inp.block_table, inp.seq_lens.clone(), e4m3=(0.01, 0.01)))
+        else:
+            caches.append(Cache(hq, inp.k_pages, inp.v_pages, inp.block_table, inp.seq_lens.clone()))
         starts.append(inp.seq_lens.clone())
     r = wl.make_router_inputs(B, Hr, bf, device=dev, seed=60)
     loop = StepLoop(ctx, *caches, r.w, 0.0, 0.5, nd, nt)

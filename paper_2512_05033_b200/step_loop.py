@@ -13,6 +13,9 @@ work it causes:
                  drops z_d and absorbs z_t
   target cache   absorbs accepted draft steps as one chunk; generates z_t token by token for the escalated
 
+A cache may be an E4M3 cache (Cache.e4m3 = its two scales): the reduced-precision cache of a quantised draft
+(Section 5.1).  Its writes go through arb_kv_append_e4m3 and its attention through arb_attn_e4m3.
+
 Which sequences take part in a phase comes from arb_phase_lens / arb_phase_lens_tokens on the device.  A round is therefore a fixed
 list of kernel launches for given maximum step lengths and can be captured in a CUDA graph.
 """
@@ -33,6 +36,7 @@ class Cache:
     v_pages: torch.Tensor
     block_table: torch.Tensor  # int32 [B, max_pages]
     seq_lens: torch.Tensor     # int32 [B], advanced and rolled back in place
+    e4m3: tuple | None = None  # (k_scale, v_scale): the pools hold E4M3 codes (uint8), keys = k_scale * code
 
 
 class StepLoop:
@@ -58,10 +62,15 @@ class StepLoop:
     # -- building blocks ---------------------------------------------------------------------------
     def _absorb(self, name: str, c: Cache, k_new, v_new, q, lens, max_len: int):
         """The cache takes `lens[b]` new tokens per sequence and attends from them (causal chunk)."""
-        self.ctx.kv_append(k_new, v_new, c.block_table, c.seq_lens, lens, c.k_pages, c.v_pages)
         out = self.out.get(name)
         if out is None or out.shape != q.shape:
             out = self.out[name] = torch.zeros_like(q)
+        if c.e4m3 is not None:   # a quantised cache: quantising append, attention over the codes
+            ks, vs = c.e4m3
+            self.ctx.kv_append_e4m3(k_new, v_new, 1.0 / ks, 1.0 / vs, c.block_table, c.seq_lens, lens, c.k_pages, c.v_pages)
+            self.ctx.attn_e4m3(q, c.k_pages, c.v_pages, ks, vs, c.block_table, c.seq_lens, lens, max_len, out=out)
+            return
+        self.ctx.kv_append(k_new, v_new, c.block_table, c.seq_lens, lens, c.k_pages, c.v_pages)
         self.ctx.attn(q, c.k_pages, c.v_pages, c.block_table, c.seq_lens, lens, max_len, out=out)
 
     def _generate(self, name: str, c: Cache, step_lens, decisions, want: int, n_max: int, q, k_new, v_new):
@@ -69,6 +78,9 @@ class StepLoop:
         at token t only sequences that take part and have t < step_lens[b] are active."""
         lens = self.ctx.phase_lens_tokens(step_lens, n_max, decisions, want=want, out=self.token_lens[name])
         for t in range(n_max):   # one launch per token: cache write, attention and length update (arb_decode_step)
+            if c.e4m3 is not None:   # the quantised cache has no fused token call: append, then decode
+                self._absorb(f"{name}[{t}]", c, k_new[t], v_new[t], q[t], lens[t], 1)
+                continue
             key = f"{name}[{t}]"
             out = self.out.get(key)
             if out is None or out.shape != q[t].shape:

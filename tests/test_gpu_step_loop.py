@@ -32,15 +32,29 @@ def _acts(gen, B, nd, nt, geo):
 
 
 class OracleCache:
-    def __init__(self, inp, hq):
-        self.hq, self.k, self.v, self.bt = hq, inp.k_pages.clone(), inp.v_pages.clone(), inp.block_table
+    """The oracle's side of one cache.  e4m3 = (k_scale, v_scale): the pools hold E4M3 codes."""
+
+    def __init__(self, inp, hq, e4m3=None):
+        self.hq, self.bt, self.e4m3 = hq, inp.block_table, e4m3
         self.sl = inp.seq_lens.numpy().copy()
+        if e4m3 is None:
+            self.k, self.v = inp.k_pages.clone(), inp.v_pages.clone()
+        else:
+            self.k = torch.from_numpy(oracle.e4m3_encode(inp.k_pages, 1.0 / e4m3[0]))
+            self.v = torch.from_numpy(oracle.e4m3_encode(inp.v_pages, 1.0 / e4m3[1]))
 
     def absorb(self, k_new, v_new, q, lens):
         n = int(lens.sum())
-        self.k, self.v, self.sl, st = oracle.kv_append(k_new[:n], v_new[:n], self.bt, self.sl, lens, self.k, self.v)
-        assert st == 0
-        out, st = oracle.attn(q[:n], self.k, self.v, self.bt, self.sl, lens)
+        if self.e4m3 is None:
+            self.k, self.v, self.sl, st = oracle.kv_append(k_new[:n], v_new[:n], self.bt, self.sl, lens, self.k, self.v)
+            assert st == 0
+            out, st = oracle.attn(q[:n], self.k, self.v, self.bt, self.sl, lens)
+        else:
+            ks, vs = self.e4m3
+            self.k, self.v, self.sl, st = oracle.kv_append_e4m3(k_new[:n], v_new[:n], self.bt, self.sl, lens, self.k,
+                                                                self.v, 1.0 / ks, 1.0 / vs)
+            assert st == 0
+            out, st = oracle.attn_e4m3(q[:n], self.k, self.v, ks, vs, self.bt, self.sl, lens)
         assert st == 0
         return out
 
@@ -68,7 +82,10 @@ def _oracle_round(d, r, tg, step_d, step_t, hidden, w, b, tau, acts, nd, nt):
     return scores, dec, outs
 
 
-def test_two_rounds_of_the_step_loop_match_the_oracle():
+@pytest.mark.parametrize("draft_e4m3", [None, (0.02, 0.03)])
+def test_two_rounds_of_the_step_loop_match_the_oracle(draft_e4m3):
+    """draft_e4m3: the draft model's cache holds E4M3 codes (the quantised-draft regime): its tokens are appended
+    quantised and decoded over the codes, and the target's step reaches it as a causal chunk over the codes."""
     from paper_2512_05033_b200 import binding
     from paper_2512_05033_b200.step_loop import Cache, StepLoop
     c = H.ctx()
@@ -77,9 +94,9 @@ def test_two_rounds_of_the_step_loop_match_the_oracle():
     prefix = [300, 33, 1000, 64]
     room = 3 * (nd + nt) + 16
     inps = [_cache(B, hq, hkv, D, prefix, 400 + i, room) for i, (hq, hkv) in enumerate(geo[:3])]
-    dev_caches = [Cache(hq, i.k_pages.cuda(), i.v_pages.cuda(), i.block_table.cuda(), i.seq_lens.cuda())
-                  for i, (hq, _) in zip(inps, geo[:3])]
-    ora = [OracleCache(i, hq) for i, (hq, _) in zip(inps, geo[:3])]
+    ora = [OracleCache(i, hq, draft_e4m3 if k == 0 else None) for k, (i, (hq, _)) in enumerate(zip(inps, geo[:3]))]
+    dev_caches = [Cache(o.hq, o.k.cuda(), o.v.cuda(), i.block_table.cuda(), i.seq_lens.cuda(), e4m3=o.e4m3)
+                  for i, o in zip(inps, ora)]
     g = torch.Generator().manual_seed(12)
     w = (torch.randn(Hd, generator=g) / Hd ** 0.5).to(BF)
     loop = StepLoop(c, *dev_caches, w.cuda(), 0.0, 0.5, nd, nt)

@@ -63,7 +63,8 @@ enum {
     ARB_DEV_BAD_SEQ_LEN = 1u,        /* q_len > 0 and (seq_len < q_len or seq_len > max_pages*page) */
     ARB_DEV_BAD_PAGE = 2u,           /* block_table entry outside [0, num_pages) */
     ARB_DEV_ROLLBACK_UNDERFLOW = 4u, /* step_len < 0 or step_len > seq_len */
-    ARB_DEV_WAIT_TIMEOUT = 8u        /* a bounded wait on an asynchronous copy or MMA gave up */
+    ARB_DEV_WAIT_TIMEOUT = 8u,       /* a bounded wait on an asynchronous copy or MMA gave up */
+    ARB_DEV_CHECK_FAILED = 16u       /* bounds-check build only: an index the device derived was out of range; the access was skipped */
 };
 
 /* escalation policies of arb_policy */
@@ -481,6 +482,17 @@ arb_status arb_poll_status(arb_ctx *ctx, arb_stream_t stream, uint32_t *bits);
  * The paper has no counterpart; this is failure-detection plumbing of the library.
  */
 arb_status arb_selftest_wait_timeout(arb_ctx *ctx, int64_t limit_cycles, int32_t *report, arb_stream_t stream);
+
+/*
+ * The bounds-check build (python -m paper_2512_05033_b200.build --checks, libarb_checks.so, -DARB_CHECKS) tests
+ * the indices the kernels derive on the device before they are used (ring stage, block-table entry, workspace
+ * slot, output row, pool offset): a failing test raises ARB_DEV_CHECK_FAILED and skips the access.  In that
+ * build every buffer a ctx owns also lies between two guard zones of a fixed byte pattern.  This call counts,
+ * on `stream`, the guard bytes that no longer hold the pattern and returns the count in *bad (host pointer)
+ * after synchronising; the ordinary build owns no guard zones and returns 0.  *checked receives the number of
+ * guard bytes looked at.  The paper has no counterpart; this stands in for a memory checker.
+ */
+arb_status arb_selftest_guard_zones(arb_ctx *ctx, arb_stream_t stream, int64_t *bad, int64_t *checked);
 
 /* Number of kernels the library has launched through this ctx since arb_create. */
 uint64_t arb_launch_count(const arb_ctx *ctx);

@@ -11,7 +11,11 @@ from pathlib import Path
 
 import torch
 
-_LIB_PATH = Path(__file__).resolve().parent / "libarb.so"
+import os
+
+# ARB_LIB_VARIANT=checks selects the bounds-check build (python -m paper_2512_05033_b200.build --checks)
+_LIB_PATH = Path(__file__).resolve().parent / ("libarb_checks.so" if os.environ.get("ARB_LIB_VARIANT") == "checks"
+                                               else "libarb.so")
 if not _LIB_PATH.exists():
     raise ImportError(
         f"{_LIB_PATH} is missing: build the CUDA library first "
@@ -23,7 +27,7 @@ ARB_OK = 0
 ARB_ERR_INVALID_ARG, ARB_ERR_UNSUPPORTED, ARB_ERR_WORKSPACE, ARB_ERR_CUDA, ARB_ERR_DEVICE_STATUS = 1, 2, 3, 4, 5
 ARB_ERR_STATIC_LIMIT = 6
 ARB_F32, ARB_BF16 = 0, 1
-DEV_BAD_SEQ_LEN, DEV_BAD_PAGE, DEV_ROLLBACK_UNDERFLOW, DEV_WAIT_TIMEOUT = 1, 2, 4, 8
+DEV_BAD_SEQ_LEN, DEV_BAD_PAGE, DEV_ROLLBACK_UNDERFLOW, DEV_WAIT_TIMEOUT, DEV_CHECK_FAILED = 1, 2, 4, 8, 16
 ATTN_OVERLAP_PREVIOUS = 1
 ATTN_NO_TENSOR_CORES = 2
 POLICY_RSD, POLICY_ORACLE_THRESHOLD, POLICY_ORACLE_ARGMAX, POLICY_ORACLE_BUDGET = 0, 1, 2, 3
@@ -35,7 +39,7 @@ EXPORTS = ("arb_create", "arb_destroy", "arb_attn_workspace_bytes", "arb_attn", 
            "arb_attn_host_begin", "arb_attn_host_wait",
            "arb_attn_decode_static", "arb_decode_step",
            "arb_route", "arb_rollback", "arb_policy", "arb_route_classes", "arb_kv_append", "arb_kv_append_e4m3", "arb_attn_decode_e4m3", "arb_attn_e4m3", "arb_phase_lens", "arb_phase_lens_tokens", "arb_spearman",
-           "arb_selftest_wait_timeout", "arb_poll_status", "arb_launch_count", "arb_status_string")
+           "arb_selftest_wait_timeout", "arb_selftest_guard_zones", "arb_poll_status", "arb_launch_count", "arb_status_string")
 
 
 class AttnParams(ctypes.Structure):
@@ -90,6 +94,8 @@ lib.arb_kv_append.restype = ctypes.c_int
 lib.arb_kv_append.argtypes = [_vp, ctypes.POINTER(AttnParams), _i32, _vp, _vp, _vp, _vp, _vp, _i32, _vp, _vp, _vp]
 lib.arb_selftest_wait_timeout.restype = ctypes.c_int
 lib.arb_selftest_wait_timeout.argtypes = [_vp, ctypes.c_int64, _vp, _vp]
+lib.arb_selftest_guard_zones.restype = ctypes.c_int
+lib.arb_selftest_guard_zones.argtypes = [_vp, _vp, ctypes.POINTER(ctypes.c_int64), ctypes.POINTER(ctypes.c_int64)]
 lib.arb_poll_status.restype = ctypes.c_int
 lib.arb_poll_status.argtypes = [_vp, _vp, ctypes.POINTER(ctypes.c_uint32)]
 lib.arb_launch_count.restype = ctypes.c_uint64
@@ -442,6 +448,13 @@ class Context:
         _check(lib.arb_selftest_wait_timeout(self._h, int(limit_cycles), _dev(report, "report", torch.int32),
                                              _stream_ptr(stream)), "arb_selftest_wait_timeout")
         return report
+
+    def guard_zones(self, stream=None):
+        """(bytes of the guard zones that were overwritten, guard bytes checked); (0, 0) in the ordinary build."""
+        bad, checked = ctypes.c_int64(0), ctypes.c_int64(0)
+        _check(lib.arb_selftest_guard_zones(self._h, _stream_ptr(stream), ctypes.byref(bad), ctypes.byref(checked)),
+               "arb_selftest_guard_zones")
+        return int(bad.value), int(checked.value)
 
     # -- status -------------------------------------------------------------------------------
     def poll_status(self, stream=None) -> int:

@@ -1,6 +1,10 @@
 """Build libarb.so (the C-ABI CUDA library) in-tree with nvcc for sm_100a.
 
-    python -m paper_2512_05033_b200.build [--force] [--verbose]
+    python -m paper_2512_05033_b200.build [--force] [--verbose] [--checks]
+
+--checks builds libarb_checks.so instead: the same sources with -DARB_CHECKS (device-side range tests that raise
+ARB_DEV_CHECK_FAILED and skip the access, guard zones around the buffers a context owns).  The binding loads it when
+ARB_LIB_VARIANT=checks is set; it is for test runs, not for timing.
 """
 from __future__ import annotations
 
@@ -30,14 +34,16 @@ def _stale(target: Path, deps) -> bool:
     return any(d.stat().st_mtime > t for d in deps)
 
 
-def build(force: bool = False, verbose: bool = False) -> Path:
+def build(force: bool = False, verbose: bool = False, checks: bool = False) -> Path:
     headers = list(CSRC.glob("*.cuh")) + [HERE.parent / "include" / "arb.h", Path(__file__)]
+    OBJ = HERE / ("_build_checks" if checks else "_build")
+    LIB = HERE / ("libarb_checks.so" if checks else "libarb.so")
     OBJ.mkdir(exist_ok=True)
     jobs = []
     for src in _sources():
         obj = OBJ / (src.stem + ".o")
         if force or _stale(obj, [src] + headers):
-            cmd = [NVCC, *FLAGS, "-c", str(src), "-o", str(obj)]
+            cmd = [NVCC, *FLAGS, *(["-DARB_CHECKS"] if checks else []), "-c", str(src), "-o", str(obj)]
             if verbose:
                 cmd.insert(1, "-Xptxas=-v")
             jobs.append(cmd)
@@ -58,4 +64,4 @@ def build(force: bool = False, verbose: bool = False) -> Path:
 
 
 if __name__ == "__main__":
-    print(build(force="--force" in sys.argv, verbose="--verbose" in sys.argv))
+    print(build(force="--force" in sys.argv, verbose="--verbose" in sys.argv, checks="--checks" in sys.argv))

@@ -32,6 +32,30 @@ arb_status check_params(const arb_attn_params *p) {
     return ARB_OK;
 }
 
+// Device allocations of a ctx.  In the bounds-check build each lies between two guard zones of kGuardBytes filled
+// with kGuardPattern (kGuardBytes is 0 in the ordinary build and these are plain cudaMalloc / cudaFree).
+template <typename T>
+bool guarded_malloc(Ctx *c, T **ptr, size_t bytes) {
+    const size_t body = (bytes + 255) & ~size_t(255);
+    char *raw = nullptr;
+    if (cudaMalloc(&raw, body + 2 * kGuardBytes) != cudaSuccess) return false;
+    if (kGuardBytes > 0) {
+        if (cudaMemset(raw, kGuardPattern, kGuardBytes) != cudaSuccess ||
+            cudaMemset(raw + kGuardBytes + body, kGuardPattern, kGuardBytes) != cudaSuccess || c->n_guards + 2 > 16) {
+            cudaFree(raw);
+            return false;
+        }
+        c->guards[c->n_guards++] = reinterpret_cast<unsigned char *>(raw);
+        c->guards[c->n_guards++] = reinterpret_cast<unsigned char *>(raw + kGuardBytes + body);
+    }
+    *ptr = reinterpret_cast<T *>(raw + kGuardBytes);
+    return true;
+}
+
+void guarded_free(void *p) {
+    if (p != nullptr) cudaFree(static_cast<char *>(p) - kGuardBytes);
+}
+
 struct DeviceGuard {
     int prev = -1;
     bool ok = true;
@@ -119,26 +143,33 @@ arb_status arb_create(arb_ctx **out, int device, size_t workspace_bytes) {
     if (const char *pct = std::getenv("ARB_STEP_BOUNDARY_PCT")) c->step_boundary_pct = std::max(0, std::min(400, std::atoi(pct)));
     c->workspace_bytes = workspace_bytes ? workspace_bytes : kDefaultWorkspace;
     c->counters_len = kCounters;
-    bool ok = cudaMalloc(&c->workspace, c->workspace_bytes) == cudaSuccess;
-    ok = ok && cudaMalloc(&c->counters, sizeof(int) * (c->counters_len + 4)) == cudaSuccess;
+    bool ok = guarded_malloc(c, &c->workspace, c->workspace_bytes);
+    ok = ok && guarded_malloc(c, &c->counters, sizeof(int) * (c->counters_len + 4));
     ok = ok && cudaMemset(c->counters, 0, sizeof(int) * (c->counters_len + 4)) == cudaSuccess;
     const size_t rot_ints = (size_t)kRotSets * kRotCounters + kRotSets + 8;
-    ok = ok && cudaMalloc(&c->rot, sizeof(int) * rot_ints) == cudaSuccess;
+    ok = ok && guarded_malloc(c, &c->rot, sizeof(int) * rot_ints);
     ok = ok && cudaMemset(c->rot, 0, sizeof(int) * rot_ints) == cudaSuccess;
-    ok = ok && cudaMalloc(&c->spearman_acc, 4 * sizeof(double)) == cudaSuccess;
+    ok = ok && guarded_malloc(c, &c->spearman_acc, 4 * sizeof(double));
     c->chunk_ws_bytes = 2 * c->workspace_bytes;   // partials of long step chunks that are split over their keys
-    ok = ok && cudaMalloc(&c->chunk_ws, c->chunk_ws_bytes) == cudaSuccess;
+    ok = ok && guarded_malloc(c, &c->chunk_ws, c->chunk_ws_bytes);
+    if (ok && c->n_guards > 0) {
+        ok = cudaMalloc(&c->guards_dev, sizeof(c->guards)) == cudaSuccess &&
+             cudaMalloc(&c->guard_bad, sizeof(unsigned long long)) == cudaSuccess &&
+             cudaMemcpy(c->guards_dev, c->guards, sizeof(c->guards), cudaMemcpyHostToDevice) == cudaSuccess;
+    }
     if (ok) {  // "everything before the first call has completed"
         const uint32_t done = c->decode_gen - 1;
         ok = cudaMemcpy(c->rot + (size_t)kRotSets * kRotCounters + kRotSets, &done, sizeof(done),
                         cudaMemcpyHostToDevice) == cudaSuccess;
     }
     if (!ok) {
-        cudaFree(c->workspace);
-        cudaFree(c->counters);
-        cudaFree(c->rot);
-        cudaFree(c->spearman_acc);
-        cudaFree(c->chunk_ws);
+        guarded_free(c->workspace);
+        guarded_free(c->counters);
+        guarded_free(c->rot);
+        guarded_free(c->spearman_acc);
+        guarded_free(c->chunk_ws);
+        cudaFree(c->guards_dev);
+        cudaFree(c->guard_bad);
         delete c;
         cudaGetLastError();
         return ARB_ERR_CUDA;
@@ -152,11 +183,13 @@ arb_status arb_destroy(arb_ctx *ctx) {
     if (ctx == nullptr) return ARB_ERR_INVALID_ARG;
     Ctx *c = reinterpret_cast<Ctx *>(ctx);
     DeviceGuard guard(c->device);
-    cudaFree(c->workspace);
-    cudaFree(c->counters);
-    cudaFree(c->rot);
-    cudaFree(c->spearman_acc);
-    cudaFree(c->chunk_ws);
+    guarded_free(c->workspace);
+    guarded_free(c->counters);
+    guarded_free(c->rot);
+    guarded_free(c->spearman_acc);
+    guarded_free(c->chunk_ws);
+    cudaFree(c->guards_dev);
+    cudaFree(c->guard_bad);
     cudaFree(c->stage);
     cudaFreeHost(c->host_stage);
     pipe_teardown(c);
@@ -648,6 +681,33 @@ arb_status arb_selftest_wait_timeout(arb_ctx *ctx, int64_t limit_cycles, int32_t
     if (limit_cycles < 1 || limit_cycles > (1ll << 31)) return ARB_ERR_INVALID_ARG;   // at most about a second
     return launch_selftest_wait(reinterpret_cast<Ctx *>(ctx), limit_cycles, report, reinterpret_cast<cudaStream_t>(stream));
 }
+
+arb_status arb_selftest_guard_zones(arb_ctx *ctx, arb_stream_t stream, int64_t *bad, int64_t *checked) {
+    if (ctx == nullptr || bad == nullptr) return ARB_ERR_INVALID_ARG;
+    Ctx *c = reinterpret_cast<Ctx *>(ctx);
+    cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+    *bad = 0;
+    if (checked) *checked = (int64_t)c->n_guards * (int64_t)kGuardBytes;
+    if (c->n_guards == 0) return cudaStreamSynchronize(s) == cudaSuccess ? ARB_OK : ARB_ERR_CUDA;
+    unsigned long long host = 0;
+    if (cudaMemsetAsync(c->guard_bad, 0, sizeof(unsigned long long), s) != cudaSuccess) return ARB_ERR_CUDA;
+    const arb_status st = launch_guard_count(c, c->guards_dev, c->n_guards, kGuardBytes, c->guard_bad, s);
+    if (st != ARB_OK) return st;
+    if (cudaMemcpyAsync(&host, c->guard_bad, sizeof(host), cudaMemcpyDeviceToHost, s) != cudaSuccess) return ARB_ERR_CUDA;
+    if (cudaStreamSynchronize(s) != cudaSuccess) return ARB_ERR_CUDA;
+    *bad = (int64_t)host;
+    return ARB_OK;
+}
+
+#ifdef ARB_CHECKS
+// Bounds-check build only, for the test of the guard check itself: overwrites the last `nbytes` bytes of the guard
+// zone in front of the workspace (memory this ctx owns), as a store just below the buffer would.
+int arb_debug_poke_guard(arb_ctx *ctx, int nbytes) {
+    if (ctx == nullptr || nbytes < 1 || (size_t)nbytes > kGuardBytes) return 1;
+    Ctx *c = reinterpret_cast<Ctx *>(ctx);
+    return cudaMemset(c->workspace - nbytes, 0, (size_t)nbytes) == cudaSuccess ? 0 : 1;
+}
+#endif
 
 uint64_t arb_launch_count(const arb_ctx *ctx) {
     return ctx ? reinterpret_cast<const Ctx *>(ctx)->launches : 0;

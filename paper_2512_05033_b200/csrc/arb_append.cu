@@ -119,6 +119,7 @@ kv_append_kernel(const AppendArgs a) {
         const int page = a.block_table[(size_t)lo * a.max_pages + pos / kPage];
         const size_t dst = (((size_t)page * a.Hkv + h) * kPage + (pos % kPage)) * a.row_bytes + (size_t)vec * 16;
         const size_t src = (size_t)r * a.row_bytes + (size_t)vec * 16;
+        if (!ARB_IN_RANGE(a.status, dst + 15, (size_t)a.num_pages * a.Hkv * kPage * a.row_bytes)) continue;
         const uint4 kx = __ldg(reinterpret_cast<const uint4 *>(a.k_new + src));
         const uint4 vx = __ldg(reinterpret_cast<const uint4 *>(a.v_new + src));
         *reinterpret_cast<uint4 *>(a.k_pages + dst) = kx;

@@ -92,6 +92,7 @@ struct MmaArgs {
     int split_cap;      // slots that fit there
     int fill_ctas;      // CTAs a call should keep busy: a call with fewer than half as many work items has its
                         // sequences cut over their keys as well (0: never)
+    int rows;           // rows of q and out (bounds-check build)
     float scale_log2;   // softmax scale (times the key scale of an E4M3 cache) * log2(e)
     float v_scale;      // value scale of an E4M3 cache, 1 otherwise
 };
@@ -539,7 +540,8 @@ chunk_mma_kernel(const MmaArgs a, const __grid_constant__ CUtensorMap k_map, con
                 if (jt >= w.ntiles) return -1;
                 jt += w.t0;
                 const int np = min(kTilePages, (w.kv_len - jt * kBN + kPage - 1) / kPage);
-                return (lane < np) ? a.block_table[(size_t)w.b * a.max_pages + jt * kTilePages + lane] : -1;
+                return (lane < np && ARB_IN_RANGE(a.status, jt * kTilePages + lane, a.max_pages))
+                           ? a.block_table[(size_t)w.b * a.max_pages + jt * kTilePages + lane] : -1;
             };
             // K and V tiles are asked into L2 kPrefetchTiles ahead of their load into the ring, so the
             // ring (two tiles deep) only has to cover the L2 latency, not the DRAM latency
@@ -855,15 +857,17 @@ chunk_mma_kernel(const MmaArgs a, const __grid_constant__ CUtensorMap k_map, con
             // ---- epilogue: O / l, bf16, one 256-byte row per thread
             mbar_wait(&bars->o_full[grp], (itg - 1u) & 1u, abort, a.status);
             tc_fence_after();
+            const bool row_in = ARB_IN_RANGE(a.status, w.qrow0 + tok, a.rows);
             if (w.split) {
                 // one part of a split sequence: leave the un-normalised O row and its (max, sum)
-                float *po = a.split_ws + (size_t)(w.slot + grp) * kSlotFloats;
+                const bool slot_in = ARB_IN_RANGE(a.status, w.slot + grp, a.split_cap);
+                float *po = a.split_ws + (size_t)(slot_in ? w.slot + grp : 0) * kSlotFloats;
 #pragma unroll 1
                 for (int c4 = 0; c4 < 4; ++c4) {
                     uint32_t v[32];
                     tmem_ld32(o_tmem + c4 * 32, v);
                     tmem_wait_ld();
-                    if (row_ok) {
+                    if (row_ok && slot_in) {
                         if constexpr (E4M3) {   // values of an E4M3 cache are v_scale * code
 #pragma unroll
                             for (int k = 0; k < 32; ++k) v[k] = __float_as_uint(__uint_as_float(v[k]) * a.v_scale);
@@ -874,7 +878,7 @@ chunk_mma_kernel(const MmaArgs a, const __grid_constant__ CUtensorMap k_map, con
                                 make_uint4(v[qd * 4], v[qd * 4 + 1], v[qd * 4 + 2], v[qd * 4 + 3]);
                     }
                 }
-                if (row_ok) *reinterpret_cast<float2 *>(po + (size_t)kBM * kD + tg * 2) = make_float2(m_used, l_sum);
+                if (row_ok && slot_in) *reinterpret_cast<float2 *>(po + (size_t)kBM * kD + tg * 2) = make_float2(m_used, l_sum);
                 tc_fence_before();
                 continue;
             }
@@ -885,7 +889,7 @@ chunk_mma_kernel(const MmaArgs a, const __grid_constant__ CUtensorMap k_map, con
                 uint32_t v[32];
                 tmem_ld32(o_tmem + c4 * 32, v);
                 tmem_wait_ld();
-                if (row_ok) {
+                if (row_ok && row_in) {
 #pragma unroll
                     for (int qd = 0; qd < 4; ++qd) {
                         uint4 o4;
@@ -1049,6 +1053,7 @@ arb_status launch_chunk_tc(Ctx *ctx, const arb_attn_params &p, const void *q, co
     a.Hkv = p.num_kv_heads;
     a.num_pages = p.num_pages;
     a.max_pages = p.max_pages_per_seq;
+    a.rows = p.total_q;
     a.min_rows = kChunkMmaMinRows;
     a.work_counter = ctx->rot + (size_t)kRotSets * kRotCounters + kRotSets + 1;
     a.split_ws = ctx->chunk_ws;

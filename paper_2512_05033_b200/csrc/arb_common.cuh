@@ -67,6 +67,12 @@ struct Ctx {
     int step_boundary_pct = 100;          // single-launch decode: what a (sequence, kv head) boundary inside a CTA's range counts for
     float *chunk_ws = nullptr;            // partial results of split long sequences (step-chunk attention)
     size_t chunk_ws_bytes = 0;
+    // bounds-check build: the guard zones around the buffers above (device addresses), their copy on the device,
+    // and the counter the guard check adds up in
+    const unsigned char *guards[16] = {};
+    int n_guards = 0;
+    const unsigned char **guards_dev = nullptr;
+    unsigned long long *guard_bad = nullptr;
 };
 
 constexpr int kRotSets = 4;
@@ -83,6 +89,22 @@ inline size_t rot_region_bytes(const Ctx *ctx) { return (ctx->workspace_bytes / 
 inline void note_unnumbered_decode(Ctx *ctx, size_t bytes) {
     if (bytes > rot_region_bytes(ctx)) ctx->rot_wait_through = ctx->decode_gen + (uint32_t)kRotSets - 1u;
 }
+
+// ---------------------------------------------------------------------------------------------
+// Bounds-check build (-DARB_CHECKS): indices derived on the device are tested before use; a failing test raises
+// ARB_DEV_CHECK_FAILED and the caller skips the access.  In the ordinary build the test is `true` and costs nothing.
+// ---------------------------------------------------------------------------------------------
+#ifdef ARB_CHECKS
+#define ARB_IN_RANGE(status, idx, limit)                                  \
+    (((unsigned long long)(idx) < (unsigned long long)(limit))            \
+         ? true                                                           \
+         : (atomicOr((status), (uint32_t)ARB_DEV_CHECK_FAILED), false))
+constexpr size_t kGuardBytes = 4096;    // guard zone on either side of every buffer a ctx owns
+#else
+#define ARB_IN_RANGE(status, idx, limit) true
+constexpr size_t kGuardBytes = 0;
+#endif
+constexpr unsigned char kGuardPattern = 0xA5;
 
 // ---------------------------------------------------------------------------------------------
 // Element types
@@ -300,6 +322,8 @@ bool decode_step_supported(const arb_attn_params &p);
 arb_status launch_decode_step(Ctx *ctx, const arb_attn_params &p, const void *q, const void *k_new, const void *v_new,
                               void *k_pages, void *v_pages, const int32_t *block_table, int32_t *seq_lens,
                               const int32_t *q_lens, void *out, cudaStream_t stream);
+arb_status launch_guard_count(Ctx *ctx, const unsigned char *const *zones, int n_zones, size_t zone_bytes,
+                              unsigned long long *bad_dev, cudaStream_t stream);
 arb_status launch_selftest_wait(Ctx *ctx, long long limit_cycles, int32_t *report, cudaStream_t stream);
 size_t decode_workspace_bytes(const arb_attn_params &p, int num_sms);
 int decode_grid(int num_sms);

@@ -86,6 +86,7 @@ struct Args {
     float v_scale;      // value scale of an E4M3 cache, 1 otherwise
     // workspace rotation (see launch_decode_mma): this call's generation number, the number of
     // workspace sets, the generation of the newest completed call
+    int slots, rows;  // partial slots of a workspace set; rows of q and out (bounds-check build)
     uint32_t gen;
     int sets;
     int force_wait;
@@ -257,7 +258,7 @@ decode_mma_kernel(const Args a, const __grid_constant__ CUtensorMap k_map, const
             for (int sp0 = s.pg0; sp0 < s.pg1; sp0 += 32) {
                 const int np = min(32, s.pg1 - sp0);
                 int pid = 0;
-                if (lane < np) {
+                if (lane < np && ARB_IN_RANGE(a.status, sp0 + lane, a.max_pages)) {
                     pid = a.block_table[(size_t)s.b * a.max_pages + sp0 + lane];
                     if ((unsigned)pid >= (unsigned)a.num_pages) {
                         atomicOr(a.status, (uint32_t)ARB_DEV_BAD_PAGE);
@@ -365,6 +366,7 @@ decode_mma_kernel(const Args a, const __grid_constant__ CUtensorMap k_map, const
                 if (pk[j].nparts == 1) continue;
                 const float *rec = park + j * REC;
                 const size_t slot = (size_t)pk[j].bk + blockIdx.x;
+                if (!ARB_IN_RANGE(a.status, slot, a.slots)) continue;
                 for (int idx = tid; idx < G * kD / 4; idx += kCT)
                     reinterpret_cast<float4 *>(a.part_o + slot * G * kD)[idx] =
                         reinterpret_cast<const float4 *>(rec + 2 * GP)[idx];
@@ -602,6 +604,7 @@ decode_mma_kernel(const Args a, const __grid_constant__ CUtensorMap k_map, const
     if (any_single || blockIdx.x == 0) ensure_wait();
     for (int j = 0; j < n_parked; ++j) {
         if (pk[j].nparts != 1) continue;
+        if (!ARB_IN_RANGE(a.status, pk[j].out_base + G * kD - 1, (size_t)a.rows * a.Hq * kD)) continue;
         const float *rec = park + j * REC;
         for (int idx = tid; idx < G * kD; idx += kCT)
             reinterpret_cast<__nv_bfloat16 *>(a.out)[pk[j].out_base + idx] =
@@ -881,6 +884,8 @@ arb_status launch_decode_tc(Ctx *ctx, const arb_attn_params &p, const void *q, c
     a.sets = sets;
     a.force_wait = force_wait ? 1 : 0;
     a.status = ctx->status;
+    a.slots = (int)slots;
+    a.rows = p.total_q;
     a.batch = p.batch;
     a.Hq = p.num_q_heads;
     a.Hkv = p.num_kv_heads;

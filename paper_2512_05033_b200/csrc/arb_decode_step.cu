@@ -59,6 +59,8 @@ struct StepArgs {
     uint32_t *status;
     int batch, Hq, Hkv, num_pages, max_pages;
     int whole_rows;    // the tensor maps are 3-D: one copy per page tile instead of one per half
+    int slots;         // partial slots in the workspace region (bounds-check build)
+    int rows;          // rows of q and out
     int min_chunk;     // fewest pages worth giving a CTA
     int boundary_pct;  // cost of a (sequence, kv head) boundary inside a CTA's range: percent of min(even share, kBoundaryCap) pages
     float scale_log2;
@@ -366,7 +368,8 @@ decode_step_kernel(const StepArgs a, const __grid_constant__ CUtensorMap k_map, 
             const int pages = pl.pages_of(lo);
             int pg;
             const int kvh = small_div(r - pref[lo], pages, pg);
-            int pid = a.block_table[(size_t)lo * a.max_pages + pg];
+            int pid = ARB_IN_RANGE(a.status, pg, a.max_pages) && ARB_IN_RANGE(a.status, kvh, Hkv)
+                          ? a.block_table[(size_t)lo * a.max_pages + pg] : 0;
             if ((unsigned)pid >= (unsigned)a.num_pages) {
                 atomicOr(a.status, (uint32_t)ARB_DEV_BAD_PAGE);
                 pid = 0;
@@ -387,7 +390,8 @@ decode_step_kernel(const StepArgs a, const __grid_constant__ CUtensorMap k_map, 
                 if (i < ntiles) {
                     const uint32_t cc = c + i, st = cc % STAGES, par = (cc / STAGES) & 1u;
                     const CUtensorMap *map = (i & 1) ? &v_map : &k_map;
-                    if (mbar_wait(&tail->empty[st], par ^ 1u, abort, a.status)) {
+                    if (ARB_IN_RANGE(a.status, row, (long long)a.num_pages * Hkv * kPage) &&
+                        mbar_wait(&tail->empty[st], par ^ 1u, abort, a.status)) {
                         mbar_arrive_expect_tx(&tail->full[st], kTileBytes);
                         if (a.whole_rows) {
                             tma_box_load3(ring + st * kTileBytes, map, 0, row, 0, &tail->full[st]);
@@ -435,12 +439,14 @@ decode_step_kernel(const StepArgs a, const __grid_constant__ CUtensorMap k_map, 
         for (int j = 0; j < n_parked; ++j) {
             const float *rec = park + j * REC;
             if (pk[j].nparts == 1) {
+                if (!ARB_IN_RANGE(a.status, pk[j].out_base + G * kD - 1, (size_t)a.rows * a.Hq * kD)) continue;
                 for (int idx = tid; idx < G * kD; idx += kCT)
                     reinterpret_cast<__nv_bfloat16 *>(a.out)[pk[j].out_base + idx] =
                         __float2bfloat16_rn(rec[2 * GP + idx] / rec[GP + idx / kD]);
             } else {
                 any_multi = true;
                 const size_t slot = (size_t)pk[j].bk + blockIdx.x;
+                if (!ARB_IN_RANGE(a.status, slot, a.slots)) continue;
                 for (int idx = tid; idx < G * kD / 4; idx += kCT)
                     reinterpret_cast<float4 *>(a.part_o + slot * G * kD)[idx] =
                         reinterpret_cast<const float4 *>(rec + 2 * GP)[idx];
@@ -511,7 +517,7 @@ decode_step_kernel(const StepArgs a, const __grid_constant__ CUtensorMap k_map, 
                 const char *src = (lane < 16 ? a.k_new : a.v_new) + ((size_t)qrow * Hkv + s.kvh) * kD * 2 + (lane & 15) * 16;
                 new_row = __ldg(reinterpret_cast<const uint4 *>(src));
                 const int pid = a.block_table[(size_t)s.b * a.max_pages + last_pg];
-                if ((unsigned)pid < (unsigned)a.num_pages) {
+                if ((unsigned)pid < (unsigned)a.num_pages && ARB_IN_RANGE(a.status, qrow, a.rows)) {
                     char *dst = (lane < 16 ? a.k_pool : a.v_pool) +
                                 (((size_t)pid * Hkv + s.kvh) * kPage + new_slot) * (kD * 2) + (lane & 15) * 16;
                     *reinterpret_cast<uint4 *>(dst) = new_row;
@@ -738,7 +744,7 @@ decode_step_kernel(const StepArgs a, const __grid_constant__ CUtensorMap k_map, 
     }
 #pragma unroll
     for (int j = 0; j < 2; ++j) {
-        if (j < pend_n && mine) {
+        if (j < pend_n && mine && ARB_IN_RANGE(a.status, pend[j].out_base + G * kD - 1, (size_t)a.rows * a.Hq * kD)) {
             const float inv = 1.0f / l[j];
             uint2 o2;
             o2.x = pack_bf16(x[j].x * inv, x[j].y * inv);
@@ -828,6 +834,8 @@ arb_status launch_decode_step(Ctx *ctx, const arb_attn_params &p, const void *q,
     a.num_pages = p.num_pages;
     a.max_pages = p.max_pages_per_seq;
     a.whole_rows = whole_rows ? 1 : 0;
+    a.slots = (int)slots;
+    a.rows = p.total_q;
     a.boundary_pct = ctx->step_boundary_pct;
     a.min_chunk = ctx->step_min_chunk;
     const float scale = p.softmax_scale > 0.f ? p.softmax_scale : 1.0f / sqrtf((float)p.head_dim);

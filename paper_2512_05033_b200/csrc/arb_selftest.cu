@@ -39,7 +39,24 @@ selftest_wait_kernel(long long limit, uint32_t *status, int32_t *report) {
     }
 }
 
+// counts the bytes of the guard zones that do not hold the pattern; zones: device array of n pointers
+__global__ void guard_count_kernel(const unsigned char *const *zones, int n_zones, size_t zone_bytes,
+                                   unsigned long long *bad) {
+    unsigned long long mine = 0;
+    for (int z = 0; z < n_zones; ++z)
+        for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < zone_bytes; i += (size_t)gridDim.x * blockDim.x)
+            mine += zones[z][i] != kGuardPattern;
+    if (mine) atomicAdd(bad, mine);
+}
+
 }  // namespace
+
+arb_status launch_guard_count(Ctx *ctx, const unsigned char *const *zones, int n_zones, size_t zone_bytes,
+                              unsigned long long *bad_dev, cudaStream_t stream) {
+    guard_count_kernel<<<8, 256, 0, stream>>>(zones, n_zones, zone_bytes, bad_dev);
+    ctx->launches++;
+    return cudaGetLastError() == cudaSuccess ? ARB_OK : ARB_ERR_CUDA;
+}
 
 arb_status launch_selftest_wait(Ctx *ctx, long long limit_cycles, int32_t *report, cudaStream_t stream) {
     selftest_wait_kernel<<<1, kSelftestThreads, 0, stream>>>(limit_cycles, ctx->status, report);

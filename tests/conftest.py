@@ -26,3 +26,15 @@ def pytest_collection_modifyitems(config, items):
     for item in items:
         if "gpu" in item.keywords:
             item.add_marker(skip)
+
+
+def pytest_sessionfinish(session, exitstatus):
+    # Under the bounds-check build (ARB_LIB_VARIANT=checks) the buffers of the shared context lie between guard
+    # zones: after the last test they must still hold their pattern.
+    if os.environ.get("ARB_LIB_VARIANT") != "checks":
+        return
+    from tests import helpers
+    bad, checked = helpers.guard_zones()
+    print(f"\nguard zones: {checked} bytes checked, {bad} overwritten")
+    if bad and session.exitstatus == 0:
+        session.exitstatus = 1

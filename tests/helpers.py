@@ -19,12 +19,22 @@ def gpu_attn(inp, scale=0.0, flags=0):
     """inp: workloads.AttnInputs on the CPU.  Returns (out fp64 numpy, status bits)."""
     d = inp.to("cuda")
     max_q = int(inp.q_lens.max()) if inp.q_lens.numel() else 0
-    out = torch.full_like(d.q, float("nan"))
+    # `out` lies between two guard rows: a store before its first or past its last row would show in them
+    guard = 12345.0
+    buf = torch.full((d.q.shape[0] + 2,) + tuple(d.q.shape[1:]), guard, dtype=d.q.dtype, device="cuda")
+    out = buf[1:-1]
+    out.fill_(float("nan"))
     c = ctx()
     p = c.params_for(d.q, d.k_pages, d.block_table, max_q, scale, flags=flags)
     c.attn(d.q, d.k_pages, d.v_pages, d.block_table, d.seq_lens, d.q_lens, max_q, out=out, params=p)
     bits = c.poll_status()
+    assert bool((buf[0] == guard).all()) and bool((buf[-1] == guard).all()), "a row outside `out` was written"
     return out.double().cpu().numpy(), bits
+
+
+def guard_zones():
+    """(overwritten, checked) guard bytes of the shared context; (0, 0) unless the bounds-check build is loaded."""
+    return _ctx.guard_zones() if _ctx is not None else (0, 0)
 
 
 def oracle_attn(inp, scale=0.0):

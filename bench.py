@@ -375,6 +375,7 @@ def run_ours(args):
                                                  us2, peak, peak_kind),
                         "note": "the same calls without ARB_ATTN_OVERLAP_PREVIOUS: every call waits for the one "
                                 "before it, which is what a token of Algorithm 1 sees"}
+                result["decode_step"] = run_decode_step(ctx, dev, peak, peak_kind)
                 result["target_shaped_decode"] = run_target_decode(ctx, dev, peak)
                 result["step_scoring"] = run_step_scoring(ctx, dev)
                 result["mixed_loop"] = run_mixed_loop(ctx, dev)
@@ -383,6 +384,7 @@ def run_ours(args):
                 result["kv_append"] = run_kv_append(ctx, dev, peak)
                 result["policies"] = run_policies(ctx, dev)
                 result["e4m3_decode"] = run_e4m3_decode(ctx, dev, peak)
+                result["e4m3_chunk"] = run_e4m3_chunk(ctx, dev)
             result["cpu_baseline"] = run_cpu_baseline(work)
     if dist:
         dist.barrier()
@@ -490,6 +492,67 @@ def run_target_decode(ctx, dev, peak):
             "roofline": hbm_roofline("decode kernel, target-shaped", work.bytes["total"], us, peak, measured_peak()[1]),
             "back_to_back": {"us_per_call": round(us2, 2), "gbs": round(gbs2, 1), "frac_of_measured": round(gbs2 / peak, 4),
                              "pct_of_nominal_8TBs": round(100 * gbs2 / NOMINAL_HBM_GBS, 2)}}
+
+
+def run_decode_step(ctx, dev, peak, peak_kind, layers=LAYERS):
+    """Supplementary: the single-launch decode token (arb_decode_step: cache write + attention + combine + length
+    update) on the draft-shaped batch: `layers` calls per CUDA graph, each on its own KV pool and its own length
+    array (a layer's cache grows by one token per replay), every call waiting for the one before it."""
+    shape = wl.DRAFT_DECODE
+    inp = wl.make_attn_inputs(shape, device=dev, seed=shape.seed, extra_tokens=2048)
+    pools = [(inp.k_pages, inp.v_pages)] + [wl.make_kv_pool(shape, inp.num_pages, dev, shape.seed * 100 + l) for l in range(1, layers)]
+    lens = [inp.seq_lens.clone() for _ in pools]
+    k_new = wl.normal((shape.batch, shape.num_kv_heads, shape.head_dim), 1.0, shape.dtype, dev, 4401)
+    v_new = wl.normal((shape.batch, shape.num_kv_heads, shape.head_dim), 1.0, shape.dtype, dev, 4402)
+    out = torch.empty_like(inp.q)
+    p = ctx.params_for(inp.q, inp.k_pages, inp.block_table, 1)
+
+    def step():
+        for (k, v), sl in zip(pools, lens):
+            ctx.decode_step(inp.q, k_new, v_new, k, v, inp.block_table, sl, inp.q_lens, out=out, params=p)
+
+    step()
+    torch.cuda.synchronize()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g):
+        step()
+    ms = statistics.median(time_repeated(g.replay, 20, 5, min_total_ms=60.0)) / 20   # about 600 tokens appended per layer
+    us = ms / layers * 1e3
+    b = attn_bytes(shape, inp.seq_lens.cpu().to(torch.int64) + 300, inp.q_lens.cpu().to(torch.int64))
+    nbytes = b["total"] + 4 * shape.batch * shape.num_kv_heads * shape.head_dim * 2   # + the new rows, read and written
+    assert ctx.poll_status() == 0
+    return {"us_per_call": round(us, 3), "kv_tokens": b["tokens"],
+            "roofline": hbm_roofline("decode_step_kernel", nbytes, us, peak, peak_kind),
+            "note": f"{layers} arb_decode_step calls per CUDA graph, none overlapped: what a token of Algorithm 1 costs per layer"}
+
+
+def run_e4m3_chunk(ctx, dev):
+    """Supplementary: step chunks over an E4M3 cache (arb_attn_e4m3) on the step-scoring batch, pools of random codes."""
+    shape = wl.STEP_SCORING
+    inp = wl.make_attn_inputs(shape, device=dev, seed=shape.seed)
+    g8 = torch.Generator(device=dev)
+    g8.manual_seed(3100)
+    kc = torch.randint(0, 0x7f, inp.k_pages.shape, generator=g8, device=dev, dtype=torch.uint8)
+    vc = torch.randint(0, 0x7f, inp.k_pages.shape, generator=g8, device=dev, dtype=torch.uint8)
+    out = torch.empty_like(inp.q)
+    max_q = int(inp.q_lens.max())
+    fn = lambda: ctx.attn_e4m3(inp.q, kc, vc, 0.01, 0.01, inp.block_table, inp.seq_lens, inp.q_lens, max_q, out=out)
+    us = statistics.median(time_repeated(fn, 10, 3, min_total_ms=40.0)) / 10 * 1e3
+    sl, ql = inp.seq_lens.cpu().to(torch.int64), inp.q_lens.cpu().to(torch.int64)
+    b = attn_bytes(shape, sl, ql)
+    nbytes = b["kv"] // 2 + b["qo"] + b["table"]
+    flops = int((4 * ql * shape.num_q_heads * shape.head_dim * sl).sum())
+    burst, sustained, kind = measured_tensor_peaks()
+    hbm_peak, _ = measured_peak()
+    t_tensor, t_hbm = flops / (sustained * 1e12) * 1e6, nbytes / (hbm_peak * 1e9) * 1e6
+    tflops = flops / (us * 1e-6) / 1e12
+    return {"us_per_call": round(us, 2),
+            "roofline": {"bound": "tensor" if t_tensor >= t_hbm else "hbm", "kernel": "chunk_mma_kernel<E4M3>",
+                         "achieved": round(tflops, 1), "peak": sustained,
+                         "peak_kind": f"of {kind} (sustained bf16; f16 operands run at the same rate)", "unit": "TFLOP/s",
+                         "frac": round(max(t_tensor, t_hbm) / us, 4), "traffic": None,
+                         "algorithmic_flops_per_launch": flops, "algorithmic_bytes_per_launch": nbytes,
+                         "avg_launch_us": round(us, 2), "roofline_us": {"tensor": round(t_tensor, 1), "hbm": round(t_hbm, 1)}}}
 
 
 def run_step_scoring(ctx, dev):
@@ -831,6 +894,8 @@ def main():
                          "rollback) and nothing else")
     ap.add_argument("--profile-e4m3", action="store_true",
                     help="for runs under ncu: a few calls of the E4M3 decode on both decode workloads and nothing else")
+    ap.add_argument("--profile-decode-step", action="store_true",
+                    help="for runs under ncu: a few arb_decode_step calls on the draft-shaped batch and nothing else")
     ap.add_argument("--profile-step-loop", action="store_true",
                     help="for runs under ncu: the step loop (rounds of Algorithm 1 over three caches) and nothing else")
     ap.add_argument("--profile", action="store_true",
@@ -844,6 +909,12 @@ def main():
         from paper_2512_05033_b200 import binding
         torch.cuda.set_device(0)
         print(json.dumps({"step_scoring": run_step_scoring(binding.Context(0), torch.device("cuda", 0))}), flush=True)
+    elif args.profile_decode_step:
+        from paper_2512_05033_b200 import binding
+        torch.cuda.set_device(0)
+        peak, kind = measured_peak()
+        print(json.dumps({"decode_step": run_decode_step(binding.Context(0), torch.device("cuda", 0), peak, kind, layers=8)}),
+              flush=True)
     elif args.profile_step_loop:
         from paper_2512_05033_b200 import binding
         torch.cuda.set_device(0)

@@ -53,7 +53,7 @@ constexpr int kTmaWarp = 8, kMmaWarp = 9, kVWarp = 10;   // warp 11 has no role
 constexpr int kHalfBytes = 128 * 128;      // [128 rows x 64 bf16]: one 128-byte-swizzled half tile
 constexpr int kTileBytes = 2 * kHalfBytes;  // [128 x 128] bf16
 constexpr int kBoxBytes = kPage * 128;      // one TMA box: 16 rows x 64 bf16
-constexpr int kStagePages = 4;              // E4M3: pages of codes in flight per operand
+constexpr int kStagePages = 6;              // E4M3: pages of codes in flight per operand
 constexpr int kCodePageBytes = kPage * kD;  // 2 KB: one (page, kv head) tile of codes
 constexpr uint32_t kTmemCols = 512;         // S of tile A: columns 0..127, S of B: 128..255, O of A: 256..383, O of B: 384..511
 constexpr uint32_t kOCol = 256;
@@ -118,7 +118,7 @@ constexpr size_t kSmemFixed = 1024 /*alignment*/ + 2 * kTileBytes /*Q of A, B*/ 
                               sizeof(Bars);
 
 constexpr size_t kCodeStageBytes = 2 * kStagePages * kCodePageBytes;   // E4M3: staging of both operands
-constexpr int kMaxBatchE4m3 = 512;   // the staging takes 16 KB of what the plan tables of a larger batch would need
+constexpr int kMaxBatchE4m3 = 320;   // the staging takes 24 KB of what the plan tables of a larger batch would need
 
 inline size_t mma_smem_bytes(int batch, bool e4m3 = false) {
     return kSmemFixed + (e4m3 ? kCodeStageBytes : 0) + sizeof(int) * (7 * (size_t)batch + 2);
@@ -606,10 +606,22 @@ chunk_mma_kernel(const MmaArgs a, const __grid_constant__ CUtensorMap k_map, con
                         mbar_wait(&cfull[sl], ph, abort, a.status);
                         const char *src = stg + sl * kCodePageBytes + r * 128;
                         char *dst = ring + s * kTileBytes + h * kHalfBytes + (p * kPage + r) * 128;
+                        // the codes come into registers first, so that the slot can be asked for again at once
+                        uint4 codes[4];
+#pragma unroll
+                        for (int c4 = 0; c4 < 4; ++c4)
+                            codes[c4] = *reinterpret_cast<const uint4 *>(src + (((4 * h + c4) ^ (r & 7)) << 4));
+                        fence_async_smem();   // the slot's next writer is the TMA unit
+                        __syncwarp();
+                        {
+                            const int ahead = p + kStagePages;   // the page that takes this slot
+                            const bool there = ahead < npages || (ahead >= kTilePages && ahead - kTilePages < np_next);
+                            if (there) ask(ahead, pc + kStagePages);
+                        }
                         if (ok) {
 #pragma unroll
                             for (int c4 = 0; c4 < 4; ++c4) {
-                                const uint4 cd = *reinterpret_cast<const uint4 *>(src + (((4 * h + c4) ^ (r & 7)) << 4));
+                                const uint4 cd = codes[c4];
                                 uint4 lo, hi;
                                 lo.x = e4m3x2_to_f16x2((uint16_t)cd.x); lo.y = e4m3x2_to_f16x2((uint16_t)(cd.x >> 16));
                                 lo.z = e4m3x2_to_f16x2((uint16_t)cd.y); lo.w = e4m3x2_to_f16x2((uint16_t)(cd.y >> 16));
@@ -619,12 +631,9 @@ chunk_mma_kernel(const MmaArgs a, const __grid_constant__ CUtensorMap k_map, con
                                 *reinterpret_cast<uint4 *>(dst + (((2 * c4 + 1) ^ (r & 7)) << 4)) = hi;
                             }
                         }
-                        fence_async_smem();   // the slot's next writer is the TMA unit; the stage's reader the tensor core
-                        __syncwarp();
-                        const int ahead = p + kStagePages;   // the page that takes this slot
-                        const bool there = ahead < npages || (ahead >= kTilePages && ahead - kTilePages < np_next);
-                        if (there) ask(ahead, pc + kStagePages);
                     }
+                    fence_async_smem();   // the stage's reader is the tensor core
+                    __syncwarp();
                     if (lane == 0) mbar_arrive(&full[s]);
                 } else {
                     if (lane == 0) ok = mbar_wait(&empty[s], par ^ 1u, abort, a.status);

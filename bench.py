@@ -393,6 +393,14 @@ def run_ours(args):
         print(json.dumps(result), flush=True)
 
 
+def decode_mma_source_hash() -> str:
+    """sha1 over the sources of the headline's dominant kernel (decode_mma_kernel and the header it shares)."""
+    h = hashlib.sha1()
+    for name in ("arb_decode_mma.cu", "arb_decode_tc.cuh"):
+        h.update((ROOT / "paper_2512_05033_b200" / "csrc" / name).read_bytes())
+    return h.hexdigest()
+
+
 def read_traffic_note():
     """DRAM bytes per decode launch from the committed ncu summary; null once the kernel source has
     changed since the counters were taken."""
@@ -400,8 +408,7 @@ def read_traffic_note():
     if not note.exists():
         return None
     kv = dict(l.split("=", 1) for l in note.read_text().splitlines() if "=" in l and not l.startswith("#"))
-    src = ROOT / "paper_2512_05033_b200" / "csrc" / "arb_decode_mma.cu"
-    if kv.get("source_sha1", "").strip() != hashlib.sha1(src.read_bytes()).hexdigest():
+    if kv.get("source_sha1", "").strip() != decode_mma_source_hash():
         return None
     try:
         return float(kv["dram_bytes_per_launch"])
@@ -894,6 +901,8 @@ def main():
                          "rollback) and nothing else")
     ap.add_argument("--profile-e4m3", action="store_true",
                     help="for runs under ncu: a few calls of the E4M3 decode on both decode workloads and nothing else")
+    ap.add_argument("--profile-e4m3-chunk", action="store_true",
+                    help="for runs under ncu: a few step-chunk calls over the E4M3 cache and nothing else")
     ap.add_argument("--profile-decode-step", action="store_true",
                     help="for runs under ncu: a few arb_decode_step calls on the draft-shaped batch and nothing else")
     ap.add_argument("--profile-step-loop", action="store_true",
@@ -909,6 +918,10 @@ def main():
         from paper_2512_05033_b200 import binding
         torch.cuda.set_device(0)
         print(json.dumps({"step_scoring": run_step_scoring(binding.Context(0), torch.device("cuda", 0))}), flush=True)
+    elif args.profile_e4m3_chunk:
+        from paper_2512_05033_b200 import binding
+        torch.cuda.set_device(0)
+        print(json.dumps({"e4m3_chunk": run_e4m3_chunk(binding.Context(0), torch.device("cuda", 0))}), flush=True)
     elif args.profile_decode_step:
         from paper_2512_05033_b200 import binding
         torch.cuda.set_device(0)

@@ -392,182 +392,291 @@ decode_mma_kernel(const Args a, const __grid_constant__ CUtensorMap k_map, const
 
     while (next_segment(cur, r1, pref, slen, B, Hkv, chunk, s)) {
         const int qrow = row0[s.b];
-        // A fragments of q (16 x 128, rows >= G zero): 8 k-slices of 16 dims.  E4M3 cache: converted to f16, and
-        // k-slice ks holds dims 16 ks .. 16 ks + 15 in the order the widened codes arrive in: this lane has dims
-        // 16 ks + 4 tq + {0, 1} (k = 2 tq, + 1) and + {2, 3} (k = 8 + 2 tq, + 1)
-        uint32_t qa[8][4];
-        {
-            const char *qh = a.q + ((size_t)qrow * a.Hq + s.kvh * G + gq) * kD * 2;
+        if constexpr (!E4M3) {
+            // ---- bf16 cache: the transposed products.  S^T = K q^T puts the 16 keys of a page on the rows of the
+            //      m16n8k16 tile and the group's heads (padded to 8) on its columns, O^T += V^T P^T likewise: 8 + 8
+            //      MMAs per page instead of 16 + 16 and half the accumulator registers.  P^T reaches the second
+            //      product's B fragment through two movmatrix transposes; the row maximum is a reduction over the
+            //      lanes that share a column pair (three shuffles).
+            const bool head_ok = gq < G;               // as a B-fragment column: this lane's head is a real one
+            const int h0 = 2 * tq, h1 = 2 * tq + 1;    // as accumulator columns: the two heads this lane holds
+            uint32_t qb[8][2];                         // k-slice ks: dims 16 ks + 2 tq, + 1 and + 8 of head gq
+            {
+                const char *qh = a.q + ((size_t)qrow * a.Hq + s.kvh * G + (head_ok ? gq : 0)) * kD * 2;
 #pragma unroll
-            for (int ks = 0; ks < 8; ++ks) {
-                if constexpr (E4M3) {
-                    const uint2 raw = row_ok ? __ldg(reinterpret_cast<const uint2 *>(qh + ks * 32 + tq * 8)) : make_uint2(0u, 0u);
-                    qa[ks][0] = pack_f16(__uint_as_float(raw.x << 16), __uint_as_float(raw.x & 0xffff0000u));
-                    qa[ks][2] = pack_f16(__uint_as_float(raw.y << 16), __uint_as_float(raw.y & 0xffff0000u));
-                } else {
-                    qa[ks][0] = row_ok ? __ldg(reinterpret_cast<const uint32_t *>(qh + ks * 32 + tq * 4)) : 0u;
-                    qa[ks][2] = row_ok ? __ldg(reinterpret_cast<const uint32_t *>(qh + ks * 32 + 16 + tq * 4)) : 0u;
+                for (int ks = 0; ks < 8; ++ks) {
+                    qb[ks][0] = head_ok ? __ldg(reinterpret_cast<const uint32_t *>(qh + ks * 32 + tq * 4)) : 0u;
+                    qb[ks][1] = head_ok ? __ldg(reinterpret_cast<const uint32_t *>(qh + ks * 32 + 16 + tq * 4)) : 0u;
                 }
-                qa[ks][1] = 0u;
-                qa[ks][3] = 0u;
             }
-        }
-        // this lane's row (head gq): running max (the same in the 4 lanes of a row), its share of the
-        // sum, and 16 n-tiles of the output row: o[n][0..1] = dims 8n + 2 tq, + 1 (o[n][2..3]: rows 8..15); with an E4M3
-        // cache o[2c][0..1] = dims 16c + 4 tq, + 2 and o[2c+1][0..1] = dims 16c + 4 tq + 1, + 3
-        float m_run = -INFINITY, l_run = 0.f;
-        float o[16][4];
+            // running max of heads h0, h1 (the same in the 8 lanes of a column pair), this lane's share of their sums,
+            // and 8 m-tiles of O^T: o[mt][0..1] = dim 16 mt + gq of heads h0, h1; o[mt][2..3] = dim + 8
+            float m_run0 = -INFINITY, m_run1 = -INFINITY, l_run0 = 0.f, l_run1 = 0.f;
+            float o[8][4];
 #pragma unroll
-        for (int n = 0; n < 16; ++n) { o[n][0] = o[n][1] = o[n][2] = o[n][3] = 0.f; }
-
-        const int seg_pages = s.pg1 - s.pg0;
-        const int ngroups = (seg_pages + kGroup - 1) / kGroup;
-        for (int gi = warp; gi < ngroups; gi += kCW) {
-            const int p0 = s.pg0 + gi * kGroup;
-            const int npg = min(kGroup, s.pg1 - p0);
-            const int ntok = min(s.L - p0 * kPage, npg * kPage);
-            const uint32_t gbase = seg_base + (uint32_t)gi * 2 * kGroup;
-
-            // ---- S = q K^T for the group's pages: per page two n-tiles of 8 keys -----------------
-            float sc[kGroup * 2][4];
-#pragma unroll
-            for (int t = 0; t < kGroup; ++t) {
-#pragma unroll
-                for (int j = 0; j < 2; ++j) { sc[t * 2 + j][0] = sc[t * 2 + j][1] = sc[t * 2 + j][2] = sc[t * 2 + j][3] = 0.f; }
-                if (t < npg) {
-                    const uint32_t cc = gbase + t, st = cc % kStages, par = (cc / kStages) & 1u;
+            for (int mt = 0; mt < 8; ++mt) { o[mt][0] = o[mt][1] = o[mt][2] = o[mt][3] = 0.f; }
+            const int seg_pages = s.pg1 - s.pg0;
+            for (int gi = warp; gi < seg_pages; gi += kCW) {
+                const int pg = s.pg0 + gi;
+                const int ntok = min(s.L - pg * kPage, kPage);
+                const uint32_t ck = seg_base + 2u * (uint32_t)gi;
+                float sa[4] = {0.f, 0.f, 0.f, 0.f}, sb[4] = {0.f, 0.f, 0.f, 0.f};   // two chains, four deep
+                {
+                    const uint32_t st = ck % kStages, par = (ck / kStages) & 1u;
                     mbar_wait(&tail->full[st], par, abort, a.status);
                     const uint32_t tile = ring_addr + st * kTileBytes;
 #pragma unroll
-                    for (int j = 0; j < 2; ++j) {          // keys 8j .. 8j+7 of the page
-                        if constexpr (E4M3) {
-#pragma unroll
-                            for (int kq = 0; kq < 2; ++kq) {   // k-slices 4kq .. 4kq + 3: one 16-byte chunk of codes each
-                                uint32_t bfr[4];
-                                ldmatrix_x4(tile + tile_off<true>(8 * j + (lane & 7), 4 * kq + (lane >> 3)), bfr);
-#pragma unroll
-                                for (int i = 0; i < 4; ++i)
-                                    mma_16816<true>(sc[t * 2 + j], qa[4 * kq + i], e4m3x2_to_f16x2(bfr[i]),
-                                                    e4m3x2_to_f16x2(bfr[i] >> 16));
-                            }
-                        } else {
-#pragma unroll
-                            for (int kp = 0; kp < 4; ++kp) {   // k-slices 2kp, 2kp+1
-                                uint32_t bfr[4];
-                                ldmatrix_x4(tile + tile_off<false>(8 * j + (lane & 7), 4 * kp + (lane >> 3)), bfr);
-                                mma_16816<false>(sc[t * 2 + j], qa[2 * kp], bfr[0], bfr[1]);
-                                mma_16816<false>(sc[t * 2 + j], qa[2 * kp + 1], bfr[2], bfr[3]);
-                            }
-                        }
+                    for (int ks = 0; ks < 8; ++ks) {
+                        uint32_t af[4];   // rows: keys; matrices: (keys 0-7 | 8-15) x (dims 16 ks + 0-7 | 8-15)
+                        ldmatrix_x4(tile + tile_off<false>((lane & 7) + ((lane >> 3) & 1) * 8, 2 * ks + (lane >> 4)), af);
+                        if (ks & 1) mma_16816<false>(sb, af, qb[ks][0], qb[ks][1]);
+                        else mma_16816<false>(sa, af, qb[ks][0], qb[ks][1]);
                     }
                     __syncwarp();
                     if (lane == 0) mbar_arrive(&tail->empty[st]);
                 }
-            }
-
-            // ---- online softmax on the fragments: this lane has 2 scores per n-tile of its row ------
-            float mx = -INFINITY;
+                const bool k0 = gq < ntok, k1 = gq + 8 < ntok;   // this lane has keys gq and gq + 8
+                const float s00 = k0 ? (sa[0] + sb[0]) * a.scale_log2 : -INFINITY;
+                const float s01 = k0 ? (sa[1] + sb[1]) * a.scale_log2 : -INFINITY;
+                const float s10 = k1 ? (sa[2] + sb[2]) * a.scale_log2 : -INFINITY;
+                const float s11 = k1 ? (sa[3] + sb[3]) * a.scale_log2 : -INFINITY;
+                float mx0 = fmaxf(s00, s10), mx1 = fmaxf(s01, s11);
 #pragma unroll
-            for (int nt = 0; nt < kGroup * 2; ++nt) {
-#pragma unroll
-                for (int e = 0; e < 2; ++e) {
-                    const int key = nt * 8 + tq * 2 + e;
-                    const float v = (key < ntok) ? sc[nt][e] * a.scale_log2 : -INFINITY;
-                    sc[nt][e] = v;
-                    mx = fmaxf(mx, v);
+                for (int off = 4; off < 32; off <<= 1) {
+                    mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, off));
+                    mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, off));
                 }
-            }
-            mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
-            mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
-            const float m_new = fmaxf(m_run, mx);            // finite: the group has a visible key
-            const float f = fast_exp2(m_run - m_new);        // 0 for the first group
-            m_run = m_new;
-            uint32_t pa[kGroup][4];                          // A fragments of P: one k-slice per page
-            float lsum = 0.f;
+                const float mn0 = fmaxf(m_run0, mx0), mn1 = fmaxf(m_run1, mx1);   // finite: key 0 of the page is visible
+                const float f0 = fast_exp2(m_run0 - mn0), f1 = fast_exp2(m_run1 - mn1);
+                m_run0 = mn0;
+                m_run1 = mn1;
+                // P^T, rounded to bf16; the sums use the rounded weights, like the tensor core
+                const uint32_t w0 = pack_bf16(fast_exp2(s00 - mn0), fast_exp2(s01 - mn1));   // key gq: heads h0, h1
+                const uint32_t w1 = pack_bf16(fast_exp2(s10 - mn0), fast_exp2(s11 - mn1));   // key gq + 8
+                l_run0 = fmaf(l_run0, f0, __uint_as_float(w0 << 16) + __uint_as_float(w1 << 16));
+                l_run1 = fmaf(l_run1, f1, __uint_as_float(w0 & 0xffff0000u) + __uint_as_float(w1 & 0xffff0000u));
+                const uint32_t pb0 = movmatrix_trans(w0), pb1 = movmatrix_trans(w1);   // keys 2 tq, + 1 (and + 8) of head gq
+                if (__any_sync(0xffffffffu, f0 != 1.0f || f1 != 1.0f)) {
 #pragma unroll
-            for (int t = 0; t < kGroup; ++t) {
-                const float p00 = fast_exp2(sc[2 * t][0] - m_new), p01 = fast_exp2(sc[2 * t][1] - m_new);
-                const float p10 = fast_exp2(sc[2 * t + 1][0] - m_new), p11 = fast_exp2(sc[2 * t + 1][1] - m_new);
-                const uint32_t w0 = E4M3 ? pack_f16(p00, p01) : pack_bf16(p00, p01);
-                const uint32_t w1 = E4M3 ? pack_f16(p10, p11) : pack_bf16(p10, p11);
-                pa[t][0] = w0;   // row gq, keys 2 tq, +1
-                pa[t][2] = w1;   // row gq, keys 8 + 2 tq, +1
-                pa[t][1] = 0u;   // rows 8..15
-                pa[t][3] = 0u;
-                // the sum uses the rounded weights, like the tensor core
-                if constexpr (E4M3) {
-                    const float2 r0 = unpack_f16(w0), r1 = unpack_f16(w1);
-                    lsum += (r0.x + r0.y) + (r1.x + r1.y);
-                } else {
-                    lsum += __uint_as_float(w0 << 16) + __uint_as_float(w0 & 0xffff0000u) +
-                            __uint_as_float(w1 << 16) + __uint_as_float(w1 & 0xffff0000u);
+                    for (int mt = 0; mt < 8; ++mt) { o[mt][0] *= f0; o[mt][1] *= f1; o[mt][2] *= f0; o[mt][3] *= f1; }
                 }
-            }
-            l_run = fmaf(l_run, f, lsum);
-            if (__any_sync(0xffffffffu, f != 1.0f)) {
-#pragma unroll
-                for (int n = 0; n < 16; ++n) { o[n][0] *= f; o[n][1] *= f; }
-            }
-
-            // ---- O += P V: per page 16 n-tiles of 8 dims, one k-slice of 16 keys ------------------
-#pragma unroll
-            for (int t = 0; t < kGroup; ++t) {
-                if (t < npg) {
-                    const uint32_t cc = gbase + npg + t, st = cc % kStages, par = (cc / kStages) & 1u;
+                {
+                    const uint32_t cv = ck + 1u, st = cv % kStages, par = (cv / kStages) & 1u;
                     mbar_wait(&tail->full[st], par, abort, a.status);
-                    const uint32_t tile = ring_addr + st * kTileBytes;
-                    const int nvalid = ntok - t * kPage;
-                    if (nvalid < kPage) {
-                        // slots past the sequence end may hold anything; they must not reach the
-                        // tensor core, not even times zero: blank them in shared memory
-                        constexpr int kRowChunks = kTileBytes / kPage / 16;   // 16-byte chunks of a row: 16 or 8
-                        for (int i = lane; i < (kPage - nvalid) * kRowChunks; i += 32) {
-                            const int r = nvalid + i / kRowChunks, c = i % kRowChunks;
-                            *reinterpret_cast<uint4 *>(ring + st * kTileBytes + tile_off<E4M3>(r, c)) = make_uint4(0, 0, 0, 0);
-                        }
+                    if (ntok < kPage) {
+                        // slots past the sequence end may hold anything; they must not reach the tensor core, not
+                        // even times zero: blank them in shared memory
+                        for (int i = lane; i < (kPage - ntok) * 16; i += 32)
+                            *reinterpret_cast<uint4 *>(ring + st * kTileBytes + tile_off<false>(ntok + (i >> 4), i & 15)) = make_uint4(0, 0, 0, 0);
                         __syncwarp();
                     }
+                    const uint32_t tile = ring_addr + st * kTileBytes;
 #pragma unroll
-                    for (int np2 = 0; np2 < (E4M3 ? 4 : 8); ++np2) {    // two 16-byte chunks of a row: 16 dims, or 32 dims of codes
-                        uint32_t bfr[4];
-                        // blocks: (keys 0-7, chunk 2np2), (keys 8-15, 2np2), (keys 0-7, 2np2+1), (keys 8-15, 2np2+1)
-                        ldmatrix_x4_trans(tile + tile_off<E4M3>((lane & 7) + ((lane >> 3) & 1) * 8, 2 * np2 + (lane >> 4)), bfr);
-                        if constexpr (E4M3) {
-                            // a lane has (key 2tq: dims d, d+1 | key 2tq+1: dims d, d+1) with d = 16 chunk + 2 gq
-#pragma unroll
-                            for (int h = 0; h < 2; ++h) {      // chunk 2np2 + h
-                                // bytes -> (key 2tq, key 2tq+1) of dim d | the same of dim d + 1
-                                const uint32_t lo = byte_perm(bfr[2 * h], 0x3120u), hi = byte_perm(bfr[2 * h + 1], 0x3120u);
-                                mma_16816<true>(o[4 * np2 + 2 * h], pa[t], e4m3x2_to_f16x2(lo), e4m3x2_to_f16x2(hi));
-                                mma_16816<true>(o[4 * np2 + 2 * h + 1], pa[t], e4m3x2_to_f16x2(lo >> 16), e4m3x2_to_f16x2(hi >> 16));
-                            }
-                        } else {
-                            mma_16816<false>(o[2 * np2], pa[t], bfr[0], bfr[1]);
-                            mma_16816<false>(o[2 * np2 + 1], pa[t], bfr[2], bfr[3]);
-                        }
+                    for (int mt = 0; mt < 8; ++mt) {
+                        uint32_t af[4];   // transposed on the way: rows dims (16 mt + 0-7 | 8-15), columns keys (0-7 | 8-15)
+                        ldmatrix_x4_trans(tile + tile_off<false>((lane & 7) + (lane >> 4) * 8, 2 * mt + ((lane >> 3) & 1)), af);
+                        mma_16816<false>(o[mt], af, pb0, pb1);
                     }
                     __syncwarp();
                     if (lane == 0) mbar_arrive(&tail->empty[st]);
                 }
             }
-        }
-        seg_base += 2u * (uint32_t)seg_pages;
-
-        // ---- segment end: every warp leaves (max, sum, row accumulators); all threads merge them ------
-        l_run += __shfl_xor_sync(0xffffffffu, l_run, 1);
-        l_run += __shfl_xor_sync(0xffffffffu, l_run, 2);
-        float *rec = osm + warp * REC;
-        if (row_ok) {
+            seg_base += 2u * (uint32_t)seg_pages;
+            // ---- segment end: every warp leaves (max, sum, accumulators) in the record layout the merge reads
 #pragma unroll
-            if constexpr (E4M3) {
-                for (int c = 0; c < 8; ++c)   // four consecutive dims per 16-dim group
-                    *reinterpret_cast<float4 *>(rec + 2 * GP + gq * kD + 16 * c + 4 * tq) =
-                        make_float4(o[2 * c][0], o[2 * c + 1][0], o[2 * c][1], o[2 * c + 1][1]);
-            } else {
-                for (int n = 0; n < 16; ++n)
-                    *reinterpret_cast<float2 *>(rec + 2 * GP + gq * kD + 8 * n + tq * 2) = make_float2(o[n][0], o[n][1]);
+            for (int off = 4; off < 32; off <<= 1) {
+                l_run0 += __shfl_xor_sync(0xffffffffu, l_run0, off);
+                l_run1 += __shfl_xor_sync(0xffffffffu, l_run1, off);
             }
-            if (tq == 0) { rec[gq] = m_run; rec[GP + gq] = l_run; }
+            float *rec = osm + warp * REC;
+            if (gq == 0) {
+                if (h0 < G) { rec[h0] = m_run0; rec[GP + h0] = l_run0; }
+                if (h1 < G) { rec[h1] = m_run1; rec[GP + h1] = l_run1; }
+            }
+#pragma unroll
+            for (int mt = 0; mt < 8; ++mt) {
+                const int d = 16 * mt + gq;
+                if (h0 < G) { rec[2 * GP + h0 * kD + d] = o[mt][0]; rec[2 * GP + h0 * kD + d + 8] = o[mt][2]; }
+                if (h1 < G) { rec[2 * GP + h1 * kD + d] = o[mt][1]; rec[2 * GP + h1 * kD + d + 8] = o[mt][3]; }
+            }
+        } else {
+            // A fragments of q (16 x 128, rows >= G zero): 8 k-slices of 16 dims.  E4M3 cache: converted to f16, and
+            // k-slice ks holds dims 16 ks .. 16 ks + 15 in the order the widened codes arrive in: this lane has dims
+            // 16 ks + 4 tq + {0, 1} (k = 2 tq, + 1) and + {2, 3} (k = 8 + 2 tq, + 1)
+            uint32_t qa[8][4];
+            {
+                const char *qh = a.q + ((size_t)qrow * a.Hq + s.kvh * G + gq) * kD * 2;
+    #pragma unroll
+                for (int ks = 0; ks < 8; ++ks) {
+                    if constexpr (E4M3) {
+                        const uint2 raw = row_ok ? __ldg(reinterpret_cast<const uint2 *>(qh + ks * 32 + tq * 8)) : make_uint2(0u, 0u);
+                        qa[ks][0] = pack_f16(__uint_as_float(raw.x << 16), __uint_as_float(raw.x & 0xffff0000u));
+                        qa[ks][2] = pack_f16(__uint_as_float(raw.y << 16), __uint_as_float(raw.y & 0xffff0000u));
+                    } else {
+                        qa[ks][0] = row_ok ? __ldg(reinterpret_cast<const uint32_t *>(qh + ks * 32 + tq * 4)) : 0u;
+                        qa[ks][2] = row_ok ? __ldg(reinterpret_cast<const uint32_t *>(qh + ks * 32 + 16 + tq * 4)) : 0u;
+                    }
+                    qa[ks][1] = 0u;
+                    qa[ks][3] = 0u;
+                }
+            }
+            // this lane's row (head gq): running max (the same in the 4 lanes of a row), its share of the
+            // sum, and 16 n-tiles of the output row: o[n][0..1] = dims 8n + 2 tq, + 1 (o[n][2..3]: rows 8..15); with an E4M3
+            // cache o[2c][0..1] = dims 16c + 4 tq, + 2 and o[2c+1][0..1] = dims 16c + 4 tq + 1, + 3
+            float m_run = -INFINITY, l_run = 0.f;
+            float o[16][4];
+    #pragma unroll
+            for (int n = 0; n < 16; ++n) { o[n][0] = o[n][1] = o[n][2] = o[n][3] = 0.f; }
+
+            const int seg_pages = s.pg1 - s.pg0;
+            const int ngroups = (seg_pages + kGroup - 1) / kGroup;
+            for (int gi = warp; gi < ngroups; gi += kCW) {
+                const int p0 = s.pg0 + gi * kGroup;
+                const int npg = min(kGroup, s.pg1 - p0);
+                const int ntok = min(s.L - p0 * kPage, npg * kPage);
+                const uint32_t gbase = seg_base + (uint32_t)gi * 2 * kGroup;
+
+                // ---- S = q K^T for the group's pages: per page two n-tiles of 8 keys -----------------
+                float sc[kGroup * 2][4];
+    #pragma unroll
+                for (int t = 0; t < kGroup; ++t) {
+    #pragma unroll
+                    for (int j = 0; j < 2; ++j) { sc[t * 2 + j][0] = sc[t * 2 + j][1] = sc[t * 2 + j][2] = sc[t * 2 + j][3] = 0.f; }
+                    if (t < npg) {
+                        const uint32_t cc = gbase + t, st = cc % kStages, par = (cc / kStages) & 1u;
+                        mbar_wait(&tail->full[st], par, abort, a.status);
+                        const uint32_t tile = ring_addr + st * kTileBytes;
+    #pragma unroll
+                        for (int j = 0; j < 2; ++j) {          // keys 8j .. 8j+7 of the page
+                            if constexpr (E4M3) {
+    #pragma unroll
+                                for (int kq = 0; kq < 2; ++kq) {   // k-slices 4kq .. 4kq + 3: one 16-byte chunk of codes each
+                                    uint32_t bfr[4];
+                                    ldmatrix_x4(tile + tile_off<true>(8 * j + (lane & 7), 4 * kq + (lane >> 3)), bfr);
+    #pragma unroll
+                                    for (int i = 0; i < 4; ++i)
+                                        mma_16816<true>(sc[t * 2 + j], qa[4 * kq + i], e4m3x2_to_f16x2(bfr[i]),
+                                                        e4m3x2_to_f16x2(bfr[i] >> 16));
+                                }
+                            } else {
+    #pragma unroll
+                                for (int kp = 0; kp < 4; ++kp) {   // k-slices 2kp, 2kp+1
+                                    uint32_t bfr[4];
+                                    ldmatrix_x4(tile + tile_off<false>(8 * j + (lane & 7), 4 * kp + (lane >> 3)), bfr);
+                                    mma_16816<false>(sc[t * 2 + j], qa[2 * kp], bfr[0], bfr[1]);
+                                    mma_16816<false>(sc[t * 2 + j], qa[2 * kp + 1], bfr[2], bfr[3]);
+                                }
+                            }
+                        }
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(&tail->empty[st]);
+                    }
+                }
+
+                // ---- online softmax on the fragments: this lane has 2 scores per n-tile of its row ------
+                float mx = -INFINITY;
+    #pragma unroll
+                for (int nt = 0; nt < kGroup * 2; ++nt) {
+    #pragma unroll
+                    for (int e = 0; e < 2; ++e) {
+                        const int key = nt * 8 + tq * 2 + e;
+                        const float v = (key < ntok) ? sc[nt][e] * a.scale_log2 : -INFINITY;
+                        sc[nt][e] = v;
+                        mx = fmaxf(mx, v);
+                    }
+                }
+                mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
+                mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
+                const float m_new = fmaxf(m_run, mx);            // finite: the group has a visible key
+                const float f = fast_exp2(m_run - m_new);        // 0 for the first group
+                m_run = m_new;
+                uint32_t pa[kGroup][4];                          // A fragments of P: one k-slice per page
+                float lsum = 0.f;
+    #pragma unroll
+                for (int t = 0; t < kGroup; ++t) {
+                    const float p00 = fast_exp2(sc[2 * t][0] - m_new), p01 = fast_exp2(sc[2 * t][1] - m_new);
+                    const float p10 = fast_exp2(sc[2 * t + 1][0] - m_new), p11 = fast_exp2(sc[2 * t + 1][1] - m_new);
+                    const uint32_t w0 = E4M3 ? pack_f16(p00, p01) : pack_bf16(p00, p01);
+                    const uint32_t w1 = E4M3 ? pack_f16(p10, p11) : pack_bf16(p10, p11);
+                    pa[t][0] = w0;   // row gq, keys 2 tq, +1
+                    pa[t][2] = w1;   // row gq, keys 8 + 2 tq, +1
+                    pa[t][1] = 0u;   // rows 8..15
+                    pa[t][3] = 0u;
+                    // the sum uses the rounded weights, like the tensor core
+                    if constexpr (E4M3) {
+                        const float2 r0 = unpack_f16(w0), r1 = unpack_f16(w1);
+                        lsum += (r0.x + r0.y) + (r1.x + r1.y);
+                    } else {
+                        lsum += __uint_as_float(w0 << 16) + __uint_as_float(w0 & 0xffff0000u) +
+                                __uint_as_float(w1 << 16) + __uint_as_float(w1 & 0xffff0000u);
+                    }
+                }
+                l_run = fmaf(l_run, f, lsum);
+                if (__any_sync(0xffffffffu, f != 1.0f)) {
+    #pragma unroll
+                    for (int n = 0; n < 16; ++n) { o[n][0] *= f; o[n][1] *= f; }
+                }
+
+                // ---- O += P V: per page 16 n-tiles of 8 dims, one k-slice of 16 keys ------------------
+    #pragma unroll
+                for (int t = 0; t < kGroup; ++t) {
+                    if (t < npg) {
+                        const uint32_t cc = gbase + npg + t, st = cc % kStages, par = (cc / kStages) & 1u;
+                        mbar_wait(&tail->full[st], par, abort, a.status);
+                        const uint32_t tile = ring_addr + st * kTileBytes;
+                        const int nvalid = ntok - t * kPage;
+                        if (nvalid < kPage) {
+                            // slots past the sequence end may hold anything; they must not reach the
+                            // tensor core, not even times zero: blank them in shared memory
+                            constexpr int kRowChunks = kTileBytes / kPage / 16;   // 16-byte chunks of a row: 16 or 8
+                            for (int i = lane; i < (kPage - nvalid) * kRowChunks; i += 32) {
+                                const int r = nvalid + i / kRowChunks, c = i % kRowChunks;
+                                *reinterpret_cast<uint4 *>(ring + st * kTileBytes + tile_off<E4M3>(r, c)) = make_uint4(0, 0, 0, 0);
+                            }
+                            __syncwarp();
+                        }
+    #pragma unroll
+                        for (int np2 = 0; np2 < (E4M3 ? 4 : 8); ++np2) {    // two 16-byte chunks of a row: 16 dims, or 32 dims of codes
+                            uint32_t bfr[4];
+                            // blocks: (keys 0-7, chunk 2np2), (keys 8-15, 2np2), (keys 0-7, 2np2+1), (keys 8-15, 2np2+1)
+                            ldmatrix_x4_trans(tile + tile_off<E4M3>((lane & 7) + ((lane >> 3) & 1) * 8, 2 * np2 + (lane >> 4)), bfr);
+                            if constexpr (E4M3) {
+                                // a lane has (key 2tq: dims d, d+1 | key 2tq+1: dims d, d+1) with d = 16 chunk + 2 gq
+    #pragma unroll
+                                for (int h = 0; h < 2; ++h) {      // chunk 2np2 + h
+                                    // bytes -> (key 2tq, key 2tq+1) of dim d | the same of dim d + 1
+                                    const uint32_t lo = byte_perm(bfr[2 * h], 0x3120u), hi = byte_perm(bfr[2 * h + 1], 0x3120u);
+                                    mma_16816<true>(o[4 * np2 + 2 * h], pa[t], e4m3x2_to_f16x2(lo), e4m3x2_to_f16x2(hi));
+                                    mma_16816<true>(o[4 * np2 + 2 * h + 1], pa[t], e4m3x2_to_f16x2(lo >> 16), e4m3x2_to_f16x2(hi >> 16));
+                                }
+                            } else {
+                                mma_16816<false>(o[2 * np2], pa[t], bfr[0], bfr[1]);
+                                mma_16816<false>(o[2 * np2 + 1], pa[t], bfr[2], bfr[3]);
+                            }
+                        }
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(&tail->empty[st]);
+                    }
+                }
+            }
+            seg_base += 2u * (uint32_t)seg_pages;
+
+            // ---- segment end: every warp leaves (max, sum, row accumulators); all threads merge them ------
+            l_run += __shfl_xor_sync(0xffffffffu, l_run, 1);
+            l_run += __shfl_xor_sync(0xffffffffu, l_run, 2);
+            float *rec = osm + warp * REC;
+            if (row_ok) {
+    #pragma unroll
+                if constexpr (E4M3) {
+                    for (int c = 0; c < 8; ++c)   // four consecutive dims per 16-dim group
+                        *reinterpret_cast<float4 *>(rec + 2 * GP + gq * kD + 16 * c + 4 * tq) =
+                            make_float4(o[2 * c][0], o[2 * c + 1][0], o[2 * c][1], o[2 * c + 1][1]);
+                } else {
+                    for (int n = 0; n < 16; ++n)
+                        *reinterpret_cast<float2 *>(rec + 2 * GP + gq * kD + 8 * n + tq * 2) = make_float2(o[n][0], o[n][1]);
+                }
+                if (tq == 0) { rec[gq] = m_run; rec[GP + gq] = l_run; }
+            }
         }
         if (n_parked == kParked) flush(false);  // uniform across the consumer threads
         named_barrier(1, kCT);

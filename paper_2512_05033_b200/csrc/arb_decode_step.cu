@@ -105,13 +105,6 @@ __device__ __forceinline__ uint32_t tile_off(int r, int c) {   // 16-byte chunk 
     return (uint32_t)((c >> 3) * kHalfTile + r * 128 + (((c & 7) ^ (r & 7)) << 4));
 }
 
-// transposes an 8 x 8 matrix of 16-bit elements held one row per four lanes, two elements per lane
-__device__ __forceinline__ uint32_t movmatrix_trans(uint32_t v) {
-    uint32_t r;
-    asm volatile("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;" : "=r"(r) : "r"(v));
-    return r;
-}
-
 __device__ __forceinline__ void fence_proxy_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 
 // A sequence takes part when it decodes (q_len 1) and its length after the token fits the block table.

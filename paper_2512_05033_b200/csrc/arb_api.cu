@@ -152,6 +152,8 @@ arb_status arb_create(arb_ctx **out, int device, size_t workspace_bytes) {
     ok = ok && guarded_malloc(c, &c->spearman_acc, 4 * sizeof(double));
     c->chunk_ws_bytes = 2 * c->workspace_bytes;   // partials of long step chunks that are split over their keys
     ok = ok && guarded_malloc(c, &c->chunk_ws, c->chunk_ws_bytes);
+    ok = ok && guarded_malloc(c, &c->step_hint, decode_step_hint_bytes(sms));
+    ok = ok && cudaMemset(c->step_hint, 0, decode_step_hint_bytes(sms)) == cudaSuccess;
     if (ok && c->n_guards > 0) {
         ok = cudaMalloc(&c->guards_dev, sizeof(c->guards)) == cudaSuccess &&
              cudaMalloc(&c->guard_bad, sizeof(unsigned long long)) == cudaSuccess &&
@@ -168,6 +170,7 @@ arb_status arb_create(arb_ctx **out, int device, size_t workspace_bytes) {
         guarded_free(c->rot);
         guarded_free(c->spearman_acc);
         guarded_free(c->chunk_ws);
+        guarded_free(c->step_hint);
         cudaFree(c->guards_dev);
         cudaFree(c->guard_bad);
         delete c;
@@ -188,6 +191,7 @@ arb_status arb_destroy(arb_ctx *ctx) {
     guarded_free(c->rot);
     guarded_free(c->spearman_acc);
     guarded_free(c->chunk_ws);
+    guarded_free(c->step_hint);
     cudaFree(c->guards_dev);
     cudaFree(c->guard_bad);
     cudaFree(c->stage);

@@ -63,6 +63,7 @@ struct Ctx {
     uint32_t decode_gen = 1000;          // generation of the next tensor-core decode call
     uint32_t rot_wait_through = 0;        // tensor-core decode calls up to this generation wait for their predecessor
     double *spearman_acc = nullptr;       // three fp64 accumulators of arb_spearman
+    int *step_hint = nullptr;             // single-launch decode: the page tiles each CTA streamed last (arb_decode_step.cu)
     int step_min_chunk = 16;              // single-launch decode: fewest pages worth giving a CTA
     int step_boundary_pct = 100;          // single-launch decode: what a (sequence, kv head) boundary inside a CTA's range counts for
     float *chunk_ws = nullptr;            // partial results of split long sequences (step-chunk attention)
@@ -319,6 +320,7 @@ arb_status launch_decode_e4m3(Ctx *ctx, const arb_attn_params &p, const void *q,
                               const void *v_pages, float k_scale, float v_scale, const int32_t *block_table,
                               const int32_t *seq_lens, const int32_t *q_lens, void *out, cudaStream_t stream);
 bool decode_step_supported(const arb_attn_params &p);
+size_t decode_step_hint_bytes(int num_sms);
 arb_status launch_decode_step(Ctx *ctx, const arb_attn_params &p, const void *q, const void *k_new, const void *v_new,
                               void *k_pages, void *v_pages, const int32_t *block_table, int32_t *seq_lens,
                               const int32_t *q_lens, void *out, cudaStream_t stream);

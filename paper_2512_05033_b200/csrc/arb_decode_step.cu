@@ -43,6 +43,13 @@ constexpr int kOStride = kD + 4;              // floats between two heads of a w
 // What a boundary costs is time (the warps meet, a second arrival, perhaps a second merge), a few microseconds
 // whatever the call's size: as pages it is the CTA's even share, but no more than this many.
 constexpr int kBoundaryCap = 32;
+// Hints for the next call: every CTA leaves the pool rows of the first kHintPages page tiles of its range in a record
+// of the context.  The next call of the same shape asks for those tiles into L2 before it waits for its predecessor
+// (the bookkeeping warp does, off every other warp's path): in a chain of dependent calls the bytes of call n + 1
+// cross from HBM while call n is in its latency-bound tail.  A prefetch is a hint: rows are range-checked, a stale or
+// foreign record costs some bandwidth and nothing else, and every real read comes after the wait.
+constexpr int kHintPages = 64;
+constexpr int kHintStride = kHintPages + 4;   // [tag, count, -, -, rows ...]
 
 struct StepArgs {
     const char *q;
@@ -56,6 +63,8 @@ struct StepArgs {
     float *part_ml;    // [slots][GP][2]
     int *counters;     // [batch * Hkv] arrival counters, zero between calls
     int *lens_counter; // CTAs that have read the lengths, zero between calls
+    int *hint;         // [grid][kHintStride] the page tiles each CTA streamed last time (see kHintPages)
+    int hint_tag;      // shape of this call; a record with another tag is ignored
     uint32_t *status;
     int batch, Hq, Hkv, num_pages, max_pages;
     int whole_rows;    // the tensor maps are 3-D: one copy per page tile instead of one per half
@@ -235,11 +244,31 @@ decode_step_kernel(const StepArgs a, const __grid_constant__ CUtensorMap k_map, 
         row0[0] = 0;
         act[0] = 0;
     }
+    int *hint = a.hint + (size_t)blockIdx.x * kHintStride;
+    if (warp == kAuxWarp) {
+        // the tiles this CTA streamed last time are asked into L2 while the predecessor is still at work
+        const int tag = __ldcg(hint), cnt = __ldcg(hint + 1);
+        if (tag == a.hint_tag) {
+            const int n = min(cnt, kHintPages);
+            for (int i = lane; i < n; i += 32) {
+                const int row = __ldcg(hint + 4 + i);
+                if ((unsigned)row < (unsigned)(a.num_pages * Hkv * kPage)) {
+                    const size_t off = (size_t)row * (kD * 2);
+                    asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(a.k_pool + off), "r"(kTileBytes) : "memory");
+                    asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(a.v_pool + off), "r"(kTileBytes) : "memory");
+                }
+            }
+        }
+    }
     // Everything below may read what the kernel before this one wrote (lengths, q, new rows, the cache).
     wait_for_predecessor();
 
-    // ---- prologue: lengths -> page counts and q row offsets ------------------------------------------
-    for (int b = tid; b < B; b += kNT) {
+    // ---- prologue: lengths -> page counts and q row offsets (the bookkeeping warp joins when the plan is there) ----
+    constexpr int kPT = kNT - 32;   // threads of the prologue: all but the bookkeeping warp
+    if (warp == kAuxWarp) {
+        asm volatile("bar.sync 3, %0;" ::"r"(kNT) : "memory");
+    } else {
+    for (int b = tid; b < B; b += kPT) {
         const int n = a.q_lens[b], L0 = a.seq_lens[b];
         const bool ok = step_ok<APPEND>(n, L0, a.max_pages);
         const int L = L0 + (APPEND ? 1 : 0);
@@ -248,7 +277,7 @@ decode_step_kernel(const StepArgs a, const __grid_constant__ CUtensorMap k_map, 
         act[b + 1] = ok ? 1 : 0;
         slen[b] = L;
     }
-    __syncthreads();
+    named_barrier(2, kPT);
     if (warp == 0) {
         int carry_p = 0, carry_r = 0, carry_a = 0;
         for (int b0 = 0; b0 < B; b0 += 32) {
@@ -300,7 +329,9 @@ decode_step_kernel(const StepArgs a, const __grid_constant__ CUtensorMap k_map, 
             plan_s[4] = seq0;
         }
     }
-    __syncthreads();
+    named_barrier(2, kPT);
+    asm volatile("bar.arrive 3, %0;" ::"r"(kNT) : "memory");   // the plan is there: the bookkeeping warp may go on
+    }
 
     if (warp == kAuxWarp) {
         // ================================ bookkeeping warp ==========================================
@@ -345,7 +376,10 @@ decode_step_kernel(const StepArgs a, const __grid_constant__ CUtensorMap k_map, 
     pl.pen = plan_s[2];
     pl.chunk = plan_s[3];
     pl.total_padded = 0;   // only the cut needs it
-    if (r0 >= r1) return;
+    if (r0 >= r1) {
+        if (tid == 0) hint[1] = 0;   // nothing streamed: nothing to ask for next time
+        return;
+    }
     volatile int *abort = &tail->abort;
 
     if (warp == kProdWarp) {
@@ -371,8 +405,13 @@ decode_step_kernel(const StepArgs a, const __grid_constant__ CUtensorMap k_map, 
         };
         uint32_t c = 0;
         int row_next = lane < nflat ? tile_row(r0 + lane) : 0;
+        if (lane == 0) {
+            hint[0] = a.hint_tag;
+            hint[1] = nflat;
+        }
         for (int g0 = 0; g0 < nflat; g0 += 32) {
             const int row_cur = row_next;
+            if (g0 + lane < min(nflat, kHintPages)) hint[4 + g0 + lane] = row_cur;
             const int ntiles = 2 * min(32, nflat - g0);
 #pragma unroll 1
             for (int i0 = 0; i0 < ntiles; i0 += kBatch) {
@@ -784,6 +823,8 @@ arb_status launch_g(Ctx *ctx, const StepArgs &a, const CUtensorMap &km, const CU
 
 }  // namespace
 
+size_t decode_step_hint_bytes(int num_sms) { return sizeof(int) * (size_t)num_sms * kHintStride; }
+
 bool decode_step_supported(const arb_attn_params &p) {
     const int g = p.num_q_heads / p.num_kv_heads;
     return p.dtype == ARB_BF16 && p.head_dim == kD && g >= 1 && g <= 8 && tma_available();
@@ -820,6 +861,9 @@ arb_status launch_decode_step(Ctx *ctx, const arb_attn_params &p, const void *q,
     a.part_ml = a.part_o + part_o_floats;
     a.counters = ctx->rot;                                                       // [kRotCounters]
     a.lens_counter = ctx->rot + (size_t)kRotSets * kRotCounters + kRotSets + 4;
+    a.hint = ctx->step_hint;
+    a.hint_tag = (int)(((uint32_t)p.batch * 2654435761u) ^ ((uint32_t)p.num_kv_heads * 40503u) ^
+                       ((uint32_t)p.num_pages * 2246822519u) ^ ((uint32_t)p.max_pages_per_seq * 3266489917u)) | 1;
     a.status = ctx->status;
     a.batch = p.batch;
     a.Hq = p.num_q_heads;

@@ -181,6 +181,19 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity) {
     return ok != 0;
 }
 
+// The non-blocking form: true if the phase with the given parity has completed, else false at once.
+__device__ __forceinline__ bool mbar_test_wait(uint64_t *bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(smem_u32(bar)), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+
 // Wait for the phase with the given parity.  Every wait is bounded: after `limit` cycles (kWaitCycles in
 // every production kernel), or as soon as another thread of the block has given up (*abort != 0), it returns
 // false and the caller carries on with whatever is in shared memory; the status word then carries

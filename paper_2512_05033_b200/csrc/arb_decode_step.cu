@@ -419,11 +419,16 @@ decode_step_kernel(const StepArgs a, const __grid_constant__ CUtensorMap k_map, 
                 if (i0 == kBatch && g0 + 32 + lane < nflat) row_next = tile_row(r0 + g0 + 32 + lane);
                 const int i = i0 + lane;
                 const int row = __shfl_sync(0xffffffffu, row_cur, (i >> 1) & 31);
-                if (i < ntiles) {
-                    const uint32_t cc = c + i, st = cc % STAGES, par = (cc / STAGES) & 1u;
-                    const CUtensorMap *map = (i & 1) ? &v_map : &k_map;
-                    if (ARB_IN_RANGE(a.status, row, (long long)a.num_pages * Hkv * kPage) &&
-                        mbar_wait(&tail->empty[st], par ^ 1u, abort, a.status)) {
+                const uint32_t cc = c + i, st = cc % STAGES, par = (cc / STAGES) & 1u;
+                const CUtensorMap *map = (i & 1) ? &v_map : &k_map;
+                // The lanes wait for 32 different stages.  A blocking wait would put the whole warp to sleep until its
+                // time limit whenever one stage is not free yet, and copies for stages that are would go out late, in
+                // clumps (seen: 0.7 us apart).  So the warp polls, converged: every round each lane tests its own
+                // stage without blocking and issues its copy the moment the stage is free.
+                bool pending = i < ntiles && ARB_IN_RANGE(a.status, row, (long long)a.num_pages * Hkv * kPage);
+                const long long t0 = clock64();
+                while (__any_sync(0xffffffffu, pending)) {
+                    if (pending && mbar_test_wait(&tail->empty[st], par ^ 1u)) {
                         mbar_arrive_expect_tx(&tail->full[st], kTileBytes);
                         if (a.whole_rows) {
                             tma_box_load3(ring + st * kTileBytes, map, 0, row, 0, &tail->full[st]);
@@ -431,9 +436,16 @@ decode_step_kernel(const StepArgs a, const __grid_constant__ CUtensorMap k_map, 
                             tma_box_load(ring + st * kTileBytes, map, 0, row, &tail->full[st]);
                             tma_box_load(ring + st * kTileBytes + kHalfTile, map, 64, row, &tail->full[st]);
                         }
+                        pending = false;
+                    }
+                    if (pending && (*abort || clock64() - t0 > kWaitCycles)) {   // give up, like every other wait
+                        if (!*abort) {
+                            *abort = 1;
+                            atomicOr(a.status, (uint32_t)ARB_DEV_WAIT_TIMEOUT);
+                        }
+                        pending = false;
                     }
                 }
-                __syncwarp();
             }
             if (ntiles <= kBatch && g0 + 32 + lane < nflat) row_next = tile_row(r0 + g0 + 32 + lane);
             c += ntiles;

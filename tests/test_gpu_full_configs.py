@@ -143,3 +143,46 @@ def test_mixed_serving_loop_full():
         np.testing.assert_array_equal(seq.cpu().numpy(), seq_ref)
         escalated += int((dec.cpu().numpy() * (ql.cpu().numpy() > 1)).sum())
     assert 0 < escalated < B * len(m.q_lens) // 2
+
+
+def test_draft_shaped_decode_step_full():
+    """The single-launch token (arb_decode_step) on the draft-shaped batch, in the chain bench.py times: three tokens in a
+    row on one cache, every call finding what the one before it left; pools bit for bit, lengths exact, every row."""
+    shape = wl.DRAFT_DECODE
+    inp = wl.make_attn_inputs(shape, extra_tokens=8)
+    d = inp.to("cuda")
+    c = H.ctx()
+    sl = inp.seq_lens.numpy().copy()
+    k_ref, v_ref = inp.k_pages, inp.v_pages
+    ones = torch.ones(shape.batch, dtype=torch.int32)
+    outs, news = [], []
+    for t in range(3):
+        q = wl.normal((shape.batch, shape.num_q_heads, shape.head_dim), 1.0, BF, "cpu", 9100 + t)
+        kn = wl.normal((shape.batch, shape.num_kv_heads, shape.head_dim), 1.0, BF, "cpu", 9200 + t)
+        vn = wl.normal((shape.batch, shape.num_kv_heads, shape.head_dim), 1.0, BF, "cpu", 9300 + t)
+        news.append((q, kn, vn))
+        outs.append(c.decode_step(q.cuda(), kn.cuda(), vn.cuda(), d.k_pages, d.v_pages, d.block_table, d.seq_lens, d.q_lens))
+    assert c.poll_status() == 0
+    for (q, kn, vn), out in zip(news, outs):
+        k_ref, v_ref, sl, st = oracle.kv_append(kn, vn, inp.block_table, sl, ones, k_ref, v_ref)
+        ref, st2 = oracle.attn(q, k_ref, v_ref, inp.block_table, sl, ones)
+        assert st == 0 and st2 == 0
+        H.assert_close(out.double().cpu().numpy(), ref, BF, tight=3e-3)
+    assert np.array_equal(d.seq_lens.cpu().numpy(), sl)
+    assert torch.equal(d.k_pages.cpu(), k_ref) and torch.equal(d.v_pages.cpu(), v_ref)
+
+
+def test_step_scoring_full_over_the_e4m3_cache():
+    """arb_attn_e4m3 on the step-scoring batch at full size (pools quantised by the oracle), every element."""
+    shape = wl.STEP_SCORING
+    inp = wl.make_attn_inputs(shape)
+    ks, vs = 0.012, 0.015
+    kc = torch.from_numpy(oracle.e4m3_encode(inp.k_pages, 1 / ks))
+    vc = torch.from_numpy(oracle.e4m3_encode(inp.v_pages, 1 / vs))
+    d = inp.to("cuda")
+    c = H.ctx()
+    out = c.attn_e4m3(d.q, kc.cuda(), vc.cuda(), ks, vs, d.block_table, d.seq_lens, d.q_lens, int(inp.q_lens.max()))
+    assert c.poll_status() == 0
+    ref, st = oracle.attn_e4m3(inp.q, kc, vc, ks, vs, inp.block_table, inp.seq_lens, inp.q_lens)
+    assert st == 0
+    H.assert_close(out.double().cpu().numpy(), ref, BF, tight=3e-3)

@@ -425,6 +425,28 @@ arb_status arb_kv_append_e4m3(arb_ctx *ctx, const arb_attn_params *params, int32
                               uint8_t *v_codes, arb_stream_t stream);
 
 /*
+ * One decode token of a quantised draft in one launch: arb_kv_append_e4m3 of the token's K/V rows (update_lens = 1),
+ * arb_attn_decode_e4m3 over the cache that now holds them, and the length update, fused -- arb_decode_step for an
+ * E4M3 cache (Section 3.1: z_i ~ q(z_i | x, z_<i), one call per token and layer; Section 5.1's quantised drafts).
+ *
+ *   params, q, out, k_new, v_new, block_table, seq_lens, q_lens
+ *              as for arb_decode_step; dtype ARB_BF16 (q, out, k_new, v_new), head_dim 128, g <= 8.
+ *   k_codes,
+ *   v_codes    uint8 pools [num_pages, Hkv, P, D], written (code = e4m3(x * inv_scale): product in fp32, nearest
+ *              code, ties to even, saturating at +-448) and read (key = k_scale * code, value = v_scale * code).
+ *   k_scale, v_scale, k_inv_scale, v_inv_scale   > 0; the caller keeps inv_scale = 1 / scale (the library does not
+ *              divide, so that the codes are those of arb_kv_append_e4m3 given the same inv_scale).
+ * The codes written are bit-identical to arb_kv_append_e4m3's, the rows equal arb_attn_decode_e4m3's within its
+ * tolerance.  Refused sequences, idle slots, status bits and stream behaviour as for arb_decode_step.
+ * Errors: ARB_ERR_INVALID_ARG, ARB_ERR_UNSUPPORTED (dtype, head_dim, g > 8, ARB_ATTN_NO_TENSOR_CORES),
+ * ARB_ERR_WORKSPACE, ARB_ERR_CUDA.
+ */
+arb_status arb_decode_step_e4m3(arb_ctx *ctx, const arb_attn_params *params, const void *q, const void *k_new,
+                                const void *v_new, uint8_t *k_codes, uint8_t *v_codes, float k_scale, float v_scale,
+                                float k_inv_scale, float v_inv_scale, const int32_t *block_table, int32_t *seq_lens,
+                                const int32_t *q_lens, void *out, arb_stream_t stream);
+
+/*
  * Spearman's rank correlation of two samples (Section 4.2, "Evaluation", and Tables 1-3 of the paper:
  * the correlation between the router's predicted scores and the oracle advantage Delta).  Each value is
  * replaced by its rank within its sample, equal values sharing the mean of the ranks they span, and

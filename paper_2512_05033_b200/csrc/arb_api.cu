@@ -237,7 +237,7 @@ arb_status arb_attn(arb_ctx *ctx, const arb_attn_params *params, const void *q, 
         const bool series = (params->flags & ARB_ATTN_OVERLAP_PREVIOUS) != 0;
         if (tensor_cores && !series && decode_step_supported(*params))
             st = launch_decode_step(c, *params, q, nullptr, nullptr, const_cast<void *>(k_pages),
-                                    const_cast<void *>(v_pages), block_table, const_cast<int32_t *>(seq_lens), q_lens, out, s);
+                                    const_cast<void *>(v_pages), nullptr, block_table, const_cast<int32_t *>(seq_lens), q_lens, out, s);
         else if (tensor_cores && decode_mma_supported(*params))
             st = launch_decode_mma(c, *params, q, k_pages, v_pages, block_table, seq_lens, q_lens, out, s);
         else {
@@ -281,12 +281,38 @@ arb_status arb_decode_step(arb_ctx *ctx, const arb_attn_params *params, const vo
     if (decode_workspace_bytes(*params, c->num_sms) > c->workspace_bytes) return ARB_ERR_WORKSPACE;
     cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
     if ((params->flags & ARB_ATTN_NO_TENSOR_CORES) == 0 && decode_step_supported(*params))
-        return launch_decode_step(c, *params, q, k_new, v_new, k_pages, v_pages, block_table, seq_lens, q_lens, out, s);
+        return launch_decode_step(c, *params, q, k_new, v_new, k_pages, v_pages, nullptr, block_table, seq_lens, q_lens, out, s);
     // shapes the single launch does not serve (fp32, head_dim 64): the same step as two launches
     st = launch_kv_append(c, *params, params->total_q, k_new, v_new, block_table, seq_lens, q_lens, 1, k_pages, v_pages, s);
     if (st != ARB_OK) return st;
     note_unnumbered_decode(c, decode_workspace_bytes(*params, c->num_sms));
     return launch_decode(c, *params, q, k_pages, v_pages, block_table, seq_lens, q_lens, out, s);
+}
+
+arb_status arb_decode_step_e4m3(arb_ctx *ctx, const arb_attn_params *params, const void *q, const void *k_new,
+                                const void *v_new, uint8_t *k_codes, uint8_t *v_codes, float k_scale, float v_scale,
+                                float k_inv_scale, float v_inv_scale, const int32_t *block_table, int32_t *seq_lens,
+                                const int32_t *q_lens, void *out, arb_stream_t stream) {
+    if (ctx == nullptr) return ARB_ERR_INVALID_ARG;
+    arb_status st = check_params(params);
+    if (st != ARB_OK) return st;
+    if (params->dtype != ARB_BF16 || params->head_dim != 128) return ARB_ERR_UNSUPPORTED;
+    if (params->flags & ARB_ATTN_NO_TENSOR_CORES) return ARB_ERR_UNSUPPORTED;
+    if (params->max_q_len != 1 || params->total_q < 0 || params->total_q > params->batch) return ARB_ERR_INVALID_ARG;
+    if (params->flags & ARB_ATTN_OVERLAP_PREVIOUS) return ARB_ERR_INVALID_ARG;   // the call writes the cache it reads
+    if (!(k_scale > 0.f) || !(v_scale > 0.f) || !(k_inv_scale > 0.f) || !(v_inv_scale > 0.f)) return ARB_ERR_INVALID_ARG;
+    if (!k_codes || !v_codes || !block_table || !seq_lens || !q_lens) return ARB_ERR_INVALID_ARG;
+    if (params->total_q == 0) return ARB_OK;
+    if (!q || !out || !k_new || !v_new) return ARB_ERR_INVALID_ARG;
+    if (!aligned16(q) || !aligned16(out) || !aligned16(k_codes) || !aligned16(v_codes) || !aligned16(k_new) ||
+        !aligned16(v_new))
+        return ARB_ERR_INVALID_ARG;
+    Ctx *c = reinterpret_cast<Ctx *>(ctx);
+    if (decode_workspace_bytes(*params, c->num_sms) > c->workspace_bytes) return ARB_ERR_WORKSPACE;
+    if (!decode_step_supported(*params)) return ARB_ERR_UNSUPPORTED;
+    const float scales[4] = {k_scale, v_scale, k_inv_scale, v_inv_scale};
+    return launch_decode_step(c, *params, q, k_new, v_new, k_codes, v_codes, scales, block_table, seq_lens, q_lens, out,
+                              reinterpret_cast<cudaStream_t>(stream));
 }
 
 arb_status arb_attn_decode_static(const arb_attn_params *params, const void *q, const void *k_pages,

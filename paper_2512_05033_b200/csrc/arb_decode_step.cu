@@ -24,6 +24,13 @@
 //   - With k_new / v_new given, the warp that owns a sequence's last page puts the token's new row into the
 //     tile in shared memory (the tile arrives with whatever the slot held) and stores it to the pool; the
 //     lengths move forward once every CTA has read them (a counter in the prologue tells the last reader).
+//
+// Compiled a second time (template parameter E4M3) the kernel serves an E4M3 cache (arb_decode_step_e4m3: the token
+// of a quantised draft).  A page tile is 2 KB of codes; the consumer warp that owns it widens it to f16 (exact) into
+// a tile of its own in shared memory, laid out like a bf16 tile, frees the ring stage at once, and runs the same
+// fragment loads and MMAs on f16 operands (q converted bf16 -> f16, P rounded to f16).  The token's new rows are
+// quantised by the warp that patches them in (x * inv_scale, nearest code, saturating: the arithmetic of
+// arb_kv_append_e4m3), stored to the pool as codes and patched into the widened tile.
 #include "arb_decode_tc.cuh"
 
 namespace arb {
@@ -37,6 +44,7 @@ constexpr int kAuxWarp = kCW + 1;             // bookkeeping: length update, row
 constexpr int kNT = kCT + 64;
 constexpr int kTileBytes = kPage * kD * 2;    // 4 KB: one (page, kv head) tile of K or of V
 constexpr int kHalfTile = kTileBytes / 2;
+constexpr int kCodeTileBytes = kPage * kD;    // 2 KB: the same tile of an E4M3 cache
 constexpr int kBatch = 32;                    // producer lanes issuing side by side
 constexpr int kParked = 2;                    // segment results parked in shared memory before they are written
 constexpr int kOStride = kD + 4;              // floats between two heads of a warp record (spreads the banks)
@@ -72,7 +80,9 @@ struct StepArgs {
     int rows;          // rows of q and out
     int min_chunk;     // fewest pages worth giving a CTA
     int boundary_pct;  // cost of a (sequence, kv head) boundary inside a CTA's range: percent of min(even share, kBoundaryCap) pages
-    float scale_log2;
+    float scale_log2;  // softmax scale (times the key scale of an E4M3 cache) * log2(e)
+    float v_scale;     // value scale of an E4M3 cache, 1 otherwise
+    float k_inv_scale, v_inv_scale;   // E4M3 cache with a cache write: code = e4m3(x * inv_scale)
 };
 
 template <int STAGES>
@@ -93,11 +103,12 @@ struct Cfg {
     static constexpr int PARK_BYTES = kParked * REC * 4;
 };
 
-template <int G, int STAGES>
+// E4M3: the ring holds tiles of codes; every consumer warp has a widened K tile and a widened V tile of its own
+template <int G, int STAGES, bool E4M3>
 size_t smem_bytes(int batch) {
     using C = Cfg<G>;
-    return 1024 + (size_t)STAGES * kTileBytes + C::OSM_BYTES + C::PARK_BYTES + sizeof(Tail<STAGES>) +
-           sizeof(int) * (4 * (size_t)batch + 3 + 8);
+    const size_t tiles = E4M3 ? (size_t)STAGES * kCodeTileBytes + (size_t)kCW * 2 * kTileBytes : (size_t)STAGES * kTileBytes;
+    return 1024 + tiles + C::OSM_BYTES + C::PARK_BYTES + sizeof(Tail<STAGES>) + sizeof(int) * (4 * (size_t)batch + 3 + 8);
 }
 
 struct Parked {
@@ -112,6 +123,49 @@ struct Pending {   // a split (sequence, kv head) this CTA was the last to reach
 
 __device__ __forceinline__ uint32_t tile_off(int r, int c) {   // 16-byte chunk c of row r of a swizzled bf16 tile
     return (uint32_t)((c >> 3) * kHalfTile + r * 128 + (((c & 7) ^ (r & 7)) << 4));
+}
+
+__device__ __forceinline__ uint32_t pack_f16(float lo, float hi) {
+    uint32_t r;
+    asm("cvt.rn.f16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+    return r;
+}
+__device__ __forceinline__ float2 unpack_f16(uint32_t v) {
+    float lo, hi;
+    asm("{\n\t.reg .b16 l, h;\n\tmov.b32 {l, h}, %2;\n\tcvt.f32.f16 %0, l;\n\tcvt.f32.f16 %1, h;\n\t}" : "=f"(lo), "=f"(hi) : "r"(v));
+    return make_float2(lo, hi);
+}
+__device__ __forceinline__ uint32_t bf16x2_to_f16x2(uint32_t v) {
+    return pack_f16(__uint_as_float(v << 16), __uint_as_float(v & 0xffff0000u));
+}
+// two E4M3 codes (a 16-bit pair) -> f16x2, exact; the low byte lands in the low half
+__device__ __forceinline__ uint32_t e4m3x2_to_f16x2(uint16_t v) {
+    uint32_t r;
+    asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(r) : "h"(v));
+    return r;
+}
+// two values -> two E4M3 codes (nearest, ties to even, saturating); lo lands in the low byte
+__device__ __forceinline__ uint32_t e4m3x2_from_f32(float lo, float hi) {
+    uint16_t r;
+    asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(r) : "f"(hi), "f"(lo));
+    return r;
+}
+// A warp widens a tile of codes (16 rows x 128 B, 128-byte swizzle) into an f16 tile laid out like a bf16 tile:
+// lane (r, h) = (lane / 2, lane % 2) takes the 64 codes of half h of row r, four 16-byte pieces in, eight out.
+__device__ __forceinline__ void widen_tile(const char *codes, char *dst, int lane) {
+    const int r = lane >> 1, h = lane & 1;
+#pragma unroll
+    for (int c4 = 0; c4 < 4; ++c4) {
+        const int c = 4 * h + c4;
+        const uint4 cd = *reinterpret_cast<const uint4 *>(codes + r * 128 + ((c ^ (r & 7)) << 4));
+        uint4 lo, hi;
+        lo.x = e4m3x2_to_f16x2((uint16_t)cd.x); lo.y = e4m3x2_to_f16x2((uint16_t)(cd.x >> 16));
+        lo.z = e4m3x2_to_f16x2((uint16_t)cd.y); lo.w = e4m3x2_to_f16x2((uint16_t)(cd.y >> 16));
+        hi.x = e4m3x2_to_f16x2((uint16_t)cd.z); hi.y = e4m3x2_to_f16x2((uint16_t)(cd.z >> 16));
+        hi.z = e4m3x2_to_f16x2((uint16_t)cd.w); hi.w = e4m3x2_to_f16x2((uint16_t)(cd.w >> 16));
+        *reinterpret_cast<uint4 *>(dst + tile_off(r, 2 * c)) = lo;
+        *reinterpret_cast<uint4 *>(dst + tile_off(r, 2 * c + 1)) = hi;
+    }
 }
 
 __device__ __forceinline__ void fence_proxy_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
@@ -202,13 +256,16 @@ __device__ __forceinline__ void parts_of(const Plan &pl, Segment &s) {
     s.nparts = pl.cta_of(s.b, s.kvh, pages, pages - 1) - s.c_first + 1;
 }
 
-template <int G, int STAGES, bool APPEND>
+template <int G, int STAGES, bool APPEND, bool E4M3>
 __global__ void __launch_bounds__(kNT, 1)
 decode_step_kernel(const StepArgs a, const __grid_constant__ CUtensorMap k_map, const __grid_constant__ CUtensorMap v_map) {
     using C = Cfg<G>;
     using Tail = arb::Tail<STAGES>;
     constexpr int GP = C::GP, WREC = C::WREC, REC = C::REC;
-    constexpr int kRingBytes = STAGES * kTileBytes;
+    constexpr int kStageBytes = E4M3 ? kCodeTileBytes : kTileBytes;   // what one TMA copy brings
+    constexpr int kElt = E4M3 ? 1 : 2;                                  // bytes of a cache element
+    constexpr int kWideBytes = E4M3 ? kCW * 2 * kTileBytes : 0;         // E4M3: a widened K and V tile per consumer warp
+    constexpr int kRingBytes = STAGES * kStageBytes + kWideBytes;       // the merges use all of it
     static_assert(G >= 1 && G <= 8, "the group's heads are the 8 columns of the tile");
     static_assert(STAGES % (2 * kCW) == 0 && kBatch <= STAGES, "a ring stage always belongs to the same warp of a segment");
 
@@ -253,9 +310,9 @@ decode_step_kernel(const StepArgs a, const __grid_constant__ CUtensorMap k_map, 
             for (int i = lane; i < n; i += 32) {
                 const int row = __ldcg(hint + 4 + i);
                 if ((unsigned)row < (unsigned)(a.num_pages * Hkv * kPage)) {
-                    const size_t off = (size_t)row * (kD * 2);
-                    asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(a.k_pool + off), "r"(kTileBytes) : "memory");
-                    asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(a.v_pool + off), "r"(kTileBytes) : "memory");
+                    const size_t off = (size_t)row * (kD * kElt);
+                    asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(a.k_pool + off), "r"(kStageBytes) : "memory");
+                    asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(a.v_pool + off), "r"(kStageBytes) : "memory");
                 }
             }
         }
@@ -429,8 +486,10 @@ decode_step_kernel(const StepArgs a, const __grid_constant__ CUtensorMap k_map, 
                 const long long t0 = clock64();
                 while (__any_sync(0xffffffffu, pending)) {
                     if (pending && mbar_test_wait(&tail->empty[st], par ^ 1u)) {
-                        mbar_arrive_expect_tx(&tail->full[st], kTileBytes);
-                        if (a.whole_rows) {
+                        mbar_arrive_expect_tx(&tail->full[st], kStageBytes);
+                        if constexpr (E4M3) {
+                            tma_box_load(ring + st * kStageBytes, map, 0, row, &tail->full[st]);   // 16 rows x 128 codes
+                        } else if (a.whole_rows) {
                             tma_box_load3(ring + st * kTileBytes, map, 0, row, 0, &tail->full[st]);
                         } else {
                             tma_box_load(ring + st * kTileBytes, map, 0, row, &tail->full[st]);
@@ -468,7 +527,6 @@ decode_step_kernel(const StepArgs a, const __grid_constant__ CUtensorMap k_map, 
     const int gq = lane >> 2, tq = lane & 3;   // fragment coordinates
     const bool head_ok = gq < G;               // as a B-fragment column: this lane's head is a real one
     const int h0 = 2 * tq, h1 = 2 * tq + 1;    // as accumulator columns: the two heads this lane holds
-    const uint32_t ring_addr = smem_u32(ring);
     uint32_t seg_base = 0;                     // ring counter of the segment's first tile
     int cur = r0;
     Segment s;
@@ -538,8 +596,14 @@ decode_step_kernel(const StepArgs a, const __grid_constant__ CUtensorMap k_map, 
         for (int ks = 0; ks < 8; ++ks) {
             dst[ks][0] = head_ok ? __ldg(reinterpret_cast<const uint32_t *>(qh + ks * 32 + tq * 4)) : 0u;
             dst[ks][1] = head_ok ? __ldg(reinterpret_cast<const uint32_t *>(qh + ks * 32 + 16 + tq * 4)) : 0u;
+            if constexpr (E4M3) {   // the operands of one MMA share a type: q goes to f16 like the widened codes
+                dst[ks][0] = bf16x2_to_f16x2(dst[ks][0]);
+                dst[ks][1] = bf16x2_to_f16x2(dst[ks][1]);
+            }
         }
     };
+    // E4M3: this warp's widened K and V tiles
+    char *wide_k = ring + STAGES * kStageBytes + warp * 2 * kTileBytes, *wide_v = wide_k + kTileBytes;
     Segment s_next;
     int seq_at = seq0;
     bool have = next_segment(cur, r1, seq_at, pl, s);
@@ -561,11 +625,29 @@ decode_step_kernel(const StepArgs a, const __grid_constant__ CUtensorMap k_map, 
                 const char *src = (lane < 16 ? a.k_new : a.v_new) + ((size_t)qrow * Hkv + s.kvh) * kD * 2 + (lane & 15) * 16;
                 new_row = __ldg(reinterpret_cast<const uint4 *>(src));
                 const int pid = a.block_table[(size_t)s.b * a.max_pages + last_pg];
-                if ((unsigned)pid < (unsigned)a.num_pages && ARB_IN_RANGE(a.status, qrow, a.rows)) {
+                const bool store = (unsigned)pid < (unsigned)a.num_pages && ARB_IN_RANGE(a.status, qrow, a.rows);
+                // (a page outside the pool: the producer has raised ARB_DEV_BAD_PAGE; nothing is written)
+                if constexpr (E4M3) {
+                    // quantise this lane's eight values as arb_kv_append_e4m3 does (x * inv_scale in fp32, nearest code,
+                    // ties to even, saturating), store the codes, and keep their widened form for the tile
+                    const float inv = lane < 16 ? a.k_inv_scale : a.v_inv_scale;
+                    const uint32_t w[4] = {new_row.x, new_row.y, new_row.z, new_row.w};
+                    uint32_t code[4];
+#pragma unroll
+                    for (int j = 0; j < 4; ++j)
+                        code[j] = e4m3x2_from_f32(__uint_as_float(w[j] << 16) * inv, __uint_as_float(w[j] & 0xffff0000u) * inv);
+                    if (store) {
+                        char *dst = (lane < 16 ? a.k_pool : a.v_pool) +
+                                    (((size_t)pid * Hkv + s.kvh) * kPage + new_slot) * kD + (lane & 15) * 8;
+                        *reinterpret_cast<uint2 *>(dst) = make_uint2(code[0] | (code[1] << 16), code[2] | (code[3] << 16));
+                    }
+                    new_row = make_uint4(e4m3x2_to_f16x2((uint16_t)code[0]), e4m3x2_to_f16x2((uint16_t)code[1]),
+                                         e4m3x2_to_f16x2((uint16_t)code[2]), e4m3x2_to_f16x2((uint16_t)code[3]));
+                } else if (store) {
                     char *dst = (lane < 16 ? a.k_pool : a.v_pool) +
                                 (((size_t)pid * Hkv + s.kvh) * kPage + new_slot) * (kD * 2) + (lane & 15) * 16;
                     *reinterpret_cast<uint4 *>(dst) = new_row;
-                }   // a page outside the pool: the producer has raised ARB_DEV_BAD_PAGE; nothing is written
+                }
             }
         }
 
@@ -587,21 +669,30 @@ decode_step_kernel(const StepArgs a, const __grid_constant__ CUtensorMap k_map, 
             {
                 const uint32_t st = ck % STAGES, par = (ck / STAGES) & 1u;
                 mbar_wait(&tail->full[st], par, abort, a.status);
+                char *tile_p = ring + st * kStageBytes;
+                if constexpr (E4M3) {   // widen into this warp's tile; the ring stage is free at once
+                    widen_tile(tile_p, wide_k, lane);
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&tail->empty[st]);
+                    tile_p = wide_k;
+                }
                 if (patch_here) {
-                    if (lane < 16) *reinterpret_cast<uint4 *>(ring + st * kTileBytes + tile_off(new_slot, lane)) = new_row;
+                    if (lane < 16) *reinterpret_cast<uint4 *>(tile_p + tile_off(new_slot, lane)) = new_row;
                     __syncwarp();
                 }
-                const uint32_t tile = ring_addr + st * kTileBytes;
+                const uint32_t tile = smem_u32(tile_p);
 #pragma unroll
                 for (int ks = 0; ks < 8; ++ks) {
                     uint32_t af[4];   // rows: keys; matrices: (keys 0-7 | 8-15) x (dims 16 ks + 0-7 | 8-15)
                     ldmatrix_x4(tile + tile_off((lane & 7) + ((lane >> 3) & 1) * 8, 2 * ks + (lane >> 4)), af);
-                    if (ks & 1) mma_16816<false>(sb, af, qb[ks][0], qb[ks][1]);
-                    else mma_16816<false>(sa, af, qb[ks][0], qb[ks][1]);
+                    if (ks & 1) mma_16816<E4M3>(sb, af, qb[ks][0], qb[ks][1]);
+                    else mma_16816<E4M3>(sa, af, qb[ks][0], qb[ks][1]);
                 }
                 __syncwarp();
-                if (patch_here) fence_proxy_async_smem();   // the stage's next writer is the TMA unit
-                if (lane == 0) mbar_arrive(&tail->empty[st]);
+                if constexpr (!E4M3) {
+                    if (patch_here) fence_proxy_async_smem();   // the stage's next writer is the TMA unit
+                    if (lane == 0) mbar_arrive(&tail->empty[st]);
+                }
             }
 
             // ---- online softmax: this lane has keys gq and gq + 8 of heads h0 and h1 -------------------
@@ -620,11 +711,19 @@ decode_step_kernel(const StepArgs a, const __grid_constant__ CUtensorMap k_map, 
             const float f0 = fast_exp2(m_run0 - mn0), f1 = fast_exp2(m_run1 - mn1);   // 0 on the first page
             m_run0 = mn0;
             m_run1 = mn1;
-            // P^T, rounded to bf16; the sums use the rounded weights, like the tensor core
-            const uint32_t w0 = pack_bf16(fast_exp2(s00 - mn0), fast_exp2(s01 - mn1));   // key gq:     heads h0, h1
-            const uint32_t w1 = pack_bf16(fast_exp2(s10 - mn0), fast_exp2(s11 - mn1));   // key gq + 8
-            l_run0 = fmaf(l_run0, f0, __uint_as_float(w0 << 16) + __uint_as_float(w1 << 16));
-            l_run1 = fmaf(l_run1, f1, __uint_as_float(w0 & 0xffff0000u) + __uint_as_float(w1 & 0xffff0000u));
+            // P^T, rounded to bf16 (f16 over an E4M3 cache); the sums use the rounded weights, like the tensor core
+            const float p00 = fast_exp2(s00 - mn0), p01 = fast_exp2(s01 - mn1);
+            const float p10 = fast_exp2(s10 - mn0), p11 = fast_exp2(s11 - mn1);
+            const uint32_t w0 = E4M3 ? pack_f16(p00, p01) : pack_bf16(p00, p01);   // key gq:     heads h0, h1
+            const uint32_t w1 = E4M3 ? pack_f16(p10, p11) : pack_bf16(p10, p11);   // key gq + 8
+            if constexpr (E4M3) {
+                const float2 r0 = unpack_f16(w0), r1 = unpack_f16(w1);
+                l_run0 = fmaf(l_run0, f0, r0.x + r1.x);
+                l_run1 = fmaf(l_run1, f1, r0.y + r1.y);
+            } else {
+                l_run0 = fmaf(l_run0, f0, __uint_as_float(w0 << 16) + __uint_as_float(w1 << 16));
+                l_run1 = fmaf(l_run1, f1, __uint_as_float(w0 & 0xffff0000u) + __uint_as_float(w1 & 0xffff0000u));
+            }
             // B fragment of P^T (16 keys x 8 heads): keys 2 tq, + 1 (and + 8) of head gq
             const uint32_t pb0 = movmatrix_trans(w0), pb1 = movmatrix_trans(w1);
             if (__any_sync(0xffffffffu, f0 != 1.0f || f1 != 1.0f)) {
@@ -636,27 +735,36 @@ decode_step_kernel(const StepArgs a, const __grid_constant__ CUtensorMap k_map, 
             {
                 const uint32_t cv = ck + 1u, st = cv % STAGES, par = (cv / STAGES) & 1u;
                 mbar_wait(&tail->full[st], par, abort, a.status);
+                char *tile_p = ring + st * kStageBytes;
+                if constexpr (E4M3) {
+                    widen_tile(tile_p, wide_v, lane);
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&tail->empty[st]);
+                    tile_p = wide_v;
+                }
                 if (patch_here) {
-                    if (lane >= 16) *reinterpret_cast<uint4 *>(ring + st * kTileBytes + tile_off(new_slot, lane - 16)) = new_row;
+                    if (lane >= 16) *reinterpret_cast<uint4 *>(tile_p + tile_off(new_slot, lane - 16)) = new_row;
                     __syncwarp();
                 }
                 if (ntok < kPage) {
                     // slots past the sequence end may hold anything; they must not reach the tensor core, not even
                     // times zero: blank them in shared memory
                     for (int i = lane; i < (kPage - ntok) * 16; i += 32)
-                        *reinterpret_cast<uint4 *>(ring + st * kTileBytes + tile_off(ntok + (i >> 4), i & 15)) = make_uint4(0, 0, 0, 0);
+                        *reinterpret_cast<uint4 *>(tile_p + tile_off(ntok + (i >> 4), i & 15)) = make_uint4(0, 0, 0, 0);
                     __syncwarp();
                 }
-                const uint32_t tile = ring_addr + st * kTileBytes;
+                const uint32_t tile = smem_u32(tile_p);
 #pragma unroll
                 for (int mt = 0; mt < 8; ++mt) {
                     uint32_t af[4];   // transposed on the way: rows dims (16 mt + 0-7 | 8-15), columns keys (0-7 | 8-15)
                     ldmatrix_x4_trans(tile + tile_off((lane & 7) + (lane >> 4) * 8, 2 * mt + ((lane >> 3) & 1)), af);
-                    mma_16816<false>(o[mt], af, pb0, pb1);
+                    mma_16816<E4M3>(o[mt], af, pb0, pb1);
                 }
                 __syncwarp();
-                if (patch_here || ntok < kPage) fence_proxy_async_smem();
-                if (lane == 0) mbar_arrive(&tail->empty[st]);
+                if constexpr (!E4M3) {
+                    if (patch_here || ntok < kPage) fence_proxy_async_smem();
+                    if (lane == 0) mbar_arrive(&tail->empty[st]);
+                }
             }
         }
         seg_base += 2u * (uint32_t)seg_pages;
@@ -693,7 +801,7 @@ decode_step_kernel(const StepArgs a, const __grid_constant__ CUtensorMap k_map, 
                 l = fmaf(ff, osm[w * WREC + 8 + h], l);
                 acc = fmaf(ff, osm[w * WREC + 16 + h * kOStride + d], acc);
             }
-            dst[2 * GP + idx] = acc;
+            dst[2 * GP + idx] = E4M3 ? acc * a.v_scale : acc;   // values of an E4M3 cache are v_scale * code
             if (d == 0) { dst[h] = M; dst[GP + h] = l; }
         }
         parts_of(pl, s);
@@ -804,12 +912,12 @@ decode_step_kernel(const StepArgs a, const __grid_constant__ CUtensorMap k_map, 
 // kernel's CTAs leave anyway.
 constexpr int kStages = 32;
 
-template <int G, bool APPEND>
+template <int G, bool APPEND, bool E4M3>
 arb_status launch_variant(Ctx *ctx, const StepArgs &a, const CUtensorMap &km, const CUtensorMap &vm, cudaStream_t stream) {
     static bool attr_set[64] = {};
     if (!attr_set[ctx->device & 63]) {
-        if (cudaFuncSetAttribute(decode_step_kernel<G, kStages, APPEND>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 (int)smem_bytes<G, kStages>(kMaxBatch)) != cudaSuccess)
+        if (cudaFuncSetAttribute(decode_step_kernel<G, kStages, APPEND, E4M3>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 (int)smem_bytes<G, kStages, E4M3>(kMaxBatch)) != cudaSuccess)
             return ARB_ERR_CUDA;
         attr_set[ctx->device & 63] = true;
     }
@@ -819,18 +927,21 @@ arb_status launch_variant(Ctx *ctx, const StepArgs &a, const CUtensorMap &km, co
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(ctx->num_sms);
     cfg.blockDim = dim3(kNT);
-    cfg.dynamicSmemBytes = smem_bytes<G, kStages>(a.batch);
+    cfg.dynamicSmemBytes = smem_bytes<G, kStages, E4M3>(a.batch);
     cfg.stream = stream;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    if (cudaLaunchKernelEx(&cfg, decode_step_kernel<G, kStages, APPEND>, a, km, vm) != cudaSuccess) return ARB_ERR_CUDA;
+    if (cudaLaunchKernelEx(&cfg, decode_step_kernel<G, kStages, APPEND, E4M3>, a, km, vm) != cudaSuccess) return ARB_ERR_CUDA;
     ctx->launches++;
     return ARB_OK;
 }
 
+// The E4M3 form exists with the cache write only: decode alone over an E4M3 cache is arb_attn_decode_e4m3.
 template <int G>
-arb_status launch_g(Ctx *ctx, const StepArgs &a, const CUtensorMap &km, const CUtensorMap &vm, cudaStream_t stream) {
-    return a.k_new != nullptr ? launch_variant<G, true>(ctx, a, km, vm, stream) : launch_variant<G, false>(ctx, a, km, vm, stream);
+arb_status launch_g(Ctx *ctx, const StepArgs &a, bool e4m3, const CUtensorMap &km, const CUtensorMap &vm, cudaStream_t stream) {
+    if (e4m3) return launch_variant<G, true, true>(ctx, a, km, vm, stream);
+    return a.k_new != nullptr ? launch_variant<G, true, false>(ctx, a, km, vm, stream)
+                              : launch_variant<G, false, false>(ctx, a, km, vm, stream);
 }
 
 }  // namespace
@@ -842,16 +953,26 @@ bool decode_step_supported(const arb_attn_params &p) {
     return p.dtype == ARB_BF16 && p.head_dim == kD && g >= 1 && g <= 8 && tma_available();
 }
 
-// k_new == nullptr: attention only (seq_lens is not written).
+// k_new == nullptr: attention only (seq_lens is not written).  scales == nullptr: a bf16 cache; else an E4M3 cache
+// with scales = {k_scale, v_scale, k_inv_scale, v_inv_scale} (k_new is required then).
 arb_status launch_decode_step(Ctx *ctx, const arb_attn_params &p, const void *q, const void *k_new, const void *v_new,
-                              void *k_pages, void *v_pages, const int32_t *block_table, int32_t *seq_lens,
-                              const int32_t *q_lens, void *out, cudaStream_t stream) {
+                              void *k_pages, void *v_pages, const float *scales, const int32_t *block_table,
+                              int32_t *seq_lens, const int32_t *q_lens, void *out, cudaStream_t stream) {
     alignas(64) CUtensorMap km, vm;
-    bool whole_rows = pool_map(ctx, &km, k_pages, p.num_pages, p.num_kv_heads, PoolView::kBf16WholeRows) &&
-                      pool_map(ctx, &vm, v_pages, p.num_pages, p.num_kv_heads, PoolView::kBf16WholeRows);
-    if (!whole_rows && (!pool_map(ctx, &km, k_pages, p.num_pages, p.num_kv_heads, PoolView::kBf16HalfRows) ||
-                        !pool_map(ctx, &vm, v_pages, p.num_pages, p.num_kv_heads, PoolView::kBf16HalfRows)))
-        return ARB_ERR_CUDA;
+    const bool e4m3 = scales != nullptr;
+    if (e4m3 && k_new == nullptr) return ARB_ERR_INVALID_ARG;
+    bool whole_rows = false;
+    if (e4m3) {
+        if (!pool_map(ctx, &km, k_pages, p.num_pages, p.num_kv_heads, PoolView::kE4m3) ||
+            !pool_map(ctx, &vm, v_pages, p.num_pages, p.num_kv_heads, PoolView::kE4m3))
+            return ARB_ERR_CUDA;
+    } else {
+        whole_rows = pool_map(ctx, &km, k_pages, p.num_pages, p.num_kv_heads, PoolView::kBf16WholeRows) &&
+                     pool_map(ctx, &vm, v_pages, p.num_pages, p.num_kv_heads, PoolView::kBf16WholeRows);
+        if (!whole_rows && (!pool_map(ctx, &km, k_pages, p.num_pages, p.num_kv_heads, PoolView::kBf16HalfRows) ||
+                            !pool_map(ctx, &vm, v_pages, p.num_pages, p.num_kv_heads, PoolView::kBf16HalfRows)))
+            return ARB_ERR_CUDA;
+    }
     const int g = p.num_q_heads / p.num_kv_heads;
     const int gp = (g + 3) / 4 * 4;
     const size_t slots = (size_t)p.batch * p.num_kv_heads + (size_t)ctx->num_sms;
@@ -888,16 +1009,19 @@ arb_status launch_decode_step(Ctx *ctx, const arb_attn_params &p, const void *q,
     a.boundary_pct = ctx->step_boundary_pct;
     a.min_chunk = ctx->step_min_chunk;
     const float scale = p.softmax_scale > 0.f ? p.softmax_scale : 1.0f / sqrtf((float)p.head_dim);
-    a.scale_log2 = scale * 1.4426950408889634f;
+    a.scale_log2 = scale * (e4m3 ? scales[0] : 1.0f) * 1.4426950408889634f;
+    a.v_scale = e4m3 ? scales[1] : 1.0f;
+    a.k_inv_scale = e4m3 ? scales[2] : 1.0f;
+    a.v_inv_scale = e4m3 ? scales[3] : 1.0f;
     switch (g) {
-        case 1: return launch_g<1>(ctx, a, km, vm, stream);
-        case 2: return launch_g<2>(ctx, a, km, vm, stream);
-        case 3: return launch_g<3>(ctx, a, km, vm, stream);
-        case 4: return launch_g<4>(ctx, a, km, vm, stream);
-        case 5: return launch_g<5>(ctx, a, km, vm, stream);
-        case 6: return launch_g<6>(ctx, a, km, vm, stream);
-        case 7: return launch_g<7>(ctx, a, km, vm, stream);
-        case 8: return launch_g<8>(ctx, a, km, vm, stream);
+        case 1: return launch_g<1>(ctx, a, e4m3, km, vm, stream);
+        case 2: return launch_g<2>(ctx, a, e4m3, km, vm, stream);
+        case 3: return launch_g<3>(ctx, a, e4m3, km, vm, stream);
+        case 4: return launch_g<4>(ctx, a, e4m3, km, vm, stream);
+        case 5: return launch_g<5>(ctx, a, e4m3, km, vm, stream);
+        case 6: return launch_g<6>(ctx, a, e4m3, km, vm, stream);
+        case 7: return launch_g<7>(ctx, a, e4m3, km, vm, stream);
+        case 8: return launch_g<8>(ctx, a, e4m3, km, vm, stream);
         default: return ARB_ERR_UNSUPPORTED;
     }
 }

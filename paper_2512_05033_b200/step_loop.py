@@ -14,7 +14,8 @@ work it causes:
   target cache   absorbs accepted draft steps as one chunk; generates z_t token by token for the escalated
 
 A cache may be an E4M3 cache (Cache.e4m3 = its two scales): the reduced-precision cache of a quantised draft
-(Section 5.1).  Its writes go through arb_kv_append_e4m3 and its attention through arb_attn_e4m3.
+(Section 5.1).  Its tokens go through arb_decode_step_e4m3, the chunks it absorbs through arb_kv_append_e4m3 and
+arb_attn_e4m3.
 
 Which sequences take part in a phase comes from arb_phase_lens / arb_phase_lens_tokens on the device.  A round is therefore a fixed
 list of kernel launches for given maximum step lengths and can be captured in a CUDA graph.
@@ -78,13 +79,15 @@ class StepLoop:
         at token t only sequences that take part and have t < step_lens[b] are active."""
         lens = self.ctx.phase_lens_tokens(step_lens, n_max, decisions, want=want, out=self.token_lens[name])
         for t in range(n_max):   # one launch per token: cache write, attention and length update (arb_decode_step)
-            if c.e4m3 is not None:   # the quantised cache has no fused token call: append, then decode
-                self._absorb(f"{name}[{t}]", c, k_new[t], v_new[t], q[t], lens[t], 1)
-                continue
             key = f"{name}[{t}]"
             out = self.out.get(key)
             if out is None or out.shape != q[t].shape:
                 out = self.out[key] = torch.zeros_like(q[t])
+            if c.e4m3 is not None:   # a quantised cache: the same token over codes (arb_decode_step_e4m3)
+                ks, vs = c.e4m3
+                self.ctx.decode_step_e4m3(q[t], k_new[t], v_new[t], c.k_pages, c.v_pages, ks, vs, 1.0 / ks, 1.0 / vs,
+                                          c.block_table, c.seq_lens, lens[t], out=out)
+                continue
             self.ctx.decode_step(q[t], k_new[t], v_new[t], c.k_pages, c.v_pages, c.block_table, c.seq_lens, lens[t],
                                  out=out)
 

@@ -178,3 +178,139 @@ def test_decode_step_refuses_what_does_not_fit():
     p = c.params_for(d2.q, d2.k_pages, d2.block_table, 1, flags=binding.ATTN_OVERLAP_PREVIOUS)
     with pytest.raises(binding.ArbError):
         c.decode_step(d2.q, kn2.cuda(), vn2.cuda(), d2.k_pages, d2.v_pages, d2.block_table, d2.seq_lens, d2.q_lens, params=p)
+
+
+# ---- arb_decode_step_e4m3: the same token over an E4M3 cache -------------------------------------------------------
+
+E4M3_STEP_CASES = [
+    # (B, Hq, Hkv, lengths before the token, q_lens)
+    (3, 12, 2, [15, 16, 17], [1, 1, 1]),
+    (4, 12, 2, [0, 1, 31, 32], [1, 1, 1, 1]),
+    (8, 12, 2, [1025, 2000, 3001, 777, 4096, 1, 640, 5555], [1] * 8),
+    (4, 32, 8, [4100, 9000, 33, 12000], [1, 1, 1, 1]),
+    (2, 28, 4, [3000, 150], [1, 1]),
+    (5, 16, 2, [2100, 5, 900, 77, 4000], [1, 0, 1, 0, 1]),
+    (1, 5, 1, [40000], [1]),
+    (2, 8, 8, [260, 100], [1, 1]),
+]
+KS, VS = 0.011, 0.017     # N(0,1) values / scale reach about 400: the whole range of the format is used
+
+
+def _e4m3_case(B, Hq, Hkv, sl, ql, seed, extra=4):
+    inp = wl.small_attn_case(B, Hq, Hkv, 128, BF, sl, ql, seed=seed, extra_tokens=extra)
+    kc = torch.from_numpy(oracle.e4m3_encode(inp.k_pages, 1 / KS))
+    vc = torch.from_numpy(oracle.e4m3_encode(inp.v_pages, 1 / VS))
+    for b in range(B):              # stale slots past the ends hold NaN codes: they must never reach the arithmetic
+        for pos in range(sl[b], sl[b] + extra):
+            page = int(inp.block_table[b, pos // 16])
+            kc[page, :, pos % 16, :] = 0x7f
+            vc[page, :, pos % 16, :] = 0xff
+    return inp, kc, vc
+
+
+@pytest.mark.parametrize("case", E4M3_STEP_CASES)
+def test_decode_step_e4m3_matches_quantising_append_then_attention(case):
+    B, Hq, Hkv, sl, ql = case
+    inp, kc, vc = _e4m3_case(B, Hq, Hkv, sl, ql, 900 + len(sl) + Hq)
+    k_new, v_new = _new_rows(inp, sum(ql), 9100 + Hq)
+    k_new[0, 0, :4] = torch.tensor([1e4, -1e4, 0.0, 448 * KS])          # saturation on both sides, zero, the edge
+    c = H.ctx()
+    d = inp.to("cuda")
+    dk, dv = kc.cuda(), vc.cuda()
+    out = torch.full_like(d.q, float("nan"))
+    c.decode_step_e4m3(d.q, k_new.cuda(), v_new.cuda(), dk, dv, KS, VS, 1 / KS, 1 / VS, d.block_table, d.seq_lens,
+                       d.q_lens, out=out)
+    assert c.poll_status() == 0
+    ok, ov, osl, st = oracle.kv_append_e4m3(k_new, v_new, inp.block_table, inp.seq_lens, inp.q_lens, kc, vc, 1 / KS, 1 / VS)
+    ref, st2 = oracle.attn_e4m3(inp.q, ok, ov, KS, VS, inp.block_table, osl, inp.q_lens)
+    assert st == 0 and st2 == 0
+    assert np.array_equal(d.seq_lens.cpu().numpy(), osl)
+    assert torch.equal(dk.cpu(), ok) and torch.equal(dv.cpu(), ov)       # codes: bit for bit
+    H.assert_close(out.double().cpu().numpy(), ref, BF, tight=3e-3)
+
+
+def test_decode_step_e4m3_chain_equals_the_two_calls():
+    """Twelve tokens in a row, in place, then as one CUDA graph: codes and lengths equal those the two separate
+    calls (arb_kv_append_e4m3, arb_attn_decode_e4m3) leave on a copy of the cache, rows equal the oracle's."""
+    c = H.ctx()
+    B, T = 5, 12
+    inp, kc, vc = _e4m3_case(B, 12, 2, [500, 33, 2100, 0, 1500], [1] * B, 93, extra=T + 2)
+    q = wl.normal((T, B, 12, 128), 1.0, BF, "cpu", 94)
+    kn = wl.normal((T, B, 2, 128), 1.0, BF, "cpu", 95)
+    vn = wl.normal((T, B, 2, 128), 1.0, BF, "cpu", 96)
+    d = inp.to("cuda")
+    dk, dv = kc.cuda(), vc.cuda()
+    start = (dk.clone(), dv.clone(), d.seq_lens.clone())
+    dq, dkn, dvn = q.cuda(), kn.cuda(), vn.cuda()
+    outs = [torch.full((B, 12, 128), float("nan"), dtype=BF, device="cuda") for _ in range(T)]
+    p = c.params_for(dq[0], dk, d.block_table, 1)
+
+    def chain():
+        for t in range(T):
+            c.decode_step_e4m3(dq[t], dkn[t], dvn[t], dk, dv, KS, VS, 1 / KS, 1 / VS, d.block_table, d.seq_lens,
+                               d.q_lens, out=outs[t], params=p)
+
+    chain()
+    assert c.poll_status() == 0
+    k, v, sl = kc, vc, inp.seq_lens.numpy()
+    for t in range(T):
+        k, v, sl, st = oracle.kv_append_e4m3(kn[t], vn[t], inp.block_table, sl, inp.q_lens, k, v, 1 / KS, 1 / VS)
+        ref, st2 = oracle.attn_e4m3(q[t], k, v, KS, VS, inp.block_table, sl, inp.q_lens)
+        assert st == 0 and st2 == 0
+        H.assert_close(outs[t].double().cpu().numpy(), ref, BF, tight=3e-3)
+    assert np.array_equal(d.seq_lens.cpu().numpy(), sl)
+    assert torch.equal(dk.cpu(), k) and torch.equal(dv.cpu(), v)
+    # the two separate calls on a copy of the starting cache
+    k2, v2, sl2 = (t_.clone() for t_ in start)
+    for t in range(T):
+        c.kv_append_e4m3(dkn[t], dvn[t], 1 / KS, 1 / VS, d.block_table, sl2, d.q_lens, k2, v2)
+        two = c.attn_decode_e4m3(dq[t], k2, v2, KS, VS, d.block_table, sl2, d.q_lens)
+        assert float((two.float() - outs[t].float()).abs().max()) <= 2e-2
+    assert torch.equal(k2, dk) and torch.equal(v2, dv) and torch.equal(sl2, d.seq_lens)
+    eager = [o.clone() for o in outs]
+    gr = torch.cuda.CUDAGraph()
+    for t_, s_ in zip((dk, dv, d.seq_lens), start):
+        t_.copy_(s_)
+    with torch.cuda.graph(gr):
+        chain()
+    for rep in range(2):
+        for t_, s_ in zip((dk, dv, d.seq_lens), start):
+            t_.copy_(s_)
+        for o in outs:
+            o.fill_(float("nan"))
+        gr.replay()
+        torch.cuda.synchronize()
+        for t in range(T):
+            assert torch.equal(outs[t], eager[t]), (rep, t)
+        assert np.array_equal(d.seq_lens.cpu().numpy(), sl)
+
+
+def test_decode_step_e4m3_refusals():
+    """Host-side refusals, and a token that does not fit: sequence untouched, zero row, status bit."""
+    from paper_2512_05033_b200 import binding
+    c = H.ctx()
+    inp, kc, vc = _e4m3_case(3, 12, 2, [100, 64, 300], [1, 1, 1], 97, extra=0)
+    k_new, v_new = _new_rows(inp, 3, 98)
+    d = inp.to("cuda")
+    with pytest.raises(binding.ArbError):      # a scale that is not positive
+        c.decode_step_e4m3(d.q, k_new.cuda(), v_new.cuda(), kc.cuda(), vc.cuda(), 0.0, VS, 1 / KS, 1 / VS, d.block_table,
+                           d.seq_lens, d.q_lens)
+    with pytest.raises(binding.ArbError):      # a series flag: the call writes the cache it reads
+        p = c.params_for(d.q, kc.cuda(), d.block_table, 1, flags=binding.ATTN_OVERLAP_PREVIOUS)
+        c.decode_step_e4m3(d.q, k_new.cuda(), v_new.cuda(), kc.cuda(), vc.cuda(), KS, VS, 1 / KS, 1 / VS, d.block_table,
+                           d.seq_lens, d.q_lens, params=p)
+    inp.seq_lens[1] = inp.block_table.shape[1] * 16          # full: one more token does not fit
+    d = inp.to("cuda")
+    dk, dv = kc.cuda(), vc.cuda()
+    out = torch.full_like(d.q, float("nan"))
+    c.decode_step_e4m3(d.q, k_new.cuda(), v_new.cuda(), dk, dv, KS, VS, 1 / KS, 1 / VS, d.block_table, d.seq_lens,
+                       d.q_lens, out=out)
+    assert c.poll_status() == binding.DEV_BAD_SEQ_LEN
+    ok, ov, osl, st = oracle.kv_append_e4m3(k_new, v_new, inp.block_table, inp.seq_lens, inp.q_lens, kc, vc, 1 / KS, 1 / VS)
+    assert st == oracle.BAD_SEQ_LEN
+    assert np.array_equal(d.seq_lens.cpu().numpy(), osl)
+    assert torch.equal(dk.cpu(), ok) and torch.equal(dv.cpu(), ov)
+    assert float(out[1].abs().max()) == 0.0
+    keep = torch.tensor([1, 0, 1], dtype=torch.int32)
+    ref, _ = oracle.attn_e4m3(inp.q[[0, 2]], ok, ov, KS, VS, inp.block_table, osl, keep)
+    H.assert_close(out[[0, 2]].double().cpu().numpy(), ref, BF, tight=3e-3)

@@ -376,6 +376,7 @@ def run_ours(args):
                         "note": "the same calls without ARB_ATTN_OVERLAP_PREVIOUS: every call waits for the one "
                                 "before it, which is what a token of Algorithm 1 sees"}
                 result["decode_step"] = run_decode_step(ctx, dev, peak, peak_kind)
+                result["decode_step"]["e4m3"] = run_decode_step(ctx, dev, peak, peak_kind, e4m3=True)
                 result["target_shaped_decode"] = run_target_decode(ctx, dev, peak)
                 result["step_scoring"] = run_step_scoring(ctx, dev)
                 result["mixed_loop"] = run_mixed_loop(ctx, dev)
@@ -501,22 +502,33 @@ def run_target_decode(ctx, dev, peak):
                              "pct_of_nominal_8TBs": round(100 * gbs2 / NOMINAL_HBM_GBS, 2)}}
 
 
-def run_decode_step(ctx, dev, peak, peak_kind, layers=LAYERS):
+def run_decode_step(ctx, dev, peak, peak_kind, layers=LAYERS, e4m3=False):
     """Supplementary: the single-launch decode token (arb_decode_step: cache write + attention + combine + length
     update) on the draft-shaped batch: `layers` calls per CUDA graph, each on its own KV pool and its own length
-    array (a layer's cache grows by one token per replay), every call waiting for the one before it."""
+    array (a layer's cache grows by one token per replay), every call waiting for the one before it.  e4m3: the
+    same over pools of E4M3 codes (arb_decode_step_e4m3)."""
     shape = wl.DRAFT_DECODE
     inp = wl.make_attn_inputs(shape, device=dev, seed=shape.seed, extra_tokens=2048)
-    pools = [(inp.k_pages, inp.v_pages)] + [wl.make_kv_pool(shape, inp.num_pages, dev, shape.seed * 100 + l) for l in range(1, layers)]
+    if e4m3:
+        g8 = torch.Generator(device=dev)
+        g8.manual_seed(3200)
+        pools = [tuple(torch.randint(0, 0x7f, inp.k_pages.shape, generator=g8, device=dev, dtype=torch.uint8) for _ in range(2))
+                 for _ in range(layers)]
+    else:
+        pools = [(inp.k_pages, inp.v_pages)] + [wl.make_kv_pool(shape, inp.num_pages, dev, shape.seed * 100 + l) for l in range(1, layers)]
     lens = [inp.seq_lens.clone() for _ in pools]
     k_new = wl.normal((shape.batch, shape.num_kv_heads, shape.head_dim), 1.0, shape.dtype, dev, 4401)
     v_new = wl.normal((shape.batch, shape.num_kv_heads, shape.head_dim), 1.0, shape.dtype, dev, 4402)
     out = torch.empty_like(inp.q)
-    p = ctx.params_for(inp.q, inp.k_pages, inp.block_table, 1)
+    p = ctx.params_for(inp.q, pools[0][0], inp.block_table, 1)
 
     def step():
         for (k, v), sl in zip(pools, lens):
-            ctx.decode_step(inp.q, k_new, v_new, k, v, inp.block_table, sl, inp.q_lens, out=out, params=p)
+            if e4m3:
+                ctx.decode_step_e4m3(inp.q, k_new, v_new, k, v, 0.01, 0.01, 100.0, 100.0, inp.block_table, sl, inp.q_lens,
+                                     out=out, params=p)
+            else:
+                ctx.decode_step(inp.q, k_new, v_new, k, v, inp.block_table, sl, inp.q_lens, out=out, params=p)
 
     step()
     torch.cuda.synchronize()
@@ -526,11 +538,16 @@ def run_decode_step(ctx, dev, peak, peak_kind, layers=LAYERS):
     ms = statistics.median(time_repeated(g.replay, 20, 5, min_total_ms=60.0)) / 20   # about 600 tokens appended per layer
     us = ms / layers * 1e3
     b = attn_bytes(shape, inp.seq_lens.cpu().to(torch.int64) + 300, inp.q_lens.cpu().to(torch.int64))
-    nbytes = b["total"] + 4 * shape.batch * shape.num_kv_heads * shape.head_dim * 2   # + the new rows, read and written
+    rows = shape.batch * shape.num_kv_heads * shape.head_dim
+    if e4m3:   # codes: one byte per cache element; the new rows are read as bf16 and written as codes
+        nbytes = b["kv"] // 2 + b["qo"] + b["table"] + 2 * rows * 3
+    else:
+        nbytes = b["total"] + 4 * rows * 2   # + the new rows, read and written
     assert ctx.poll_status() == 0
+    name = "arb_decode_step_e4m3" if e4m3 else "arb_decode_step"
     return {"us_per_call": round(us, 3), "kv_tokens": b["tokens"],
-            "roofline": hbm_roofline("decode_step_kernel", nbytes, us, peak, peak_kind),
-            "note": f"{layers} arb_decode_step calls per CUDA graph, none overlapped: what a token of Algorithm 1 costs per layer"}
+            "roofline": hbm_roofline("decode_step_kernel<E4M3>" if e4m3 else "decode_step_kernel", nbytes, us, peak, peak_kind),
+            "note": f"{layers} {name} calls per CUDA graph, none overlapped: what a token of Algorithm 1 costs per layer"}
 
 
 def run_e4m3_chunk(ctx, dev):

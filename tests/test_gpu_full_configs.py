@@ -172,6 +172,37 @@ def test_draft_shaped_decode_step_full():
     assert torch.equal(d.k_pages.cpu(), k_ref) and torch.equal(d.v_pages.cpu(), v_ref)
 
 
+def test_draft_shaped_decode_step_e4m3_full():
+    """arb_decode_step_e4m3 on the draft-shaped batch: two tokens in a row on one E4M3 cache; codes bit for bit,
+    lengths exact, every row."""
+    shape = wl.DRAFT_DECODE
+    inp = wl.make_attn_inputs(shape, extra_tokens=8)
+    ks, vs = 0.012, 0.015
+    kc = torch.from_numpy(oracle.e4m3_encode(inp.k_pages, 1 / ks))
+    vc = torch.from_numpy(oracle.e4m3_encode(inp.v_pages, 1 / vs))
+    d = inp.to("cuda")
+    dk, dv = kc.cuda(), vc.cuda()
+    c = H.ctx()
+    sl = inp.seq_lens.numpy().copy()
+    ones = torch.ones(shape.batch, dtype=torch.int32)
+    outs, news = [], []
+    for t in range(2):
+        q = wl.normal((shape.batch, shape.num_q_heads, shape.head_dim), 1.0, BF, "cpu", 9400 + t)
+        kn = wl.normal((shape.batch, shape.num_kv_heads, shape.head_dim), 1.0, BF, "cpu", 9500 + t)
+        vn = wl.normal((shape.batch, shape.num_kv_heads, shape.head_dim), 1.0, BF, "cpu", 9600 + t)
+        news.append((q, kn, vn))
+        outs.append(c.decode_step_e4m3(q.cuda(), kn.cuda(), vn.cuda(), dk, dv, ks, vs, 1 / ks, 1 / vs, d.block_table,
+                                       d.seq_lens, d.q_lens))
+    assert c.poll_status() == 0
+    for (q, kn, vn), out in zip(news, outs):
+        kc, vc, sl, st = oracle.kv_append_e4m3(kn, vn, inp.block_table, sl, ones, kc, vc, 1 / ks, 1 / vs)
+        ref, st2 = oracle.attn_e4m3(q, kc, vc, ks, vs, inp.block_table, sl, ones)
+        assert st == 0 and st2 == 0
+        H.assert_close(out.double().cpu().numpy(), ref, BF, tight=3e-3)
+    assert np.array_equal(d.seq_lens.cpu().numpy(), sl)
+    assert torch.equal(dk.cpu(), kc) and torch.equal(dv.cpu(), vc)
+
+
 def test_step_scoring_full_over_the_e4m3_cache():
     """arb_attn_e4m3 on the step-scoring batch at full size (pools quantised by the oracle), every element."""
     shape = wl.STEP_SCORING

@@ -49,13 +49,14 @@ constexpr int kStages = 2;
 constexpr int kSoftmaxThreads = 128;        // per row tile
 constexpr int kThreads = 3 * kSoftmaxThreads;   // two softmax groups and a group of service warps; registers are
                                                 // handed out per 128 threads, so the third group's spare warps cost none
-constexpr int kTmaWarp = 8, kMmaWarp = 9, kVWarp = 10;   // warp 11 has no role
+constexpr int kTmaWarp = 8, kMmaWarp = 9, kVWarp = 10, kPvWarp = 11;
 constexpr int kHalfBytes = 128 * 128;      // [128 rows x 64 bf16]: one 128-byte-swizzled half tile
 constexpr int kTileBytes = 2 * kHalfBytes;  // [128 x 128] bf16
 constexpr int kBoxBytes = kPage * 128;      // one TMA box: 16 rows x 64 bf16
 constexpr int kStagePages = 6;              // E4M3: pages of codes in flight per operand
 constexpr int kCodePageBytes = kPage * kD;  // 2 KB: one (page, kv head) tile of codes
-constexpr uint32_t kTmemCols = 512;         // S of tile A: columns 0..127, S of B: 128..255, O of A: 256..383, O of B: 384..511
+constexpr uint32_t kTmemCols = 512;         // S (shared): columns 0..127, P of group A: 128..191, of B: 192..255,
+constexpr uint32_t kPCol = 128;             // O of group A: 256..383, of B: 384..511
 constexpr uint32_t kOCol = 256;
 constexpr float kRescaleThreshold = 8.0f;   // log2 units
 constexpr int kItemSlots = 8;               // work items announced ahead of their use
@@ -106,6 +107,8 @@ struct Bars {
     uint64_t s_full[2];          // S = Q K^T of row tile A / B is in TMEM
     uint64_t p_full[2];          // P of row tile A / B is in TMEM (over S)
     uint64_t o_full[2];          // O += P V of row tile A / B has completed
+    uint64_t s_free[2];          // group A / B holds the S it was given in registers: the S region is free
+    uint64_t ml_full;            // an item with one row tile: both softmax groups have left their (max, sum)
     uint64_t item_full[kItemSlots];   // the producer warp has fetched the next work item
     uint64_t item_empty[kItemSlots];  // the MMA thread, the V producer and the softmax threads have read it
     uint64_t code_full[2][kStagePages];   // E4M3: a page of codes of K / of V has landed in its staging slot
@@ -479,9 +482,12 @@ chunk_mma_kernel(const MmaArgs a, const __grid_constant__ CUtensorMap k_map, con
         mbar_init(&bars->p_full[1], kSoftmaxThreads);
         mbar_init(&bars->o_full[0], 1);
         mbar_init(&bars->o_full[1], 1);
+        mbar_init(&bars->s_free[0], kSoftmaxThreads);
+        mbar_init(&bars->s_free[1], kSoftmaxThreads);
+        mbar_init(&bars->ml_full, 2 * kSoftmaxThreads);
         for (int i = 0; i < kItemSlots; ++i) {
             mbar_init(&bars->item_full[i], 1);
-            mbar_init(&bars->item_empty[i], 2 + 2 * kSoftmaxThreads);   // MMA thread, V warp, softmax threads
+            mbar_init(&bars->item_empty[i], 3 + 2 * kSoftmaxThreads);   // the two MMA threads, V warp, softmax threads
         }
         for (int i = 0; i < kStagePages; ++i) {
             mbar_init(&bars->code_full[0][i], 1);
@@ -649,15 +655,21 @@ chunk_mma_kernel(const MmaArgs a, const __grid_constant__ CUtensorMap k_map, con
             }
         }
     } else if (warp == kMmaWarp) {
-        // ====================================== MMA issue ===========================================
-        // Per KV tile: S_A = Q_A K^T, S_B = Q_B K^T, then -- as each softmax group delivers its P --
-        // O_A += P_A V and O_B += P_B V.  The next tile's Q K^T of a row tile is issued right after
-        // that row tile's P V, so the tensor core works for one row tile while the other one's
-        // softmax group is busy.
+        // ================================ MMA issue: S = Q K^T ======================================
+        // An item is a sequence of units, each the work of one softmax group on one KV tile: for a pair of row tiles
+        // unit u is (row tile u % 2, KV tile u / 2); for a single row tile it is (row tile A, KV tile u), the KV tiles
+        // alternating between the two groups, which merge their two O in the epilogue.  All units share ONE S region
+        // in TMEM; P and O have a region per group.  So S of unit u + 1 is computed as soon as the group of unit u holds
+        // S of unit u in registers, under that group's exponentials, and the softmax groups never wait for a product
+        // of their own.  The two kinds of product are issued by two threads (this one: S = Q K^T; warp kPvWarp:
+        // O += P V): issuing an MMA holds the thread until the tensor core has room for it, and finding a barrier
+        // complete costs about a hundred cycles, so one thread issuing both kinds leaves the tensor core idle while it
+        // looks at its barriers.
         if (lane == 0) {
-            constexpr uint32_t idesc_qk = instr_desc(false, E4M3), idesc_pv = instr_desc(true, E4M3);
+            constexpr uint32_t idesc_qk = instr_desc(false, E4M3);
             const uint32_t q_addr = smem_u32(q_s);
-            uint32_t it = 0, nitem = 0, nproc = 0, itg[2] = {0u, 0u};  // KV tiles so far: all, per row tile
+            uint32_t it = 0, nitem = 0, nproc = 0;   // KV tiles so far, items, items with work
+            uint32_t nfree[2] = {0u, 0u};            // S loads so far per group
             Item w;
             for (;; ++nitem) {
                 const uint32_t slot = nitem % kItemSlots, qpar = (nitem / kItemSlots) & 1u;
@@ -668,56 +680,71 @@ chunk_mma_kernel(const MmaArgs a, const __grid_constant__ CUtensorMap k_map, con
                 if (w.ntiles == 0) continue;   // a part the pair sees nothing of: no role does anything for it
                 mbar_wait(&bars->q_full, nproc & 1u, abort, a.status);
                 ++nproc;
-                const bool has_b = w.rows[1] > 0;
-                // S of row tile g for KV tile `itx`: 8 steps of 16 dims, 4 per 64-dim half; K-major
-                // operands, SBO = 8 rows
-                auto issue_qk = [&](int g, uint32_t itx) {
-                    const uint32_t s = itx % kStages;
+                const bool lone = w.rows[1] == 0;
+                const int units = lone ? w.ntiles : 2 * w.ntiles;
+                // S of unit u: 8 steps of 16 dims, 4 per 64-dim half; K-major operands, SBO = 8 rows.  A K stage is
+                // waited for by the first unit that reads it and released behind the last one.
+                auto issue_qk = [&](int u) {
+                    const uint32_t itx = it + (lone ? u : (u >> 1)), s = itx % kStages;
+                    const int g = u & 1, qt = lone ? 0 : g;
+                    if (lone || g == 0) mbar_wait(&bars->k_full[s], (itx / kStages) & 1u, abort, a.status);
                     const uint32_t k_addr = smem_u32(k_s + s * kTileBytes);
                     tc_fence_after();
 #pragma unroll
                     for (int ks = 0; ks < kD / 16; ++ks) {
                         const uint32_t off = (ks >> 2) * kHalfBytes + (ks & 3) * 32;
-                        mma_f16_ss(tmem + g * kBN, smem_desc(q_addr + g * kTileBytes + off, 16, 1024),
+                        mma_f16_ss(tmem, smem_desc(q_addr + qt * kTileBytes + off, 16, 1024),
                                    smem_desc(k_addr + off, 16, 1024), idesc_qk, ks > 0 ? 1u : 0u);
                     }
                     mma_commit(&bars->s_full[g]);
+                    if (lone || g == 1) mma_commit(&bars->k_empty[s]);
                 };
-                // O of row tile g += P V for KV tile `itx`: 8 steps of 16 keys; P from TMEM (first 64
-                // columns of the tile's S, 8 columns per step); V MN-major: 64-dim halves LBO apart,
-                // 8-key groups SBO apart
-                auto issue_pv = [&](int g, uint32_t itx, bool first) {
-                    const uint32_t s = itx % kStages;
+                issue_qk(0);
+                for (int u = 0; u < units; ++u) {
+                    const int g = u & 1;
+                    mbar_wait(&bars->s_free[g], nfree[g] & 1u, abort, a.status);   // S of unit u is in registers
+                    ++nfree[g];
+                    if (u + 1 < units) issue_qk(u + 1);
+                }
+                it += w.ntiles;
+            }
+        }
+        __syncwarp();
+    } else if (warp == kPvWarp) {
+        // ================================ MMA issue: O += P V =======================================
+        if (lane == 0) {
+            constexpr uint32_t idesc_pv = instr_desc(true, E4M3);
+            uint32_t it = 0, nitem = 0, itg[2] = {0u, 0u};  // KV tiles so far, items, units so far per group
+            Item w;
+            for (;; ++nitem) {
+                const uint32_t slot = nitem % kItemSlots, qpar = (nitem / kItemSlots) & 1u;
+                if (!mbar_wait(&bars->item_full[slot], qpar, abort, a.status)) break;
+                const int item = bars->item_id[slot];
+                mbar_arrive(&bars->item_empty[slot]);
+                if (!get_item<G>(item, total, pl, B, Hkv, a, w)) break;
+                if (w.ntiles == 0) continue;
+                const bool lone = w.rows[1] == 0;
+                const int units = lone ? w.ntiles : 2 * w.ntiles;
+                // O of the unit's group += P V: 8 steps of 16 keys; P from the group's TMEM columns (two keys per
+                // column, 8 columns per step); V MN-major: 64-dim halves LBO apart, 8-key groups SBO apart.  A V stage
+                // is waited for by the first unit that reads it and released behind the last one.
+                for (int u = 0; u < units; ++u) {
+                    const uint32_t itx = it + (lone ? u : (u >> 1)), s = itx % kStages;
+                    const int g = u & 1;
+                    if (lone || g == 0) mbar_wait(&bars->v_full[s], (itx / kStages) & 1u, abort, a.status);
                     const uint32_t v_addr = smem_u32(v_s + s * kTileBytes);
                     mbar_wait(&bars->p_full[g], itg[g] & 1u, abort, a.status);
                     tc_fence_after();
 #pragma unroll
                     for (int ks = 0; ks < kBN / 16; ++ks)
-                        mma_f16_ts(tmem + kOCol + g * kBN, tmem + g * kBN + ks * 8,
+                        mma_f16_ts(tmem + kOCol + g * kBN, tmem + kPCol + g * (kBN / 2) + ks * 8,
                                    smem_desc(v_addr + ks * 2 * 1024, kHalfBytes, 1024), idesc_pv,
-                                   (!first || ks > 0) ? 1u : 0u);
+                                   (u >= 2 || ks > 0) ? 1u : 0u);
                     mma_commit(&bars->o_full[g]);
                     ++itg[g];
-                };
-                mbar_wait(&bars->k_full[it % kStages], (it / kStages) & 1u, abort, a.status);
-                issue_qk(0, it);
-                if (has_b) issue_qk(1, it);
-                mma_commit(&bars->k_empty[it % kStages]);
-                for (int j = 0; j < w.ntiles; ++j, ++it) {
-                    const uint32_t s = it % kStages, par = (it / kStages) & 1u;
-                    const bool more = j + 1 < w.ntiles;
-                    if (more) mbar_wait(&bars->k_full[(it + 1) % kStages], ((it + 1) / kStages) & 1u, abort, a.status);
-                    mbar_wait(&bars->v_full[s], par, abort, a.status);
-                    issue_pv(0, it, j == 0);
-                    if (more) issue_qk(0, it + 1);
-                    if (has_b) {
-                        issue_pv(1, it, j == 0);
-                        if (more) issue_qk(1, it + 1);
-                    }
-                    // everything issued so far has read V of this tile and K of the next one
-                    mma_commit(&bars->v_empty[s]);
-                    if (more) mma_commit(&bars->k_empty[(it + 1) % kStages]);
+                    if (lone || g == 1) mma_commit(&bars->v_empty[s]);
                 }
+                it += w.ntiles;
             }
         }
         __syncwarp();
@@ -726,11 +753,13 @@ chunk_mma_kernel(const MmaArgs a, const __grid_constant__ CUtensorMap k_map, con
         // two groups of 128 threads: group g owns row tile g; thread tg of a group owns TMEM lane tg
         const int grp = warp >> 2, tg = tid & (kSoftmaxThreads - 1);
         const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;  // this warp's TMEM lane quadrant
-        const uint32_t s_tmem = tmem + lane_base + grp * kBN;
+        const uint32_t s_tmem = tmem + lane_base;                                  // S: one region for both groups
+        const uint32_t p_tmem = tmem + lane_base + kPCol + grp * (kBN / 2);        // this group's P
         const uint32_t o_tmem = tmem + lane_base + kOCol + grp * kBN;
         char *q_tile = q_s + grp * kTileBytes;
         const int swz = tg & 7;
-        uint32_t it = 0, itg = 0, nitem = 0;  // KV tiles so far: of all items, of items that had this row tile
+        uint32_t it = 0, itg = 0, nitem = 0;  // KV tiles so far: of all items, of those this group has worked on
+        uint32_t nlone = 0;                   // items with one row tile so far
         Item w;
         for (;; ++nitem) {
             const uint32_t slot = nitem % kItemSlots, qpar = (nitem / kItemSlots) & 1u;
@@ -739,14 +768,17 @@ chunk_mma_kernel(const MmaArgs a, const __grid_constant__ CUtensorMap k_map, con
             mbar_arrive(&bars->item_empty[slot]);
             if (!get_item<G>(item, total, pl, B, Hkv, a, w)) break;
             if (w.ntiles == 0) continue;   // a part the pair sees nothing of
-            const int rows_here = w.rows[grp];
+            // An item with one row tile is worked on by both groups: even KV tiles by group A, odd ones by group B,
+            // each with an O of its own, merged in the epilogue.
+            const bool lone = w.rows[1] == 0;
+            const int rows_here = lone ? w.rows[0] : w.rows[grp];
             const bool row_ok = tg < rows_here;
-            const int r = min(w.r_begin + grp * kBM + tg, w.rows_total - 1);
+            const int r = min(w.r_begin + (lone ? 0 : grp * kBM) + tg, w.rows_total - 1);
             const int tok = r / G, head = r - tok * G;
             const int lim = w.L - w.n + tok + 1;  // keys this row may see
             const size_t grow = ((size_t)(w.qrow0 + tok) * a.Hq + w.kvh * G + head) * kD;
             // ---- Q tile: row `tg`, 16 chunks of 8 dims, chunk c of a half stored at c ^ (row & 7)
-            {
+            if (!(lone && grp == 1)) {   // (the second group of such an item reads Q tile A as well)
                 const uint4 *src = reinterpret_cast<const uint4 *>(a.q + grow * 2);
 #pragma unroll
                 for (int c = 0; c < 16; ++c) {
@@ -758,15 +790,14 @@ chunk_mma_kernel(const MmaArgs a, const __grid_constant__ CUtensorMap k_map, con
                     *reinterpret_cast<uint4 *>(q_tile + (c >> 3) * kHalfBytes + tg * 128 + (((c & 7) ^ swz) << 4)) = v;
                 }
                 fence_async_smem();
-                mbar_arrive(&bars->q_full);
             }
-            if (rows_here == 0) {  // this item has no second row tile: nothing is issued for it
-                it += w.ntiles;
-                continue;
-            }
+            mbar_arrive(&bars->q_full);
             float m_used = -INFINITY, l_sum = 0.f;
-            for (int j = 0; j < w.ntiles; ++j, ++it, ++itg) {
-                const uint32_t s = it % kStages, par = (it / kStages) & 1u;
+            const uint32_t it0 = it;
+            it += w.ntiles;
+            const int my_tiles = lone ? (w.ntiles + 1 - grp) / 2 : w.ntiles;   // KV tiles this group works on
+            for (int j = lone ? grp : 0, jt = 0; j < w.ntiles; j += lone ? 2 : 1, ++itg, ++jt) {
+                const uint32_t s = (it0 + j) % kStages, par = ((it0 + j) / kStages) & 1u;
                 const int key0 = (w.t0 + j) * kBN;
                 const int nvis = lim - key0;  // columns < nvis are visible to this row (may be <= 0)
                 mbar_wait(&bars->s_full[grp], itg & 1u, abort, a.status);
@@ -778,6 +809,8 @@ chunk_mma_kernel(const MmaArgs a, const __grid_constant__ CUtensorMap k_map, con
                 tmem_ld32<64>(s_tmem + 64, v);
                 tmem_ld32<96>(s_tmem + 96, v);
                 tmem_wait_ld();
+                tc_fence_before();
+                mbar_arrive(&bars->s_free[grp]);   // the next unit's S may be computed
                 if (nvis < kBN) {  // causal edge or end of the sequence: hidden keys weigh exp2(-inf) = 0
 #pragma unroll
                     for (int k = 0; k < kBN; ++k)
@@ -796,13 +829,17 @@ chunk_mma_kernel(const MmaArgs a, const __grid_constant__ CUtensorMap k_map, con
                 bool rescale = false;
                 if (m_tile > m_used + kRescaleThreshold || (m_used == -INFINITY && m_tile > -INFINITY)) {
                     factor = fast_exp2(m_used - m_tile);  // 0 the first time
-                    rescale = j > 0;
+                    rescale = m_used > -INFINITY;          // (nothing has been accumulated before the first visible key)
                     l_sum *= factor;
                     m_used = m_tile;
                 }
+                // this group's previous product must have completed before its P is overwritten or its O rescaled
+                // (it was issued when the group delivered that P, a whole softmax pass ago)
+                if (jt > 0) {
+                    mbar_wait(&bars->o_full[grp], (itg - 1u) & 1u, abort, a.status);
+                    tc_fence_after();
+                }
                 if (__any_sync(0xffffffffu, rescale)) {
-                    // O of the previous tiles is complete: this tile's S was issued, and committed,
-                    // after the previous tile's second product of this row tile
 #pragma unroll 1
                     for (int c4 = 0; c4 < 4; ++c4) {
                         uint32_t o[32];
@@ -836,7 +873,7 @@ chunk_mma_kernel(const MmaArgs a, const __grid_constant__ CUtensorMap k_map, con
                         pk[k] = E4M3 ? pack_f16(e0, e1) : pack_bf16(e0, e1);
                         l2[k & 3] = add_f32x2(l2[k & 3], pack_f32x2(e0, e1));
                     }
-                    tmem_st16(s_tmem + c4 * 16, pk);
+                    tmem_st16(p_tmem + c4 * 16, pk);
                 }
                 {
                     float x0, x1, y0, y1;
@@ -848,7 +885,7 @@ chunk_mma_kernel(const MmaArgs a, const __grid_constant__ CUtensorMap k_map, con
                 // ---- V rows past the last visible key of the item (stale slots, pages never loaded)
                 //      must not reach the tensor core, not even times zero
                 const int nvalid = w.kv_len - key0;
-                if (nvalid < kBN && grp == 0) {   // group A always exists and its P is waited for first
+                if (nvalid < kBN && (grp == 0 || lone)) {   // the P of group A (of a pair) is waited for first
                     mbar_wait(&bars->v_full[s], par, abort, a.status);
                     if (tg >= nvalid) {
                         char *vrow = v_s + s * kTileBytes + tg * 128;
@@ -864,9 +901,71 @@ chunk_mma_kernel(const MmaArgs a, const __grid_constant__ CUtensorMap k_map, con
                 mbar_arrive(&bars->p_full[grp]);
             }
             // ---- epilogue: O / l, bf16, one 256-byte row per thread
-            mbar_wait(&bars->o_full[grp], (itg - 1u) & 1u, abort, a.status);
+            if (my_tiles > 0) mbar_wait(&bars->o_full[grp], (itg - 1u) & 1u, abort, a.status);
             tc_fence_after();
             const bool row_in = ARB_IN_RANGE(a.status, w.qrow0 + tok, a.rows);
+            if (lone) {
+                // The two groups hold O, max and sum over the even and over the odd KV tiles of the same rows.  They
+                // exchange (max, sum) through the shared memory of Q tile B, which such an item does not use, and
+                // each merges and writes 64 of the 128 dimensions: thread tg of either group owns TMEM lane tg and
+                // reads that lane of both O.
+                float2 *ml = reinterpret_cast<float2 *>(q_s + kTileBytes);
+                ml[grp * kSoftmaxThreads + tg] = make_float2(m_used, l_sum);
+                tc_fence_before();
+                mbar_arrive(&bars->ml_full);
+                mbar_wait(&bars->ml_full, nlone & 1u, abort, a.status);
+                ++nlone;
+                tc_fence_after();
+                const float2 ml0 = ml[tg], ml1 = ml[kSoftmaxThreads + tg];
+                const bool two = w.ntiles > 1;                       // else group B has worked on nothing: its O is undefined
+                const float m = fmaxf(ml0.x, two ? ml1.x : -INFINITY);
+                const float w0 = ml0.x == -INFINITY ? 0.f : fast_exp2(ml0.x - m);
+                const float w1 = (!two || ml1.x == -INFINITY) ? 0.f : fast_exp2(ml1.x - m);
+                const float l = ml0.y * w0 + (two ? ml1.y * w1 : 0.f);
+                const bool slot_in = !w.split || ARB_IN_RANGE(a.status, w.slot, a.split_cap);
+                float *po = a.split_ws + (size_t)(w.split && slot_in ? w.slot : 0) * kSlotFloats;
+                const float norm = w.split ? (E4M3 ? a.v_scale : 1.0f) : (E4M3 ? a.v_scale : 1.0f) / l;
+                const uint32_t oa = tmem + lane_base + kOCol, ob = oa + kBN;
+                uint4 *dst = reinterpret_cast<uint4 *>(a.out + grow * 2);
+#pragma unroll 1
+                for (int c4 = 2 * grp; c4 < 2 * grp + 2; ++c4) {
+                    uint32_t va[32];
+                    float o[32];
+                    tmem_ld32(oa + c4 * 32, va);
+                    tmem_wait_ld();
+                    const float n0 = w0 * norm, n1 = w1 * norm;
+#pragma unroll
+                    for (int k = 0; k < 32; ++k) o[k] = __uint_as_float(va[k]) * n0;
+                    if (two) {
+                        tmem_ld32(ob + c4 * 32, va);
+                        tmem_wait_ld();
+#pragma unroll
+                        for (int k = 0; k < 32; ++k) o[k] = fmaf(__uint_as_float(va[k]), n1, o[k]);
+                    }
+                    if (w.split) {
+                        if (row_ok && slot_in) {
+#pragma unroll
+                            for (int qd = 0; qd < 8; ++qd)
+                                *reinterpret_cast<float4 *>(po + ((size_t)(c4 * 8 + qd) * kBM + tg) * 4) =
+                                    make_float4(o[qd * 4], o[qd * 4 + 1], o[qd * 4 + 2], o[qd * 4 + 3]);
+                        }
+                    } else if (row_ok && row_in) {
+#pragma unroll
+                        for (int qd = 0; qd < 4; ++qd) {
+                            uint4 o4;
+                            o4.x = pack_bf16(o[qd * 8 + 0], o[qd * 8 + 1]);
+                            o4.y = pack_bf16(o[qd * 8 + 2], o[qd * 8 + 3]);
+                            o4.z = pack_bf16(o[qd * 8 + 4], o[qd * 8 + 5]);
+                            o4.w = pack_bf16(o[qd * 8 + 6], o[qd * 8 + 7]);
+                            dst[c4 * 4 + qd] = o4;
+                        }
+                    }
+                }
+                if (w.split && grp == 0 && row_ok && slot_in)
+                    *reinterpret_cast<float2 *>(po + (size_t)kBM * kD + tg * 2) = make_float2(m, l);
+                tc_fence_before();
+                continue;
+            }
             if (w.split) {
                 // one part of a split sequence: leave the un-normalised O row and its (max, sum)
                 const bool slot_in = ARB_IN_RANGE(a.status, w.slot + grp, a.split_cap);

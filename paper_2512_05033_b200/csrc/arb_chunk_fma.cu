@@ -30,46 +30,23 @@ struct ChunkArgs {
     int n_lo, n_hi;  // this kernel owns the sequences with n_lo <= q_len <= n_hi ...
     int skip_rows;   // ... except valid ones with q_len * group >= skip_rows (> 0): the tensor-core kernel has them
     const int *needed;  // with skip_rows > 0: written by the tensor-core kernel, 0 = nothing is left for this one
+    int jobs;        // (query row, kv head) pairs: total_q * Hkv; the CTAs take them in turn
     float scale_log2;
 };
 
+// One (query row, kv head) pair; every thread of the block takes part.  rec: [NGROUPS][REC] floats of shared
+// memory; row0: the prefix sums of the q_lens.
 template <typename T, int D, int G>
-__global__ void __launch_bounds__(kThreads) chunk_fma_kernel(const ChunkArgs a) {
+__device__ void chunk_fma_job(const ChunkArgs &a, int job, float *rec, const int *row0) {
     constexpr int EPL = Elt<T>::kPerVec;
     constexpr int ROW_BYTES = D * (int)sizeof(T);
     constexpr int LPR = ROW_BYTES / 16;
     constexpr int RPP = 32 / LPR;
     constexpr int NGROUPS = kWarps * RPP;
     constexpr int REC = G * (D + 2);  // floats per group record: m[G], l[G], o[G][D]
-
-    extern __shared__ float sm[];
-    float *rec = sm;                                      // [NGROUPS][REC]
-    int *row0 = reinterpret_cast<int *>(sm + NGROUPS * REC);  // [B + 1]
-
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int B = a.batch;
-    const int row = blockIdx.x / a.Hkv, kvh = blockIdx.x - row * a.Hkv;
-    pdl_enter();
-    if (a.skip_rows > 0 && a.needed != nullptr && *a.needed == 0) return;  // the usual case: every chunk was large
-
-    if (tid == 0) row0[0] = 0;
-    for (int b = tid; b < B; b += kThreads) row0[b + 1] = max(a.q_lens[b], 0);
-    __syncthreads();
-    if (warp == 0) {
-        int carry = 0;
-        for (int b0 = 0; b0 < B; b0 += 32) {
-            const int b = b0 + lane;
-            int v = b < B ? row0[b + 1] : 0;
-#pragma unroll
-            for (int off = 1; off < 32; off <<= 1) {
-                const int t = __shfl_up_sync(0xffffffffu, v, off);
-                if (lane >= off) v += t;
-            }
-            if (b < B) row0[b + 1] = v + carry;
-            carry += __shfl_sync(0xffffffffu, v, 31);
-        }
-    }
-    __syncthreads();
+    const int row = job / a.Hkv, kvh = job - row * a.Hkv;
     if (row >= row0[B]) return;
     int lo = 0, hi = B;  // largest b with row0[b] <= row
     while (hi - lo > 1) {
@@ -182,6 +159,49 @@ __global__ void __launch_bounds__(kThreads) chunk_fma_kernel(const ChunkArgs a) 
 }
 
 template <typename T, int D, int G>
+__global__ void __launch_bounds__(kThreads) chunk_fma_kernel(const ChunkArgs a) {
+    constexpr int ROW_BYTES = D * (int)sizeof(T);
+    constexpr int LPR = ROW_BYTES / 16;
+    constexpr int RPP = 32 / LPR;
+    constexpr int NGROUPS = kWarps * RPP;
+    constexpr int REC = G * (D + 2);
+
+    extern __shared__ float sm[];
+    float *rec = sm;                                      // [NGROUPS][REC]
+    int *row0 = reinterpret_cast<int *>(sm + NGROUPS * REC);  // [B + 1]
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int B = a.batch;
+    pdl_enter();
+    if (a.skip_rows > 0 && a.needed != nullptr && *a.needed == 0) return;  // the usual case: every chunk was large
+
+    if (tid == 0) row0[0] = 0;
+    for (int b = tid; b < B; b += kThreads) row0[b + 1] = max(a.q_lens[b], 0);
+    __syncthreads();
+    if (warp == 0) {
+        int carry = 0;
+        for (int b0 = 0; b0 < B; b0 += 32) {
+            const int b = b0 + lane;
+            int v = b < B ? row0[b + 1] : 0;
+#pragma unroll
+            for (int off = 1; off < 32; off <<= 1) {
+                const int t = __shfl_up_sync(0xffffffffu, v, off);
+                if (lane >= off) v += t;
+            }
+            if (b < B) row0[b + 1] = v + carry;
+            carry += __shfl_sync(0xffffffffu, v, 31);
+        }
+    }
+    __syncthreads();
+    // the grid is bounded (a call whose chunks all went to the tensor cores would otherwise start, and end at once,
+    // one CTA per query row and kv head): the CTAs take the jobs in turn
+    for (int job = blockIdx.x; job < a.jobs; job += gridDim.x) {
+        chunk_fma_job<T, D, G>(a, job, rec, row0);
+        __syncthreads();   // the records are free again
+    }
+}
+
+template <typename T, int D, int G>
 arb_status launch_one(Ctx *ctx, const ChunkArgs &a, int total_q, cudaStream_t stream) {
     constexpr int LPR = D * (int)sizeof(T) / 16;
     constexpr int NGROUPS = kWarps * (32 / LPR);
@@ -194,7 +214,8 @@ arb_status launch_one(Ctx *ctx, const ChunkArgs &a, int total_q, cudaStream_t st
             return ARB_ERR_CUDA;
         attr_set[ctx->device & 63] = true;
     }
-    const cudaError_t err = launch_pdl(chunk_fma_kernel<T, D, G>, dim3(total_q * a.Hkv), dim3(kThreads), smem, stream, a);
+    const int grid = a.jobs < 8 * ctx->num_sms ? a.jobs : 8 * ctx->num_sms;
+    const cudaError_t err = launch_pdl(chunk_fma_kernel<T, D, G>, dim3(grid), dim3(kThreads), smem, stream, a);
     ctx->launches++;
     return err == cudaSuccess ? ARB_OK : ARB_ERR_CUDA;
 }
@@ -239,6 +260,7 @@ arb_status launch_chunk_fma(Ctx *ctx, const arb_attn_params &p, const void *q, c
     a.n_hi = n_hi;
     a.skip_rows = skip_rows;
     a.needed = needed;
+    a.jobs = p.total_q * p.num_kv_heads;
     const float scale = p.softmax_scale > 0.f ? p.softmax_scale : 1.0f / sqrtf((float)p.head_dim);
     a.scale_log2 = scale * 1.4426950408889634f;
     const int g = p.num_q_heads / p.num_kv_heads;

@@ -8,21 +8,26 @@
 // both row tiles use every K/V tile that is loaded.  Per row tile and KV tile:
 //
 //     S = Q K^T      tcgen05.mma, A = Q tile, B = K tile, both K-major in shared memory (128-byte
-//                    swizzle), fp32 accumulator in the row tile's 128 TMEM columns for S
-//     P = exp2(scale * S - m)   by the row tile's 128 softmax threads, one TMEM lane (= query row)
+//                    swizzle), fp32 accumulator in the 128 TMEM columns for S
+//     P = exp2(scale * S - m)   by a softmax group of 128 threads, one TMEM lane (= query row)
 //                    each: tcgen05.ld, causal / length mask, row max, exponentials; P, rounded to
-//                    bf16, overwrites S in place (tcgen05.st, two keys per column)
+//                    bf16, goes to the group's own TMEM columns (tcgen05.st, two keys per column)
 //     O += P V       tcgen05.mma with P as the TMEM A operand and the V tile read MN-major straight
-//                    from its page layout; fp32 accumulator in the row tile's 128 TMEM columns for O
+//                    from its page layout; fp32 accumulator in the group's 128 TMEM columns for O
 //
-// TMEM: S_A 0-127, S_B 128-255, O_A 256-383, O_B 384-511.  The MMA thread interleaves the two row
-// tiles (P V of A, next Q K^T of A, P V of B, next Q K^T of B), so the tensor core works for one
-// row tile while the other one's softmax group is busy.  The running max is lazy: O is rescaled
+// TMEM: S 0-127 (one region for both groups), P_A 128-191, P_B 192-255, O_A 256-383, O_B 384-511.  The
+// work of an item is a sequence of units (one group on one KV tile; the groups alternate).  S of a unit is
+// wanted only until its group holds it in registers, so one S region serves both groups, and with P in
+// columns of its own the next unit's Q K^T runs under this unit's exponentials: a softmax group goes from
+// one unit to its next without waiting for a product.  Q K^T and P V are issued by two threads of two
+// warps, so that neither kind waits while the other thread looks at its barriers.  An item with a single row
+// tile gives its KV tiles to the two groups in turn (both against Q tile A); they merge their two O in the
+// epilogue.  The running max is lazy: O is rescaled
 // (tcgen05.ld / st) only when a row's max grows by more than 2^8, otherwise the stale max keeps the
 // exponentials bounded by 2^8 and nothing is touched.  K and V tiles are fetched page by page with
 // tiled TMA copies (one 16 x 64 box per page and half of head_dim, landing in the canonical swizzled
-// layout) into a two-stage ring.  Roles: warps 0-3 softmax and epilogue of row tile A, warps 4-7 of
-// row tile B, warp 8 TMA producer of K, warp 10 of V, warp 9 MMA issue and TMEM allocation.  Work items are
+// layout) into a two-stage ring.  Roles: warps 0-3 softmax group A, warps 4-7 group B (softmax and epilogue),
+// warp 8 TMA producer of K, warp 10 of V, warp 9 issue of Q K^T and TMEM allocation, warp 11 issue of P V.  Work items are
 // handed out dynamically, longest sequences first: the K producer takes the next item from an atomic
 // counter and announces it to the other roles through a small queue in shared memory.  Every mbarrier wait
 // is bounded; TMEM is released on every path.
@@ -750,7 +755,8 @@ chunk_mma_kernel(const MmaArgs a, const __grid_constant__ CUtensorMap k_map, con
         __syncwarp();
     } else if (warp < 2 * kSoftmaxThreads / 32) {
         // ================================ softmax and epilogue ====================================
-        // two groups of 128 threads: group g owns row tile g; thread tg of a group owns TMEM lane tg
+        // two groups of 128 threads: group g works on row tile g of a pair (on every second KV tile of a single row
+        // tile); thread tg of a group owns TMEM lane tg
         const int grp = warp >> 2, tg = tid & (kSoftmaxThreads - 1);
         const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;  // this warp's TMEM lane quadrant
         const uint32_t s_tmem = tmem + lane_base;                                  // S: one region for both groups
@@ -855,8 +861,7 @@ chunk_mma_kernel(const MmaArgs a, const __grid_constant__ CUtensorMap k_map, con
                 //      (fma.f32x2, add.f32x2; ex2 and the bf16 conversion have none).  The denominator sums
                 //      the fp32 weights, the tensor core the same weights rounded to bf16: the two differ by
                 //      independent relative errors of at most 2^-9 per key, which the sum averages out.
-                //      P overwrites S in place: keys 32 c .. 32 c + 31 -> columns 16 c .. 16 c + 15 (all
-                //      of S is in registers).
+                //      Keys 32 c .. 32 c + 31 -> columns 16 c .. 16 c + 15 of the group's P region.
                 const float neg_m = (m_used == -INFINITY) ? 0.f : -m_used;
                 const uint64_t sc2 = pack_f32x2(a.scale_log2, a.scale_log2), nm2 = pack_f32x2(neg_m, neg_m);
                 uint64_t l2[4] = {0ull, 0ull, 0ull, 0ull};

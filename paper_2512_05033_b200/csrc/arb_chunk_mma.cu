@@ -58,7 +58,9 @@ constexpr int kTmaWarp = 8, kMmaWarp = 9, kVWarp = 10, kPvWarp = 11;
 constexpr int kHalfBytes = 128 * 128;      // [128 rows x 64 bf16]: one 128-byte-swizzled half tile
 constexpr int kTileBytes = 2 * kHalfBytes;  // [128 x 128] bf16
 constexpr int kBoxBytes = kPage * 128;      // one TMA box: 16 rows x 64 bf16
-constexpr int kStagePages = 6;              // E4M3: pages of codes in flight per operand
+constexpr int kStagePages = 6;              // E4M3: pages of codes in flight per operand ...
+constexpr int kStagePairs = kStagePages / 2;   // ... asked for, waited for and widened two at a time
+constexpr int kTilePairs = kTilePages / 2;
 constexpr int kCodePageBytes = kPage * kD;  // 2 KB: one (page, kv head) tile of codes
 constexpr uint32_t kTmemCols = 512;         // S (shared): columns 0..127, P of group A: 128..191, of B: 192..255,
 constexpr uint32_t kPCol = 128;             // O of group A: 256..383, of B: 384..511
@@ -584,9 +586,11 @@ chunk_mma_kernel(const MmaArgs a, const __grid_constant__ CUtensorMap k_map, con
                 const int row = (__shfl_sync(0xffffffffu, pid, pg) * Hkv + w.kvh) * kPage;
                 bool ok = true;
                 if constexpr (E4M3) {
-                    // Pages of codes go through the staging slots: wait for a page, widen it into the operand stage,
-                    // ask for the page kStagePages ahead (of this tile or of the next).  Lane (r, h) = (lane / 2,
-                    // lane % 2) widens the 64 codes of half h of row r: four 16-byte pieces in, eight out.
+                    // Codes go through the staging slots two pages at a time (a slot: 2 pages = 4 KB, one barrier):
+                    // wait for a pair, take its codes into registers, ask for the pair kStagePairs ahead (of this tile
+                    // or of the next), widen.  Every wait, fence and request costs the warp 100-250 cycles whatever it
+                    // covers, so they are paid per pair, not per page.  Lane (r, h) = (lane / 2, lane % 2) widens
+                    // the 64 codes of half h of row r of each page: four 16-byte pieces in, eight out.
                     char *stg = code_s + (is_v ? kStagePages * kCodePageBytes : 0);
                     uint64_t *cfull = bars->code_full[is_v ? 1 : 0];
                     // (an entry of the next tile that lies outside the pool is reported when that tile is the current one)
@@ -594,52 +598,60 @@ chunk_mma_kernel(const MmaArgs a, const __grid_constant__ CUtensorMap k_map, con
                     const int row_next = (((unsigned)pid_ahead < (unsigned)a.num_pages ? pid_ahead : 0) * Hkv + w.kvh) * kPage;
                     const int left = min(kTilePages, (w.kv_len - (jg + 1) * kBN + kPage - 1) / kPage);   // pages of the next tile
                     const int np_next = (j + 1 < w.ntiles) ? max(left, 0) : 0;
-                    auto ask = [&](int p_in_tile, uint32_t at) {   // lane 0: page p of this tile (or p - 8 of the next)
-                        const int rr = p_in_tile < kTilePages ? __shfl_sync(0xffffffffu, row, p_in_tile & 7)
-                                                              : __shfl_sync(0xffffffffu, row_next, p_in_tile & 7);
-                        if (lane == 0) {
-                            const uint32_t sl = at % kStagePages;
-                            mbar_arrive_expect_tx(&cfull[sl], kCodePageBytes);
-                            tma_box_load(stg + sl * kCodePageBytes, map, 0, rr, &cfull[sl]);
-                        }
+                    // pair q of this tile (q < kTilePairs) or pair q - kTilePairs of the next one, into slot `at` % kStagePairs
+                    auto ask = [&](int q, uint32_t at) {
+                        const bool nxt = q >= kTilePairs;
+                        const int p0 = 2 * (nxt ? q - kTilePairs : q);
+                        const int cnt = min(2, (nxt ? np_next : npages) - p0);   // pages of the pair that exist
+                        if (cnt <= 0) return;
+                        const int rr = nxt ? __shfl_sync(0xffffffffu, row_next, (p0 + (lane & 1)) & 7)
+                                           : __shfl_sync(0xffffffffu, row, (p0 + (lane & 1)) & 7);
+                        const uint32_t sl = at % kStagePairs;
+                        if (lane == 0) mbar_arrive_expect_tx(&cfull[sl], (uint32_t)cnt * kCodePageBytes);
+                        __syncwarp();
+                        if (lane < cnt) tma_box_load(stg + (sl * 2 + lane) * kCodePageBytes, map, 0, rr, &cfull[sl]);
                     };
                     if (j == 0) {   // a new item: nothing of it is in flight yet
-                        for (int p = 0; p < kStagePages; ++p) {
-                            const bool there = p < npages || (p >= kTilePages && p - kTilePages < np_next);
-                            if (__shfl_sync(0xffffffffu, there ? 1 : 0, 0)) ask(p, pc + p);
-                        }
+                        for (int q = 0; q < kStagePairs; ++q) ask(q, pc + q);
                     }
                     if (lane == 0) ok = mbar_wait(&empty[s], par ^ 1u, abort, a.status);
                     ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
                     const int r = lane >> 1, h = lane & 1;
-                    for (int p = 0; p < npages; ++p, ++pc) {
-                        const uint32_t sl = pc % kStagePages, ph = (pc / kStagePages) & 1u;
+                    const int npairs = (npages + 1) >> 1;
+                    for (int q = 0; q < npairs; ++q, ++pc) {
+                        const uint32_t sl = pc % kStagePairs, ph = (pc / kStagePairs) & 1u;
+                        const int cnt = min(2, npages - 2 * q);
                         mbar_wait(&cfull[sl], ph, abort, a.status);
-                        const char *src = stg + sl * kCodePageBytes + r * 128;
-                        char *dst = ring + s * kTileBytes + h * kHalfBytes + (p * kPage + r) * 128;
                         // the codes come into registers first, so that the slot can be asked for again at once
-                        uint4 codes[4];
+                        uint4 codes[2][4];
 #pragma unroll
-                        for (int c4 = 0; c4 < 4; ++c4)
-                            codes[c4] = *reinterpret_cast<const uint4 *>(src + (((4 * h + c4) ^ (r & 7)) << 4));
+                        for (int pp = 0; pp < 2; ++pp) {
+                            const char *src = stg + (sl * 2 + pp) * kCodePageBytes + r * 128;
+#pragma unroll
+                            for (int c4 = 0; c4 < 4; ++c4)
+                                codes[pp][c4] = (pp < cnt) ? *reinterpret_cast<const uint4 *>(src + (((4 * h + c4) ^ (r & 7)) << 4))
+                                                           : make_uint4(0, 0, 0, 0);
+                        }
                         fence_async_smem();   // the slot's next writer is the TMA unit
                         __syncwarp();
-                        {
-                            const int ahead = p + kStagePages;   // the page that takes this slot
-                            const bool there = ahead < npages || (ahead >= kTilePages && ahead - kTilePages < np_next);
-                            if (there) ask(ahead, pc + kStagePages);
-                        }
+                        ask(q + kStagePairs, pc + kStagePairs);
                         if (ok) {
 #pragma unroll
-                            for (int c4 = 0; c4 < 4; ++c4) {
-                                const uint4 cd = codes[c4];
-                                uint4 lo, hi;
-                                lo.x = e4m3x2_to_f16x2((uint16_t)cd.x); lo.y = e4m3x2_to_f16x2((uint16_t)(cd.x >> 16));
-                                lo.z = e4m3x2_to_f16x2((uint16_t)cd.y); lo.w = e4m3x2_to_f16x2((uint16_t)(cd.y >> 16));
-                                hi.x = e4m3x2_to_f16x2((uint16_t)cd.z); hi.y = e4m3x2_to_f16x2((uint16_t)(cd.z >> 16));
-                                hi.z = e4m3x2_to_f16x2((uint16_t)cd.w); hi.w = e4m3x2_to_f16x2((uint16_t)(cd.w >> 16));
-                                *reinterpret_cast<uint4 *>(dst + (((2 * c4) ^ (r & 7)) << 4)) = lo;
-                                *reinterpret_cast<uint4 *>(dst + (((2 * c4 + 1) ^ (r & 7)) << 4)) = hi;
+                            for (int pp = 0; pp < 2; ++pp) {
+                                if (pp < cnt) {
+                                    char *dst = ring + s * kTileBytes + h * kHalfBytes + ((2 * q + pp) * kPage + r) * 128;
+#pragma unroll
+                                    for (int c4 = 0; c4 < 4; ++c4) {
+                                        const uint4 cd = codes[pp][c4];
+                                        uint4 lo, hi;
+                                        lo.x = e4m3x2_to_f16x2((uint16_t)cd.x); lo.y = e4m3x2_to_f16x2((uint16_t)(cd.x >> 16));
+                                        lo.z = e4m3x2_to_f16x2((uint16_t)cd.y); lo.w = e4m3x2_to_f16x2((uint16_t)(cd.y >> 16));
+                                        hi.x = e4m3x2_to_f16x2((uint16_t)cd.z); hi.y = e4m3x2_to_f16x2((uint16_t)(cd.z >> 16));
+                                        hi.z = e4m3x2_to_f16x2((uint16_t)cd.w); hi.w = e4m3x2_to_f16x2((uint16_t)(cd.w >> 16));
+                                        *reinterpret_cast<uint4 *>(dst + (((2 * c4) ^ (r & 7)) << 4)) = lo;
+                                        *reinterpret_cast<uint4 *>(dst + (((2 * c4 + 1) ^ (r & 7)) << 4)) = hi;
+                                    }
+                                }
                             }
                         }
                     }

@@ -55,6 +55,12 @@ constexpr int kSoftmaxThreads = 128;        // per row tile
 constexpr int kThreads = 3 * kSoftmaxThreads;   // two softmax groups and a group of service warps; registers are
                                                 // handed out per 128 threads, so the third group's spare warps cost none
 constexpr int kTmaWarp = 8, kMmaWarp = 9, kVWarp = 10, kPvWarp = 11;
+// The E4M3 form runs a fourth group of warps: warps 12 and 14 widen every second pair of pages of K and of V beside
+// warps 8 and 10 (one warp per operand widens a tile in about twice the time the tensor core and the softmax groups
+// need for it).  512 threads start with 128 registers each; the softmax groups then take 168 and the two service
+// groups keep 88 (setmaxnreg; 2 * 168 + 2 * 88 = 4 * 128).
+constexpr int kKHelpWarp = 12, kVHelpWarp = 14;
+__host__ __device__ constexpr int threads_of(bool e4m3) { return e4m3 ? 4 * kSoftmaxThreads : kThreads; }
 constexpr int kHalfBytes = 128 * 128;      // [128 rows x 64 bf16]: one 128-byte-swizzled half tile
 constexpr int kTileBytes = 2 * kHalfBytes;  // [128 x 128] bf16
 constexpr int kBoxBytes = kPage * 128;      // one TMA box: 16 rows x 64 bf16
@@ -460,7 +466,7 @@ __device__ __forceinline__ bool get_item(int item, int total, const Plan &pl, in
 }
 
 template <int G, bool E4M3>
-__global__ void __launch_bounds__(kThreads, 1)
+__global__ void __launch_bounds__(threads_of(E4M3), 1)
 chunk_mma_kernel(const MmaArgs a, const __grid_constant__ CUtensorMap k_map, const __grid_constant__ CUtensorMap v_map) {
     extern __shared__ char smem_raw[];
     char *base = reinterpret_cast<char *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -478,8 +484,8 @@ chunk_mma_kernel(const MmaArgs a, const __grid_constant__ CUtensorMap k_map, con
     if (tid == 0) {
         mbar_init(&bars->q_full, 2 * kSoftmaxThreads);
         for (int s = 0; s < kStages; ++s) {
-            mbar_init(&bars->k_full[s], 1);
-            mbar_init(&bars->v_full[s], 1);
+            mbar_init(&bars->k_full[s], E4M3 ? 2 : 1);   // E4M3: both widening warps of the operand arrive
+            mbar_init(&bars->v_full[s], E4M3 ? 2 : 1);
             mbar_init(&bars->k_empty[s], 1);
             mbar_init(&bars->v_empty[s], 1);
         }
@@ -494,7 +500,8 @@ chunk_mma_kernel(const MmaArgs a, const __grid_constant__ CUtensorMap k_map, con
         mbar_init(&bars->ml_full, 2 * kSoftmaxThreads);
         for (int i = 0; i < kItemSlots; ++i) {
             mbar_init(&bars->item_full[i], 1);
-            mbar_init(&bars->item_empty[i], 3 + 2 * kSoftmaxThreads);   // the two MMA threads, V warp, softmax threads
+            // the two MMA threads, the V warp, the softmax threads (E4M3: and the two helping warps)
+            mbar_init(&bars->item_empty[i], 3 + 2 * kSoftmaxThreads + (E4M3 ? 2 : 0));
         }
         for (int i = 0; i < kStagePages; ++i) {
             mbar_init(&bars->code_full[0][i], 1);
@@ -504,7 +511,7 @@ chunk_mma_kernel(const MmaArgs a, const __grid_constant__ CUtensorMap k_map, con
         mbar_fence_init();
     }
     wait_for_predecessor();   // everything below reads what the kernel before this one may have written
-    make_plan<G>(a, pl, tid, kThreads, a.work_counter + 1);
+    make_plan<G>(a, pl, tid, threads_of(E4M3), a.work_counter + 1);
     const int total = pl.pref[B];
     if ((int)blockIdx.x >= total) return;  // nothing for this CTA; no TMEM taken, no barrier pending
 
@@ -515,7 +522,10 @@ chunk_mma_kernel(const MmaArgs a, const __grid_constant__ CUtensorMap k_map, con
     const uint32_t tmem = bars->tmem_base;
     volatile int *abort = &bars->abort;
 
-    if (warp == kTmaWarp || warp == kVWarp) {
+    const bool helper = E4M3 && (warp == kKHelpWarp || warp == kVHelpWarp);   // widens the odd pairs of pages
+    if (warp >= 2 * kSoftmaxThreads / 32) {   // the service warps
+    if constexpr (E4M3) asm volatile("setmaxnreg.dec.sync.aligned.u32 88;");
+    if (warp == kTmaWarp || warp == kVWarp || helper) {
         // ================================= TMA producers: K warp, V warp ==========================
         // One warp per operand: a tiled TMA copy is issued per (page, 64-dim half), sixteen to a tile, and one
         // warp issues them one after the other (about 1500 cycles per tile), so K and V of a tile are in
@@ -523,7 +533,7 @@ chunk_mma_kernel(const MmaArgs a, const __grid_constant__ CUtensorMap k_map, con
         // from an atomic counter (longest sequences first) and are announced to every other role, the V warp
         // included, through a small queue in shared memory.  Both run ahead of the consumers as far as their
         // two-stage rings allow.
-        const bool is_v = warp == kVWarp;
+        const bool is_v = warp == kVWarp || warp == kVHelpWarp;
         uint64_t *full = is_v ? bars->v_full : bars->k_full, *empty = is_v ? bars->v_empty : bars->k_empty;
         char *ring = is_v ? v_s : k_s;
         const CUtensorMap *map = is_v ? &v_map : &k_map;
@@ -535,7 +545,7 @@ chunk_mma_kernel(const MmaArgs a, const __grid_constant__ CUtensorMap k_map, con
             const uint32_t slot = nq % kItemSlots, qpar = (nq / kItemSlots) & 1u;
             int item = total;
             if (lane == 0) {
-                if (!is_v) {
+                if (!is_v && !helper) {
                     if (mbar_wait(&bars->item_empty[slot], qpar ^ 1u, abort, a.status)) item = atomicAdd(a.work_counter, 1);
                     bars->item_id[slot] = item;
                     mbar_arrive(&bars->item_full[slot]);
@@ -559,7 +569,7 @@ chunk_mma_kernel(const MmaArgs a, const __grid_constant__ CUtensorMap k_map, con
             // K and V tiles are asked into L2 kPrefetchTiles ahead of their load into the ring, so the
             // ring (two tiles deep) only has to cover the L2 latency, not the DRAM latency
             auto prefetch_pages = [&](int pf) {
-                if ((unsigned)pf < (unsigned)a.num_pages) {
+                if ((unsigned)pf < (unsigned)a.num_pages && !helper) {
                     constexpr int kPageBytes = kPage * kD * (E4M3 ? 1 : 2);
                     const char *src = pool + ((size_t)pf * Hkv + w.kvh) * kPageBytes;
                     asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(src), "r"(kPageBytes) : "memory");
@@ -611,7 +621,7 @@ chunk_mma_kernel(const MmaArgs a, const __grid_constant__ CUtensorMap k_map, con
                         __syncwarp();
                         if (lane < cnt) tma_box_load(stg + (sl * 2 + lane) * kCodePageBytes, map, 0, rr, &cfull[sl]);
                     };
-                    if (j == 0) {   // a new item: nothing of it is in flight yet
+                    if (j == 0 && !helper) {   // a new item: nothing of it is in flight yet
                         for (int q = 0; q < kStagePairs; ++q) ask(q, pc + q);
                     }
                     if (lane == 0) ok = mbar_wait(&empty[s], par ^ 1u, abort, a.status);
@@ -619,6 +629,7 @@ chunk_mma_kernel(const MmaArgs a, const __grid_constant__ CUtensorMap k_map, con
                     const int r = lane >> 1, h = lane & 1;
                     const int npairs = (npages + 1) >> 1;
                     for (int q = 0; q < npairs; ++q, ++pc) {
+                        if ((q & 1) != (helper ? 1 : 0)) continue;   // the operand's two warps take the pairs in turn
                         const uint32_t sl = pc % kStagePairs, ph = (pc / kStagePairs) & 1u;
                         const int cnt = min(2, npages - 2 * q);
                         mbar_wait(&cfull[sl], ph, abort, a.status);
@@ -765,8 +776,10 @@ chunk_mma_kernel(const MmaArgs a, const __grid_constant__ CUtensorMap k_map, con
             }
         }
         __syncwarp();
-    } else if (warp < 2 * kSoftmaxThreads / 32) {
+    }
+    } else {
         // ================================ softmax and epilogue ====================================
+        if constexpr (E4M3) asm volatile("setmaxnreg.inc.sync.aligned.u32 168;");
         // two groups of 128 threads: group g works on row tile g of a pair (on every second KV tile of a single row
         // tile); thread tg of a group owns TMEM lane tg
         const int grp = warp >> 2, tg = tid & (kSoftmaxThreads - 1);
@@ -1133,7 +1146,7 @@ arb_status launch_one(Ctx *ctx, const MmaArgs &a, const CUtensorMap &km, const C
         attr_set[ctx->device & 63] = true;
     }
     const int grid = max_items < ctx->num_sms ? max_items : ctx->num_sms;
-    const cudaError_t err = launch_pdl(chunk_mma_kernel<G, E4M3>, dim3(grid), dim3(kThreads), smem, stream, a, km, vm);
+    const cudaError_t err = launch_pdl(chunk_mma_kernel<G, E4M3>, dim3(grid), dim3(threads_of(E4M3)), smem, stream, a, km, vm);
     ctx->launches++;
     if (err != cudaSuccess) return ARB_ERR_CUDA;
     // the merge of split sequences, when the block table is long enough for a sequence to be split at all

@@ -295,3 +295,77 @@ def attn_e4m3(q, k_codes, v_codes, k_scale: float, v_scale: float, block_table, 
     vf = torch.from_numpy(e4m3_decode(v_codes))
     out, st = attn(q.float(), kf, vf, block_table, seq_lens, q_lens, sm * float(k_scale))
     return out * float(v_scale), st
+
+
+# ---- 4-bit KV cache (this library's format, stated here in full) ------------------------------------------
+#
+# Every (token, kv head) row of D values has one fp32 scale s = max|x| / 7 (IEEE division in fp32; s = 0 for a row
+# of zeros) and D codes c = clamp(rint(x * (7 / max|x|)), -7, 7): the reciprocal 7 / max|x| by IEEE division in fp32,
+# the product in fp32, rint to nearest with ties to even; c = 0 for a row of zeros.  The value read back is s * c.
+# A nibble holds c + 8 (1 .. 15).  The D / 2 bytes of a row are packed per group of 8 dimensions d0 .. d7 into one
+# little-endian 32-bit word whose nibbles 0 .. 7 (from the least significant) hold d0, d2, d4, d6, d1, d3, d5, d7:
+# the pair (nibble i, nibble i + 4) is the pair of neighbouring dimensions (2i, 2i + 1).
+# A quantised draft (Section 5.1 runs 4-bit and 3-bit drafts) is the reason for the cache; the format itself is not
+# the paper's.  NaN or infinite inputs are outside the format (the row's scale would not be finite).
+
+_I4_NIBBLE_OF_DIM = (0, 4, 1, 5, 2, 6, 3, 7)   # dimension d of a group of 8 sits in nibble _I4_NIBBLE_OF_DIM[d]
+
+
+def i4_encode(x):
+    """values [..., D] -> (codes uint8 [..., D / 2], scales fp32 [...])."""
+    a = _f32(x)
+    D = a.shape[-1]
+    assert D % 8 == 0
+    m = np.max(np.abs(a), axis=-1).astype(np.float32)
+    with np.errstate(divide="ignore", invalid="ignore"):
+        scale = np.where(m > 0, m / np.float32(7), np.float32(0)).astype(np.float32)
+        inv = np.where(m > 0, np.float32(7) / m, np.float32(0)).astype(np.float32)
+    c = np.rint((a * inv[..., None]).astype(np.float32))          # fp32 product, ties to even
+    c = np.clip(c, -7, 7).astype(np.int64) + 8                      # nibble values 1 .. 15
+    g = c.reshape(a.shape[:-1] + (D // 8, 8))
+    word = np.zeros(g.shape[:-1], dtype=np.uint64)
+    for d in range(8):
+        word |= g[..., d].astype(np.uint64) << np.uint64(4 * _I4_NIBBLE_OF_DIM[d])
+    word = word.astype(np.uint32)
+    codes = np.stack([(word >> np.uint32(8 * b)) & np.uint32(0xff) for b in range(4)], axis=-1).astype(np.uint8)
+    return codes.reshape(a.shape[:-1] + (D // 2,)), scale
+
+
+def i4_decode(codes, scales):
+    """(codes uint8 [..., D / 2], scales fp32 [...]) -> float64 values [..., D] = scale * code (exact)."""
+    c = np.ascontiguousarray(codes.detach().cpu().numpy() if hasattr(codes, "detach") else np.asarray(codes), dtype=np.uint8)
+    s = _f32(scales).astype(np.float64)
+    half = c.shape[-1]
+    b = c.reshape(c.shape[:-1] + (half // 4, 4)).astype(np.uint32)
+    word = b[..., 0] | (b[..., 1] << np.uint32(8)) | (b[..., 2] << np.uint32(16)) | (b[..., 3] << np.uint32(24))
+    out = np.zeros(word.shape + (8,), dtype=np.float64)
+    for d in range(8):
+        out[..., d] = ((word >> np.uint32(4 * _I4_NIBBLE_OF_DIM[d])) & np.uint32(0xf)).astype(np.float64) - 8.0
+    return out.reshape(c.shape[:-1] + (2 * half,)) * s[..., None]
+
+
+def kv_append_i4(k_new, v_new, block_table, seq_lens, new_lens, k_codes, v_codes, k_scales, v_scales,
+                 update_lens: bool = True):
+    """Quantising append into copies of the code pools [num_pages, Hkv, P, D / 2] and scale pools [num_pages, Hkv, P]:
+    the placement rule and the refusals are kv_append's (a scale is a one-element row of the same slot)."""
+    import torch
+
+    kc, ks = i4_encode(k_new)
+    vc, vs = i4_encode(v_new)
+    ok, ov, sl, st = kv_append(torch.from_numpy(kc), torch.from_numpy(vc), block_table, seq_lens, new_lens, k_codes, v_codes,
+                               update_lens)
+    ks_p = torch.as_tensor(np.asarray(_f32(k_scales)))[..., None]
+    vs_p = torch.as_tensor(np.asarray(_f32(v_scales)))[..., None]
+    oks, ovs, _, _ = kv_append(torch.from_numpy(ks)[..., None], torch.from_numpy(vs)[..., None], block_table, seq_lens,
+                               new_lens, ks_p, vs_p, update_lens)
+    return ok, ov, oks[..., 0], ovs[..., 0], sl, st
+
+
+def attn_i4(q, k_codes, v_codes, k_scales, v_scales, block_table, seq_lens, q_lens, scale: float = 0.0):
+    """Attention over a 4-bit cache: keys and values are i4_decode of the pools, handed to `attn` as fp32 (its input
+    type: the product scale * code is rounded once, 2^-24 relative; fp64 from there on)."""
+    import torch
+
+    kf = torch.from_numpy(i4_decode(k_codes, k_scales).astype(np.float32))
+    vf = torch.from_numpy(i4_decode(v_codes, v_scales).astype(np.float32))
+    return attn(q.float(), kf, vf, block_table, seq_lens, q_lens, scale)

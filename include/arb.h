@@ -447,6 +447,34 @@ arb_status arb_decode_step_e4m3(arb_ctx *ctx, const arb_attn_params *params, con
                                 const int32_t *q_lens, void *out, arb_stream_t stream);
 
 /*
+ * One decode token over a 4-bit KV cache in one launch: arb_decode_step with the token's K/V rows quantised on the
+ * way in (Section 3.1: z_i ~ q(z_i | x, z_<i); Section 5.1 runs 4-bit and 3-bit drafts; the cache format is this
+ * library's own and is fixed here).
+ *
+ * Format.  Every (token, kv head) row of D = 128 values x has one fp32 scale s = max|x| / 7 (IEEE division in fp32;
+ * 0 for a row of zeros) and 128 codes c = clamp(rint(x * (7 / max|x|)), -7, 7) (the reciprocal by IEEE division in
+ * fp32, the product in fp32, nearest with ties to even; 0 for a row of zeros); the value read back is s * c.  A
+ * nibble holds c + 8.  A group of 8 dimensions d0 .. d7 is one little-endian 32-bit word whose nibbles 0 .. 7 (from the
+ * least significant) hold d0, d2, d4, d6, d1, d3, d5, d7.  NaN and infinities are outside the format.
+ *
+ *   params, q, out, k_new, v_new, block_table, seq_lens, q_lens
+ *              as for arb_decode_step; dtype ARB_BF16 (q, out, k_new, v_new), head_dim 128, g <= 8.
+ *   k_codes,
+ *   v_codes    uint8 pools [num_pages, Hkv, P, D / 2], written (one row per sequence and kv head) and read.
+ *   k_scales,
+ *   v_scales   fp32 pools [num_pages, Hkv, P], written and read; 16-byte aligned.
+ * Codes and scales written are bit-identical to the format's definition; the rows are attention over s * c within
+ * the tolerance of arb_attn (the weights that reach the tensor core are rounded to bf16 after they took the value
+ * scale).  Refused sequences, idle slots, status bits and stream behaviour as for arb_decode_step.
+ * Errors: ARB_ERR_INVALID_ARG, ARB_ERR_UNSUPPORTED (dtype, head_dim, g > 8, ARB_ATTN_NO_TENSOR_CORES),
+ * ARB_ERR_WORKSPACE, ARB_ERR_CUDA.
+ */
+arb_status arb_decode_step_i4(arb_ctx *ctx, const arb_attn_params *params, const void *q, const void *k_new,
+                              const void *v_new, uint8_t *k_codes, uint8_t *v_codes, float *k_scales, float *v_scales,
+                              const int32_t *block_table, int32_t *seq_lens, const int32_t *q_lens, void *out,
+                              arb_stream_t stream);
+
+/*
  * Spearman's rank correlation of two samples (Section 4.2, "Evaluation", and Tables 1-3 of the paper:
  * the correlation between the router's predicted scores and the oracle advantage Delta).  Each value is
  * replaced by its rank within its sample, equal values sharing the mean of the ranks they span, and

@@ -37,7 +37,7 @@ MAX_CLASSES = 16
 # every symbol include/arb.h declares
 EXPORTS = ("arb_create", "arb_destroy", "arb_attn_workspace_bytes", "arb_attn", "arb_attn_host",
            "arb_attn_host_begin", "arb_attn_host_wait",
-           "arb_attn_decode_static", "arb_decode_step", "arb_decode_step_e4m3",
+           "arb_attn_decode_static", "arb_decode_step", "arb_decode_step_e4m3", "arb_decode_step_i4",
            "arb_route", "arb_rollback", "arb_policy", "arb_route_classes", "arb_kv_append", "arb_kv_append_e4m3", "arb_attn_decode_e4m3", "arb_attn_e4m3", "arb_phase_lens", "arb_phase_lens_tokens", "arb_spearman",
            "arb_selftest_wait_timeout", "arb_selftest_guard_zones", "arb_poll_status", "arb_launch_count", "arb_status_string")
 
@@ -69,6 +69,8 @@ lib.arb_attn_decode_static.restype = ctypes.c_int
 lib.arb_attn_decode_static.argtypes = [ctypes.POINTER(AttnParams), _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp]
 lib.arb_decode_step.restype = ctypes.c_int
 lib.arb_decode_step.argtypes = [_vp, ctypes.POINTER(AttnParams), _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp]
+lib.arb_decode_step_i4.restype = ctypes.c_int
+lib.arb_decode_step_i4.argtypes = [_vp, ctypes.POINTER(AttnParams)] + [_vp] * 12
 lib.arb_decode_step_e4m3.restype = ctypes.c_int
 lib.arb_decode_step_e4m3.argtypes = [_vp, ctypes.POINTER(AttnParams), _vp, _vp, _vp, _vp, _vp, ctypes.c_float, ctypes.c_float,
                                      ctypes.c_float, ctypes.c_float, _vp, _vp, _vp, _vp, _vp]
@@ -294,6 +296,28 @@ class Context:
                                       _dev(seq_lens, "seq_lens", torch.int32), _dev(q_lens, "q_lens", torch.int32),
                                       _dev(out, "out", torch.bfloat16), _stream_ptr(stream))
         _check(st, "arb_decode_step_e4m3")
+        return out
+
+    # -- arb_decode_step_i4 -------------------------------------------------------------------
+    def decode_step_i4(self, q, k_new, v_new, k_codes, v_codes, k_scales, v_scales, block_table, seq_lens, q_lens,
+                       out=None, softmax_scale: float = 0.0, stream=None, params: AttnParams | None = None):
+        """decode_step over a 4-bit cache (codes uint8 [pages, Hkv, P, D / 2], scales fp32 [pages, Hkv, P]): the new
+        rows are quantised into the pools, out = attention over scale * code including them, seq_lens += q_lens."""
+        if out is None:
+            out = torch.empty_like(q)
+        if params is None:
+            num_pages, Hkv, P, _ = k_codes.shape
+            B, max_pages = block_table.shape
+            params = attn_params(_dtype_code(q), B, q.shape[1], Hkv, q.shape[2], num_pages, max_pages, q.shape[0], 1,
+                                 softmax_scale, P, 0)
+        st = lib.arb_decode_step_i4(self._h, ctypes.byref(params), _dev(q, "q", torch.bfloat16),
+                                    _dev(k_new, "k_new", torch.bfloat16), _dev(v_new, "v_new", torch.bfloat16),
+                                    _dev(k_codes, "k_codes", torch.uint8), _dev(v_codes, "v_codes", torch.uint8),
+                                    _dev(k_scales, "k_scales", torch.float32), _dev(v_scales, "v_scales", torch.float32),
+                                    _dev(block_table, "block_table", torch.int32),
+                                    _dev(seq_lens, "seq_lens", torch.int32), _dev(q_lens, "q_lens", torch.int32),
+                                    _dev(out, "out", torch.bfloat16), _stream_ptr(stream))
+        _check(st, "arb_decode_step_i4")
         return out
 
     # -- arb_route ----------------------------------------------------------------------------

@@ -315,6 +315,30 @@ arb_status arb_decode_step_e4m3(arb_ctx *ctx, const arb_attn_params *params, con
                               reinterpret_cast<cudaStream_t>(stream));
 }
 
+arb_status arb_decode_step_i4(arb_ctx *ctx, const arb_attn_params *params, const void *q, const void *k_new,
+                              const void *v_new, uint8_t *k_codes, uint8_t *v_codes, float *k_scales, float *v_scales,
+                              const int32_t *block_table, int32_t *seq_lens, const int32_t *q_lens, void *out,
+                              arb_stream_t stream) {
+    if (ctx == nullptr) return ARB_ERR_INVALID_ARG;
+    arb_status st = check_params(params);
+    if (st != ARB_OK) return st;
+    if (params->dtype != ARB_BF16 || params->head_dim != 128) return ARB_ERR_UNSUPPORTED;
+    if (params->flags & ARB_ATTN_NO_TENSOR_CORES) return ARB_ERR_UNSUPPORTED;
+    if (params->max_q_len != 1 || params->total_q < 0 || params->total_q > params->batch) return ARB_ERR_INVALID_ARG;
+    if (params->flags & ARB_ATTN_OVERLAP_PREVIOUS) return ARB_ERR_INVALID_ARG;   // the call writes the cache it reads
+    if (!k_codes || !v_codes || !k_scales || !v_scales || !block_table || !seq_lens || !q_lens) return ARB_ERR_INVALID_ARG;
+    if (params->total_q == 0) return ARB_OK;
+    if (!q || !out || !k_new || !v_new) return ARB_ERR_INVALID_ARG;
+    if (!aligned16(q) || !aligned16(out) || !aligned16(k_codes) || !aligned16(v_codes) || !aligned16(k_new) ||
+        !aligned16(v_new) || !aligned16(k_scales) || !aligned16(v_scales))
+        return ARB_ERR_INVALID_ARG;
+    Ctx *c = reinterpret_cast<Ctx *>(ctx);
+    if (decode_workspace_bytes(*params, c->num_sms) > c->workspace_bytes) return ARB_ERR_WORKSPACE;
+    if (!decode_step_supported(*params)) return ARB_ERR_UNSUPPORTED;
+    return launch_decode_step(c, *params, q, k_new, v_new, k_codes, v_codes, nullptr, block_table, seq_lens, q_lens, out,
+                              reinterpret_cast<cudaStream_t>(stream), k_scales, v_scales);
+}
+
 arb_status arb_attn_decode_static(const arb_attn_params *params, const void *q, const void *k_pages,
                                   const void *v_pages, const int32_t *block_table, const int32_t *seq_lens,
                                   const int32_t *q_lens, void *out, uint32_t *device_status, arb_stream_t stream) {

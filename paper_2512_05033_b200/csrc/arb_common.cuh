@@ -336,7 +336,8 @@ bool decode_step_supported(const arb_attn_params &p);
 size_t decode_step_hint_bytes(int num_sms);
 arb_status launch_decode_step(Ctx *ctx, const arb_attn_params &p, const void *q, const void *k_new, const void *v_new,
                               void *k_pages, void *v_pages, const float *scales, const int32_t *block_table,
-                              int32_t *seq_lens, const int32_t *q_lens, void *out, cudaStream_t stream);
+                              int32_t *seq_lens, const int32_t *q_lens, void *out, cudaStream_t stream,
+                              float *k_row_scales = nullptr, float *v_row_scales = nullptr);
 arb_status launch_guard_count(Ctx *ctx, const unsigned char *const *zones, int n_zones, size_t zone_bytes,
                               unsigned long long *bad_dev, cudaStream_t stream);
 arb_status launch_selftest_wait(Ctx *ctx, long long limit_cycles, int32_t *report, cudaStream_t stream);

@@ -45,6 +45,10 @@ constexpr int kNT = kCT + 64;
 constexpr int kTileBytes = kPage * kD * 2;    // 4 KB: one (page, kv head) tile of K or of V
 constexpr int kHalfTile = kTileBytes / 2;
 constexpr int kCodeTileBytes = kPage * kD;    // 2 KB: the same tile of an E4M3 cache
+constexpr int kI4CodeBytes = kPage * kD / 2;  // 1 KB: the same tile of a 4-bit cache (16 rows x 64 bytes, not swizzled) ...
+constexpr int kI4ScaleBytes = kPage * 4;      // ... followed by the 16 fp32 scales of its rows
+constexpr int kI4StageBytes = 1152;           // both, rounded up to 128
+enum { kKvBf16 = 0, kKvE4m3 = 1, kKvI4 = 2 }; // the cache a kernel instance reads
 constexpr int kBatch = 32;                    // producer lanes issuing side by side
 constexpr int kParked = 2;                    // segment results parked in shared memory before they are written
 constexpr int kOStride = kD + 4;              // floats between two heads of a warp record (spreads the banks)
@@ -83,6 +87,7 @@ struct StepArgs {
     float scale_log2;  // softmax scale (times the key scale of an E4M3 cache) * log2(e)
     float v_scale;     // value scale of an E4M3 cache, 1 otherwise
     float k_inv_scale, v_inv_scale;   // E4M3 cache with a cache write: code = e4m3(x * inv_scale)
+    float *k_scales, *v_scales;       // 4-bit cache: the scale pools [num_pages, Hkv, 16]
 };
 
 template <int STAGES>
@@ -104,10 +109,12 @@ struct Cfg {
 };
 
 // E4M3: the ring holds tiles of codes; every consumer warp has a widened K tile and a widened V tile of its own
-template <int G, int STAGES, bool E4M3>
+template <int G, int STAGES, int KV>
 size_t smem_bytes(int batch) {
     using C = Cfg<G>;
-    const size_t tiles = E4M3 ? (size_t)STAGES * kCodeTileBytes + (size_t)kCW * 2 * kTileBytes : (size_t)STAGES * kTileBytes;
+    const size_t wide = (size_t)kCW * 2 * kTileBytes;
+    const size_t tiles = KV == kKvE4m3 ? (size_t)STAGES * kCodeTileBytes + wide
+                         : KV == kKvI4 ? (size_t)STAGES * kI4StageBytes + wide : (size_t)STAGES * kTileBytes;
     return 1024 + tiles + C::OSM_BYTES + C::PARK_BYTES + sizeof(Tail<STAGES>) + sizeof(int) * (4 * (size_t)batch + 3 + 8);
 }
 
@@ -166,6 +173,29 @@ __device__ __forceinline__ void widen_tile(const char *codes, char *dst, int lan
         *reinterpret_cast<uint4 *>(dst + tile_off(r, 2 * c)) = lo;
         *reinterpret_cast<uint4 *>(dst + tile_off(r, 2 * c + 1)) = hi;
     }
+}
+
+// 4-bit cache: a 32-bit word holds 8 dimensions as nibbles (code + 8), nibble i and nibble i + 4 being the neighbouring
+// dimensions 2i and 2i + 1.  (word >> 4i) & 0x000F000F | 0x43004300 is the bf16 pair (128 + nibble i, 128 + nibble i + 4)
+// -- a bf16 with exponent 2^7 counts in ones -- and subtracting 136 leaves the two codes, exactly.
+__device__ __forceinline__ uint4 i4_word_to_bf16x8(uint32_t w) {
+    uint32_t r[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const uint32_t biased = ((w >> (4 * i)) & 0x000F000Fu) | 0x43004300u;
+        asm("fma.rn.bf16x2 %0, %1, %2, %3;" : "=r"(r[i]) : "r"(biased), "r"(0x3F803F80u), "r"(0xC308C308u));
+    }
+    return make_uint4(r[0], r[1], r[2], r[3]);
+}
+// A warp widens a tile of 4-bit codes (16 rows x 64 bytes, plain row-major) into a bf16 tile laid out like a tile of
+// a bf16 cache: lane (r, h) = (lane / 2, lane % 2) takes the 32 bytes (64 dimensions) of half h of row r.
+__device__ __forceinline__ void widen_tile_i4(const char *codes, char *dst, int lane) {
+    const int r = lane >> 1, h = lane & 1;
+    const uint4 c0 = *reinterpret_cast<const uint4 *>(codes + r * 64 + h * 32);
+    const uint4 c1 = *reinterpret_cast<const uint4 *>(codes + r * 64 + h * 32 + 16);
+    const uint32_t w[8] = {c0.x, c0.y, c0.z, c0.w, c1.x, c1.y, c1.z, c1.w};
+#pragma unroll
+    for (int i = 0; i < 8; ++i) *reinterpret_cast<uint4 *>(dst + tile_off(r, 8 * h + i)) = i4_word_to_bf16x8(w[i]);
 }
 
 __device__ __forceinline__ void fence_proxy_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
@@ -256,15 +286,17 @@ __device__ __forceinline__ void parts_of(const Plan &pl, Segment &s) {
     s.nparts = pl.cta_of(s.b, s.kvh, pages, pages - 1) - s.c_first + 1;
 }
 
-template <int G, int STAGES, bool APPEND, bool E4M3>
+template <int G, int STAGES, bool APPEND, int KV>
 __global__ void __launch_bounds__(kNT, 1)
 decode_step_kernel(const StepArgs a, const __grid_constant__ CUtensorMap k_map, const __grid_constant__ CUtensorMap v_map) {
     using C = Cfg<G>;
     using Tail = arb::Tail<STAGES>;
     constexpr int GP = C::GP, WREC = C::WREC, REC = C::REC;
-    constexpr int kStageBytes = E4M3 ? kCodeTileBytes : kTileBytes;   // what one TMA copy brings
-    constexpr int kElt = E4M3 ? 1 : 2;                                  // bytes of a cache element
-    constexpr int kWideBytes = E4M3 ? kCW * 2 * kTileBytes : 0;         // E4M3: a widened K and V tile per consumer warp
+    constexpr bool E4M3 = KV == kKvE4m3, I4 = KV == kKvI4, WIDE = KV != kKvBf16;
+    constexpr int kStageBytes = E4M3 ? kCodeTileBytes : I4 ? kI4StageBytes : kTileBytes;   // a ring stage
+    constexpr int kTxBytes = I4 ? kI4CodeBytes + kI4ScaleBytes : kStageBytes;               // what the copies of a stage bring
+    constexpr int kRowBytes = E4M3 ? kD : I4 ? kD / 2 : kD * 2;         // bytes of a cache row
+    constexpr int kWideBytes = WIDE ? kCW * 2 * kTileBytes : 0;         // codes: a widened K and V tile per consumer warp
     constexpr int kRingBytes = STAGES * kStageBytes + kWideBytes;       // the merges use all of it
     static_assert(G >= 1 && G <= 8, "the group's heads are the 8 columns of the tile");
     static_assert(STAGES % (2 * kCW) == 0 && kBatch <= STAGES, "a ring stage always belongs to the same warp of a segment");
@@ -310,9 +342,9 @@ decode_step_kernel(const StepArgs a, const __grid_constant__ CUtensorMap k_map, 
             for (int i = lane; i < n; i += 32) {
                 const int row = __ldcg(hint + 4 + i);
                 if ((unsigned)row < (unsigned)(a.num_pages * Hkv * kPage)) {
-                    const size_t off = (size_t)row * (kD * kElt);
-                    asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(a.k_pool + off), "r"(kStageBytes) : "memory");
-                    asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(a.v_pool + off), "r"(kStageBytes) : "memory");
+                    const size_t off = (size_t)row * kRowBytes;
+                    asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(a.k_pool + off), "r"(kPage * kRowBytes) : "memory");
+                    asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(a.v_pool + off), "r"(kPage * kRowBytes) : "memory");
                 }
             }
         }
@@ -486,8 +518,12 @@ decode_step_kernel(const StepArgs a, const __grid_constant__ CUtensorMap k_map, 
                 const long long t0 = clock64();
                 while (__any_sync(0xffffffffu, pending)) {
                     if (pending && mbar_test_wait(&tail->empty[st], par ^ 1u)) {
-                        mbar_arrive_expect_tx(&tail->full[st], kStageBytes);
-                        if constexpr (E4M3) {
+                        mbar_arrive_expect_tx(&tail->full[st], kTxBytes);
+                        if constexpr (I4) {   // 16 rows x 64 bytes of codes, then the rows' 16 scales
+                            tma_box_load(ring + st * kStageBytes, map, 0, row, &tail->full[st]);
+                            bulk_load(ring + st * kStageBytes + kI4CodeBytes, ((i & 1) ? a.v_scales : a.k_scales) + row,
+                                      kI4ScaleBytes, &tail->full[st]);
+                        } else if constexpr (E4M3) {
                             tma_box_load(ring + st * kStageBytes, map, 0, row, &tail->full[st]);   // 16 rows x 128 codes
                         } else if (a.whole_rows) {
                             tma_box_load3(ring + st * kTileBytes, map, 0, row, 0, &tail->full[st]);
@@ -619,6 +655,7 @@ decode_step_kernel(const StepArgs a, const __grid_constant__ CUtensorMap k_map, 
         const int last_pg = (s.L - 1) / kPage, new_slot = (s.L - 1) % kPage;
         bool patch = false;
         uint4 new_row = make_uint4(0, 0, 0, 0);
+        float new_scale = 0.f;   // 4-bit cache: the scale of the new K row (lanes 0..15) / V row (lanes 16..31)
         if constexpr (APPEND) {
             patch = last_pg >= s.pg0 && last_pg < s.pg1 && ((last_pg - s.pg0) % kCW) == warp;
             if (patch) {
@@ -627,7 +664,37 @@ decode_step_kernel(const StepArgs a, const __grid_constant__ CUtensorMap k_map, 
                 const int pid = a.block_table[(size_t)s.b * a.max_pages + last_pg];
                 const bool store = (unsigned)pid < (unsigned)a.num_pages && ARB_IN_RANGE(a.status, qrow, a.rows);
                 // (a page outside the pool: the producer has raised ARB_DEV_BAD_PAGE; nothing is written)
-                if constexpr (E4M3) {
+                if constexpr (I4) {
+                    // The row's scale is max|x| / 7 over its 128 values (16 lanes), the codes rint(x * (7 / max|x|))
+                    // clamped to -7 .. 7, both divisions IEEE; this lane's eight values are one word of nibbles
+                    // (code + 8; nibbles 0..7 = dimensions 0, 2, 4, 6, 1, 3, 5, 7 of the eight).
+                    const uint32_t w[4] = {new_row.x, new_row.y, new_row.z, new_row.w};
+                    float x[8];
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        x[2 * j] = __uint_as_float(w[j] << 16);
+                        x[2 * j + 1] = __uint_as_float(w[j] & 0xffff0000u);
+                    }
+                    float m = 0.f;
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) m = fmaxf(m, fabsf(x[j]));
+#pragma unroll
+                    for (int off = 8; off >= 1; off >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, off));
+                    new_scale = m > 0.f ? __fdiv_rn(m, 7.f) : 0.f;
+                    const float inv = m > 0.f ? __fdiv_rn(7.f, m) : 0.f;
+                    uint32_t word = 0;
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) {
+                        const int c = max(-7, min(7, __float2int_rn(__fmul_rn(x[j], inv))));
+                        word |= (uint32_t)(c + 8) << (4 * ((j >> 1) + 4 * (j & 1)));
+                    }
+                    if (store) {
+                        const size_t slot_row = ((size_t)pid * Hkv + s.kvh) * kPage + new_slot;
+                        *reinterpret_cast<uint32_t *>((lane < 16 ? a.k_pool : a.v_pool) + slot_row * (kD / 2) + (lane & 15) * 4) = word;
+                        if ((lane & 15) == 0) (lane < 16 ? a.k_scales : a.v_scales)[slot_row] = new_scale;
+                    }
+                    new_row = i4_word_to_bf16x8(word);
+                } else if constexpr (E4M3) {
                     // quantise this lane's eight values as arb_kv_append_e4m3 does (x * inv_scale in fp32, nearest code,
                     // ties to even, saturating), store the codes, and keep their widened form for the tile
                     const float inv = lane < 16 ? a.k_inv_scale : a.v_inv_scale;
@@ -666,18 +733,31 @@ decode_step_kernel(const StepArgs a, const __grid_constant__ CUtensorMap k_map, 
 
             // ---- S^T = K q^T: 16 keys x 8 heads, two accumulators so that the chain is four deep ----------
             float sa[4] = {0.f, 0.f, 0.f, 0.f}, sb[4] = {0.f, 0.f, 0.f, 0.f};
+            float ksc0 = 1.f, ksc1 = 1.f, vsc0 = 1.f, vsc1 = 1.f;   // 4-bit cache: the scales of keys gq and gq + 8
             {
                 const uint32_t st = ck % STAGES, par = (ck / STAGES) & 1u;
                 mbar_wait(&tail->full[st], par, abort, a.status);
                 char *tile_p = ring + st * kStageBytes;
-                if constexpr (E4M3) {   // widen into this warp's tile; the ring stage is free at once
-                    widen_tile(tile_p, wide_k, lane);
+                if constexpr (WIDE) {   // widen into this warp's tile; the ring stage is free at once
+                    if constexpr (I4) {
+                        widen_tile_i4(tile_p, wide_k, lane);
+                        const float *sc = reinterpret_cast<const float *>(tile_p + kI4CodeBytes);
+                        ksc0 = sc[gq];
+                        ksc1 = sc[gq + 8];
+                    } else {
+                        widen_tile(tile_p, wide_k, lane);
+                    }
                     __syncwarp();
                     if (lane == 0) mbar_arrive(&tail->empty[st]);
                     tile_p = wide_k;
                 }
                 if (patch_here) {
                     if (lane < 16) *reinterpret_cast<uint4 *>(tile_p + tile_off(new_slot, lane)) = new_row;
+                    if constexpr (I4) {
+                        const float ns = __shfl_sync(0xffffffffu, new_scale, 0);
+                        if (gq == new_slot) ksc0 = ns;
+                        if (gq + 8 == new_slot) ksc1 = ns;
+                    }
                     __syncwarp();
                 }
                 const uint32_t tile = smem_u32(tile_p);
@@ -689,10 +769,14 @@ decode_step_kernel(const StepArgs a, const __grid_constant__ CUtensorMap k_map, 
                     else mma_16816<E4M3>(sa, af, qb[ks][0], qb[ks][1]);
                 }
                 __syncwarp();
-                if constexpr (!E4M3) {
+                if constexpr (!WIDE) {
                     if (patch_here) fence_proxy_async_smem();   // the stage's next writer is the TMA unit
                     if (lane == 0) mbar_arrive(&tail->empty[st]);
                 }
+            }
+            if constexpr (I4) {   // a key is scale * code: the scores of keys gq and gq + 8 take their rows' scales
+                sa[0] *= ksc0; sa[1] *= ksc0; sb[0] *= ksc0; sb[1] *= ksc0;
+                sa[2] *= ksc1; sa[3] *= ksc1; sb[2] *= ksc1; sb[3] *= ksc1;
             }
 
             // ---- online softmax: this lane has keys gq and gq + 8 of heads h0 and h1 -------------------
@@ -714,9 +798,12 @@ decode_step_kernel(const StepArgs a, const __grid_constant__ CUtensorMap k_map, 
             // P^T, rounded to bf16 (f16 over an E4M3 cache); the sums use the rounded weights, like the tensor core
             const float p00 = fast_exp2(s00 - mn0), p01 = fast_exp2(s01 - mn1);
             const float p10 = fast_exp2(s10 - mn0), p11 = fast_exp2(s11 - mn1);
-            const uint32_t w0 = E4M3 ? pack_f16(p00, p01) : pack_bf16(p00, p01);   // key gq:     heads h0, h1
-            const uint32_t w1 = E4M3 ? pack_f16(p10, p11) : pack_bf16(p10, p11);   // key gq + 8
-            if constexpr (E4M3) {
+            uint32_t w0 = E4M3 ? pack_f16(p00, p01) : pack_bf16(p00, p01);   // key gq:     heads h0, h1
+            uint32_t w1 = E4M3 ? pack_f16(p10, p11) : pack_bf16(p10, p11);   // key gq + 8
+            if constexpr (I4) {   // (the weights that reach the tensor core carry the value scales: packed below)
+                l_run0 = fmaf(l_run0, f0, p00 + p10);
+                l_run1 = fmaf(l_run1, f1, p01 + p11);
+            } else if constexpr (E4M3) {
                 const float2 r0 = unpack_f16(w0), r1 = unpack_f16(w1);
                 l_run0 = fmaf(l_run0, f0, r0.x + r1.x);
                 l_run1 = fmaf(l_run1, f1, r0.y + r1.y);
@@ -725,7 +812,11 @@ decode_step_kernel(const StepArgs a, const __grid_constant__ CUtensorMap k_map, 
                 l_run1 = fmaf(l_run1, f1, __uint_as_float(w0 & 0xffff0000u) + __uint_as_float(w1 & 0xffff0000u));
             }
             // B fragment of P^T (16 keys x 8 heads): keys 2 tq, + 1 (and + 8) of head gq
-            const uint32_t pb0 = movmatrix_trans(w0), pb1 = movmatrix_trans(w1);
+            uint32_t pb0 = 0, pb1 = 0;
+            if constexpr (!I4) {
+                pb0 = movmatrix_trans(w0);
+                pb1 = movmatrix_trans(w1);
+            }
             if (__any_sync(0xffffffffu, f0 != 1.0f || f1 != 1.0f)) {
 #pragma unroll
                 for (int mt = 0; mt < 8; ++mt) { o[mt][0] *= f0; o[mt][1] *= f1; o[mt][2] *= f0; o[mt][3] *= f1; }
@@ -736,15 +827,33 @@ decode_step_kernel(const StepArgs a, const __grid_constant__ CUtensorMap k_map, 
                 const uint32_t cv = ck + 1u, st = cv % STAGES, par = (cv / STAGES) & 1u;
                 mbar_wait(&tail->full[st], par, abort, a.status);
                 char *tile_p = ring + st * kStageBytes;
-                if constexpr (E4M3) {
-                    widen_tile(tile_p, wide_v, lane);
+                if constexpr (WIDE) {
+                    if constexpr (I4) {
+                        widen_tile_i4(tile_p, wide_v, lane);
+                        const float *sc = reinterpret_cast<const float *>(tile_p + kI4CodeBytes);
+                        vsc0 = k0 ? sc[gq] : 0.f;        // (the scale of a slot past the sequence end may be anything)
+                        vsc1 = k1 ? sc[gq + 8] : 0.f;
+                    } else {
+                        widen_tile(tile_p, wide_v, lane);
+                    }
                     __syncwarp();
                     if (lane == 0) mbar_arrive(&tail->empty[st]);
                     tile_p = wide_v;
                 }
                 if (patch_here) {
                     if (lane >= 16) *reinterpret_cast<uint4 *>(tile_p + tile_off(new_slot, lane - 16)) = new_row;
+                    if constexpr (I4) {
+                        const float ns = __shfl_sync(0xffffffffu, new_scale, 16);
+                        if (gq == new_slot) vsc0 = ns;
+                        if (gq + 8 == new_slot) vsc1 = ns;
+                    }
                     __syncwarp();
+                }
+                if constexpr (I4) {   // a value is scale * code: the weight of a key takes its row's scale
+                    w0 = pack_bf16(p00 * vsc0, p01 * vsc0);
+                    w1 = pack_bf16(p10 * vsc1, p11 * vsc1);
+                    pb0 = movmatrix_trans(w0);
+                    pb1 = movmatrix_trans(w1);
                 }
                 if (ntok < kPage) {
                     // slots past the sequence end may hold anything; they must not reach the tensor core, not even
@@ -761,7 +870,7 @@ decode_step_kernel(const StepArgs a, const __grid_constant__ CUtensorMap k_map, 
                     mma_16816<E4M3>(o[mt], af, pb0, pb1);
                 }
                 __syncwarp();
-                if constexpr (!E4M3) {
+                if constexpr (!WIDE) {
                     if (patch_here || ntok < kPage) fence_proxy_async_smem();
                     if (lane == 0) mbar_arrive(&tail->empty[st]);
                 }
@@ -912,12 +1021,12 @@ decode_step_kernel(const StepArgs a, const __grid_constant__ CUtensorMap k_map, 
 // kernel's CTAs leave anyway.
 constexpr int kStages = 32;
 
-template <int G, bool APPEND, bool E4M3>
+template <int G, bool APPEND, int KV>
 arb_status launch_variant(Ctx *ctx, const StepArgs &a, const CUtensorMap &km, const CUtensorMap &vm, cudaStream_t stream) {
     static bool attr_set[64] = {};
     if (!attr_set[ctx->device & 63]) {
-        if (cudaFuncSetAttribute(decode_step_kernel<G, kStages, APPEND, E4M3>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 (int)smem_bytes<G, kStages, E4M3>(kMaxBatch)) != cudaSuccess)
+        if (cudaFuncSetAttribute(decode_step_kernel<G, kStages, APPEND, KV>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 (int)smem_bytes<G, kStages, KV>(kMaxBatch)) != cudaSuccess)
             return ARB_ERR_CUDA;
         attr_set[ctx->device & 63] = true;
     }
@@ -927,21 +1036,22 @@ arb_status launch_variant(Ctx *ctx, const StepArgs &a, const CUtensorMap &km, co
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(ctx->num_sms);
     cfg.blockDim = dim3(kNT);
-    cfg.dynamicSmemBytes = smem_bytes<G, kStages, E4M3>(a.batch);
+    cfg.dynamicSmemBytes = smem_bytes<G, kStages, KV>(a.batch);
     cfg.stream = stream;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    if (cudaLaunchKernelEx(&cfg, decode_step_kernel<G, kStages, APPEND, E4M3>, a, km, vm) != cudaSuccess) return ARB_ERR_CUDA;
+    if (cudaLaunchKernelEx(&cfg, decode_step_kernel<G, kStages, APPEND, KV>, a, km, vm) != cudaSuccess) return ARB_ERR_CUDA;
     ctx->launches++;
     return ARB_OK;
 }
 
-// The E4M3 form exists with the cache write only: decode alone over an E4M3 cache is arb_attn_decode_e4m3.
+// The E4M3 and the 4-bit forms exist with the cache write only (decode alone over an E4M3 cache is arb_attn_decode_e4m3).
 template <int G>
-arb_status launch_g(Ctx *ctx, const StepArgs &a, bool e4m3, const CUtensorMap &km, const CUtensorMap &vm, cudaStream_t stream) {
-    if (e4m3) return launch_variant<G, true, true>(ctx, a, km, vm, stream);
-    return a.k_new != nullptr ? launch_variant<G, true, false>(ctx, a, km, vm, stream)
-                              : launch_variant<G, false, false>(ctx, a, km, vm, stream);
+arb_status launch_g(Ctx *ctx, const StepArgs &a, int kv, const CUtensorMap &km, const CUtensorMap &vm, cudaStream_t stream) {
+    if (kv == kKvE4m3) return launch_variant<G, true, kKvE4m3>(ctx, a, km, vm, stream);
+    if (kv == kKvI4) return launch_variant<G, true, kKvI4>(ctx, a, km, vm, stream);
+    return a.k_new != nullptr ? launch_variant<G, true, kKvBf16>(ctx, a, km, vm, stream)
+                              : launch_variant<G, false, kKvBf16>(ctx, a, km, vm, stream);
 }
 
 }  // namespace
@@ -953,16 +1063,23 @@ bool decode_step_supported(const arb_attn_params &p) {
     return p.dtype == ARB_BF16 && p.head_dim == kD && g >= 1 && g <= 8 && tma_available();
 }
 
-// k_new == nullptr: attention only (seq_lens is not written).  scales == nullptr: a bf16 cache; else an E4M3 cache
-// with scales = {k_scale, v_scale, k_inv_scale, v_inv_scale} (k_new is required then).
+// k_new == nullptr: attention only (seq_lens is not written).  scales != nullptr: an E4M3 cache with scales =
+// {k_scale, v_scale, k_inv_scale, v_inv_scale}; k_row_scales != nullptr: a 4-bit cache with its two scale pools
+// (k_new is required for both); neither: a bf16 cache.
 arb_status launch_decode_step(Ctx *ctx, const arb_attn_params &p, const void *q, const void *k_new, const void *v_new,
                               void *k_pages, void *v_pages, const float *scales, const int32_t *block_table,
-                              int32_t *seq_lens, const int32_t *q_lens, void *out, cudaStream_t stream) {
+                              int32_t *seq_lens, const int32_t *q_lens, void *out, cudaStream_t stream,
+                              float *k_row_scales, float *v_row_scales) {
     alignas(64) CUtensorMap km, vm;
-    const bool e4m3 = scales != nullptr;
-    if (e4m3 && k_new == nullptr) return ARB_ERR_INVALID_ARG;
+    const bool e4m3 = scales != nullptr, i4 = k_row_scales != nullptr;
+    if ((e4m3 || i4) && k_new == nullptr) return ARB_ERR_INVALID_ARG;
+    if (e4m3 && i4) return ARB_ERR_INVALID_ARG;
     bool whole_rows = false;
-    if (e4m3) {
+    if (i4) {
+        if (!pool_map(ctx, &km, k_pages, p.num_pages, p.num_kv_heads, PoolView::kI4) ||
+            !pool_map(ctx, &vm, v_pages, p.num_pages, p.num_kv_heads, PoolView::kI4))
+            return ARB_ERR_CUDA;
+    } else if (e4m3) {
         if (!pool_map(ctx, &km, k_pages, p.num_pages, p.num_kv_heads, PoolView::kE4m3) ||
             !pool_map(ctx, &vm, v_pages, p.num_pages, p.num_kv_heads, PoolView::kE4m3))
             return ARB_ERR_CUDA;
@@ -1013,15 +1130,18 @@ arb_status launch_decode_step(Ctx *ctx, const arb_attn_params &p, const void *q,
     a.v_scale = e4m3 ? scales[1] : 1.0f;
     a.k_inv_scale = e4m3 ? scales[2] : 1.0f;
     a.v_inv_scale = e4m3 ? scales[3] : 1.0f;
+    a.k_scales = k_row_scales;
+    a.v_scales = v_row_scales;
+    const int kv = i4 ? kKvI4 : e4m3 ? kKvE4m3 : kKvBf16;
     switch (g) {
-        case 1: return launch_g<1>(ctx, a, e4m3, km, vm, stream);
-        case 2: return launch_g<2>(ctx, a, e4m3, km, vm, stream);
-        case 3: return launch_g<3>(ctx, a, e4m3, km, vm, stream);
-        case 4: return launch_g<4>(ctx, a, e4m3, km, vm, stream);
-        case 5: return launch_g<5>(ctx, a, e4m3, km, vm, stream);
-        case 6: return launch_g<6>(ctx, a, e4m3, km, vm, stream);
-        case 7: return launch_g<7>(ctx, a, e4m3, km, vm, stream);
-        case 8: return launch_g<8>(ctx, a, e4m3, km, vm, stream);
+        case 1: return launch_g<1>(ctx, a, kv, km, vm, stream);
+        case 2: return launch_g<2>(ctx, a, kv, km, vm, stream);
+        case 3: return launch_g<3>(ctx, a, kv, km, vm, stream);
+        case 4: return launch_g<4>(ctx, a, kv, km, vm, stream);
+        case 5: return launch_g<5>(ctx, a, kv, km, vm, stream);
+        case 6: return launch_g<6>(ctx, a, kv, km, vm, stream);
+        case 7: return launch_g<7>(ctx, a, kv, km, vm, stream);
+        case 8: return launch_g<8>(ctx, a, kv, km, vm, stream);
         default: return ARB_ERR_UNSUPPORTED;
     }
 }

@@ -68,8 +68,23 @@ bool encode_pool_map3(CUtensorMap *map, const void *pool, int num_pages, int num
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// A pool of 4-bit codes: rows of 64 bytes; one box is the 16 rows of a (page, kv head), landing row-major (no swizzle:
+// the rows are read by plain shared-memory loads, 32 bytes per lane, before they are widened).
+bool encode_pool_map_i4(CUtensorMap *map, const void *pool, int num_pages, int num_kv_heads) {
+    EncodeTiledFn fn = encode_tiled_fn();
+    if (!fn) return false;
+    const cuuint64_t dims[2] = {(cuuint64_t)kD / 2, (cuuint64_t)num_pages * num_kv_heads * kPage};
+    const cuuint64_t strides[1] = {(cuuint64_t)kD / 2};
+    const cuuint32_t box[2] = {(cuuint32_t)kD / 2, (cuuint32_t)kPage};
+    const cuuint32_t estr[2] = {1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void *>(pool), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 namespace {
 bool encode_view(CUtensorMap *map, const void *pool, int num_pages, int num_kv_heads, PoolView view) {
+    if (view == PoolView::kI4) return encode_pool_map_i4(map, pool, num_pages, num_kv_heads);
     if (view == PoolView::kBf16WholeRows) return encode_pool_map3(map, pool, num_pages, num_kv_heads);
     return encode_pool_map(map, pool, num_pages, num_kv_heads, view == PoolView::kE4m3);
 }

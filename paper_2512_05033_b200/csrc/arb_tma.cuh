@@ -20,6 +20,7 @@ enum class PoolView : int {
     kBf16HalfRows = 0,    // 2-D, box 16 rows x 64 elements (one 128-byte-swizzled half tile)
     kE4m3 = 1,            // 2-D over E4M3 codes, box 16 whole rows of 128 bytes
     kBf16WholeRows = 2,   // 3-D (64 elements, rows, 2 halves), box 16 rows x both halves: a page in one copy
+    kI4 = 3,              // 2-D over 4-bit codes, box 16 whole rows of 64 bytes, not swizzled
 };
 
 // 3-D view kBf16WholeRows; false if the driver refuses the encoding (the caller then uses kBf16HalfRows).

@@ -314,3 +314,145 @@ def test_decode_step_e4m3_refusals():
     keep = torch.tensor([1, 0, 1], dtype=torch.int32)
     ref, _ = oracle.attn_e4m3(inp.q[[0, 2]], ok, ov, KS, VS, inp.block_table, osl, keep)
     H.assert_close(out[[0, 2]].double().cpu().numpy(), ref, BF, tight=3e-3)
+
+
+# ---- arb_decode_step_i4: the same token over a 4-bit cache (per-row scales) ----------------------------------------
+
+def _i4_case(B, Hq, Hkv, sl, ql, seed, extra=4, row_std=None):
+    """Pools quantised by the oracle; slots past the ends hold nibble 0 (a code the format never writes) and NaN scales."""
+    inp = wl.small_attn_case(B, Hq, Hkv, 128, BF, sl, ql, seed=seed, extra_tokens=extra)
+    if row_std is not None:     # rows of very different magnitude: the per-row scales matter
+        g = torch.Generator().manual_seed(seed + 1)
+        for pool in (inp.k_pages, inp.v_pages):
+            f = torch.exp(torch.randn(pool.shape[:3], generator=g) * row_std)[..., None]
+            pool.copy_((pool.float() * f).to(pool.dtype))
+    kc, ks = oracle.i4_encode(inp.k_pages)
+    vc, vs = oracle.i4_encode(inp.v_pages)
+    kc, vc, ks, vs = torch.from_numpy(kc), torch.from_numpy(vc), torch.from_numpy(ks), torch.from_numpy(vs)
+    for b in range(B):
+        for pos in range(sl[b], sl[b] + extra):
+            page = int(inp.block_table[b, pos // 16])
+            kc[page, :, pos % 16, :] = 0
+            vc[page, :, pos % 16, :] = 0
+            ks[page, :, pos % 16] = float("nan")
+            vs[page, :, pos % 16] = float("nan")
+    return inp, kc, vc, ks, vs
+
+
+def _i4_close(out, ref, v_scales):
+    """The bar of the other decode tests (bf16 rounding of the output, 2^-8 |ref|, plus 3e-3 for N(0,1) values), its
+    absolute part scaled with the size of the values: the weights reach the tensor core rounded to bf16, an error of
+    2^-9 of weight x value per key, and the largest value of a pool of N(0,1) rows is about 4.5."""
+    s = np.asarray(v_scales, dtype=np.float64)
+    vmax = float(np.nanmax(s)) * 7.0
+    err = np.abs(out.double().cpu().numpy() - ref)
+    assert np.isfinite(out.float().cpu().numpy()).all()
+    bar = 2.0 ** -8 * np.abs(ref) + 3e-3 * max(1.0, vmax / 4.5)
+    assert (err <= bar).all(), f"error {err.max():.3e} above the bar (largest value {vmax:.1f})"
+
+
+def _same_f32_bits(a, b):
+    return torch.equal(a.cpu().contiguous().view(torch.int32), torch.as_tensor(np.asarray(b)).contiguous().view(torch.int32))
+
+
+@pytest.mark.parametrize("case", E4M3_STEP_CASES)
+def test_decode_step_i4_matches_quantising_append_then_attention(case):
+    B, Hq, Hkv, sl, ql = case
+    inp, kc, vc, ks, vs = _i4_case(B, Hq, Hkv, sl, ql, 950 + len(sl) + Hq, row_std=1.0 if B % 2 else None)
+    k_new, v_new = _new_rows(inp, sum(ql), 9700 + Hq)
+    k_new[0, 0, :] = 0.0                                             # a row of zeros: scale 0, codes 0
+    v_new[0, 0, :8] = torch.tensor([7, -7, 3.5, 2.5, -0.5, 0.49, 6.5, -6.5])   # ties (when the row's max is 7)
+    v_new[0, 0, 8:] = 0.0
+    c = H.ctx()
+    d = inp.to("cuda")
+    dk, dv, dks, dvs = kc.cuda(), vc.cuda(), ks.cuda(), vs.cuda()
+    out = torch.full_like(d.q, float("nan"))
+    c.decode_step_i4(d.q, k_new.cuda(), v_new.cuda(), dk, dv, dks, dvs, d.block_table, d.seq_lens, d.q_lens, out=out)
+    assert c.poll_status() == 0
+    ok, ov, oks, ovs, osl, st = oracle.kv_append_i4(k_new, v_new, inp.block_table, inp.seq_lens, inp.q_lens, kc, vc, ks, vs)
+    ref, st2 = oracle.attn_i4(inp.q, _live(ok, oks, inp, osl)[0], _live(ov, ovs, inp, osl)[0], _live(ok, oks, inp, osl)[1],
+                              _live(ov, ovs, inp, osl)[1], inp.block_table, osl, inp.q_lens)
+    assert st == 0 and st2 == 0
+    assert np.array_equal(d.seq_lens.cpu().numpy(), osl)
+    assert torch.equal(dk.cpu(), ok) and torch.equal(dv.cpu(), ov)                    # codes: bit for bit
+    assert _same_f32_bits(dks, oks) and _same_f32_bits(dvs, ovs)                      # scales: bit for bit (NaN included)
+    _i4_close(out, ref, ovs)
+
+
+def _live(codes, scales, inp, lens):
+    """The pools with every slot past a sequence's end given a finite scale (the oracle's attention decodes whole pools
+    before it looks at the lengths; what those slots hold must not matter to the result)."""
+    s = torch.as_tensor(np.asarray(scales)).clone()
+    s[torch.isnan(s)] = 0.0
+    return codes, s
+
+
+def test_decode_step_i4_chain_in_place_and_as_a_graph():
+    c = H.ctx()
+    B, T = 5, 10
+    inp, kc, vc, ks, vs = _i4_case(B, 12, 2, [500, 33, 2100, 0, 1500], [1] * B, 961, extra=T + 2, row_std=0.7)
+    q = wl.normal((T, B, 12, 128), 1.0, BF, "cpu", 962)
+    kn = wl.normal((T, B, 2, 128), 1.0, BF, "cpu", 963)
+    vn = wl.normal((T, B, 2, 128), 3.0, BF, "cpu", 964)
+    d = inp.to("cuda")
+    pools = [kc.cuda(), vc.cuda(), ks.cuda(), vs.cuda()]
+    start = [t.clone() for t in pools] + [d.seq_lens.clone()]
+    dq, dkn, dvn = q.cuda(), kn.cuda(), vn.cuda()
+    outs = [torch.full((B, 12, 128), float("nan"), dtype=BF, device="cuda") for _ in range(T)]
+
+    def chain():
+        for t in range(T):
+            c.decode_step_i4(dq[t], dkn[t], dvn[t], *pools, d.block_table, d.seq_lens, d.q_lens, out=outs[t])
+
+    chain()
+    assert c.poll_status() == 0
+    k, v, sk, sv, sl = kc, vc, ks, vs, inp.seq_lens.numpy()
+    for t in range(T):
+        k, v, sk, sv, sl, st = oracle.kv_append_i4(kn[t], vn[t], inp.block_table, sl, inp.q_lens, k, v, sk, sv)
+        ref, st2 = oracle.attn_i4(q[t], k, v, _live(k, sk, inp, sl)[1], _live(v, sv, inp, sl)[1], inp.block_table, sl, inp.q_lens)
+        assert st == 0 and st2 == 0
+        _i4_close(outs[t], ref, sv)
+    assert np.array_equal(d.seq_lens.cpu().numpy(), sl)
+    assert torch.equal(pools[0].cpu(), k) and torch.equal(pools[1].cpu(), v)
+    assert _same_f32_bits(pools[2], sk) and _same_f32_bits(pools[3], sv)
+    eager = [o.clone() for o in outs]
+    gr = torch.cuda.CUDAGraph()
+    for t_, s_ in zip(pools + [d.seq_lens], start):
+        t_.copy_(s_)
+    with torch.cuda.graph(gr):
+        chain()
+    for t_, s_ in zip(pools + [d.seq_lens], start):
+        t_.copy_(s_)
+    gr.replay()
+    torch.cuda.synchronize()
+    for t in range(T):
+        assert torch.equal(outs[t], eager[t]), t
+
+
+def test_decode_step_i4_refusals():
+    from paper_2512_05033_b200 import binding
+    c = H.ctx()
+    inp, kc, vc, ks, vs = _i4_case(3, 12, 2, [100, 64, 300], [1, 1, 1], 971, extra=0)
+    k_new, v_new = _new_rows(inp, 3, 972)
+    inp.seq_lens[1] = inp.block_table.shape[1] * 16          # full: one more token does not fit
+    d = inp.to("cuda")
+    pools = [kc.cuda(), vc.cuda(), ks.cuda(), vs.cuda()]
+    out = torch.full_like(d.q, float("nan"))
+    c.decode_step_i4(d.q, k_new.cuda(), v_new.cuda(), *pools, d.block_table, d.seq_lens, d.q_lens, out=out)
+    assert c.poll_status() == binding.DEV_BAD_SEQ_LEN
+    ok, ov, oks, ovs, osl, st = oracle.kv_append_i4(k_new, v_new, inp.block_table, inp.seq_lens, inp.q_lens, kc, vc, ks, vs)
+    assert st == oracle.BAD_SEQ_LEN
+    assert np.array_equal(d.seq_lens.cpu().numpy(), osl)
+    assert torch.equal(pools[0].cpu(), ok) and torch.equal(pools[1].cpu(), ov)
+    assert _same_f32_bits(pools[2], oks) and _same_f32_bits(pools[3], ovs)
+    assert float(out[1].abs().max()) == 0.0
+    keep = torch.tensor([1, 0, 1], dtype=torch.int32)
+    ref, _ = oracle.attn_i4(inp.q[[0, 2]], ok, ov, oks, ovs, inp.block_table, osl, keep)
+    H.assert_close(out[[0, 2]].double().cpu().numpy(), ref, BF, tight=3e-3)
+    with pytest.raises(binding.ArbError):      # scale pools are required: a null pool is refused by the library
+        p = c.params_for(d.q, inp.k_pages, d.block_table, 1)
+        st = binding.lib.arb_decode_step_i4(c._h, __import__("ctypes").byref(p), d.q.data_ptr(), k_new.cuda().data_ptr(),
+                                            v_new.cuda().data_ptr(), pools[0].data_ptr(), pools[1].data_ptr(), None, None,
+                                            d.block_table.data_ptr(), d.seq_lens.data_ptr(), d.q_lens.data_ptr(),
+                                            out.data_ptr(), None)
+        binding._check(st, "arb_decode_step_i4")

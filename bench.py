@@ -377,6 +377,7 @@ def run_ours(args):
                                 "before it, which is what a token of Algorithm 1 sees"}
                 result["decode_step"] = run_decode_step(ctx, dev, peak, peak_kind)
                 result["decode_step"]["e4m3"] = run_decode_step(ctx, dev, peak, peak_kind, e4m3=True)
+                result["decode_step"]["i4"] = run_decode_step(ctx, dev, peak, peak_kind, i4=True)
                 result["target_shaped_decode"] = run_target_decode(ctx, dev, peak)
                 result["step_scoring"] = run_step_scoring(ctx, dev)
                 result["mixed_loop"] = run_mixed_loop(ctx, dev)
@@ -502,18 +503,29 @@ def run_target_decode(ctx, dev, peak):
                              "pct_of_nominal_8TBs": round(100 * gbs2 / NOMINAL_HBM_GBS, 2)}}
 
 
-def run_decode_step(ctx, dev, peak, peak_kind, layers=LAYERS, e4m3=False):
+def run_decode_step(ctx, dev, peak, peak_kind, layers=LAYERS, e4m3=False, i4=False, shape=None):
     """Supplementary: the single-launch decode token (arb_decode_step: cache write + attention + combine + length
     update) on the draft-shaped batch: `layers` calls per CUDA graph, each on its own KV pool and its own length
     array (a layer's cache grows by one token per replay), every call waiting for the one before it.  e4m3: the
     same over pools of E4M3 codes (arb_decode_step_e4m3)."""
-    shape = wl.DRAFT_DECODE
+    shape = shape or wl.DRAFT_DECODE
     inp = wl.make_attn_inputs(shape, device=dev, seed=shape.seed, extra_tokens=2048)
     if e4m3:
         g8 = torch.Generator(device=dev)
         g8.manual_seed(3200)
         pools = [tuple(torch.randint(0, 0x7f, inp.k_pages.shape, generator=g8, device=dev, dtype=torch.uint8) for _ in range(2))
                  for _ in range(layers)]
+    elif i4:   # pools of random nibbles 1..15 and scales around 0.15 (what N(0,1) rows of 128 values give)
+        g4 = torch.Generator(device=dev)
+        g4.manual_seed(3300)
+        cshape = inp.k_pages.shape[:3] + (shape.head_dim // 2,)
+        def codes():
+            lo = torch.randint(1, 16, cshape, generator=g4, device=dev, dtype=torch.uint8)
+            hi = torch.randint(1, 16, cshape, generator=g4, device=dev, dtype=torch.uint8)
+            return lo | (hi << 4)
+        def scales():
+            return 0.1 + 0.1 * torch.rand(inp.k_pages.shape[:3], generator=g4, device=dev, dtype=torch.float32)
+        pools = [(codes(), codes(), scales(), scales()) for _ in range(layers)]
     else:
         pools = [(inp.k_pages, inp.v_pages)] + [wl.make_kv_pool(shape, inp.num_pages, dev, shape.seed * 100 + l) for l in range(1, layers)]
     lens = [inp.seq_lens.clone() for _ in pools]
@@ -523,7 +535,11 @@ def run_decode_step(ctx, dev, peak, peak_kind, layers=LAYERS, e4m3=False):
     p = ctx.params_for(inp.q, pools[0][0], inp.block_table, 1)
 
     def step():
-        for (k, v), sl in zip(pools, lens):
+        for pool, sl in zip(pools, lens):
+            if i4:
+                ctx.decode_step_i4(inp.q, k_new, v_new, *pool, inp.block_table, sl, inp.q_lens, out=out, params=p)
+                continue
+            k, v = pool
             if e4m3:
                 ctx.decode_step_e4m3(inp.q, k_new, v_new, k, v, 0.01, 0.01, 100.0, 100.0, inp.block_table, sl, inp.q_lens,
                                      out=out, params=p)
@@ -539,14 +555,17 @@ def run_decode_step(ctx, dev, peak, peak_kind, layers=LAYERS, e4m3=False):
     us = ms / layers * 1e3
     b = attn_bytes(shape, inp.seq_lens.cpu().to(torch.int64) + 300, inp.q_lens.cpu().to(torch.int64))
     rows = shape.batch * shape.num_kv_heads * shape.head_dim
-    if e4m3:   # codes: one byte per cache element; the new rows are read as bf16 and written as codes
+    if i4:     # codes: half a byte per element and 4 bytes of scale per row of 128
+        nbytes = b["kv"] // 4 + b["kv"] // 64 + b["qo"] + b["table"] + 2 * rows * 2 + rows // 2
+    elif e4m3:   # codes: one byte per cache element; the new rows are read as bf16 and written as codes
         nbytes = b["kv"] // 2 + b["qo"] + b["table"] + 2 * rows * 3
     else:
         nbytes = b["total"] + 4 * rows * 2   # + the new rows, read and written
     assert ctx.poll_status() == 0
-    name = "arb_decode_step_e4m3" if e4m3 else "arb_decode_step"
+    name = "arb_decode_step_i4" if i4 else "arb_decode_step_e4m3" if e4m3 else "arb_decode_step"
     return {"us_per_call": round(us, 3), "kv_tokens": b["tokens"],
-            "roofline": hbm_roofline("decode_step_kernel<E4M3>" if e4m3 else "decode_step_kernel", nbytes, us, peak, peak_kind),
+            "roofline": hbm_roofline("decode_step_kernel<4-bit>" if i4 else "decode_step_kernel<E4M3>" if e4m3 else "decode_step_kernel", nbytes, us,
+                                    peak, peak_kind),
             "note": f"{layers} {name} calls per CUDA graph, none overlapped: what a token of Algorithm 1 costs per layer"}
 
 

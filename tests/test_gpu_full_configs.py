@@ -203,6 +203,36 @@ def test_draft_shaped_decode_step_e4m3_full():
     assert torch.equal(dk.cpu(), kc) and torch.equal(dv.cpu(), vc)
 
 
+def test_draft_shaped_decode_step_i4_full():
+    """arb_decode_step_i4 on the draft-shaped batch: two tokens in a row on one 4-bit cache; codes and scales bit for
+    bit, lengths exact, every row."""
+    shape = wl.DRAFT_DECODE
+    inp = wl.make_attn_inputs(shape, extra_tokens=8)
+    kc, ks = (torch.from_numpy(x) for x in oracle.i4_encode(inp.k_pages))
+    vc, vs = (torch.from_numpy(x) for x in oracle.i4_encode(inp.v_pages))
+    d = inp.to("cuda")
+    pools = [kc.cuda(), vc.cuda(), ks.cuda(), vs.cuda()]
+    c = H.ctx()
+    sl = inp.seq_lens.numpy().copy()
+    ones = torch.ones(shape.batch, dtype=torch.int32)
+    outs, news = [], []
+    for t in range(2):
+        q = wl.normal((shape.batch, shape.num_q_heads, shape.head_dim), 1.0, BF, "cpu", 9700 + t)
+        kn = wl.normal((shape.batch, shape.num_kv_heads, shape.head_dim), 1.0, BF, "cpu", 9800 + t)
+        vn = wl.normal((shape.batch, shape.num_kv_heads, shape.head_dim), 1.0, BF, "cpu", 9900 + t)
+        news.append((q, kn, vn))
+        outs.append(c.decode_step_i4(q.cuda(), kn.cuda(), vn.cuda(), *pools, d.block_table, d.seq_lens, d.q_lens))
+    assert c.poll_status() == 0
+    for (q, kn, vn), out in zip(news, outs):
+        kc, vc, ks, vs, sl, st = oracle.kv_append_i4(kn, vn, inp.block_table, sl, ones, kc, vc, ks, vs)
+        ref, st2 = oracle.attn_i4(q, kc, vc, ks, vs, inp.block_table, sl, ones)
+        assert st == 0 and st2 == 0
+        H.assert_close(out.double().cpu().numpy(), ref, BF, tight=3e-3)
+    assert np.array_equal(d.seq_lens.cpu().numpy(), sl)
+    assert torch.equal(pools[0].cpu(), kc) and torch.equal(pools[1].cpu(), vc)
+    assert torch.equal(pools[2].cpu(), torch.as_tensor(np.asarray(ks))) and torch.equal(pools[3].cpu(), torch.as_tensor(np.asarray(vs)))
+
+
 def test_step_scoring_full_over_the_e4m3_cache():
     """arb_attn_e4m3 on the step-scoring batch at full size (pools quantised by the oracle), every element."""
     shape = wl.STEP_SCORING

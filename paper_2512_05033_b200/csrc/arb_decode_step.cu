@@ -25,12 +25,16 @@
 //     tile in shared memory (the tile arrives with whatever the slot held) and stores it to the pool; the
 //     lengths move forward once every CTA has read them (a counter in the prologue tells the last reader).
 //
-// Compiled a second time (template parameter E4M3) the kernel serves an E4M3 cache (arb_decode_step_e4m3: the token
+// The template parameter KV names the cache.  Compiled a second time (KV = E4M3) the kernel serves an E4M3 cache (arb_decode_step_e4m3: the token
 // of a quantised draft).  A page tile is 2 KB of codes; the consumer warp that owns it widens it to f16 (exact) into
 // a tile of its own in shared memory, laid out like a bf16 tile, frees the ring stage at once, and runs the same
 // fragment loads and MMAs on f16 operands (q converted bf16 -> f16, P rounded to f16).  The token's new rows are
 // quantised by the warp that patches them in (x * inv_scale, nearest code, saturating: the arithmetic of
 // arb_kv_append_e4m3), stored to the pool as codes and patched into the widened tile.
+// A third time (KV = 4-bit; arb_decode_step_i4) it serves a cache of 4-bit codes with one fp32 scale per (token, kv head)
+// row: a stage is 1 KB of codes and the rows' 16 scales; the consumer warp widens the codes to bf16 (exact), keeps the
+// scales of its two keys in registers, multiplies them into the scores and into the weights, and runs the bf16 MMAs; the
+// token's rows are quantised in the kernel (row max by shuffles, IEEE divisions, nearest with ties to even).
 #include "arb_decode_tc.cuh"
 
 namespace arb {

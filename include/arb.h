@@ -475,6 +475,22 @@ arb_status arb_decode_step_i4(arb_ctx *ctx, const arb_attn_params *params, const
                               arb_stream_t stream);
 
 /*
+ * The 4-bit cache's quantising append: arb_kv_append with the rows encoded on the way in (the format of
+ * arb_decode_step_i4: per-row scale max|x| / 7, codes rint(x * 7 / max|x|) in -7 .. 7, interleaved nibbles).  The cache
+ * write of a step's tokens, or of a prefix (Algorithm 1 absorbs steps into the caches; Section 5.1's quantised drafts).
+ *
+ *   params, total_new, k_new, v_new, block_table, seq_lens, new_lens, update_lens
+ *              as for arb_kv_append; dtype ARB_BF16 (the type of k_new / v_new), head_dim 128.
+ *   k_codes, v_codes    uint8 pools [num_pages, Hkv, P, D / 2];  k_scales, v_scales    fp32 pools [num_pages, Hkv, P].
+ * Placement, refusals and status bits are arb_kv_append's; codes and scales are bit-identical to the format's definition.
+ * Errors: ARB_ERR_INVALID_ARG, ARB_ERR_UNSUPPORTED (dtype, head_dim, page size, batch), ARB_ERR_CUDA.
+ */
+arb_status arb_kv_append_i4(arb_ctx *ctx, const arb_attn_params *params, int32_t total_new, const void *k_new,
+                            const void *v_new, const int32_t *block_table, int32_t *seq_lens, const int32_t *new_lens,
+                            int32_t update_lens, uint8_t *k_codes, uint8_t *v_codes, float *k_scales, float *v_scales,
+                            arb_stream_t stream);
+
+/*
  * Spearman's rank correlation of two samples (Section 4.2, "Evaluation", and Tables 1-3 of the paper:
  * the correlation between the router's predicted scores and the oracle advantage Delta).  Each value is
  * replaced by its rank within its sample, equal values sharing the mean of the ranks they span, and

@@ -37,7 +37,7 @@ MAX_CLASSES = 16
 # every symbol include/arb.h declares
 EXPORTS = ("arb_create", "arb_destroy", "arb_attn_workspace_bytes", "arb_attn", "arb_attn_host",
            "arb_attn_host_begin", "arb_attn_host_wait",
-           "arb_attn_decode_static", "arb_decode_step", "arb_decode_step_e4m3", "arb_decode_step_i4",
+           "arb_attn_decode_static", "arb_decode_step", "arb_decode_step_e4m3", "arb_decode_step_i4", "arb_kv_append_i4",
            "arb_route", "arb_rollback", "arb_policy", "arb_route_classes", "arb_kv_append", "arb_kv_append_e4m3", "arb_attn_decode_e4m3", "arb_attn_e4m3", "arb_phase_lens", "arb_phase_lens_tokens", "arb_spearman",
            "arb_selftest_wait_timeout", "arb_selftest_guard_zones", "arb_poll_status", "arb_launch_count", "arb_status_string")
 
@@ -69,6 +69,9 @@ lib.arb_attn_decode_static.restype = ctypes.c_int
 lib.arb_attn_decode_static.argtypes = [ctypes.POINTER(AttnParams), _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp]
 lib.arb_decode_step.restype = ctypes.c_int
 lib.arb_decode_step.argtypes = [_vp, ctypes.POINTER(AttnParams), _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp]
+lib.arb_kv_append_i4.restype = ctypes.c_int
+lib.arb_kv_append_i4.argtypes = [_vp, ctypes.POINTER(AttnParams), ctypes.c_int32, _vp, _vp, _vp, _vp, _vp, ctypes.c_int32,
+                                 _vp, _vp, _vp, _vp, _vp]
 lib.arb_decode_step_i4.restype = ctypes.c_int
 lib.arb_decode_step_i4.argtypes = [_vp, ctypes.POINTER(AttnParams)] + [_vp] * 12
 lib.arb_decode_step_e4m3.restype = ctypes.c_int
@@ -319,6 +322,21 @@ class Context:
                                     _dev(out, "out", torch.bfloat16), _stream_ptr(stream))
         _check(st, "arb_decode_step_i4")
         return out
+
+    # -- arb_kv_append_i4 ---------------------------------------------------------------------
+    def kv_append_i4(self, k_new, v_new, block_table, seq_lens, new_lens, k_codes, v_codes, k_scales, v_scales,
+                     update_lens: bool = True, stream=None):
+        """In place: the new rows are quantised to the 4-bit format and written behind each sequence's tokens."""
+        num_pages, Hkv, P, half = k_codes.shape
+        B, max_pages = block_table.shape
+        p = attn_params(_dtype_code(k_new), B, Hkv, Hkv, 2 * half, num_pages, max_pages, 0, 0, 0.0, P, 0)
+        st = lib.arb_kv_append_i4(self._h, ctypes.byref(p), k_new.shape[0], _dev(k_new, "k_new", torch.bfloat16),
+                                  _dev(v_new, "v_new", torch.bfloat16), _dev(block_table, "block_table", torch.int32),
+                                  _dev(seq_lens, "seq_lens", torch.int32), _dev(new_lens, "new_lens", torch.int32),
+                                  1 if update_lens else 0, _dev(k_codes, "k_codes", torch.uint8),
+                                  _dev(v_codes, "v_codes", torch.uint8), _dev(k_scales, "k_scales", torch.float32),
+                                  _dev(v_scales, "v_scales", torch.float32), _stream_ptr(stream))
+        _check(st, "arb_kv_append_i4")
 
     # -- arb_route ----------------------------------------------------------------------------
     def route(self, hidden, w, b: float, tau: float, scores=None, decisions=None, stream=None):

@@ -712,6 +712,26 @@ arb_status arb_kv_append_e4m3(arb_ctx *ctx, const arb_attn_params *params, int32
                                  reinterpret_cast<cudaStream_t>(stream));
 }
 
+arb_status arb_kv_append_i4(arb_ctx *ctx, const arb_attn_params *params, int32_t total_new, const void *k_new,
+                            const void *v_new, const int32_t *block_table, int32_t *seq_lens, const int32_t *new_lens,
+                            int32_t update_lens, uint8_t *k_codes, uint8_t *v_codes, float *k_scales, float *v_scales,
+                            arb_stream_t stream) {
+    if (ctx == nullptr || params == nullptr || total_new < 0) return ARB_ERR_INVALID_ARG;
+    if (params->batch < 1 || params->num_kv_heads < 1 || params->num_pages < 1 || params->max_pages_per_seq < 1)
+        return ARB_ERR_INVALID_ARG;
+    if (params->dtype != ARB_BF16 || params->head_dim != 128) return ARB_ERR_UNSUPPORTED;
+    if (params->page_size != kPage || params->batch > kMaxBatch) return ARB_ERR_UNSUPPORTED;
+    if (!block_table || !seq_lens || !new_lens || !k_codes || !v_codes || !k_scales || !v_scales) return ARB_ERR_INVALID_ARG;
+    if (total_new == 0) return ARB_OK;
+    if (!k_new || !v_new) return ARB_ERR_INVALID_ARG;
+    if (!aligned16(k_new) || !aligned16(v_new) || !aligned16(k_codes) || !aligned16(v_codes) || !aligned16(k_scales) ||
+        !aligned16(v_scales))
+        return ARB_ERR_INVALID_ARG;
+    return launch_kv_append_i4(reinterpret_cast<Ctx *>(ctx), *params, total_new, k_new, v_new, block_table, seq_lens,
+                               new_lens, update_lens, k_codes, v_codes, k_scales, v_scales,
+                               reinterpret_cast<cudaStream_t>(stream));
+}
+
 arb_status arb_poll_status(arb_ctx *ctx, arb_stream_t stream, uint32_t *bits) {
     if (ctx == nullptr) return ARB_ERR_INVALID_ARG;
     Ctx *c = reinterpret_cast<Ctx *>(ctx);

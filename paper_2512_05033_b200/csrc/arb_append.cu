@@ -209,6 +209,92 @@ kv_append_e4m3_kernel(const AppendArgs a, float k_inv_scale, float v_inv_scale) 
     advance_lens_when_last(a, okay);
 }
 
+// The 4-bit cache's quantising append (bf16 rows of 128 values).  A row is held by 16 neighbouring threads, 8 values
+// each: its scale is max|x| / 7 over the 16 threads (shuffles within the half warp), its codes rint(x * (7 / max|x|))
+// clamped to -7 .. 7, both divisions IEEE; a thread's eight codes are one 32-bit word of nibbles (code + 8; nibbles
+// 0..7 = dimensions 0, 2, 4, 6, 1, 3, 5, 7 of the eight).  Same plan, same checks as kv_append_kernel.
+__device__ __forceinline__ uint32_t i4_word(const float (&x)[8], float m, float &scale) {
+    scale = m > 0.f ? __fdiv_rn(m, 7.f) : 0.f;
+    const float inv = m > 0.f ? __fdiv_rn(7.f, m) : 0.f;
+    uint32_t word = 0;
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+        const int c = max(-7, min(7, __float2int_rn(__fmul_rn(x[j], inv))));
+        word |= (uint32_t)(c + 8) << (4 * ((j >> 1) + 4 * (j & 1)));
+    }
+    return word;
+}
+
+__global__ void __launch_bounds__(kAppendThreads)
+kv_append_i4_kernel(const AppendArgs a, float *k_scales, float *v_scales) {
+    extern __shared__ int asm_[];
+    int *pref = asm_;
+    int *okay = pref + a.batch + 1;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int B = a.batch;
+    pdl_enter();
+    if (tid == 0) pref[0] = 0;
+    for (int b = tid; b < B; b += kAppendThreads) {
+        const uint32_t bad = append_check(a, b);
+        if (bad && blockIdx.x == 0) atomicOr(a.status, bad);
+        okay[b] = bad == 0;
+        const int n = a.new_lens[b];
+        pref[b + 1] = n > 0 ? n : 0;
+    }
+    __syncthreads();
+    if (warp == 0) {
+        int carry = 0;
+        for (int b0 = 0; b0 < B; b0 += 32) {
+            const int b = b0 + lane;
+            int v = b < B ? pref[b + 1] : 0;
+#pragma unroll
+            for (int off = 1; off < 32; off <<= 1) {
+                const int t = __shfl_up_sync(0xffffffffu, v, off);
+                if (lane >= off) v += t;
+            }
+            if (b < B) pref[b + 1] = v + carry;
+            carry += __shfl_sync(0xffffffffu, v, 31);
+        }
+    }
+    __syncthreads();
+    const int total = min(pref[B], a.total_new);
+    constexpr int kVecs = 16;                      // 16-byte pieces of a bf16 row of 128 values
+    constexpr int kRowsPerPass = kAppendThreads / kVecs;
+    const int sub = tid / kVecs, vec = tid - sub * kVecs;
+    const uint32_t half_mask = 0xffffu << (lane & 16);   // the 16 lanes that hold this row
+    const long long nrows = (long long)total * a.Hkv;
+    for (long long r = (long long)blockIdx.x * kRowsPerPass + sub; r < nrows; r += (long long)gridDim.x * kRowsPerPass) {
+        const int tok = (int)(r / a.Hkv), h = (int)(r - (long long)tok * a.Hkv);
+        int lo = 0, hi = B;
+        while (hi - lo > 1) {
+            const int mid = (lo + hi) >> 1;
+            if (pref[mid] <= tok) lo = mid; else hi = mid;
+        }
+        if (!okay[lo]) continue;   // (the same for the 16 lanes of the row)
+        const int pos = a.seq_lens[lo] + (tok - pref[lo]);
+        const int page = a.block_table[(size_t)lo * a.max_pages + pos / kPage];
+        const size_t slot_row = ((size_t)page * a.Hkv + h) * kPage + (pos % kPage);
+        const size_t src = (size_t)r * a.row_bytes + (size_t)vec * 16;
+        float kf[8], vf[8];
+        Elt<__nv_bfloat16>::unpack(__ldg(reinterpret_cast<const uint4 *>(a.k_new + src)), kf);
+        Elt<__nv_bfloat16>::unpack(__ldg(reinterpret_cast<const uint4 *>(a.v_new + src)), vf);
+        float mk = 0.f, mv = 0.f;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) { mk = fmaxf(mk, fabsf(kf[j])); mv = fmaxf(mv, fabsf(vf[j])); }
+#pragma unroll
+        for (int off = 8; off >= 1; off >>= 1) {
+            mk = fmaxf(mk, __shfl_xor_sync(half_mask, mk, off));
+            mv = fmaxf(mv, __shfl_xor_sync(half_mask, mv, off));
+        }
+        float ks, vs;
+        const uint32_t kw = i4_word(kf, mk, ks), vw = i4_word(vf, mv, vs);
+        *reinterpret_cast<uint32_t *>(a.k_pages + slot_row * 64 + vec * 4) = kw;
+        *reinterpret_cast<uint32_t *>(a.v_pages + slot_row * 64 + vec * 4) = vw;
+        if (vec == 0) { k_scales[slot_row] = ks; v_scales[slot_row] = vs; }
+    }
+    advance_lens_when_last(a, okay);
+}
+
 }  // namespace
 
 arb_status launch_kv_append(Ctx *ctx, const arb_attn_params &p, int total_new, const void *k_new, const void *v_new,
@@ -273,6 +359,37 @@ arb_status launch_kv_append_e4m3(Ctx *ctx, const arb_attn_params &p, int total_n
         p.dtype == ARB_BF16
             ? launch_pdl(kv_append_e4m3_kernel<__nv_bfloat16>, dim3(grid), dim3(kAppendThreads), smem, stream, a, k_inv_scale, v_inv_scale)
             : launch_pdl(kv_append_e4m3_kernel<float>, dim3(grid), dim3(kAppendThreads), smem, stream, a, k_inv_scale, v_inv_scale);
+    ctx->launches++;
+    return err == cudaSuccess ? ARB_OK : ARB_ERR_CUDA;
+}
+
+arb_status launch_kv_append_i4(Ctx *ctx, const arb_attn_params &p, int total_new, const void *k_new, const void *v_new,
+                               const int32_t *block_table, int32_t *seq_lens, const int32_t *new_lens, int update_lens,
+                               void *k_codes, void *v_codes, float *k_scales, float *v_scales, cudaStream_t stream) {
+    AppendArgs a;
+    a.k_new = static_cast<const char *>(k_new);
+    a.v_new = static_cast<const char *>(v_new);
+    a.k_pages = static_cast<char *>(k_codes);
+    a.v_pages = static_cast<char *>(v_codes);
+    a.block_table = block_table;
+    a.seq_lens = seq_lens;
+    a.new_lens = new_lens;
+    a.status = ctx->status;
+    a.batch = p.batch;
+    a.Hkv = p.num_kv_heads;
+    a.num_pages = p.num_pages;
+    a.max_pages = p.max_pages_per_seq;
+    a.row_bytes = p.head_dim * 2;   // of the bf16 source rows
+    a.total_new = total_new;
+    a.update_lens = update_lens;
+    a.done_counter = ctx->rot + (size_t)kRotSets * kRotCounters + kRotSets + 3;
+    const int rows_per_pass = kAppendThreads / 16;
+    const long long nrows = (long long)total_new * p.num_kv_heads;
+    long long want = (nrows + rows_per_pass - 1) / rows_per_pass;
+    const long long cap = (long long)ctx->num_sms * 4;
+    const int grid = (int)(want < 1 ? 1 : (want > cap ? cap : want));
+    const size_t smem = sizeof(int) * (2 * (size_t)p.batch + 1);
+    const cudaError_t err = launch_pdl(kv_append_i4_kernel, dim3(grid), dim3(kAppendThreads), smem, stream, a, k_scales, v_scales);
     ctx->launches++;
     return err == cudaSuccess ? ARB_OK : ARB_ERR_CUDA;
 }

@@ -332,6 +332,9 @@ arb_status launch_kv_append_e4m3(Ctx *ctx, const arb_attn_params &p, int total_n
 arb_status launch_decode_e4m3(Ctx *ctx, const arb_attn_params &p, const void *q, const void *k_pages,
                               const void *v_pages, float k_scale, float v_scale, const int32_t *block_table,
                               const int32_t *seq_lens, const int32_t *q_lens, void *out, cudaStream_t stream);
+arb_status launch_kv_append_i4(Ctx *ctx, const arb_attn_params &p, int total_new, const void *k_new, const void *v_new,
+                               const int32_t *block_table, int32_t *seq_lens, const int32_t *new_lens, int update_lens,
+                               void *k_codes, void *v_codes, float *k_scales, float *v_scales, cudaStream_t stream);
 bool decode_step_supported(const arb_attn_params &p);
 size_t decode_step_hint_bytes(int num_sms);
 arb_status launch_decode_step(Ctx *ctx, const arb_attn_params &p, const void *q, const void *k_new, const void *v_new,

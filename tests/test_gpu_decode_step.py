@@ -456,3 +456,43 @@ def test_decode_step_i4_refusals():
                                             d.block_table.data_ptr(), d.seq_lens.data_ptr(), d.q_lens.data_ptr(),
                                             out.data_ptr(), None)
         binding._check(st, "arb_decode_step_i4")
+
+
+def test_kv_append_i4_prefill_then_tokens():
+    """arb_kv_append_i4 writes a ragged batch of new rows (a prefix for an empty sequence, a step for others, none for
+    one, one that does not fit), bit for bit like the oracle's encoder; arb_decode_step_i4 then runs on that cache."""
+    from paper_2512_05033_b200 import binding
+    c = H.ctx()
+    sl = [0, 40, 1000, 31, 200]
+    inp, kc, vc, ks, vs = _i4_case(5, 12, 2, sl, [1] * 5, 981, extra=70, row_std=0.5)
+    new = torch.tensor([64, 17, 0, 1, 33], dtype=torch.int32)
+    n = int(new.sum())
+    kn = wl.normal((n, 2, 128), 1.0, BF, "cpu", 982)
+    vn = wl.normal((n, 2, 128), 2.0, BF, "cpu", 983)
+    kn[3] = 0.0                                   # rows of zeros
+    d = inp.to("cuda")
+    pools = [kc.cuda(), vc.cuda(), ks.cuda(), vs.cuda()]
+    c.kv_append_i4(kn.cuda(), vn.cuda(), d.block_table, d.seq_lens, new.cuda(), *pools)
+    assert c.poll_status() == 0
+    ok, ov, oks, ovs, osl, st = oracle.kv_append_i4(kn, vn, inp.block_table, inp.seq_lens, new, kc, vc, ks, vs)
+    assert st == 0 and np.array_equal(d.seq_lens.cpu().numpy(), osl)
+    assert torch.equal(pools[0].cpu(), ok) and torch.equal(pools[1].cpu(), ov)
+    assert _same_f32_bits(pools[2], oks) and _same_f32_bits(pools[3], ovs)
+    # a token on top of it
+    k1, v1 = _new_rows(inp, 5, 984)
+    out = c.decode_step_i4(d.q, k1.cuda(), v1.cuda(), *pools, d.block_table, d.seq_lens, d.q_lens)
+    assert c.poll_status() == 0
+    ok, ov, oks, ovs, osl2, st = oracle.kv_append_i4(k1, v1, inp.block_table, osl, inp.q_lens, ok, ov, oks, ovs)
+    ref, st2 = oracle.attn_i4(inp.q, ok, ov, _live(ok, oks, inp, osl2)[1], _live(ov, ovs, inp, osl2)[1], inp.block_table, osl2,
+                              inp.q_lens)
+    assert st == 0 and st2 == 0
+    _i4_close(out, ref, ovs)
+    assert torch.equal(pools[0].cpu(), ok) and _same_f32_bits(pools[3], ovs)
+    # a sequence whose rows do not fit is left untouched, with the status bit
+    too_many = torch.tensor([0, 0, 0, 0, inp.block_table.shape[1] * 16], dtype=torch.int32)
+    before = [t.clone() for t in pools] + [d.seq_lens.clone()]
+    big = wl.normal((int(too_many.sum()), 2, 128), 1.0, BF, "cuda", 985)
+    c.kv_append_i4(big, big, d.block_table, d.seq_lens, too_many.cuda(), *pools)
+    assert c.poll_status() == binding.DEV_BAD_SEQ_LEN
+    for t_, b_ in zip(pools + [d.seq_lens], before):
+        assert torch.equal(t_.view(torch.uint8) if t_.dtype == torch.float32 else t_, b_.view(torch.uint8) if b_.dtype == torch.float32 else b_)

@@ -1023,14 +1023,19 @@ decode_step_kernel(const StepArgs a, const __grid_constant__ CUtensorMap k_map, 
 // CTAs per SM (so that the next kernel of a chain is resident before this one ends) was measured and is slower on
 // every workload: a lone call is bound by bytes in flight, and the successor's CTAs come up SM by SM as this
 // kernel's CTAs leave anyway.
-constexpr int kStages = 32;
+// Ring stages.  What is in flight per SM is stages x bytes of a stage, and it has to cover latency x bandwidth: 32 tiles
+// of a bf16 cache are 128 KB; the tiles of the code caches are 2 KB and 1.1 KB, so their rings are deeper (with 32
+// stages a large call over 4-bit codes could keep 16 KB per SM in flight: 1.4 TB/s).  The widened tiles of the code
+// forms take 64 KB beside the ring.
+template <int KV>
+constexpr int stages_of() { return KV == kKvBf16 ? 32 : KV == kKvE4m3 ? 48 : 80; }
 
 template <int G, bool APPEND, int KV>
 arb_status launch_variant(Ctx *ctx, const StepArgs &a, const CUtensorMap &km, const CUtensorMap &vm, cudaStream_t stream) {
     static bool attr_set[64] = {};
     if (!attr_set[ctx->device & 63]) {
-        if (cudaFuncSetAttribute(decode_step_kernel<G, kStages, APPEND, KV>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 (int)smem_bytes<G, kStages, KV>(kMaxBatch)) != cudaSuccess)
+        if (cudaFuncSetAttribute(decode_step_kernel<G, stages_of<KV>(), APPEND, KV>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 (int)smem_bytes<G, stages_of<KV>(), KV>(kMaxBatch)) != cudaSuccess)
             return ARB_ERR_CUDA;
         attr_set[ctx->device & 63] = true;
     }
@@ -1040,11 +1045,11 @@ arb_status launch_variant(Ctx *ctx, const StepArgs &a, const CUtensorMap &km, co
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(ctx->num_sms);
     cfg.blockDim = dim3(kNT);
-    cfg.dynamicSmemBytes = smem_bytes<G, kStages, KV>(a.batch);
+    cfg.dynamicSmemBytes = smem_bytes<G, stages_of<KV>(), KV>(a.batch);
     cfg.stream = stream;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    if (cudaLaunchKernelEx(&cfg, decode_step_kernel<G, kStages, APPEND, KV>, a, km, vm) != cudaSuccess) return ARB_ERR_CUDA;
+    if (cudaLaunchKernelEx(&cfg, decode_step_kernel<G, stages_of<KV>(), APPEND, KV>, a, km, vm) != cudaSuccess) return ARB_ERR_CUDA;
     ctx->launches++;
     return ARB_OK;
 }

@@ -55,11 +55,15 @@ constexpr int kSoftmaxThreads = 128;        // per row tile
 constexpr int kThreads = 3 * kSoftmaxThreads;   // two softmax groups and a group of service warps; registers are
                                                 // handed out per 128 threads, so the third group's spare warps cost none
 constexpr int kTmaWarp = 8, kMmaWarp = 9, kVWarp = 10, kPvWarp = 11;
-// The E4M3 form runs a fourth group of warps: warps 12 and 14 widen every second pair of pages of K and of V beside
-// warps 8 and 10 (one warp per operand widens a tile in about twice the time the tensor core and the softmax groups
-// need for it).  512 threads start with 128 registers each; the softmax groups then take 168 and the two service
-// groups keep 88 (setmaxnreg; 2 * 168 + 2 * 88 = 4 * 128).
-constexpr int kKHelpWarp = 12, kVHelpWarp = 14;
+// The E4M3 form runs a fourth group of warps: warps 12, 13 widen pairs of pages of K beside warp 8, warps 14, 15 pairs of
+// V beside warp 10 (one warp per operand widens a tile in about twice the time the tensor core and the softmax groups
+// need for it).  The pairs of an operand are numbered through the tiles; pair n belongs to warp n % 3 of the operand and
+// to staging slot n % 3, so every warp has a slot of its own, asks for its own next pair, and takes part in every
+// tile (four consecutive numbers cover the three residues).  512 threads start with 128 registers each; the softmax
+// groups then take 168 and the two service groups keep 88 (setmaxnreg; 2 * 168 + 2 * 88 = 4 * 128).
+constexpr int kKHelpWarp = 12, kVHelpWarp = 14;   // and the warp after each
+constexpr int kWideners = 3;                      // warps per operand in the E4M3 form
+static_assert(kWideners == 3 && kWideners <= 4, "a slot per widening warp; every warp has a pair in every full tile");
 __host__ __device__ constexpr int threads_of(bool e4m3) { return e4m3 ? 4 * kSoftmaxThreads : kThreads; }
 constexpr int kHalfBytes = 128 * 128;      // [128 rows x 64 bf16]: one 128-byte-swizzled half tile
 constexpr int kTileBytes = 2 * kHalfBytes;  // [128 x 128] bf16
@@ -484,8 +488,8 @@ chunk_mma_kernel(const MmaArgs a, const __grid_constant__ CUtensorMap k_map, con
     if (tid == 0) {
         mbar_init(&bars->q_full, 2 * kSoftmaxThreads);
         for (int s = 0; s < kStages; ++s) {
-            mbar_init(&bars->k_full[s], E4M3 ? 2 : 1);   // E4M3: both widening warps of the operand arrive
-            mbar_init(&bars->v_full[s], E4M3 ? 2 : 1);
+            mbar_init(&bars->k_full[s], E4M3 ? kWideners : 1);   // E4M3: every widening warp of the operand arrives
+            mbar_init(&bars->v_full[s], E4M3 ? kWideners : 1);
             mbar_init(&bars->k_empty[s], 1);
             mbar_init(&bars->v_empty[s], 1);
         }
@@ -500,8 +504,8 @@ chunk_mma_kernel(const MmaArgs a, const __grid_constant__ CUtensorMap k_map, con
         mbar_init(&bars->ml_full, 2 * kSoftmaxThreads);
         for (int i = 0; i < kItemSlots; ++i) {
             mbar_init(&bars->item_full[i], 1);
-            // the two MMA threads, the V warp, the softmax threads (E4M3: and the two helping warps)
-            mbar_init(&bars->item_empty[i], 3 + 2 * kSoftmaxThreads + (E4M3 ? 2 : 0));
+            // the two MMA threads, the V warp, the softmax threads (E4M3: and the four helping warps)
+            mbar_init(&bars->item_empty[i], 3 + 2 * kSoftmaxThreads + (E4M3 ? 2 * (kWideners - 1) : 0));
         }
         for (int i = 0; i < kStagePages; ++i) {
             mbar_init(&bars->code_full[0][i], 1);
@@ -522,7 +526,8 @@ chunk_mma_kernel(const MmaArgs a, const __grid_constant__ CUtensorMap k_map, con
     const uint32_t tmem = bars->tmem_base;
     volatile int *abort = &bars->abort;
 
-    const bool helper = E4M3 && (warp == kKHelpWarp || warp == kVHelpWarp);   // widens the odd pairs of pages
+    const bool helper = E4M3 && warp >= kKHelpWarp;                          // a widening warp of the fourth group
+    const int widx = helper ? 1 + (warp & 1) : 0;                            // which of the operand's wideners
     if (warp >= 2 * kSoftmaxThreads / 32) {   // the service warps
     if constexpr (E4M3) asm volatile("setmaxnreg.dec.sync.aligned.u32 88;");
     if (warp == kTmaWarp || warp == kVWarp || helper) {
@@ -533,7 +538,7 @@ chunk_mma_kernel(const MmaArgs a, const __grid_constant__ CUtensorMap k_map, con
         // from an atomic counter (longest sequences first) and are announced to every other role, the V warp
         // included, through a small queue in shared memory.  Both run ahead of the consumers as far as their
         // two-stage rings allow.
-        const bool is_v = warp == kVWarp || warp == kVHelpWarp;
+        const bool is_v = warp == kVWarp || warp >= kVHelpWarp;
         uint64_t *full = is_v ? bars->v_full : bars->k_full, *empty = is_v ? bars->v_empty : bars->k_empty;
         char *ring = is_v ? v_s : k_s;
         const CUtensorMap *map = is_v ? &v_map : &k_map;
@@ -621,15 +626,16 @@ chunk_mma_kernel(const MmaArgs a, const __grid_constant__ CUtensorMap k_map, con
                         __syncwarp();
                         if (lane < cnt) tma_box_load(stg + (sl * 2 + lane) * kCodePageBytes, map, 0, rr, &cfull[sl]);
                     };
-                    if (j == 0 && !helper) {   // a new item: nothing of it is in flight yet
-                        for (int q = 0; q < kStagePairs; ++q) ask(q, pc + q);
+                    if (j == 0) {   // a new item: nothing of it is in flight yet; every warp asks for its first pair
+                        for (int q = 0; q < kStagePairs; ++q)
+                            if ((int)((pc + q) % kWideners) == widx) ask(q, pc + q);
                     }
                     if (lane == 0) ok = mbar_wait(&empty[s], par ^ 1u, abort, a.status);
                     ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
                     const int r = lane >> 1, h = lane & 1;
                     const int npairs = (npages + 1) >> 1;
                     for (int q = 0; q < npairs; ++q, ++pc) {
-                        if ((q & 1) != (helper ? 1 : 0)) continue;   // the operand's two warps take the pairs in turn
+                        if ((int)(pc % kWideners) != widx) continue;   // the operand's warps take the pairs in turn
                         const uint32_t sl = pc % kStagePairs, ph = (pc / kStagePairs) & 1u;
                         const int cnt = min(2, npages - 2 * q);
                         mbar_wait(&cfull[sl], ph, abort, a.status);

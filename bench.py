@@ -639,6 +639,13 @@ def run_step_scoring(ctx, dev):
     hbm_peak, hbm_kind = measured_peak()
     t_tensor, t_hbm = flops / (sustained * 1e12) * 1e6, b["total"] / (hbm_peak * 1e9) * 1e6
     tflops = flops / (us_attn * 1e-6) / 1e12
+    # per case: a sequence's chunk is tensor-bound when its M = q_len * group rows exceed peak flops / peak bytes
+    g = shape.num_q_heads // shape.num_kv_heads
+    ridge = sustained * 1e12 / (hbm_peak * 1e9)
+    case_flops = (4 * ql * shape.num_q_heads * shape.head_dim * sl).double()
+    case_bytes = (4 * sl * shape.num_kv_heads * shape.head_dim).double()          # K and V, bf16
+    case_us = torch.maximum(case_flops / (sustained * 1e12), case_bytes / (hbm_peak * 1e9)) * 1e6
+    tensor_cases = int((ql * g > ridge).sum())
     roof = {"bound": "tensor" if t_tensor >= t_hbm else "hbm", "kernel": "chunk_mma_kernel",
             "achieved": round(tflops, 1), "peak": sustained, "peak_kind": f"of {kind} (sustained bf16)", "unit": "TFLOP/s",
             "frac": round(max(t_tensor, t_hbm) / us_attn, 4), "traffic": None, "algorithmic_flops_per_launch": flops,
@@ -646,7 +653,12 @@ def run_step_scoring(ctx, dev):
             "roofline_us": {"tensor": round(t_tensor, 1), "hbm": round(t_hbm, 1)},
             "tensor_utilisation": round(tflops / sustained, 4), "tensor_utilisation_of_burst_peak": round(tflops / burst, 4),
             "hbm_utilisation": round(b["total"] / (us_attn * 1e-6) / 1e9 / hbm_peak, 4),
-            "note": "frac = max(bytes / HBM peak, flops / tensor peak) / measured time"}
+            "per_case": {"ridge_rows": round(ridge, 1), "tensor_bound_sequences": tensor_cases,
+                         "hbm_bound_sequences": int(shape.batch) - tensor_cases,
+                         "sum_of_case_rooflines_us": round(float(case_us.sum()), 1),
+                         "frac_of_sum": round(float(case_us.sum()) / us_attn, 4)},
+            "note": "frac = max(bytes / HBM peak, flops / tensor peak) / measured time; per_case: the same maximum taken "
+                    "sequence by sequence (M = q_len * group rows against the ridge) and summed"}
     return {"steps_scored_routed_per_s": res, "escalation_rate": esc, "layer_calls_per_step": 1,
             "route_only_steps_per_s": round(shape.batch / (ms_route / 200 * 1e-3), 1),
             "kv_tokens": b["tokens"], "rows": int(inp.q_lens.sum()), "attn_us_per_call": round(us_attn, 2),
